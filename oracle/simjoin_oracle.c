@@ -1,0 +1,273 @@
+/*
+ * CPU ORACLE for the thresholded all-pairs similarity join.
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  Only the tests, the
+ * smoke check and the benchmark's cpu_baseline / reference legs may build,
+ * load or call it.  It shares no code, header, table or constant with the CUDA
+ * library and includes nothing from it.
+ *
+ * What it computes: the definition of the similarity join in Section 4 of the
+ * paper (P join_r Q = all pairs (x, y) in P x Q whose distance is at most r),
+ * taken over index pairs (i, j), for the ip-distances Section 4 lists, written
+ * as the plain double loop over (i, j) with an inner loop over the d
+ * coordinates.  The paper's brute-force TCU algorithm (Section 4, the product
+ * F_P * G_Q^T evaluated with Theorem 1's tiling) reaches exactly this set, so
+ * the definition itself is the oracle: no tiling, blocking or reordering here.
+ *
+ * Readings where the paper is silent (each one is listed in the design notes):
+ *   - similarities (inner product, cosine) pass when score >= t, distances
+ *     (Euclidean) when distance <= r; both inclusive, as "D(x,y) <= r" is.
+ *   - points are identified by their row index; duplicates are distinct rows;
+ *     a self join keeps the diagonal and both orientations.
+ *   - int8 inputs: exact integer arithmetic.  Inner product: pass iff
+ *     s >= t over the reals (s is an integer below 2^53, so the double compare
+ *     is exact).  Euclidean: pass iff the integer squared distance D satisfies
+ *     (double)D <= r*r, r*r being the double product.
+ *   - bf16 inputs: the 16-bit patterns are the inputs; each is widened exactly
+ *     to fp64 and all sums run in fp64 with k ascending.
+ *     cosine of a zero vector is defined as 0.
+ *     Euclidean uses the difference form sqrt(sum (x_k-y_k)^2), not the norm
+ *     expansion.
+ *
+ * Output: pairs sorted by (i, j); the return value is the total number of
+ * passing pairs even when it exceeds `capacity` (then only the first
+ * `capacity` pairs in sorted order are written).  -1 on invalid arguments.
+ *
+ * Threads only split the outer loop into contiguous row blocks whose results
+ * are concatenated in block order; they do not change any arithmetic.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { KIND_IP = 0, KIND_COS = 1, KIND_L2 = 2 };
+
+/* ---------------------------------------------------------------- scores */
+
+/* <x,y> over int8 coordinates, exact. */
+int64_t oracle_ip_i8(const int8_t *x, const int8_t *y, int32_t d) {
+    int64_t s = 0;
+    for (int32_t k = 0; k < d; ++k) s += (int64_t)x[k] * (int64_t)y[k];
+    return s;
+}
+
+/* sum_k (x_k - y_k)^2 over int8 coordinates, exact. */
+int64_t oracle_sqdist_i8(const int8_t *x, const int8_t *y, int32_t d) {
+    int64_t s = 0;
+    for (int32_t k = 0; k < d; ++k) {
+        int64_t e = (int64_t)x[k] - (int64_t)y[k];
+        s += e * e;
+    }
+    return s;
+}
+
+/* The value a bfloat16 bit pattern denotes, as fp64 (exact). */
+double oracle_bf16_to_f64(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+static double dot_f64(const double *x, const double *y, int32_t d) {
+    double s = 0.0;
+    for (int32_t k = 0; k < d; ++k) s += x[k] * y[k];
+    return s;
+}
+
+/* Score of one pair of already widened rows; nx2, ny2 are sum x_k^2, sum y_k^2
+ * (used by the cosine only). */
+static double score_f64(const double *x, const double *y, int32_t d, int kind, double nx2, double ny2) {
+    if (kind == KIND_IP) return dot_f64(x, y, d);
+    if (kind == KIND_COS) {
+        if (nx2 == 0.0 || ny2 == 0.0) return 0.0;
+        return dot_f64(x, y, d) / (sqrt(nx2) * sqrt(ny2));
+    }
+    double s = 0.0;
+    for (int32_t k = 0; k < d; ++k) {
+        double e = x[k] - y[k];
+        s += e * e;
+    }
+    return sqrt(s);
+}
+
+static double *widen_rows(const uint16_t *X, int64_t rows, int32_t d) {
+    size_t cnt = (size_t)rows * (size_t)d;
+    double *W = (double *)malloc((cnt ? cnt : 1) * sizeof(double));
+    if (!W) return NULL;
+    for (size_t t = 0; t < cnt; ++t) W[t] = oracle_bf16_to_f64(X[t]);
+    return W;
+}
+
+static double *row_sq_norms(const double *W, int64_t rows, int32_t d) {
+    double *N = (double *)malloc((rows ? rows : 1) * sizeof(double));
+    if (!N) return NULL;
+    for (int64_t i = 0; i < rows; ++i) N[i] = dot_f64(W + (size_t)i * d, W + (size_t)i * d, d);
+    return N;
+}
+
+/* Score of the bf16 pair (row i of P, row j of Q), fp64. */
+double oracle_score_bf16(const uint16_t *P, int64_t i, const uint16_t *Q, int64_t j, int32_t d, int32_t kind) {
+    double *x = widen_rows(P + (size_t)i * d, 1, d);
+    double *y = widen_rows(Q + (size_t)j * d, 1, d);
+    double s = score_f64(x, y, d, kind, dot_f64(x, x, d), dot_f64(y, y, d));
+    free(x);
+    free(y);
+    return s;
+}
+
+/* Scores of a list of pairs: out[p] = score(P[pairs[2p]], Q[pairs[2p+1]]).
+ * int8: inner product (KIND_IP) or squared distance (KIND_L2) as int64 in out_i;
+ * bf16: fp64 score in out_f. */
+int32_t oracle_scores_i8(const int8_t *P, const int8_t *Q, int32_t d, int32_t kind,
+                         const int32_t *pairs, int64_t npairs, int64_t *out_i) {
+    if (kind != KIND_IP && kind != KIND_L2) return -1;
+    for (int64_t p = 0; p < npairs; ++p) {
+        const int8_t *x = P + (size_t)pairs[2 * p] * d, *y = Q + (size_t)pairs[2 * p + 1] * d;
+        out_i[p] = kind == KIND_IP ? oracle_ip_i8(x, y, d) : oracle_sqdist_i8(x, y, d);
+    }
+    return 0;
+}
+
+int32_t oracle_scores_bf16(const uint16_t *P, const uint16_t *Q, int32_t d, int32_t kind,
+                           const int32_t *pairs, int64_t npairs, double *out_f) {
+    if (kind < KIND_IP || kind > KIND_L2) return -1;
+    for (int64_t p = 0; p < npairs; ++p)
+        out_f[p] = oracle_score_bf16(P, pairs[2 * p], Q, pairs[2 * p + 1], d, kind);
+    return 0;
+}
+
+/* Row squared norms in fp64 (bf16 rows) / exact int64 (int8 rows). */
+void oracle_sq_norms_bf16(const uint16_t *X, int64_t rows, int32_t d, double *out) {
+    for (int64_t i = 0; i < rows; ++i) {
+        double s = 0.0;
+        for (int32_t k = 0; k < d; ++k) {
+            double v = oracle_bf16_to_f64(X[(size_t)i * d + k]);
+            s += v * v;
+        }
+        out[i] = s;
+    }
+}
+
+void oracle_sq_norms_i8(const int8_t *X, int64_t rows, int32_t d, int64_t *out) {
+    for (int64_t i = 0; i < rows; ++i) out[i] = oracle_ip_i8(X + (size_t)i * d, X + (size_t)i * d, d);
+}
+
+/* ------------------------------------------------------------- the join */
+
+typedef struct {
+    int32_t *v;     /* (i, j) pairs of this row block, in (i, j) order */
+    int64_t cnt, cap;
+    int oom;
+} pairbuf;
+
+static void pb_push(pairbuf *b, int64_t i, int64_t j) {
+    if (b->cnt == b->cap) {
+        int64_t nc = b->cap ? 2 * b->cap : 64;
+        int32_t *nv = (int32_t *)realloc(b->v, (size_t)nc * 2 * sizeof(int32_t));
+        if (!nv) { b->oom = 1; return; }
+        b->v = nv;
+        b->cap = nc;
+    }
+    b->v[2 * b->cnt] = (int32_t)i;
+    b->v[2 * b->cnt + 1] = (int32_t)j;
+    b->cnt++;
+}
+
+static int pass_i8(const int8_t *x, const int8_t *y, int32_t d, int kind, double thr) {
+    if (kind == KIND_IP) return (double)oracle_ip_i8(x, y, d) >= thr;
+    return (double)oracle_sqdist_i8(x, y, d) <= thr * thr;
+}
+
+static int pass_f64(double score, int kind, double thr) {
+    return kind == KIND_L2 ? score <= thr : score >= thr;
+}
+
+static int64_t num_blocks(int64_t n, int nthreads) {
+    int64_t nb = (int64_t)nthreads * 64;
+    if (nb > n) nb = n;
+    if (nb < 1) nb = 1;
+    return nb;
+}
+
+static int64_t gather(pairbuf *blk, int64_t nb, int32_t *out_pairs, int64_t capacity) {
+    int64_t total = 0, written = 0;
+    int oom = 0;
+    for (int64_t b = 0; b < nb; ++b) {
+        oom |= blk[b].oom;
+        for (int64_t p = 0; p < blk[b].cnt && written < capacity; ++p, ++written) {
+            out_pairs[2 * written] = blk[b].v[2 * p];
+            out_pairs[2 * written + 1] = blk[b].v[2 * p + 1];
+        }
+        total += blk[b].cnt;
+        free(blk[b].v);
+    }
+    free(blk);
+    return oom ? -1 : total;
+}
+
+static int resolve_threads(int32_t nthreads) {
+#ifdef _OPENMP
+    return nthreads > 0 ? nthreads : omp_get_max_threads();
+#else
+    (void)nthreads;
+    return 1;
+#endif
+}
+
+int32_t oracle_max_threads(void) { return resolve_threads(0); }
+
+int64_t oracle_join_i8(const int8_t *P, int64_t n, const int8_t *Q, int64_t m, int32_t d, int32_t kind,
+                       double threshold, int32_t *out_pairs, int64_t capacity, int32_t nthreads) {
+    if (n < 0 || m < 0 || d <= 0 || capacity < 0 || (kind != KIND_IP && kind != KIND_L2)) return -1;
+    if (isnan(threshold) || (kind == KIND_L2 && threshold < 0)) return -1;
+    if (n >= INT32_MAX || m >= INT32_MAX) return -1;
+    int nt = resolve_threads(nthreads);
+    int64_t nb = num_blocks(n, nt);
+    pairbuf *blk = (pairbuf *)calloc((size_t)nb, sizeof(pairbuf));
+    if (!blk) return -1;
+#pragma omp parallel for schedule(dynamic, 1) num_threads(nt)
+    for (int64_t b = 0; b < nb; ++b) {
+        int64_t i0 = n * b / nb, i1 = n * (b + 1) / nb;
+        for (int64_t i = i0; i < i1; ++i)
+            for (int64_t j = 0; j < m; ++j)
+                if (pass_i8(P + (size_t)i * d, Q + (size_t)j * d, d, kind, threshold)) pb_push(&blk[b], i, j);
+    }
+    return gather(blk, nb, out_pairs, capacity);
+}
+
+int64_t oracle_join_bf16(const uint16_t *P, int64_t n, const uint16_t *Q, int64_t m, int32_t d, int32_t kind,
+                         double threshold, int32_t *out_pairs, int64_t capacity, int32_t nthreads) {
+    if (n < 0 || m < 0 || d <= 0 || capacity < 0 || kind < KIND_IP || kind > KIND_L2) return -1;
+    if (isnan(threshold) || (kind == KIND_L2 && threshold < 0)) return -1;
+    if (n >= INT32_MAX || m >= INT32_MAX) return -1;
+    int nt = resolve_threads(nthreads);
+    double *WP = widen_rows(P, n, d), *WQ = widen_rows(Q, m, d);
+    double *NP = WP ? row_sq_norms(WP, n, d) : NULL, *NQ = WQ ? row_sq_norms(WQ, m, d) : NULL;
+    int64_t nb = num_blocks(n, nt);
+    pairbuf *blk = (pairbuf *)calloc((size_t)nb, sizeof(pairbuf));
+    int64_t total = -1;
+    if (WP && WQ && NP && NQ && blk) {
+#pragma omp parallel for schedule(dynamic, 1) num_threads(nt)
+        for (int64_t b = 0; b < nb; ++b) {
+            int64_t i0 = n * b / nb, i1 = n * (b + 1) / nb;
+            for (int64_t i = i0; i < i1; ++i)
+                for (int64_t j = 0; j < m; ++j) {
+                    double s = score_f64(WP + (size_t)i * d, WQ + (size_t)j * d, d, kind, NP[i], NQ[j]);
+                    if (pass_f64(s, kind, threshold)) pb_push(&blk[b], i, j);
+                }
+        }
+        total = gather(blk, nb, out_pairs, capacity);
+    } else {
+        free(blk);
+    }
+    free(WP);
+    free(WQ);
+    free(NP);
+    free(NQ);
+    return total;
+}

@@ -1,0 +1,175 @@
+"""ctypes front end of the CPU oracle (``simjoin_oracle.c``).
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT: only the tests, the smoke check and the
+benchmark's cpu_baseline / reference legs may import this module.  It imports
+nothing from the CUDA package and the CUDA package imports nothing from here.
+
+The C file is the oracle: the join's definition (Section 4 of the paper) as a
+plain double loop in exact integer / fp64 arithmetic.  This module only builds
+it with gcc on first use, marshals numpy arrays and derives the band sets used
+to compare floating-point joins (a pure re-run of the same oracle at a shifted
+threshold).
+"""
+from __future__ import annotations
+
+import ctypes
+import hashlib
+import os
+import subprocess
+from typing import Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "simjoin_oracle.c")
+KIND = {"ip": 0, "cos": 1, "l2": 2}
+_lib = None
+
+
+def _cpu_tag() -> str:
+    """Short tag of the host CPU so a library built with -march=native on one
+    machine is never loaded on a different one."""
+    try:
+        with open("/proc/cpuinfo") as f:
+            txt = f.read()
+        lines = [l for l in txt.splitlines() if l.startswith(("model name", "flags"))][:2]
+        return hashlib.sha1("\n".join(lines).encode()).hexdigest()[:10]
+    except OSError:
+        return "generic"
+
+
+def lib_path() -> str:
+    return os.path.join(_HERE, f"liboracle_simjoin_{_cpu_tag()}.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O3 -march=native -fopenmp); returns the .so path."""
+    out = lib_path()
+    if not force and os.path.exists(out) and os.path.getmtime(out) >= os.path.getmtime(_SRC):
+        return out
+    tmp = out + f".tmp{os.getpid()}"
+    cmd = ["gcc", "-O3", "-march=native", "-fopenmp", "-fno-fast-math", "-shared", "-fPIC",
+           "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True, capture_output=True)
+    os.replace(tmp, out)
+    return out
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = ctypes.CDLL(build())
+    c = ctypes
+    vp, i64, i32, dbl = c.c_void_p, c.c_int64, c.c_int32, c.c_double
+    for name in ("oracle_join_i8", "oracle_join_bf16"):
+        fn = getattr(lib, name)
+        fn.restype = i64
+        fn.argtypes = [vp, i64, vp, i64, i32, i32, dbl, vp, i64, i32]
+    lib.oracle_scores_i8.restype = i32
+    lib.oracle_scores_i8.argtypes = [vp, vp, i32, i32, vp, i64, vp]
+    lib.oracle_scores_bf16.restype = i32
+    lib.oracle_scores_bf16.argtypes = [vp, vp, i32, i32, vp, i64, vp]
+    lib.oracle_sq_norms_bf16.restype = None
+    lib.oracle_sq_norms_bf16.argtypes = [vp, i64, i32, vp]
+    lib.oracle_sq_norms_i8.restype = None
+    lib.oracle_sq_norms_i8.argtypes = [vp, i64, i32, vp]
+    lib.oracle_max_threads.restype = i32
+    lib.oracle_max_threads.argtypes = []
+    _lib = lib
+    return lib
+
+
+def max_threads() -> int:
+    return int(_load().oracle_max_threads())
+
+
+def _check(X: np.ndarray, dtype: str) -> np.ndarray:
+    want = np.int8 if dtype == "i8" else np.uint16
+    if X.dtype != want or X.ndim != 2:
+        raise TypeError(f"expected 2-D {want.__name__} array for dtype {dtype}, got {X.dtype} ndim {X.ndim}")
+    return np.ascontiguousarray(X)
+
+
+def join(P: np.ndarray, Q: np.ndarray, kind: str, threshold: float, dtype: str,
+         capacity: int | None = None, threads: int = 0) -> Tuple[np.ndarray, int]:
+    """All (i, j) with score(P[i], Q[j]) >= threshold (ip, cos) or
+    distance <= threshold (l2), sorted by (i, j).
+
+    Returns (pairs[min(count, capacity), 2] int32, count).  With capacity=None
+    the call is repeated with a larger buffer until everything fits.
+    """
+    lib = _load()
+    P = _check(P, dtype)
+    Q = _check(Q, dtype)
+    n, d = P.shape
+    m, d2 = Q.shape
+    if d != d2:
+        raise ValueError("P and Q must have the same number of columns")
+    fn = lib.oracle_join_i8 if dtype == "i8" else lib.oracle_join_bf16
+    cap = 1 << 16 if capacity is None else int(capacity)
+    while True:
+        out = np.empty((max(cap, 1), 2), dtype=np.int32)
+        cnt = fn(P.ctypes.data, n, Q.ctypes.data, m, d, KIND[kind], float(threshold),
+                 out.ctypes.data, cap, threads)
+        if cnt < 0:
+            raise ValueError("oracle rejected the arguments")
+        if capacity is not None or cnt <= cap:
+            return out[:min(cnt, cap)].copy(), int(cnt)
+        cap = int(cnt)
+
+
+def band_sets(P, Q, kind, threshold, dtype, rel: float = 1e-2, threads: int = 0):
+    """(S_strict, S_exact, S_loose): the join at the threshold moved by rel*|t|
+    towards fewer pairs, at the threshold itself, and moved towards more pairs.
+    A floating-point join G is accepted when S_strict <= G <= S_loose."""
+    t = float(threshold)
+    delta = rel * abs(t)
+    if kind == "l2":
+        strict_t, loose_t = t - delta, t + delta
+    else:
+        strict_t, loose_t = t + delta, t - delta
+    s_strict, _ = join(P, Q, kind, strict_t, dtype, threads=threads)
+    s_exact, _ = join(P, Q, kind, t, dtype, threads=threads)
+    s_loose, _ = join(P, Q, kind, loose_t, dtype, threads=threads)
+    return s_strict, s_exact, s_loose
+
+
+def scores(P, Q, kind: str, dtype: str, pairs: np.ndarray) -> np.ndarray:
+    """Score of each listed (i, j): int64 inner product / squared distance for
+    int8 rows, fp64 inner product / cosine / distance for bf16 rows."""
+    lib = _load()
+    P = _check(P, dtype)
+    Q = _check(Q, dtype)
+    pairs = np.ascontiguousarray(pairs, dtype=np.int32).reshape(-1, 2)
+    d = P.shape[1]
+    if len(pairs) and (pairs[:, 0].max() >= P.shape[0] or pairs[:, 1].max() >= Q.shape[0] or pairs.min() < 0):
+        raise IndexError("pair index out of range")
+    if dtype == "i8":
+        out = np.empty(len(pairs), dtype=np.int64)
+        rc = lib.oracle_scores_i8(P.ctypes.data, Q.ctypes.data, d, KIND[kind], pairs.ctypes.data, len(pairs), out.ctypes.data)
+    else:
+        out = np.empty(len(pairs), dtype=np.float64)
+        rc = lib.oracle_scores_bf16(P.ctypes.data, Q.ctypes.data, d, KIND[kind], pairs.ctypes.data, len(pairs), out.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return out
+
+
+def sq_norms(X: np.ndarray, dtype: str) -> np.ndarray:
+    """Row squared norms: exact int64 (int8 rows) or fp64 (bf16 rows)."""
+    lib = _load()
+    X = _check(X, dtype)
+    if dtype == "i8":
+        out = np.empty(X.shape[0], dtype=np.int64)
+        lib.oracle_sq_norms_i8(X.ctypes.data, X.shape[0], X.shape[1], out.ctypes.data)
+    else:
+        out = np.empty(X.shape[0], dtype=np.float64)
+        lib.oracle_sq_norms_bf16(X.ctypes.data, X.shape[0], X.shape[1], out.ctypes.data)
+    return out
+
+
+def pairs_to_set(pairs: np.ndarray) -> np.ndarray:
+    """Encode (i, j) rows as sorted unique int64 keys i*2^32 + j (for set algebra)."""
+    p = np.asarray(pairs, dtype=np.int64).reshape(-1, 2)
+    return np.unique((p[:, 0] << 32) | p[:, 1])

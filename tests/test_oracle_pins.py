@@ -1,0 +1,305 @@
+"""Pins for the CPU oracle: everything here checks the oracle against something
+other than itself -- hand-worked joins (tests/golden), closed forms, an
+independent bit-counting formulation, exact rational brute force, a BLAS
+product, and the invariants the join's definition (Section 4) fixes.  No GPU."""
+import glob
+import itertools
+import json
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import simjoin_oracle as O
+from paper_2006_12608_b200 import workloads as W
+
+
+def as_set(pairs):
+    return set(map(tuple, np.asarray(pairs).reshape(-1, 2).tolist()))
+
+
+def to_arr(rows, dtype):
+    a = np.asarray(rows, dtype=np.float64)
+    if dtype == "i8":
+        return a.astype(np.int8)
+    bits = W.f32_to_bf16_bits(a.astype(np.float32))
+    assert np.array_equal(W.bf16_bits_to_f32(bits).astype(np.float64), a), "fixture value not exact in bf16"
+    return bits
+
+
+# ------------------------------------------------------------------ hand-worked
+GOLDEN = sorted(glob.glob(os.path.join(os.path.dirname(__file__), "golden", "*.json")))
+
+
+@pytest.mark.parametrize("path", GOLDEN, ids=[os.path.basename(p) for p in GOLDEN])
+def test_hand_worked_cases(path):
+    with open(path) as f:
+        g = json.load(f)
+    P, Q = to_arr(g["P"], g["dtype"]), to_arr(g["Q"], g["dtype"])
+    allp = np.array(list(itertools.product(range(len(P)), range(len(Q)))), dtype=np.int32)
+    sc = O.scores(P, Q, g["kind"], g["dtype"], allp).reshape(len(P), len(Q))
+    np.testing.assert_allclose(sc, np.array(g["scores"], dtype=np.float64), rtol=1e-15, atol=0)
+    for case in g["cases"]:
+        pairs, cnt = O.join(P, Q, g["kind"], case["threshold"], g["dtype"])
+        assert cnt == len(case["pairs"]), case
+        assert pairs.tolist() == sorted(case["pairs"]), case      # sorted by (i, j)
+
+
+# ------------------------------------------------- independent formulations
+def _packbits_rows(X):
+    return np.packbits(X > 0, axis=1)
+
+
+_POP8 = np.array([bin(v).count("1") for v in range(256)], dtype=np.int32)
+
+
+def hamming_matrix(P, Q):
+    """Hamming distance of +-1 rows through XOR + popcount: no multiply, no sum of products."""
+    bp, bq = _packbits_rows(P), _packbits_rows(Q)
+    return _POP8[bp[:, None, :] ^ bq[None, :, :]].sum(axis=2)
+
+
+def test_pm1_inner_product_is_d_minus_2_hamming_cfg1_full():
+    # <x,y> = d - 2*Hamming(x,y) for +-1 vectors: the Hamming ip-distance of Section 4 in disguise.
+    w = W.make_workload(1)
+    pairs, cnt = O.join(w.P, w.Q, "ip", w.threshold, "i8")
+    want = set()
+    for i0 in range(0, w.n, 256):
+        ham = hamming_matrix(w.P[i0:i0 + 256], w.Q)
+        ii, jj = np.nonzero(w.d - 2 * ham >= w.threshold)
+        want |= set(zip((ii + i0).tolist(), jj.tolist()))
+    assert as_set(pairs) == want and cnt == len(want)
+    assert as_set(w.planted) <= want
+    # closed-form tail: background pairs pass with p = P[Bin(64,1/2) <= 12]; expectation ~0.96
+    p_bg = sum(math.comb(64, k) for k in range(13)) / 2.0 ** 64
+    assert abs(p_bg * 2048 * 2048 - 0.958) < 0.01
+    assert 32 <= cnt <= 32 + 8
+
+
+def test_binomial_tail_closed_form_pins_count():
+    # iid +-1 rows, no planted pairs: count ~ Binomial(n*m, P[Bin(d,1/2) <= (d-t)/2])
+    n = m = 1024
+    d, t = 64, 16
+    w = W.make_workload(1, n=n, m=m, planted=0, seed=5)
+    _, cnt = O.join(w.P, w.Q, "ip", t, "i8")
+    p = sum(math.comb(d, k) for k in range((d - t) // 2 + 1)) / 2.0 ** d
+    mean, sd = n * m * p, math.sqrt(n * m * p * (1 - p))
+    assert abs(cnt - mean) < 5 * sd, (cnt, mean, sd)
+
+
+@pytest.mark.parametrize("cfg,kw", [(3, dict(n=700, m=900, planted=25)), (4, dict(n=1000, m=513, planted=40))])
+def test_blas_product_gives_same_integer_set(cfg, kw):
+    w = W.make_workload(cfg, **kw)
+    S = w.P.astype(np.float64) @ w.Q.astype(np.float64).T          # exact: all values < 2^53
+    ii, jj = np.nonzero(S >= w.threshold)
+    pairs, cnt = O.join(w.P, w.Q, "ip", w.threshold, "i8")
+    assert as_set(pairs) == set(zip(ii.tolist(), jj.tolist())) and cnt == len(ii)
+    assert as_set(w.planted) <= as_set(pairs)
+    assert cnt >= kw["planted"]
+
+
+def test_blas_product_outside_band_bf16():
+    w = W.make_workload(2, n=600, m=500, planted=30)
+    Pf, Qf = W.bf16_bits_to_f32(w.P).astype(np.float64), W.bf16_bits_to_f32(w.Q).astype(np.float64)
+    C = (Pf @ Qf.T) / np.outer(np.linalg.norm(Pf, axis=1), np.linalg.norm(Qf, axis=1))
+    pairs, _ = O.join(w.P, w.Q, "cos", w.threshold, "bf16")
+    got = np.zeros(C.shape, dtype=bool)
+    got[pairs[:, 0], pairs[:, 1]] = True
+    clear = np.abs(C - w.threshold) > 1e-9
+    assert np.array_equal(got[clear], (C >= w.threshold)[clear])
+    assert as_set(w.planted) <= as_set(pairs)
+
+
+def test_mixture_join_is_same_cluster_relation():
+    w = W.make_workload(5, n=1500, m=1300, centers=40)
+    pairs, cnt = O.join(w.P, w.Q, "l2", w.threshold, "bf16")
+    ii, jj = np.nonzero(w.labels_p[:, None] == w.labels_q[None, :])
+    assert as_set(pairs) == set(zip(ii.tolist(), jj.tolist()))
+    wl = W.make_workload(5, n=1500, m=1300, centers=40, sigma_reading="percoord")
+    _, cnt_lit = O.join(wl.P, wl.Q, "l2", wl.threshold, "bf16")
+    assert cnt_lit == 0
+
+
+# ------------------------------------------------------ exact rational brute force
+def frac_rows(X, dtype):
+    if dtype == "i8":
+        return [[Fraction(int(v)) for v in r] for r in X]
+    return [[Fraction(float(v)) for v in r] for r in W.bf16_bits_to_f32(X)]
+
+
+def frac_pass(x, y, kind, t):
+    s = sum(a * b for a, b in zip(x, y))
+    if kind == "ip":
+        return s >= t, s - t
+    if kind == "l2":
+        dd = sum((a - b) ** 2 for a, b in zip(x, y))
+        return dd <= t * t, dd - t * t
+    nx, ny = sum(a * a for a in x), sum(b * b for b in y)
+    if nx == 0 or ny == 0:
+        return Fraction(0) >= t, Fraction(1)
+    # s/(sqrt(nx) sqrt(ny)) >= t without square roots
+    lhs, rhs = s * s, t * t * nx * ny
+    if t >= 0:
+        return (s >= 0 and lhs >= rhs), lhs - rhs
+    return (s >= 0 or lhs <= rhs), lhs - rhs
+
+
+@pytest.mark.parametrize("dtype,kind", [("i8", "ip"), ("i8", "l2"), ("bf16", "ip"), ("bf16", "cos"), ("bf16", "l2")])
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_exact_rational_brute_force(dtype, kind, seed):
+    n, m, d = 7, 9, 5
+    P = W.random_points(dtype, n, d, seed)
+    Q = W.random_points(dtype, m, d, seed + 100)
+    if dtype == "bf16" and seed == 2:
+        P[3] = 0                                            # a zero row (bits of +0.0)
+    FP, FQ = frac_rows(P, dtype), frac_rows(Q, dtype)
+    thresholds = {"ip": [-2.5, 0, 1, 3.25], "cos": [-0.5, 0.0, 0.3, 0.8], "l2": [0.0, 1.5, 3.0, 4.75]}[kind]
+    for t in thresholds:
+        ft = Fraction(t)
+        want = set()
+        for i, j in itertools.product(range(n), range(m)):
+            ok, margin = frac_pass(FP[i], FQ[j], kind, ft)
+            if dtype == "bf16" and kind != "ip" and margin != 0 and abs(margin) < Fraction(1, 10 ** 9):
+                pytest.skip("near tie: fp64 rounding may decide")
+            if ok:
+                want.add((i, j))
+        pairs, cnt = O.join(P, Q, kind, t, dtype)
+        assert as_set(pairs) == want and cnt == len(want), (kind, dtype, t)
+
+
+# ------------------------------------------------ the paper's f, g embeddings
+def test_hamming_embedding_identity():
+    # Section 4: f(x) = (x_0, 1-x_0, ...), g(y) = (1-y_0, y_0, ...) on {0,1}^d gives Hamming(x,y);
+    # on binary vectors Hamming equals the squared Euclidean distance the oracle computes.
+    rng = np.random.default_rng(3)
+    X = rng.integers(0, 2, size=(6, 11), dtype=np.int8)
+    Y = rng.integers(0, 2, size=(5, 11), dtype=np.int8)
+    f = np.stack([X, 1 - X], axis=2).reshape(len(X), -1).astype(np.int64)
+    g = np.stack([1 - Y, Y], axis=2).reshape(len(Y), -1).astype(np.int64)
+    allp = np.array(list(itertools.product(range(6), range(5))), dtype=np.int32)
+    got = O.scores(X, Y, "l2", "i8", allp).reshape(6, 5)
+    assert np.array_equal(got, f @ g.T)
+    assert np.array_equal(got, (X[:, None, :] != Y[None, :, :]).sum(axis=2))
+
+
+def test_squared_l2_embedding_identity():
+    # Section 4 (g is misprinted there): f(x) = (x_k^2, 1, -2 x_k)_k, g(y) = (1, y_k^2, y_k)_k.
+    rng = np.random.default_rng(4)
+    X = rng.integers(-9, 10, size=(6, 7), dtype=np.int8)
+    Y = rng.integers(-9, 10, size=(5, 7), dtype=np.int8)
+    x, y = X.astype(np.int64), Y.astype(np.int64)
+    f = np.stack([x * x, np.ones_like(x), -2 * x], axis=2).reshape(len(X), -1)
+    g = np.stack([np.ones_like(y), y * y, y], axis=2).reshape(len(Y), -1)
+    allp = np.array(list(itertools.product(range(6), range(5))), dtype=np.int32)
+    assert np.array_equal(O.scores(X, Y, "l2", "i8", allp).reshape(6, 5), f @ g.T)
+    # and the norm expansion the GPU path uses: ||x||^2 + ||y||^2 - 2<x,y>
+    ip = O.scores(X, Y, "ip", "i8", allp).reshape(6, 5)
+    nx, ny = O.sq_norms(X, "i8"), O.sq_norms(Y, "i8")
+    assert np.array_equal(nx[:, None] + ny[None, :] - 2 * ip, f @ g.T)
+    assert np.array_equal(nx, (x * x).sum(axis=1))
+
+
+def test_cosine_embedding_identity():
+    X = W.random_points("bf16", 6, 9, 11)
+    Y = W.random_points("bf16", 5, 9, 12)
+    xf, yf = W.bf16_bits_to_f32(X).astype(np.float64), W.bf16_bits_to_f32(Y).astype(np.float64)
+    f = xf / np.sqrt((xf * xf).sum(axis=1, keepdims=True))
+    g = yf / np.sqrt((yf * yf).sum(axis=1, keepdims=True))
+    allp = np.array(list(itertools.product(range(6), range(5))), dtype=np.int32)
+    np.testing.assert_allclose(O.scores(X, Y, "cos", "bf16", allp).reshape(6, 5), f @ g.T, rtol=0, atol=1e-14)
+    np.testing.assert_allclose(O.sq_norms(X, "bf16"), (xf * xf).sum(axis=1), rtol=1e-15)
+    d2 = O.scores(X, Y, "l2", "bf16", allp).reshape(6, 5) ** 2
+    np.testing.assert_allclose(d2, ((xf[:, None, :] - yf[None, :, :]) ** 2).sum(axis=2), rtol=1e-14)
+
+
+# ------------------------------------------------------------------ invariants
+CASES = [("i8", "ip", 3, 2.0), ("i8", "l2", None, 9.5), ("bf16", "ip", None, 1.0),
+         ("bf16", "cos", None, 0.2), ("bf16", "l2", None, 3.5)]
+
+
+@pytest.mark.parametrize("dtype,kind,_,t", CASES)
+def test_invariants(dtype, kind, _, t):
+    n, m, d = 90, 70, 16
+    P, Q = W.random_points(dtype, n, d, 1), W.random_points(dtype, m, d, 2)
+    base, cnt = O.join(P, Q, kind, t, dtype)
+    S = as_set(base)
+    assert 0 < cnt < n * m, "test threshold should split the pairs"
+    # join(Q, P) is the transpose
+    tr, _c = O.join(Q, P, kind, t, dtype)
+    assert {(j, i) for (i, j) in as_set(tr)} == S
+    # self join: symmetric and (for these kinds at these thresholds) reflexive where defined
+    self_pairs, _c = O.join(P, P, kind, t, dtype)
+    SS = as_set(self_pairs)
+    assert {(j, i) for (i, j) in SS} == SS
+    if kind in ("l2", "cos"):
+        assert all((i, i) in SS for i in range(n))
+    # monotone in the threshold
+    t_more = t + 0.5 if kind == "l2" else t - 0.5
+    more, _c = O.join(P, Q, kind, t_more, dtype)
+    assert S <= as_set(more)
+    # extreme thresholds: everything / nothing
+    big = 1e30
+    everything, c_all = O.join(P, Q, kind, big if kind == "l2" else -big, dtype)
+    assert c_all == n * m and everything.tolist() == [[i, j] for i in range(n) for j in range(m)]
+    if kind != "l2":
+        assert O.join(P, Q, kind, big, dtype)[1] == 0
+    # Theorem 1's block decomposition: the union over any row/column split is the whole join
+    for r_cut, c_cut in [(1, 1), (37, 64), (89, 3)]:
+        U = set()
+        for (r0, r1) in [(0, r_cut), (r_cut, n)]:
+            for (c0, c1) in [(0, c_cut), (c_cut, m)]:
+                part, _c = O.join(P[r0:r1], Q[c0:c1], kind, t, dtype)
+                U |= {(i + r0, j + c0) for (i, j) in as_set(part)}
+        assert U == S
+    # permuting the rows of P permutes i
+    perm = np.random.default_rng(9).permutation(n)
+    pp, _c = O.join(P[perm], Q, kind, t, dtype)
+    assert {(int(perm[i]), j) for (i, j) in as_set(pp)} == S
+    # appending zero columns changes no score
+    Pz = np.concatenate([P, np.zeros((n, 5), dtype=P.dtype)], axis=1)
+    Qz = np.concatenate([Q, np.zeros((m, 5), dtype=Q.dtype)], axis=1)
+    assert as_set(O.join(Pz, Qz, kind, t, dtype)[0]) == S
+    # capacity smaller than the result: count is still the total, prefix is the sorted prefix
+    few, c_few = O.join(P, Q, kind, t, dtype, capacity=5)
+    assert c_few == cnt and few.tolist() == base[:5].tolist()
+    # thread count does not change the result
+    one, c_one = O.join(P, Q, kind, t, dtype, threads=1)
+    assert c_one == cnt and np.array_equal(one, base)
+
+
+def test_band_sets_are_nested():
+    w = W.make_workload(2, n=300, m=300, planted=20)
+    s_strict, s_exact, s_loose = O.band_sets(w.P, w.Q, "cos", 0.1, "bf16")
+    assert as_set(s_strict) <= as_set(s_exact) <= as_set(s_loose)
+    assert len(s_strict) < len(s_loose)
+    w5 = W.make_workload(5, n=300, m=300, centers=8)
+    a, b, c = O.band_sets(w5.P, w5.Q, "l2", 0.07, "bf16")
+    assert as_set(a) <= as_set(b) <= as_set(c) and len(a) < len(c)
+
+
+def test_empty_and_rejected_inputs():
+    P = np.zeros((0, 8), dtype=np.int8)
+    Q = np.ones((4, 8), dtype=np.int8)
+    assert O.join(P, Q, "ip", 0, "i8")[1] == 0
+    assert O.join(Q, P, "ip", 0, "i8")[1] == 0
+    with pytest.raises(ValueError):
+        O.join(Q, Q, "l2", -1.0, "i8")
+    with pytest.raises(ValueError):
+        O.join(Q, Q, "ip", float("nan"), "i8")
+    with pytest.raises(ValueError):
+        O.join(Q, Q, "cos", 0.5, "i8")
+
+
+def test_planted_scores_match_the_recipes():
+    w1 = W.make_workload(1)
+    assert np.all(O.scores(w1.P, w1.Q, "ip", "i8", w1.planted) == 64 - 2 * 4)
+    w4 = W.make_workload(4, n=3000, m=2000, planted=100)
+    assert np.all(O.scores(w4.P, w4.Q, "ip", "i8", w4.planted) == 128 - 2 * 8)
+    w3 = W.make_workload(3, n=3000, m=2000, planted=100)
+    s3 = O.scores(w3.P, w3.Q, "ip", "i8", w3.planted)
+    assert s3.min() > 4000 and abs(s3.mean() - 256 * 24) < 300     # E<x,x> = d*E[x^2] = 256*24
+    w2 = W.make_workload(2, n=3000, m=2000, planted=100)
+    c2 = O.scores(w2.P, w2.Q, "cos", "bf16", w2.planted)
+    assert c2.min() > 0.93 and abs(c2.mean() - 1 / math.sqrt(1.09)) < 5e-3

@@ -1,0 +1,53 @@
+"""The seeded input generators: determinism, shapes, value ranges, planted structure.
+Nothing here evaluates a join score."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2006_12608_b200 import workloads as W
+
+
+def test_bf16_bit_conversion_matches_torch_cast():
+    a = np.random.default_rng(0).standard_normal(10000).astype(np.float32) * 3
+    a[:4] = [0.0, -0.0, 1.0, 65504.0]
+    bits = W.f32_to_bf16_bits(a)
+    t = torch.from_numpy(a).to(torch.bfloat16)
+    assert np.array_equal(bits.view(np.int16), t.view(torch.int16).numpy())
+    assert np.array_equal(W.bf16_bits_to_f32(bits), t.to(torch.float32).numpy())
+
+
+@pytest.mark.parametrize("cfg,kw", [(1, {}), (2, dict(n=500, m=300, planted=20)), (3, dict(n=400, m=600, planted=30)),
+                                    (4, dict(n=700, m=900, planted=50)), (5, dict(n=500, m=400, centers=16))])
+def test_deterministic_and_well_formed(cfg, kw):
+    a, b = W.make_workload(cfg, **kw), W.make_workload(cfg, **kw)
+    assert np.array_equal(a.P, b.P) and np.array_equal(a.Q, b.Q) and np.array_equal(a.planted, b.planted)
+    c = W.make_workload(cfg, seed=1, **kw)
+    assert not np.array_equal(a.P, c.P)
+    assert a.P.shape == (a.n, a.d) and a.Q.shape == (a.m, a.d)
+    assert a.P.dtype == (np.int8 if a.dtype == "i8" else np.uint16)
+    assert a.P.flags["C_CONTIGUOUS"] and a.Q.flags["C_CONTIGUOUS"]
+    assert a.ops == 2 * a.n * a.m * a.d
+    if len(a.planted):
+        assert len(np.unique(a.planted[:, 0])) == len(a.planted) == len(np.unique(a.planted[:, 1]))
+
+
+def test_planted_structure():
+    w = W.make_workload(1)
+    assert set(np.unique(w.P)) == {-1, 1} and set(np.unique(w.Q)) == {-1, 1}
+    x, y = w.P[w.planted[:, 0]], w.Q[w.planted[:, 1]]
+    assert np.all((x != y).sum(axis=1) == 4)
+    w4 = W.make_workload(4, n=5000, m=4000, planted=300)
+    assert np.all((w4.P[w4.planted[:, 0]] != w4.Q[w4.planted[:, 1]]).sum(axis=1) == 8)
+    w3 = W.make_workload(3, n=5000, m=4000, planted=300)
+    assert w3.P.min() == -8 and w3.P.max() == 8
+    e = w3.Q[w3.planted[:, 1]].astype(int) - w3.P[w3.planted[:, 0]].astype(int)
+    assert set(np.unique(e)) == {-1, 0, 1} and abs(w3.Q).max() == 9
+
+
+def test_full_size_parameters_match_the_benchmark_table():
+    c = W.CONFIGS
+    assert (c[1]["n"], c[1]["d"], c[1]["threshold"], c[1]["planted"]) == (2048, 64, 40.0, 32)
+    assert (c[2]["n"], c[2]["d"], c[2]["threshold"], c[2]["planted"]) == (65536, 128, 0.9, 1000)
+    assert (c[3]["n"], c[3]["d"], c[3]["threshold"], c[3]["planted"]) == (262144, 256, 3000.0, 10000)
+    assert (c[4]["n"], c[4]["d"], c[4]["threshold"], c[4]["planted"]) == (1048576, 128, 100.0, 100000)
+    assert (c[5]["n"], c[5]["d"], c[5]["threshold"], c[5]["centers"]) == (524288, 64, 0.25, 1024)
