@@ -1,0 +1,154 @@
+/*
+ * simjoin.h -- C ABI of the B200 (sm_100a) thresholded all-pairs similarity join.
+ *
+ * The operation is the similarity join of Section 4 of arXiv 2006.12608:
+ *   P join_r Q = { (x, y) : x in P, y in Q, D(x, y) <= r }
+ * for the ip-distances that section lists, evaluated by the brute-force route
+ * it describes: the product F_P * G_Q^T, decomposed into small dense tile
+ * products (Theorem 1) that run on the tensor cores.  Rows are identified by
+ * their index, so the result is a set of index pairs (i, j), 0-based, i a row
+ * of P and j a row of Q.  The n x m score matrix is never materialised: the
+ * threshold and the compaction of passing pairs are fused behind each tile
+ * product.
+ *
+ * Conventions
+ *   - "device pointer": memory of the context's CUDA device (e.g. the
+ *     data_ptr() of a torch tensor).  "host pointer": ordinary host memory.
+ *   - Matrices are row-major with the d coordinates of a point contiguous.
+ *     Rows must start on 16-byte boundaries: the base pointer is 16-byte
+ *     aligned and d * sizeof(element) is a multiple of 16 (pad with zero
+ *     columns otherwise: zero columns change no score).
+ *   - Nothing the caller passes is freed or retained after a call returns.
+ *     P and Q are only read.
+ *   - No function throws, prints or exits; every failure is a status code.
+ *   - A context is not thread-safe; use one per host thread / stream.
+ */
+#ifndef SIMJOIN_H_
+#define SIMJOIN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct simjoin_ctx simjoin_ctx; /* opaque; owned by the library */
+
+typedef enum {
+    SIMJOIN_I8 = 0,  /* int8 coordinates, exact int32 accumulation              */
+    SIMJOIN_BF16 = 1 /* bfloat16 coordinates, fp32 accumulation                 */
+} simjoin_dtype;
+
+typedef enum {
+    SIMJOIN_IP = 0,  /* keep (i,j) when <x_i, y_j>                  >= threshold */
+    SIMJOIN_COS = 1, /* keep (i,j) when <x_i, y_j>/(|x_i| |y_j|)    >= threshold;
+                        the cosine with a zero vector counts as 0                */
+    SIMJOIN_L2 = 2   /* keep (i,j) when |x_i - y_j| <= threshold (threshold >= 0),
+                        evaluated as |x|^2 + |y|^2 - 2<x,y> <= threshold^2       */
+} simjoin_kind;
+
+typedef enum {
+    SIMJOIN_OK = 0,
+    SIMJOIN_ERR_ARG = 1,         /* null / negative / NaN / wrong pointer kind    */
+    SIMJOIN_ERR_UNSUPPORTED = 2, /* alignment, d too large, dtype x kind missing  */
+    SIMJOIN_ERR_CAPACITY = 3,    /* more passing pairs than `capacity`            */
+    SIMJOIN_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed           */
+    SIMJOIN_ERR_TIMEOUT = 5,     /* a bounded wait inside the kernel ran out      */
+    SIMJOIN_ERR_ARCH = 6         /* the device is not compute capability 10.x     */
+} simjoin_status;
+
+/* Limits of this build. */
+#define SIMJOIN_MAX_ROWS 2147483647LL /* n, m < 2^31 (pairs are int32)          */
+#define SIMJOIN_MAX_ROW_BYTES 8192    /* d * sizeof(element) <= 8192             */
+
+/*
+ * Create a context for joins over `dtype` points on CUDA device `device`,
+ * enqueueing on `cuda_stream` (a cudaStream_t; NULL = the legacy default
+ * stream).  The stream stays owned by the caller and must outlive the context.
+ * The context owns its scratch (row norms, per-tile norm bounds, a 64-byte
+ * counter/status block, staging buffers of simjoin_run_host), grown on demand
+ * with cudaMalloc and released by simjoin_destroy.
+ * Errors: ERR_ARG (null ctx, unknown dtype, bad device), ERR_ARCH, ERR_CUDA.
+ */
+simjoin_status simjoin_create(simjoin_ctx **ctx, simjoin_dtype dtype, int device, void *cuda_stream);
+
+/*
+ * The join (Section 4: join definition; brute-force product F_P * G_Q^T).
+ *
+ *   P, Q        device pointers, n x d and m x d, row-major, read-only.
+ *   kind        see simjoin_kind.  Supported: I8 x {IP, L2}, BF16 x {IP, COS, L2}.
+ *   threshold   t (IP, COS) or r (L2).  I8/IP passes when the integer score s
+ *               satisfies s >= t over the reals; I8/L2 when the integer squared
+ *               distance D satisfies D <= floor(r*r), r*r the double product.
+ *               BF16 kinds compare fp32 scores; pairs whose exact score lies
+ *               within 1e-2*|threshold| of the threshold may fall on either side.
+ *   out_pairs   device pointer to capacity x 2 int32, written as (i, j) rows.
+ *               May be NULL when capacity == 0 (count-only mode).
+ *   count       HOST pointer; receives the total number of passing pairs, even
+ *               when that exceeds `capacity`.
+ *
+ * Exactly min(*count, capacity) rows of out_pairs are written, each passing
+ * pair at most once, in unspecified order.  When *count > capacity the written
+ * subset is arbitrary but valid and the call returns ERR_CAPACITY.
+ * The call enqueues on the context's stream and synchronises that stream
+ * before it returns.  n == 0 or m == 0 gives OK with *count = 0.
+ *
+ * Errors, all detected before any launch: ERR_ARG (null ctx/P/Q/count, n or m
+ * negative or >= 2^31, d <= 0, NaN threshold, L2 with threshold < 0, a host
+ * pointer where a device pointer is required, out_pairs NULL with capacity > 0);
+ * ERR_UNSUPPORTED (misaligned base pointer, d*sizeof(element) not a multiple
+ * of 16 or above SIMJOIN_MAX_ROW_BYTES, I8 x COS).  After launch: ERR_CUDA,
+ * ERR_TIMEOUT (a wait in the kernel gave up; the context stays usable),
+ * ERR_CAPACITY.
+ */
+simjoin_status simjoin_run(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m,
+                           int32_t d, simjoin_kind kind, double threshold, int32_t *out_pairs,
+                           uint64_t capacity, uint64_t *count);
+
+/*
+ * Same join with HOST buffers: P, Q and out_pairs are host pointers.  The call
+ * copies P and Q to device staging owned by the context, runs the join, and
+ * copies min(*count, capacity) pairs back; all on the context's stream,
+ * synchronised before return.  Pinned host memory makes the copies faster but
+ * is not required.  Errors as simjoin_run (device pointers are rejected here).
+ */
+simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n, const void *Q_host,
+                                int64_t m, int32_t d, simjoin_kind kind, double threshold,
+                                int32_t *out_pairs_host, uint64_t capacity, uint64_t *count);
+
+/*
+ * Row squared norms, the pre-pass behind the |x|^2 and |y|^2 terms of the
+ * squared-L2 and cosine ip-distances (Section 4).  X: device pointer, rows x d.
+ * out: device pointer to `rows` values -- int32 (exact) for I8 contexts, fp32
+ * for BF16 contexts.  Synchronises the stream before returning.
+ * Errors: ERR_ARG, ERR_UNSUPPORTED (alignment / row bytes as above), ERR_CUDA.
+ */
+simjoin_status simjoin_row_norms(simjoin_ctx *ctx, const void *X, int64_t rows, int32_t d, void *out);
+
+/*
+ * Offsets added to every emitted pair: (i + row_offset_p, j + row_offset_q).
+ * Lets a caller that shards P (or Q) by row blocks over several GPUs or calls
+ * obtain global indices directly (Theorem 1's block decomposition: the union
+ * of the joins of the blocks is the join).  Both default to 0.  The sums must
+ * stay below 2^31: ERR_ARG otherwise (checked again in simjoin_run).
+ */
+simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64_t row_offset_q);
+
+/*
+ * Device time of the kernels of the last successful simjoin_run /
+ * simjoin_run_host on this context, in milliseconds, measured with CUDA events
+ * on the context's stream: the norm pre-pass (0 when the kind needs none) and
+ * the join kernel.  Either pointer may be NULL.  ERR_ARG if nothing has run.
+ */
+simjoin_status simjoin_last_kernel_ms(simjoin_ctx *ctx, float *prepass_ms, float *join_ms);
+
+/* Release the context and its scratch.  NULL is accepted. */
+simjoin_status simjoin_destroy(simjoin_ctx *ctx);
+
+/* Static, human-readable name of a status code. */
+const char *simjoin_strerror(simjoin_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SIMJOIN_H_ */

@@ -1,0 +1,375 @@
+// The fused similarity-join kernel for sm_100a.
+//
+// Section 4 of the paper reduces the join to the product F_P * G_Q^T and Theorem 1
+// decomposes that product into small dense tile products.  Here one tile product is a
+// 128 x 256 block of scores: 128 rows of P against 256 rows of Q over all d coordinates,
+// computed by tcgen05.mma from 128-byte-swizzled shared-memory tiles that TMA fills, with
+// the accumulator in tensor memory.  The rest of the ip-distance (row norms, Section 4's
+// squared-L2 and cosine forms) and the threshold are applied to the accumulator in
+// registers and passing (i, j) are compacted straight into the output list.
+//
+// CTA layout (384 threads, one CTA per SM, persistent):
+//   warp 0      TMA producer: P row block (resident while its Q sweep lasts) + Q chunk ring
+//   warp 1      MMA issuer (lane 0 issues), double-buffered 2 x 256-column accumulators
+//   warp 2      TMEM allocation / release
+//   warp 3      idle
+//   warps 4-11  epilogue: warp w reads TMEM lanes 32*(w%4).., column half (w-4)/4
+// Every mbarrier wait is bounded; on expiry the CTA raises a status word and drains.
+#pragma once
+#include "ptx_sm100.cuh"
+
+namespace sj {
+
+constexpr int DT_I8 = 0, DT_BF16 = 1;
+constexpr int KIND_IP = 0, KIND_COS = 1, KIND_L2 = 2;
+
+constexpr int TILE_M = 128;                       // rows of P per tile
+constexpr int TILE_N = 256;                       // rows of Q per tile
+constexpr int CHUNK_BYTES = 128;                  // K bytes per shared-memory chunk (one swizzle atom)
+constexpr int A_CHUNK_BYTES = TILE_M * CHUNK_BYTES;   // 16 KiB
+constexpr int B_CHUNK_BYTES = TILE_N * CHUNK_BYTES;   // 32 KiB
+constexpr int MAX_STAGES = 6;
+constexpr int MAX_STATIONARY_CHUNKS = 4;          // P block kept resident up to 512-byte rows
+constexpr int NUM_THREADS = 384;
+constexpr int EPI_WARP0 = 4;
+constexpr int NUM_EPI_WARPS = 8;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;  // ~1 s: far beyond any legitimate wait
+constexpr int CTRL_BYTES = 256;
+
+struct JoinParams {
+    long long n, m;          // rows of P, Q
+    int kc;                  // 128-byte K chunks per row = ceil(row_bytes / 128)
+    int last_ksteps;         // 32-byte MMA K steps in the last chunk (1..4)
+    int elems_per_chunk;     // 128 / sizeof(element)
+    int stationary;          // 1: the P block stays in shared memory for its whole Q sweep
+    int nstages;             // ring depth
+    int PB, QT;              // number of 128-row P blocks, 256-row Q tiles
+    int thr_i;               // I8/IP: ceil(t);  I8/L2: floor(r*r); both clamped
+    float thr_f;             // BF16: t (IP, COS) or r*r (L2)
+    const void *nx;          // per-row term of P: int32 |x|^2 (I8/L2), fp32 |x| (COS) or |x|^2 (L2)
+    const void *ny;          // same for Q
+    const void *qstat;       // per 256-row Q tile: (min, max) of ny over the tile's valid rows
+    int2 *out;               // capacity x (i, j)
+    unsigned long long capacity;
+    unsigned long long *counter;   // total passing pairs
+    unsigned int *status;          // 0 = ok, else 0x80000000 | wait site that timed out
+    int ioff, joff;          // added to emitted indices
+};
+
+struct Ctrl {
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES];
+    uint64_t pfull[2], pempty[2];
+    uint64_t tfull[2], tempty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    volatile uint32_t abort;
+};
+static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
+
+// One unit of work: P block `pb` against Q tiles [q0, q1).  CTAs take whole Q sweeps in
+// waves of gridDim.x P blocks (all CTAs then walk Q together, so a Q tile is fetched from
+// HBM once and served from L2 to everyone else); the last, partial wave splits each of
+// its sweeps over several CTAs.
+struct Unit { int pb, q0, q1; };
+__device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
+    const int G = gridDim.x, c = blockIdx.x;
+    const int full = p.PB / G, rem = p.PB - full * G;
+    if (u < full) { un.pb = u * G + c; un.q0 = 0; un.q1 = p.QT; return true; }
+    if (u == full && rem > 0) {
+        const int S = G / rem, idx = c / S, seg = c - idx * S;
+        if (idx >= rem) return false;
+        un.pb = full * G + idx;
+        un.q0 = (int)((long long)seg * p.QT / S);
+        un.q1 = (int)((long long)(seg + 1) * p.QT / S);
+        return un.q1 > un.q0;
+    }
+    return false;
+}
+
+// Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting.
+__device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *ctrl, unsigned int *status, uint32_t site) {
+    const uint32_t addr = smem_u32(bar);
+    if (mbar_try_wait(addr, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(addr, parity)) return true;
+        if ((it & 0x3F) == 0) {
+            if (ctrl->abort) return false;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                ctrl->abort = 1;
+                atomicCAS(status, 0u, 0x80000000u | site);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool wait_bar_warp(uint64_t *bar, uint32_t parity, Ctrl *ctrl, unsigned int *status, uint32_t site) {
+    const bool ok = wait_bar(bar, parity, ctrl, status, site);
+    return __all_sync(0xffffffffu, ok);
+}
+
+// Compact the pairs (i, j0 + c), c in `mask`, of the 32 rows this warp owns into the
+// output list: popcount prefix over the warp, one atomic per warp, 8-byte stores.
+__device__ __forceinline__ void emit_pairs(const JoinParams &p, uint32_t mask, int lane, long long i, long long j0) {
+    const int cnt = __popc(mask);
+    int incl = cnt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += t;
+    }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    if (total == 0) return;
+    unsigned long long base = 0;
+    if (lane == 0) base = atomicAdd(p.counter, (unsigned long long)total);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    unsigned long long slot = base + (unsigned long long)(incl - cnt);
+    while (mask) {
+        const int c = __ffs(mask) - 1;
+        mask &= mask - 1;
+        if (slot < p.capacity) p.out[slot] = make_int2((int)(i + p.ioff), (int)(j0 + c + p.joff));
+        ++slot;
+    }
+}
+
+template <int DT, int KIND>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ, const JoinParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // 1024-byte alignment: the 128-byte swizzle pattern repeats every 1024 bytes.
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int p_bytes = p.stationary ? 2 * p.kc * A_CHUNK_BYTES : 0;
+    const int stage_bytes = B_CHUNK_BYTES + (p.stationary ? 0 : A_CHUNK_BYTES);
+    uint8_t *smem_p = smem;
+    uint8_t *smem_ring = smem + p_bytes;
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem_ring + (size_t)p.nstages * stage_bytes);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.nstages; ++s) { mbar_init(smem_u32(&ctrl->full[s]), 1); mbar_init(smem_u32(&ctrl->empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&ctrl->pfull[b]), 1);
+            mbar_init(smem_u32(&ctrl->pempty[b]), 1);
+            mbar_init(smem_u32(&ctrl->tfull[b]), 1);
+            mbar_init(smem_u32(&ctrl->tempty[b]), NUM_EPI_WARPS);
+        }
+        mbar_init(smem_u32(&ctrl->drain), 1);
+        ctrl->abort = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&mapP);
+        prefetch_tensormap(&mapQ);
+    }
+    if (warp == 2) {
+        tmem_alloc(smem_u32(&ctrl->tmem_base), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------- TMA producer
+        uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0;
+        bool ok = true;
+        Unit un;
+        for (int u = 0; ok && get_unit(p, u, un); ++u) {
+            if (p.stationary) {
+                ok = wait_bar_warp(&ctrl->pempty[pbuf], pphase ^ 1, ctrl, p.status, 1);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t bar = smem_u32(&ctrl->pfull[pbuf]);
+                    mbar_arrive_expect_tx(bar, (uint32_t)(p.kc * A_CHUNK_BYTES));
+                    for (int c = 0; c < p.kc; ++c)
+                        tma_load_2d(smem_u32(smem_p + (size_t)(pbuf * p.kc + c) * A_CHUNK_BYTES), &mapP, bar,
+                                    c * p.elems_per_chunk, un.pb * TILE_M);
+                }
+                __syncwarp();
+                pbuf ^= 1;
+                if (pbuf == 0) pphase ^= 1;
+            }
+            for (int qt = un.q0; ok && qt < un.q1; ++qt) {
+                for (int c = 0; c < p.kc; ++c) {
+                    ok = wait_bar_warp(&ctrl->empty[stage], phase ^ 1, ctrl, p.status, 2);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        const uint32_t bar = smem_u32(&ctrl->full[stage]);
+                        uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
+                        mbar_arrive_expect_tx(bar, (uint32_t)stage_bytes);
+                        tma_load_2d(smem_u32(sb), &mapQ, bar, c * p.elems_per_chunk, qt * TILE_N);
+                        if (!p.stationary)
+                            tma_load_2d(smem_u32(sb + B_CHUNK_BYTES), &mapP, bar, c * p.elems_per_chunk, un.pb * TILE_M);
+                    }
+                    __syncwarp();
+                    if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+        if (!ok && lane == 0) {
+            // aborting: give copies already in flight time to land before shared memory is released
+            for (int t = 0; t < 200; ++t) __nanosleep(1000);
+        }
+    } else if (warp == 1) {
+        // --------------------------------------------------------------- MMA issuer
+        constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, TILE_N);
+        uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0, acc = 0, accphase = 0;
+        bool ok = true;
+        Unit un;
+        for (int u = 0; ok && get_unit(p, u, un); ++u) {
+            if (p.stationary) {
+                ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
+                if (!ok) break;
+            }
+            for (int qt = un.q0; ok && qt < un.q1; ++qt) {
+                ok = wait_bar_warp(&ctrl->tempty[acc], accphase ^ 1, ctrl, p.status, 4);
+                if (!ok) break;
+                tc_fence_after();
+                for (int c = 0; c < p.kc; ++c) {
+                    ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
+                        const uint32_t a_addr = p.stationary ? smem_u32(smem_p + (size_t)(pbuf * p.kc + c) * A_CHUNK_BYTES)
+                                                             : smem_u32(sb + B_CHUNK_BYTES);
+                        const uint64_t adesc = umma_desc_sw128_kmajor(a_addr);
+                        const uint64_t bdesc = umma_desc_sw128_kmajor(smem_u32(sb));
+                        const int ksteps = (c == p.kc - 1) ? p.last_ksteps : 4;
+                        for (int k = 0; k < ksteps; ++k)
+                            umma_ss<DT == DT_I8>(tmem_base + acc * TILE_N, adesc + 2 * k, bdesc + 2 * k, idesc,
+                                                 (c | k) != 0 ? 1u : 0u);
+                        umma_commit(smem_u32(&ctrl->empty[stage]));
+                    }
+                    __syncwarp();
+                    if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                if (lane == 0) umma_commit(smem_u32(&ctrl->tfull[acc]));
+                __syncwarp();
+                acc ^= 1;
+                if (acc == 0) accphase ^= 1;
+            }
+            if (ok && p.stationary) {
+                if (lane == 0) umma_commit(smem_u32(&ctrl->pempty[pbuf]));
+                __syncwarp();
+                pbuf ^= 1;
+                if (pbuf == 0) pphase ^= 1;
+            }
+        }
+        if (!ok) {
+            // aborting: wait (bounded) until the MMAs already issued have retired
+            if (lane == 0) {
+                umma_commit(smem_u32(&ctrl->drain));
+                const long long t0 = clock64();
+                while (!mbar_try_wait(smem_u32(&ctrl->drain), 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+            }
+            __syncwarp();
+        }
+    } else if (warp >= EPI_WARP0) {
+        // ------------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;               // TMEM lane quarter this warp may read
+        const int half = (warp - EPI_WARP0) >> 2;   // which 128 of the tile's 256 columns
+        const int row_in_tile = quarter * 32 + lane;
+        uint32_t acc = 0, accphase = 0;
+        bool ok = true;
+        Unit un;
+        for (int u = 0; ok && get_unit(p, u, un); ++u) {
+            const long long i = (long long)un.pb * TILE_M + row_in_tile;
+            const bool row_ok = i < p.n;
+            int ri = 0;          // I8/L2: |x|^2 - floor(r^2)
+            float rf = 0.f;      // COS: t*|x|;  BF16/L2: |x|^2
+            bool rzero = false;  // COS: x is the zero vector
+            if (row_ok) {
+                if constexpr (DT == DT_I8 && KIND == KIND_L2) ri = reinterpret_cast<const int *>(p.nx)[i] - p.thr_i;
+                if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
+                    const float nxr = reinterpret_cast<const float *>(p.nx)[i];
+                    rf = p.thr_f * nxr;
+                    rzero = nxr == 0.f;
+                }
+                if constexpr (DT == DT_BF16 && KIND == KIND_L2) rf = reinterpret_cast<const float *>(p.nx)[i];
+            }
+            for (int qt = un.q0; ok && qt < un.q1; ++qt) {
+                // per-tile filter bound: a necessary condition on max_j s_ij for row i to have any hit
+                int fi = p.thr_i;
+                float ff = p.thr_f;
+                if constexpr (DT == DT_I8 && KIND == KIND_L2) {
+                    const int2 st = reinterpret_cast<const int2 *>(p.qstat)[qt];
+                    fi = (ri + st.x + 1) >> 1;                    // 2s >= |x|^2 - R + min|y|^2
+                }
+                if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
+                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt];
+                    ff = rf * (p.thr_f >= 0.f ? st.x : st.y);     // s >= t|x| * min|y| (max|y| when t < 0)
+                }
+                if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
+                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt];
+                    ff = rf + st.x;                               // (|x|^2 + min|y|^2) - 2s <= r^2
+                }
+                ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll 1
+                for (int cc = 0; cc < 4; ++cc) {
+                    const int col = half * 128 + cc * 32;
+                    uint32_t v[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + col, v);
+                    bool hit;
+                    if constexpr (DT == DT_I8) {
+                        int mx = (int)v[0];
+#pragma unroll
+                        for (int c = 1; c < 31; c += 2) mx = __vimax3_s32(mx, (int)v[c], (int)v[c + 1]);
+                        mx = max(mx, (int)v[31]);
+                        hit = row_ok && mx >= fi;
+                    } else {
+                        float mx = __uint_as_float(v[0]);
+#pragma unroll
+                        for (int c = 1; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(v[c]));
+                        if constexpr (KIND == KIND_L2) hit = row_ok && (ff - 2.f * mx) <= p.thr_f;
+                        else hit = row_ok && mx >= ff;
+                    }
+                    if (__any_sync(0xffffffffu, hit)) {
+                        // exact per-element test for this 32 x 32 block
+                        const long long j0 = (long long)qt * TILE_N + col;
+                        uint32_t mask = 0;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            const long long j = j0 + c;
+                            bool pass = false;
+                            if (j < p.m) {
+                                if constexpr (DT == DT_I8 && KIND == KIND_IP) pass = (int)v[c] >= p.thr_i;
+                                if constexpr (DT == DT_I8 && KIND == KIND_L2)
+                                    pass = 2 * (int)v[c] - reinterpret_cast<const int *>(p.ny)[j] >= ri;
+                                if constexpr (DT == DT_BF16 && KIND == KIND_IP) pass = __uint_as_float(v[c]) >= p.thr_f;
+                                if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
+                                    const float nyr = reinterpret_cast<const float *>(p.ny)[j];
+                                    pass = (rzero || nyr == 0.f) ? (p.thr_f <= 0.f) : (__uint_as_float(v[c]) >= rf * nyr);
+                                }
+                                if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
+                                    const float ny2 = reinterpret_cast<const float *>(p.ny)[j];
+                                    pass = ((rf + ny2) - 2.f * __uint_as_float(v[c])) <= p.thr_f;
+                                }
+                            }
+                            mask |= (pass ? 1u : 0u) << c;
+                        }
+                        if (!row_ok) mask = 0;
+                        emit_pairs(p, mask, lane, i, j0);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                acc ^= 1;
+                if (acc == 0) accphase ^= 1;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace sj

@@ -1,0 +1,108 @@
+// Row-norm pre-pass: |x|^2 per row (the |x|^2, |y|^2 terms of Section 4's squared-L2
+// ip-distance and the 1/|x| scaling of its cosine form), plus, per 256-row tile, the
+// minimum and maximum of the stored values, which the join kernel turns into a per-tile
+// bound that lets it skip whole blocks of the score tile.  Memory-bound: every input
+// byte is read once with 16-byte loads.
+#pragma once
+#include <cstdint>
+#include <cuda_bf16.h>
+
+namespace sj {
+
+constexpr int NORM_TILE_ROWS = 256;
+constexpr int NORM_THREADS = 256;
+
+template <bool kInt8>
+struct NormAcc;
+template <>
+struct NormAcc<true> {
+    using type = int;
+    static __device__ __forceinline__ int add16(int acc, const uint4 &q) {
+        acc = __dp4a((int)q.x, (int)q.x, acc);
+        acc = __dp4a((int)q.y, (int)q.y, acc);
+        acc = __dp4a((int)q.z, (int)q.z, acc);
+        acc = __dp4a((int)q.w, (int)q.w, acc);
+        return acc;
+    }
+};
+template <>
+struct NormAcc<false> {
+    using type = float;
+    static __device__ __forceinline__ float add16(float acc, const uint4 &q) {
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const float lo = __uint_as_float(w[t] << 16), hi = __uint_as_float(w[t] & 0xffff0000u);
+            acc = fmaf(lo, lo, acc);
+            acc = fmaf(hi, hi, acc);
+        }
+        return acc;
+    }
+};
+
+// X: rows x (g * 16 bytes).  norms[r] = sum of squares of row r (fp32: its square root when
+// sqrt_out).  tile_minmax[b] = (min, max) of norms over the valid rows of tile b (may be null).
+template <bool kInt8>
+__global__ void __launch_bounds__(NORM_THREADS)
+row_norms_kernel(const uint4 *__restrict__ X, long long rows, int g, int sqrt_out,
+                 typename NormAcc<kInt8>::type *__restrict__ norms,
+                 typename NormAcc<kInt8>::type *__restrict__ tile_minmax) {
+    using T = typename NormAcc<kInt8>::type;
+    __shared__ T s_val[NORM_TILE_ROWS];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long row0 = (long long)blockIdx.x * NORM_TILE_ROWS + warp * 32;   // this warp's 32 rows
+    const bool pow2 = g <= 32 && (g & (g - 1)) == 0;
+    if (pow2) {
+        // g lanes share a row: 32/g rows per pass, g passes; all loads of a warp are contiguous
+        const int rpp = 32 / g, sub = lane / g, chunk = lane - sub * g;
+#pragma unroll 4
+        for (int pass = 0; pass < g; ++pass) {
+            const int rl = pass * rpp + sub;
+            const long long r = row0 + rl;
+            T acc = 0;
+            if (r < rows) acc = NormAcc<kInt8>::add16(acc, __ldg(X + r * g + chunk));
+            for (int off = g >> 1; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            if (chunk == 0) s_val[warp * 32 + rl] = acc;
+        }
+    } else {
+        for (int rl = 0; rl < 32; ++rl) {
+            const long long r = row0 + rl;
+            T acc = 0;
+            if (r < rows)
+                for (int c = lane; c < g; c += 32) acc = NormAcc<kInt8>::add16(acc, __ldg(X + r * g + c));
+            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            if (lane == 0) s_val[warp * 32 + rl] = acc;
+        }
+    }
+    __syncthreads();
+    const long long r = (long long)blockIdx.x * NORM_TILE_ROWS + threadIdx.x;
+    T v = s_val[threadIdx.x];
+    if constexpr (!kInt8) { if (sqrt_out) v = sqrtf(v); }
+    const bool valid = r < rows;
+    if (valid) norms[r] = v;
+    if (tile_minmax == nullptr) return;
+    // block min / max over valid rows (row 0 of a launched tile is always valid)
+    __syncthreads();
+    s_val[threadIdx.x] = v;
+    __syncthreads();
+    const T first = s_val[0];
+    T mn = valid ? v : first, mx = mn;
+    for (int off = 16; off > 0; off >>= 1) {
+        const T a = __shfl_xor_sync(0xffffffffu, mn, off), b = __shfl_xor_sync(0xffffffffu, mx, off);
+        mn = a < mn ? a : mn;
+        mx = b > mx ? b : mx;
+    }
+    __shared__ T s_mn[NORM_THREADS / 32], s_mx[NORM_THREADS / 32];
+    if (lane == 0) { s_mn[warp] = mn; s_mx[warp] = mx; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < NORM_THREADS / 32; ++w) {
+            mn = s_mn[w] < mn ? s_mn[w] : mn;
+            mx = s_mx[w] > mx ? s_mx[w] : mx;
+        }
+        tile_minmax[2 * (long long)blockIdx.x] = mn;
+        tile_minmax[2 * (long long)blockIdx.x + 1] = mx;
+    }
+}
+
+}  // namespace sj

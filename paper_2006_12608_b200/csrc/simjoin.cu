@@ -1,0 +1,426 @@
+// Host side of the C ABI declared in include/simjoin.h: argument checks, scratch
+// management, TMA descriptors, launches of the pre-pass and the fused join kernel.
+#include "../../include/simjoin.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "join_kernel.cuh"
+#include "prepass_kernel.cuh"
+
+namespace {
+
+using namespace sj;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DevBuf {
+    void *ptr = nullptr;
+    size_t bytes = 0;
+};
+
+}  // namespace
+
+struct simjoin_ctx {
+    simjoin_dtype dtype;
+    int device;
+    cudaStream_t stream;
+    int num_sms;
+    int max_smem_optin;
+    EncodeTiledFn encode;
+    DevBuf nx, ny, qstat, pstat;        // row terms and per-tile bounds
+    DevBuf stage_p, stage_q, stage_out; // device staging of simjoin_run_host
+    unsigned long long *d_ctrl;         // [0] pair counter, [1] status word (low 32 bits)
+    unsigned long long *h_ctrl;         // pinned mirror
+    cudaEvent_t ev[4];
+    bool have_timing;
+    float prepass_ms, join_ms;
+    long long ioff, joff;
+    bool attr_set[2][3];
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+bool grow(DevBuf &b, size_t bytes) {
+    if (bytes <= b.bytes) return true;
+    if (b.ptr) cudaFree(b.ptr);
+    b.ptr = nullptr;
+    b.bytes = 0;
+    if (cudaMalloc(&b.ptr, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    b.bytes = bytes;
+    return true;
+}
+
+void release(DevBuf &b) {
+    if (b.ptr) cudaFree(b.ptr);
+    b.ptr = nullptr;
+    b.bytes = 0;
+}
+
+size_t elem_size(simjoin_dtype t) { return t == SIMJOIN_I8 ? 1 : 2; }
+
+// 1 = device memory of `device`, 0 = host / unregistered / other device.
+int is_device_ptr(const void *p, int device) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    if (a.type == cudaMemoryTypeDevice || a.type == cudaMemoryTypeManaged) return a.device == device;
+    return 0;
+}
+
+simjoin_status check_matrix_args(const simjoin_ctx *ctx, const void *X, int64_t rows, int32_t d) {
+    if (!X || rows < 0 || rows >= SIMJOIN_MAX_ROWS || d <= 0) return SIMJOIN_ERR_ARG;
+    const size_t row_bytes = (size_t)d * elem_size(ctx->dtype);
+    if (row_bytes % 16 != 0 || row_bytes > SIMJOIN_MAX_ROW_BYTES) return SIMJOIN_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(X) & 15u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
+    return SIMJOIN_OK;
+}
+
+simjoin_status check_join_args(const simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
+                               simjoin_kind kind, double threshold, const int32_t *out_pairs, uint64_t capacity,
+                               const uint64_t *count) {
+    if (!ctx || !count) return SIMJOIN_ERR_ARG;
+    if (kind != SIMJOIN_IP && kind != SIMJOIN_COS && kind != SIMJOIN_L2) return SIMJOIN_ERR_ARG;
+    if (std::isnan(threshold) || (kind == SIMJOIN_L2 && threshold < 0)) return SIMJOIN_ERR_ARG;
+    if (!out_pairs && capacity > 0) return SIMJOIN_ERR_ARG;
+    simjoin_status st = check_matrix_args(ctx, P, n, d);
+    if (st == SIMJOIN_OK || st == SIMJOIN_ERR_UNSUPPORTED) {
+        const simjoin_status sq = check_matrix_args(ctx, Q, m, d);
+        if (sq == SIMJOIN_ERR_ARG || st == SIMJOIN_OK) st = sq;
+    }
+    if (st != SIMJOIN_OK) return st;
+    if (n + ctx->ioff >= SIMJOIN_MAX_ROWS || m + ctx->joff >= SIMJOIN_MAX_ROWS) return SIMJOIN_ERR_ARG;
+    if (ctx->dtype == SIMJOIN_I8 && kind == SIMJOIN_COS) return SIMJOIN_ERR_UNSUPPORTED;
+    return SIMJOIN_OK;
+}
+
+bool encode_rows_map(const simjoin_ctx *ctx, CUtensorMap *map, const void *X, int64_t rows, int32_t d, int box_rows) {
+    const size_t es = elem_size(ctx->dtype);
+    const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)d * es};
+    const cuuint32_t box[2] = {(cuuint32_t)(CHUNK_BYTES / es), (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapDataType dt = ctx->dtype == SIMJOIN_I8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUresult r = ctx->encode(map, dt, 2, const_cast<void *>(X), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+template <bool kInt8>
+cudaError_t launch_norms(const simjoin_ctx *ctx, const void *X, int64_t rows, int32_t d, int sqrt_out, void *norms,
+                         void *minmax) {
+    using T = typename NormAcc<kInt8>::type;
+    if (rows == 0) return cudaSuccess;
+    const int g = (int)((size_t)d * elem_size(ctx->dtype) / 16);
+    const unsigned blocks = (unsigned)((rows + NORM_TILE_ROWS - 1) / NORM_TILE_ROWS);
+    row_norms_kernel<kInt8><<<blocks, NORM_THREADS, 0, ctx->stream>>>(reinterpret_cast<const uint4 *>(X), rows, g, sqrt_out,
+                                                                     reinterpret_cast<T *>(norms), reinterpret_cast<T *>(minmax));
+    return cudaGetLastError();
+}
+
+template <int DT, int KIND>
+cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
+                        size_t smem) {
+    auto kern = join_kernel<DT, KIND>;
+    if (!ctx->attr_set[DT][KIND]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
+        if (e != cudaSuccess) return e;
+        ctx->attr_set[DT][KIND] = true;
+    }
+    kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
+    return cudaGetLastError();
+}
+
+int clamp_to_i32(double v) {
+    if (v >= 2147483647.0) return 2147483647;
+    if (v <= -2147483648.0) return (-2147483647 - 1);
+    return (int)v;
+}
+
+// The join on device buffers.  Arguments were validated by the caller.
+simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
+                          simjoin_kind kind, double threshold, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+    *count = 0;
+    ctx->have_timing = false;
+    if (n == 0 || m == 0) return SIMJOIN_OK;
+    const bool i8 = ctx->dtype == SIMJOIN_I8;
+    const size_t es = elem_size(ctx->dtype);
+    const int row_bytes = (int)(d * es);
+
+    JoinParams jp;
+    std::memset(&jp, 0, sizeof jp);
+    jp.n = n;
+    jp.m = m;
+    jp.kc = (row_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES;
+    const int last_bytes = row_bytes - (jp.kc - 1) * CHUNK_BYTES;
+    jp.last_ksteps = (last_bytes + 31) / 32;
+    jp.elems_per_chunk = (int)(CHUNK_BYTES / es);
+    jp.stationary = jp.kc <= MAX_STATIONARY_CHUNKS ? 1 : 0;
+    const int p_bytes = jp.stationary ? 2 * jp.kc * A_CHUNK_BYTES : 0;
+    const int stage_bytes = B_CHUNK_BYTES + (jp.stationary ? 0 : A_CHUNK_BYTES);
+    int nstages = (ctx->max_smem_optin - 1024 - CTRL_BYTES - p_bytes) / stage_bytes;
+    if (nstages > MAX_STAGES) nstages = MAX_STAGES;
+    if (nstages < 2) return SIMJOIN_ERR_UNSUPPORTED;
+    jp.nstages = nstages;
+    const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + CTRL_BYTES;
+    jp.PB = (int)((n + TILE_M - 1) / TILE_M);
+    jp.QT = (int)((m + TILE_N - 1) / TILE_N);
+    jp.out = reinterpret_cast<int2 *>(out_pairs);
+    jp.capacity = capacity;
+    jp.counter = ctx->d_ctrl;
+    jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
+    jp.ioff = (int)ctx->ioff;
+    jp.joff = (int)ctx->joff;
+
+    // thresholds in the precision each path decides in
+    if (i8) {
+        if (kind == SIMJOIN_IP) jp.thr_i = clamp_to_i32(std::ceil(threshold));
+        else {
+            const double r2 = std::floor(threshold * threshold);
+            jp.thr_i = r2 >= 1073741824.0 ? 1073741824 : (int)r2;   // 2^30 exceeds every int8 squared distance here
+        }
+    } else {
+        jp.thr_f = kind == SIMJOIN_L2 ? (float)(threshold * threshold) : (float)threshold;
+    }
+
+    const bool need_norms = kind != SIMJOIN_IP;
+    if (need_norms) {
+        if (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, (size_t)m * 4) || !grow(ctx->qstat, (size_t)jp.QT * 8))
+            return SIMJOIN_ERR_CUDA;
+        jp.nx = ctx->nx.ptr;
+        jp.ny = ctx->ny.ptr;
+        jp.qstat = ctx->qstat.ptr;
+    }
+
+    CUtensorMap mapP, mapQ;
+    if (!encode_rows_map(ctx, &mapP, P, n, d, TILE_M) || !encode_rows_map(ctx, &mapQ, Q, m, d, TILE_N))
+        return SIMJOIN_ERR_CUDA;
+
+    cudaStream_t s = ctx->stream;
+    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    cudaEventRecord(ctx->ev[0], s);
+    if (need_norms) {
+        const int sq = kind == SIMJOIN_COS ? 1 : 0;
+        cudaError_t e1, e2;
+        if (i8) {
+            e1 = launch_norms<true>(ctx, P, n, d, 0, ctx->nx.ptr, nullptr);
+            e2 = launch_norms<true>(ctx, Q, m, d, 0, ctx->ny.ptr, ctx->qstat.ptr);
+        } else {
+            e1 = launch_norms<false>(ctx, P, n, d, sq, ctx->nx.ptr, nullptr);
+            e2 = launch_norms<false>(ctx, Q, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
+        }
+        if (e1 != cudaSuccess || e2 != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    }
+    cudaEventRecord(ctx->ev[1], s);
+    const int grid = ctx->num_sms;
+    cudaError_t e = cudaErrorInvalidValue;
+    if (i8 && kind == SIMJOIN_IP) e = launch_join<DT_I8, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
+    else if (i8 && kind == SIMJOIN_L2) e = launch_join<DT_I8, KIND_L2>(ctx, mapP, mapQ, jp, grid, smem);
+    else if (!i8 && kind == SIMJOIN_IP) e = launch_join<DT_BF16, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
+    else if (!i8 && kind == SIMJOIN_COS) e = launch_join<DT_BF16, KIND_COS>(ctx, mapP, mapQ, jp, grid, smem);
+    else if (!i8 && kind == SIMJOIN_L2) e = launch_join<DT_BF16, KIND_L2>(ctx, mapP, mapQ, jp, grid, smem);
+    if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    cudaEventRecord(ctx->ev[2], s);
+    if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    const unsigned int kstatus = (unsigned int)(ctx->h_ctrl[1] & 0xffffffffu);
+    if (kstatus != 0) return SIMJOIN_ERR_TIMEOUT;
+    *count = ctx->h_ctrl[0];
+    float a = 0.f, b = 0.f;
+    if (cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess &&
+        cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
+        ctx->prepass_ms = need_norms ? a : 0.f;
+        ctx->join_ms = b;
+        ctx->have_timing = true;
+    }
+    return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+simjoin_status simjoin_create(simjoin_ctx **out, simjoin_dtype dtype, int device, void *cuda_stream) {
+    if (!out) return SIMJOIN_ERR_ARG;
+    *out = nullptr;
+    if (dtype != SIMJOIN_I8 && dtype != SIMJOIN_BF16) return SIMJOIN_ERR_ARG;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    if (device < 0 || device >= ndev) return SIMJOIN_ERR_ARG;
+    int major = 0, sms = 0, smem = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
+        return SIMJOIN_ERR_CUDA;
+    if (major != 10) return SIMJOIN_ERR_ARCH;
+    DeviceGuard guard(device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    simjoin_ctx *ctx = new (std::nothrow) simjoin_ctx();
+    if (!ctx) return SIMJOIN_ERR_CUDA;
+    ctx->dtype = dtype;
+    ctx->device = device;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->num_sms = sms;
+    ctx->max_smem_optin = smem;
+    ctx->d_ctrl = nullptr;
+    ctx->h_ctrl = nullptr;
+    ctx->have_timing = false;
+    ctx->ioff = ctx->joff = 0;
+    std::memset(ctx->attr_set, 0, sizeof ctx->attr_set);
+    for (auto &e : ctx->ev) e = nullptr;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    bool ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+              qres == cudaDriverEntryPointSuccess && fn != nullptr;
+    ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    ok = ok && cudaMalloc(reinterpret_cast<void **>(&ctx->d_ctrl), 64) == cudaSuccess;
+    ok = ok && cudaMallocHost(reinterpret_cast<void **>(&ctx->h_ctrl), 64) == cudaSuccess;
+    for (auto &e : ctx->ev) ok = ok && cudaEventCreate(&e) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        simjoin_destroy(ctx);
+        return SIMJOIN_ERR_CUDA;
+    }
+    *out = ctx;
+    return SIMJOIN_OK;
+}
+
+simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
+    if (!ctx) return SIMJOIN_OK;
+    DeviceGuard guard(ctx->device);
+    release(ctx->nx);
+    release(ctx->ny);
+    release(ctx->qstat);
+    release(ctx->pstat);
+    release(ctx->stage_p);
+    release(ctx->stage_q);
+    release(ctx->stage_out);
+    if (ctx->d_ctrl) cudaFree(ctx->d_ctrl);
+    if (ctx->h_ctrl) cudaFreeHost(ctx->h_ctrl);
+    for (auto &e : ctx->ev)
+        if (e) cudaEventDestroy(e);
+    delete ctx;
+    return SIMJOIN_OK;
+}
+
+simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64_t row_offset_q) {
+    if (!ctx || row_offset_p < 0 || row_offset_q < 0 || row_offset_p >= SIMJOIN_MAX_ROWS || row_offset_q >= SIMJOIN_MAX_ROWS)
+        return SIMJOIN_ERR_ARG;
+    ctx->ioff = row_offset_p;
+    ctx->joff = row_offset_q;
+    return SIMJOIN_OK;
+}
+
+simjoin_status simjoin_run(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
+                           simjoin_kind kind, double threshold, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+    simjoin_status st = check_join_args(ctx, P, n, Q, m, d, kind, threshold, out_pairs, capacity, count);
+    if (st != SIMJOIN_OK) return st;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    if ((n > 0 && !is_device_ptr(P, ctx->device)) || (m > 0 && !is_device_ptr(Q, ctx->device))) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && !is_device_ptr(out_pairs, ctx->device)) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
+    return run_device(ctx, P, n, Q, m, d, kind, threshold, out_pairs, capacity, count);
+}
+
+simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n, const void *Q_host, int64_t m, int32_t d,
+                                simjoin_kind kind, double threshold, int32_t *out_pairs_host, uint64_t capacity,
+                                uint64_t *count) {
+    simjoin_status st = check_join_args(ctx, P_host, n, Q_host, m, d, kind, threshold, out_pairs_host, capacity, count);
+    if (st != SIMJOIN_OK) return st;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    if (is_device_ptr(P_host, ctx->device) || is_device_ptr(Q_host, ctx->device)) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && is_device_ptr(out_pairs_host, ctx->device)) return SIMJOIN_ERR_ARG;
+    *count = 0;
+    if (n == 0 || m == 0) return SIMJOIN_OK;
+    const size_t es = elem_size(ctx->dtype);
+    const size_t pb = (size_t)n * d * es, qb = (size_t)m * d * es, ob = (size_t)capacity * 8;
+    if (!grow(ctx->stage_p, pb) || !grow(ctx->stage_q, qb) || !grow(ctx->stage_out, ob ? ob : 8)) return SIMJOIN_ERR_CUDA;
+    cudaStream_t s = ctx->stream;
+    if (cudaMemcpyAsync(ctx->stage_p.ptr, P_host, pb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->stage_q.ptr, Q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return SIMJOIN_ERR_CUDA;
+    st = run_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, kind, threshold,
+                    capacity ? reinterpret_cast<int32_t *>(ctx->stage_out.ptr) : nullptr, capacity, count);
+    if (st != SIMJOIN_OK && st != SIMJOIN_ERR_CAPACITY) return st;
+    const uint64_t wrote = *count < capacity ? *count : capacity;
+    if (wrote > 0) {
+        if (cudaMemcpyAsync(out_pairs_host, ctx->stage_out.ptr, (size_t)wrote * 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) {
+            cudaGetLastError();
+            return SIMJOIN_ERR_CUDA;
+        }
+    }
+    return st;
+}
+
+simjoin_status simjoin_row_norms(simjoin_ctx *ctx, const void *X, int64_t rows, int32_t d, void *out) {
+    if (!ctx || !out) return SIMJOIN_ERR_ARG;
+    simjoin_status st = check_matrix_args(ctx, X, rows, d);
+    if (st != SIMJOIN_OK) return st;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    if (rows == 0) return SIMJOIN_OK;
+    if (!is_device_ptr(X, ctx->device) || !is_device_ptr(out, ctx->device)) return SIMJOIN_ERR_ARG;
+    const cudaError_t e = ctx->dtype == SIMJOIN_I8 ? launch_norms<true>(ctx, X, rows, d, 0, out, nullptr)
+                                                   : launch_norms<false>(ctx, X, rows, d, 0, out, nullptr);
+    if (e != cudaSuccess || cudaStreamSynchronize(ctx->stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    return SIMJOIN_OK;
+}
+
+simjoin_status simjoin_last_kernel_ms(simjoin_ctx *ctx, float *prepass_ms, float *join_ms) {
+    if (!ctx || !ctx->have_timing) return SIMJOIN_ERR_ARG;
+    if (prepass_ms) *prepass_ms = ctx->prepass_ms;
+    if (join_ms) *join_ms = ctx->join_ms;
+    return SIMJOIN_OK;
+}
+
+const char *simjoin_strerror(simjoin_status status) {
+    switch (status) {
+        case SIMJOIN_OK: return "ok";
+        case SIMJOIN_ERR_ARG: return "invalid argument";
+        case SIMJOIN_ERR_UNSUPPORTED: return "unsupported shape, alignment or dtype/kind combination";
+        case SIMJOIN_ERR_CAPACITY: return "more passing pairs than the output capacity";
+        case SIMJOIN_ERR_CUDA: return "a CUDA call failed";
+        case SIMJOIN_ERR_TIMEOUT: return "a bounded wait inside the join kernel expired";
+        case SIMJOIN_ERR_ARCH: return "device is not compute capability 10.x";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

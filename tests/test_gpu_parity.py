@@ -1,0 +1,291 @@
+"""Parity of the CUDA join (through the C ABI) with the CPU oracle, element by element.
+
+int8 joins must equal the oracle's sorted pair set bit for bit.  bf16 joins must lie
+between the oracle's strict and loose band sets (scores within 1e-2*|t| of the
+threshold may fall on either side); in-band disagreements are reported."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import simjoin_oracle as O
+from paper_2006_12608_b200 import binding as B
+from paper_2006_12608_b200 import build
+from paper_2006_12608_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+BAND_REL = 1e-2      # the band half-width relative to |threshold| (spec tolerance)
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    B.load()
+
+
+@pytest.fixture(scope="module")
+def ctx_i8():
+    c = B.Simjoin("i8", 0)
+    yield c
+    c.close()
+
+
+@pytest.fixture(scope="module")
+def ctx_bf16():
+    c = B.Simjoin("bf16", 0)
+    yield c
+    c.close()
+
+
+def gpu_join(ctx, P, Q, kind, t, capacity=None):
+    dP, dQ = B.to_device(P), B.to_device(Q)
+    cap = 1 << 16 if capacity is None else capacity
+    while True:
+        out = torch.full((max(cap, 1) + 4, 2), -7, dtype=torch.int32, device="cuda:0")   # 4 canary rows
+        st, cnt = ctx.simjoin_run(dP, P.shape[0], dQ, Q.shape[0], P.shape[1], kind, t, out if cap else None, cap)
+        assert st in (B.SIMJOIN_OK, B.SIMJOIN_ERR_CAPACITY), B.strerror(st)
+        assert (st == B.SIMJOIN_ERR_CAPACITY) == (cnt > cap)
+        host = out.cpu().numpy()
+        assert np.all(host[cap:] == -7), "wrote past capacity"
+        wrote = min(cnt, cap)
+        assert np.all(host[wrote:cap] == -7), "wrote more rows than min(count, capacity)"
+        if capacity is not None or cnt <= cap:
+            return host[:wrote], cnt
+        cap = cnt
+
+
+def keys(pairs):
+    p = np.asarray(pairs, dtype=np.int64).reshape(-1, 2)
+    return (p[:, 0] << 32) | p[:, 1]
+
+
+def assert_exact(gpu_pairs, cnt, P, Q, kind, t, dtype="i8"):
+    want, wcnt = O.join(P, Q, kind, t, dtype)
+    assert cnt == wcnt
+    g = np.sort(keys(gpu_pairs))
+    assert len(np.unique(g)) == len(g), "duplicate pairs"
+    assert np.array_equal(g, keys(want))            # oracle output is already sorted by (i, j)
+
+
+def assert_band(gpu_pairs, cnt, P, Q, kind, t):
+    s_strict, s_exact, s_loose = O.band_sets(P, Q, kind, t, "bf16", rel=BAND_REL)
+    g = np.sort(keys(gpu_pairs))
+    assert len(g) == cnt and len(np.unique(g)) == len(g), "duplicate pairs"
+    assert np.isin(keys(s_strict), g).all(), "missing a pair that is clearly inside the threshold"
+    assert np.isin(g, keys(s_loose)).all(), "emitted a pair that is clearly outside the threshold"
+    disagreements = len(np.setxor1d(g, keys(s_exact)))
+    in_band = len(s_loose) - len(s_strict)
+    print(f"[band] kind={kind} t={t}: |GPU|={len(g)} |exact|={len(s_exact)} in-band={in_band} disagreements={disagreements}")
+    return disagreements, in_band
+
+
+# ------------------------------------------------------------------ configuration 1, full size
+def test_cfg1_full_bit_exact(ctx_i8):
+    w = W.make_workload(1)
+    pairs, cnt = gpu_join(ctx_i8, w.P, w.Q, "ip", w.threshold)
+    assert_exact(pairs, cnt, w.P, w.Q, "ip", w.threshold)
+    assert np.isin(keys(w.planted), keys(pairs)).all()
+
+
+# ------------------------------------------------------------------ shapes: ragged tails, K chunks
+I8_SHAPES = [(1, 1, 16), (5, 3, 16), (128, 256, 128), (129, 257, 128), (300, 700, 64), (1000, 513, 144),
+             (257, 1030, 256), (77, 300, 384), (200, 260, 512), (130, 520, 640), (140, 300, 1024), (64, 64, 8192)]
+
+
+@pytest.mark.parametrize("n,m,d", I8_SHAPES)
+def test_i8_ip_shapes(ctx_i8, n, m, d):
+    P, Q = W.random_points("i8", n, d, 1), W.random_points("i8", m, d, 2)
+    sd = (d * (28.0 / 7.0) ** 2) ** 0.5        # std of <x,y> for iid uniform{-3..3}: var(x)=4
+    for t in (2.0 * sd, 0.5 * sd + 0.5):
+        pairs, cnt = gpu_join(ctx_i8, P, Q, "ip", t)
+        assert_exact(pairs, cnt, P, Q, "ip", t)
+
+
+@pytest.mark.parametrize("n,m,d", [(5, 3, 16), (129, 257, 128), (300, 700, 64), (257, 1030, 256), (140, 300, 1024)])
+def test_i8_l2_shapes(ctx_i8, n, m, d):
+    P, Q = W.random_points("i8", n, d, 3), W.random_points("i8", m, d, 4)
+    mean = (8.0 * d) ** 0.5                     # E|x-y|^2 = 2*var*d = 8d
+    for r in (0.93 * mean, 0.8 * mean, float(int(mean))):
+        pairs, cnt = gpu_join(ctx_i8, P, Q, "l2", r)
+        assert_exact(pairs, cnt, P, Q, "l2", r)
+
+
+BF_SHAPES = [(1, 1, 8), (5, 3, 8), (128, 256, 64), (129, 257, 64), (300, 700, 128), (513, 1000, 72),
+             (257, 1030, 256), (140, 300, 512), (64, 64, 4096)]
+
+
+@pytest.mark.parametrize("kind", ["ip", "cos", "l2"])
+@pytest.mark.parametrize("n,m,d", BF_SHAPES)
+def test_bf16_shapes(ctx_bf16, kind, n, m, d):
+    P, Q = W.random_points("bf16", n, d, 5), W.random_points("bf16", m, d, 6)
+    t = {"ip": 1.5 * d ** 0.5, "cos": 1.5 / d ** 0.5, "l2": (2 * d) ** 0.5 - 1.2}[kind]
+    pairs, cnt = gpu_join(ctx_bf16, P, Q, kind, t)
+    assert_band(pairs, cnt, P, Q, kind, t)
+
+
+def test_bf16_negative_threshold_and_zero_rows(ctx_bf16):
+    P, Q = W.random_points("bf16", 200, 32, 7), W.random_points("bf16", 300, 32, 8)
+    P[17] = 0
+    Q[5] = 0
+    Q[299] = 0
+    for t in (-0.2, 0.0, 0.25):
+        pairs, cnt = gpu_join(ctx_bf16, P, Q, "cos", t)
+        assert_band(pairs, cnt, P, Q, "cos", t) if t != 0.0 else None
+        want, _c = O.join(P, Q, "cos", t, "bf16")
+        zero_rows = {(i, j) for (i, j) in map(tuple, want.tolist()) if i == 17 or j in (5, 299)}
+        got = set(map(tuple, pairs.tolist()))
+        assert {(i, j) for (i, j) in got if i == 17 or j in (5, 299)} == zero_rows   # cosine with 0 counts as 0
+    pairs, cnt = gpu_join(ctx_bf16, P, Q, "ip", -1.0)
+    assert_band(pairs, cnt, P, Q, "ip", -1.0)
+
+
+# ------------------------------------------------------------------ degenerate thresholds and sizes
+def test_everything_and_nothing(ctx_i8, ctx_bf16):
+    P, Q = W.random_points("i8", 200, 64, 9), W.random_points("i8", 300, 64, 10)
+    pairs, cnt = gpu_join(ctx_i8, P, Q, "ip", -1e30)
+    assert cnt == 200 * 300 and np.array_equal(np.sort(keys(pairs)), keys([[i, j] for i in range(200) for j in range(300)]))
+    assert gpu_join(ctx_i8, P, Q, "ip", 1e30)[1] == 0
+    assert gpu_join(ctx_i8, P, Q, "ip", float("inf"))[1] == 0
+    assert gpu_join(ctx_i8, P, Q, "ip", float("-inf"))[1] == 200 * 300
+    assert gpu_join(ctx_i8, P, Q, "l2", 1e9)[1] == 200 * 300
+    pairs, cnt = gpu_join(ctx_i8, P, P, "l2", 0.0)                     # only identical rows
+    assert_exact(pairs, cnt, P, P, "l2", 0.0)
+    assert cnt >= 200
+    Pb, Qb = W.random_points("bf16", 150, 64, 11), W.random_points("bf16", 260, 64, 12)
+    assert gpu_join(ctx_bf16, Pb, Qb, "l2", 1e18)[1] == 150 * 260
+    assert gpu_join(ctx_bf16, Pb, Qb, "cos", -1.5)[1] == 150 * 260
+    assert gpu_join(ctx_bf16, Pb, Qb, "cos", 1.5)[1] == 0
+    assert gpu_join(ctx_bf16, Pb, Qb, "ip", float("inf"))[1] == 0
+
+
+def test_self_join_is_symmetric_with_diagonal(ctx_i8):
+    w = W.make_workload(3, n=700, m=700, planted=0)
+    pairs, cnt = gpu_join(ctx_i8, w.P, w.P, "ip", 3000.0)
+    S = set(map(tuple, pairs.tolist()))
+    assert {(j, i) for (i, j) in S} == S and all((i, i) in S for i in range(700))
+    assert_exact(pairs, cnt, w.P, w.P, "ip", 3000.0)
+
+
+def test_empty_inputs_count_only_and_capacity(ctx_i8):
+    P, Q = W.random_points("i8", 300, 64, 13), W.random_points("i8", 500, 64, 14)
+    dP, dQ = B.to_device(P), B.to_device(Q)
+    out = torch.zeros((8, 2), dtype=torch.int32, device="cuda:0")
+    assert ctx_i8.simjoin_run(dP, 0, dQ, 500, 64, "ip", 0.0, out, 8) == (B.SIMJOIN_OK, 0)
+    assert ctx_i8.simjoin_run(dP, 300, dQ, 0, 64, "ip", 0.0, out, 8) == (B.SIMJOIN_OK, 0)
+    want, wcnt = O.join(P, Q, "ip", 20.0, "i8")
+    assert wcnt > 100
+    st, cnt = ctx_i8.simjoin_run(dP, 300, dQ, 500, 64, "ip", 20.0, None, 0)       # count-only mode
+    assert (st, cnt) == (B.SIMJOIN_ERR_CAPACITY, wcnt)
+    part, cnt = gpu_join(ctx_i8, P, Q, "ip", 20.0, capacity=37)                   # overflow: valid subset
+    assert cnt == wcnt and len(part) == 37
+    k = keys(part)
+    assert len(np.unique(k)) == 37 and np.isin(k, keys(want)).all()
+
+
+def test_offsets_shift_emitted_indices(ctx_i8):
+    P, Q = W.random_points("i8", 260, 64, 15), W.random_points("i8", 300, 64, 16)
+    base, cnt = gpu_join(ctx_i8, P, Q, "ip", 18.0)
+    assert ctx_i8.simjoin_set_offsets(1000, 70000) == B.SIMJOIN_OK
+    try:
+        shifted, cnt2 = gpu_join(ctx_i8, P, Q, "ip", 18.0)
+    finally:
+        assert ctx_i8.simjoin_set_offsets(0, 0) == B.SIMJOIN_OK
+    assert cnt2 == cnt and np.array_equal(np.sort(keys(shifted - np.array([1000, 70000]))), np.sort(keys(base)))
+    assert ctx_i8.simjoin_set_offsets(-1, 0) == B.SIMJOIN_ERR_ARG
+
+
+def test_bad_arguments_are_rejected_before_launch(ctx_i8, ctx_bf16):
+    P = B.to_device(W.random_points("i8", 64, 64, 17))
+    out = torch.zeros((8, 2), dtype=torch.int32, device="cuda:0")
+    E = B.SIMJOIN_ERR_ARG
+    assert ctx_i8.simjoin_run(None, 64, P, 64, 64, "ip", 0.0, out, 8)[0] == E
+    assert ctx_i8.simjoin_run(P, -1, P, 64, 64, "ip", 0.0, out, 8)[0] == E
+    assert ctx_i8.simjoin_run(P, 64, P, 64, 0, "ip", 0.0, out, 8)[0] == E
+    assert ctx_i8.simjoin_run(P, 64, P, 64, 64, "ip", float("nan"), out, 8)[0] == E
+    assert ctx_i8.simjoin_run(P, 64, P, 64, 64, "l2", -1.0, out, 8)[0] == E
+    assert ctx_i8.simjoin_run(P, 64, P, 64, 64, "ip", 0.0, None, 8)[0] == E
+    assert ctx_i8.simjoin_run(P.cpu().numpy(), 64, P, 64, 64, "ip", 0.0, out, 8)[0] == E     # host pointer
+    assert ctx_i8.simjoin_run(P, 64, P, 64, 64, "ip", 0.0, out.cpu().numpy(), 8)[0] == E
+    U = B.SIMJOIN_ERR_UNSUPPORTED
+    assert ctx_i8.simjoin_run(P, 64, P, 64, 24, "ip", 0.0, out, 8)[0] == U                   # 24 B rows
+    assert ctx_i8.simjoin_run(P.data_ptr() + 1, 32, P, 64, 64, "ip", 0.0, out, 8)[0] == U    # misaligned
+    assert ctx_i8.simjoin_run(P, 64, P, 64, 64, "cos", 0.5, out, 8)[0] == U
+    assert ctx_i8.simjoin_run(P, 1, P, 1, 16384, "ip", 0.0, out, 8)[0] == U                  # row too long
+    assert ctx_i8.simjoin_last_kernel_ms()[0] in (B.SIMJOIN_OK, B.SIMJOIN_ERR_ARG)
+    # the context is still usable afterwards
+    assert ctx_i8.simjoin_run(P, 64, P, 64, 64, "ip", 1e9, out, 8) == (B.SIMJOIN_OK, 0)
+
+
+def test_run_host_matches_device_path(ctx_i8):
+    w = W.make_workload(4, n=3000, m=2500, planted=120)
+    want, wcnt = O.join(w.P, w.Q, "ip", w.threshold, "i8")
+    out = np.full((wcnt + 10, 2), -7, dtype=np.int32)
+    st, cnt = ctx_i8.simjoin_run_host(w.P, w.n, w.Q, w.m, w.d, "ip", w.threshold, out, wcnt + 10)
+    assert (st, cnt) == (B.SIMJOIN_OK, wcnt)
+    assert np.array_equal(np.sort(keys(out[:cnt])), keys(want)) and np.all(out[cnt:] == -7)
+    dP = B.to_device(w.P)
+    assert ctx_i8.simjoin_run_host(dP, w.n, w.Q, w.m, w.d, "ip", w.threshold, out, 10)[0] == B.SIMJOIN_ERR_ARG
+
+
+def test_row_norms_prepass(ctx_i8, ctx_bf16):
+    for rows, d in [(1, 16), (300, 64), (1000, 144), (513, 1024)]:
+        X = W.random_points("i8", rows, d, 18, lo=-128, hi=127)
+        out = torch.zeros(rows, dtype=torch.int32, device="cuda:0")
+        assert ctx_i8.simjoin_row_norms(B.to_device(X), rows, d, out) == B.SIMJOIN_OK
+        assert np.array_equal(out.cpu().numpy().astype(np.int64), O.sq_norms(X, "i8"))       # exact
+    for rows, d in [(1, 8), (300, 64), (1000, 72), (513, 512)]:
+        X = W.random_points("bf16", rows, d, 19, scale=3.0)
+        out = torch.zeros(rows, dtype=torch.float32, device="cuda:0")
+        assert ctx_bf16.simjoin_row_norms(B.to_device(X), rows, d, out) == B.SIMJOIN_OK
+        np.testing.assert_allclose(out.cpu().numpy().astype(np.float64), O.sq_norms(X, "bf16"), rtol=2e-6)
+
+
+# ------------------------------------------------------------------ scheduling: several waves + a split tail
+def test_multiple_waves_and_split_tail(ctx_i8):
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n = 128 * (sms + 21) + 5           # one full wave, then a 22-block tail split over the CTAs
+    w = W.make_workload(4, n=n, m=2048 + 77, planted=500)
+    pairs, cnt = gpu_join(ctx_i8, w.P, w.Q, "ip", w.threshold)
+    assert_exact(pairs, cnt, w.P, w.Q, "ip", w.threshold)
+    assert np.isin(keys(w.planted), keys(pairs)).all()
+
+
+# ------------------------------------------------------------------ the five configurations, reduced
+def test_cfg2_reduced(ctx_bf16):
+    w = W.make_workload(2, n=6000, m=5000, planted=200)
+    pairs, cnt = gpu_join(ctx_bf16, w.P, w.Q, "cos", w.threshold)
+    dis, _band = assert_band(pairs, cnt, w.P, w.Q, "cos", w.threshold)
+    assert np.isin(keys(w.planted), keys(pairs)).all() and dis == 0
+
+
+def test_cfg3_reduced(ctx_i8):
+    w = W.make_workload(3, n=5000, m=4100, planted=300)
+    pairs, cnt = gpu_join(ctx_i8, w.P, w.Q, "ip", w.threshold)
+    assert_exact(pairs, cnt, w.P, w.Q, "ip", w.threshold)
+    assert np.isin(keys(w.planted), keys(pairs)).all()
+
+
+def test_cfg4_reduced(ctx_i8):
+    w = W.make_workload(4, n=9000, m=7000, planted=900)
+    pairs, cnt = gpu_join(ctx_i8, w.P, w.Q, "ip", w.threshold)
+    assert_exact(pairs, cnt, w.P, w.Q, "ip", w.threshold)
+    assert np.isin(keys(w.planted), keys(pairs)).all()
+
+
+@pytest.mark.parametrize("reading", ["radial", "percoord"])
+def test_cfg5_reduced(ctx_bf16, reading):
+    w = W.make_workload(5, n=6000, m=5000, centers=50, sigma_reading=reading)
+    pairs, cnt = gpu_join(ctx_bf16, w.P, w.Q, "l2", w.threshold, capacity=1 << 20)
+    assert_band(pairs, cnt, w.P, w.Q, "l2", w.threshold)
+    if reading == "radial":     # dense: exactly the same-cluster relation
+        assert cnt == int(sum(np.sum(w.labels_p == c) * np.sum(w.labels_q == c) for c in range(50)))
+        assert np.all(w.labels_p[pairs[:, 0]] == w.labels_q[pairs[:, 1]])
+    else:
+        assert cnt == 0
+
+
+def test_repeated_runs_give_the_same_set(ctx_bf16):
+    w = W.make_workload(5, n=3000, m=3000, centers=30)
+    a, ca = gpu_join(ctx_bf16, w.P, w.Q, "l2", w.threshold, capacity=1 << 19)
+    b, cb = gpu_join(ctx_bf16, w.P, w.Q, "l2", w.threshold, capacity=1 << 19)
+    assert ca == cb and np.array_equal(np.sort(keys(a)), np.sort(keys(b)))
