@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the similarity-join hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+One "step" is one pass of the whole hot path (norm pre-pass where the kind needs
+it, tile streaming, tile products, fused threshold + compaction, counter read-back)
+over one synthetic workload through ``simjoin_run`` of the C-ABI library.  The
+default workload is the throughput-headline configuration (inner-product join,
+n = m = 1 048 576, d = 128, int8 +-1, t = 100).  Rank 0 prints ONE JSON line.
+
+Metric: pair-TOPS = 2*n*m*d / time.  With N > 1 ranks (torchrun) every rank joins
+its own row block of P against a replicated Q (weak scaling, no data-path
+collective); the value is the ops of all ranks over the slowest rank's time.
+
+``--impl reference`` times the CPU oracle (as it stands) on a bounded row slab of
+the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2006_12608_b200 import workloads as W  # noqa: E402
+
+METRIC = "join pair-TOPS (2*n*m*d/s)"
+UNIT = "TOPS"
+NOMINAL_TOPS = {"i8": 4500.0, "bf16": 2250.0}          # dense, per GPU (context only)
+# DRAM bytes per join-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
+# captures summarised under profiles/, scaled to the full workload by (#P-block waves x |Q|).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p["bf16_tflops_sustained"]), "source": "measured"}
+    except (OSError, KeyError, ValueError):
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        import torch
+        self.gpu_id = str(device_index)
+        try:
+            self.gpu_id = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+        except Exception:
+            pass
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread:
+            self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[2:6]):
+                if v == "Active":
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_slab(w, rows: int):
+    """Time the CPU oracle on the first `rows` rows of P against all of Q. Returns (seconds, count, threads)."""
+    from oracle import simjoin_oracle as O
+    t0 = time.perf_counter()
+    _pairs, cnt = O.join(w.P[:rows], w.Q, w.kind, w.threshold, w.dtype)
+    return time.perf_counter() - t0, cnt, O.max_threads()
+
+
+def slab_rows_for(w, seconds: float) -> int:
+    """Rows of P whose oracle join takes roughly `seconds` (rates measured on 8 cores: ~25 GMAC/s
+    int8, ~3.3 GMAC/s bf16/fp64; scaled by the core count)."""
+    cores = os.cpu_count() or 1
+    rate = (25e9 if w.dtype == "i8" else 3.3e9) * cores / 8.0
+    rows = int(seconds * rate / (w.m * w.d))
+    return max(1, min(w.n, rows))
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import simjoin_oracle as O
+    O.build()
+    rows = slab_rows_for(w, 4.0)
+    times = []
+    for it in range(args.warmup + args.steps):
+        dt, _cnt, threads = oracle_slab(w, rows)
+        if it >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    ops_per_step = 2.0 * rows * w.m * w.d
+    value = ops_per_step * len(times) / total / 1e12
+    sample = f"first {rows} rows of P x all {w.m} rows of Q per step (the oracle's cost is linear in rows)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int64" if w.dtype == "i8" else "f64", "data": "synthetic",
+            "config": {"workload": w.name, "n": w.n, "m": w.m, "d": w.d, "kind": w.kind, "threshold": w.threshold,
+                       "sample_rows": rows},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def size_kw(args):
+    kw = {}
+    if args.n is not None:
+        kw["n"] = args.n
+    if args.m is not None:
+        kw["m"] = args.m
+    if args.planted is not None and args.config != 5:
+        kw["planted"] = args.planted
+    return kw
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=4, help="1..5, the benchmark configuration (default 4: the headline)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--n", type=int, default=None, help="override the row count of P (profiling / experiments)")
+    ap.add_argument("--m", type=int, default=None, help="override the row count of Q")
+    ap.add_argument("--planted", type=int, default=None)
+    ap.add_argument("--sigma-reading", default="radial")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        w = W.make_workload(args.config, sigma_reading=args.sigma_reading, **size_kw(args)) if rank == 0 else None
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2006_12608_b200 import binding as B
+    from paper_2006_12608_b200 import build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the join has no CPU path")
+    if rank == 0 and not os.path.exists(B.LIB_PATH):
+        build.build()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    B.load()
+
+    # Each rank owns one row block of a (world * n)-row P and a full copy of Q.
+    w = W.make_workload(args.config, seed=rank, sigma_reading=args.sigma_reading, **size_kw(args))
+    if world > 1:
+        w.Q = W.make_workload(args.config, seed=0, sigma_reading=args.sigma_reading, **size_kw(args)).Q if rank else w.Q
+        w.planted = w.planted if rank == 0 else np.zeros((0, 2), np.int64)
+    dev = torch.device("cuda", local_rank)
+    dP, dQ = B.to_device(w.P, dev), B.to_device(w.Q, dev)
+    same_cluster = None
+    if w.cfg_id == 5 and args.sigma_reading == "radial":
+        same_cluster = int(sum(int(np.sum(w.labels_p == c)) * int(np.sum(w.labels_q == c)) for c in range(1024)))
+    capacity = int(same_cluster * 1.05) if same_cluster else max(4 * len(w.planted), 1 << 20)
+    out = torch.empty((capacity, 2), dtype=torch.int32, device=dev)
+    ctx = B.Simjoin(w.dtype, local_rank)
+    ctx.simjoin_set_offsets(rank * w.n, 0)
+
+    def step():
+        st, cnt = ctx.simjoin_run(dP, w.n, dQ, w.m, w.d, w.kind, w.threshold, out, capacity)
+        if st != B.SIMJOIN_OK:
+            raise RuntimeError(f"simjoin_run: {B.strerror(st)}")
+        return cnt
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    cnt = 0
+    for _ in range(args.warmup):
+        cnt = step()
+    # result sanity (not timed): every planted pair is in the output, nothing is duplicated
+    got = out[:cnt].cpu().numpy().astype(np.int64)
+    keys = (got[:, 0] << 32) | got[:, 1]
+    assert len(np.unique(keys)) == cnt, "duplicate pairs in the join output"
+    if len(w.planted):
+        pk = ((w.planted[:, 0] + rank * w.n) << 32) | w.planted[:, 1]
+        assert np.isin(pk, keys).all(), "a planted pair is missing from the join output"
+    if same_cluster is not None:
+        assert cnt == same_cluster, (cnt, same_cluster)
+
+    sampler = ClockSampler(local_rank)
+    sync_all()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    join_ms, pre_ms = [], []
+    e0.record()
+    for _ in range(args.steps):
+        step()
+        _st, a, b = ctx.simjoin_last_kernel_ms()
+        pre_ms.append(a)
+        join_ms.append(b)
+    e1.record()
+    sync_all()
+    clocks = sampler.stop()
+    elapsed_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * w.ops / (ms_per_step * 1e-3) / 1e12
+
+    e2e = None
+    if not args.no_e2e:
+        e2e = measure_e2e(args, ctx, w, capacity, cnt, world, dev, sync_all)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+    finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks, e2e)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def measure_e2e(args, ctx, w, capacity, cnt, world, dev, sync_all):
+    """End to end: host buffers in, host pairs out, copies inside the timed region."""
+    import torch
+    import torch.distributed as dist
+    from paper_2006_12608_b200 import binding as B
+    hP = torch.from_numpy(w.P.view(np.int16) if w.P.dtype == np.uint16 else w.P).pin_memory()
+    hQ = torch.from_numpy(w.Q.view(np.int16) if w.Q.dtype == np.uint16 else w.Q).pin_memory()
+    hout = torch.empty((capacity, 2), dtype=torch.int32).pin_memory()
+    e2e_steps = max(1, min(args.steps, 5))
+
+    def e2e_step():
+        st, c = ctx.simjoin_run_host(hP, w.n, hQ, w.m, w.d, w.kind, w.threshold, hout, capacity)
+        if st != B.SIMJOIN_OK:
+            raise RuntimeError(f"simjoin_run_host: {B.strerror(st)}")
+        return c
+
+    e2e_step()
+    sync_all()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        c2 = e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = world * w.ops * e2e_steps / e2e_s / 1e12
+    assert c2 == cnt
+    return {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(w.P.nbytes + w.Q.nbytes),
+            "d2h_bytes_per_step": int(cnt * 8 + 16), "steps": e2e_steps}
+
+
+def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks, e2e):
+    peaks = measured_peaks()
+    jm = statistics.mean(join_ms)
+    achieved = w.ops / (jm * 1e-3) / 1e12
+    ratio = 2.0 if w.dtype == "i8" else 1.0          # nominal dense int8 : bf16 rate
+    peak = peaks["bf16_tflops_sustained"] * ratio
+    roofline = {"bound": "tensor", "kernel": "join_kernel", "achieved": achieved, "peak": peak, "unit": "TOP/s",
+                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.cfg_id),
+                "peak_source": f"{peaks['source']}: cuBLAS bf16 sustained {peaks['bf16_tflops_sustained']} TFLOP/s"
+                               + (" x 2 (nominal int8:bf16 ratio)" if ratio == 2.0 else ""),
+                "frac_of_nominal": achieved / NOMINAL_TOPS[w.dtype], "kernel_ms": jm,
+                "prepass_ms": statistics.mean(pre_ms)}
+    launches_per_step = 1 + (2 if w.kind != "ip" else 0)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int32" if w.dtype == "i8" else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "n": w.n, "m": w.m, "d": w.d, "kind": w.kind, "in_dtype": w.dtype,
+                       "threshold": w.threshold, "pairs_found": int(cnt), "l2": "inputs (P+Q) larger than L2; no flush",
+                       "sharding": f"P row blocks x{world}, Q replicated" if world > 1 else "single GPU",
+                       "note": w.note},
+            "clocks": clocks,
+            "e2e": e2e,
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline}
+    if not args.no_cpu_baseline and world == 1:
+        rows = slab_rows_for(w, 12.0)
+        dt, _c, threads = oracle_slab(w, rows)
+        line["cpu_baseline"] = {"value": 2.0 * rows * w.m * w.d / dt / 1e12, "unit": UNIT, "cores": threads,
+                                "kind": "oracle",
+                                "sample": f"first {rows} rows of P x all {w.m} rows of Q, {dt:.1f} s "
+                                          "(the oracle's cost is linear in rows)"}
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()
