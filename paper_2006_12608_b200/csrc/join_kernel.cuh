@@ -9,8 +9,8 @@
 // registers and passing (i, j) are compacted straight into the output list.
 //
 // CTA layout (384 threads, one CTA per SM, persistent):
-//   warp 0      TMA producer: P row block (resident while its Q sweep lasts) + Q chunk ring
-//   warp 1      MMA issuer (lane 0 issues), double-buffered 2 x 256-column accumulators
+//   warp 0      TMA producer (one thread): P row block (resident while its Q sweep lasts) + Q chunk ring
+//   warp 1      MMA issuer (one thread), double-buffered 2 x 256-column accumulators
 //   warp 2      TMEM allocation / release
 //   warp 3      idle
 //   warps 4-11  epilogue: warp w reads TMEM lanes 32*(w%4).., column half (w-4)/4
@@ -44,6 +44,7 @@ struct JoinParams {
     int elems_per_chunk;     // 128 / sizeof(element)
     int stationary;          // 1: the P block stays in shared memory for its whole Q sweep
     int nstages;             // ring depth
+    int epi_release;         // 1: the epilogue hands ring stages back (one commit per tile); needs nstages >= 2*kc
     int PB, QT;              // number of 128-row P blocks, 256-row Q tiles
     int thr_i;               // I8/IP: ceil(t);  I8/L2: floor(r*r); both clamped
     float thr_f;             // BF16: t (IP, COS) or r*r (L2)
@@ -94,7 +95,7 @@ __device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *c
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(addr, parity)) return true;
-        if ((it & 0x3F) == 0) {
+        {
             if (ctrl->abort) return false;
             if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
                 ctrl->abort = 1;
@@ -109,10 +110,41 @@ __device__ __forceinline__ bool wait_bar_warp(uint64_t *bar, uint32_t parity, Ct
     return __all_sync(0xffffffffu, ok);
 }
 
-// Compact the pairs (i, j0 + c), c in `mask`, of the 32 rows this warp owns into the
+// Tree maximum over N accumulator words (3-input max per step keeps the dependency chain
+// at log3(N) instead of N).
+template <int N, bool kInt>
+struct TreeMax {
+    static __device__ __forceinline__ uint32_t run(const uint32_t *a) {
+        constexpr int M = (N + 2) / 3;
+        uint32_t t[M];
+#pragma unroll
+        for (int c = 0; c < M; ++c) {
+            if constexpr (kInt) {
+                if (3 * c + 2 < N) t[c] = (uint32_t)__vimax3_s32((int)a[3 * c], (int)a[3 * c + 1], (int)a[3 * c + 2]);
+                else if (3 * c + 1 < N) t[c] = (uint32_t)max((int)a[3 * c], (int)a[3 * c + 1]);
+                else t[c] = a[3 * c];
+            } else {
+                if (3 * c + 2 < N)
+                    t[c] = __float_as_uint(fmaxf(fmaxf(__uint_as_float(a[3 * c]), __uint_as_float(a[3 * c + 1])), __uint_as_float(a[3 * c + 2])));
+                else if (3 * c + 1 < N) t[c] = __float_as_uint(fmaxf(__uint_as_float(a[3 * c]), __uint_as_float(a[3 * c + 1])));
+                else t[c] = a[3 * c];
+            }
+        }
+        return TreeMax<M, kInt>::run(t);
+    }
+};
+template <bool kInt>
+struct TreeMax<1, kInt> {
+    static __device__ __forceinline__ uint32_t run(const uint32_t *a) { return a[0]; }
+};
+
+// Compact the pairs (i, j0 + 32*q + c), c in mask[q], of the 32 rows this warp owns into the
 // output list: popcount prefix over the warp, one atomic per warp, 8-byte stores.
-__device__ __forceinline__ void emit_pairs(const JoinParams &p, uint32_t mask, int lane, long long i, long long j0) {
-    const int cnt = __popc(mask);
+template <int NQ>
+__device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (&mask)[NQ], int lane, long long i, long long j0) {
+    int cnt = 0;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) cnt += __popc(mask[q]);
     int incl = cnt;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -125,11 +157,15 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, uint32_t mask, i
     if (lane == 0) base = atomicAdd(p.counter, (unsigned long long)total);
     base = __shfl_sync(0xffffffffu, base, 0);
     unsigned long long slot = base + (unsigned long long)(incl - cnt);
-    while (mask) {
-        const int c = __ffs(mask) - 1;
-        mask &= mask - 1;
-        if (slot < p.capacity) p.out[slot] = make_int2((int)(i + p.ioff), (int)(j0 + c + p.joff));
-        ++slot;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        uint32_t mk = mask[q];
+        while (mk) {
+            const int c = __ffs(mk) - 1;
+            mk &= mk - 1;
+            if (slot < p.capacity) p.out[slot] = make_int2((int)(i + p.ioff), (int)(j0 + 32 * q + c + p.joff));
+            ++slot;
+        }
     }
 }
 
@@ -171,6 +207,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
+        // The whole warp walks the loop converged; one elected lane issues the copies.
         uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0;
         bool ok = true;
         Unit un;
@@ -178,7 +215,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             if (p.stationary) {
                 ok = wait_bar_warp(&ctrl->pempty[pbuf], pphase ^ 1, ctrl, p.status, 1);
                 if (!ok) break;
-                if (lane == 0) {
+                if (elect_one()) {
                     const uint32_t bar = smem_u32(&ctrl->pfull[pbuf]);
                     mbar_arrive_expect_tx(bar, (uint32_t)(p.kc * A_CHUNK_BYTES));
                     for (int c = 0; c < p.kc; ++c)
@@ -193,7 +230,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 for (int c = 0; c < p.kc; ++c) {
                     ok = wait_bar_warp(&ctrl->empty[stage], phase ^ 1, ctrl, p.status, 2);
                     if (!ok) break;
-                    if (lane == 0) {
+                    if (elect_one()) {
                         const uint32_t bar = smem_u32(&ctrl->full[stage]);
                         uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
                         mbar_arrive_expect_tx(bar, (uint32_t)stage_bytes);
@@ -210,8 +247,12 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             // aborting: give copies already in flight time to land before shared memory is released
             for (int t = 0; t < 200; ++t) __nanosleep(1000);
         }
+        __syncwarp();
     } else if (warp == 1) {
         // --------------------------------------------------------------- MMA issuer
+        // One tcgen05.commit per tile: commits are expensive (~70 cycles of tensor-pipe time
+        // each, measured), so when a whole tile's chunks fit in the ring twice over the stages of
+        // a tile are handed back to the producer by the epilogue once it has seen the tile's commit.
         constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, TILE_N);
         uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0, acc = 0, accphase = 0;
         bool ok = true;
@@ -229,7 +270,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
                     if (!ok) break;
                     tc_fence_after();
-                    if (lane == 0) {
+                    if (elect_one()) {
                         uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
                         const uint32_t a_addr = p.stationary ? smem_u32(smem_p + (size_t)(pbuf * p.kc + c) * A_CHUNK_BYTES)
                                                              : smem_u32(sb + B_CHUNK_BYTES);
@@ -239,19 +280,18 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         for (int k = 0; k < ksteps; ++k)
                             umma_ss<DT == DT_I8>(tmem_base + acc * TILE_N, adesc + 2 * k, bdesc + 2 * k, idesc,
                                                  (c | k) != 0 ? 1u : 0u);
-                        umma_commit(smem_u32(&ctrl->empty[stage]));
+                        if (!p.epi_release) umma_commit(smem_u32(&ctrl->empty[stage]));
+                        if (c == p.kc - 1) umma_commit(smem_u32(&ctrl->tfull[acc]));
                     }
                     __syncwarp();
                     if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
-                if (lane == 0) umma_commit(smem_u32(&ctrl->tfull[acc]));
-                __syncwarp();
                 acc ^= 1;
                 if (acc == 0) accphase ^= 1;
             }
             if (ok && p.stationary) {
-                if (lane == 0) umma_commit(smem_u32(&ctrl->pempty[pbuf]));
+                if (elect_one()) umma_commit(smem_u32(&ctrl->pempty[pbuf]));
                 __syncwarp();
                 pbuf ^= 1;
                 if (pbuf == 0) pphase ^= 1;
@@ -271,7 +311,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
         const int half = (warp - EPI_WARP0) >> 2;   // which 128 of the tile's 256 columns
         const int row_in_tile = quarter * 32 + lane;
-        uint32_t acc = 0, accphase = 0;
+        uint32_t acc = 0, accphase = 0, rstage = 0;   // rstage: next ring stage to hand back
         bool ok = true;
         Unit un;
         for (int u = 0; ok && get_unit(p, u, un); ++u) {
@@ -308,56 +348,62 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
                 if (!ok) break;
                 tc_fence_after();
-#pragma unroll 1
-                for (int cc = 0; cc < 4; ++cc) {
-                    const int col = half * 128 + cc * 32;
-                    uint32_t v[32];
-                    tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + col, v);
-                    bool hit;
-                    if constexpr (DT == DT_I8) {
-                        int mx = (int)v[0];
-#pragma unroll
-                        for (int c = 1; c < 31; c += 2) mx = __vimax3_s32(mx, (int)v[c], (int)v[c + 1]);
-                        mx = max(mx, (int)v[31]);
-                        hit = row_ok && mx >= fi;
-                    } else {
-                        float mx = __uint_as_float(v[0]);
-#pragma unroll
-                        for (int c = 1; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(v[c]));
-                        if constexpr (KIND == KIND_L2) hit = row_ok && (ff - 2.f * mx) <= p.thr_f;
-                        else hit = row_ok && mx >= ff;
-                    }
-                    if (__any_sync(0xffffffffu, hit)) {
-                        // exact per-element test for this 32 x 32 block
-                        const long long j0 = (long long)qt * TILE_N + col;
-                        uint32_t mask = 0;
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const long long j = j0 + c;
-                            bool pass = false;
-                            if (j < p.m) {
-                                if constexpr (DT == DT_I8 && KIND == KIND_IP) pass = (int)v[c] >= p.thr_i;
-                                if constexpr (DT == DT_I8 && KIND == KIND_L2)
-                                    pass = 2 * (int)v[c] - reinterpret_cast<const int *>(p.ny)[j] >= ri;
-                                if constexpr (DT == DT_BF16 && KIND == KIND_IP) pass = __uint_as_float(v[c]) >= p.thr_f;
-                                if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
-                                    const float nyr = reinterpret_cast<const float *>(p.ny)[j];
-                                    pass = (rzero || nyr == 0.f) ? (p.thr_f <= 0.f) : (__uint_as_float(v[c]) >= rf * nyr);
-                                }
-                                if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
-                                    const float ny2 = reinterpret_cast<const float *>(p.ny)[j];
-                                    pass = ((rf + ny2) - 2.f * __uint_as_float(v[c])) <= p.thr_f;
-                                }
-                            }
-                            mask |= (pass ? 1u : 0u) << c;
+                if (p.epi_release && warp == EPI_WARP0) {
+                    // the tile's MMAs have retired: its ring stages are free again
+                    if (lane == 0)
+                        for (int c = 0; c < p.kc; ++c) {
+                            mbar_arrive(smem_u32(&ctrl->empty[rstage]));
+                            if (++rstage == (uint32_t)p.nstages) rstage = 0;
                         }
-                        if (!row_ok) mask = 0;
-                        emit_pairs(p, mask, lane, i, j0);
-                    }
+                    __syncwarp();
                 }
+                // this warp's 128 columns of the tile, then hand the accumulator back to the MMA warp
+                uint32_t v[128];
+                tmem_ld_32x32_x128(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * 128, v);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                bool hit;
+                if constexpr (DT == DT_I8) {
+                    const int mx = (int)TreeMax<128, true>::run(v);
+                    hit = row_ok && mx >= fi;
+                } else {
+                    const float mx = __uint_as_float(TreeMax<128, false>::run(v));
+                    if constexpr (KIND == KIND_L2) hit = row_ok && (ff - 2.f * mx) <= p.thr_f;
+                    else hit = row_ok && mx >= ff;
+                }
+                if (__any_sync(0xffffffffu, hit)) {
+                    // exact per-element test for this 32 x 128 block
+                    const long long j0 = (long long)qt * TILE_N + half * 128;
+                    uint32_t mask[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t mk = 0;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            const long long j = j0 + q * 32 + c;
+                            const uint32_t x = v[q * 32 + c];
+                            bool pass = false;
+                            if (j < p.m) {
+                                if constexpr (DT == DT_I8 && KIND == KIND_IP) pass = (int)x >= p.thr_i;
+                                if constexpr (DT == DT_I8 && KIND == KIND_L2)
+                                    pass = 2 * (int)x - reinterpret_cast<const int *>(p.ny)[j] >= ri;
+                                if constexpr (DT == DT_BF16 && KIND == KIND_IP) pass = __uint_as_float(x) >= p.thr_f;
+                                if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
+                                    const float nyr = reinterpret_cast<const float *>(p.ny)[j];
+                                    pass = (rzero || nyr == 0.f) ? (p.thr_f <= 0.f) : (__uint_as_float(x) >= rf * nyr);
+                                }
+                                if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
+                                    const float ny2 = reinterpret_cast<const float *>(p.ny)[j];
+                                    pass = ((rf + ny2) - 2.f * __uint_as_float(x)) <= p.thr_f;
+                                }
+                            }
+                            mk |= (pass ? 1u : 0u) << c;
+                        }
+                        mask[q] = row_ok ? mk : 0u;
+                    }
+                    emit_pairs<4>(p, mask, lane, i, j0);
+                }
                 acc ^= 1;
                 if (acc == 0) accphase ^= 1;
             }

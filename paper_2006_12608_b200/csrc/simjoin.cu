@@ -187,6 +187,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     if (nstages > MAX_STAGES) nstages = MAX_STAGES;
     if (nstages < 2) return SIMJOIN_ERR_UNSUPPORTED;
     jp.nstages = nstages;
+    jp.epi_release = (jp.stationary && nstages >= 2 * jp.kc) ? 1 : 0;
     const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + CTRL_BYTES;
     jp.PB = (int)((n + TILE_M - 1) / TILE_M);
     jp.QT = (int)((m + TILE_N - 1) / TILE_N);
@@ -304,8 +305,8 @@ simjoin_status simjoin_create(simjoin_ctx **out, simjoin_dtype dtype, int device
     bool ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
               qres == cudaDriverEntryPointSuccess && fn != nullptr;
     ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
-    ok = ok && cudaMalloc(reinterpret_cast<void **>(&ctx->d_ctrl), 64) == cudaSuccess;
-    ok = ok && cudaMallocHost(reinterpret_cast<void **>(&ctx->h_ctrl), 64) == cudaSuccess;
+    ok = ok && cudaMalloc(reinterpret_cast<void **>(&ctx->d_ctrl), 128) == cudaSuccess;
+    ok = ok && cudaMallocHost(reinterpret_cast<void **>(&ctx->h_ctrl), 128) == cudaSuccess;
     for (auto &e : ctx->ev) ok = ok && cudaEventCreate(&e) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
