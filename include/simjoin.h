@@ -142,6 +142,40 @@ simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64
  */
 simjoin_status simjoin_last_kernel_ms(simjoin_ctx *ctx, float *prepass_ms, float *join_ms);
 
+/*
+ * Allocation-free join.  (The paper has no counterpart: this entry point exists for the
+ * sake of callers, not of the method.)
+ *
+ * Some callers must not trigger a device allocation while they run: a serving loop whose
+ * memory is handed out once by a pool and whose latency budget cannot absorb the implicit
+ * device synchronisation of cudaMalloc / cudaFree, a plugin that runs under a host
+ * framework owning all device memory, code on a path where an out-of-memory failure is not
+ * an option.  simjoin_create / simjoin_run grow scratch with cudaMalloc; this call does not.
+ * It calls no cudaMalloc, cudaFree, cudaMallocHost, event or stream creation, nor any other
+ * allocating routine: the scratch of the norm pre-pass and of the join kernel (row norms,
+ * per-tile norm bounds, the counter / status block) lives in a fixed array inside the
+ * library's device image, about 0.5 MiB that every GPU loading the library holds until the
+ * process exits.  There is no context: device, stream and dtype are arguments.
+ *
+ * Same semantics, supported kinds and error codes as simjoin_run, with these differences:
+ *   - n and m must not exceed SIMJOIN_NOALLOC_MAX_ROWS; larger inputs are rejected with
+ *     SIMJOIN_ERR_UNSUPPORTED before anything is launched (use simjoin_run instead).
+ *   - emitted indices carry no offsets; no kernel timings are recorded.
+ *   - the first call on each device looks up the device address of the scratch array and
+ *     sets kernel attributes; make that first call before any stream capture begins, and
+ *     not concurrently with another first call on the same device.
+ *   - all calls on a device share the one scratch array, which keeps the previous call's
+ *     contents (this call clears the words that must start at zero).  Two calls whose
+ *     kernels overlap on the GPU -- different streams, or different host threads -- race
+ *     on it and give wrong results: serialise them.
+ * P, Q, out_pairs are device pointers, count a host pointer, exactly as in simjoin_run;
+ * the call synchronises `cuda_stream` before it returns.
+ */
+#define SIMJOIN_NOALLOC_MAX_ROWS 65536
+simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype dtype, const void *P, int64_t n,
+                                   const void *Q, int64_t m, int32_t d, simjoin_kind kind, double threshold,
+                                   int32_t *out_pairs, uint64_t capacity, uint64_t *count);
+
 /* Release the context and its scratch.  NULL is accepted. */
 simjoin_status simjoin_destroy(simjoin_ctx *ctx);
 

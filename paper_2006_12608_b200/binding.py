@@ -22,7 +22,8 @@ DTYPE = {"i8": SIMJOIN_I8, "bf16": SIMJOIN_BF16}
 KIND = {"ip": SIMJOIN_IP, "cos": SIMJOIN_COS, "l2": SIMJOIN_L2}
 
 EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_row_norms", "simjoin_set_offsets",
-           "simjoin_last_kernel_ms", "simjoin_destroy", "simjoin_strerror")
+           "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_destroy", "simjoin_strerror")
+SIMJOIN_NOALLOC_MAX_ROWS = 65536
 
 _lib = None
 
@@ -50,6 +51,8 @@ def load() -> ctypes.CDLL:
         fn = getattr(lib, name)
         fn.restype = c.c_int
         fn.argtypes = [vp, vp, i64, vp, i64, i32, c.c_int, dbl, vp, u64, c.POINTER(u64)]
+    lib.simjoin_run_noalloc.restype = c.c_int
+    lib.simjoin_run_noalloc.argtypes = [c.c_int, vp, c.c_int, vp, i64, vp, i64, i32, c.c_int, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_row_norms.restype = c.c_int
     lib.simjoin_row_norms.argtypes = [vp, vp, i64, i32, vp]
     lib.simjoin_set_offsets.restype = c.c_int
@@ -79,6 +82,18 @@ def _ptr(x) -> Tuple[Optional[int], object]:
     if hasattr(x, "ctypes"):
         return x.ctypes.data, x
     raise TypeError(f"cannot take the address of {type(x)}")
+
+
+def simjoin_run_noalloc(device, stream, dtype, P, n, Q, m, d, kind, threshold, out_pairs, capacity):
+    """The allocation-free entry point (no context): returns (status, count) without raising.
+    For callers that may not allocate device memory while they run; rows are limited to
+    SIMJOIN_NOALLOC_MAX_ROWS and overlapping calls on one device race on the shared scratch."""
+    cnt = ctypes.c_uint64(0)
+    (pp, _a), (qp, _b), (op, _c) = _ptr(P), _ptr(Q), _ptr(out_pairs)
+    st = load().simjoin_run_noalloc(int(device), ctypes.c_void_p(stream), DTYPE[dtype] if isinstance(dtype, str) else dtype,
+                                    pp, n, qp, m, d, KIND[kind] if isinstance(kind, str) else kind, float(threshold),
+                                    op, capacity, ctypes.byref(cnt))
+    return st, cnt.value
 
 
 class Simjoin:

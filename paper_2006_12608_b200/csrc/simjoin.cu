@@ -411,6 +411,178 @@ simjoin_status simjoin_last_kernel_ms(simjoin_ctx *ctx, float *prepass_ms, float
     return SIMJOIN_OK;
 }
 
+// ------------------------------------------------------------------------------------
+// Allocation-free variant (no counterpart in the paper).  All scratch of the norm pre-pass
+// and the join kernel lives in one file-scope device array; its device address is looked up
+// once per device with cudaGetSymbolAddress (the array's name is only a host-side stand-in
+// and must never be handed to a kernel directly).
+namespace {
+
+constexpr size_t NA_ROWS = SIMJOIN_NOALLOC_MAX_ROWS;
+constexpr size_t NA_OFF_CTRL = 0;                                    // 64 B counter / status block
+constexpr size_t NA_OFF_NX = 256;                                    // NA_ROWS x 4 B
+constexpr size_t NA_OFF_NY = NA_OFF_NX + NA_ROWS * 4;                // NA_ROWS x 4 B
+constexpr size_t NA_OFF_QSTAT = NA_OFF_NY + NA_ROWS * 4;             // (NA_ROWS / 256) x 8 B
+constexpr size_t NA_BYTES = NA_OFF_QSTAT + (NA_ROWS / NORM_TILE_ROWS) * 8 + 256;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NA_BYTES];
+
+constexpr int NA_MAX_DEVICES = 64;
+struct NoAllocDevice {
+    bool ready;
+    unsigned char *scratch;   // device address of g_noalloc_scratch on this device
+    int sms, smem_optin;
+    bool attr_set[2][3];
+};
+NoAllocDevice g_na_dev[NA_MAX_DEVICES];
+EncodeTiledFn g_na_encode = nullptr;
+
+// Once per device, with that device current.
+simjoin_status noalloc_setup(int device) {
+    NoAllocDevice &nd = g_na_dev[device];
+    if (nd.ready) return SIMJOIN_OK;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&nd.sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&nd.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    if (major != 10) return SIMJOIN_ERR_ARCH;
+    if (!g_na_encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || !fn) {
+            cudaGetLastError();
+            return SIMJOIN_ERR_CUDA;
+        }
+        g_na_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    nd.scratch = static_cast<unsigned char *>(ptr);
+    std::memset(nd.attr_set, 0, sizeof nd.attr_set);
+    nd.ready = true;
+    return SIMJOIN_OK;
+}
+
+}  // namespace
+
+simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype dtype, const void *P, int64_t n,
+                                   const void *Q, int64_t m, int32_t d, simjoin_kind kind, double threshold,
+                                   int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+    if (dtype != SIMJOIN_I8 && dtype != SIMJOIN_BF16) return SIMJOIN_ERR_ARG;
+    if (device < 0 || device >= NA_MAX_DEVICES) return SIMJOIN_ERR_ARG;
+    // a stack context carries dtype / stream / limits to the helpers; it owns nothing
+    simjoin_ctx tmp{};
+    tmp.dtype = dtype;
+    tmp.device = device;
+    tmp.stream = static_cast<cudaStream_t>(cuda_stream);
+    tmp.ioff = tmp.joff = 0;
+    simjoin_status st = check_join_args(&tmp, P, n, Q, m, d, kind, threshold, out_pairs, capacity, count);
+    if (st != SIMJOIN_OK) return st;
+    if ((uint64_t)n > NA_ROWS || (uint64_t)m > NA_ROWS) return SIMJOIN_ERR_UNSUPPORTED;   // beyond the static scratch
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    if (device >= ndev) return SIMJOIN_ERR_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    st = noalloc_setup(device);
+    if (st != SIMJOIN_OK) return st;
+    NoAllocDevice &nd = g_na_dev[device];
+    if ((n > 0 && !is_device_ptr(P, device)) || (m > 0 && !is_device_ptr(Q, device))) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && !is_device_ptr(out_pairs, device)) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
+    *count = 0;
+    if (n == 0 || m == 0) return SIMJOIN_OK;
+    tmp.num_sms = nd.sms;
+    tmp.max_smem_optin = nd.smem_optin;
+    tmp.encode = g_na_encode;
+    std::memcpy(tmp.attr_set, nd.attr_set, sizeof nd.attr_set);
+
+    const bool i8 = dtype == SIMJOIN_I8;
+    const size_t es = elem_size(dtype);
+    const int row_bytes = (int)(d * es);
+    JoinParams jp;
+    std::memset(&jp, 0, sizeof jp);
+    jp.n = n;
+    jp.m = m;
+    jp.kc = (row_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES;
+    jp.last_ksteps = (row_bytes - (jp.kc - 1) * CHUNK_BYTES + 31) / 32;
+    jp.elems_per_chunk = (int)(CHUNK_BYTES / es);
+    jp.stationary = jp.kc <= MAX_STATIONARY_CHUNKS ? 1 : 0;
+    const int p_bytes = jp.stationary ? 2 * jp.kc * A_CHUNK_BYTES : 0;
+    const int stage_bytes = B_CHUNK_BYTES + (jp.stationary ? 0 : A_CHUNK_BYTES);
+    int nstages = (nd.smem_optin - 1024 - CTRL_BYTES - p_bytes) / stage_bytes;
+    if (nstages > MAX_STAGES) nstages = MAX_STAGES;
+    if (nstages < 2) return SIMJOIN_ERR_UNSUPPORTED;
+    jp.nstages = nstages;
+    jp.epi_release = (jp.stationary && nstages >= 2 * jp.kc) ? 1 : 0;
+    const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + CTRL_BYTES;
+    jp.PB = (int)((n + TILE_M - 1) / TILE_M);
+    jp.QT = (int)((m + TILE_N - 1) / TILE_N);
+    jp.out = reinterpret_cast<int2 *>(out_pairs);
+    jp.capacity = capacity;
+    unsigned long long *ctrl = reinterpret_cast<unsigned long long *>(nd.scratch + NA_OFF_CTRL);
+    jp.counter = ctrl;
+    jp.status = reinterpret_cast<unsigned int *>(ctrl + 1);
+    if (i8) {
+        if (kind == SIMJOIN_IP) jp.thr_i = clamp_to_i32(std::ceil(threshold));
+        else {
+            const double r2 = std::floor(threshold * threshold);
+            jp.thr_i = r2 >= 1073741824.0 ? 1073741824 : (int)r2;
+        }
+    } else {
+        jp.thr_f = kind == SIMJOIN_L2 ? (float)(threshold * threshold) : (float)threshold;
+    }
+    jp.nx = nd.scratch + NA_OFF_NX;
+    jp.ny = nd.scratch + NA_OFF_NY;
+    jp.qstat = nd.scratch + NA_OFF_QSTAT;
+
+    CUtensorMap mapP, mapQ;
+    if (!encode_rows_map(&tmp, &mapP, P, n, d, TILE_M) || !encode_rows_map(&tmp, &mapQ, Q, m, d, TILE_N))
+        return SIMJOIN_ERR_CUDA;
+    cudaStream_t s = tmp.stream;
+    // the array keeps the previous call's contents: the counter / status block must start at zero
+    if (cudaMemsetAsync(ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (kind != SIMJOIN_IP) {
+        const int sq = kind == SIMJOIN_COS ? 1 : 0;
+        cudaError_t e1, e2;
+        if (i8) {
+            e1 = launch_norms<true>(&tmp, P, n, d, 0, const_cast<void *>(jp.nx), nullptr);
+            e2 = launch_norms<true>(&tmp, Q, m, d, 0, const_cast<void *>(jp.ny), const_cast<void *>(jp.qstat));
+        } else {
+            e1 = launch_norms<false>(&tmp, P, n, d, sq, const_cast<void *>(jp.nx), nullptr);
+            e2 = launch_norms<false>(&tmp, Q, m, d, sq, const_cast<void *>(jp.ny), const_cast<void *>(jp.qstat));
+        }
+        if (e1 != cudaSuccess || e2 != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    }
+    cudaError_t e = cudaErrorInvalidValue;
+    if (i8 && kind == SIMJOIN_IP) e = launch_join<DT_I8, KIND_IP>(&tmp, mapP, mapQ, jp, nd.sms, smem);
+    else if (i8 && kind == SIMJOIN_L2) e = launch_join<DT_I8, KIND_L2>(&tmp, mapP, mapQ, jp, nd.sms, smem);
+    else if (!i8 && kind == SIMJOIN_IP) e = launch_join<DT_BF16, KIND_IP>(&tmp, mapP, mapQ, jp, nd.sms, smem);
+    else if (!i8 && kind == SIMJOIN_COS) e = launch_join<DT_BF16, KIND_COS>(&tmp, mapP, mapQ, jp, nd.sms, smem);
+    else if (!i8 && kind == SIMJOIN_L2) e = launch_join<DT_BF16, KIND_L2>(&tmp, mapP, mapQ, jp, nd.sms, smem);
+    std::memcpy(nd.attr_set, tmp.attr_set, sizeof nd.attr_set);
+    if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    unsigned long long host_ctrl[2] = {0, 0};
+    if (cudaMemcpyAsync(host_ctrl, ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    if ((host_ctrl[1] & 0xffffffffu) != 0) return SIMJOIN_ERR_TIMEOUT;
+    *count = host_ctrl[0];
+    return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
+}
+
 const char *simjoin_strerror(simjoin_status status) {
     switch (status) {
         case SIMJOIN_OK: return "ok";
