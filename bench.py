@@ -337,7 +337,7 @@ def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks
                                + (" x 2 (nominal int8:bf16 ratio)" if ratio == 2.0 else ""),
                 "frac_of_nominal": achieved / NOMINAL_TOPS[w.dtype], "kernel_ms": jm,
                 "prepass_ms": statistics.mean(pre_ms)}
-    launches_per_step = 1 + (2 if w.kind != "ip" else 0)
+    launches_per_step = 1 + (2 if w.kind != "ip" else 0) + (2 if w.dtype == "i8" else 0)   # join + norms + max|x|
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32" if w.dtype == "i8" else "f32", "data": "synthetic",

@@ -10,9 +10,8 @@
 //
 // CTA layout (384 threads, one CTA per SM, persistent):
 //   warp 0      TMA producer (one thread): P row block (resident while its Q sweep lasts) + Q chunk ring
-//   warp 1      MMA issuer (one thread), double-buffered 2 x 256-column accumulators
+//   warps 1, 3  MMA issuers: warp 1 even tiles -> accumulator 0, warp 3 odd tiles -> accumulator 1
 //   warp 2      TMEM allocation / release
-//   warp 3      idle
 //   warps 4-11  epilogue: warp w reads TMEM lanes 32*(w%4).., column half (w-4)/4
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word and drains.
 #pragma once
@@ -30,12 +29,20 @@ constexpr int A_CHUNK_BYTES = TILE_M * CHUNK_BYTES;   // 16 KiB
 constexpr int B_CHUNK_BYTES = TILE_N * CHUNK_BYTES;   // 32 KiB
 constexpr int MAX_STAGES = 6;
 constexpr int MAX_STATIONARY_CHUNKS = 4;          // P block kept resident up to 512-byte rows
-constexpr int NUM_THREADS = 384;
 constexpr int EPI_WARP0 = 4;
-constexpr int NUM_EPI_WARPS = 8;
+constexpr int NUM_EPI_WARPS = 8;                               // 2 per TMEM lane quarter (16 measured no faster)
+constexpr int EPI_COLS = TILE_N / (NUM_EPI_WARPS / 4);         // accumulator columns per epilogue warp
+constexpr int NUM_THREADS = 32 * (EPI_WARP0 + NUM_EPI_WARPS);
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 constexpr int CTRL_BYTES = 256;
+
+// Compile-time tuning switches for experiments (never set in the product build):
+// 1 = epilogue skips the TMEM load and the reduction, 2 = epilogue loads but skips the reduction,
+// 4 = MMA warp does not wait for operands, 8 = no producer and no stage hand-back (implies 4).
+#ifndef SIMJOIN_TUNE
+#define SIMJOIN_TUNE 0
+#endif
 
 struct JoinParams {
     long long n, m;          // rows of P, Q
@@ -62,7 +69,7 @@ struct Ctrl {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES];
     uint64_t pfull[2], pempty[2];
     uint64_t tfull[2], tempty[2];
-    uint64_t drain;
+    uint64_t drain[2];
     uint32_t tmem_base;
     volatile uint32_t abort;
 };
@@ -88,16 +95,19 @@ __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
     return false;
 }
 
-// Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting.
+// Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting.  The hot loop is a
+// bare try_wait (the hardware suspends the thread inside it); the abort flag and the cycle budget
+// are only looked at every 256 failed attempts so that they stay off the critical path.
 __device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *ctrl, unsigned int *status, uint32_t site) {
     const uint32_t addr = smem_u32(bar);
-    if (mbar_try_wait(addr, parity)) return true;
-    const long long t0 = clock64();
+    long long t0 = 0;
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(addr, parity)) return true;
-        {
+        if ((it & 0xFF) == 0) {
             if (ctrl->abort) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > WAIT_LIMIT_CYCLES) {
                 ctrl->abort = 1;
                 atomicCAS(status, 0u, 0x80000000u | site);
                 return false;
@@ -110,31 +120,31 @@ __device__ __forceinline__ bool wait_bar_warp(uint64_t *bar, uint32_t parity, Ct
     return __all_sync(0xffffffffu, ok);
 }
 
-// Tree maximum over N accumulator words (3-input max per step keeps the dependency chain
-// at log3(N) instead of N).
-template <int N, bool kInt>
+// Tree maximum over N accumulator words (3-input max per step keeps the dependency chain at
+// log3(N) instead of N).  MODE 0: fp32, 1: int32, 2: two signed 16-bit values per word.
+constexpr int MAX_F32 = 0, MAX_S32 = 1, MAX_S16X2 = 2;
+template <int MODE>
+__device__ __forceinline__ uint32_t max3_words(uint32_t a, uint32_t b, uint32_t c) {
+    if constexpr (MODE == MAX_S32) return (uint32_t)__vimax3_s32((int)a, (int)b, (int)c);
+    else if constexpr (MODE == MAX_S16X2) return __vimax3_s16x2(a, b, c);
+    else return __float_as_uint(fmaxf(fmaxf(__uint_as_float(a), __uint_as_float(b)), __uint_as_float(c)));
+}
+template <int N, int MODE>
 struct TreeMax {
     static __device__ __forceinline__ uint32_t run(const uint32_t *a) {
         constexpr int M = (N + 2) / 3;
         uint32_t t[M];
 #pragma unroll
         for (int c = 0; c < M; ++c) {
-            if constexpr (kInt) {
-                if (3 * c + 2 < N) t[c] = (uint32_t)__vimax3_s32((int)a[3 * c], (int)a[3 * c + 1], (int)a[3 * c + 2]);
-                else if (3 * c + 1 < N) t[c] = (uint32_t)max((int)a[3 * c], (int)a[3 * c + 1]);
-                else t[c] = a[3 * c];
-            } else {
-                if (3 * c + 2 < N)
-                    t[c] = __float_as_uint(fmaxf(fmaxf(__uint_as_float(a[3 * c]), __uint_as_float(a[3 * c + 1])), __uint_as_float(a[3 * c + 2])));
-                else if (3 * c + 1 < N) t[c] = __float_as_uint(fmaxf(__uint_as_float(a[3 * c]), __uint_as_float(a[3 * c + 1])));
-                else t[c] = a[3 * c];
-            }
+            if (3 * c + 2 < N) t[c] = max3_words<MODE>(a[3 * c], a[3 * c + 1], a[3 * c + 2]);
+            else if (3 * c + 1 < N) t[c] = max3_words<MODE>(a[3 * c], a[3 * c + 1], a[3 * c + 1]);
+            else t[c] = a[3 * c];
         }
-        return TreeMax<M, kInt>::run(t);
+        return TreeMax<M, MODE>::run(t);
     }
 };
-template <bool kInt>
-struct TreeMax<1, kInt> {
+template <int MODE>
+struct TreeMax<1, MODE> {
     static __device__ __forceinline__ uint32_t run(const uint32_t *a) { return a[0]; }
 };
 
@@ -169,7 +179,10 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     }
 }
 
-template <int DT, int KIND>
+// NARROW (int8 only): the host has verified that every score fits in 16 bits, so the epilogue
+// loads the accumulator packed two columns per register and reduces it with packed 16-bit max --
+// half the registers and half the ALU work of the 32-bit path, which is what bounds short-K tiles.
+template <int DT, int KIND, bool NARROW = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ, const JoinParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -186,11 +199,12 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         for (int s = 0; s < p.nstages; ++s) { mbar_init(smem_u32(&ctrl->full[s]), 1); mbar_init(smem_u32(&ctrl->empty[s]), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctrl->pfull[b]), 1);
-            mbar_init(smem_u32(&ctrl->pempty[b]), 1);
+            mbar_init(smem_u32(&ctrl->pempty[b]), 2);
             mbar_init(smem_u32(&ctrl->tfull[b]), 1);
             mbar_init(smem_u32(&ctrl->tempty[b]), NUM_EPI_WARPS);
         }
-        mbar_init(smem_u32(&ctrl->drain), 1);
+        mbar_init(smem_u32(&ctrl->drain[0]), 1);
+        mbar_init(smem_u32(&ctrl->drain[1]), 1);
         ctrl->abort = 0;
         fence_mbar_init();
         prefetch_tensormap(&mapP);
@@ -227,6 +241,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 if (pbuf == 0) pphase ^= 1;
             }
             for (int qt = un.q0; ok && qt < un.q1; ++qt) {
+#if SIMJOIN_TUNE & 8
+                if (u > 0 || qt >= un.q0 + p.nstages) continue;
+#endif
                 for (int c = 0; c < p.kc; ++c) {
                     ok = wait_bar_warp(&ctrl->empty[stage], phase ^ 1, ctrl, p.status, 2);
                     if (!ok) break;
@@ -248,13 +265,19 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             for (int t = 0; t < 200; ++t) __nanosleep(1000);
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // --------------------------------------------------------------- MMA issuer
-        // One tcgen05.commit per tile: commits are expensive (~70 cycles of tensor-pipe time
-        // each, measured), so when a whole tile's chunks fit in the ring twice over the stages of
-        // a tile are handed back to the producer by the epilogue once it has seen the tile's commit.
+    } else if (warp == 1 || warp == 3) {
+        // -------------------------------------------------------------- MMA issuers
+        // Issuing is the serial bottleneck of a short-K tile: measured on B200, a tcgen05.mma takes
+        // ~70 cycles to issue, a tcgen05.commit ~70 and every mbarrier wait ~120 even when it is
+        // already complete -- more than the 512 cycles the tensor core needs for the tile.  So two
+        // warps issue: warp 1 owns the even tiles and accumulator 0, warp 3 the odd tiles and
+        // accumulator 1; both walk the same tile sequence and skip each other's ring stages.
+        // One tcgen05.commit per tile: when a whole tile's chunks fit in the ring twice over, its
+        // stages are handed back to the producer by the epilogue once it has seen that commit.
         constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, TILE_N);
-        uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0, acc = 0, accphase = 0;
+        const uint32_t mid = warp == 1 ? 0u : 1u;
+        const uint32_t d_tmem = tmem_base + mid * TILE_N;
+        uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0, accphase = 0, tsel = 0;
         bool ok = true;
         Unit un;
         for (int u = 0; ok && get_unit(p, u, un); ++u) {
@@ -262,35 +285,46 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
                 if (!ok) break;
             }
-            for (int qt = un.q0; ok && qt < un.q1; ++qt) {
-                ok = wait_bar_warp(&ctrl->tempty[acc], accphase ^ 1, ctrl, p.status, 4);
+            for (int qt = un.q0; ok && qt < un.q1; ++qt, tsel ^= 1) {
+                if (tsel != mid) {
+                    // the other issuer's tile: step over its chunks in the ring
+                    stage += (uint32_t)p.kc;
+                    while (stage >= (uint32_t)p.nstages) { stage -= (uint32_t)p.nstages; phase ^= 1; }
+                    continue;
+                }
+                ok = wait_bar_warp(&ctrl->tempty[mid], accphase ^ 1, ctrl, p.status, 4);
                 if (!ok) break;
-                tc_fence_after();
                 for (int c = 0; c < p.kc; ++c) {
+#if !(SIMJOIN_TUNE & 12)
                     ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
                     if (!ok) break;
+#endif
                     tc_fence_after();
+                    // operands are computed by the whole (converged) warp so that they stay warp-uniform;
+                    // the four K steps are unrolled: a loop around single tcgen05.mma issues is slow
+                    uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
+                    const uint32_t a_addr = p.stationary ? smem_u32(smem_p + (size_t)(pbuf * p.kc + c) * A_CHUNK_BYTES)
+                                                         : smem_u32(sb + B_CHUNK_BYTES);
+                    const uint64_t adesc = umma_desc_sw128_kmajor(a_addr);
+                    const uint64_t bdesc = umma_desc_sw128_kmajor(smem_u32(sb));
+                    const bool last_chunk = c == p.kc - 1;
+                    const int ksteps = last_chunk ? p.last_ksteps : 4;
                     if (elect_one()) {
-                        uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
-                        const uint32_t a_addr = p.stationary ? smem_u32(smem_p + (size_t)(pbuf * p.kc + c) * A_CHUNK_BYTES)
-                                                             : smem_u32(sb + B_CHUNK_BYTES);
-                        const uint64_t adesc = umma_desc_sw128_kmajor(a_addr);
-                        const uint64_t bdesc = umma_desc_sw128_kmajor(smem_u32(sb));
-                        const int ksteps = (c == p.kc - 1) ? p.last_ksteps : 4;
-                        for (int k = 0; k < ksteps; ++k)
-                            umma_ss<DT == DT_I8>(tmem_base + acc * TILE_N, adesc + 2 * k, bdesc + 2 * k, idesc,
-                                                 (c | k) != 0 ? 1u : 0u);
+                        umma_ss<DT == DT_I8>(d_tmem, adesc, bdesc, idesc, c != 0 ? 1u : 0u);
+                        if (ksteps > 1) umma_ss<DT == DT_I8>(d_tmem, adesc + 2, bdesc + 2, idesc, 1u);
+                        if (ksteps > 2) umma_ss<DT == DT_I8>(d_tmem, adesc + 4, bdesc + 4, idesc, 1u);
+                        if (ksteps > 3) umma_ss<DT == DT_I8>(d_tmem, adesc + 6, bdesc + 6, idesc, 1u);
                         if (!p.epi_release) umma_commit(smem_u32(&ctrl->empty[stage]));
-                        if (c == p.kc - 1) umma_commit(smem_u32(&ctrl->tfull[acc]));
+                        if (last_chunk) umma_commit(smem_u32(&ctrl->tfull[mid]));
                     }
                     __syncwarp();
                     if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
-                acc ^= 1;
-                if (acc == 0) accphase ^= 1;
+                accphase ^= 1;
             }
             if (ok && p.stationary) {
+                // the P block may be overwritten once the MMAs of both issuers have retired
                 if (elect_one()) umma_commit(smem_u32(&ctrl->pempty[pbuf]));
                 __syncwarp();
                 pbuf ^= 1;
@@ -300,16 +334,16 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         if (!ok) {
             // aborting: wait (bounded) until the MMAs already issued have retired
             if (lane == 0) {
-                umma_commit(smem_u32(&ctrl->drain));
+                umma_commit(smem_u32(&ctrl->drain[mid]));
                 const long long t0 = clock64();
-                while (!mbar_try_wait(smem_u32(&ctrl->drain), 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+                while (!mbar_try_wait(smem_u32(&ctrl->drain[mid]), 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
             }
             __syncwarp();
         }
     } else if (warp >= EPI_WARP0) {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
-        const int half = (warp - EPI_WARP0) >> 2;   // which 128 of the tile's 256 columns
+        const int half = (warp - EPI_WARP0) >> 2;   // which EPI_COLS-wide slice of the tile's 256 columns
         const int row_in_tile = quarter * 32 + lane;
         uint32_t acc = 0, accphase = 0, rstage = 0;   // rstage: next ring stage to hand back
         bool ok = true;
@@ -348,7 +382,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
                 if (!ok) break;
                 tc_fence_after();
-                if (p.epi_release && warp == EPI_WARP0) {
+                if (p.epi_release && warp == EPI_WARP0 && !(SIMJOIN_TUNE & 8)) {
                     // the tile's MMAs have retired: its ring stages are free again
                     if (lane == 0)
                         for (int c = 0; c < p.kc; ++c) {
@@ -358,31 +392,55 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     __syncwarp();
                 }
                 // this warp's 128 columns of the tile, then hand the accumulator back to the MMA warp
-                uint32_t v[128];
-                tmem_ld_32x32_x128(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * 128, v);
+#if SIMJOIN_TUNE & 1
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                acc ^= 1;
+                if (acc == 0) accphase ^= 1;
+                continue;
+#endif
+                constexpr int NV = NARROW ? EPI_COLS / 2 : EPI_COLS;
+                uint32_t v[NV];
+                if constexpr (NARROW) tmem_ld_32x32_x64_pack16(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * EPI_COLS, v);
+                else tmem_ld_32x32_x128(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * EPI_COLS, v);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
                 bool hit;
-                if constexpr (DT == DT_I8) {
-                    const int mx = (int)TreeMax<128, true>::run(v);
+#if SIMJOIN_TUNE & 2
+                hit = row_ok && (int)(v[5] | v[57]) == 0x12345678;
+                if (false)
+#endif
+                if constexpr (DT == DT_I8 && NARROW) {
+                    const uint32_t m2 = TreeMax<NV, MAX_S16X2>::run(v);
+                    const int mx = max((int)(short)(m2 & 0xffffu), (int)m2 >> 16);
+                    hit = row_ok && mx >= fi;
+                } else if constexpr (DT == DT_I8) {
+                    const int mx = (int)TreeMax<EPI_COLS, MAX_S32>::run(v);
                     hit = row_ok && mx >= fi;
                 } else {
-                    const float mx = __uint_as_float(TreeMax<128, false>::run(v));
+                    const float mx = __uint_as_float(TreeMax<EPI_COLS, MAX_F32>::run(v));
                     if constexpr (KIND == KIND_L2) hit = row_ok && (ff - 2.f * mx) <= p.thr_f;
                     else hit = row_ok && mx >= ff;
                 }
                 if (__any_sync(0xffffffffu, hit)) {
-                    // exact per-element test for this 32 x 128 block
-                    const long long j0 = (long long)qt * TILE_N + half * 128;
-                    uint32_t mask[4];
+                    // exact per-element test for this 32 x EPI_COLS block
+                    const long long j0 = (long long)qt * TILE_N + half * EPI_COLS;
+                    uint32_t mask[EPI_COLS / 32];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
+                    for (int q = 0; q < EPI_COLS / 32; ++q) {
                         uint32_t mk = 0;
 #pragma unroll
                         for (int c = 0; c < 32; ++c) {
                             const long long j = j0 + q * 32 + c;
-                            const uint32_t x = v[q * 32 + c];
+                            uint32_t x;
+                            if constexpr (NARROW) {
+                                const uint32_t w = v[(q * 32 + c) >> 1];
+                                x = (c & 1) ? (uint32_t)((int)w >> 16) : (uint32_t)(int)(short)(w & 0xffffu);
+                            } else {
+                                x = v[q * 32 + c];
+                            }
                             bool pass = false;
                             if (j < p.m) {
                                 if constexpr (DT == DT_I8 && KIND == KIND_IP) pass = (int)x >= p.thr_i;
@@ -402,7 +460,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         }
                         mask[q] = row_ok ? mk : 0u;
                     }
-                    emit_pairs<4>(p, mask, lane, i, j0);
+                    emit_pairs<EPI_COLS / 32>(p, mask, lane, i, j0);
                 }
                 acc ^= 1;
                 if (acc == 0) accphase ^= 1;

@@ -105,4 +105,17 @@ row_norms_kernel(const uint4 *__restrict__ X, long long rows, int g, int sqrt_ou
     }
 }
 
+// max |x| over an int8 buffer of n16 16-byte words, folded into *out with atomicMax.  The host
+// uses it to prove that d * max|P| * max|Q| fits in 16 bits before choosing the packed epilogue.
+__global__ void __launch_bounds__(256) maxabs_i8_kernel(const uint4 *__restrict__ X, long long n16, unsigned int *out) {
+    unsigned int m = 0;   // four unsigned byte maxima
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (long long)gridDim.x * blockDim.x) {
+        const uint4 q = __ldg(X + i);
+        m = __vmaxu4(m, __vmaxu4(__vmaxu4(__vabs4(q.x), __vabs4(q.y)), __vmaxu4(__vabs4(q.z), __vabs4(q.w))));
+    }
+    unsigned int v = max(max(m & 0xffu, (m >> 8) & 0xffu), max((m >> 16) & 0xffu, m >> 24));
+    v = __reduce_max_sync(0xffffffffu, v);
+    if ((threadIdx.x & 31) == 0 && v > 0) atomicMax(out, v);
+}
+
 }  // namespace sj

@@ -44,7 +44,7 @@ struct simjoin_ctx {
     bool have_timing;
     float prepass_ms, join_ms;
     long long ioff, joff;
-    bool attr_set[2][3];
+    bool attr_set[2][3][2];
 };
 
 namespace {
@@ -143,14 +143,14 @@ cudaError_t launch_norms(const simjoin_ctx *ctx, const void *X, int64_t rows, in
     return cudaGetLastError();
 }
 
-template <int DT, int KIND>
+template <int DT, int KIND, bool NARROW = false>
 cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
                         size_t smem) {
-    auto kern = join_kernel<DT, KIND>;
-    if (!ctx->attr_set[DT][KIND]) {
+    auto kern = join_kernel<DT, KIND, NARROW>;
+    if (!ctx->attr_set[DT][KIND][NARROW ? 1 : 0]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
         if (e != cudaSuccess) return e;
-        ctx->attr_set[DT][KIND] = true;
+        ctx->attr_set[DT][KIND][NARROW ? 1 : 0] = true;
     }
     kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
     return cudaGetLastError();
@@ -224,6 +224,22 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
 
     cudaStream_t s = ctx->stream;
     if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    // int8: if d * max|P| * max|Q| fits in 16 bits, every score does, and the packed epilogue applies
+    bool narrow = false;
+    if (i8) {
+        unsigned int *d_max = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 2);
+        const int blocks = ctx->num_sms * 8;
+        maxabs_i8_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const uint4 *>(P), (long long)n * row_bytes / 16, d_max);
+        maxabs_i8_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const uint4 *>(Q), (long long)m * row_bytes / 16, d_max + 1);
+        if (cudaGetLastError() != cudaSuccess ||
+            cudaMemcpyAsync(ctx->h_ctrl + 2, ctx->d_ctrl + 2, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) {
+            cudaGetLastError();
+            return SIMJOIN_ERR_CUDA;
+        }
+        const unsigned int *h_max = reinterpret_cast<const unsigned int *>(ctx->h_ctrl + 2);
+        narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
+    }
     cudaEventRecord(ctx->ev[0], s);
     if (need_norms) {
         const int sq = kind == SIMJOIN_COS ? 1 : 0;
@@ -240,7 +256,9 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     cudaEventRecord(ctx->ev[1], s);
     const int grid = ctx->num_sms;
     cudaError_t e = cudaErrorInvalidValue;
-    if (i8 && kind == SIMJOIN_IP) e = launch_join<DT_I8, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
+    if (i8 && kind == SIMJOIN_IP && narrow) e = launch_join<DT_I8, KIND_IP, true>(ctx, mapP, mapQ, jp, grid, smem);
+    else if (i8 && kind == SIMJOIN_L2 && narrow) e = launch_join<DT_I8, KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
+    else if (i8 && kind == SIMJOIN_IP) e = launch_join<DT_I8, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_L2) e = launch_join<DT_I8, KIND_L2>(ctx, mapP, mapQ, jp, grid, smem);
     else if (!i8 && kind == SIMJOIN_IP) e = launch_join<DT_BF16, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
     else if (!i8 && kind == SIMJOIN_COS) e = launch_join<DT_BF16, KIND_COS>(ctx, mapP, mapQ, jp, grid, smem);
@@ -432,7 +450,7 @@ struct NoAllocDevice {
     bool ready;
     unsigned char *scratch;   // device address of g_noalloc_scratch on this device
     int sms, smem_optin;
-    bool attr_set[2][3];
+    bool attr_set[2][3][2];
 };
 NoAllocDevice g_na_dev[NA_MAX_DEVICES];
 EncodeTiledFn g_na_encode = nullptr;

@@ -139,6 +139,27 @@ def test_bf16_negative_threshold_and_zero_rows(ctx_bf16):
     assert_band(pairs, cnt, P, Q, "ip", -1.0)
 
 
+def test_i8_packed_16_bit_epilogue_boundary(ctx_i8):
+    """int8 scores that provably fit in 16 bits take a packed epilogue; check both sides of that
+    decision and scores at the very ends of the 16-bit range."""
+    d = 16
+    for amp, narrow in ((45, True), (46, False), (127, False)):     # d*amp*amp = 32400 / 33856 / 258064
+        P = W.random_points("i8", 300, d, 31, lo=-amp, hi=amp)
+        Q = W.random_points("i8", 520, d, 32, lo=-amp, hi=amp)
+        P[7] = amp
+        Q[11] = amp                  # score +d*amp^2
+        Q[12] = -amp                 # score -d*amp^2
+        if amp == 127:
+            P[8] = -128
+            Q[13] = -128             # score d*128*128 = 262144
+        top = d * amp * amp
+        for kind, t in (("ip", top), ("ip", top - 1.5), ("ip", 0.6 * top), ("ip", -top), ("ip", -top + 0.5),
+                        ("l2", 0.0), ("l2", 0.35 * (2 * top) ** 0.5), ("l2", 2.0 * (top ** 0.5) * 2)):
+            pairs, cnt = gpu_join(ctx_i8, P, Q, kind, t)
+            assert_exact(pairs, cnt, P, Q, kind, t)
+        assert (d * amp * amp <= 32767) == narrow
+
+
 # ------------------------------------------------------------------ degenerate thresholds and sizes
 def test_everything_and_nothing(ctx_i8, ctx_bf16):
     P, Q = W.random_points("i8", 200, 64, 9), W.random_points("i8", 300, 64, 10)
