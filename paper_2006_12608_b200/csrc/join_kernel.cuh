@@ -12,7 +12,9 @@
 //   warp 0      TMA producer (one thread): P row block (resident while its Q sweep lasts) + Q chunk ring
 //   warps 1, 3  MMA issuers: warp 1 even tiles -> accumulator 0, warp 3 odd tiles -> accumulator 1
 //   warp 2      TMEM allocation / release
-//   warps 4-11  epilogue: warp w reads TMEM lanes 32*(w%4).., column half (w-4)/4
+//   warps 4-11  epilogue: warp w reads TMEM lanes 32*(w%4).., column half (w-4)/4; row max vs a
+//               per-tile bound, then 16-column group maxima, then the exact test; passing pairs go
+//               through a per-warp shared-memory staging buffer to the output list
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word and drains.
 #pragma once
 #include "ptx_sm100.cuh"
@@ -29,6 +31,10 @@ constexpr int A_CHUNK_BYTES = TILE_M * CHUNK_BYTES;   // 16 KiB
 constexpr int B_CHUNK_BYTES = TILE_N * CHUNK_BYTES;   // 32 KiB
 constexpr int MAX_STAGES = 6;
 constexpr int MAX_STATIONARY_CHUNKS = 4;          // P block kept resident up to 512-byte rows
+#ifndef SIMJOIN_P_BUFS
+#define SIMJOIN_P_BUFS 1
+#endif
+constexpr int P_BUFS = SIMJOIN_P_BUFS;            // resident P blocks: 1 (a short bubble per Q sweep) or 2
 constexpr int EPI_WARP0 = 4;
 constexpr int NUM_EPI_WARPS = 8;                               // 2 per TMEM lane quarter (16 measured no faster)
 constexpr int EPI_COLS = TILE_N / (NUM_EPI_WARPS / 4);         // accumulator columns per epilogue warp
@@ -36,6 +42,8 @@ constexpr int NUM_THREADS = 32 * (EPI_WARP0 + NUM_EPI_WARPS);
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 constexpr int CTRL_BYTES = 256;
+constexpr int STAGE_PAIRS = 256;                               // per epilogue warp: pairs staged in shared memory
+constexpr int STAGING_BYTES = NUM_EPI_WARPS * STAGE_PAIRS * 8;  // 16 KiB
 
 // Compile-time tuning switches for experiments (never set in the product build):
 // 1 = epilogue skips the TMEM load and the reduction, 2 = epilogue loads but skips the reduction,
@@ -67,7 +75,7 @@ struct JoinParams {
 
 struct Ctrl {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES];
-    uint64_t pfull[2], pempty[2];
+    uint64_t pfull[2], pempty[2];      // P_BUFS of each are used
     uint64_t tfull[2], tempty[2];
     uint64_t drain[2];
     uint32_t tmem_base;
@@ -148,10 +156,28 @@ struct TreeMax<1, MODE> {
     static __device__ __forceinline__ uint32_t run(const uint32_t *a) { return a[0]; }
 };
 
-// Compact the pairs (i, j0 + 32*q + c), c in mask[q], of the 32 rows this warp owns into the
-// output list: popcount prefix over the warp, one atomic per warp, 8-byte stores.
+// Write `fill` staged pairs of this warp to the output list: one atomic reserves the slots, the
+// stores are coalesced.
+__device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf, int fill, int lane) {
+    if (fill == 0) return;
+    unsigned long long base = 0;
+    if (lane == 0) base = atomicAdd(p.counter, (unsigned long long)fill);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    __syncwarp();
+    for (int k = lane; k < fill; k += 32) {
+        const unsigned long long slot = base + (unsigned long long)k;
+        if (slot < p.capacity) p.out[slot] = buf[k];
+    }
+    __syncwarp();
+}
+
+// Compact the pairs (i, j0 + 32*q + c), c in mask[q], of the 32 rows this warp owns: popcount
+// prefix over the warp, then into the warp's shared-memory staging buffer, which is flushed with
+// one global atomic per ~STAGE_PAIRS pairs.  A block with more hits than the buffer holds goes
+// straight to global memory.  `fill` (warp-uniform) is the number of pairs staged so far.
 template <int NQ>
-__device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (&mask)[NQ], int lane, long long i, long long j0) {
+__device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (&mask)[NQ], int lane, long long i, long long j0,
+                                           int2 *buf, int &fill) {
     int cnt = 0;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) cnt += __popc(mask[q]);
@@ -163,20 +189,41 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     }
     const int total = __shfl_sync(0xffffffffu, incl, 31);
     if (total == 0) return;
-    unsigned long long base = 0;
-    if (lane == 0) base = atomicAdd(p.counter, (unsigned long long)total);
-    base = __shfl_sync(0xffffffffu, base, 0);
-    unsigned long long slot = base + (unsigned long long)(incl - cnt);
+    if (fill + total > STAGE_PAIRS) {
+        flush_pairs(p, buf, fill, lane);
+        fill = 0;
+    }
+    const int ii = (int)(i + p.ioff);
+    const int jj = (int)(j0 + p.joff);
+    if (total > STAGE_PAIRS) {
+        unsigned long long base = 0;
+        if (lane == 0) base = atomicAdd(p.counter, (unsigned long long)total);
+        base = __shfl_sync(0xffffffffu, base, 0);
+        unsigned long long slot = base + (unsigned long long)(incl - cnt);
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            uint32_t mk = mask[q];
+            while (mk) {
+                const int c = __ffs(mk) - 1;
+                mk &= mk - 1;
+                if (slot < p.capacity) p.out[slot] = make_int2(ii, jj + 32 * q + c);
+                ++slot;
+            }
+        }
+        return;
+    }
+    int pos = fill + incl - cnt;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
         uint32_t mk = mask[q];
         while (mk) {
             const int c = __ffs(mk) - 1;
             mk &= mk - 1;
-            if (slot < p.capacity) p.out[slot] = make_int2((int)(i + p.ioff), (int)(j0 + 32 * q + c + p.joff));
-            ++slot;
+            buf[pos++] = make_int2(ii, jj + 32 * q + c);
         }
     }
+    fill += total;
+    __syncwarp();
 }
 
 // NARROW (int8 only): the host has verified that every score fits in 16 bits, so the epilogue
@@ -189,11 +236,12 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     // 1024-byte alignment: the 128-byte swizzle pattern repeats every 1024 bytes.
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int p_bytes = p.stationary ? 2 * p.kc * A_CHUNK_BYTES : 0;
+    const int p_bytes = p.stationary ? P_BUFS * p.kc * A_CHUNK_BYTES : 0;
     const int stage_bytes = B_CHUNK_BYTES + (p.stationary ? 0 : A_CHUNK_BYTES);
     uint8_t *smem_p = smem;
     uint8_t *smem_ring = smem + p_bytes;
-    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem_ring + (size_t)p.nstages * stage_bytes);
+    int2 *smem_staging = reinterpret_cast<int2 *>(smem_ring + (size_t)p.nstages * stage_bytes);
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem_ring + (size_t)p.nstages * stage_bytes + STAGING_BYTES);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.nstages; ++s) { mbar_init(smem_u32(&ctrl->full[s]), 1); mbar_init(smem_u32(&ctrl->empty[s]), 1); }
@@ -237,8 +285,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                                     c * p.elems_per_chunk, un.pb * TILE_M);
                 }
                 __syncwarp();
-                pbuf ^= 1;
-                if (pbuf == 0) pphase ^= 1;
+                if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }
             }
             for (int qt = un.q0; ok && qt < un.q1; ++qt) {
 #if SIMJOIN_TUNE & 8
@@ -327,8 +374,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 // the P block may be overwritten once the MMAs of both issuers have retired
                 if (elect_one()) umma_commit(smem_u32(&ctrl->pempty[pbuf]));
                 __syncwarp();
-                pbuf ^= 1;
-                if (pbuf == 0) pphase ^= 1;
+                if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }
             }
         }
         if (!ok) {
@@ -346,6 +392,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         const int half = (warp - EPI_WARP0) >> 2;   // which EPI_COLS-wide slice of the tile's 256 columns
         const int row_in_tile = quarter * 32 + lane;
         uint32_t acc = 0, accphase = 0, rstage = 0;   // rstage: next ring stage to hand back
+        int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * STAGE_PAIRS;
+        int stage_fill = 0;
         bool ok = true;
         Unit un;
         for (int u = 0; ok && get_unit(p, u, un); ++u) {
@@ -379,6 +427,12 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt];
                     ff = rf + st.x;                               // (|x|^2 + min|y|^2) - 2s <= r^2
                 }
+                // per-column terms of this warp's 128 columns, 4 per lane, fetched while the tile is still
+                // being multiplied so that the exact test never waits on global memory
+                uint4 yq = make_uint4(0, 0, 0, 0);
+                if constexpr (KIND != KIND_IP)
+                    yq = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint32_t *>(p.ny) +
+                                                               ((long long)qt * TILE_N + half * EPI_COLS)) + lane);
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
                 if (!ok) break;
                 tc_fence_after();
@@ -400,72 +454,91 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 if (acc == 0) accphase ^= 1;
                 continue;
 #endif
-                constexpr int NV = NARROW ? EPI_COLS / 2 : EPI_COLS;
+                constexpr int NV = NARROW ? EPI_COLS / 2 : EPI_COLS;      // accumulator words per thread
+                constexpr int NG = 8, GW = NV / NG, GCOLS = EPI_COLS / NG;   // 8 groups of 16 columns
+                constexpr int MODE = DT == DT_BF16 ? MAX_F32 : (NARROW ? MAX_S16X2 : MAX_S32);
                 uint32_t v[NV];
                 if constexpr (NARROW) tmem_ld_32x32_x64_pack16(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * EPI_COLS, v);
                 else tmem_ld_32x32_x128(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * EPI_COLS, v);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
-                bool hit;
+                // level 0: the row maximum over this warp's 128 columns against the per-tile bound
+                // (a necessary condition of the exact test, in the same arithmetic)
+                auto bound_ok = [&](uint32_t word) -> bool {
+                    if constexpr (DT == DT_I8) {
+                        const int mx = NARROW ? max((int)(short)(word & 0xffffu), (int)word >> 16) : (int)word;
+                        return mx >= fi;
+                    } else if constexpr (KIND == KIND_L2) {
+                        return (ff - 2.f * __uint_as_float(word)) <= p.thr_f;
+                    } else {
+                        return __uint_as_float(word) >= ff;
+                    }
+                };
+                bool hit = row_ok && bound_ok(TreeMax<NV, MODE>::run(v));
 #if SIMJOIN_TUNE & 2
                 hit = row_ok && (int)(v[5] | v[57]) == 0x12345678;
-                if (false)
 #endif
-                if constexpr (DT == DT_I8 && NARROW) {
-                    const uint32_t m2 = TreeMax<NV, MAX_S16X2>::run(v);
-                    const int mx = max((int)(short)(m2 & 0xffffu), (int)m2 >> 16);
-                    hit = row_ok && mx >= fi;
-                } else if constexpr (DT == DT_I8) {
-                    const int mx = (int)TreeMax<EPI_COLS, MAX_S32>::run(v);
-                    hit = row_ok && mx >= fi;
-                } else {
-                    const float mx = __uint_as_float(TreeMax<EPI_COLS, MAX_F32>::run(v));
-                    if constexpr (KIND == KIND_L2) hit = row_ok && (ff - 2.f * mx) <= p.thr_f;
-                    else hit = row_ok && mx >= ff;
-                }
                 if (__any_sync(0xffffffffu, hit)) {
-                    // exact per-element test for this 32 x EPI_COLS block
+                    // level 1: which 16-column groups can hold a hit for this row
+                    uint32_t gm = 0;
+#pragma unroll
+                    for (int k = 0; k < NG; ++k) gm |= (bound_ok(TreeMax<GW, MODE>::run(v + k * GW)) ? 1u : 0u) << k;
+                    if (!row_ok) gm = 0;
                     const long long j0 = (long long)qt * TILE_N + half * EPI_COLS;
                     uint32_t mask[EPI_COLS / 32];
 #pragma unroll
-                    for (int q = 0; q < EPI_COLS / 32; ++q) {
+                    for (int q = 0; q < EPI_COLS / 32; ++q) mask[q] = 0;
+#pragma unroll
+                    for (int k = 0; k < NG; ++k) {
+                        if (!__any_sync(0xffffffffu, (gm >> k) & 1u)) continue;
+                        // level 2: the exact test on the 16 columns of group k
+                        const long long jg = j0 + k * GCOLS;
+                        const long long left = p.m - jg;                       // columns of this group inside Q
+                        const uint32_t valid = left >= GCOLS ? 0xffffu : (left <= 0 ? 0u : ((1u << (int)left) - 1u));
+                        uint32_t yw[GCOLS];                                     // per-column term of Q (norm kinds)
+                        if constexpr (KIND != KIND_IP) {
+#pragma unroll
+                            for (int t = 0; t < GCOLS / 4; ++t) {              // column k*16 + 4t + e lives in lane k*4 + t
+                                yw[4 * t] = __shfl_sync(0xffffffffu, yq.x, k * (GCOLS / 4) + t);
+                                yw[4 * t + 1] = __shfl_sync(0xffffffffu, yq.y, k * (GCOLS / 4) + t);
+                                yw[4 * t + 2] = __shfl_sync(0xffffffffu, yq.z, k * (GCOLS / 4) + t);
+                                yw[4 * t + 3] = __shfl_sync(0xffffffffu, yq.w, k * (GCOLS / 4) + t);
+                            }
+                        }
                         uint32_t mk = 0;
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const long long j = j0 + q * 32 + c;
+                        for (int c = 0; c < GCOLS; ++c) {
                             uint32_t x;
                             if constexpr (NARROW) {
-                                const uint32_t w = v[(q * 32 + c) >> 1];
+                                const uint32_t w = v[(k * GCOLS + c) >> 1];
                                 x = (c & 1) ? (uint32_t)((int)w >> 16) : (uint32_t)(int)(short)(w & 0xffffu);
                             } else {
-                                x = v[q * 32 + c];
+                                x = v[k * GCOLS + c];
                             }
                             bool pass = false;
-                            if (j < p.m) {
-                                if constexpr (DT == DT_I8 && KIND == KIND_IP) pass = (int)x >= p.thr_i;
-                                if constexpr (DT == DT_I8 && KIND == KIND_L2)
-                                    pass = 2 * (int)x - reinterpret_cast<const int *>(p.ny)[j] >= ri;
-                                if constexpr (DT == DT_BF16 && KIND == KIND_IP) pass = __uint_as_float(x) >= p.thr_f;
-                                if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
-                                    const float nyr = reinterpret_cast<const float *>(p.ny)[j];
-                                    pass = (rzero || nyr == 0.f) ? (p.thr_f <= 0.f) : (__uint_as_float(x) >= rf * nyr);
-                                }
-                                if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
-                                    const float ny2 = reinterpret_cast<const float *>(p.ny)[j];
-                                    pass = ((rf + ny2) - 2.f * __uint_as_float(x)) <= p.thr_f;
-                                }
+                            if constexpr (DT == DT_I8 && KIND == KIND_IP) pass = (int)x >= p.thr_i;
+                            if constexpr (DT == DT_I8 && KIND == KIND_L2) pass = 2 * (int)x - (int)yw[c] >= ri;
+                            if constexpr (DT == DT_BF16 && KIND == KIND_IP) pass = __uint_as_float(x) >= p.thr_f;
+                            if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
+                                const float nyr = __uint_as_float(yw[c]);
+                                pass = (rzero || nyr == 0.f) ? (p.thr_f <= 0.f) : (__uint_as_float(x) >= rf * nyr);
                             }
+                            if constexpr (DT == DT_BF16 && KIND == KIND_L2)
+                                pass = ((rf + __uint_as_float(yw[c])) - 2.f * __uint_as_float(x)) <= p.thr_f;
                             mk |= (pass ? 1u : 0u) << c;
                         }
-                        mask[q] = row_ok ? mk : 0u;
+                        mk &= valid;
+                        if (!((gm >> k) & 1u)) mk = 0;       // the group bound is necessary: nothing can pass here
+                        mask[k >> 1] |= mk << ((k & 1) * 16);
                     }
-                    emit_pairs<EPI_COLS / 32>(p, mask, lane, i, j0);
+                    emit_pairs<EPI_COLS / 32>(p, mask, lane, i, j0, stage_buf, stage_fill);
                 }
                 acc ^= 1;
                 if (acc == 0) accphase ^= 1;
             }
         }
+        if (ok) flush_pairs(p, stage_buf, stage_fill, lane);
     }
 
     tc_fence_before();

@@ -40,6 +40,33 @@ struct NormAcc<false> {
     }
 };
 
+// One warp, 32 consecutive rows of G 16-byte chunks each (G a power of two <= 32): G lanes share a
+// row; the row sums land in out[0..31].
+template <bool kInt8, int G>
+__device__ __forceinline__ void warp_rows_pow2(const uint4 *__restrict__ X, long long rows, long long row0, int lane,
+                                               typename NormAcc<kInt8>::type *out) {
+    using T = typename NormAcc<kInt8>::type;
+    constexpr int RPP = 32 / G;                 // rows per pass
+    constexpr int BATCH = G < 8 ? G : 8;        // passes whose loads are in flight together
+    const int sub = lane / G, chunk = lane - sub * G;
+#pragma unroll
+    for (int p0 = 0; p0 < G; p0 += BATCH) {
+        uint4 q[BATCH];
+#pragma unroll
+        for (int b = 0; b < BATCH; ++b) {
+            const long long r = row0 + (p0 + b) * RPP + sub;
+            q[b] = r < rows ? __ldg(X + r * G + chunk) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int b = 0; b < BATCH; ++b) {
+            T acc = NormAcc<kInt8>::add16(T(0), q[b]);
+#pragma unroll
+            for (int off = G >> 1; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            if (chunk == 0) out[(p0 + b) * RPP + sub] = acc;
+        }
+    }
+}
+
 // X: rows x (g * 16 bytes).  norms[r] = sum of squares of row r (fp32: its square root when
 // sqrt_out).  tile_minmax[b] = (min, max) of norms over the valid rows of tile b (may be null).
 template <bool kInt8>
@@ -53,16 +80,15 @@ row_norms_kernel(const uint4 *__restrict__ X, long long rows, int g, int sqrt_ou
     const long long row0 = (long long)blockIdx.x * NORM_TILE_ROWS + warp * 32;   // this warp's 32 rows
     const bool pow2 = g <= 32 && (g & (g - 1)) == 0;
     if (pow2) {
-        // g lanes share a row: 32/g rows per pass, g passes; all loads of a warp are contiguous
-        const int rpp = 32 / g, sub = lane / g, chunk = lane - sub * g;
-#pragma unroll 4
-        for (int pass = 0; pass < g; ++pass) {
-            const int rl = pass * rpp + sub;
-            const long long r = row0 + rl;
-            T acc = 0;
-            if (r < rows) acc = NormAcc<kInt8>::add16(acc, __ldg(X + r * g + chunk));
-            for (int off = g >> 1; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            if (chunk == 0) s_val[warp * 32 + rl] = acc;
+        // g lanes share a row: 32/g rows per pass, g passes; all loads of a warp are contiguous.
+        // Loads are issued in batches of up to 8 before anything is reduced (bytes in flight).
+        switch (g) {
+            case 1: warp_rows_pow2<kInt8, 1>(X, rows, row0, lane, s_val + warp * 32); break;
+            case 2: warp_rows_pow2<kInt8, 2>(X, rows, row0, lane, s_val + warp * 32); break;
+            case 4: warp_rows_pow2<kInt8, 4>(X, rows, row0, lane, s_val + warp * 32); break;
+            case 8: warp_rows_pow2<kInt8, 8>(X, rows, row0, lane, s_val + warp * 32); break;
+            case 16: warp_rows_pow2<kInt8, 16>(X, rows, row0, lane, s_val + warp * 32); break;
+            default: warp_rows_pow2<kInt8, 32>(X, rows, row0, lane, s_val + warp * 32); break;
         }
     } else {
         for (int rl = 0; rl < 32; ++rl) {

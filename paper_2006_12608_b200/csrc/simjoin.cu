@@ -181,14 +181,14 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.last_ksteps = (last_bytes + 31) / 32;
     jp.elems_per_chunk = (int)(CHUNK_BYTES / es);
     jp.stationary = jp.kc <= MAX_STATIONARY_CHUNKS ? 1 : 0;
-    const int p_bytes = jp.stationary ? 2 * jp.kc * A_CHUNK_BYTES : 0;
+    const int p_bytes = jp.stationary ? P_BUFS * jp.kc * A_CHUNK_BYTES : 0;
     const int stage_bytes = B_CHUNK_BYTES + (jp.stationary ? 0 : A_CHUNK_BYTES);
-    int nstages = (ctx->max_smem_optin - 1024 - CTRL_BYTES - p_bytes) / stage_bytes;
+    int nstages = (ctx->max_smem_optin - 1024 - CTRL_BYTES - STAGING_BYTES - p_bytes) / stage_bytes;
     if (nstages > MAX_STAGES) nstages = MAX_STAGES;
     if (nstages < 2) return SIMJOIN_ERR_UNSUPPORTED;
     jp.nstages = nstages;
     jp.epi_release = (jp.stationary && nstages >= 2 * jp.kc) ? 1 : 0;
-    const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + CTRL_BYTES;
+    const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + STAGING_BYTES + CTRL_BYTES;
     jp.PB = (int)((n + TILE_M - 1) / TILE_M);
     jp.QT = (int)((m + TILE_N - 1) / TILE_N);
     jp.out = reinterpret_cast<int2 *>(out_pairs);
@@ -211,7 +211,8 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
 
     const bool need_norms = kind != SIMJOIN_IP;
     if (need_norms) {
-        if (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, (size_t)m * 4) || !grow(ctx->qstat, (size_t)jp.QT * 8))
+        // ny is read in 16-entry groups up to the end of the last 256-row tile: pad it to whole tiles
+        if (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, (size_t)jp.QT * TILE_N * 4) || !grow(ctx->qstat, (size_t)jp.QT * 8))
             return SIMJOIN_ERR_CUDA;
         jp.nx = ctx->nx.ptr;
         jp.ny = ctx->ny.ptr;
@@ -536,14 +537,14 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     jp.last_ksteps = (row_bytes - (jp.kc - 1) * CHUNK_BYTES + 31) / 32;
     jp.elems_per_chunk = (int)(CHUNK_BYTES / es);
     jp.stationary = jp.kc <= MAX_STATIONARY_CHUNKS ? 1 : 0;
-    const int p_bytes = jp.stationary ? 2 * jp.kc * A_CHUNK_BYTES : 0;
+    const int p_bytes = jp.stationary ? P_BUFS * jp.kc * A_CHUNK_BYTES : 0;
     const int stage_bytes = B_CHUNK_BYTES + (jp.stationary ? 0 : A_CHUNK_BYTES);
-    int nstages = (nd.smem_optin - 1024 - CTRL_BYTES - p_bytes) / stage_bytes;
+    int nstages = (nd.smem_optin - 1024 - CTRL_BYTES - STAGING_BYTES - p_bytes) / stage_bytes;
     if (nstages > MAX_STAGES) nstages = MAX_STAGES;
     if (nstages < 2) return SIMJOIN_ERR_UNSUPPORTED;
     jp.nstages = nstages;
     jp.epi_release = (jp.stationary && nstages >= 2 * jp.kc) ? 1 : 0;
-    const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + CTRL_BYTES;
+    const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + STAGING_BYTES + CTRL_BYTES;
     jp.PB = (int)((n + TILE_M - 1) / TILE_M);
     jp.QT = (int)((m + TILE_N - 1) / TILE_N);
     jp.out = reinterpret_cast<int2 *>(out_pairs);
