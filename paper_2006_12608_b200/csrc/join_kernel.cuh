@@ -45,13 +45,6 @@ constexpr int CTRL_BYTES = 256;
 constexpr int STAGE_PAIRS = 256;                               // per epilogue warp: pairs staged in shared memory
 constexpr int STAGING_BYTES = NUM_EPI_WARPS * STAGE_PAIRS * 8;  // 16 KiB
 
-// Compile-time tuning switches for experiments (never set in the product build):
-// 1 = epilogue skips the TMEM load and the reduction, 2 = epilogue loads but skips the reduction,
-// 4 = MMA warp does not wait for operands, 8 = no producer and no stage hand-back (implies 4).
-#ifndef SIMJOIN_TUNE
-#define SIMJOIN_TUNE 0
-#endif
-
 struct JoinParams {
     long long n, m;          // rows of P, Q
     int kc;                  // 128-byte K chunks per row = ceil(row_bytes / 128)
@@ -288,9 +281,6 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }
             }
             for (int qt = un.q0; ok && qt < un.q1; ++qt) {
-#if SIMJOIN_TUNE & 8
-                if (u > 0 || qt >= un.q0 + p.nstages) continue;
-#endif
                 for (int c = 0; c < p.kc; ++c) {
                     ok = wait_bar_warp(&ctrl->empty[stage], phase ^ 1, ctrl, p.status, 2);
                     if (!ok) break;
@@ -342,10 +332,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 ok = wait_bar_warp(&ctrl->tempty[mid], accphase ^ 1, ctrl, p.status, 4);
                 if (!ok) break;
                 for (int c = 0; c < p.kc; ++c) {
-#if !(SIMJOIN_TUNE & 12)
                     ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
                     if (!ok) break;
-#endif
                     tc_fence_after();
                     // operands are computed by the whole (converged) warp so that they stay warp-uniform;
                     // the four K steps are unrolled: a loop around single tcgen05.mma issues is slow
@@ -436,7 +424,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
                 if (!ok) break;
                 tc_fence_after();
-                if (p.epi_release && warp == EPI_WARP0 && !(SIMJOIN_TUNE & 8)) {
+                if (p.epi_release && warp == EPI_WARP0) {
                     // the tile's MMAs have retired: its ring stages are free again
                     if (lane == 0)
                         for (int c = 0; c < p.kc; ++c) {
@@ -446,14 +434,6 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     __syncwarp();
                 }
                 // this warp's 128 columns of the tile, then hand the accumulator back to the MMA warp
-#if SIMJOIN_TUNE & 1
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
-                acc ^= 1;
-                if (acc == 0) accphase ^= 1;
-                continue;
-#endif
                 constexpr int NV = NARROW ? EPI_COLS / 2 : EPI_COLS;      // accumulator words per thread
                 constexpr int NG = 8, GW = NV / NG, GCOLS = EPI_COLS / NG;   // 8 groups of 16 columns
                 constexpr int MODE = DT == DT_BF16 ? MAX_F32 : (NARROW ? MAX_S16X2 : MAX_S32);
@@ -476,9 +456,6 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     }
                 };
                 bool hit = row_ok && bound_ok(TreeMax<NV, MODE>::run(v));
-#if SIMJOIN_TUNE & 2
-                hit = row_ok && (int)(v[5] | v[57]) == 0x12345678;
-#endif
                 if (__any_sync(0xffffffffu, hit)) {
                     // level 1: which 16-column groups can hold a hit for this row
                     uint32_t gm = 0;

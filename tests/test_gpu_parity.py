@@ -160,6 +160,20 @@ def test_i8_packed_16_bit_epilogue_boundary(ctx_i8):
         assert (d * amp * amp <= 32767) == narrow
 
 
+def test_staged_compaction_flush_paths(ctx_i8, ctx_bf16):
+    """Several tiles per CTA with ~100 hits per 32x128 warp block: the per-warp staging buffer
+    (256 pairs) fills and is flushed mid-kernel, not only at the end; a lower threshold then sends
+    blocks with more hits than the buffer holds straight to global memory."""
+    P, Q = W.random_points("i8", 2048, 64, 51), W.random_points("i8", 8192 + 37, 64, 52)
+    sd = (64 * 16.0) ** 0.5
+    for t in (2.0 * sd, 1.2 * sd, 0.2 * sd):
+        pairs, cnt = gpu_join(ctx_i8, P, Q, "ip", t, capacity=1 << 23)
+        assert_exact(pairs, cnt, P, Q, "ip", t)
+    Pb, Qb = W.random_points("bf16", 1100, 32, 53), W.random_points("bf16", 4096 + 5, 32, 54)
+    pairs, cnt = gpu_join(ctx_bf16, Pb, Qb, "l2", 6.5, capacity=1 << 22)
+    assert_band(pairs, cnt, Pb, Qb, "l2", 6.5)
+
+
 # ------------------------------------------------------------------ degenerate thresholds and sizes
 def test_everything_and_nothing(ctx_i8, ctx_bf16):
     P, Q = W.random_points("i8", 200, 64, 9), W.random_points("i8", 300, 64, 10)
