@@ -38,9 +38,9 @@ from paper_2006_12608_b200 import workloads as W  # noqa: E402
 METRIC = "join pair-TOPS (2*n*m*d/s)"
 UNIT = "TOPS"
 NOMINAL_TOPS = {"i8": 4500.0, "bf16": 2250.0}          # dense, per GPU (context only)
-# DRAM bytes per join-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
-# captures summarised under profiles/, scaled to the full workload by (#P-block waves x |Q|).
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes per join-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum), from a one-pass ncu
+# capture of the full-size launch (profiles/join_kernel_dram_traffic_cfg4_full.md).
+NCU_TRAFFIC_BYTES = {4: 735.62e6 + 5.89e6}
 
 
 def measured_peaks():

@@ -54,6 +54,7 @@ struct JoinParams {
     int nstages;             // ring depth
     int epi_release;         // 1: the epilogue hands ring stages back (one commit per tile); needs nstages >= 2*kc
     int PB, QT;              // number of 128-row P blocks, 256-row Q tiles
+    int qpanel;              // Q tiles per L2-resident panel
     int thr_i;               // I8/IP: ceil(t);  I8/L2: floor(r*r); both clamped
     float thr_f;             // BF16: t (IP, COS) or r*r (L2)
     const void *nx;          // per-row term of P: int32 |x|^2 (I8/L2), fp32 |x| (COS) or |x|^2 (L2)
@@ -76,24 +77,27 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
 
-// One unit of work: P block `pb` against Q tiles [q0, q1).  CTAs take whole Q sweeps in
-// waves of gridDim.x P blocks (all CTAs then walk Q together, so a Q tile is fetched from
-// HBM once and served from L2 to everyone else); the last, partial wave splits each of
-// its sweeps over several CTAs.
+// One unit of work: P block `pb` against Q tiles [q0, q1).  Q is cut into panels of `qpanel` tiles
+// that fit in L2; within a panel CTAs take whole sweeps in waves of gridDim.x P blocks (all CTAs
+// then walk the panel together, so a Q tile is fetched from HBM once and served from L2 to everyone
+// else, wave after wave); the last, partial wave of a panel splits each of its sweeps over several CTAs.
 struct Unit { int pb, q0, q1; };
 __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
     const int G = gridDim.x, c = blockIdx.x;
     const int full = p.PB / G, rem = p.PB - full * G;
-    if (u < full) { un.pb = u * G + c; un.q0 = 0; un.q1 = p.QT; return true; }
-    if (u == full && rem > 0) {
-        const int S = G / rem, idx = c / S, seg = c - idx * S;
-        if (idx >= rem) return false;
-        un.pb = full * G + idx;
-        un.q0 = (int)((long long)seg * p.QT / S);
-        un.q1 = (int)((long long)(seg + 1) * p.QT / S);
-        return un.q1 > un.q0;
-    }
-    return false;
+    const int per_panel = full + (rem > 0 ? 1 : 0);
+    const int panel = u / per_panel, v = u - panel * per_panel;
+    const int pq0 = panel * p.qpanel;
+    if (pq0 >= p.QT) return false;
+    const int pq1 = min(pq0 + p.qpanel, p.QT);
+    if (v < full) { un.pb = v * G + c; un.q0 = pq0; un.q1 = pq1; return true; }
+    // v == full, rem > 0: the partial wave
+    const int S = G / rem, idx = c / S, seg = c - idx * S;
+    un.pb = full * G + (idx < rem ? idx : 0);
+    const int len = pq1 - pq0;
+    un.q0 = pq0 + (int)((long long)seg * len / S);
+    un.q1 = idx < rem ? pq0 + (int)((long long)(seg + 1) * len / S) : un.q0;   // empty for spare CTAs
+    return true;
 }
 
 // Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting.  The hot loop is a
@@ -267,6 +271,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         bool ok = true;
         Unit un;
         for (int u = 0; ok && get_unit(p, u, un); ++u) {
+            if (un.q1 <= un.q0) continue;            // nothing for this CTA in this wave (all roles skip it)
             if (p.stationary) {
                 ok = wait_bar_warp(&ctrl->pempty[pbuf], pphase ^ 1, ctrl, p.status, 1);
                 if (!ok) break;
@@ -318,6 +323,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         bool ok = true;
         Unit un;
         for (int u = 0; ok && get_unit(p, u, un); ++u) {
+            if (un.q1 <= un.q0) continue;
             if (p.stationary) {
                 ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
                 if (!ok) break;
@@ -385,6 +391,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         bool ok = true;
         Unit un;
         for (int u = 0; ok && get_unit(p, u, un); ++u) {
+            if (un.q1 <= un.q0) continue;
             const long long i = (long long)un.pb * TILE_M + row_in_tile;
             const bool row_ok = i < p.n;
             int ri = 0;          // I8/L2: |x|^2 - floor(r^2)
