@@ -244,7 +244,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         for (int s = 0; s < p.nstages; ++s) { mbar_init(smem_u32(&ctrl->full[s]), 1); mbar_init(smem_u32(&ctrl->empty[s]), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctrl->pfull[b]), 1);
-            mbar_init(smem_u32(&ctrl->pempty[b]), 2);
+            mbar_init(smem_u32(&ctrl->pempty[b]), p.epi_release ? 2 : 1);   // one commit per issuing warp
             mbar_init(smem_u32(&ctrl->tfull[b]), 1);
             mbar_init(smem_u32(&ctrl->tempty[b]), NUM_EPI_WARPS);
         }
@@ -316,26 +316,33 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         // accumulator 1; both walk the same tile sequence and skip each other's ring stages.
         // One tcgen05.commit per tile: when a whole tile's chunks fit in the ring twice over, its
         // stages are handed back to the producer by the epilogue once it has seen that commit.
+        // Two issuers are only safe when consecutive tiles never share a ring stage (nstages >= 2*kc,
+        // the same condition as the epilogue hand-back): otherwise the second issuer would wait on a
+        // barrier that is still one phase behind, and a parity wait cannot tell phases two apart.
+        // In that case warp 1 issues every tile and warp 3 stays out.
         constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, TILE_N);
+        const bool dual = p.epi_release != 0;
         const uint32_t mid = warp == 1 ? 0u : 1u;
-        const uint32_t d_tmem = tmem_base + mid * TILE_N;
-        uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0, accphase = 0, tsel = 0;
+        uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0, tsel = 0;
+        uint32_t accph0 = 0, accph1 = 0;            // phase of each accumulator's hand-back barrier
         bool ok = true;
         Unit un;
-        for (int u = 0; ok && get_unit(p, u, un); ++u) {
+        for (int u = 0; ok && (dual || mid == 0) && get_unit(p, u, un); ++u) {
             if (un.q1 <= un.q0) continue;
             if (p.stationary) {
                 ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
                 if (!ok) break;
             }
             for (int qt = un.q0; ok && qt < un.q1; ++qt, tsel ^= 1) {
-                if (tsel != mid) {
+                if (dual && tsel != mid) {
                     // the other issuer's tile: step over its chunks in the ring
                     stage += (uint32_t)p.kc;
                     while (stage >= (uint32_t)p.nstages) { stage -= (uint32_t)p.nstages; phase ^= 1; }
                     continue;
                 }
-                ok = wait_bar_warp(&ctrl->tempty[mid], accphase ^ 1, ctrl, p.status, 4);
+                const uint32_t a = tsel;                       // accumulator of this tile
+                const uint32_t d_tmem = tmem_base + a * TILE_N;
+                ok = wait_bar_warp(&ctrl->tempty[a], (a ? accph1 : accph0) ^ 1, ctrl, p.status, 4);
                 if (!ok) break;
                 for (int c = 0; c < p.kc; ++c) {
                     ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
@@ -356,16 +363,16 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         if (ksteps > 2) umma_ss<DT == DT_I8>(d_tmem, adesc + 4, bdesc + 4, idesc, 1u);
                         if (ksteps > 3) umma_ss<DT == DT_I8>(d_tmem, adesc + 6, bdesc + 6, idesc, 1u);
                         if (!p.epi_release) umma_commit(smem_u32(&ctrl->empty[stage]));
-                        if (last_chunk) umma_commit(smem_u32(&ctrl->tfull[mid]));
+                        if (last_chunk) umma_commit(smem_u32(&ctrl->tfull[a]));
                     }
                     __syncwarp();
                     if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
-                accphase ^= 1;
+                if (a) accph1 ^= 1; else accph0 ^= 1;
             }
             if (ok && p.stationary) {
-                // the P block may be overwritten once the MMAs of both issuers have retired
+                // the P block may be overwritten once the MMAs of every issuer have retired
                 if (elect_one()) umma_commit(smem_u32(&ctrl->pempty[pbuf]));
                 __syncwarp();
                 if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }

@@ -285,6 +285,31 @@ def test_multiple_waves_and_split_tail(ctx_i8):
     assert np.isin(keys(w.planted), keys(pairs)).all()
 
 
+@pytest.mark.parametrize("d", [384, 512, 640, 2048])
+def test_many_tiles_per_cta_with_long_rows(ctx_i8, d):
+    """3, 4, 5 and 16 K chunks per tile with a dozen tiles per CTA: consecutive tiles share ring stages
+    here, which is the case where only one warp may issue MMAs."""
+    P, Q = W.random_points("i8", 1024 + 19, d, 71), W.random_points("i8", 40 * 256 + 3, d, 72)
+    t = 2.4 * (d * 16.0) ** 0.5
+    pairs, cnt = gpu_join(ctx_i8, P, Q, "ip", t, capacity=1 << 20)
+    assert_exact(pairs, cnt, P, Q, "ip", t)
+    assert cnt > 1000
+
+
+def test_several_q_panels(ctx_i8, ctx_bf16):
+    """Long rows make the L2-sized Q panels short (16 tiles at 8 KiB rows), so m = 9000 spans three
+    panels with a ragged last one; every panel has its own split partial wave."""
+    P, Q = W.random_points("i8", 300, 8192, 61), W.random_points("i8", 9000, 8192, 62)
+    t = 2.2 * (8192 * 16.0) ** 0.5
+    pairs, cnt = gpu_join(ctx_i8, P, Q, "ip", t, capacity=1 << 20)
+    assert_exact(pairs, cnt, P, Q, "ip", t)
+    assert cnt > 1000
+    Pb, Qb = W.random_points("bf16", 200, 4096, 63), W.random_points("bf16", 8500, 4096, 64)
+    pairs, cnt = gpu_join(ctx_bf16, Pb, Qb, "cos", 0.03, capacity=1 << 20)
+    assert_band(pairs, cnt, Pb, Qb, "cos", 0.03)
+    assert cnt > 1000
+
+
 # ------------------------------------------------------------------ the five configurations, reduced
 def test_cfg2_reduced(ctx_bf16):
     w = W.make_workload(2, n=6000, m=5000, planted=200)
