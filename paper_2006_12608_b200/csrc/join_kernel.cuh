@@ -17,6 +17,8 @@
 //               through a per-warp shared-memory staging buffer to the output list
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word and drains.
 #pragma once
+#include <type_traits>
+
 #include "ptx_sm100.cuh"
 
 namespace sj {
@@ -36,13 +38,16 @@ constexpr int MAX_STATIONARY_CHUNKS = 4;          // P block kept resident up to
 #endif
 constexpr int P_BUFS = SIMJOIN_P_BUFS;            // resident P blocks: 1 (a short bubble per Q sweep) or 2
 constexpr int EPI_WARP0 = 4;
-constexpr int NUM_EPI_WARPS = 8;                               // 2 per TMEM lane quarter (16 measured no faster)
+#ifndef SIMJOIN_EPI_WARPS
+#define SIMJOIN_EPI_WARPS 8
+#endif
+constexpr int NUM_EPI_WARPS = SIMJOIN_EPI_WARPS;               // 8 or 16: 2 or 4 per TMEM lane quarter
 constexpr int EPI_COLS = TILE_N / (NUM_EPI_WARPS / 4);         // accumulator columns per epilogue warp
 constexpr int NUM_THREADS = 32 * (EPI_WARP0 + NUM_EPI_WARPS);
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 constexpr int CTRL_BYTES = 256;
-constexpr int STAGE_PAIRS = 256;                               // per epilogue warp: pairs staged in shared memory
+constexpr int STAGE_PAIRS = 2048 / NUM_EPI_WARPS;                // per epilogue warp: pairs staged in shared memory
 constexpr int STAGING_BYTES = NUM_EPI_WARPS * STAGE_PAIRS * 8;  // 16 KiB
 
 struct JoinParams {
@@ -100,6 +105,23 @@ __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
     return true;
 }
 
+// The k-th tile a CTA visits in its unit.  Every CTA starts its sweep at a different offset and wraps
+// around, so that at any moment the CTAs read different Q tiles instead of all hitting the same L2
+// lines at once (measured: the aligned sweep is ~5 % slower on two-chunk tiles once Q is L2-resident).
+#ifndef SIMJOIN_ROTATE
+#define SIMJOIN_ROTATE 1
+#endif
+__device__ __forceinline__ int tile_at(const Unit &un, int k) {
+#if SIMJOIN_ROTATE
+    const int len = un.q1 - un.q0;
+    int idx = k + (int)((long long)blockIdx.x * len / gridDim.x);
+    if (idx >= len) idx -= len;
+    return un.q0 + idx;
+#else
+    return un.q0 + k;
+#endif
+}
+
 // Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting.  The hot loop is a
 // bare try_wait (the hardware suspends the thread inside it); the abort flag and the cycle budget
 // are only looked at every 256 failed attempts so that they stay off the critical path.
@@ -124,6 +146,12 @@ __device__ __forceinline__ bool wait_bar_warp(uint64_t *bar, uint32_t parity, Ct
     const bool ok = wait_bar(bar, parity, ctrl, status, site);
     return __all_sync(0xffffffffu, ok);
 }
+
+// One TMEM load of a warp's EPI_COLS columns: 32-bit words, or two 16-bit columns per word.
+__device__ __forceinline__ void tmem_ld_words(uint32_t taddr, uint32_t (&v)[128], std::false_type) { tmem_ld_32x32_x128(taddr, v); }
+__device__ __forceinline__ void tmem_ld_words(uint32_t taddr, uint32_t (&v)[64], std::false_type) { tmem_ld_32x32_x64(taddr, v); }
+__device__ __forceinline__ void tmem_ld_words(uint32_t taddr, uint32_t (&v)[64], std::true_type) { tmem_ld_32x32_x64_pack16(taddr, v); }
+__device__ __forceinline__ void tmem_ld_words(uint32_t taddr, uint32_t (&v)[32], std::true_type) { tmem_ld_32x32_x32_pack16(taddr, v); }
 
 // Tree maximum over N accumulator words (3-input max per step keeps the dependency chain at
 // log3(N) instead of N).  MODE 0: fp32, 1: int32, 2: two signed 16-bit values per word.
@@ -285,7 +313,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 __syncwarp();
                 if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }
             }
-            for (int qt = un.q0; ok && qt < un.q1; ++qt) {
+            for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
+                const int qt = tile_at(un, k);
                 for (int c = 0; c < p.kc; ++c) {
                     ok = wait_bar_warp(&ctrl->empty[stage], phase ^ 1, ctrl, p.status, 2);
                     if (!ok) break;
@@ -333,7 +362,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
                 if (!ok) break;
             }
-            for (int qt = un.q0; ok && qt < un.q1; ++qt, tsel ^= 1) {
+            for (int k = 0; ok && k < un.q1 - un.q0; ++k, tsel ^= 1) {
                 if (dual && tsel != mid) {
                     // the other issuer's tile: step over its chunks in the ring
                     stage += (uint32_t)p.kc;
@@ -413,7 +442,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 }
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) rf = reinterpret_cast<const float *>(p.nx)[i];
             }
-            for (int qt = un.q0; ok && qt < un.q1; ++qt) {
+            for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
+                const int qt = tile_at(un, k);
                 // per-tile filter bound: a necessary condition on max_j s_ij for row i to have any hit
                 int fi = p.thr_i;
                 float ff = p.thr_f;
@@ -429,10 +459,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt];
                     ff = rf + st.x;                               // (|x|^2 + min|y|^2) - 2s <= r^2
                 }
-                // per-column terms of this warp's 128 columns, 4 per lane, fetched while the tile is still
+                // per-column terms of this warp's columns, 4 per lane, fetched while the tile is still
                 // being multiplied so that the exact test never waits on global memory
                 uint4 yq = make_uint4(0, 0, 0, 0);
-                if constexpr (KIND != KIND_IP)
+                if (KIND != KIND_IP && lane < EPI_COLS / 4)
                     yq = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint32_t *>(p.ny) +
                                                                ((long long)qt * TILE_N + half * EPI_COLS)) + lane);
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
@@ -449,11 +479,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 }
                 // this warp's 128 columns of the tile, then hand the accumulator back to the MMA warp
                 constexpr int NV = NARROW ? EPI_COLS / 2 : EPI_COLS;      // accumulator words per thread
-                constexpr int NG = 8, GW = NV / NG, GCOLS = EPI_COLS / NG;   // 8 groups of 16 columns
+                constexpr int GCOLS = 16, NG = EPI_COLS / GCOLS, GW = NV / NG;  // groups of 16 columns
                 constexpr int MODE = DT == DT_BF16 ? MAX_F32 : (NARROW ? MAX_S16X2 : MAX_S32);
                 uint32_t v[NV];
-                if constexpr (NARROW) tmem_ld_32x32_x64_pack16(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * EPI_COLS, v);
-                else tmem_ld_32x32_x128(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * EPI_COLS, v);
+                tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * EPI_COLS, v, std::integral_constant<bool, NARROW>{});
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
