@@ -143,6 +143,16 @@ simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64
 simjoin_status simjoin_last_kernel_ms(simjoin_ctx *ctx, float *prepass_ms, float *join_ms);
 
 /*
+ * Self-test of the kernel's failure path.  Every wait inside the join kernel is bounded: when one
+ * expires the kernel raises a status word, drains and returns, and the call reports ERR_TIMEOUT
+ * with the context still usable.  This entry point launches a one-warp kernel that waits, with a
+ * ~1 ms budget, on a barrier nothing ever completes, and reads the status back the same way
+ * simjoin_run does.  Returns SIMJOIN_ERR_TIMEOUT when the path works (the expected result),
+ * SIMJOIN_ERR_CUDA otherwise.  It faults nothing and leaves the context usable.
+ */
+simjoin_status simjoin_selftest_wait_timeout(simjoin_ctx *ctx);
+
+/*
  * Allocation-free join.  (The paper has no counterpart: this entry point exists for the
  * sake of callers, not of the method.)
  *

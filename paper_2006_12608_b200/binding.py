@@ -22,7 +22,8 @@ DTYPE = {"i8": SIMJOIN_I8, "bf16": SIMJOIN_BF16}
 KIND = {"ip": SIMJOIN_IP, "cos": SIMJOIN_COS, "l2": SIMJOIN_L2}
 
 EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_row_norms", "simjoin_set_offsets",
-           "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_destroy", "simjoin_strerror")
+           "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_selftest_wait_timeout", "simjoin_destroy",
+           "simjoin_strerror")
 SIMJOIN_NOALLOC_MAX_ROWS = 65536
 
 _lib = None
@@ -59,6 +60,8 @@ def load() -> ctypes.CDLL:
     lib.simjoin_set_offsets.argtypes = [vp, i64, i64]
     lib.simjoin_last_kernel_ms.restype = c.c_int
     lib.simjoin_last_kernel_ms.argtypes = [vp, c.POINTER(c.c_float), c.POINTER(c.c_float)]
+    lib.simjoin_selftest_wait_timeout.restype = c.c_int
+    lib.simjoin_selftest_wait_timeout.argtypes = [vp]
     lib.simjoin_destroy.restype = c.c_int
     lib.simjoin_destroy.argtypes = [vp]
     lib.simjoin_strerror.restype = c.c_char_p
@@ -133,6 +136,9 @@ class Simjoin:
 
     def simjoin_set_offsets(self, row_offset_p: int, row_offset_q: int):
         return load().simjoin_set_offsets(self._h, row_offset_p, row_offset_q)
+
+    def simjoin_selftest_wait_timeout(self):
+        return load().simjoin_selftest_wait_timeout(self._h)
 
     def simjoin_last_kernel_ms(self):
         a, b = ctypes.c_float(0), ctypes.c_float(0)

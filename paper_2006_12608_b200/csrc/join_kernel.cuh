@@ -125,7 +125,8 @@ __device__ __forceinline__ int tile_at(const Unit &un, int k) {
 // Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting.  The hot loop is a
 // bare try_wait (the hardware suspends the thread inside it); the abort flag and the cycle budget
 // are only looked at every 256 failed attempts so that they stay off the critical path.
-__device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *ctrl, unsigned int *status, uint32_t site) {
+__device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *ctrl, unsigned int *status, uint32_t site,
+                                         long long limit = WAIT_LIMIT_CYCLES) {
     const uint32_t addr = smem_u32(bar);
     long long t0 = 0;
     for (uint32_t it = 1;; ++it) {
@@ -134,7 +135,7 @@ __device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *c
             if (ctrl->abort) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            if (now - t0 > WAIT_LIMIT_CYCLES) {
+            if (now - t0 > limit) {
                 ctrl->abort = 1;
                 atomicCAS(status, 0u, 0x80000000u | site);
                 return false;
@@ -567,6 +568,20 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
+}
+
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever completes, with a
+// short cycle budget.  The wait must give up, raise the status word and let the kernel return.
+__global__ void wait_timeout_selftest_kernel(unsigned int *status, long long limit_cycles) {
+    __shared__ Ctrl ctrl;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&ctrl.full[0]), 1);
+        ctrl.abort = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    const bool ok = wait_bar(&ctrl.full[0], 0, &ctrl, status, 0x7f, limit_cycles);
+    if (ok && threadIdx.x == 0) atomicCAS(status, 0u, 0x40000000u);   // must not happen: flags a false wake-up
 }
 
 }  // namespace sj

@@ -437,6 +437,23 @@ simjoin_status simjoin_row_norms(simjoin_ctx *ctx, const void *X, int64_t rows, 
     return SIMJOIN_OK;
 }
 
+simjoin_status simjoin_selftest_wait_timeout(simjoin_ctx *ctx) {
+    if (!ctx) return SIMJOIN_ERR_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    cudaStream_t s = ctx->stream;
+    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1), 2000000LL);   // ~1 ms
+    if (cudaGetLastError() != cudaSuccess ||
+        cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    const unsigned int kstatus = (unsigned int)(ctx->h_ctrl[1] & 0xffffffffu);
+    return kstatus == (0x80000000u | 0x7fu) ? SIMJOIN_ERR_TIMEOUT : SIMJOIN_ERR_CUDA;
+}
+
 simjoin_status simjoin_last_kernel_ms(simjoin_ctx *ctx, float *prepass_ms, float *join_ms) {
     if (!ctx || !ctx->have_timing) return SIMJOIN_ERR_ARG;
     if (prepass_ms) *prepass_ms = ctx->prepass_ms;

@@ -251,6 +251,15 @@ def test_bad_arguments_are_rejected_before_launch(ctx_i8, ctx_bf16):
     assert ctx_i8.simjoin_run(P, 64, P, 64, 64, "ip", 1e9, out, 8) == (B.SIMJOIN_OK, 0)
 
 
+def test_bounded_wait_gives_up_and_context_survives(ctx_i8):
+    """A wait on a barrier nothing completes must expire (status ERR_TIMEOUT), not hang; the context
+    keeps working afterwards.  Nothing is faulted: the wait simply runs out of its cycle budget."""
+    assert ctx_i8.simjoin_selftest_wait_timeout() == B.SIMJOIN_ERR_TIMEOUT
+    w = W.make_workload(1)
+    pairs, cnt = gpu_join(ctx_i8, w.P, w.Q, "ip", w.threshold)
+    assert_exact(pairs, cnt, w.P, w.Q, "ip", w.threshold)
+
+
 def test_run_host_matches_device_path(ctx_i8):
     w = W.make_workload(4, n=3000, m=2500, planted=120)
     want, wcnt = O.join(w.P, w.Q, "ip", w.threshold, "i8")
