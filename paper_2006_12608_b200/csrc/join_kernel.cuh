@@ -252,6 +252,88 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     __syncwarp();
 }
 
+// The MMA-issuing role (warps 1 and 3).  KC > 0 is a fast path with the chunks per tile known at
+// compile time (resident P block, full 128-byte chunks, two issuers): measured on B200, a chunk loop
+// with a run-time trip count around the tcgen05.mma issues costs ~80 cycles per tile, the run-time
+// operand-address select another ~25.  KC == 0 is the general path.
+template <int DT, int KC>
+__device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl, uint8_t *smem_p, uint8_t *smem_ring,
+                                                const int stage_bytes_rt, const uint32_t tmem_base, const int warp, const int lane) {
+    constexpr bool FAST = KC > 0;
+    constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, TILE_N);
+    const int kc = FAST ? KC : p.kc;
+    const bool stationary = FAST ? true : p.stationary != 0;
+    const bool epi_release = FAST ? true : p.epi_release != 0;
+    const int stage_bytes = FAST ? B_CHUNK_BYTES : stage_bytes_rt;
+    const bool dual = epi_release;
+    const uint32_t mid = warp == 1 ? 0u : 1u;
+    uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0, tsel = 0;
+    uint32_t accph0 = 0, accph1 = 0;            // phase of each accumulator's hand-back barrier
+    bool ok = true;
+    Unit un;
+    for (int u = 0; ok && (dual || mid == 0) && get_unit(p, u, un); ++u) {
+        if (un.q1 <= un.q0) continue;
+        if (stationary) {
+            ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
+            if (!ok) break;
+        }
+        for (int k = 0; ok && k < un.q1 - un.q0; ++k, tsel ^= 1) {
+            if (dual && tsel != mid) {
+                // the other issuer's tile: step over its chunks in the ring
+                stage += (uint32_t)kc;
+                while (stage >= (uint32_t)p.nstages) { stage -= (uint32_t)p.nstages; phase ^= 1; }
+                continue;
+            }
+            const uint32_t a = tsel;                       // accumulator of this tile
+            const uint32_t d_tmem = tmem_base + a * TILE_N;
+            ok = wait_bar_warp(&ctrl->tempty[a], (a ? accph1 : accph0) ^ 1, ctrl, p.status, 4);
+            if (!ok) break;
+#pragma unroll
+            for (int c = 0; c < (FAST ? KC : kc); ++c) {
+                ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
+                if (!ok) break;
+                tc_fence_after();
+                // operands are computed by the whole (converged) warp so that they stay warp-uniform;
+                // the four K steps are unrolled: a loop around single tcgen05.mma issues is slow
+                uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
+                const uint32_t a_addr = stationary ? smem_u32(smem_p + (size_t)(pbuf * kc + c) * A_CHUNK_BYTES)
+                                                   : smem_u32(sb + B_CHUNK_BYTES);
+                const uint64_t adesc = umma_desc_sw128_kmajor(a_addr);
+                const uint64_t bdesc = umma_desc_sw128_kmajor(smem_u32(sb));
+                const bool last_chunk = c == kc - 1;
+                const int ksteps = FAST ? 4 : (last_chunk ? p.last_ksteps : 4);
+                if (elect_one()) {
+                    umma_ss<DT == DT_I8>(d_tmem, adesc, bdesc, idesc, c != 0 ? 1u : 0u);
+                    if (ksteps > 1) umma_ss<DT == DT_I8>(d_tmem, adesc + 2, bdesc + 2, idesc, 1u);
+                    if (ksteps > 2) umma_ss<DT == DT_I8>(d_tmem, adesc + 4, bdesc + 4, idesc, 1u);
+                    if (ksteps > 3) umma_ss<DT == DT_I8>(d_tmem, adesc + 6, bdesc + 6, idesc, 1u);
+                    if (!epi_release) umma_commit(smem_u32(&ctrl->empty[stage]));
+                    if (last_chunk) umma_commit(smem_u32(&ctrl->tfull[a]));
+                }
+                __syncwarp();
+                if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
+            }
+            if (!ok) break;
+            if (a) accph1 ^= 1; else accph0 ^= 1;
+        }
+        if (ok && stationary) {
+            // the P block may be overwritten once the MMAs of every issuer have retired
+            if (elect_one()) umma_commit(smem_u32(&ctrl->pempty[pbuf]));
+            __syncwarp();
+            if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }
+        }
+    }
+    if (!ok) {
+        // aborting: wait (bounded) until the MMAs already issued have retired
+        if (lane == 0) {
+            umma_commit(smem_u32(&ctrl->drain[mid]));
+            const long long t0 = clock64();
+            while (!mbar_try_wait(smem_u32(&ctrl->drain[mid]), 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+        __syncwarp();
+    }
+}
+
 // NARROW (int8 only): the host has verified that every score fits in 16 bits, so the epilogue
 // loads the accumulator packed two columns per register and reduces it with packed 16-bit max --
 // half the registers and half the ALU work of the 32-bit path, which is what bounds short-K tiles.
@@ -350,73 +432,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         // the same condition as the epilogue hand-back): otherwise the second issuer would wait on a
         // barrier that is still one phase behind, and a parity wait cannot tell phases two apart.
         // In that case warp 1 issues every tile and warp 3 stays out.
-        constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, TILE_N);
-        const bool dual = p.epi_release != 0;
-        const uint32_t mid = warp == 1 ? 0u : 1u;
-        uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0, tsel = 0;
-        uint32_t accph0 = 0, accph1 = 0;            // phase of each accumulator's hand-back barrier
-        bool ok = true;
-        Unit un;
-        for (int u = 0; ok && (dual || mid == 0) && get_unit(p, u, un); ++u) {
-            if (un.q1 <= un.q0) continue;
-            if (p.stationary) {
-                ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
-                if (!ok) break;
-            }
-            for (int k = 0; ok && k < un.q1 - un.q0; ++k, tsel ^= 1) {
-                if (dual && tsel != mid) {
-                    // the other issuer's tile: step over its chunks in the ring
-                    stage += (uint32_t)p.kc;
-                    while (stage >= (uint32_t)p.nstages) { stage -= (uint32_t)p.nstages; phase ^= 1; }
-                    continue;
-                }
-                const uint32_t a = tsel;                       // accumulator of this tile
-                const uint32_t d_tmem = tmem_base + a * TILE_N;
-                ok = wait_bar_warp(&ctrl->tempty[a], (a ? accph1 : accph0) ^ 1, ctrl, p.status, 4);
-                if (!ok) break;
-                for (int c = 0; c < p.kc; ++c) {
-                    ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
-                    if (!ok) break;
-                    tc_fence_after();
-                    // operands are computed by the whole (converged) warp so that they stay warp-uniform;
-                    // the four K steps are unrolled: a loop around single tcgen05.mma issues is slow
-                    uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
-                    const uint32_t a_addr = p.stationary ? smem_u32(smem_p + (size_t)(pbuf * p.kc + c) * A_CHUNK_BYTES)
-                                                         : smem_u32(sb + B_CHUNK_BYTES);
-                    const uint64_t adesc = umma_desc_sw128_kmajor(a_addr);
-                    const uint64_t bdesc = umma_desc_sw128_kmajor(smem_u32(sb));
-                    const bool last_chunk = c == p.kc - 1;
-                    const int ksteps = last_chunk ? p.last_ksteps : 4;
-                    if (elect_one()) {
-                        umma_ss<DT == DT_I8>(d_tmem, adesc, bdesc, idesc, c != 0 ? 1u : 0u);
-                        if (ksteps > 1) umma_ss<DT == DT_I8>(d_tmem, adesc + 2, bdesc + 2, idesc, 1u);
-                        if (ksteps > 2) umma_ss<DT == DT_I8>(d_tmem, adesc + 4, bdesc + 4, idesc, 1u);
-                        if (ksteps > 3) umma_ss<DT == DT_I8>(d_tmem, adesc + 6, bdesc + 6, idesc, 1u);
-                        if (!p.epi_release) umma_commit(smem_u32(&ctrl->empty[stage]));
-                        if (last_chunk) umma_commit(smem_u32(&ctrl->tfull[a]));
-                    }
-                    __syncwarp();
-                    if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
-                }
-                if (!ok) break;
-                if (a) accph1 ^= 1; else accph0 ^= 1;
-            }
-            if (ok && p.stationary) {
-                // the P block may be overwritten once the MMAs of every issuer have retired
-                if (elect_one()) umma_commit(smem_u32(&ctrl->pempty[pbuf]));
-                __syncwarp();
-                if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }
-            }
-        }
-        if (!ok) {
-            // aborting: wait (bounded) until the MMAs already issued have retired
-            if (lane == 0) {
-                umma_commit(smem_u32(&ctrl->drain[mid]));
-                const long long t0 = clock64();
-                while (!mbar_try_wait(smem_u32(&ctrl->drain[mid]), 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
-            }
-            __syncwarp();
-        }
+        const bool fast = p.stationary && p.epi_release && p.last_ksteps == 4;
+        if (fast && p.kc == 1) mma_issuer_role<DT, 1>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        else if (fast && p.kc == 2) mma_issuer_role<DT, 2>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        else mma_issuer_role<DT, 0>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
     } else if (warp >= EPI_WARP0) {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
