@@ -490,11 +490,24 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 tc_fence_after();
                 if (p.epi_release && warp == EPI_WARP0) {
                     // the tile's MMAs have retired: its ring stages are free again
-                    if (lane == 0)
-                        for (int c = 0; c < p.kc; ++c) {
+                    // (straight-line for one or two chunks: this sits on the accumulator hand-back path
+                    // of the whole CTA, and a loop with a run-time trip count costs ~40 cycles per tile)
+                    if (p.kc == 1) {
+                        if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[rstage]));
+                        if (++rstage == (uint32_t)p.nstages) rstage = 0;
+                    } else if (p.kc == 2) {
+                        const uint32_t r2 = rstage + 1 == (uint32_t)p.nstages ? 0u : rstage + 1;
+                        if (lane == 0) {
                             mbar_arrive(smem_u32(&ctrl->empty[rstage]));
+                            mbar_arrive(smem_u32(&ctrl->empty[r2]));
+                        }
+                        rstage = r2 + 1 == (uint32_t)p.nstages ? 0u : r2 + 1;
+                    } else {
+                        for (int c = 0; c < p.kc; ++c) {
+                            if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[rstage]));
                             if (++rstage == (uint32_t)p.nstages) rstage = 0;
                         }
+                    }
                     __syncwarp();
                 }
                 // this warp's 128 columns of the tile, then hand the accumulator back to the MMA warp
@@ -519,7 +532,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     }
                 };
                 bool hit = row_ok && bound_ok(TreeMax<NV, MODE>::run(v));
-                if (__any_sync(0xffffffffu, hit)) {
+                if (__builtin_expect(__any_sync(0xffffffffu, hit) != 0, 0)) {   // rare for sparse joins: keep it out of line
                     // level 1: which 16-column groups can hold a hit for this row
                     uint32_t gm = 0;
 #pragma unroll
