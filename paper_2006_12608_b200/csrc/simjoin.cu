@@ -44,7 +44,7 @@ struct simjoin_ctx {
     bool have_timing;
     float prepass_ms, join_ms;
     long long ioff, joff;
-    bool attr_set[2][3][2];
+    bool attr_set[2][3][2][3];
 };
 
 namespace {
@@ -143,17 +143,27 @@ cudaError_t launch_norms(const simjoin_ctx *ctx, const void *X, int64_t rows, in
     return cudaGetLastError();
 }
 
-template <int DT, int KIND, bool NARROW = false>
-cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
-                        size_t smem) {
-    auto kern = join_kernel<DT, KIND, NARROW>;
-    if (!ctx->attr_set[DT][KIND][NARROW ? 1 : 0]) {
+template <int DT, int KIND, bool NARROW, int KC>
+cudaError_t launch_join_kc(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
+                           size_t smem) {
+    auto kern = join_kernel<DT, KIND, NARROW, KC>;
+    if (!ctx->attr_set[DT][KIND][NARROW ? 1 : 0][KC]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
         if (e != cudaSuccess) return e;
-        ctx->attr_set[DT][KIND][NARROW ? 1 : 0] = true;
+        ctx->attr_set[DT][KIND][NARROW ? 1 : 0][KC] = true;
     }
     kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
     return cudaGetLastError();
+}
+
+// Picks the instantiation with compile-time chunk count when the run-time parameters match it.
+template <int DT, int KIND, bool NARROW = false>
+cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
+                        size_t smem) {
+    const bool fast = jp.stationary && jp.epi_release && jp.last_ksteps == 4;
+    if (fast && jp.kc == 1 && jp.nstages == fast_nstages(1)) return launch_join_kc<DT, KIND, NARROW, 1>(ctx, mp, mq, jp, grid, smem);
+    if (fast && jp.kc == 2 && jp.nstages == fast_nstages(2)) return launch_join_kc<DT, KIND, NARROW, 2>(ctx, mp, mq, jp, grid, smem);
+    return launch_join_kc<DT, KIND, NARROW, 0>(ctx, mp, mq, jp, grid, smem);
 }
 
 // Q tiles per panel.  A Q of up to 64 MiB is swept whole (it mostly stays in L2 and measured faster
@@ -482,7 +492,7 @@ struct NoAllocDevice {
     bool ready;
     unsigned char *scratch;   // device address of g_noalloc_scratch on this device
     int sms, smem_optin;
-    bool attr_set[2][3][2];
+    bool attr_set[2][3][2][3];
 };
 NoAllocDevice g_na_dev[NA_MAX_DEVICES];
 EncodeTiledFn g_na_encode = nullptr;
