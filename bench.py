@@ -40,7 +40,7 @@ UNIT = "TOPS"
 NOMINAL_TOPS = {"i8": 4500.0, "bf16": 2250.0}          # dense, per GPU (context only)
 # DRAM bytes per join-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum), from a one-pass ncu
 # capture of the full-size launch (profiles/join_kernel_dram_traffic_cfg4_full.md).
-NCU_TRAFFIC_BYTES = {4: 735.62e6 + 5.89e6}
+NCU_TRAFFIC_BYTES = {4: 726.13e6 + 6.28e6}
 
 
 def measured_peaks():
