@@ -240,6 +240,37 @@ int64_t oracle_join_i8(const int8_t *P, int64_t n, const int8_t *Q, int64_t m, i
     return gather(blk, nb, out_pairs, capacity);
 }
 
+/* Hamming distance of two bit-packed rows of d coordinates (d/8 bytes each; coordinate k is bit
+ * k%8 of byte k/8): the number of coordinates that differ -- Section 4's first ip-distance. */
+int64_t oracle_hamming_bits(const uint8_t *x, const uint8_t *y, int32_t d) {
+    int64_t h = 0;
+    for (int32_t k = 0; k < d; ++k) {
+        int bx = (x[k >> 3] >> (k & 7)) & 1, by = (y[k >> 3] >> (k & 7)) & 1;
+        h += bx != by;
+    }
+    return h;
+}
+
+/* All (i, j) with Hamming(P[i], Q[j]) <= r over bit-packed rows; output as in the other joins. */
+int64_t oracle_join_hamming_bits(const uint8_t *P, int64_t n, const uint8_t *Q, int64_t m, int32_t d, double r,
+                                 int32_t *out_pairs, int64_t capacity, int32_t nthreads) {
+    if (n < 0 || m < 0 || d <= 0 || (d & 7) || capacity < 0 || isnan(r) || r < 0) return -1;
+    if (n >= INT32_MAX || m >= INT32_MAX) return -1;
+    int nt = resolve_threads(nthreads);
+    int64_t nb = num_blocks(n, nt);
+    pairbuf *blk = (pairbuf *)calloc((size_t)nb, sizeof(pairbuf));
+    if (!blk) return -1;
+    const size_t rb = (size_t)d / 8;
+#pragma omp parallel for schedule(dynamic, 1) num_threads(nt)
+    for (int64_t b = 0; b < nb; ++b) {
+        int64_t i0 = n * b / nb, i1 = n * (b + 1) / nb;
+        for (int64_t i = i0; i < i1; ++i)
+            for (int64_t j = 0; j < m; ++j)
+                if ((double)oracle_hamming_bits(P + (size_t)i * rb, Q + (size_t)j * rb, d) <= r) pb_push(&blk[b], i, j);
+    }
+    return gather(blk, nb, out_pairs, capacity);
+}
+
 int64_t oracle_join_bf16(const uint16_t *P, int64_t n, const uint16_t *Q, int64_t m, int32_t d, int32_t kind,
                          double threshold, int32_t *out_pairs, int64_t capacity, int32_t nthreads) {
     if (n < 0 || m < 0 || d <= 0 || capacity < 0 || kind < KIND_IP || kind > KIND_L2) return -1;

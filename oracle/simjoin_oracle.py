@@ -66,6 +66,10 @@ def _load():
         fn = getattr(lib, name)
         fn.restype = i64
         fn.argtypes = [vp, i64, vp, i64, i32, i32, dbl, vp, i64, i32]
+    lib.oracle_join_hamming_bits.restype = i64
+    lib.oracle_join_hamming_bits.argtypes = [vp, i64, vp, i64, i32, dbl, vp, i64, i32]
+    lib.oracle_hamming_bits.restype = i64
+    lib.oracle_hamming_bits.argtypes = [vp, vp, i32]
     lib.oracle_scores_i8.restype = i32
     lib.oracle_scores_i8.argtypes = [vp, vp, i32, i32, vp, i64, vp]
     lib.oracle_scores_bf16.restype = i32
@@ -117,6 +121,33 @@ def join(P: np.ndarray, Q: np.ndarray, kind: str, threshold: float, dtype: str,
         if capacity is not None or cnt <= cap:
             return out[:min(cnt, cap)].copy(), int(cnt)
         cap = int(cnt)
+
+
+def join_hamming(Pbits: np.ndarray, Qbits: np.ndarray, d: int, r: float, threads: int = 0):
+    """All (i, j) with Hamming(P[i], Q[j]) <= r over bit-packed uint8 rows (d/8 bytes per row, bit k%8 of
+    byte k/8 is coordinate k), sorted by (i, j).  Returns (pairs, count)."""
+    lib = _load()
+    if Pbits.dtype != np.uint8 or Qbits.dtype != np.uint8 or Pbits.ndim != 2 or Qbits.ndim != 2:
+        raise TypeError("expected 2-D uint8 arrays of packed bits")
+    if Pbits.shape[1] * 8 != d or Qbits.shape[1] * 8 != d:
+        raise ValueError("rows must hold d/8 bytes")
+    Pbits, Qbits = np.ascontiguousarray(Pbits), np.ascontiguousarray(Qbits)
+    cap = 1 << 16
+    while True:
+        out = np.empty((cap, 2), dtype=np.int32)
+        cnt = lib.oracle_join_hamming_bits(Pbits.ctypes.data, Pbits.shape[0], Qbits.ctypes.data, Qbits.shape[0], d,
+                                           float(r), out.ctypes.data, cap, threads)
+        if cnt < 0:
+            raise ValueError("oracle rejected the arguments")
+        if cnt <= cap:
+            return out[:cnt].copy(), int(cnt)
+        cap = int(cnt)
+
+
+def hamming(x: np.ndarray, y: np.ndarray, d: int) -> int:
+    """Hamming distance of two bit-packed rows."""
+    x, y = np.ascontiguousarray(x, dtype=np.uint8), np.ascontiguousarray(y, dtype=np.uint8)
+    return int(_load().oracle_hamming_bits(x.ctypes.data, y.ctypes.data, d))
 
 
 def band_sets(P, Q, kind, threshold, dtype, rel: float = 1e-2, threads: int = 0):

@@ -183,3 +183,23 @@ def random_points(dtype: str, rows: int, d: int, seed: int, lo: int = -3, hi: in
     if dtype == "bf16":
         return f32_to_bf16_bits(np.float32(scale) * rng.standard_normal((rows, d), dtype=np.float32))
     raise ValueError(dtype)
+
+
+def random_bits(rows: int, d: int, seed: int, planted_from=None, flips: int = 0):
+    """Bit-packed points in {0,1}^d: uint8 array (rows, d/8), coordinate k = bit k%8 of byte k/8.
+    With `planted_from` (another packed array) the first len(planted_from) rows are copies of it with
+    `flips` distinct coordinates flipped each (near pairs at Hamming distance `flips`)."""
+    if d % 8:
+        raise ValueError("d must be a multiple of 8")
+    rng = np.random.default_rng([seed, rows, d, 99])
+    bits = rng.integers(0, 2, size=(rows, d), dtype=np.uint8)
+    if planted_from is not None:
+        src = np.unpackbits(planted_from, axis=1, bitorder="little")[:, :d]
+        k = len(src)
+        cols = _distinct_coords(rng, k, d, flips)
+        src = src.copy()
+        if flips:
+            rr = np.repeat(np.arange(k), flips)
+            src[rr, cols.ravel()] ^= 1
+        bits[:k] = src
+    return np.packbits(bits, axis=1, bitorder="little")

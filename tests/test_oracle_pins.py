@@ -30,7 +30,8 @@ def to_arr(rows, dtype):
 
 
 # ------------------------------------------------------------------ hand-worked
-GOLDEN = sorted(glob.glob(os.path.join(os.path.dirname(__file__), "golden", "*.json")))
+GOLDEN = sorted(g for g in glob.glob(os.path.join(os.path.dirname(__file__), "golden", "*.json"))
+                if not os.path.basename(g).startswith("hamming"))
 
 
 @pytest.mark.parametrize("path", GOLDEN, ids=[os.path.basename(p) for p in GOLDEN])
@@ -45,6 +46,44 @@ def test_hand_worked_cases(path):
         pairs, cnt = O.join(P, Q, g["kind"], case["threshold"], g["dtype"])
         assert cnt == len(case["pairs"]), case
         assert pairs.tolist() == sorted(case["pairs"]), case      # sorted by (i, j)
+
+
+def test_hamming_hand_worked_case():
+    with open(os.path.join(os.path.dirname(__file__), "golden", "hamming_bits_d16.json")) as f:
+        g = json.load(f)
+    d = g["d"]
+    P = np.packbits(np.array(g["P"], dtype=np.uint8), axis=1, bitorder="little")
+    Q = np.packbits(np.array(g["Q"], dtype=np.uint8), axis=1, bitorder="little")
+    for i in range(len(P)):
+        for j in range(len(Q)):
+            assert O.hamming(P[i], Q[j], d) == g["distances"][i][j]
+    for case in g["cases"]:
+        pairs, cnt = O.join_hamming(P, Q, d, case["r"])
+        assert cnt == len(case["pairs"]) and pairs.tolist() == sorted(case["pairs"]), case
+
+
+def test_hamming_oracle_against_embeddings_and_pm1_inner_product():
+    # three independent routes to the same set: (a) the paper's f, g embedding with d' = 2d,
+    # (b) <x+-, y+-> = d - 2*Hamming through the int8 inner-product oracle, (c) numpy on unpacked bits
+    d = 128
+    P = W.random_bits(60, d, 1)
+    Q = W.random_bits(90, d, 2, planted_from=P[:12], flips=9)
+    pu = np.unpackbits(P, axis=1, bitorder="little").astype(np.int64)
+    qu = np.unpackbits(Q, axis=1, bitorder="little").astype(np.int64)
+    f = np.stack([pu, 1 - pu], axis=2).reshape(len(P), -1)
+    g = np.stack([1 - qu, qu], axis=2).reshape(len(Q), -1)
+    H = f @ g.T
+    assert np.array_equal(H, (pu[:, None, :] != qu[None, :, :]).sum(axis=2))
+    for r in (0, 9, 40.5, 58, 64):
+        pairs, cnt = O.join_hamming(P, Q, d, r)
+        ii, jj = np.nonzero(H <= r)
+        assert as_set(pairs) == set(zip(ii.tolist(), jj.tolist())) and cnt == len(ii)
+        pm_p, pm_q = (2 * pu - 1).astype(np.int8), (2 * qu - 1).astype(np.int8)
+        ip_pairs, _c = O.join(pm_p, pm_q, "ip", d - 2 * math.floor(r), "i8")
+        assert as_set(ip_pairs) == as_set(pairs)
+    assert all((i, i) in as_set(O.join_hamming(P, Q, d, 9)[0]) for i in range(12))      # planted at distance 9
+    with pytest.raises(ValueError):
+        O.join_hamming(P, Q, d, -1.0)
 
 
 # ------------------------------------------------- independent formulations
