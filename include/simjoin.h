@@ -117,6 +117,23 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
                                 int32_t *out_pairs_host, uint64_t capacity, uint64_t *count);
 
 /*
+ * Hamming join on bit-packed points (Section 4: Hamming is the first ip-distance listed, with the
+ * embedding f(x) = (x_k, 1-x_k)_k, g(y) = (1-y_k, y_k)_k).  keep (i, j) when Hamming(x_i, y_j) <= r.
+ *
+ *   P_bits, Q_bits  device pointers, n and m rows of d/8 bytes; coordinate k of a row is bit k%8
+ *                   (least significant first) of byte k/8.  d must be a multiple of 128 (16-byte rows),
+ *                   base pointers 16-byte aligned.  I8 contexts only (ERR_UNSUPPORTED otherwise).
+ *   r               >= 0; a real r acts as floor(r).  ERR_ARG for NaN or negative r.
+ *
+ * The library applies the operand transform x -> 2x-1 on the device (bits to +-1 int8 rows in staging
+ * owned by the context: d' = d instead of the paper's 2d, because <x+-, y+-> = d - 2*Hamming) and runs
+ * the int8 inner-product join with threshold d - 2*floor(r).  Result, count, capacity and error
+ * semantics are those of simjoin_run; the pair set is exact.
+ */
+simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t n, const void *Q_bits, int64_t m,
+                                   int32_t d, double r, int32_t *out_pairs, uint64_t capacity, uint64_t *count);
+
+/*
  * Row squared norms, the pre-pass behind the |x|^2 and |y|^2 terms of the
  * squared-L2 and cosine ip-distances (Section 4).  X: device pointer, rows x d.
  * out: device pointer to `rows` values -- int32 (exact) for I8 contexts, fp32

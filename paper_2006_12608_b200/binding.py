@@ -21,7 +21,7 @@ SIMJOIN_IP, SIMJOIN_COS, SIMJOIN_L2 = 0, 1, 2
 DTYPE = {"i8": SIMJOIN_I8, "bf16": SIMJOIN_BF16}
 KIND = {"ip": SIMJOIN_IP, "cos": SIMJOIN_COS, "l2": SIMJOIN_L2}
 
-EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_row_norms", "simjoin_set_offsets",
+EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_hamming", "simjoin_row_norms", "simjoin_set_offsets",
            "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_selftest_wait_timeout", "simjoin_destroy",
            "simjoin_strerror")
 SIMJOIN_NOALLOC_MAX_ROWS = 65536
@@ -52,6 +52,8 @@ def load() -> ctypes.CDLL:
         fn = getattr(lib, name)
         fn.restype = c.c_int
         fn.argtypes = [vp, vp, i64, vp, i64, i32, c.c_int, dbl, vp, u64, c.POINTER(u64)]
+    lib.simjoin_run_hamming.restype = c.c_int
+    lib.simjoin_run_hamming.argtypes = [vp, vp, i64, vp, i64, i32, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_run_noalloc.restype = c.c_int
     lib.simjoin_run_noalloc.argtypes = [c.c_int, vp, c.c_int, vp, i64, vp, i64, i32, c.c_int, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_row_norms.restype = c.c_int
@@ -128,6 +130,12 @@ class Simjoin:
         (pp, _a), (qp, _b), (op, _c) = _ptr(P), _ptr(Q), _ptr(out_pairs)
         st = load().simjoin_run_host(self._h, pp, n, qp, m, d, KIND[kind] if isinstance(kind, str) else kind,
                                      float(threshold), op, capacity, ctypes.byref(cnt))
+        return st, cnt.value
+
+    def simjoin_run_hamming(self, P_bits, n, Q_bits, m, d, r, out_pairs, capacity):
+        cnt = ctypes.c_uint64(0)
+        (pp, _a), (qp, _b), (op, _c) = _ptr(P_bits), _ptr(Q_bits), _ptr(out_pairs)
+        st = load().simjoin_run_hamming(self._h, pp, n, qp, m, d, float(r), op, capacity, ctypes.byref(cnt))
         return st, cnt.value
 
     def simjoin_row_norms(self, X, rows, d, out):

@@ -144,4 +144,22 @@ __global__ void __launch_bounds__(256) maxabs_i8_kernel(const uint4 *__restrict_
     if ((threadIdx.x & 31) == 0 && v > 0) atomicMax(out, v);
 }
 
+// Operand transform for the Hamming ip-distance (Section 4): bit-packed {0,1} coordinates -> +-1 int8
+// rows, so that <x, y> = d - 2 * Hamming(x, y) and the int8 inner-product join applies with d' = d.
+// One thread expands 16 bits (coordinate k = bit k%8 of byte k/8) into 16 bytes: 1 -> +1, 0 -> -1.
+__global__ void __launch_bounds__(256) unpack_bits_pm1_kernel(const uint16_t *__restrict__ bits, long long nhalf,
+                                                              uint4 *__restrict__ out) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= nhalf) return;
+    const uint32_t h = bits[t];
+    uint32_t w[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint32_t nib = (h >> (4 * q)) & 0xfu;
+        const uint32_t ones = (nib * 0x00204081u) & 0x01010101u;        // bit i of the nibble -> byte i
+        w[q] = ones | ((ones ^ 0x01010101u) * 0xffu);                   // 0x01 where set, 0xff (-1) where clear
+    }
+    out[t] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 }  // namespace sj

@@ -430,6 +430,37 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
     return st;
 }
 
+simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t n, const void *Q_bits, int64_t m, int32_t d,
+                                   double r, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+    if (!ctx || !count || !P_bits || !Q_bits) return SIMJOIN_ERR_ARG;
+    if (ctx->dtype != SIMJOIN_I8) return SIMJOIN_ERR_UNSUPPORTED;
+    if (n < 0 || m < 0 || n >= SIMJOIN_MAX_ROWS || m >= SIMJOIN_MAX_ROWS || d <= 0) return SIMJOIN_ERR_ARG;
+    if (std::isnan(r) || r < 0) return SIMJOIN_ERR_ARG;
+    if (!out_pairs && capacity > 0) return SIMJOIN_ERR_ARG;
+    if (d % 128 != 0 || d > SIMJOIN_MAX_ROW_BYTES) return SIMJOIN_ERR_UNSUPPORTED;    // 16-byte packed rows
+    if ((reinterpret_cast<uintptr_t>(P_bits) & 15u) || (reinterpret_cast<uintptr_t>(Q_bits) & 15u)) return SIMJOIN_ERR_UNSUPPORTED;
+    if (n + ctx->ioff >= SIMJOIN_MAX_ROWS || m + ctx->joff >= SIMJOIN_MAX_ROWS) return SIMJOIN_ERR_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    if ((n > 0 && !is_device_ptr(P_bits, ctx->device)) || (m > 0 && !is_device_ptr(Q_bits, ctx->device))) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && !is_device_ptr(out_pairs, ctx->device)) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
+    *count = 0;
+    if (n == 0 || m == 0) return SIMJOIN_OK;
+    const size_t pb = (size_t)n * d, qb = (size_t)m * d;
+    if (!grow(ctx->stage_p, pb) || !grow(ctx->stage_q, qb)) return SIMJOIN_ERR_CUDA;
+    cudaStream_t s = ctx->stream;
+    const long long ph = (long long)n * d / 16, qh = (long long)m * d / 16;      // 16-bit groups
+    unpack_bits_pm1_kernel<<<(unsigned)((ph + 255) / 256), 256, 0, s>>>(reinterpret_cast<const uint16_t *>(P_bits), ph,
+                                                                         reinterpret_cast<uint4 *>(ctx->stage_p.ptr));
+    unpack_bits_pm1_kernel<<<(unsigned)((qh + 255) / 256), 256, 0, s>>>(reinterpret_cast<const uint16_t *>(Q_bits), qh,
+                                                                         reinterpret_cast<uint4 *>(ctx->stage_q.ptr));
+    if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    // Hamming <= r  <=>  Hamming <= floor(r)  <=>  d - 2*Hamming >= d - 2*floor(r)
+    const double t = (double)d - 2.0 * std::floor(r);
+    return run_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, SIMJOIN_IP, t, out_pairs, capacity, count);
+}
+
 simjoin_status simjoin_row_norms(simjoin_ctx *ctx, const void *X, int64_t rows, int32_t d, void *out) {
     if (!ctx || !out) return SIMJOIN_ERR_ARG;
     simjoin_status st = check_matrix_args(ctx, X, rows, d);
