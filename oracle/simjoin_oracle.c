@@ -271,6 +271,69 @@ int64_t oracle_join_hamming_bits(const uint8_t *P, int64_t n, const uint8_t *Q, 
     return gather(blk, nb, out_pairs, capacity);
 }
 
+/* ------------------------------------------------------------------ LSH-bucketed join
+ * Section 4's second algorithm: L repetitions; in each, every point gets a hash that concatenates k
+ * base hashes, the points are split into buckets by that hash, and the brute-force join runs inside
+ * each bucket; the result is the union over the repetitions.  With a fixed hash family the result is
+ * therefore exactly { (i, j) in the brute-force join : the hashes of x_i and y_j agree in at least
+ * one repetition } -- which is what this oracle enumerates, with no buckets at all.
+ * Base hash (bit sampling, the classic monotone LSH for Hamming / +-1 data): h(x) = [x_c > 0] for a
+ * sampled coordinate c.  Coordinate of repetition l, bit b: splitmix64(seed, l*64 + b) mod d -- a
+ * counter-based generator that the CUDA library implements on its own. */
+static uint64_t splitmix64_at(uint64_t seed, uint64_t idx) {
+    uint64_t z = seed + (idx + 1) * 0x9E3779B97F4A7C15ULL;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+
+int32_t oracle_lsh_coordinate(uint64_t seed, int32_t rep, int32_t bit, int32_t d) {
+    return (int32_t)(splitmix64_at(seed, (uint64_t)rep * 64u + (uint64_t)bit) % (uint64_t)d);
+}
+
+/* keys[l * rows + i] = the k-bit hash of row i in repetition l (bit b = [x_{c(l,b)} > 0]). */
+void oracle_lsh_keys_i8(const int8_t *X, int64_t rows, int32_t d, int32_t L, int32_t k, uint64_t seed, uint32_t *keys) {
+    for (int32_t l = 0; l < L; ++l)
+        for (int64_t i = 0; i < rows; ++i) {
+            uint32_t key = 0;
+            for (int32_t b = 0; b < k; ++b)
+                if (X[(size_t)i * d + oracle_lsh_coordinate(seed, l, b, d)] > 0) key |= 1u << b;
+            keys[(size_t)l * rows + i] = key;
+        }
+}
+
+int64_t oracle_lsh_join_i8(const int8_t *P, int64_t n, const int8_t *Q, int64_t m, int32_t d, double threshold,
+                           int32_t L, int32_t k, uint64_t seed, int32_t *out_pairs, int64_t capacity, int32_t nthreads) {
+    if (n < 0 || m < 0 || d <= 0 || capacity < 0 || isnan(threshold) || L < 1 || L > 64 || k < 0 || k > 20) return -1;
+    if (n >= INT32_MAX || m >= INT32_MAX) return -1;
+    int nt = resolve_threads(nthreads);
+    uint32_t *KP = (uint32_t *)malloc(((size_t)L * n + 1) * sizeof(uint32_t));
+    uint32_t *KQ = (uint32_t *)malloc(((size_t)L * m + 1) * sizeof(uint32_t));
+    int64_t nb = num_blocks(n, nt);
+    pairbuf *blk = (pairbuf *)calloc((size_t)nb, sizeof(pairbuf));
+    int64_t total = -1;
+    if (KP && KQ && blk) {
+        oracle_lsh_keys_i8(P, n, d, L, k, seed, KP);
+        oracle_lsh_keys_i8(Q, m, d, L, k, seed, KQ);
+#pragma omp parallel for schedule(dynamic, 1) num_threads(nt)
+        for (int64_t b = 0; b < nb; ++b) {
+            int64_t i0 = n * b / nb, i1 = n * (b + 1) / nb;
+            for (int64_t i = i0; i < i1; ++i)
+                for (int64_t j = 0; j < m; ++j) {
+                    int collide = 0;
+                    for (int32_t l = 0; l < L && !collide; ++l) collide = KP[(size_t)l * n + i] == KQ[(size_t)l * m + j];
+                    if (collide && (double)oracle_ip_i8(P + (size_t)i * d, Q + (size_t)j * d, d) >= threshold) pb_push(&blk[b], i, j);
+                }
+        }
+        total = gather(blk, nb, out_pairs, capacity);
+    } else {
+        free(blk);
+    }
+    free(KP);
+    free(KQ);
+    return total;
+}
+
 int64_t oracle_join_bf16(const uint16_t *P, int64_t n, const uint16_t *Q, int64_t m, int32_t d, int32_t kind,
                          double threshold, int32_t *out_pairs, int64_t capacity, int32_t nthreads) {
     if (n < 0 || m < 0 || d <= 0 || capacity < 0 || kind < KIND_IP || kind > KIND_L2) return -1;

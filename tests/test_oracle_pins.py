@@ -86,6 +86,51 @@ def test_hamming_oracle_against_embeddings_and_pm1_inner_product():
         O.join_hamming(P, Q, d, -1.0)
 
 
+# ------------------------------------------------------------------ LSH-bucketed join
+def _splitmix64(seed, idx):
+    M = (1 << 64) - 1
+    z = (seed + (idx + 1) * 0x9E3779B97F4A7C15) & M
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & M
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & M
+    return z ^ (z >> 31)
+
+
+def test_lsh_join_is_brute_force_restricted_to_colliding_pairs():
+    # independent route: python-int splitmix64 for the sampled coordinates, numpy for keys and scores
+    w = W.make_workload(4, n=700, m=600, planted=80)
+    L, k, seed, d = 5, 4, 1234, w.d
+    coords = np.array([[_splitmix64(seed, l * 64 + b) % d for b in range(k)] for l in range(L)])
+    assert all(O.lsh_coordinate(seed, l, b, d) == coords[l, b] for l in range(L) for b in range(k))
+    kp = ((w.P[:, coords] > 0).astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T      # (L, n)
+    kq = ((w.Q[:, coords] > 0).astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T
+    assert np.array_equal(kp, O.lsh_keys(w.P, L, k, seed)) and np.array_equal(kq, O.lsh_keys(w.Q, L, k, seed))
+    collide = (kp[:, :, None] == kq[:, None, :]).any(axis=0)
+    S = w.P.astype(np.int64) @ w.Q.astype(np.int64).T
+    for t in (100.0, 40.0, 24.0):
+        ii, jj = np.nonzero(collide & (S >= t))
+        pairs, cnt = O.lsh_join(w.P, w.Q, t, L, k, seed)
+        assert as_set(pairs) == set(zip(ii.tolist(), jj.tolist())) and cnt == len(ii)
+        exact, _c = O.join(w.P, w.Q, "ip", t, "i8")
+        assert as_set(pairs) <= as_set(exact)                       # precision is 1 by construction
+    # no hash bits: everything collides and the LSH join is the brute-force join
+    all_pairs, _c = O.lsh_join(w.P, w.Q, 40.0, 3, 0, seed)
+    assert as_set(all_pairs) == as_set(O.join(w.P, w.Q, "ip", 40.0, "i8")[0])
+
+
+def test_lsh_recall_matches_the_collision_probability():
+    # planted pairs differ in h = 8 of d = 128 coordinates: one k-bit sample collides with probability close
+    # to (1 - h/d)^k, so the recall over L repetitions is about 1 - (1 - (1-h/d)^k)^L
+    w = W.make_workload(4, n=4000, m=4000, planted=2000)
+    L, k = 4, 8
+    pairs, _c = O.lsh_join(w.P, w.Q, w.threshold, L, k, 99)
+    found = np.isin(O.pairs_to_set(w.planted), O.pairs_to_set(pairs)).mean()
+    p1 = (1 - 8 / 128) ** k
+    expect = 1 - (1 - p1) ** L
+    assert abs(found - expect) < 0.04, (found, expect)
+    with pytest.raises(ValueError):
+        O.lsh_join(w.P, w.Q, 1.0, 0, 4, 1)
+
+
 # ------------------------------------------------- independent formulations
 def _packbits_rows(X):
     return np.packbits(X > 0, axis=1)
