@@ -70,6 +70,13 @@ struct JoinParams {
     unsigned long long *counter;   // total passing pairs
     unsigned int *status;          // 0 = ok, else 0x80000000 | wait site that timed out
     int ioff, joff;          // added to emitted indices
+    // Bucketed mode (the LSH join): the rows of P and Q have been regrouped so that each bucket is a
+    // contiguous row range, and the work list names (P row range, Q row range) units instead of the grid.
+    const int4 *units;             // per unit: first P row, P rows (<= 128), first Q row, Q rows
+    const unsigned int *nunits;    // number of units (written by the kernel that builds the list)
+    const int *perm_p, *perm_q;    // regrouped position -> original row
+    const uint32_t *keys_p, *keys_q;   // [repetition][original row] hash keys, strides n and m
+    int rep;                       // repetitions already joined: a pair whose keys agreed in one of them is not reported again
 };
 
 struct Ctrl {
@@ -86,9 +93,24 @@ static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
 // that fit in L2; within a panel CTAs take whole sweeps in waves of gridDim.x P blocks (all CTAs
 // then walk the panel together, so a Q tile is fetched from HBM once and served from L2 to everyone
 // else, wave after wave); the last, partial wave of a panel splits each of its sweeps over several CTAs.
-struct Unit { int pb, q0, q1; };
+struct Unit {
+    int pb, q0, q1;
+    int prow0, prows, qrow0, qrows;   // bucketed mode only
+};
+template <bool GROUPED>
 __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
     const int G = gridDim.x, c = blockIdx.x;
+    if constexpr (GROUPED) {
+        // units are listed bucket by bucket, so neighbouring CTAs sweep the same Q rows
+        const long long idx = (long long)u * G + c;
+        if (idx >= (long long)__ldg(p.nunits)) return false;
+        const int4 e = __ldg(p.units + idx);
+        un.pb = 0;
+        un.q0 = 0;
+        un.q1 = (e.w + TILE_N - 1) / TILE_N;
+        un.prow0 = e.x; un.prows = e.y; un.qrow0 = e.z; un.qrows = e.w;
+        return true;
+    }
     const int full = p.PB / G, rem = p.PB - full * G;
     const int per_panel = full + (rem > 0 ? 1 : 0);
     const int panel = u / per_panel, v = u - panel * per_panel;
@@ -111,7 +133,9 @@ __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
 #ifndef SIMJOIN_ROTATE
 #define SIMJOIN_ROTATE 1
 #endif
+template <bool GROUPED>
 __device__ __forceinline__ int tile_at(const Unit &un, int k) {
+    if constexpr (GROUPED) return k;
 #if SIMJOIN_ROTATE
     const int len = un.q1 - un.q0;
     int idx = k + (int)((long long)blockIdx.x * len / gridDim.x);
@@ -184,6 +208,12 @@ struct TreeMax<1, MODE> {
 
 // Write `fill` staged pairs of this warp to the output list: one atomic reserves the slots, the
 // stores are coalesced.
+template <bool GROUPED>
+__device__ __forceinline__ int2 final_pair(const JoinParams &p, int2 pr) {
+    if constexpr (GROUPED) return make_int2(__ldg(p.perm_p + pr.x) + p.ioff, __ldg(p.perm_q + pr.y) + p.joff);
+    return pr;
+}
+template <bool GROUPED>
 __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf, int fill, int lane) {
     if (fill == 0) return;
     unsigned long long base = 0;
@@ -192,7 +222,7 @@ __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf
     __syncwarp();
     for (int k = lane; k < fill; k += 32) {
         const unsigned long long slot = base + (unsigned long long)k;
-        if (slot < p.capacity) p.out[slot] = buf[k];
+        if (slot < p.capacity) p.out[slot] = final_pair<GROUPED>(p, buf[k]);
     }
     __syncwarp();
 }
@@ -201,7 +231,7 @@ __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf
 // prefix over the warp, then into the warp's shared-memory staging buffer, which is flushed with
 // one global atomic per ~STAGE_PAIRS pairs.  A block with more hits than the buffer holds goes
 // straight to global memory.  `fill` (warp-uniform) is the number of pairs staged so far.
-template <int NQ>
+template <int NQ, bool GROUPED>
 __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (&mask)[NQ], int lane, long long i, long long j0,
                                            int2 *buf, int &fill) {
     int cnt = 0;
@@ -216,11 +246,12 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     const int total = __shfl_sync(0xffffffffu, incl, 31);
     if (total == 0) return;
     if (fill + total > STAGE_PAIRS) {
-        flush_pairs(p, buf, fill, lane);
+        flush_pairs<GROUPED>(p, buf, fill, lane);
         fill = 0;
     }
-    const int ii = (int)(i + p.ioff);
-    const int jj = (int)(j0 + p.joff);
+    // bucketed mode stages regrouped positions; they become original rows when they leave the CTA
+    const int ii = (int)(i + (GROUPED ? 0 : p.ioff));
+    const int jj = (int)(j0 + (GROUPED ? 0 : p.joff));
     if (total > STAGE_PAIRS) {
         unsigned long long base = 0;
         if (lane == 0) base = atomicAdd(p.counter, (unsigned long long)total);
@@ -232,7 +263,7 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
             while (mk) {
                 const int c = __ffs(mk) - 1;
                 mk &= mk - 1;
-                if (slot < p.capacity) p.out[slot] = make_int2(ii, jj + 32 * q + c);
+                if (slot < p.capacity) p.out[slot] = final_pair<GROUPED>(p, make_int2(ii, jj + 32 * q + c));
                 ++slot;
             }
         }
@@ -252,11 +283,37 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     __syncwarp();
 }
 
+// Bucketed mode, repetition > 0: clear the candidates whose hash keys already agreed in an earlier
+// repetition -- that repetition found and reported them (Section 4's union over repetitions).
+template <int NQ>
+__device__ __forceinline__ void drop_reported(const JoinParams &p, uint32_t (&mask)[NQ], long long i, long long j0) {
+    uint32_t anyb = 0;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) anyb |= mask[q];
+    if (anyb == 0) return;
+    const long long pi = __ldg(p.perm_p + i);
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        uint32_t mk = mask[q], keep = mk;
+        while (mk) {
+            const int c = __ffs(mk) - 1;
+            mk &= mk - 1;
+            const long long qj = __ldg(p.perm_q + (j0 + 32 * q + c));
+            for (int r = 0; r < p.rep; ++r)
+                if (__ldg(p.keys_p + (long long)r * p.n + pi) == __ldg(p.keys_q + (long long)r * p.m + qj)) {
+                    keep &= ~(1u << c);
+                    break;
+                }
+        }
+        mask[q] = keep;
+    }
+}
+
 // The MMA-issuing role (warps 1 and 3).  KC > 0 is a fast path with the chunks per tile known at
 // compile time (resident P block, full 128-byte chunks, two issuers): measured on B200, a chunk loop
 // with a run-time trip count around the tcgen05.mma issues costs ~80 cycles per tile, the run-time
 // operand-address select another ~25.  KC == 0 is the general path.
-template <int DT, int KC>
+template <int DT, int KC, bool GROUPED>
 __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl, uint8_t *smem_p, uint8_t *smem_ring,
                                                 const int stage_bytes_rt, const uint32_t tmem_base, const int warp, const int lane) {
     constexpr bool FAST = KC > 0;
@@ -271,7 +328,7 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
     uint32_t accph0 = 0, accph1 = 0;            // phase of each accumulator's hand-back barrier
     bool ok = true;
     Unit un;
-    for (int u = 0; ok && (dual || mid == 0) && get_unit(p, u, un); ++u) {
+    for (int u = 0; ok && (dual || mid == 0) && get_unit<GROUPED>(p, u, un); ++u) {
         if (un.q1 <= un.q0) continue;
         if (stationary) {
             ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
@@ -345,7 +402,8 @@ __host__ __device__ constexpr int fast_nstages(int kc) {
                ? MAX_STAGES
                : (232448 - 1024 - CTRL_BYTES - STAGING_BYTES - P_BUFS * kc * A_CHUNK_BYTES) / B_CHUNK_BYTES;
 }
-template <int DT, int KIND, bool NARROW = false, int KC = 0>
+// GROUPED: bucketed mode (int8 inner product only) -- see JoinParams::units.
+template <int DT, int KIND, bool NARROW = false, int KC = 0, bool GROUPED = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ, const JoinParams p_in) {
     JoinParams p = p_in;
@@ -397,8 +455,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0;
         bool ok = true;
         Unit un;
-        for (int u = 0; ok && get_unit(p, u, un); ++u) {
+        for (int u = 0; ok && get_unit<GROUPED>(p, u, un); ++u) {
             if (un.q1 <= un.q0) continue;            // nothing for this CTA in this wave (all roles skip it)
+            const int p_row = GROUPED ? un.prow0 : un.pb * TILE_M;
             if (p.stationary) {
                 ok = wait_bar_warp(&ctrl->pempty[pbuf], pphase ^ 1, ctrl, p.status, 1);
                 if (!ok) break;
@@ -407,13 +466,13 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     mbar_arrive_expect_tx(bar, (uint32_t)(p.kc * A_CHUNK_BYTES));
                     for (int c = 0; c < p.kc; ++c)
                         tma_load_2d(smem_u32(smem_p + (size_t)(pbuf * p.kc + c) * A_CHUNK_BYTES), &mapP, bar,
-                                    c * p.elems_per_chunk, un.pb * TILE_M);
+                                    c * p.elems_per_chunk, p_row);
                 }
                 __syncwarp();
                 if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }
             }
             for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
-                const int qt = tile_at(un, k);
+                const int q_row = (GROUPED ? un.qrow0 : 0) + tile_at<GROUPED>(un, k) * TILE_N;
                 for (int c = 0; c < p.kc; ++c) {
                     ok = wait_bar_warp(&ctrl->empty[stage], phase ^ 1, ctrl, p.status, 2);
                     if (!ok) break;
@@ -421,9 +480,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         const uint32_t bar = smem_u32(&ctrl->full[stage]);
                         uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
                         mbar_arrive_expect_tx(bar, (uint32_t)stage_bytes);
-                        tma_load_2d(smem_u32(sb), &mapQ, bar, c * p.elems_per_chunk, qt * TILE_N);
+                        tma_load_2d(smem_u32(sb), &mapQ, bar, c * p.elems_per_chunk, q_row);
                         if (!p.stationary)
-                            tma_load_2d(smem_u32(sb + B_CHUNK_BYTES), &mapP, bar, c * p.elems_per_chunk, un.pb * TILE_M);
+                            tma_load_2d(smem_u32(sb + B_CHUNK_BYTES), &mapP, bar, c * p.elems_per_chunk, p_row);
                     }
                     __syncwarp();
                     if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
@@ -449,9 +508,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         // barrier that is still one phase behind, and a parity wait cannot tell phases two apart.
         // In that case warp 1 issues every tile and warp 3 stays out.
         const bool fast = p.stationary && p.epi_release && p.last_ksteps == 4;
-        if (fast && p.kc == 1) mma_issuer_role<DT, 1>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
-        else if (fast && p.kc == 2) mma_issuer_role<DT, 2>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
-        else mma_issuer_role<DT, 0>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        if (fast && p.kc == 1) mma_issuer_role<DT, 1, GROUPED>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        else if (fast && p.kc == 2) mma_issuer_role<DT, 2, GROUPED>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        else mma_issuer_role<DT, 0, GROUPED>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
     } else if (warp >= EPI_WARP0) {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
@@ -462,10 +521,12 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         int stage_fill = 0;
         bool ok = true;
         Unit un;
-        for (int u = 0; ok && get_unit(p, u, un); ++u) {
+        for (int u = 0; ok && get_unit<GROUPED>(p, u, un); ++u) {
             if (un.q1 <= un.q0) continue;
-            const long long i = (long long)un.pb * TILE_M + row_in_tile;
-            const bool row_ok = i < p.n;
+            const long long i = GROUPED ? (long long)un.prow0 + row_in_tile : (long long)un.pb * TILE_M + row_in_tile;
+            const bool row_ok = GROUPED ? row_in_tile < un.prows : i < p.n;
+            const long long q_base = GROUPED ? un.qrow0 : 0;                          // Q row of tile 0
+            const long long q_end = GROUPED ? (long long)un.qrow0 + un.qrows : p.m;   // end of the Q rows of this unit
             int ri = 0;          // I8/L2: |x|^2 - floor(r^2)
             float rf = 0.f;      // COS: t*|x|;  BF16/L2: |x|^2
             bool rzero = false;  // COS: x is the zero vector
@@ -479,7 +540,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) rf = reinterpret_cast<const float *>(p.nx)[i];
             }
             for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
-                const int qt = tile_at(un, k);
+                const int qt = tile_at<GROUPED>(un, k);
                 // per-tile filter bound: a necessary condition on max_j s_ij for row i to have any hit
                 int fi = p.thr_i;
                 float ff = p.thr_f;
@@ -554,7 +615,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
 #pragma unroll
                     for (int k = 0; k < NG; ++k) gm |= (bound_ok(TreeMax<GW, MODE>::run(v + k * GW)) ? 1u : 0u) << k;
                     if (!row_ok) gm = 0;
-                    const long long j0 = (long long)qt * TILE_N + half * EPI_COLS;
+                    const long long j0 = q_base + (long long)qt * TILE_N + half * EPI_COLS;
                     uint32_t mask[EPI_COLS / 32];
 #pragma unroll
                     for (int q = 0; q < EPI_COLS / 32; ++q) mask[q] = 0;
@@ -563,7 +624,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         if (!__any_sync(0xffffffffu, (gm >> k) & 1u)) continue;
                         // level 2: the exact test on the 16 columns of group k
                         const long long jg = j0 + k * GCOLS;
-                        const long long left = p.m - jg;                       // columns of this group inside Q
+                        const long long left = q_end - jg;                     // columns of this group inside Q (the bucket)
                         const uint32_t valid = left >= GCOLS ? 0xffffu : (left <= 0 ? 0u : ((1u << (int)left) - 1u));
                         uint32_t yw[GCOLS];                                     // per-column term of Q (norm kinds)
                         if constexpr (KIND != KIND_IP) {
@@ -601,13 +662,16 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         if (!((gm >> k) & 1u)) mk = 0;       // the group bound is necessary: nothing can pass here
                         mask[k >> 1] |= mk << ((k & 1) * 16);
                     }
-                    emit_pairs<EPI_COLS / 32>(p, mask, lane, i, j0, stage_buf, stage_fill);
+                    if constexpr (GROUPED) {
+                        if (p.rep > 0) drop_reported<EPI_COLS / 32>(p, mask, i, j0);
+                    }
+                    emit_pairs<EPI_COLS / 32, GROUPED>(p, mask, lane, i, j0, stage_buf, stage_fill);
                 }
                 acc ^= 1;
                 if (acc == 0) accphase ^= 1;
             }
         }
-        if (ok) flush_pairs(p, stage_buf, stage_fill, lane);
+        if (ok) flush_pairs<GROUPED>(p, stage_buf, stage_fill, lane);
     }
 
     tc_fence_before();

@@ -1,0 +1,173 @@
+// Bucketing kernels of the LSH join (Section 4, second algorithm): hash every point L times with a
+// concatenation of k base hashes, and for each repetition regroup the rows of P and Q so that every
+// bucket is one contiguous row range, then list the (P row block, Q bucket) units the join kernel sweeps.
+//
+// Base hash: bit sampling, h(x) = [x_c > 0] for a sampled coordinate c -- the classic monotone family
+// for Hamming distance / +-1 data.  The coordinate of repetition l, bit b is
+// splitmix64(seed, l * 64 + b) mod d, a counter-based generator, so nothing random is stored.
+#pragma once
+#include <cstdint>
+
+namespace sj {
+
+constexpr int LSH_MAX_BITS = 12;                    // buckets per repetition <= 4096 (shared-memory histograms)
+constexpr int LSH_MAX_BUCKETS = 1 << LSH_MAX_BITS;
+constexpr int LSH_MAX_REPS = 64;
+constexpr int LSH_SORT_THREADS = 256;
+constexpr int LSH_SORT_ITEMS = 8;                   // rows per thread in the scatter kernel
+
+__host__ __device__ inline uint64_t lsh_splitmix64(uint64_t seed, uint64_t idx) {
+    uint64_t z = seed + (idx + 1) * 0x9E3779B97F4A7C15ULL;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+
+// keys[l * rows + i] = k-bit key of row i in repetition l.  One thread per row; the L*k sampled
+// coordinates are computed once per block.
+__global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict__ X, long long rows, int d, int L, int k,
+                                                       unsigned long long seed, uint32_t *__restrict__ keys) {
+    __shared__ int s_coord[LSH_MAX_REPS * LSH_MAX_BITS];
+    for (int t = threadIdx.x; t < L * k; t += blockDim.x) {
+        const int l = t / k, b = t - l * k;
+        s_coord[t] = (int)(lsh_splitmix64(seed, (uint64_t)l * 64u + (uint64_t)b) % (uint64_t)d);
+    }
+    __syncthreads();
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows) return;
+    const int8_t *x = X + i * d;
+    for (int l = 0; l < L; ++l) {
+        uint32_t key = 0;
+        for (int b = 0; b < k; ++b) key |= (x[s_coord[l * k + b]] > 0 ? 1u : 0u) << b;
+        keys[(long long)l * rows + i] = key;
+    }
+}
+
+// hist[key] += number of rows with that key (block-private histogram in shared memory first).
+__global__ void __launch_bounds__(LSH_SORT_THREADS) lsh_hist_kernel(const uint32_t *__restrict__ keys, long long rows, int nb,
+                                                                    unsigned int *__restrict__ hist) {
+    __shared__ unsigned int s_cnt[LSH_MAX_BUCKETS];
+    for (int b = threadIdx.x; b < nb; b += blockDim.x) s_cnt[b] = 0;
+    __syncthreads();
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < rows; i += (long long)gridDim.x * blockDim.x)
+        atomicAdd(&s_cnt[keys[i]], 1u);
+    __syncthreads();
+    for (int b = threadIdx.x; b < nb; b += blockDim.x)
+        if (s_cnt[b]) atomicAdd(&hist[b], s_cnt[b]);
+}
+
+// Exclusive scan of up to LSH_MAX_BUCKETS values by one 1024-thread block (4 per thread); returns the total.
+__device__ __forceinline__ unsigned int block_scan4(unsigned int (&v)[4], unsigned int *s_warp) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned int mine = v[0] + v[1] + v[2] + v[3];
+    unsigned int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int t = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += t;
+    }
+    __syncthreads();                         // s_warp may still be read from a previous scan
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const unsigned int w = s_warp[lane];
+        unsigned int wi = w;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned int t = __shfl_up_sync(0xffffffffu, wi, off);
+            if (lane >= off) wi += t;
+        }
+        s_warp[lane] = wi - w;               // exclusive prefix of the warp totals
+        if (lane == 31) s_warp[32] = wi;     // grand total
+    }
+    __syncthreads();
+    unsigned int run = s_warp[warp] + incl - mine;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const unsigned int x = v[t];
+        v[t] = run;
+        run += x;
+    }
+    return s_warp[32];
+}
+
+// One block: bucket offsets of P and Q (exclusive scans of the histograms; also copied to the scatter
+// cursors) and the work list -- for every bucket that holds points of both sets, one unit per 128-row
+// block of its P rows, each against all of the bucket's Q rows.  Units of a bucket are adjacent.
+__global__ void __launch_bounds__(1024) lsh_offsets_units_kernel(const unsigned int *__restrict__ hist_p,
+                                                                 const unsigned int *__restrict__ hist_q, int nb,
+                                                                 unsigned int *__restrict__ cursor_p,
+                                                                 unsigned int *__restrict__ cursor_q, int4 *__restrict__ units,
+                                                                 unsigned int *__restrict__ nunits, int rows_per_unit) {
+    __shared__ unsigned int s_warp[33];
+    unsigned int pc[4], qc[4], po[4], qo[4], ub[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const int b = threadIdx.x * 4 + t;
+        pc[t] = b < nb ? hist_p[b] : 0u;
+        qc[t] = b < nb ? hist_q[b] : 0u;
+        po[t] = pc[t];
+        qo[t] = qc[t];
+        ub[t] = (pc[t] && qc[t]) ? (pc[t] + rows_per_unit - 1) / rows_per_unit : 0u;
+    }
+    block_scan4(po, s_warp);
+    block_scan4(qo, s_warp);
+    const unsigned int total = block_scan4(ub, s_warp);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const int b = threadIdx.x * 4 + t;
+        if (b >= nb) continue;
+        cursor_p[b] = po[t];
+        cursor_q[b] = qo[t];
+        if (pc[t] && qc[t]) {
+            const unsigned int nblk = (pc[t] + rows_per_unit - 1) / rows_per_unit;
+            for (unsigned int j = 0; j < nblk; ++j) {
+                const unsigned int r0 = j * rows_per_unit;
+                const unsigned int rr = pc[t] - r0 < (unsigned)rows_per_unit ? pc[t] - r0 : (unsigned)rows_per_unit;
+                units[ub[t] + j] = make_int4((int)(po[t] + r0), (int)rr, (int)qo[t], (int)qc[t]);
+            }
+        }
+    }
+    if (threadIdx.x == 0) *nunits = total;
+}
+
+// perm[position] = row, positions grouped by key: each block ranks its rows inside shared-memory
+// counters, reserves one range per key with a single global atomic, and writes its rows there.
+__global__ void __launch_bounds__(LSH_SORT_THREADS) lsh_scatter_kernel(const uint32_t *__restrict__ keys, long long rows, int nb,
+                                                                       unsigned int *__restrict__ cursor, int *__restrict__ perm) {
+    __shared__ unsigned int s_cnt[LSH_MAX_BUCKETS];
+    for (int b = threadIdx.x; b < nb; b += blockDim.x) s_cnt[b] = 0;
+    __syncthreads();
+    const long long base = (long long)blockIdx.x * (LSH_SORT_THREADS * LSH_SORT_ITEMS);
+    uint32_t key[LSH_SORT_ITEMS];
+    unsigned int rank[LSH_SORT_ITEMS];
+#pragma unroll
+    for (int t = 0; t < LSH_SORT_ITEMS; ++t) {
+        const long long i = base + t * LSH_SORT_THREADS + threadIdx.x;
+        key[t] = i < rows ? keys[i] : 0u;
+        rank[t] = i < rows ? atomicAdd(&s_cnt[key[t]], 1u) : 0u;
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < nb; b += blockDim.x) {
+        const unsigned int c = s_cnt[b];
+        if (c) s_cnt[b] = atomicAdd(&cursor[b], c);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int t = 0; t < LSH_SORT_ITEMS; ++t) {
+        const long long i = base + t * LSH_SORT_THREADS + threadIdx.x;
+        if (i < rows) perm[s_cnt[key[t]] + rank[t]] = (int)i;
+    }
+}
+
+// out row `pos` = X row perm[pos]; rows are g 16-byte words.
+__global__ void __launch_bounds__(256) lsh_gather_rows_kernel(const uint4 *__restrict__ X, const int *__restrict__ perm,
+                                                              long long rows, int g, uint4 *__restrict__ out) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows * g) return;
+    const long long pos = t / g;
+    const int c = (int)(t - pos * g);
+    out[t] = __ldg(X + (long long)__ldg(perm + pos) * g + c);
+}
+
+}  // namespace sj

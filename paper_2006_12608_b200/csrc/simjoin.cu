@@ -12,6 +12,7 @@
 #include <new>
 
 #include "join_kernel.cuh"
+#include "lsh_kernel.cuh"
 #include "prepass_kernel.cuh"
 
 namespace {
@@ -44,7 +45,9 @@ struct simjoin_ctx {
     bool have_timing;
     float prepass_ms, join_ms;
     long long ioff, joff;
-    bool attr_set[2][3][2][3];
+    bool attr_set[2][3][2][3][2];
+    // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
+    DevBuf lsh_keys_p, lsh_keys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
 };
 
 namespace {
@@ -143,27 +146,29 @@ cudaError_t launch_norms(const simjoin_ctx *ctx, const void *X, int64_t rows, in
     return cudaGetLastError();
 }
 
-template <int DT, int KIND, bool NARROW, int KC>
+template <int DT, int KIND, bool NARROW, int KC, bool GROUPED>
 cudaError_t launch_join_kc(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
                            size_t smem) {
-    auto kern = join_kernel<DT, KIND, NARROW, KC>;
-    if (!ctx->attr_set[DT][KIND][NARROW ? 1 : 0][KC]) {
+    auto kern = join_kernel<DT, KIND, NARROW, KC, GROUPED>;
+    if (!ctx->attr_set[DT][KIND][NARROW ? 1 : 0][KC][GROUPED ? 1 : 0]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
         if (e != cudaSuccess) return e;
-        ctx->attr_set[DT][KIND][NARROW ? 1 : 0][KC] = true;
+        ctx->attr_set[DT][KIND][NARROW ? 1 : 0][KC][GROUPED ? 1 : 0] = true;
     }
     kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
     return cudaGetLastError();
 }
 
 // Picks the instantiation with compile-time chunk count when the run-time parameters match it.
-template <int DT, int KIND, bool NARROW = false>
+template <int DT, int KIND, bool NARROW = false, bool GROUPED = false>
 cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
                         size_t smem) {
     const bool fast = jp.stationary && jp.epi_release && jp.last_ksteps == 4;
-    if (fast && jp.kc == 1 && jp.nstages == fast_nstages(1)) return launch_join_kc<DT, KIND, NARROW, 1>(ctx, mp, mq, jp, grid, smem);
-    if (fast && jp.kc == 2 && jp.nstages == fast_nstages(2)) return launch_join_kc<DT, KIND, NARROW, 2>(ctx, mp, mq, jp, grid, smem);
-    return launch_join_kc<DT, KIND, NARROW, 0>(ctx, mp, mq, jp, grid, smem);
+    if (fast && jp.kc == 1 && jp.nstages == fast_nstages(1))
+        return launch_join_kc<DT, KIND, NARROW, 1, GROUPED>(ctx, mp, mq, jp, grid, smem);
+    if (fast && jp.kc == 2 && jp.nstages == fast_nstages(2))
+        return launch_join_kc<DT, KIND, NARROW, 2, GROUPED>(ctx, mp, mq, jp, grid, smem);
+    return launch_join_kc<DT, KIND, NARROW, 0, GROUPED>(ctx, mp, mq, jp, grid, smem);
 }
 
 // Q tiles per panel.  A Q of up to 64 MiB is swept whole (it mostly stays in L2 and measured faster
@@ -185,17 +190,9 @@ int clamp_to_i32(double v) {
     return (int)v;
 }
 
-// The join on device buffers.  Arguments were validated by the caller.
-simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
-                          simjoin_kind kind, double threshold, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
-    *count = 0;
-    ctx->have_timing = false;
-    if (n == 0 || m == 0) return SIMJOIN_OK;
-    const bool i8 = ctx->dtype == SIMJOIN_I8;
-    const size_t es = elem_size(ctx->dtype);
-    const int row_bytes = (int)(d * es);
-
-    JoinParams jp;
+// Tile geometry of a join over rows of `row_bytes` bytes: chunks per tile, resident-P mode, ring depth,
+// dynamic shared memory.  False when the ring would be too shallow.
+bool tile_geometry(const simjoin_ctx *ctx, int64_t n, int64_t m, int row_bytes, size_t es, JoinParams &jp, size_t &smem) {
     std::memset(&jp, 0, sizeof jp);
     jp.n = n;
     jp.m = m;
@@ -208,10 +205,26 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     const int stage_bytes = B_CHUNK_BYTES + (jp.stationary ? 0 : A_CHUNK_BYTES);
     int nstages = (ctx->max_smem_optin - 1024 - CTRL_BYTES - STAGING_BYTES - p_bytes) / stage_bytes;
     if (nstages > MAX_STAGES) nstages = MAX_STAGES;
-    if (nstages < 2) return SIMJOIN_ERR_UNSUPPORTED;
+    if (nstages < 2) return false;
     jp.nstages = nstages;
     jp.epi_release = (jp.stationary && nstages >= 2 * jp.kc) ? 1 : 0;
-    const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + STAGING_BYTES + CTRL_BYTES;
+    smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + STAGING_BYTES + CTRL_BYTES;
+    return true;
+}
+
+// The join on device buffers.  Arguments were validated by the caller.
+simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
+                          simjoin_kind kind, double threshold, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+    *count = 0;
+    ctx->have_timing = false;
+    if (n == 0 || m == 0) return SIMJOIN_OK;
+    const bool i8 = ctx->dtype == SIMJOIN_I8;
+    const size_t es = elem_size(ctx->dtype);
+    const int row_bytes = (int)(d * es);
+
+    JoinParams jp;
+    size_t smem = 0;
+    if (!tile_geometry(ctx, n, m, row_bytes, es, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
     jp.PB = (int)((n + TILE_M - 1) / TILE_M);
     jp.QT = (int)((m + TILE_N - 1) / TILE_N);
     jp.qpanel = q_panel_tiles(jp.QT, row_bytes);
@@ -370,6 +383,13 @@ simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
     release(ctx->stage_p);
     release(ctx->stage_q);
     release(ctx->stage_out);
+    release(ctx->lsh_keys_p);
+    release(ctx->lsh_keys_q);
+    release(ctx->lsh_perm_p);
+    release(ctx->lsh_perm_q);
+    release(ctx->lsh_sorted_p);
+    release(ctx->lsh_sorted_q);
+    release(ctx->lsh_misc);
     if (ctx->d_ctrl) cudaFree(ctx->d_ctrl);
     if (ctx->h_ctrl) cudaFreeHost(ctx->h_ctrl);
     for (auto &e : ctx->ev)
@@ -461,6 +481,119 @@ simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t
     return run_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, SIMJOIN_IP, t, out_pairs, capacity, count);
 }
 
+simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, double threshold,
+                               int32_t L, int32_t k, uint64_t seed, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+    simjoin_status st = check_join_args(ctx, P, n, Q, m, d, SIMJOIN_IP, threshold, out_pairs, capacity, count);
+    if (st != SIMJOIN_OK) return st;
+    if (ctx->dtype != SIMJOIN_I8) return SIMJOIN_ERR_UNSUPPORTED;
+    if (L < 1 || L > LSH_MAX_REPS || k < 0) return SIMJOIN_ERR_ARG;
+    if (k > LSH_MAX_BITS) return SIMJOIN_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    if ((n > 0 && !is_device_ptr(P, ctx->device)) || (m > 0 && !is_device_ptr(Q, ctx->device))) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && !is_device_ptr(out_pairs, ctx->device)) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
+    *count = 0;
+    ctx->have_timing = false;
+    if (n == 0 || m == 0) return SIMJOIN_OK;
+
+    JoinParams jp;
+    size_t smem = 0;
+    if (!tile_geometry(ctx, n, m, d, 1, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
+    const int nb = 1 << k;
+    const size_t max_units = (size_t)((n + TILE_M - 1) / TILE_M) + (size_t)nb;
+    // misc: hist_p | hist_q | cursor_p | cursor_q (nb words each) | nunits (padded to 16 B) | units
+    const size_t off_units = ((size_t)4 * nb * 4 + 16 + 15) & ~(size_t)15;
+    if (!grow(ctx->lsh_keys_p, (size_t)L * n * 4) || !grow(ctx->lsh_keys_q, (size_t)L * m * 4) ||
+        !grow(ctx->lsh_perm_p, (size_t)n * 4) || !grow(ctx->lsh_perm_q, (size_t)m * 4) ||
+        !grow(ctx->lsh_sorted_p, (size_t)n * d) || !grow(ctx->lsh_sorted_q, (size_t)m * d) ||
+        !grow(ctx->lsh_misc, off_units + max_units * 16))
+        return SIMJOIN_ERR_CUDA;
+    unsigned int *hist_p = reinterpret_cast<unsigned int *>(ctx->lsh_misc.ptr);
+    unsigned int *hist_q = hist_p + nb, *cursor_p = hist_q + nb, *cursor_q = cursor_p + nb, *nunits = cursor_q + nb;
+    int4 *units = reinterpret_cast<int4 *>(reinterpret_cast<unsigned char *>(ctx->lsh_misc.ptr) + off_units);
+    uint32_t *keys_p = reinterpret_cast<uint32_t *>(ctx->lsh_keys_p.ptr), *keys_q = reinterpret_cast<uint32_t *>(ctx->lsh_keys_q.ptr);
+    int *perm_p = reinterpret_cast<int *>(ctx->lsh_perm_p.ptr), *perm_q = reinterpret_cast<int *>(ctx->lsh_perm_q.ptr);
+
+    jp.out = reinterpret_cast<int2 *>(out_pairs);
+    jp.capacity = capacity;
+    jp.counter = ctx->d_ctrl;
+    jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
+    jp.ioff = (int)ctx->ioff;
+    jp.joff = (int)ctx->joff;
+    jp.thr_i = clamp_to_i32(std::ceil(threshold));
+    jp.units = units;
+    jp.nunits = nunits;
+    jp.perm_p = perm_p;
+    jp.perm_q = perm_q;
+    jp.keys_p = keys_p;
+    jp.keys_q = keys_q;
+
+    CUtensorMap mapP, mapQ;
+    if (!encode_rows_map(ctx, &mapP, ctx->lsh_sorted_p.ptr, n, d, TILE_M) ||
+        !encode_rows_map(ctx, &mapQ, ctx->lsh_sorted_q.ptr, m, d, TILE_N))
+        return SIMJOIN_ERR_CUDA;
+
+    cudaStream_t s = ctx->stream;
+    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    // 16-bit epilogue when every score provably fits (as in the brute-force join)
+    unsigned int *d_max = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 2);
+    maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(P), (long long)n * d / 16, d_max);
+    maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(Q), (long long)m * d / 16, d_max + 1);
+    if (cudaGetLastError() != cudaSuccess ||
+        cudaMemcpyAsync(ctx->h_ctrl + 2, ctx->d_ctrl + 2, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    const unsigned int *h_max = reinterpret_cast<const unsigned int *>(ctx->h_ctrl + 2);
+    const bool narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
+
+    cudaEventRecord(ctx->ev[0], s);
+    lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, k, seed, keys_p);
+    lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, k, seed, keys_q);
+    if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    cudaEventRecord(ctx->ev[1], s);
+    const int g = d / 16;
+    const unsigned hist_blocks = (unsigned)ctx->num_sms * 4;
+    const int rows_per_block = LSH_SORT_THREADS * LSH_SORT_ITEMS;
+    for (int l = 0; l < L; ++l) {
+        const uint32_t *kp = keys_p + (size_t)l * n, *kq = keys_q + (size_t)l * m;
+        if (cudaMemsetAsync(hist_p, 0, (size_t)2 * nb * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kp, n, nb, hist_p);
+        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kq, m, nb, hist_q);
+        lsh_offsets_units_kernel<<<1, 1024, 0, s>>>(hist_p, hist_q, nb, cursor_p, cursor_q, units, nunits, TILE_M);
+        lsh_scatter_kernel<<<(unsigned)((n + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kp, n, nb, cursor_p,
+                                                                                                              perm_p);
+        lsh_scatter_kernel<<<(unsigned)((m + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kq, m, nb, cursor_q,
+                                                                                                              perm_q);
+        lsh_gather_rows_kernel<<<(unsigned)(((long long)n * g + 255) / 256), 256, 0, s>>>(
+            reinterpret_cast<const uint4 *>(P), perm_p, n, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_p.ptr));
+        lsh_gather_rows_kernel<<<(unsigned)(((long long)m * g + 255) / 256), 256, 0, s>>>(
+            reinterpret_cast<const uint4 *>(Q), perm_q, m, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_q.ptr));
+        if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        jp.rep = l;
+        const cudaError_t e = narrow ? launch_join<DT_I8, KIND_IP, true, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem)
+                                     : launch_join<DT_I8, KIND_IP, false, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem);
+        if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    }
+    cudaEventRecord(ctx->ev[2], s);
+    if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    if ((unsigned int)(ctx->h_ctrl[1] & 0xffffffffu) != 0) return SIMJOIN_ERR_TIMEOUT;
+    *count = ctx->h_ctrl[0];
+    float a = 0.f, b = 0.f;
+    if (cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess && cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
+        ctx->prepass_ms = a;       // hashing
+        ctx->join_ms = b;          // L x (regroup + bucketed join)
+        ctx->have_timing = true;
+    }
+    return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
+}
+
 simjoin_status simjoin_row_norms(simjoin_ctx *ctx, const void *X, int64_t rows, int32_t d, void *out) {
     if (!ctx || !out) return SIMJOIN_ERR_ARG;
     simjoin_status st = check_matrix_args(ctx, X, rows, d);
@@ -523,7 +656,7 @@ struct NoAllocDevice {
     bool ready;
     unsigned char *scratch;   // device address of g_noalloc_scratch on this device
     int sms, smem_optin;
-    bool attr_set[2][3][2][3];
+    bool attr_set[2][3][2][3][2];
 };
 NoAllocDevice g_na_dev[NA_MAX_DEVICES];
 EncodeTiledFn g_na_encode = nullptr;

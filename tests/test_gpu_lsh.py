@@ -1,0 +1,116 @@
+"""LSH-bucketed inner-product join (Section 4, second algorithm) through the C ABI: hashing, regrouping,
+work list and bucketed tile join all on the device.  The result is a set fixed by (L, k, seed), so it is
+compared with the oracle pair by pair; no pair may be reported twice."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import simjoin_oracle as O
+from paper_2006_12608_b200 import binding as B
+from paper_2006_12608_b200 import build
+from paper_2006_12608_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    build.build()
+    c = B.Simjoin("i8", 0)
+    yield c
+    c.close()
+
+
+def keys(p):
+    p = np.asarray(p, dtype=np.int64).reshape(-1, 2)
+    return np.sort((p[:, 0] << 32) | p[:, 1])
+
+
+def gpu_lsh(ctx, P, Q, t, L, k, seed, cap=1 << 21, expect=B.SIMJOIN_OK):
+    dP, dQ = torch.from_numpy(P).cuda(), torch.from_numpy(Q).cuda()
+    out = torch.full((cap + 2, 2), -5, dtype=torch.int32, device="cuda:0")
+    st, cnt = ctx.simjoin_run_lsh(dP, P.shape[0], dQ, Q.shape[0], P.shape[1], t, L, k, seed, out, cap)
+    assert st == expect, B.strerror(st)
+    host = out.cpu().numpy()
+    assert np.all(host[min(cnt, cap):] == -5)
+    return host[:min(cnt, cap)], cnt
+
+
+def check(ctx, P, Q, t, L, k, seed):
+    pairs, cnt = gpu_lsh(ctx, P, Q, t, L, k, seed)
+    want, wcnt = O.lsh_join(P, Q, t, L, k, seed)
+    got = keys(pairs)
+    assert len(np.unique(got)) == len(got), "a pair was reported twice"
+    assert cnt == wcnt and np.array_equal(got, keys(want)), (P.shape, Q.shape, t, L, k, cnt, wcnt)
+    return cnt
+
+
+@pytest.mark.parametrize("n,m,L,k", [(700, 600, 5, 4), (1, 1, 1, 0), (129, 257, 3, 1), (5000, 7000, 4, 3),
+                                      (3000, 2500, 2, 12), (20000, 30000, 6, 5)])
+def test_lsh_join_matches_oracle(ctx, n, m, L, k):
+    w = W.make_workload(4, n=n, m=m, planted=min(n, m, 300))
+    total = 0
+    for t in (w.threshold, 40.0, 26.0 if n * m < 10**8 else 34.0):
+        total += check(ctx, w.P, w.Q, t, L, k, 1234 + k)
+    assert total > 0 or min(n, m) == 1
+
+
+def test_no_hash_bits_is_the_brute_force_join(ctx):
+    w = W.make_workload(4, n=3000, m=4100, planted=200)
+    pairs, cnt = gpu_lsh(ctx, w.P, w.Q, 30.0, 3, 0, 7)
+    want, wcnt = O.join(w.P, w.Q, "ip", 30.0, "i8")
+    assert cnt == wcnt and np.array_equal(keys(pairs), keys(want))
+
+
+@pytest.mark.parametrize("d", [64, 256, 384, 1024])
+def test_lsh_row_lengths(ctx, d):
+    # 64: partial chunk; 256: two-chunk fast path; 384: three chunks; 1024: streamed P
+    P = W.random_points("i8", 2100, d, 11, lo=-1, hi=1)
+    Q = W.random_points("i8", 2600, d, 12, lo=-1, hi=1)
+    Q[:100] = P[:100]
+    check(ctx, P, Q, 0.25 * d, 4, 3, 99)
+
+
+def test_lsh_wide_values_use_the_32_bit_epilogue(ctx):
+    P = W.random_points("i8", 1500, 128, 21, lo=-127, hi=127)
+    Q = W.random_points("i8", 1700, 128, 22, lo=-127, hi=127)
+    Q[:64] = P[:64]
+    assert check(ctx, P, Q, 150000.0, 4, 4, 5) >= 1
+
+
+def test_lsh_recall_on_planted_pairs(ctx):
+    # planted pairs differ in 8 of 128 coordinates; 8 repetitions of 6 bits miss one with probability ~1e-4
+    w = W.make_workload(4, n=40000, m=40000, planted=4000)
+    pairs, cnt = gpu_lsh(ctx, w.P, w.Q, w.threshold, 8, 6, 3)
+    found = np.isin(keys(w.planted), keys(pairs)).mean()
+    assert found > 0.995, found
+    exact, _ = O.join(w.P, w.Q, "ip", w.threshold, "i8")
+    assert np.isin(keys(pairs), keys(exact)).all()
+
+
+def test_lsh_offsets_capacity_and_errors(ctx):
+    w = W.make_workload(4, n=2000, m=2000, planted=300)
+    dP, dQ = torch.from_numpy(w.P).cuda(), torch.from_numpy(w.Q).cuda()
+    want, wcnt = O.lsh_join(w.P, w.Q, w.threshold, 4, 3, 17)
+    assert wcnt > 50
+    assert ctx.simjoin_set_offsets(1000, 50000) == B.SIMJOIN_OK
+    try:
+        pairs, cnt = gpu_lsh(ctx, w.P, w.Q, w.threshold, 4, 3, 17)
+    finally:
+        ctx.simjoin_set_offsets(0, 0)
+    assert np.array_equal(keys(pairs), keys(want + np.array([1000, 50000])))
+    # too small an output list: the count is still the full one, only `capacity` pairs are written
+    pairs, cnt = gpu_lsh(ctx, w.P, w.Q, w.threshold, 4, 3, 17, cap=20, expect=B.SIMJOIN_ERR_CAPACITY)
+    assert cnt == wcnt and np.isin(keys(pairs), keys(want)).all() and len(pairs) == 20
+    out = torch.zeros((8, 2), dtype=torch.int32, device="cuda:0")
+    args = (dP, 2000, dQ, 2000, 128, 100.0)
+    assert ctx.simjoin_run_lsh(*args, 0, 3, 1, out, 8)[0] == B.SIMJOIN_ERR_ARG
+    assert ctx.simjoin_run_lsh(*args, 65, 3, 1, out, 8)[0] == B.SIMJOIN_ERR_ARG
+    assert ctx.simjoin_run_lsh(*args, 2, -1, 1, out, 8)[0] == B.SIMJOIN_ERR_ARG
+    assert ctx.simjoin_run_lsh(*args, 2, 13, 1, out, 8)[0] == B.SIMJOIN_ERR_UNSUPPORTED
+    assert ctx.simjoin_run_lsh(dP, 0, dQ, 2000, 128, 100.0, 2, 3, 1, out, 8) == (B.SIMJOIN_OK, 0)
+    with B.Simjoin("bf16", 0) as cb:
+        assert cb.simjoin_run_lsh(*args, 2, 3, 1, out, 8)[0] == B.SIMJOIN_ERR_UNSUPPORTED
+    # the plain join still works on the same context afterwards
+    got, cnt = ctx.join(dP, dQ, "ip", w.threshold, 1 << 16)
+    assert cnt == O.join(w.P, w.Q, "ip", w.threshold, "i8")[1]
