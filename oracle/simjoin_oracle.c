@@ -279,7 +279,10 @@ int64_t oracle_join_hamming_bits(const uint8_t *P, int64_t n, const uint8_t *Q, 
  * one repetition } -- which is what this oracle enumerates, with no buckets at all.
  * Base hash (bit sampling, the classic monotone LSH for Hamming / +-1 data): h(x) = [x_c > 0] for a
  * sampled coordinate c.  Coordinate of repetition l, bit b: splitmix64(seed, l*64 + b) mod d -- a
- * counter-based generator that the CUDA library implements on its own. */
+ * counter-based generator that the CUDA library implements on its own.
+ * When the number of base hashes the analysis asks for is not an integer, the paper builds L_high
+ * tables from ceil(k) base hashes and L_low tables from floor(k): here the first L_high repetitions
+ * use k bits and the following L_low use k - 1. */
 static uint64_t splitmix64_at(uint64_t seed, uint64_t idx) {
     uint64_t z = seed + (idx + 1) * 0x9E3779B97F4A7C15ULL;
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
@@ -291,20 +294,27 @@ int32_t oracle_lsh_coordinate(uint64_t seed, int32_t rep, int32_t bit, int32_t d
     return (int32_t)(splitmix64_at(seed, (uint64_t)rep * 64u + (uint64_t)bit) % (uint64_t)d);
 }
 
-/* keys[l * rows + i] = the k-bit hash of row i in repetition l (bit b = [x_{c(l,b)} > 0]). */
-void oracle_lsh_keys_i8(const int8_t *X, int64_t rows, int32_t d, int32_t L, int32_t k, uint64_t seed, uint32_t *keys) {
-    for (int32_t l = 0; l < L; ++l)
+/* keys[l * rows + i] = the hash of row i in repetition l (bit b = [x_{c(l,b)} > 0]); k bits in the
+ * first L_high repetitions, k - 1 in the next L_low. */
+void oracle_lsh_keys_i8(const int8_t *X, int64_t rows, int32_t d, int32_t L_high, int32_t L_low, int32_t k, uint64_t seed,
+                        uint32_t *keys) {
+    for (int32_t l = 0; l < L_high + L_low; ++l)
         for (int64_t i = 0; i < rows; ++i) {
             uint32_t key = 0;
-            for (int32_t b = 0; b < k; ++b)
+            const int32_t bits = l < L_high ? k : k - 1;
+            for (int32_t b = 0; b < bits; ++b)
                 if (X[(size_t)i * d + oracle_lsh_coordinate(seed, l, b, d)] > 0) key |= 1u << b;
             keys[(size_t)l * rows + i] = key;
         }
 }
 
 int64_t oracle_lsh_join_i8(const int8_t *P, int64_t n, const int8_t *Q, int64_t m, int32_t d, double threshold,
-                           int32_t L, int32_t k, uint64_t seed, int32_t *out_pairs, int64_t capacity, int32_t nthreads) {
-    if (n < 0 || m < 0 || d <= 0 || capacity < 0 || isnan(threshold) || L < 1 || L > 64 || k < 0 || k > 20) return -1;
+                           int32_t L_high, int32_t L_low, int32_t k, uint64_t seed, int32_t *out_pairs, int64_t capacity,
+                           int32_t nthreads) {
+    const int32_t L = L_high + L_low;
+    if (n < 0 || m < 0 || d <= 0 || capacity < 0 || isnan(threshold) || L_high < 0 || L_low < 0 || L < 1 || L > 64 || k < 0 ||
+        k > 20 || (L_low > 0 && k < 1))
+        return -1;
     if (n >= INT32_MAX || m >= INT32_MAX) return -1;
     int nt = resolve_threads(nthreads);
     uint32_t *KP = (uint32_t *)malloc(((size_t)L * n + 1) * sizeof(uint32_t));
@@ -313,8 +323,8 @@ int64_t oracle_lsh_join_i8(const int8_t *P, int64_t n, const int8_t *Q, int64_t 
     pairbuf *blk = (pairbuf *)calloc((size_t)nb, sizeof(pairbuf));
     int64_t total = -1;
     if (KP && KQ && blk) {
-        oracle_lsh_keys_i8(P, n, d, L, k, seed, KP);
-        oracle_lsh_keys_i8(Q, m, d, L, k, seed, KQ);
+        oracle_lsh_keys_i8(P, n, d, L_high, L_low, k, seed, KP);
+        oracle_lsh_keys_i8(Q, m, d, L_high, L_low, k, seed, KQ);
 #pragma omp parallel for schedule(dynamic, 1) num_threads(nt)
         for (int64_t b = 0; b < nb; ++b) {
             int64_t i0 = n * b / nb, i1 = n * (b + 1) / nb;

@@ -71,9 +71,9 @@ def _load():
     lib.oracle_hamming_bits.restype = i64
     lib.oracle_hamming_bits.argtypes = [vp, vp, i32]
     lib.oracle_lsh_join_i8.restype = i64
-    lib.oracle_lsh_join_i8.argtypes = [vp, i64, vp, i64, i32, dbl, i32, i32, c.c_uint64, vp, i64, i32]
+    lib.oracle_lsh_join_i8.argtypes = [vp, i64, vp, i64, i32, dbl, i32, i32, i32, c.c_uint64, vp, i64, i32]
     lib.oracle_lsh_keys_i8.restype = None
-    lib.oracle_lsh_keys_i8.argtypes = [vp, i64, i32, i32, i32, c.c_uint64, vp]
+    lib.oracle_lsh_keys_i8.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, vp]
     lib.oracle_lsh_coordinate.restype = i32
     lib.oracle_lsh_coordinate.argtypes = [c.c_uint64, i32, i32, i32]
     lib.oracle_scores_i8.restype = i32
@@ -156,9 +156,10 @@ def hamming(x: np.ndarray, y: np.ndarray, d: int) -> int:
     return int(_load().oracle_hamming_bits(x.ctypes.data, y.ctypes.data, d))
 
 
-def lsh_join(P: np.ndarray, Q: np.ndarray, threshold: float, L: int, k: int, seed: int, threads: int = 0):
+def lsh_join(P: np.ndarray, Q: np.ndarray, threshold: float, L: int, k: int, seed: int, threads: int = 0, L_low: int = 0):
     """The LSH-bucketed inner-product join over int8 rows with bit-sampling hashes: all (i, j) of the
-    brute-force join whose k-bit hashes agree in at least one of L repetitions.  Returns (pairs, count)."""
+    brute-force join whose hashes agree in at least one repetition -- L repetitions of k bits followed by
+    L_low repetitions of k - 1 bits.  Returns (pairs, count)."""
     lib = _load()
     P, Q = _check(P, "i8"), _check(Q, "i8")
     n, d = P.shape
@@ -166,7 +167,7 @@ def lsh_join(P: np.ndarray, Q: np.ndarray, threshold: float, L: int, k: int, see
     cap = 1 << 16
     while True:
         out = np.empty((cap, 2), dtype=np.int32)
-        cnt = lib.oracle_lsh_join_i8(P.ctypes.data, n, Q.ctypes.data, m, d, float(threshold), L, k, seed,
+        cnt = lib.oracle_lsh_join_i8(P.ctypes.data, n, Q.ctypes.data, m, d, float(threshold), L, L_low, k, seed,
                                      out.ctypes.data, cap, threads)
         if cnt < 0:
             raise ValueError("oracle rejected the arguments")
@@ -175,12 +176,12 @@ def lsh_join(P: np.ndarray, Q: np.ndarray, threshold: float, L: int, k: int, see
         cap = int(cnt)
 
 
-def lsh_keys(X: np.ndarray, L: int, k: int, seed: int) -> np.ndarray:
-    """(L, rows) uint32 hash keys of int8 rows."""
+def lsh_keys(X: np.ndarray, L: int, k: int, seed: int, L_low: int = 0) -> np.ndarray:
+    """(L + L_low, rows) uint32 hash keys of int8 rows."""
     lib = _load()
     X = _check(X, "i8")
-    out = np.empty((L, X.shape[0]), dtype=np.uint32)
-    lib.oracle_lsh_keys_i8(X.ctypes.data, X.shape[0], X.shape[1], L, k, seed, out.ctypes.data)
+    out = np.empty((L + L_low, X.shape[0]), dtype=np.uint32)
+    lib.oracle_lsh_keys_i8(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, out.ctypes.data)
     return out
 
 

@@ -112,6 +112,13 @@ def test_lsh_join_is_brute_force_restricted_to_colliding_pairs():
         assert as_set(pairs) == set(zip(ii.tolist(), jj.tolist())) and cnt == len(ii)
         exact, _c = O.join(w.P, w.Q, "ip", t, "i8")
         assert as_set(pairs) <= as_set(exact)                       # precision is 1 by construction
+    # mixed tables: 3 repetitions of k bits, then 2 of k - 1 bits (the low bits of the same samples)
+    kmix = np.concatenate([kp[:3], kp[3:] & ((1 << (k - 1)) - 1)]), np.concatenate([kq[:3], kq[3:] & ((1 << (k - 1)) - 1)])
+    assert np.array_equal(kmix[0], O.lsh_keys(w.P, 3, k, seed, L_low=2))
+    cmix = (kmix[0][:, :, None] == kmix[1][:, None, :]).any(axis=0)
+    ii, jj = np.nonzero(cmix & (S >= 40.0))
+    pairs, cnt = O.lsh_join(w.P, w.Q, 40.0, 3, k, seed, L_low=2)
+    assert as_set(pairs) == set(zip(ii.tolist(), jj.tolist())) and cnt == len(ii)
     # no hash bits: everything collides and the LSH join is the brute-force join
     all_pairs, _c = O.lsh_join(w.P, w.Q, 40.0, 3, 0, seed)
     assert as_set(all_pairs) == as_set(O.join(w.P, w.Q, "ip", 40.0, "i8")[0])
@@ -129,6 +136,8 @@ def test_lsh_recall_matches_the_collision_probability():
     assert abs(found - expect) < 0.04, (found, expect)
     with pytest.raises(ValueError):
         O.lsh_join(w.P, w.Q, 1.0, 0, 4, 1)
+    with pytest.raises(ValueError):
+        O.lsh_join(w.P, w.Q, 1.0, 1, 0, 1, L_low=1)          # k - 1 bits needs k >= 1
 
 
 # ------------------------------------------------- independent formulations
