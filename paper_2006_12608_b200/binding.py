@@ -55,7 +55,7 @@ def load() -> ctypes.CDLL:
     lib.simjoin_run_hamming.restype = c.c_int
     lib.simjoin_run_hamming.argtypes = [vp, vp, i64, vp, i64, i32, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_run_lsh.restype = c.c_int
-    lib.simjoin_run_lsh.argtypes = [vp, vp, i64, vp, i64, i32, dbl, i32, i32, u64, vp, u64, c.POINTER(u64)]
+    lib.simjoin_run_lsh.argtypes = [vp, vp, i64, vp, i64, i32, dbl, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
     lib.simjoin_run_noalloc.restype = c.c_int
     lib.simjoin_run_noalloc.argtypes = [c.c_int, vp, c.c_int, vp, i64, vp, i64, i32, c.c_int, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_row_norms.restype = c.c_int
@@ -140,10 +140,10 @@ class Simjoin:
         st = load().simjoin_run_hamming(self._h, pp, n, qp, m, d, float(r), op, capacity, ctypes.byref(cnt))
         return st, cnt.value
 
-    def simjoin_run_lsh(self, P, n, Q, m, d, threshold, L, k, seed, out_pairs, capacity):
+    def simjoin_run_lsh(self, P, n, Q, m, d, threshold, L, k, seed, out_pairs, capacity, L_low=0):
         cnt = ctypes.c_uint64(0)
         (pp, _a), (qp, _b), (op, _c) = _ptr(P), _ptr(Q), _ptr(out_pairs)
-        st = load().simjoin_run_lsh(self._h, pp, n, qp, m, d, float(threshold), int(L), int(k), int(seed), op, capacity,
+        st = load().simjoin_run_lsh(self._h, pp, n, qp, m, d, float(threshold), int(L), int(L_low), int(k), int(seed), op, capacity,
                                     ctypes.byref(cnt))
         return st, cnt.value
 

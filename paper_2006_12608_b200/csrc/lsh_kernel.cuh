@@ -23,11 +23,13 @@ __host__ __device__ inline uint64_t lsh_splitmix64(uint64_t seed, uint64_t idx) 
     return z ^ (z >> 31);
 }
 
-// keys[l * rows + i] = k-bit key of row i in repetition l.  One thread per row; the L*k sampled
-// coordinates are computed once per block.
-__global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict__ X, long long rows, int d, int L, int k,
-                                                       unsigned long long seed, uint32_t *__restrict__ keys) {
+// keys[l * rows + i] = key of row i in repetition l: k bits in the first L_high repetitions, k - 1 (the
+// same samples without the last) in the following L_low -- the paper's mix of tables for a fractional
+// number of base hashes.  One thread per row; the sampled coordinates are computed once per block.
+__global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict__ X, long long rows, int d, int L_high, int L_low,
+                                                       int k, unsigned long long seed, uint32_t *__restrict__ keys) {
     __shared__ int s_coord[LSH_MAX_REPS * LSH_MAX_BITS];
+    const int L = L_high + L_low;
     for (int t = threadIdx.x; t < L * k; t += blockDim.x) {
         const int l = t / k, b = t - l * k;
         s_coord[t] = (int)(lsh_splitmix64(seed, (uint64_t)l * 64u + (uint64_t)b) % (uint64_t)d);
@@ -38,7 +40,8 @@ __global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict_
     const int8_t *x = X + i * d;
     for (int l = 0; l < L; ++l) {
         uint32_t key = 0;
-        for (int b = 0; b < k; ++b) key |= (x[s_coord[l * k + b]] > 0 ? 1u : 0u) << b;
+        const int bits = l < L_high ? k : k - 1;
+        for (int b = 0; b < bits; ++b) key |= (x[s_coord[l * k + b]] > 0 ? 1u : 0u) << b;
         keys[(long long)l * rows + i] = key;
     }
 }

@@ -482,11 +482,12 @@ simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t
 }
 
 simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, double threshold,
-                               int32_t L, int32_t k, uint64_t seed, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+                               int32_t L, int32_t L_low, int32_t k, uint64_t seed, int32_t *out_pairs, uint64_t capacity,
+                               uint64_t *count) {
     simjoin_status st = check_join_args(ctx, P, n, Q, m, d, SIMJOIN_IP, threshold, out_pairs, capacity, count);
     if (st != SIMJOIN_OK) return st;
     if (ctx->dtype != SIMJOIN_I8) return SIMJOIN_ERR_UNSUPPORTED;
-    if (L < 1 || L > LSH_MAX_REPS || k < 0) return SIMJOIN_ERR_ARG;
+    if (L < 0 || L_low < 0 || L + L_low < 1 || L + L_low > LSH_MAX_REPS || k < 0 || (L_low > 0 && k < 1)) return SIMJOIN_ERR_ARG;
     if (k > LSH_MAX_BITS) return SIMJOIN_ERR_UNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SIMJOIN_ERR_CUDA;
@@ -500,17 +501,18 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     JoinParams jp;
     size_t smem = 0;
     if (!tile_geometry(ctx, n, m, d, 1, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
-    const int nb = 1 << k;
-    const size_t max_units = (size_t)((n + TILE_M - 1) / TILE_M) + (size_t)nb;
+    const int nb_max = 1 << k;
+    const size_t max_units = (size_t)((n + TILE_M - 1) / TILE_M) + (size_t)nb_max;
     // misc: hist_p | hist_q | cursor_p | cursor_q (nb words each) | nunits (padded to 16 B) | units
-    const size_t off_units = ((size_t)4 * nb * 4 + 16 + 15) & ~(size_t)15;
-    if (!grow(ctx->lsh_keys_p, (size_t)L * n * 4) || !grow(ctx->lsh_keys_q, (size_t)L * m * 4) ||
+    const size_t off_units = ((size_t)4 * nb_max * 4 + 16 + 15) & ~(size_t)15;
+    const int reps = L + L_low;
+    if (!grow(ctx->lsh_keys_p, (size_t)reps * n * 4) || !grow(ctx->lsh_keys_q, (size_t)reps * m * 4) ||
         !grow(ctx->lsh_perm_p, (size_t)n * 4) || !grow(ctx->lsh_perm_q, (size_t)m * 4) ||
         !grow(ctx->lsh_sorted_p, (size_t)n * d) || !grow(ctx->lsh_sorted_q, (size_t)m * d) ||
         !grow(ctx->lsh_misc, off_units + max_units * 16))
         return SIMJOIN_ERR_CUDA;
     unsigned int *hist_p = reinterpret_cast<unsigned int *>(ctx->lsh_misc.ptr);
-    unsigned int *hist_q = hist_p + nb, *cursor_p = hist_q + nb, *cursor_q = cursor_p + nb, *nunits = cursor_q + nb;
+    unsigned int *hist_q = hist_p + nb_max, *cursor_p = hist_q + nb_max, *cursor_q = cursor_p + nb_max, *nunits = cursor_q + nb_max;
     int4 *units = reinterpret_cast<int4 *>(reinterpret_cast<unsigned char *>(ctx->lsh_misc.ptr) + off_units);
     uint32_t *keys_p = reinterpret_cast<uint32_t *>(ctx->lsh_keys_p.ptr), *keys_q = reinterpret_cast<uint32_t *>(ctx->lsh_keys_q.ptr);
     int *perm_p = reinterpret_cast<int *>(ctx->lsh_perm_p.ptr), *perm_q = reinterpret_cast<int *>(ctx->lsh_perm_q.ptr);
@@ -550,16 +552,17 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     const bool narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
 
     cudaEventRecord(ctx->ev[0], s);
-    lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, k, seed, keys_p);
-    lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, k, seed, keys_q);
+    lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p);
+    lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q);
     if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
     cudaEventRecord(ctx->ev[1], s);
     const int g = d / 16;
     const unsigned hist_blocks = (unsigned)ctx->num_sms * 4;
     const int rows_per_block = LSH_SORT_THREADS * LSH_SORT_ITEMS;
-    for (int l = 0; l < L; ++l) {
+    for (int l = 0; l < reps; ++l) {
         const uint32_t *kp = keys_p + (size_t)l * n, *kq = keys_q + (size_t)l * m;
-        if (cudaMemsetAsync(hist_p, 0, (size_t)2 * nb * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        const int nb = l < L ? nb_max : nb_max / 2;          // buckets of this repetition
+        if (cudaMemsetAsync(hist_p, 0, (size_t)2 * nb_max * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
         lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kp, n, nb, hist_p);
         lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kq, m, nb, hist_q);
         lsh_offsets_units_kernel<<<1, 1024, 0, s>>>(hist_p, hist_q, nb, cursor_p, cursor_q, units, nunits, TILE_M);

@@ -26,19 +26,19 @@ def keys(p):
     return np.sort((p[:, 0] << 32) | p[:, 1])
 
 
-def gpu_lsh(ctx, P, Q, t, L, k, seed, cap=1 << 21, expect=B.SIMJOIN_OK):
+def gpu_lsh(ctx, P, Q, t, L, k, seed, cap=1 << 21, expect=B.SIMJOIN_OK, L_low=0):
     dP, dQ = torch.from_numpy(P).cuda(), torch.from_numpy(Q).cuda()
     out = torch.full((cap + 2, 2), -5, dtype=torch.int32, device="cuda:0")
-    st, cnt = ctx.simjoin_run_lsh(dP, P.shape[0], dQ, Q.shape[0], P.shape[1], t, L, k, seed, out, cap)
+    st, cnt = ctx.simjoin_run_lsh(dP, P.shape[0], dQ, Q.shape[0], P.shape[1], t, L, k, seed, out, cap, L_low=L_low)
     assert st == expect, B.strerror(st)
     host = out.cpu().numpy()
     assert np.all(host[min(cnt, cap):] == -5)
     return host[:min(cnt, cap)], cnt
 
 
-def check(ctx, P, Q, t, L, k, seed):
-    pairs, cnt = gpu_lsh(ctx, P, Q, t, L, k, seed)
-    want, wcnt = O.lsh_join(P, Q, t, L, k, seed)
+def check(ctx, P, Q, t, L, k, seed, L_low=0):
+    pairs, cnt = gpu_lsh(ctx, P, Q, t, L, k, seed, L_low=L_low)
+    want, wcnt = O.lsh_join(P, Q, t, L, k, seed, L_low=L_low)
     got = keys(pairs)
     assert len(np.unique(got)) == len(got), "a pair was reported twice"
     assert cnt == wcnt and np.array_equal(got, keys(want)), (P.shape, Q.shape, t, L, k, cnt, wcnt)
@@ -53,6 +53,14 @@ def test_lsh_join_matches_oracle(ctx, n, m, L, k):
     for t in (w.threshold, 40.0, 26.0 if n * m < 10**8 else 34.0):
         total += check(ctx, w.P, w.Q, t, L, k, 1234 + k)
     assert total > 0 or min(n, m) == 1
+
+
+@pytest.mark.parametrize("L,L_low,k", [(3, 2, 4), (0, 4, 3), (2, 3, 1), (1, 1, 12)])
+def test_lsh_mixed_tables(ctx, L, L_low, k):
+    # the paper's remedy for a fractional number of base hashes: L tables of k bits, L_low of k - 1
+    w = W.make_workload(4, n=4000, m=5000, planted=300)
+    for t in (w.threshold, 36.0):
+        assert check(ctx, w.P, w.Q, t, L, k, 77, L_low=L_low) > 0
 
 
 def test_no_hash_bits_is_the_brute_force_join(ctx):
@@ -108,6 +116,8 @@ def test_lsh_offsets_capacity_and_errors(ctx):
     assert ctx.simjoin_run_lsh(*args, 65, 3, 1, out, 8)[0] == B.SIMJOIN_ERR_ARG
     assert ctx.simjoin_run_lsh(*args, 2, -1, 1, out, 8)[0] == B.SIMJOIN_ERR_ARG
     assert ctx.simjoin_run_lsh(*args, 2, 13, 1, out, 8)[0] == B.SIMJOIN_ERR_UNSUPPORTED
+    assert ctx.simjoin_run_lsh(*args, 2, 0, 1, out, 8, L_low=1)[0] == B.SIMJOIN_ERR_ARG          # k - 1 bits needs k >= 1
+    assert ctx.simjoin_run_lsh(*args, 60, 3, 1, out, 8, L_low=5)[0] == B.SIMJOIN_ERR_ARG
     assert ctx.simjoin_run_lsh(dP, 0, dQ, 2000, 128, 100.0, 2, 3, 1, out, 8) == (B.SIMJOIN_OK, 0)
     with B.Simjoin("bf16", 0) as cb:
         assert cb.simjoin_run_lsh(*args, 2, 3, 1, out, 8)[0] == B.SIMJOIN_ERR_UNSUPPORTED
