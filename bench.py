@@ -182,7 +182,13 @@ def main():
     ap.add_argument("--m", type=int, default=None, help="override the row count of Q")
     ap.add_argument("--planted", type=int, default=None)
     ap.add_argument("--sigma-reading", default="radial")
+    ap.add_argument("--lsh", default=None, metavar="L,k[,L_low]",
+                    help="time the LSH-bucketed join (int8 inner-product configs) instead of the brute-force join: "
+                         "L tables of k bits (+ L_low of k-1); not the headline metric, the line says so")
     args = ap.parse_args()
+    args.lsh = tuple(int(x) for x in args.lsh.split(",")) if args.lsh else None
+    if args.lsh and args.impl == "reference":
+        raise SystemExit("--lsh times the CUDA path only")
     if args.warmup < 3:
         args.warmup = 3
 
@@ -227,8 +233,16 @@ def main():
     ctx = B.Simjoin(w.dtype, local_rank)
     ctx.simjoin_set_offsets(rank * w.n, 0)
 
+    if args.lsh and (w.dtype != "i8" or w.kind != "ip"):
+        raise SystemExit("--lsh needs an int8 inner-product configuration (1, 3, 4)")
+
     def step():
-        st, cnt = ctx.simjoin_run(dP, w.n, dQ, w.m, w.d, w.kind, w.threshold, out, capacity)
+        if args.lsh:
+            L, k = args.lsh[0], args.lsh[1]
+            st, cnt = ctx.simjoin_run_lsh(dP, w.n, dQ, w.m, w.d, w.threshold, L, k, 2006, out, capacity,
+                                          L_low=args.lsh[2] if len(args.lsh) > 2 else 0)
+        else:
+            st, cnt = ctx.simjoin_run(dP, w.n, dQ, w.m, w.d, w.kind, w.threshold, out, capacity)
         if st != B.SIMJOIN_OK:
             raise RuntimeError(f"simjoin_run: {B.strerror(st)}")
         return cnt
@@ -249,9 +263,13 @@ def main():
         assert len(np.unique(keys)) == cnt, "duplicate pairs in the join output"
     if w.labels_p is not None and cnt:
         assert np.all(w.labels_p[got[:, 0] - rank * w.n] == w.labels_q[got[:, 1]]), "pair across clusters"
+    args.recall = None
     if len(w.planted):
         pk = ((w.planted[:, 0] + rank * w.n) << 32) | w.planted[:, 1]
-        assert np.isin(pk, keys).all(), "a planted pair is missing from the join output"
+        if args.lsh:
+            args.recall = float(np.isin(pk, keys).mean())       # the LSH join is approximate by design
+        else:
+            assert np.isin(pk, keys).all(), "a planted pair is missing from the join output"
     if same_cluster is not None:
         assert cnt == same_cluster, (cnt, same_cluster)
 
@@ -278,7 +296,7 @@ def main():
     value = world * w.ops / (ms_per_step * 1e-3) / 1e12
 
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.lsh:
         e2e = measure_e2e(args, ctx, w, capacity, cnt, world, dev, sync_all)
 
     if rank != 0:
@@ -342,6 +360,12 @@ def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks
                 "frac_of_nominal": achieved / NOMINAL_TOPS[w.dtype], "kernel_ms": jm,
                 "prepass_ms": statistics.mean(pre_ms)}
     launches_per_step = 1 + (2 if w.kind != "ip" else 0) + (2 if w.dtype == "i8" else 0)   # join + norms + max|x|
+    if args.lsh:
+        # max|x| x2, keys x2, then per table: 2 histograms, offsets + work list, 2 scatters, 2 row gathers, the join,
+        # and from the second table on 2 gathers of the key records
+        tables = args.lsh[0] + (args.lsh[2] if len(args.lsh) > 2 else 0)
+        launches_per_step = 4 + 8 * tables + 2 * (tables - 1)
+        roofline = None
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32" if w.dtype == "i8" else "f32", "data": "synthetic",
@@ -353,7 +377,13 @@ def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks
             "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline}
-    if not args.no_cpu_baseline and world == 1:
+    if args.lsh:
+        line["algorithm"] = {"name": "lsh-bucketed join (simjoin_run_lsh)", "L": args.lsh[0], "k": args.lsh[1],
+                             "L_low": args.lsh[2] if len(args.lsh) > 2 else 0, "recall_on_planted_pairs": args.recall,
+                             "hash_ms": statistics.mean(pre_ms), "tables_ms": jm,
+                             "note": "value = 2*n*m*d over the step time: the brute-force-equivalent rate of an approximate "
+                                     "join, not the headline metric; precision is 1, recall as given"}
+    if not args.no_cpu_baseline and world == 1 and not args.lsh:
         rows = slab_rows_for(w, 12.0)
         dt, _c, threads = oracle_slab(w, rows)
         line["cpu_baseline"] = {"value": 2.0 * rows * w.m * w.d / dt / 1e12, "unit": UNIT, "cores": threads,

@@ -37,6 +37,10 @@ constexpr int MAX_STATIONARY_CHUNKS = 4;          // P block kept resident up to
 #define SIMJOIN_P_BUFS 1
 #endif
 constexpr int P_BUFS = SIMJOIN_P_BUFS;            // resident P blocks: 1 (a short bubble per Q sweep) or 2
+// Bucketed mode sweeps only a bucket's Q rows per P block (tens of tiles, not thousands): there the bubble
+// matters, and the next P block is fetched while the current one is still being multiplied (rows of up to
+// two chunks; longer rows would pay for the second block with ring depth).
+__host__ __device__ constexpr int p_bufs(bool grouped, int kc) { return grouped && kc <= 2 ? 2 : P_BUFS; }
 constexpr int EPI_WARP0 = 4;
 #ifndef SIMJOIN_EPI_WARPS
 #define SIMJOIN_EPI_WARPS 8
@@ -75,7 +79,8 @@ struct JoinParams {
     const int4 *units;             // per unit: first P row, P rows (<= 128), first Q row, Q rows
     const unsigned int *nunits;    // number of units (written by the kernel that builds the list)
     const int *perm_p, *perm_q;    // regrouped position -> original row
-    const uint32_t *keys_p, *keys_q;   // [repetition][original row] hash keys, strides n and m
+    const uint4 *rec_p, *rec_q;    // per regrouped position: the 16-bit hash keys of all repetitions, rec_words x 16 bytes
+    int rec_words;
     int rep;                       // repetitions already joined: a pair whose keys agreed in one of them is not reported again
 };
 
@@ -208,6 +213,24 @@ struct TreeMax<1, MODE> {
 
 // Write `fill` staged pairs of this warp to the output list: one atomic reserves the slots, the
 // stores are coalesced.
+// Bucketed mode, repetition > 0: did the hash keys of regrouped rows (i, j) already agree in an earlier
+// repetition?  Then that repetition found and reported the pair (Section 4's union over repetitions).
+// Both key records are addressed by regrouped position, so the loads of a pair go out together.
+__device__ __forceinline__ bool already_reported(const JoinParams &p, long long i, long long j) {
+    const uint4 *rp = p.rec_p + i * p.rec_words, *rq = p.rec_q + j * p.rec_words;
+    bool seen = false;
+    for (int w = 0; w * 8 < p.rep; ++w) {
+        const uint4 a = __ldg(rp + w), b = __ldg(rq + w);
+        const uint32_t x[4] = {a.x ^ b.x, a.y ^ b.y, a.z ^ b.z, a.w ^ b.w};
+#pragma unroll
+        for (int h = 0; h < 8; ++h) {
+            const uint32_t diff = (h & 1) ? (x[h >> 1] >> 16) : (x[h >> 1] & 0xffffu);
+            seen = seen || (w * 8 + h < p.rep && diff == 0);
+        }
+    }
+    return seen;
+}
+
 template <bool GROUPED>
 __device__ __forceinline__ int2 final_pair(const JoinParams &p, int2 pr) {
     if constexpr (GROUPED) return make_int2(__ldg(p.perm_p + pr.x) + p.ioff, __ldg(p.perm_q + pr.y) + p.joff);
@@ -216,6 +239,40 @@ __device__ __forceinline__ int2 final_pair(const JoinParams &p, int2 pr) {
 template <bool GROUPED>
 __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf, int fill, int lane) {
     if (fill == 0) return;
+    if constexpr (GROUPED) {
+        if (p.rep > 0) {
+            // Duplicates are dropped here, a whole buffer at a time (32 key-record lookups in flight per
+            // step), not when a hit is found: there the lookup's latency would stall the CTA's pipeline.
+            int2 *wbuf = const_cast<int2 *>(buf);
+            int kept = 0;
+            for (int k0 = 0; k0 < fill; k0 += 32) {
+                const int k = k0 + lane;
+                bool keep = false;
+                if (k < fill) {
+                    const int2 pr = wbuf[k];
+                    keep = !already_reported(p, pr.x, pr.y);
+                    if (!keep) wbuf[k].x = -1;
+                }
+                kept += __popc(__ballot_sync(0xffffffffu, keep));
+            }
+            unsigned long long base = 0;
+            if (lane == 0 && kept) base = atomicAdd(p.counter, (unsigned long long)kept);
+            base = __shfl_sync(0xffffffffu, base, 0);
+            __syncwarp();
+            int run = 0;
+            for (int k0 = 0; k0 < fill; k0 += 32) {
+                const int k = k0 + lane;
+                const int2 pr = k < fill ? wbuf[k] : make_int2(-1, 0);
+                const bool keep = pr.x >= 0;
+                const uint32_t b = __ballot_sync(0xffffffffu, keep);
+                const unsigned long long slot = base + (unsigned long long)(run + __popc(b & ((1u << lane) - 1u)));
+                if (keep && slot < p.capacity) p.out[slot] = final_pair<GROUPED>(p, pr);
+                run += __popc(b);
+            }
+            __syncwarp();
+            return;
+        }
+    }
     unsigned long long base = 0;
     if (lane == 0) base = atomicAdd(p.counter, (unsigned long long)fill);
     base = __shfl_sync(0xffffffffu, base, 0);
@@ -253,6 +310,23 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     const int ii = (int)(i + (GROUPED ? 0 : p.ioff));
     const int jj = (int)(j0 + (GROUPED ? 0 : p.joff));
     if (total > STAGE_PAIRS) {
+        if constexpr (GROUPED) {
+            if (p.rep > 0) {
+                // more hits in one block than the buffer holds (rare): check and write them one by one
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    uint32_t mk = mask[q];
+                    while (mk) {
+                        const int c = __ffs(mk) - 1;
+                        mk &= mk - 1;
+                        if (already_reported(p, ii, jj + 32 * q + c)) continue;
+                        const unsigned long long slot = atomicAdd(p.counter, 1ULL);
+                        if (slot < p.capacity) p.out[slot] = final_pair<GROUPED>(p, make_int2(ii, jj + 32 * q + c));
+                    }
+                }
+                return;
+            }
+        }
         unsigned long long base = 0;
         if (lane == 0) base = atomicAdd(p.counter, (unsigned long long)total);
         base = __shfl_sync(0xffffffffu, base, 0);
@@ -281,32 +355,6 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     }
     fill += total;
     __syncwarp();
-}
-
-// Bucketed mode, repetition > 0: clear the candidates whose hash keys already agreed in an earlier
-// repetition -- that repetition found and reported them (Section 4's union over repetitions).
-template <int NQ>
-__device__ __forceinline__ void drop_reported(const JoinParams &p, uint32_t (&mask)[NQ], long long i, long long j0) {
-    uint32_t anyb = 0;
-#pragma unroll
-    for (int q = 0; q < NQ; ++q) anyb |= mask[q];
-    if (anyb == 0) return;
-    const long long pi = __ldg(p.perm_p + i);
-#pragma unroll
-    for (int q = 0; q < NQ; ++q) {
-        uint32_t mk = mask[q], keep = mk;
-        while (mk) {
-            const int c = __ffs(mk) - 1;
-            mk &= mk - 1;
-            const long long qj = __ldg(p.perm_q + (j0 + 32 * q + c));
-            for (int r = 0; r < p.rep; ++r)
-                if (__ldg(p.keys_p + (long long)r * p.n + pi) == __ldg(p.keys_q + (long long)r * p.m + qj)) {
-                    keep &= ~(1u << c);
-                    break;
-                }
-        }
-        mask[q] = keep;
-    }
 }
 
 // The MMA-issuing role (warps 1 and 3).  KC > 0 is a fast path with the chunks per tile known at
@@ -377,7 +425,7 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
             // the P block may be overwritten once the MMAs of every issuer have retired
             if (elect_one()) umma_commit(smem_u32(&ctrl->pempty[pbuf]));
             __syncwarp();
-            if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }
+            if (++pbuf == (uint32_t)p_bufs(GROUPED, kc)) { pbuf = 0; pphase ^= 1; }
         }
     }
     if (!ok) {
@@ -397,10 +445,10 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
 // KC > 0 (1 or 2): the chunks per tile, and with them the resident-P mode, the ring depth and the
 // epilogue hand-back, are compile-time constants -- the host selects these instantiations when the
 // run-time values agree.  Measured on B200: -6 % on the one-chunk int8 join.  KC == 0: all run-time.
-__host__ __device__ constexpr int fast_nstages(int kc) {
-    return (232448 - 1024 - CTRL_BYTES - STAGING_BYTES - P_BUFS * kc * A_CHUNK_BYTES) / B_CHUNK_BYTES > MAX_STAGES
+__host__ __device__ constexpr int fast_nstages(int kc, int pbufs) {
+    return (232448 - 1024 - CTRL_BYTES - STAGING_BYTES - pbufs * kc * A_CHUNK_BYTES) / B_CHUNK_BYTES > MAX_STAGES
                ? MAX_STAGES
-               : (232448 - 1024 - CTRL_BYTES - STAGING_BYTES - P_BUFS * kc * A_CHUNK_BYTES) / B_CHUNK_BYTES;
+               : (232448 - 1024 - CTRL_BYTES - STAGING_BYTES - pbufs * kc * A_CHUNK_BYTES) / B_CHUNK_BYTES;
 }
 // GROUPED: bucketed mode (int8 inner product only) -- see JoinParams::units.
 template <int DT, int KIND, bool NARROW = false, int KC = 0, bool GROUPED = false>
@@ -411,14 +459,15 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         p.kc = KC;
         p.stationary = 1;
         p.epi_release = 1;
-        p.nstages = fast_nstages(KC);
+        p.nstages = fast_nstages(KC, p_bufs(GROUPED, KC));
         p.last_ksteps = 4;
     }
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128-byte swizzle pattern repeats every 1024 bytes.
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int p_bytes = p.stationary ? P_BUFS * p.kc * A_CHUNK_BYTES : 0;
+    const int kc = p.kc;
+    const int p_bytes = p.stationary ? p_bufs(GROUPED, kc) * kc * A_CHUNK_BYTES : 0;
     const int stage_bytes = B_CHUNK_BYTES + (p.stationary ? 0 : A_CHUNK_BYTES);
     uint8_t *smem_p = smem;
     uint8_t *smem_ring = smem + p_bytes;
@@ -469,7 +518,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                                     c * p.elems_per_chunk, p_row);
                 }
                 __syncwarp();
-                if (++pbuf == (uint32_t)P_BUFS) { pbuf = 0; pphase ^= 1; }
+                if (++pbuf == (uint32_t)p_bufs(GROUPED, kc)) { pbuf = 0; pphase ^= 1; }
             }
             for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
                 const int q_row = (GROUPED ? un.qrow0 : 0) + tile_at<GROUPED>(un, k) * TILE_N;
@@ -661,9 +710,6 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         mk &= valid;
                         if (!((gm >> k) & 1u)) mk = 0;       // the group bound is necessary: nothing can pass here
                         mask[k >> 1] |= mk << ((k & 1) * 16);
-                    }
-                    if constexpr (GROUPED) {
-                        if (p.rep > 0) drop_reported<EPI_COLS / 32>(p, mask, i, j0);
                     }
                     emit_pairs<EPI_COLS / 32, GROUPED>(p, mask, lane, i, j0, stage_buf, stage_fill);
                 }

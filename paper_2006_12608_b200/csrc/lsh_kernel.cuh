@@ -23,11 +23,12 @@ __host__ __device__ inline uint64_t lsh_splitmix64(uint64_t seed, uint64_t idx) 
     return z ^ (z >> 31);
 }
 
-// keys[l * rows + i] = key of row i in repetition l: k bits in the first L_high repetitions, k - 1 (the
+// rec[i * stride + l] = key of row i in repetition l (one record of `stride` 16-bit keys per row, so that
+// all keys of a row sit in one or two cache lines): k bits in the first L_high repetitions, k - 1 (the
 // same samples without the last) in the following L_low -- the paper's mix of tables for a fractional
 // number of base hashes.  One thread per row; the sampled coordinates are computed once per block.
 __global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict__ X, long long rows, int d, int L_high, int L_low,
-                                                       int k, unsigned long long seed, uint32_t *__restrict__ keys) {
+                                                       int k, unsigned long long seed, uint16_t *__restrict__ rec, int stride) {
     __shared__ int s_coord[LSH_MAX_REPS * LSH_MAX_BITS];
     const int L = L_high + L_low;
     for (int t = threadIdx.x; t < L * k; t += blockDim.x) {
@@ -38,22 +39,23 @@ __global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict_
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= rows) return;
     const int8_t *x = X + i * d;
-    for (int l = 0; l < L; ++l) {
+    for (int l = 0; l < stride; ++l) {
         uint32_t key = 0;
-        const int bits = l < L_high ? k : k - 1;
+        const int bits = l < L_high ? k : (l < L ? k - 1 : 0);      // padding entries stay 0
         for (int b = 0; b < bits; ++b) key |= (x[s_coord[l * k + b]] > 0 ? 1u : 0u) << b;
-        keys[(long long)l * rows + i] = key;
+        rec[i * stride + l] = (uint16_t)key;
     }
 }
 
 // hist[key] += number of rows with that key (block-private histogram in shared memory first).
-__global__ void __launch_bounds__(LSH_SORT_THREADS) lsh_hist_kernel(const uint32_t *__restrict__ keys, long long rows, int nb,
-                                                                    unsigned int *__restrict__ hist) {
+// keys: the key of row i is keys[i * stride] (one column of the key records).
+__global__ void __launch_bounds__(LSH_SORT_THREADS) lsh_hist_kernel(const uint16_t *__restrict__ keys, int stride, long long rows,
+                                                                    int nb, unsigned int *__restrict__ hist) {
     __shared__ unsigned int s_cnt[LSH_MAX_BUCKETS];
     for (int b = threadIdx.x; b < nb; b += blockDim.x) s_cnt[b] = 0;
     __syncthreads();
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < rows; i += (long long)gridDim.x * blockDim.x)
-        atomicAdd(&s_cnt[keys[i]], 1u);
+        atomicAdd(&s_cnt[keys[i * stride]], 1u);
     __syncthreads();
     for (int b = threadIdx.x; b < nb; b += blockDim.x)
         if (s_cnt[b]) atomicAdd(&hist[b], s_cnt[b]);
@@ -136,8 +138,9 @@ __global__ void __launch_bounds__(1024) lsh_offsets_units_kernel(const unsigned 
 
 // perm[position] = row, positions grouped by key: each block ranks its rows inside shared-memory
 // counters, reserves one range per key with a single global atomic, and writes its rows there.
-__global__ void __launch_bounds__(LSH_SORT_THREADS) lsh_scatter_kernel(const uint32_t *__restrict__ keys, long long rows, int nb,
-                                                                       unsigned int *__restrict__ cursor, int *__restrict__ perm) {
+__global__ void __launch_bounds__(LSH_SORT_THREADS) lsh_scatter_kernel(const uint16_t *__restrict__ keys, int stride, long long rows,
+                                                                       int nb, unsigned int *__restrict__ cursor,
+                                                                       int *__restrict__ perm) {
     __shared__ unsigned int s_cnt[LSH_MAX_BUCKETS];
     for (int b = threadIdx.x; b < nb; b += blockDim.x) s_cnt[b] = 0;
     __syncthreads();
@@ -147,7 +150,7 @@ __global__ void __launch_bounds__(LSH_SORT_THREADS) lsh_scatter_kernel(const uin
 #pragma unroll
     for (int t = 0; t < LSH_SORT_ITEMS; ++t) {
         const long long i = base + t * LSH_SORT_THREADS + threadIdx.x;
-        key[t] = i < rows ? keys[i] : 0u;
+        key[t] = i < rows ? keys[i * stride] : 0u;
         rank[t] = i < rows ? atomicAdd(&s_cnt[key[t]], 1u) : 0u;
     }
     __syncthreads();

@@ -47,7 +47,7 @@ struct simjoin_ctx {
     long long ioff, joff;
     bool attr_set[2][3][2][3][2];
     // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
-    DevBuf lsh_keys_p, lsh_keys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
+    DevBuf lsh_keys_p, lsh_keys_q, lsh_skeys_p, lsh_skeys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
 };
 
 namespace {
@@ -164,9 +164,9 @@ template <int DT, int KIND, bool NARROW = false, bool GROUPED = false>
 cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
                         size_t smem) {
     const bool fast = jp.stationary && jp.epi_release && jp.last_ksteps == 4;
-    if (fast && jp.kc == 1 && jp.nstages == fast_nstages(1))
+    if (fast && jp.kc == 1 && jp.nstages == fast_nstages(1, p_bufs(GROUPED, 1)))
         return launch_join_kc<DT, KIND, NARROW, 1, GROUPED>(ctx, mp, mq, jp, grid, smem);
-    if (fast && jp.kc == 2 && jp.nstages == fast_nstages(2))
+    if (fast && jp.kc == 2 && jp.nstages == fast_nstages(2, p_bufs(GROUPED, 2)))
         return launch_join_kc<DT, KIND, NARROW, 2, GROUPED>(ctx, mp, mq, jp, grid, smem);
     return launch_join_kc<DT, KIND, NARROW, 0, GROUPED>(ctx, mp, mq, jp, grid, smem);
 }
@@ -192,7 +192,8 @@ int clamp_to_i32(double v) {
 
 // Tile geometry of a join over rows of `row_bytes` bytes: chunks per tile, resident-P mode, ring depth,
 // dynamic shared memory.  False when the ring would be too shallow.
-bool tile_geometry(const simjoin_ctx *ctx, int64_t n, int64_t m, int row_bytes, size_t es, JoinParams &jp, size_t &smem) {
+bool tile_geometry(const simjoin_ctx *ctx, int64_t n, int64_t m, int row_bytes, size_t es, JoinParams &jp, size_t &smem,
+                   bool grouped = false) {
     std::memset(&jp, 0, sizeof jp);
     jp.n = n;
     jp.m = m;
@@ -201,7 +202,7 @@ bool tile_geometry(const simjoin_ctx *ctx, int64_t n, int64_t m, int row_bytes, 
     jp.last_ksteps = (last_bytes + 31) / 32;
     jp.elems_per_chunk = (int)(CHUNK_BYTES / es);
     jp.stationary = jp.kc <= MAX_STATIONARY_CHUNKS ? 1 : 0;
-    const int p_bytes = jp.stationary ? P_BUFS * jp.kc * A_CHUNK_BYTES : 0;
+    const int p_bytes = jp.stationary ? p_bufs(grouped, jp.kc) * jp.kc * A_CHUNK_BYTES : 0;
     const int stage_bytes = B_CHUNK_BYTES + (jp.stationary ? 0 : A_CHUNK_BYTES);
     int nstages = (ctx->max_smem_optin - 1024 - CTRL_BYTES - STAGING_BYTES - p_bytes) / stage_bytes;
     if (nstages > MAX_STAGES) nstages = MAX_STAGES;
@@ -385,6 +386,8 @@ simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
     release(ctx->stage_out);
     release(ctx->lsh_keys_p);
     release(ctx->lsh_keys_q);
+    release(ctx->lsh_skeys_p);
+    release(ctx->lsh_skeys_q);
     release(ctx->lsh_perm_p);
     release(ctx->lsh_perm_q);
     release(ctx->lsh_sorted_p);
@@ -500,13 +503,16 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
 
     JoinParams jp;
     size_t smem = 0;
-    if (!tile_geometry(ctx, n, m, d, 1, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
+    if (!tile_geometry(ctx, n, m, d, 1, jp, smem, true)) return SIMJOIN_ERR_UNSUPPORTED;
     const int nb_max = 1 << k;
     const size_t max_units = (size_t)((n + TILE_M - 1) / TILE_M) + (size_t)nb_max;
     // misc: hist_p | hist_q | cursor_p | cursor_q (nb words each) | nunits (padded to 16 B) | units
     const size_t off_units = ((size_t)4 * nb_max * 4 + 16 + 15) & ~(size_t)15;
     const int reps = L + L_low;
-    if (!grow(ctx->lsh_keys_p, (size_t)reps * n * 4) || !grow(ctx->lsh_keys_q, (size_t)reps * m * 4) ||
+    const int rec_words = (reps + 7) / 8, stride = rec_words * 8;   // key record of a row: 16-bit keys, padded to 16 bytes
+    const size_t rec_bytes = (size_t)rec_words * 16;
+    if (!grow(ctx->lsh_keys_p, n * rec_bytes) || !grow(ctx->lsh_keys_q, m * rec_bytes) ||
+        !grow(ctx->lsh_skeys_p, n * rec_bytes) || !grow(ctx->lsh_skeys_q, m * rec_bytes) ||
         !grow(ctx->lsh_perm_p, (size_t)n * 4) || !grow(ctx->lsh_perm_q, (size_t)m * 4) ||
         !grow(ctx->lsh_sorted_p, (size_t)n * d) || !grow(ctx->lsh_sorted_q, (size_t)m * d) ||
         !grow(ctx->lsh_misc, off_units + max_units * 16))
@@ -514,7 +520,7 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     unsigned int *hist_p = reinterpret_cast<unsigned int *>(ctx->lsh_misc.ptr);
     unsigned int *hist_q = hist_p + nb_max, *cursor_p = hist_q + nb_max, *cursor_q = cursor_p + nb_max, *nunits = cursor_q + nb_max;
     int4 *units = reinterpret_cast<int4 *>(reinterpret_cast<unsigned char *>(ctx->lsh_misc.ptr) + off_units);
-    uint32_t *keys_p = reinterpret_cast<uint32_t *>(ctx->lsh_keys_p.ptr), *keys_q = reinterpret_cast<uint32_t *>(ctx->lsh_keys_q.ptr);
+    uint16_t *keys_p = reinterpret_cast<uint16_t *>(ctx->lsh_keys_p.ptr), *keys_q = reinterpret_cast<uint16_t *>(ctx->lsh_keys_q.ptr);
     int *perm_p = reinterpret_cast<int *>(ctx->lsh_perm_p.ptr), *perm_q = reinterpret_cast<int *>(ctx->lsh_perm_q.ptr);
 
     jp.out = reinterpret_cast<int2 *>(out_pairs);
@@ -528,8 +534,9 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     jp.nunits = nunits;
     jp.perm_p = perm_p;
     jp.perm_q = perm_q;
-    jp.keys_p = keys_p;
-    jp.keys_q = keys_q;
+    jp.rec_p = reinterpret_cast<const uint4 *>(ctx->lsh_skeys_p.ptr);
+    jp.rec_q = reinterpret_cast<const uint4 *>(ctx->lsh_skeys_q.ptr);
+    jp.rec_words = rec_words;
 
     CUtensorMap mapP, mapQ;
     if (!encode_rows_map(ctx, &mapP, ctx->lsh_sorted_p.ptr, n, d, TILE_M) ||
@@ -552,28 +559,37 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     const bool narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
 
     cudaEventRecord(ctx->ev[0], s);
-    lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p);
-    lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q);
+    lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p,
+                                                                stride);
+    lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q,
+                                                                stride);
     if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
     cudaEventRecord(ctx->ev[1], s);
     const int g = d / 16;
     const unsigned hist_blocks = (unsigned)ctx->num_sms * 4;
     const int rows_per_block = LSH_SORT_THREADS * LSH_SORT_ITEMS;
     for (int l = 0; l < reps; ++l) {
-        const uint32_t *kp = keys_p + (size_t)l * n, *kq = keys_q + (size_t)l * m;
+        const uint16_t *kp = keys_p + l, *kq = keys_q + l;          // column l of the key records
         const int nb = l < L ? nb_max : nb_max / 2;          // buckets of this repetition
         if (cudaMemsetAsync(hist_p, 0, (size_t)2 * nb_max * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kp, n, nb, hist_p);
-        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kq, m, nb, hist_q);
+        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kp, stride, n, nb, hist_p);
+        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kq, stride, m, nb, hist_q);
         lsh_offsets_units_kernel<<<1, 1024, 0, s>>>(hist_p, hist_q, nb, cursor_p, cursor_q, units, nunits, TILE_M);
-        lsh_scatter_kernel<<<(unsigned)((n + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kp, n, nb, cursor_p,
-                                                                                                              perm_p);
-        lsh_scatter_kernel<<<(unsigned)((m + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kq, m, nb, cursor_q,
-                                                                                                              perm_q);
+        lsh_scatter_kernel<<<(unsigned)((n + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kp, stride, n, nb,
+                                                                                                              cursor_p, perm_p);
+        lsh_scatter_kernel<<<(unsigned)((m + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kq, stride, m, nb,
+                                                                                                              cursor_q, perm_q);
         lsh_gather_rows_kernel<<<(unsigned)(((long long)n * g + 255) / 256), 256, 0, s>>>(
             reinterpret_cast<const uint4 *>(P), perm_p, n, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_p.ptr));
         lsh_gather_rows_kernel<<<(unsigned)(((long long)m * g + 255) / 256), 256, 0, s>>>(
             reinterpret_cast<const uint4 *>(Q), perm_q, m, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_q.ptr));
+        if (l > 0) {
+            // key records in regrouped order, for the duplicate check of the join's epilogue
+            lsh_gather_rows_kernel<<<(unsigned)(((long long)n * rec_words + 255) / 256), 256, 0, s>>>(
+                reinterpret_cast<const uint4 *>(keys_p), perm_p, n, rec_words, reinterpret_cast<uint4 *>(ctx->lsh_skeys_p.ptr));
+            lsh_gather_rows_kernel<<<(unsigned)(((long long)m * rec_words + 255) / 256), 256, 0, s>>>(
+                reinterpret_cast<const uint4 *>(keys_q), perm_q, m, rec_words, reinterpret_cast<uint4 *>(ctx->lsh_skeys_q.ptr));
+        }
         if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
         jp.rep = l;
         const cudaError_t e = narrow ? launch_join<DT_I8, KIND_IP, true, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem)

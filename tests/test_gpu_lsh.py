@@ -63,6 +63,14 @@ def test_lsh_mixed_tables(ctx, L, L_low, k):
         assert check(ctx, w.P, w.Q, t, L, k, 77, L_low=L_low) > 0
 
 
+def test_lsh_dense_output(ctx):
+    # every colliding pair passes: blocks with more hits than the staging buffer holds take the direct
+    # output path, which must drop the pairs of earlier tables too
+    w = W.make_workload(4, n=900, m=1100, planted=50)
+    assert check(ctx, w.P, w.Q, -1000.0, 4, 2, 31) > 400000
+    assert check(ctx, w.P, w.Q, 4.0, 5, 3, 32) > 50000
+
+
 def test_no_hash_bits_is_the_brute_force_join(ctx):
     w = W.make_workload(4, n=3000, m=4100, planted=200)
     pairs, cnt = gpu_lsh(ctx, w.P, w.Q, 30.0, 3, 0, 7)
