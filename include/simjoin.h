@@ -142,8 +142,9 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
  *
  * I8 contexts only (ERR_UNSUPPORTED otherwise).  Every pair is reported once, whatever the number of
  * repetitions it collides in; the order is unspecified.  The context keeps regrouped copies of P and Q
- * and two copies of a 16-bit key per row and repetition as scratch (about (n+m) * (d + 4(L+L_low) + 4) bytes).  Hashing, regrouping, the work list and
- * the bucketed join all run on the device with no host round trip between repetitions.
+ * and two copies of a record of 16-bit keys per row as scratch:
+ * (n+m) * (d + 4 + 32*ceil((L+L_low)/8)) bytes.  Hashing, regrouping, the work list and the bucketed
+ * join all run on the device with no host round trip between repetitions.
  * simjoin_last_kernel_ms then reports (hashing, all repetitions).
  */
 simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
