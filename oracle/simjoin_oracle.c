@@ -344,6 +344,64 @@ int64_t oracle_lsh_join_i8(const int8_t *P, int64_t n, const int8_t *Q, int64_t 
     return total;
 }
 
+/* ------------------------------------------------------------------ JL transform
+ * Section 3 (the lemma that constructs M and its proof): M = (I_{r_l} (x) A_l) ... (I_{r_1} (x) A_1),
+ * applied to a vector level by level: level i cuts its input into r_i consecutive blocks of c_i
+ * coordinates and maps every block with the same k_i x c_i matrix A_i.  Sizes as the proof sets them,
+ * with zeta = 2 (the value the running-time theorem uses): l = log2(d / k), r_i = 2^(l-i),
+ * k_i = i*k for i < l and k_l = k, c_1 = 2k, c_i = 2*k_(i-1).  A_i: independent random signs scaled by
+ * 1/sqrt(k_i) (the paper allows any matrix family with the strong JL moment property and names random
+ * +-1 entries); sign of entry (a, b) of A_i = bit 0 of splitmix64(seed, i * 2^40 + a * c_i + b):
+ * 1 -> +1, 0 -> -1.  Everything in fp64; inputs are bf16 bit patterns, widened exactly. */
+int32_t oracle_jl_levels(int32_t d, int32_t k) {
+    if (d <= 0 || k <= 0 || d % k != 0) return -1;
+    int32_t q = d / k, l = 0;
+    while (q > 1 && q % 2 == 0) { q /= 2; ++l; }
+    return (q == 1 && l >= 1) ? l : -1;
+}
+
+/* (r_i, c_i, k_i) of level i (1-based); returns 0 on success. */
+int32_t oracle_jl_shape(int32_t d, int32_t k, int32_t i, int32_t *r, int32_t *c, int32_t *kout) {
+    const int32_t l = oracle_jl_levels(d, k);
+    if (l < 1 || i < 1 || i > l) return -1;
+    *r = 1 << (l - i);
+    *kout = i < l ? i * k : k;
+    *c = i == 1 ? 2 * k : 2 * (i - 1) * k;
+    return 0;
+}
+
+int32_t oracle_jl_sign(uint64_t seed, int32_t level, int64_t a, int64_t b, int32_t c_i) {
+    return (splitmix64_at(seed, ((uint64_t)level << 40) + (uint64_t)(a * c_i + b)) & 1u) ? 1 : -1;
+}
+
+/* out (rows x k, fp64) = M applied to every row of X (rows x d, bf16 bits).  Returns 0, or -1 for bad sizes. */
+int32_t oracle_jl_transform_bf16(const uint16_t *X, int64_t rows, int32_t d, int32_t k, uint64_t seed, double *out) {
+    const int32_t l = oracle_jl_levels(d, k);
+    if (l < 1 || rows < 0) return -1;
+    double *cur = (double *)malloc(sizeof(double) * (size_t)d);
+    double *nxt = (double *)malloc(sizeof(double) * (size_t)d);
+    if (!cur || !nxt) { free(cur); free(nxt); return -1; }
+    for (int64_t row = 0; row < rows; ++row) {
+        for (int32_t t = 0; t < d; ++t) cur[t] = oracle_bf16_to_f64(X[(size_t)row * d + t]);
+        for (int32_t i = 1; i <= l; ++i) {
+            int32_t r, c, ki;
+            oracle_jl_shape(d, k, i, &r, &c, &ki);
+            const double scale = 1.0 / sqrt((double)ki);
+            for (int32_t blk = 0; blk < r; ++blk)
+                for (int32_t a = 0; a < ki; ++a) {
+                    double acc = 0.0;
+                    for (int32_t b = 0; b < c; ++b) acc += (double)oracle_jl_sign(seed, i, a, b, c) * cur[(size_t)blk * c + b];
+                    nxt[(size_t)blk * ki + a] = acc * scale;
+                }
+            double *tmp = cur; cur = nxt; nxt = tmp;
+        }
+        for (int32_t t = 0; t < k; ++t) out[(size_t)row * k + t] = cur[t];
+    }
+    free(cur);
+    free(nxt);
+    return 0;
+}
+
 int64_t oracle_join_bf16(const uint16_t *P, int64_t n, const uint16_t *Q, int64_t m, int32_t d, int32_t kind,
                          double threshold, int32_t *out_pairs, int64_t capacity, int32_t nthreads) {
     if (n < 0 || m < 0 || d <= 0 || capacity < 0 || kind < KIND_IP || kind > KIND_L2) return -1;

@@ -76,6 +76,14 @@ def _load():
     lib.oracle_lsh_keys_i8.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, vp]
     lib.oracle_lsh_coordinate.restype = i32
     lib.oracle_lsh_coordinate.argtypes = [c.c_uint64, i32, i32, i32]
+    lib.oracle_jl_levels.restype = i32
+    lib.oracle_jl_levels.argtypes = [i32, i32]
+    lib.oracle_jl_shape.restype = i32
+    lib.oracle_jl_shape.argtypes = [i32, i32, i32, c.POINTER(i32), c.POINTER(i32), c.POINTER(i32)]
+    lib.oracle_jl_sign.restype = i32
+    lib.oracle_jl_sign.argtypes = [c.c_uint64, i32, i64, i64, i32]
+    lib.oracle_jl_transform_bf16.restype = i32
+    lib.oracle_jl_transform_bf16.argtypes = [vp, i64, i32, i32, c.c_uint64, vp]
     lib.oracle_scores_i8.restype = i32
     lib.oracle_scores_i8.argtypes = [vp, vp, i32, i32, vp, i64, vp]
     lib.oracle_scores_bf16.restype = i32
@@ -187,6 +195,37 @@ def lsh_keys(X: np.ndarray, L: int, k: int, seed: int, L_low: int = 0) -> np.nda
 
 def lsh_coordinate(seed: int, rep: int, bit: int, d: int) -> int:
     return int(_load().oracle_lsh_coordinate(seed, rep, bit, d))
+
+
+def jl_shapes(d: int, k: int):
+    """[(r_i, c_i, k_i)] for the levels i = 1..l of the JL construction with zeta = 2; raises if d/k is not 2^l, l >= 1."""
+    lib = _load()
+    levels = lib.oracle_jl_levels(d, k)
+    if levels < 1:
+        raise ValueError("d / k must be a power of two >= 2")
+    out = []
+    for i in range(1, levels + 1):
+        r, c, ko = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+        lib.oracle_jl_shape(d, k, i, ctypes.byref(r), ctypes.byref(c), ctypes.byref(ko))
+        out.append((r.value, c.value, ko.value))
+    return out
+
+
+def jl_sign_matrix(seed: int, level: int, k_i: int, c_i: int) -> np.ndarray:
+    """The +-1 entries of A_level (k_i x c_i), unscaled."""
+    lib = _load()
+    return np.array([[lib.oracle_jl_sign(seed, level, a, b, c_i) for b in range(c_i)] for a in range(k_i)], dtype=np.int8)
+
+
+def jl_transform(X: np.ndarray, k: int, seed: int) -> np.ndarray:
+    """M x for every row x of X (bf16 bit patterns, rows x d) -> (rows, k) float64."""
+    lib = _load()
+    X = _check(X, "bf16")
+    rows, d = X.shape
+    out = np.empty((rows, k), dtype=np.float64)
+    if lib.oracle_jl_transform_bf16(X.ctypes.data, rows, d, k, seed, out.ctypes.data) != 0:
+        raise ValueError("oracle rejected the arguments (d / k must be a power of two >= 2)")
+    return out
 
 
 def band_sets(P, Q, kind, threshold, dtype, rel: float = 1e-2, threads: int = 0):

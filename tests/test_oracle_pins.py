@@ -140,6 +140,64 @@ def test_lsh_recall_matches_the_collision_probability():
         O.lsh_join(w.P, w.Q, 1.0, 1, 0, 1, L_low=1)          # k - 1 bits needs k >= 1
 
 
+# ------------------------------------------------------------------ JL transform (Section 3)
+def test_jl_level_sizes_chain_up_as_the_construction_requires():
+    # d = r_1 c_1,  r_i k_i = r_{i+1} c_{i+1},  r_l k_l = k  (the size equations of the lemma's proof), zeta = 2
+    for d, k in [(128, 64), (256, 32), (1024, 64), (4096, 8), (512, 128)]:
+        sh = O.jl_shapes(d, k)
+        assert len(sh) == int(np.log2(d // k))
+        assert sh[0][0] * sh[0][1] == d and sh[0][1] == 2 * k
+        for (r0, _c0, k0), (r1, c1, _k1) in zip(sh, sh[1:]):
+            assert r0 * k0 == r1 * c1 and r1 * 2 == r0
+        assert sh[-1][0] == 1 and sh[-1][2] == k
+        for i, (r, c, ki) in enumerate(sh, start=1):
+            assert ki == (i * k if i < len(sh) else k) and c == (2 * k if i == 1 else 2 * (i - 1) * k)
+    assert O.jl_shapes(1024, 64) == [(8, 128, 64), (4, 128, 128), (2, 256, 192), (1, 384, 64)]   # worked by hand
+    for d, k in [(96, 32), (64, 64), (100, 7)]:
+        with pytest.raises(ValueError):
+            O.jl_shapes(d, k)
+
+
+def test_jl_transform_is_the_kronecker_product_chain():
+    # M = (I_{r_l} (x) A_l) ... (I_{r_1} (x) A_1) written out with numpy.kron; signs re-derived in python ints
+    d, k, seed = 256, 16, 77
+    sh = O.jl_shapes(d, k)
+    M = np.eye(d)
+    for i, (r, c, ki) in enumerate(sh, start=1):
+        A = np.array([[1.0 if _splitmix64(seed, (i << 40) + a * c + b) & 1 else -1.0 for b in range(c)] for a in range(ki)])
+        assert np.array_equal(A.astype(np.int8), O.jl_sign_matrix(seed, i, ki, c))
+        M = np.kron(np.eye(r), A / np.sqrt(ki)) @ M
+    assert M.shape == (k, d)
+    X = W.random_points("bf16", 9, d, 5)
+    want = W.bf16_bits_to_f32(X).astype(np.float64) @ M.T
+    got = O.jl_transform(X, k, seed)
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-12)
+    # one level (d = 2k): a plain random-sign projection
+    X2 = W.random_points("bf16", 4, 32, 6)
+    A1 = O.jl_sign_matrix(3, 1, 16, 32).astype(np.float64) / 4.0
+    assert np.allclose(O.jl_transform(X2, 16, 3), W.bf16_bits_to_f32(X2).astype(np.float64) @ A1.T, rtol=1e-12, atol=1e-12)
+
+
+def test_jl_transform_preserves_norms_in_expectation_and_concentrates():
+    # E |Mx|^2 = |x|^2 for independent sign matrices scaled by 1/sqrt(k_i); the distortion of one draw is O(1/sqrt(k))
+    d, k = 512, 64
+    X = W.random_points("bf16", 6, d, 11)
+    n2 = (W.bf16_bits_to_f32(X).astype(np.float64) ** 2).sum(axis=1)
+    ratios = np.array([(O.jl_transform(X, k, seed) ** 2).sum(axis=1) / n2 for seed in range(60)])     # (60, 6)
+    assert abs(ratios.mean() - 1.0) < 0.03, ratios.mean()
+    assert np.abs(np.sqrt(ratios) - 1.0).max() < 0.45
+    # linear: M(2x) = 2 Mx, M(x + y) = Mx + My (inputs chosen so that the sums are exact in bf16)
+    ints = np.random.default_rng(1).integers(-8, 9, size=(2, d)).astype(np.float32)
+    xb, yb, sb = (W.f32_to_bf16_bits(v[None, :]) for v in (ints[0], ints[1], ints[0] + ints[1]))
+    tx, ty, ts = (O.jl_transform(v, k, 5) for v in (xb, yb, sb))
+    assert np.allclose(tx + ty, ts, rtol=1e-12, atol=1e-9)
+    # distances between points are preserved like norms (what a join after the reduction relies on)
+    Y = W.random_points("bf16", 6, d, 12)
+    dist = np.linalg.norm(W.bf16_bits_to_f32(X).astype(np.float64) - W.bf16_bits_to_f32(Y).astype(np.float64), axis=1)
+    dred = np.mean([np.linalg.norm(O.jl_transform(X, k, s) - O.jl_transform(Y, k, s), axis=1) / dist for s in range(30)])
+    assert abs(dred - 1.0) < 0.05, dred
+
+
 # ------------------------------------------------- independent formulations
 def _packbits_rows(X):
     return np.packbits(X > 0, axis=1)
