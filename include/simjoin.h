@@ -152,6 +152,30 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
                                int32_t *out_pairs, uint64_t capacity, uint64_t *count);
 
 /*
+ * JL transform (Section 3: the lemma that builds M = (I_{r_l} (x) A_l) ... (I_{r_1} (x) A_1) and computes M x
+ * as l small dense products): out = X M^T for all n rows at once, reducing d coordinates to k, as a
+ * pre-reduction before an (approximate) join on the k-dimensional rows.
+ *
+ *   X     device pointer, n x d bf16, row-major, 16-byte aligned.          out   device pointer, n x k bf16.
+ *   d, k  d / k must be a power of two >= 2 (zeta = 2, the value of the paper's running-time theorem; l =
+ *         log2(d / k) levels; ERR_ARG otherwise); k a multiple of 8 and 2*(l-1)*k*2 bytes <= SIMJOIN_MAX_ROW_BYTES
+ *         (ERR_UNSUPPORTED otherwise).  The paper's k = ceil(C eps^-2 log 1/delta) has an unspecified constant:
+ *         k is the caller's choice.
+ *   Level i (1..l) cuts every point into r_i = 2^(l-i) blocks of c_i coordinates (c_1 = 2k, c_i = 2(i-1)k) and
+ *   maps each block with the same k_i x c_i matrix A_i (k_i = i*k, k_l = k) of independent random signs scaled
+ *   by 1/sqrt(k_i); the sign of entry (a, b) is bit 0 of splitmix64(seed, i * 2^40 + a * c_i + b) (1 -> +1),
+ *   splitmix64 as in simjoin_run_lsh.  Each level is one launch of the tile kernel with A_i resident in shared
+ *   memory and the blocks streamed by TMA; products are exact in fp32 up to accumulation order, and each level's
+ *   output is rounded to bf16 (the next level's operand type).
+ *
+ * BF16 contexts only (ERR_UNSUPPORTED otherwise).  Scratch owned by the context: two buffers of n * max_i(r_i k_i)
+ * bf16 values and one level matrix.  Synchronises the stream before returning.  simjoin_last_kernel_ms then
+ * reports (0, all levels).
+ */
+simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, int32_t d, int32_t k, uint64_t seed,
+                                    void *out);
+
+/*
  * Hamming join on bit-packed points (Section 4: Hamming is the first ip-distance listed, with the
  * embedding f(x) = (x_k, 1-x_k)_k, g(y) = (1-y_k, y_k)_k).  keep (i, j) when Hamming(x_i, y_j) <= r.
  *

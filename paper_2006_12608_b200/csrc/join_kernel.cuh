@@ -17,6 +17,8 @@
 //               through a per-warp shared-memory staging buffer to the output list
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word and drains.
 #pragma once
+#include <cuda_bf16.h>
+
 #include <type_traits>
 
 #include "ptx_sm100.cuh"
@@ -25,6 +27,10 @@ namespace sj {
 
 constexpr int DT_I8 = 0, DT_BF16 = 1;
 constexpr int KIND_IP = 0, KIND_COS = 1, KIND_L2 = 2;
+// KIND_STORE (bf16): no predicate -- the scaled score tile itself is written out, transposed, as bf16:
+// out[j * store_ld + i] = bf16(store_scale * <P_i, Q_j>).  This is the dense product Q * P^T with P the
+// small, resident operand: one level of the JL transform of Section 3.
+constexpr int KIND_STORE = 3;
 
 constexpr int TILE_M = 128;                       // rows of P per tile
 constexpr int TILE_N = 256;                       // rows of Q per tile
@@ -82,6 +88,10 @@ struct JoinParams {
     const uint4 *rec_p, *rec_q;    // per regrouped position: the 16-bit hash keys of all repetitions, rec_words x 16 bytes
     int rec_words;
     int rep;                       // repetitions already joined: a pair whose keys agreed in one of them is not reported again
+    // KIND_STORE
+    uint16_t *store_out;
+    long long store_ld;
+    float store_scale;
 };
 
 struct Ctrl {
@@ -608,7 +618,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 // per-column terms of this warp's columns, 4 per lane, fetched while the tile is still
                 // being multiplied so that the exact test never waits on global memory
                 uint4 yq = make_uint4(0, 0, 0, 0);
-                if (KIND != KIND_IP && lane < EPI_COLS / 4)
+                if ((KIND == KIND_COS || KIND == KIND_L2) && lane < EPI_COLS / 4)
                     yq = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint32_t *>(p.ny) +
                                                                ((long long)qt * TILE_N + half * EPI_COLS)) + lane);
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
@@ -645,6 +655,22 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                if constexpr (KIND == KIND_STORE) {
+                    // lane <-> row of P (an output coordinate), columns <-> rows of Q (output rows): for a
+                    // fixed column the 32 lanes write 32 consecutive bf16 values
+                    const long long j0 = q_base + (long long)qt * TILE_N + half * EPI_COLS;
+                    const long long left = q_end - j0;
+                    if (row_ok) {
+                        uint16_t *o = p.store_out + j0 * p.store_ld + i;
+#pragma unroll
+                        for (int c = 0; c < EPI_COLS; ++c)
+                            if (c < left)
+                                o[(long long)c * p.store_ld] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[c]) * p.store_scale));
+                    }
+                    acc ^= 1;
+                    if (acc == 0) accphase ^= 1;
+                    continue;
+                }
                 // level 0: the row maximum over this warp's 128 columns against the per-tile bound
                 // (a necessary condition of the exact test, in the same arithmetic)
                 auto bound_ok = [&](uint32_t word) -> bool {

@@ -12,6 +12,7 @@
 #include <new>
 
 #include "join_kernel.cuh"
+#include "jl_kernel.cuh"
 #include "lsh_kernel.cuh"
 #include "prepass_kernel.cuh"
 
@@ -45,8 +46,9 @@ struct simjoin_ctx {
     bool have_timing;
     float prepass_ms, join_ms;
     long long ioff, joff;
-    bool attr_set[2][3][2][3][2];
+    bool attr_set[2][4][2][3][2];
     // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
+    DevBuf jl_a, jl_buf[2];             // JL transform: level matrix, ping-pong level outputs
     DevBuf lsh_keys_p, lsh_keys_q, lsh_skeys_p, lsh_skeys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
 };
 
@@ -384,6 +386,9 @@ simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
     release(ctx->stage_p);
     release(ctx->stage_q);
     release(ctx->stage_out);
+    release(ctx->jl_a);
+    release(ctx->jl_buf[0]);
+    release(ctx->jl_buf[1]);
     release(ctx->lsh_keys_p);
     release(ctx->lsh_keys_q);
     release(ctx->lsh_skeys_p);
@@ -613,6 +618,81 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
 }
 
+simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, int32_t d, int32_t k, uint64_t seed, void *out) {
+    if (!ctx || !X || !out || n < 0 || d <= 0 || k <= 0) return SIMJOIN_ERR_ARG;
+    if (ctx->dtype != SIMJOIN_BF16) return SIMJOIN_ERR_UNSUPPORTED;
+    if (d % k != 0) return SIMJOIN_ERR_ARG;
+    int levels = 0;
+    for (int q = d / k; q > 1; q /= 2, ++levels)
+        if (q % 2 != 0) return SIMJOIN_ERR_ARG;                       // zeta = 2: d / k must be a power of two
+    if (levels < 1) return SIMJOIN_ERR_ARG;
+    if (k % 8 != 0) return SIMJOIN_ERR_UNSUPPORTED;                   // 16-byte rows at every level
+    const int c_max = levels == 1 ? 2 * k : 2 * (levels - 1) * k;     // widest block: the last level's
+    if ((size_t)c_max * 2 > SIMJOIN_MAX_ROW_BYTES || (size_t)d * 2 > SIMJOIN_MAX_ROW_BYTES) return SIMJOIN_ERR_UNSUPPORTED;
+    if (n * (int64_t)(d / (2 * k)) >= SIMJOIN_MAX_ROWS) return SIMJOIN_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(X) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) return SIMJOIN_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    ctx->have_timing = false;
+    if (n == 0) return SIMJOIN_OK;
+    if (!is_device_ptr(X, ctx->device) || !is_device_ptr(out, ctx->device)) return SIMJOIN_ERR_ARG;
+    // ping-pong level outputs (at most d/2 coordinates per point) and the largest level matrix
+    size_t a_elems = 0, mid_elems = 0;
+    for (int i = 1; i <= levels; ++i) {
+        const size_t ki = i < levels ? (size_t)i * k : (size_t)k, ci = i == 1 ? (size_t)2 * k : (size_t)2 * (i - 1) * k;
+        const size_t ri = (size_t)1 << (levels - i);
+        if (ki * ci > a_elems) a_elems = ki * ci;
+        if (i < levels && ri * ki > mid_elems) mid_elems = ri * ki;
+    }
+    if (!grow(ctx->jl_a, a_elems * 2) || (levels > 1 && (!grow(ctx->jl_buf[0], (size_t)n * mid_elems * 2) ||
+                                                          (levels > 2 && !grow(ctx->jl_buf[1], (size_t)n * mid_elems * 2)))))
+        return SIMJOIN_ERR_CUDA;
+    cudaStream_t s = ctx->stream;
+    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    cudaEventRecord(ctx->ev[0], s);
+    cudaEventRecord(ctx->ev[1], s);
+    const void *src = X;
+    for (int i = 1; i <= levels; ++i) {
+        const int ki = i < levels ? i * k : k, ci = i == 1 ? 2 * k : 2 * (i - 1) * k;
+        const int64_t rows = n * ((int64_t)1 << (levels - i));        // n * r_i blocks of c_i coordinates
+        void *dst = i == levels ? out : ctx->jl_buf[(i - 1) & 1].ptr;
+        jl_sign_matrix_kernel<<<(unsigned)(((long long)ki * ci + 255) / 256), 256, 0, s>>>(seed, i, ki, ci,
+                                                                                         reinterpret_cast<uint16_t *>(ctx->jl_a.ptr));
+        if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        // the tile kernel with the level matrix as the resident operand and the blocks as the streamed one
+        JoinParams jp;
+        size_t smem = 0;
+        if (!tile_geometry(ctx, ki, rows, ci * 2, 2, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
+        jp.PB = (ki + TILE_M - 1) / TILE_M;
+        jp.QT = (int)((rows + TILE_N - 1) / TILE_N);
+        jp.qpanel = q_panel_tiles(jp.QT, ci * 2);
+        jp.counter = ctx->d_ctrl;
+        jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
+        jp.store_out = reinterpret_cast<uint16_t *>(dst);
+        jp.store_ld = ki;
+        jp.store_scale = (float)(1.0 / std::sqrt((double)ki));
+        CUtensorMap mapA, mapX;
+        if (!encode_rows_map(ctx, &mapA, ctx->jl_a.ptr, ki, ci, TILE_M) || !encode_rows_map(ctx, &mapX, src, rows, ci, TILE_N))
+            return SIMJOIN_ERR_CUDA;
+        if (launch_join<DT_BF16, KIND_STORE>(ctx, mapA, mapX, jp, ctx->num_sms, smem) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        src = dst;
+    }
+    cudaEventRecord(ctx->ev[2], s);
+    if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    if ((unsigned int)(ctx->h_ctrl[1] & 0xffffffffu) != 0) return SIMJOIN_ERR_TIMEOUT;
+    float b = 0.f;
+    if (cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
+        ctx->prepass_ms = 0.f;
+        ctx->join_ms = b;          // all levels
+        ctx->have_timing = true;
+    }
+    return SIMJOIN_OK;
+}
+
 simjoin_status simjoin_row_norms(simjoin_ctx *ctx, const void *X, int64_t rows, int32_t d, void *out) {
     if (!ctx || !out) return SIMJOIN_ERR_ARG;
     simjoin_status st = check_matrix_args(ctx, X, rows, d);
@@ -675,7 +755,7 @@ struct NoAllocDevice {
     bool ready;
     unsigned char *scratch;   // device address of g_noalloc_scratch on this device
     int sms, smem_optin;
-    bool attr_set[2][3][2][3][2];
+    bool attr_set[2][4][2][3][2];
 };
 NoAllocDevice g_na_dev[NA_MAX_DEVICES];
 EncodeTiledFn g_na_encode = nullptr;
