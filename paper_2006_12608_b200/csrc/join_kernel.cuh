@@ -656,16 +656,29 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
                 if constexpr (KIND == KIND_STORE) {
-                    // lane <-> row of P (an output coordinate), columns <-> rows of Q (output rows): for a
-                    // fixed column the 32 lanes write 32 consecutive bf16 values
+                    // lane <-> row of P (an output coordinate), columns <-> rows of Q (output rows).  The warp's
+                    // 32 x EPI_COLS block is transposed through its 2 KiB of shared memory, 32 columns at a
+                    // time, so that every global store is 16 bytes and 4 lanes cover the 64 contiguous bytes
+                    // that the warp owns of one output row.
                     const long long j0 = q_base + (long long)qt * TILE_N + half * EPI_COLS;
-                    const long long left = q_end - j0;
-                    if (row_ok) {
-                        uint16_t *o = p.store_out + j0 * p.store_ld + i;
+                    uint16_t *sb = reinterpret_cast<uint16_t *>(stage_buf);          // [32 output rows][32 coordinates]
+                    const int i_base = (GROUPED ? un.prow0 : un.pb * TILE_M) + quarter * 32;
 #pragma unroll
-                        for (int c = 0; c < EPI_COLS; ++c)
-                            if (c < left)
-                                o[(long long)c * p.store_ld] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[c]) * p.store_scale));
+                    for (int rnd = 0; rnd < EPI_COLS / 32; ++rnd) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            sb[c * 32 + lane] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[rnd * 32 + c]) * p.store_scale));
+                        __syncwarp();
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const int q = t * 32 + lane, jl = q >> 2, part = q & 3;
+                            const uint4 val = *reinterpret_cast<const uint4 *>(sb + jl * 32 + part * 8);
+                            const long long j = j0 + rnd * 32 + jl;
+                            const int icol = i_base + part * 8;                        // 8 coordinates: all valid or none (k_i % 8 == 0)
+                            if (j < q_end && icol < (int)p.n)
+                                *reinterpret_cast<uint4 *>(p.store_out + j * p.store_ld + icol) = val;
+                        }
+                        __syncwarp();
                     }
                     acc ^= 1;
                     if (acc == 0) accphase ^= 1;

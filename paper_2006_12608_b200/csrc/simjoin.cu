@@ -665,7 +665,7 @@ simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, 
         if (!tile_geometry(ctx, ki, rows, ci * 2, 2, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
         jp.PB = (ki + TILE_M - 1) / TILE_M;
         jp.QT = (int)((rows + TILE_N - 1) / TILE_N);
-        jp.qpanel = q_panel_tiles(jp.QT, ci * 2);
+        jp.qpanel = jp.QT;                 // the blocks are read once: no L2 panels, one long sweep per CTA
         jp.counter = ctx->d_ctrl;
         jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
         jp.store_out = reinterpret_cast<uint16_t *>(dst);
