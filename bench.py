@@ -41,6 +41,10 @@ NOMINAL_TOPS = {"i8": 4500.0, "bf16": 2250.0}          # dense, per GPU (context
 # DRAM bytes per join-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum), from a one-pass ncu
 # capture of the full-size launch (profiles/join_kernel_dram_traffic_cfg4_full.md).
 NCU_TRAFFIC_BYTES = {4: 726.13e6 + 6.28e6}
+# the same for all levels of one JL transform call, keyed by (n, d, k) (profiles/jl_transform_*.md)
+# captured at n = 262144 (1.2956e9 read + 0.6277e9 written); the 1 048 576-point entry is that x 4 (every level's
+# traffic is proportional to n)
+NCU_JL_TRAFFIC_BYTES = {(262144, 1024, 64): 1923.3e6, (1048576, 1024, 64): 4 * 1923.3e6}
 
 
 def measured_peaks():
@@ -158,6 +162,72 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def jl_level_dims(d: int, k: int):
+    """Coordinates per point before level 1 and after every level of the JL transform (zeta = 2)."""
+    levels = int(round(np.log2(d // k)))
+    dims = [d]
+    for i in range(1, levels + 1):
+        dims.append((1 << (levels - i)) * (i * k if i < levels else k))
+    return dims
+
+
+def run_jl(args):
+    """--jl n,d,k: the JL transform of Section 3 (simjoin_jl_transform) on n synthetic bf16 points; HBM-bound.
+    Algorithmic bytes per call: every level reads its input once and writes its output once."""
+    import torch
+    from paper_2006_12608_b200 import binding as B
+    from paper_2006_12608_b200 import build
+    n, d, k = args.jl
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the transform has no CPU path")
+    if not os.path.exists(B.LIB_PATH):
+        build.build()
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device="cuda").manual_seed(2006)
+    X = torch.randn((n, d), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty((n, k), dtype=torch.bfloat16, device="cuda")
+    ctx = B.Simjoin("bf16", 0)
+
+    def step():
+        st = ctx.simjoin_jl_transform(X, n, d, k, 2006, out)
+        if st != B.SIMJOIN_OK:
+            raise RuntimeError(f"simjoin_jl_transform: {B.strerror(st)}")
+
+    for _ in range(args.warmup):
+        step()
+    ratio = float((out.float().norm(dim=1) / X.float().norm(dim=1)).mean())       # JL: close to 1
+    sampler = ClockSampler(0)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    kernel_ms = []
+    e0.record()
+    for _ in range(args.steps):
+        step()
+        kernel_ms.append(ctx.simjoin_last_kernel_ms()[2])
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms_per_step = e0.elapsed_time(e1) / args.steps
+    dims = jl_level_dims(d, k)
+    byts = sum(2.0 * n * (a + b) for a, b in zip(dims, dims[1:]))
+    peaks = measured_peaks()
+    km = statistics.mean(kernel_ms)
+    achieved = byts / (km * 1e-3) / 1e9
+    line = {"metric": "JL transform algorithmic GB/s (level inputs + outputs, bf16)", "value": byts / (ms_per_step * 1e-3) / 1e9,
+            "unit": "GB/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"jl_bf16_{n}x{d}_to_{k}", "n": n, "d": d, "k": k, "levels": len(dims) - 1,
+                       "level_dims": dims, "mean_norm_ratio": ratio, "l2": "input larger than L2; no flush",
+                       "note": "not the headline metric: the dimensionality reduction of Section 3"},
+            "clocks": clocks, "e2e": None, "gpu_launches": 2 * (len(dims) - 1) * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "join_kernel (store epilogue), all levels", "achieved": achieved,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                         "traffic": NCU_JL_TRAFFIC_BYTES.get((n, d, k)), "peak_source": f"{peaks['source']}: copy bandwidth",
+                         "kernel_ms": km, "algorithmic_bytes": byts}}
+    print(json.dumps(line), flush=True)
+
+
 def size_kw(args):
     kw = {}
     if args.n is not None:
@@ -185,7 +255,17 @@ def main():
     ap.add_argument("--lsh", default=None, metavar="L,k[,L_low]",
                     help="time the LSH-bucketed join (int8 inner-product configs) instead of the brute-force join: "
                          "L tables of k bits (+ L_low of k-1); not the headline metric, the line says so")
+    ap.add_argument("--jl", default=None, metavar="n,d,k",
+                    help="time the JL transform (simjoin_jl_transform) of n bf16 points from d to k coordinates instead "
+                         "of the join; HBM-bound, reported in algorithmic GB/s; not the headline metric")
     args = ap.parse_args()
+    if args.jl:
+        args.jl = tuple(int(x) for x in args.jl.split(","))
+        if args.warmup < 3:
+            args.warmup = 3
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_jl(args)
+        return
     args.lsh = tuple(int(x) for x in args.lsh.split(",")) if args.lsh else None
     if args.lsh and args.impl == "reference":
         raise SystemExit("--lsh times the CUDA path only")

@@ -148,9 +148,9 @@ __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
 #ifndef SIMJOIN_ROTATE
 #define SIMJOIN_ROTATE 1
 #endif
-template <bool GROUPED>
+template <bool ALIGNED>
 __device__ __forceinline__ int tile_at(const Unit &un, int k) {
-    if constexpr (GROUPED) return k;
+    if constexpr (ALIGNED) return un.q0 + k;
 #if SIMJOIN_ROTATE
     const int len = un.q1 - un.q0;
     int idx = k + (int)((long long)blockIdx.x * len / gridDim.x);
@@ -472,6 +472,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         p.nstages = fast_nstages(KC, p_bufs(GROUPED, KC));
         p.last_ksteps = 4;
     }
+    // Aligned sweeps (no per-CTA rotation): bucketed units are short, and the store kind reads the streamed
+    // operand once per 128-row block of the resident one -- the CTAs that share a segment then walk it in
+    // step, so that the second reader finds the tile in L2 (measured: rotated, that level read its input twice).
+    constexpr bool ALIGNED = GROUPED || KIND == KIND_STORE;
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128-byte swizzle pattern repeats every 1024 bytes.
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -531,7 +535,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 if (++pbuf == (uint32_t)p_bufs(GROUPED, kc)) { pbuf = 0; pphase ^= 1; }
             }
             for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
-                const int q_row = (GROUPED ? un.qrow0 : 0) + tile_at<GROUPED>(un, k) * TILE_N;
+                const int q_row = (GROUPED ? un.qrow0 : 0) + tile_at<ALIGNED>(un, k) * TILE_N;
                 for (int c = 0; c < p.kc; ++c) {
                     ok = wait_bar_warp(&ctrl->empty[stage], phase ^ 1, ctrl, p.status, 2);
                     if (!ok) break;
@@ -599,7 +603,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) rf = reinterpret_cast<const float *>(p.nx)[i];
             }
             for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
-                const int qt = tile_at<GROUPED>(un, k);
+                const int qt = tile_at<ALIGNED>(un, k);
                 // per-tile filter bound: a necessary condition on max_j s_ij for row i to have any hit
                 int fi = p.thr_i;
                 float ff = p.thr_f;
