@@ -109,3 +109,64 @@ def test_full_size_cfg5_literal_sigma_is_empty():
     w = W.make_workload(5, sigma_reading="percoord")
     pairs, cnt = run_full(w, capacity=1 << 16)
     assert cnt == 0
+
+
+def test_full_size_lsh_join_cfg4():
+    """The LSH-bucketed join at the headline size (1 048 576 x 1 048 576, 8 tables of 7 bits), as `bench.py --lsh 8,7`
+    times it.  The result is the set {brute-force pairs whose keys agree in some table}: every emitted pair is scored
+    by the oracle and its keys (the oracle's) agree in a table; nothing is emitted twice; every planted pair whose
+    oracle keys agree in a table is present, and only those; sampled rows are joined whole by the oracle."""
+    L, k, seed = 8, 7, 2006
+    w = W.make_workload(4)
+    build.build()
+    cap = 4 * len(w.planted)
+    with B.Simjoin("i8", 0) as ctx:
+        dP, dQ = B.to_device(w.P), B.to_device(w.Q)
+        out = torch.empty((cap, 2), dtype=torch.int32, device="cuda:0")
+        st, cnt = ctx.simjoin_run_lsh(dP, w.n, dQ, w.m, w.d, w.threshold, L, k, seed, out, cap)
+        assert st == B.SIMJOIN_OK, B.strerror(st)
+        pairs = out[:cnt].cpu().numpy().astype(np.int64)
+    del dP, dQ, out
+    torch.cuda.empty_cache()
+    gk = keys(pairs)
+    assert len(np.unique(gk)) == cnt
+    assert np.all(O.scores(w.P, w.Q, "ip", "i8", pairs.astype(np.int32)) >= w.threshold)
+    kp, kq = O.lsh_keys(w.P, L, k, seed), O.lsh_keys(w.Q, L, k, seed)          # (L, rows)
+    assert np.all((kp[:, pairs[:, 0]] == kq[:, pairs[:, 1]]).any(axis=0))      # every emitted pair collides in a table
+    pl = w.planted
+    collide = (kp[:, pl[:, 0]] == kq[:, pl[:, 1]]).any(axis=0)
+    assert np.array_equal(np.isin(keys(pl), gk), collide)                      # planted pairs: present iff they collide
+    assert collide.mean() > 0.999                                              # closed form: 1 - (1 - (120/128)^7)^8 = 0.9997
+    rows = sample_rows(w, pairs, k=24)
+    sub_keys = kp[:, rows]
+    want, _c = O.join(w.P[rows], w.Q, "ip", w.threshold, "i8")                 # brute force on the sampled rows ...
+    keep = (sub_keys[:, want[:, 0]] == kq[:, want[:, 1]]).any(axis=0)          # ... restricted to colliding pairs
+    want = want[keep].astype(np.int64)
+    want[:, 0] = np.asarray(rows)[want[:, 0]]
+    got = pairs[np.isin(pairs[:, 0], rows)]
+    assert np.array_equal(np.sort(keys(got)), np.sort(keys(want)))
+
+
+def test_full_size_jl_transform_sampled_rows():
+    """The JL transform at the size `bench.py --jl 1048576,1024,64` times: sampled rows against the fp64 oracle, within
+    the bound derived from the per-level bf16 rounding (see tests/test_gpu_jl.py)."""
+    n, d, k, seed = 1 << 20, 1024, 64, 2006
+    build.build()
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    X = torch.randn((n, d), generator=gen, device="cuda:0", dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty((n, k), dtype=torch.bfloat16, device="cuda:0")
+    with B.Simjoin("bf16", 0) as ctx:
+        assert ctx.simjoin_jl_transform(X, n, d, k, seed, out) == B.SIMJOIN_OK
+    rows = np.unique(np.concatenate([np.random.default_rng(5).choice(n, size=60, replace=False), [0, 127, 128, 255, 256, n - 1]]))
+    rows_t = torch.from_numpy(rows).cuda()
+    Xs = X[rows_t].view(torch.int16).cpu().numpy().view(np.uint16)
+    got = out[rows_t].float().cpu().numpy().astype(np.float64)
+    del X, out
+    torch.cuda.empty_cache()
+    want = O.jl_transform(np.ascontiguousarray(Xs), k, seed)
+    sh = O.jl_shapes(d, k)
+    xn = np.linalg.norm(W.bf16_bits_to_f32(Xs).astype(np.float64), axis=1)
+    bound = 2.0 ** -9 * xn * (1.5 * sum(np.sqrt(c / ki) for _r, c, ki in sh) + 1.0)
+    err = np.abs(got - want)
+    assert np.all(err <= bound[:, None]), (err.max(), bound.min())
+    assert np.sqrt((err ** 2).mean()) <= 4.0 * np.sqrt(len(sh)) * 2.0 ** -9 * np.sqrt((want ** 2).mean()) / np.sqrt(3.0)
