@@ -32,12 +32,24 @@ constexpr int KIND_IP = 0, KIND_COS = 1, KIND_L2 = 2;
 // small, resident operand: one level of the JL transform of Section 3.
 constexpr int KIND_STORE = 3;
 
-constexpr int TILE_M = 128;                       // rows of P per tile
-constexpr int TILE_N = 256;                       // rows of Q per tile
+// One tile is 256 rows of P (two 128-row MMA blocks, both resident in shared memory) against 128 rows of Q.
+// Every Q chunk that arrives is multiplied with both P blocks, so a tile needs half the L2 -> shared-memory
+// traffic of a 128 x 256 tile for the same work.  Measured on B200 under the 1000 W cap with a skeleton of
+// this pipeline: streaming 32 KiB per 512 tensor cycles costs 16 % of the SM clock (1400 vs 1630 MHz with
+// the traffic switched off); at 16 KiB it costs 7 % (1505 MHz) -- the kernel is power-bound, so energy per
+// tile, not cycles per tile, sets its speed.  (tcgen05.mma with N = 128 issues in 69 cycles against 64
+// ideal: the tile takes 552 cycles instead of 549.)
+constexpr int TILE_M = 128;                       // rows of P per MMA block (TMEM lanes)
+constexpr int P_SUB = 2;                          // MMA blocks per P tile
+constexpr int P_ROWS = P_SUB * TILE_M;            // rows of P per tile
+constexpr int TILE_N = 128;                       // rows of Q per tile
+constexpr int QSTAT_ROWS = 256;                   // rows of Q behind one (min, max) entry of the per-tile bound: two tiles
+constexpr int ACC_COLS = P_SUB * TILE_N;          // TMEM columns of one accumulator buffer: block s at s * TILE_N
 constexpr int CHUNK_BYTES = 128;                  // K bytes per shared-memory chunk (one swizzle atom)
-constexpr int A_CHUNK_BYTES = TILE_M * CHUNK_BYTES;   // 16 KiB
-constexpr int B_CHUNK_BYTES = TILE_N * CHUNK_BYTES;   // 32 KiB
-constexpr int MAX_STAGES = 6;
+constexpr int A_CHUNK_BYTES = P_ROWS * CHUNK_BYTES;   // 32 KiB: one K chunk of both P blocks (block s at s * 16 KiB)
+constexpr int A_SUB_BYTES = TILE_M * CHUNK_BYTES;     // 16 KiB
+constexpr int B_CHUNK_BYTES = TILE_N * CHUNK_BYTES;   // 16 KiB
+constexpr int MAX_STAGES = 8;
 constexpr int MAX_STATIONARY_CHUNKS = 4;          // P block kept resident up to 512-byte rows
 #ifndef SIMJOIN_P_BUFS
 #define SIMJOIN_P_BUFS 1
@@ -51,8 +63,9 @@ constexpr int EPI_WARP0 = 4;
 #ifndef SIMJOIN_EPI_WARPS
 #define SIMJOIN_EPI_WARPS 8
 #endif
-constexpr int NUM_EPI_WARPS = SIMJOIN_EPI_WARPS;               // 8 or 16: 2 or 4 per TMEM lane quarter
-constexpr int EPI_COLS = TILE_N / (NUM_EPI_WARPS / 4);         // accumulator columns per epilogue warp
+constexpr int NUM_EPI_WARPS = SIMJOIN_EPI_WARPS;               // 4 TMEM lane quarters x P_SUB blocks
+static_assert(NUM_EPI_WARPS == 4 * P_SUB, "one epilogue warp per TMEM lane quarter and P block");
+constexpr int EPI_COLS = TILE_N;                               // accumulator columns per epilogue warp
 constexpr int NUM_THREADS = 32 * (EPI_WARP0 + NUM_EPI_WARPS);
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;  // ~1 s: far beyond any legitimate wait
@@ -107,7 +120,9 @@ static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
 // One unit of work: P block `pb` against Q tiles [q0, q1).  Q is cut into panels of `qpanel` tiles
 // that fit in L2; within a panel CTAs take whole sweeps in waves of gridDim.x P blocks (all CTAs
 // then walk the panel together, so a Q tile is fetched from HBM once and served from L2 to everyone
-// else, wave after wave); the last, partial wave of a panel splits each of its sweeps over several CTAs.
+// else, wave after wave); the last, partial wave of a panel lays its `rem` sweeps end to end and cuts them
+// into gridDim.x equal runs, so every CTA gets the same number of tiles (a run that crosses from one sweep
+// into the next becomes two units).
 struct Unit {
     int pb, q0, q1;
     int prow0, prows, qrow0, qrows;   // bucketed mode only
@@ -127,18 +142,28 @@ __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
         return true;
     }
     const int full = p.PB / G, rem = p.PB - full * G;
-    const int per_panel = full + (rem > 0 ? 1 : 0);
+    const int per_panel = full + (rem > 0 ? 2 : 0);
     const int panel = u / per_panel, v = u - panel * per_panel;
     const int pq0 = panel * p.qpanel;
     if (pq0 >= p.QT) return false;
     const int pq1 = min(pq0 + p.qpanel, p.QT);
     if (v < full) { un.pb = v * G + c; un.q0 = pq0; un.q1 = pq1; return true; }
-    // v == full, rem > 0: the partial wave
-    const int S = G / rem, idx = c / S, seg = c - idx * S;
-    un.pb = full * G + (idx < rem ? idx : 0);
+    // v == full or full + 1, rem > 0: the partial wave.  This CTA's run is [t0, t1) of the rem * len tiles;
+    // it lies in sweep t0 / len and, if it crosses the sweep's end, in the next one (rem <= G: never further).
     const int len = pq1 - pq0;
-    un.q0 = pq0 + (int)((long long)seg * len / S);
-    un.q1 = idx < rem ? pq0 + (int)((long long)(seg + 1) * len / S) : un.q0;   // empty for spare CTAs
+    const long long T = (long long)rem * len;
+    const long long t0 = T * c / G, t1 = T * (c + 1) / G;
+    const int sweep = (int)(t0 / len);
+    const long long cut = min(t1, (long long)(sweep + 1) * len);
+    if (v == full) {
+        un.pb = full * G + sweep;
+        un.q0 = pq0 + (int)(t0 - (long long)sweep * len);
+        un.q1 = pq0 + (int)(cut - (long long)sweep * len);
+    } else {
+        un.pb = full * G + (cut < t1 ? sweep + 1 : sweep);
+        un.q0 = pq0;
+        un.q1 = pq0 + (int)(t1 - cut);                          // empty unless the run crossed into the next sweep
+    }
     return true;
 }
 
@@ -367,11 +392,43 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     __syncwarp();
 }
 
+// Store epilogue (KIND_STORE) of one warp: NC accumulator columns (rows of Q = output rows j_first ..) of its 32
+// TMEM lanes (rows of P = output coordinates i_base ..) are scaled, rounded to bf16 and transposed through the
+// warp's 2 KiB of shared memory, 32 columns at a time, so that every global store is 16 bytes and 4 lanes cover
+// the 64 contiguous bytes the warp owns of one output row.
+template <int NC>
+__device__ __forceinline__ void store_tile_part(const JoinParams &p, uint32_t taddr, uint64_t *tempty_bar, int lane, uint16_t *sb,
+                                                long long j_first, long long q_end, int i_base) {
+    uint32_t v[NC];
+    tmem_ld_words(taddr, v, std::false_type{});
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(tempty_bar));
+#pragma unroll
+    for (int rnd = 0; rnd < NC / 32; ++rnd) {
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+            sb[c * 32 + lane] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[rnd * 32 + c]) * p.store_scale));
+        __syncwarp();
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int q = t * 32 + lane, jl = q >> 2, part = q & 3;
+            const uint4 val = *reinterpret_cast<const uint4 *>(sb + jl * 32 + part * 8);
+            const long long j = j_first + rnd * 32 + jl;
+            const int icol = i_base + part * 8;                        // 8 coordinates: all valid or none (k_i % 8 == 0)
+            if (j < q_end && icol < (int)p.n) *reinterpret_cast<uint4 *>(p.store_out + j * p.store_ld + icol) = val;
+        }
+        __syncwarp();
+    }
+}
+
 // The MMA-issuing role (warps 1 and 3).  KC > 0 is a fast path with the chunks per tile known at
 // compile time (resident P block, full 128-byte chunks, two issuers): measured on B200, a chunk loop
 // with a run-time trip count around the tcgen05.mma issues costs ~80 cycles per tile, the run-time
 // operand-address select another ~25.  KC == 0 is the general path.
-template <int DT, int KC, bool GROUPED>
+// ONE_BLOCK_OK: a tile whose second P block lies wholly past the end of P skips that block's MMAs (the store
+// kind, whose resident operand often has <= 128 rows; the join kinds keep the branch out of their issue loop).
+template <int DT, int KC, bool GROUPED, bool ONE_BLOCK_OK>
 __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl, uint8_t *smem_p, uint8_t *smem_ring,
                                                 const int stage_bytes_rt, const uint32_t tmem_base, const int warp, const int lane) {
     constexpr bool FAST = KC > 0;
@@ -392,6 +449,7 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
             ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
             if (!ok) break;
         }
+        const bool two = !ONE_BLOCK_OK || (GROUPED ? un.prows > TILE_M : (long long)un.pb * P_ROWS + TILE_M < p.n);
         for (int k = 0; ok && k < un.q1 - un.q0; ++k, tsel ^= 1) {
             if (dual && tsel != mid) {
                 // the other issuer's tile: step over its chunks in the ring
@@ -400,7 +458,7 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
                 continue;
             }
             const uint32_t a = tsel;                       // accumulator of this tile
-            const uint32_t d_tmem = tmem_base + a * TILE_N;
+            const uint32_t d_tmem = tmem_base + a * ACC_COLS;
             ok = wait_bar_warp(&ctrl->tempty[a], (a ? accph1 : accph0) ^ 1, ctrl, p.status, 4);
             if (!ok) break;
 #pragma unroll
@@ -413,15 +471,23 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
                 uint8_t *sb = smem_ring + (size_t)stage * stage_bytes;
                 const uint32_t a_addr = stationary ? smem_u32(smem_p + (size_t)(pbuf * kc + c) * A_CHUNK_BYTES)
                                                    : smem_u32(sb + B_CHUNK_BYTES);
-                const uint64_t adesc = umma_desc_sw128_kmajor(a_addr);
+                const uint64_t adesc = umma_desc_sw128_kmajor(a_addr);                       // P block 0
+                const uint64_t adesc1 = umma_desc_sw128_kmajor(a_addr + A_SUB_BYTES);        // P block 1
                 const uint64_t bdesc = umma_desc_sw128_kmajor(smem_u32(sb));
                 const bool last_chunk = c == kc - 1;
                 const int ksteps = FAST ? 4 : (last_chunk ? p.last_ksteps : 4);
                 if (elect_one()) {
+                    // the Q chunk against both resident P blocks: block s accumulates in columns s * TILE_N ..
                     umma_ss<DT == DT_I8>(d_tmem, adesc, bdesc, idesc, c != 0 ? 1u : 0u);
                     if (ksteps > 1) umma_ss<DT == DT_I8>(d_tmem, adesc + 2, bdesc + 2, idesc, 1u);
                     if (ksteps > 2) umma_ss<DT == DT_I8>(d_tmem, adesc + 4, bdesc + 4, idesc, 1u);
                     if (ksteps > 3) umma_ss<DT == DT_I8>(d_tmem, adesc + 6, bdesc + 6, idesc, 1u);
+                    if (two) {
+                        umma_ss<DT == DT_I8>(d_tmem + TILE_N, adesc1, bdesc, idesc, c != 0 ? 1u : 0u);
+                        if (ksteps > 1) umma_ss<DT == DT_I8>(d_tmem + TILE_N, adesc1 + 2, bdesc + 2, idesc, 1u);
+                        if (ksteps > 2) umma_ss<DT == DT_I8>(d_tmem + TILE_N, adesc1 + 4, bdesc + 4, idesc, 1u);
+                        if (ksteps > 3) umma_ss<DT == DT_I8>(d_tmem + TILE_N, adesc1 + 6, bdesc + 6, idesc, 1u);
+                    }
                     if (!epi_release) umma_commit(smem_u32(&ctrl->empty[stage]));
                     if (last_chunk) umma_commit(smem_u32(&ctrl->tfull[a]));
                 }
@@ -520,7 +586,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         Unit un;
         for (int u = 0; ok && get_unit<GROUPED>(p, u, un); ++u) {
             if (un.q1 <= un.q0) continue;            // nothing for this CTA in this wave (all roles skip it)
-            const int p_row = GROUPED ? un.prow0 : un.pb * TILE_M;
+            const int p_row = GROUPED ? un.prow0 : un.pb * P_ROWS;
             if (p.stationary) {
                 ok = wait_bar_warp(&ctrl->pempty[pbuf], pphase ^ 1, ctrl, p.status, 1);
                 if (!ok) break;
@@ -571,14 +637,15 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         // barrier that is still one phase behind, and a parity wait cannot tell phases two apart.
         // In that case warp 1 issues every tile and warp 3 stays out.
         const bool fast = p.stationary && p.epi_release && p.last_ksteps == 4;
-        if (fast && p.kc == 1) mma_issuer_role<DT, 1, GROUPED>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
-        else if (fast && p.kc == 2) mma_issuer_role<DT, 2, GROUPED>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
-        else mma_issuer_role<DT, 0, GROUPED>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        constexpr bool OB = KIND == KIND_STORE;
+        if (fast && p.kc == 1) mma_issuer_role<DT, 1, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        else if (fast && p.kc == 2) mma_issuer_role<DT, 2, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        else mma_issuer_role<DT, 0, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
     } else if (warp >= EPI_WARP0) {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
-        const int half = (warp - EPI_WARP0) >> 2;   // which EPI_COLS-wide slice of the tile's 256 columns
-        const int row_in_tile = quarter * 32 + lane;
+        const int half = (warp - EPI_WARP0) >> 2;   // which of the tile's two P blocks (accumulator columns half * TILE_N ..)
+        const int row_in_tile = half * TILE_M + quarter * 32 + lane;
         uint32_t acc = 0, accphase = 0, rstage = 0;   // rstage: next ring stage to hand back
         int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * STAGE_PAIRS;
         int stage_fill = 0;
@@ -586,8 +653,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         Unit un;
         for (int u = 0; ok && get_unit<GROUPED>(p, u, un); ++u) {
             if (un.q1 <= un.q0) continue;
-            const long long i = GROUPED ? (long long)un.prow0 + row_in_tile : (long long)un.pb * TILE_M + row_in_tile;
+            const long long i = GROUPED ? (long long)un.prow0 + row_in_tile : (long long)un.pb * P_ROWS + row_in_tile;
             const bool row_ok = GROUPED ? row_in_tile < un.prows : i < p.n;
+            const bool two_blocks = GROUPED ? un.prows > TILE_M : (long long)un.pb * P_ROWS + TILE_M < p.n;
             const long long q_base = GROUPED ? un.qrow0 : 0;                          // Q row of tile 0
             const long long q_end = GROUPED ? (long long)un.qrow0 + un.qrows : p.m;   // end of the Q rows of this unit
             int ri = 0;          // I8/L2: |x|^2 - floor(r^2)
@@ -608,15 +676,15 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 int fi = p.thr_i;
                 float ff = p.thr_f;
                 if constexpr (DT == DT_I8 && KIND == KIND_L2) {
-                    const int2 st = reinterpret_cast<const int2 *>(p.qstat)[qt];
+                    const int2 st = reinterpret_cast<const int2 *>(p.qstat)[qt / (QSTAT_ROWS / TILE_N)];
                     fi = (ri + st.x + 1) >> 1;                    // 2s >= |x|^2 - R + min|y|^2
                 }
                 if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
-                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt];
+                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt / (QSTAT_ROWS / TILE_N)];
                     ff = rf * (p.thr_f >= 0.f ? st.x : st.y);     // s >= t|x| * min|y| (max|y| when t < 0)
                 }
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
-                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt];
+                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt / (QSTAT_ROWS / TILE_N)];
                     ff = rf + st.x;                               // (|x|^2 + min|y|^2) - 2s <= r^2
                 }
                 // per-column terms of this warp's columns, 4 per lane, fetched while the tile is still
@@ -624,7 +692,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 uint4 yq = make_uint4(0, 0, 0, 0);
                 if ((KIND == KIND_COS || KIND == KIND_L2) && lane < EPI_COLS / 4)
                     yq = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint32_t *>(p.ny) +
-                                                               ((long long)qt * TILE_N + half * EPI_COLS)) + lane);
+                                                               (long long)qt * TILE_N) + lane);
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
                 if (!ok) break;
                 tc_fence_after();
@@ -650,44 +718,31 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     }
                     __syncwarp();
                 }
+                if constexpr (KIND == KIND_STORE) {
+                    // lane <-> row of P (an output coordinate), columns <-> rows of Q (output rows).  With two P
+                    // blocks in the tile this warp stores block `half`; with one, the two warps of a lane quarter
+                    // split that block's 128 columns between them.
+                    const long long j0 = q_base + (long long)qt * TILE_N;
+                    uint16_t *sb = reinterpret_cast<uint16_t *>(stage_buf);          // [32 output rows][32 coordinates]
+                    const int i_unit = (GROUPED ? un.prow0 : un.pb * P_ROWS) + quarter * 32;
+                    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS;
+                    if (two_blocks)
+                        store_tile_part<TILE_N>(p, t_lane + half * TILE_N, &ctrl->tempty[acc], lane, sb, j0, q_end, i_unit + half * TILE_M);
+                    else
+                        store_tile_part<TILE_N / 2>(p, t_lane + half * (TILE_N / 2), &ctrl->tempty[acc], lane, sb, j0 + half * (TILE_N / 2), q_end, i_unit);
+                    acc ^= 1;
+                    if (acc == 0) accphase ^= 1;
+                    continue;
+                }
                 // this warp's 128 columns of the tile, then hand the accumulator back to the MMA warp
                 constexpr int NV = NARROW ? EPI_COLS / 2 : EPI_COLS;      // accumulator words per thread
                 constexpr int GCOLS = 16, NG = EPI_COLS / GCOLS, GW = NV / NG;  // groups of 16 columns
                 constexpr int MODE = DT == DT_BF16 ? MAX_F32 : (NARROW ? MAX_S16X2 : MAX_S32);
                 uint32_t v[NV];
-                tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * TILE_N + half * EPI_COLS, v, std::integral_constant<bool, NARROW>{});
+                tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TILE_N, v, std::integral_constant<bool, NARROW>{});
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
-                if constexpr (KIND == KIND_STORE) {
-                    // lane <-> row of P (an output coordinate), columns <-> rows of Q (output rows).  The warp's
-                    // 32 x EPI_COLS block is transposed through its 2 KiB of shared memory, 32 columns at a
-                    // time, so that every global store is 16 bytes and 4 lanes cover the 64 contiguous bytes
-                    // that the warp owns of one output row.
-                    const long long j0 = q_base + (long long)qt * TILE_N + half * EPI_COLS;
-                    uint16_t *sb = reinterpret_cast<uint16_t *>(stage_buf);          // [32 output rows][32 coordinates]
-                    const int i_base = (GROUPED ? un.prow0 : un.pb * TILE_M) + quarter * 32;
-#pragma unroll
-                    for (int rnd = 0; rnd < EPI_COLS / 32; ++rnd) {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            sb[c * 32 + lane] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[rnd * 32 + c]) * p.store_scale));
-                        __syncwarp();
-#pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            const int q = t * 32 + lane, jl = q >> 2, part = q & 3;
-                            const uint4 val = *reinterpret_cast<const uint4 *>(sb + jl * 32 + part * 8);
-                            const long long j = j0 + rnd * 32 + jl;
-                            const int icol = i_base + part * 8;                        // 8 coordinates: all valid or none (k_i % 8 == 0)
-                            if (j < q_end && icol < (int)p.n)
-                                *reinterpret_cast<uint4 *>(p.store_out + j * p.store_ld + icol) = val;
-                        }
-                        __syncwarp();
-                    }
-                    acc ^= 1;
-                    if (acc == 0) accphase ^= 1;
-                    continue;
-                }
                 // level 0: the row maximum over this warp's 128 columns against the per-tile bound
                 // (a necessary condition of the exact test, in the same arithmetic)
                 auto bound_ok = [&](uint32_t word) -> bool {
@@ -707,7 +762,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
 #pragma unroll
                     for (int k = 0; k < NG; ++k) gm |= (bound_ok(TreeMax<GW, MODE>::run(v + k * GW)) ? 1u : 0u) << k;
                     if (!row_ok) gm = 0;
-                    const long long j0 = q_base + (long long)qt * TILE_N + half * EPI_COLS;
+                    const long long j0 = q_base + (long long)qt * TILE_N;
                     uint32_t mask[EPI_COLS / 32];
 #pragma unroll
                     for (int q = 0; q < EPI_COLS / 32; ++q) mask[q] = 0;

@@ -16,6 +16,8 @@
 #include "lsh_kernel.cuh"
 #include "prepass_kernel.cuh"
 
+static_assert(sj::QSTAT_ROWS == sj::NORM_TILE_ROWS, "the join kernel indexes the per-tile bounds by 256-row blocks");
+
 namespace {
 
 using namespace sj;
@@ -228,7 +230,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     JoinParams jp;
     size_t smem = 0;
     if (!tile_geometry(ctx, n, m, row_bytes, es, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
-    jp.PB = (int)((n + TILE_M - 1) / TILE_M);
+    jp.PB = (int)((n + P_ROWS - 1) / P_ROWS);
     jp.QT = (int)((m + TILE_N - 1) / TILE_N);
     jp.qpanel = q_panel_tiles(jp.QT, row_bytes);
     jp.out = reinterpret_cast<int2 *>(out_pairs);
@@ -260,7 +262,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     }
 
     CUtensorMap mapP, mapQ;
-    if (!encode_rows_map(ctx, &mapP, P, n, d, TILE_M) || !encode_rows_map(ctx, &mapQ, Q, m, d, TILE_N))
+    if (!encode_rows_map(ctx, &mapP, P, n, d, P_ROWS) || !encode_rows_map(ctx, &mapQ, Q, m, d, TILE_N))
         return SIMJOIN_ERR_CUDA;
 
     cudaStream_t s = ctx->stream;
@@ -510,7 +512,7 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     size_t smem = 0;
     if (!tile_geometry(ctx, n, m, d, 1, jp, smem, true)) return SIMJOIN_ERR_UNSUPPORTED;
     const int nb_max = 1 << k;
-    const size_t max_units = (size_t)((n + TILE_M - 1) / TILE_M) + (size_t)nb_max;
+    const size_t max_units = (size_t)((n + P_ROWS - 1) / P_ROWS) + (size_t)nb_max;
     // misc: hist_p | hist_q | cursor_p | cursor_q (nb words each) | nunits (padded to 16 B) | units
     const size_t off_units = ((size_t)4 * nb_max * 4 + 16 + 15) & ~(size_t)15;
     const int reps = L + L_low;
@@ -544,7 +546,7 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     jp.rec_words = rec_words;
 
     CUtensorMap mapP, mapQ;
-    if (!encode_rows_map(ctx, &mapP, ctx->lsh_sorted_p.ptr, n, d, TILE_M) ||
+    if (!encode_rows_map(ctx, &mapP, ctx->lsh_sorted_p.ptr, n, d, P_ROWS) ||
         !encode_rows_map(ctx, &mapQ, ctx->lsh_sorted_q.ptr, m, d, TILE_N))
         return SIMJOIN_ERR_CUDA;
 
@@ -579,7 +581,7 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
         if (cudaMemsetAsync(hist_p, 0, (size_t)2 * nb_max * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
         lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kp, stride, n, nb, hist_p);
         lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kq, stride, m, nb, hist_q);
-        lsh_offsets_units_kernel<<<1, 1024, 0, s>>>(hist_p, hist_q, nb, cursor_p, cursor_q, units, nunits, TILE_M);
+        lsh_offsets_units_kernel<<<1, 1024, 0, s>>>(hist_p, hist_q, nb, cursor_p, cursor_q, units, nunits, P_ROWS);
         lsh_scatter_kernel<<<(unsigned)((n + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kp, stride, n, nb,
                                                                                                               cursor_p, perm_p);
         lsh_scatter_kernel<<<(unsigned)((m + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kq, stride, m, nb,
@@ -663,7 +665,7 @@ simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, 
         JoinParams jp;
         size_t smem = 0;
         if (!tile_geometry(ctx, ki, rows, ci * 2, 2, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
-        jp.PB = (ki + TILE_M - 1) / TILE_M;
+        jp.PB = (ki + P_ROWS - 1) / P_ROWS;
         jp.QT = (int)((rows + TILE_N - 1) / TILE_N);
         jp.qpanel = jp.QT;                 // the blocks are read once: no L2 panels, one long sweep per CTA
         jp.counter = ctx->d_ctrl;
@@ -672,7 +674,7 @@ simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, 
         jp.store_ld = ki;
         jp.store_scale = (float)(1.0 / std::sqrt((double)ki));
         CUtensorMap mapA, mapX;
-        if (!encode_rows_map(ctx, &mapA, ctx->jl_a.ptr, ki, ci, TILE_M) || !encode_rows_map(ctx, &mapX, src, rows, ci, TILE_N))
+        if (!encode_rows_map(ctx, &mapA, ctx->jl_a.ptr, ki, ci, P_ROWS) || !encode_rows_map(ctx, &mapX, src, rows, ci, TILE_N))
             return SIMJOIN_ERR_CUDA;
         if (launch_join<DT_BF16, KIND_STORE>(ctx, mapA, mapX, jp, ctx->num_sms, smem) != cudaSuccess) return SIMJOIN_ERR_CUDA;
         src = dst;
@@ -849,7 +851,7 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     jp.nstages = nstages;
     jp.epi_release = (jp.stationary && nstages >= 2 * jp.kc) ? 1 : 0;
     const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + STAGING_BYTES + CTRL_BYTES;
-    jp.PB = (int)((n + TILE_M - 1) / TILE_M);
+    jp.PB = (int)((n + P_ROWS - 1) / P_ROWS);
     jp.QT = (int)((m + TILE_N - 1) / TILE_N);
     jp.qpanel = q_panel_tiles(jp.QT, row_bytes);
     jp.out = reinterpret_cast<int2 *>(out_pairs);
@@ -871,7 +873,7 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     jp.qstat = nd.scratch + NA_OFF_QSTAT;
 
     CUtensorMap mapP, mapQ;
-    if (!encode_rows_map(&tmp, &mapP, P, n, d, TILE_M) || !encode_rows_map(&tmp, &mapQ, Q, m, d, TILE_N))
+    if (!encode_rows_map(&tmp, &mapP, P, n, d, P_ROWS) || !encode_rows_map(&tmp, &mapQ, Q, m, d, TILE_N))
         return SIMJOIN_ERR_CUDA;
     cudaStream_t s = tmp.stream;
     // the array keeps the previous call's contents: the counter / status block must start at zero
