@@ -2,17 +2,17 @@
 //
 // Section 4 of the paper reduces the join to the product F_P * G_Q^T and Theorem 1
 // decomposes that product into small dense tile products.  Here one tile product is a
-// 128 x 256 block of scores: 128 rows of P against 256 rows of Q over all d coordinates,
-// computed by tcgen05.mma from 128-byte-swizzled shared-memory tiles that TMA fills, with
+// 256 x 128 block of scores: 256 rows of P (two 128-row MMA blocks) against 128 rows of Q over
+// all d coordinates, computed by tcgen05.mma from 128-byte-swizzled shared-memory tiles that TMA fills, with
 // the accumulator in tensor memory.  The rest of the ip-distance (row norms, Section 4's
 // squared-L2 and cosine forms) and the threshold are applied to the accumulator in
 // registers and passing (i, j) are compacted straight into the output list.
 //
 // CTA layout (384 threads, one CTA per SM, persistent):
-//   warp 0      TMA producer (one thread): P row block (resident while its Q sweep lasts) + Q chunk ring
+//   warp 0      TMA producer (one elected lane): P tile (resident while its Q sweep lasts) + Q chunk ring
 //   warps 1, 3  MMA issuers: warp 1 even tiles -> accumulator 0, warp 3 odd tiles -> accumulator 1
 //   warp 2      TMEM allocation / release
-//   warps 4-11  epilogue: warp w reads TMEM lanes 32*(w%4).., column half (w-4)/4; row max vs a
+//   warps 4-11  epilogue: warp w reads TMEM lanes 32*(w%4).. of P block (w-4)/4; row max vs a
 //               per-tile bound, then 16-column group maxima, then the exact test; passing pairs go
 //               through a per-warp shared-memory staging buffer to the output list
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word and drains.
@@ -81,13 +81,13 @@ struct JoinParams {
     int stationary;          // 1: the P block stays in shared memory for its whole Q sweep
     int nstages;             // ring depth
     int epi_release;         // 1: the epilogue hands ring stages back (one commit per tile); needs nstages >= 2*kc
-    int PB, QT;              // number of 128-row P blocks, 256-row Q tiles
+    int PB, QT;              // number of 256-row P tiles, 128-row Q tiles
     int qpanel;              // Q tiles per L2-resident panel
     int thr_i;               // I8/IP: ceil(t);  I8/L2: floor(r*r); both clamped
     float thr_f;             // BF16: t (IP, COS) or r*r (L2)
     const void *nx;          // per-row term of P: int32 |x|^2 (I8/L2), fp32 |x| (COS) or |x|^2 (L2)
     const void *ny;          // same for Q
-    const void *qstat;       // per 256-row Q tile: (min, max) of ny over the tile's valid rows
+    const void *qstat;       // per 256 rows of Q (two tiles): (min, max) of ny over the valid rows
     int2 *out;               // capacity x (i, j)
     unsigned long long capacity;
     unsigned long long *counter;   // total passing pairs
@@ -539,7 +539,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         p.last_ksteps = 4;
     }
     // Aligned sweeps (no per-CTA rotation): bucketed units are short, and the store kind reads the streamed
-    // operand once per 128-row block of the resident one -- the CTAs that share a segment then walk it in
+    // operand once per 256-row tile of the resident one -- the CTAs that share a segment then walk it in
     // step, so that the second reader finds the tile in L2 (measured: rotated, that level read its input twice).
     constexpr bool ALIGNED = GROUPED || KIND == KIND_STORE;
     extern __shared__ uint8_t smem_raw[];

@@ -97,7 +97,7 @@ __device__ __forceinline__ unsigned int block_scan4(unsigned int (&v)[4], unsign
 }
 
 // One block: bucket offsets of P and Q (exclusive scans of the histograms; also copied to the scatter
-// cursors) and the work list -- for every bucket that holds points of both sets, one unit per 128-row
+// cursors) and the work list -- for every bucket that holds points of both sets, one unit per rows_per_unit-row
 // block of its P rows, each against all of the bucket's Q rows.  Units of a bucket are adjacent.
 __global__ void __launch_bounds__(1024) lsh_offsets_units_kernel(const unsigned int *__restrict__ hist_p,
                                                                  const unsigned int *__restrict__ hist_q, int nb,

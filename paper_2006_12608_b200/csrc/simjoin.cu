@@ -253,7 +253,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
 
     const bool need_norms = kind != SIMJOIN_IP;
     if (need_norms) {
-        // ny is read in 16-entry groups up to the end of the last 256-row tile: pad it to whole tiles
+        // ny is read in 16-entry groups up to the end of the last Q tile: pad it to whole tiles
         if (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, (size_t)jp.QT * TILE_N * 4) || !grow(ctx->qstat, (size_t)jp.QT * 8))
             return SIMJOIN_ERR_CUDA;
         jp.nx = ctx->nx.ptr;
