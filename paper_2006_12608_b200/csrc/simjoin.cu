@@ -217,6 +217,19 @@ bool tile_geometry(const simjoin_ctx *ctx, int64_t n, int64_t m, int row_bytes, 
     return true;
 }
 
+// Thresholds in the precision each path decides in.
+void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold) {
+    if (i8) {
+        if (kind == SIMJOIN_IP) jp.thr_i = clamp_to_i32(std::ceil(threshold));
+        else {
+            const double r2 = std::floor(threshold * threshold);
+            jp.thr_i = r2 >= 1073741824.0 ? 1073741824 : (int)r2;   // 2^30 exceeds every int8 squared distance here
+        }
+    } else {
+        jp.thr_f = kind == SIMJOIN_L2 ? (float)(threshold * threshold) : (float)threshold;
+    }
+}
+
 // The join on device buffers.  Arguments were validated by the caller.
 simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
                           simjoin_kind kind, double threshold, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
@@ -240,16 +253,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.ioff = (int)ctx->ioff;
     jp.joff = (int)ctx->joff;
 
-    // thresholds in the precision each path decides in
-    if (i8) {
-        if (kind == SIMJOIN_IP) jp.thr_i = clamp_to_i32(std::ceil(threshold));
-        else {
-            const double r2 = std::floor(threshold * threshold);
-            jp.thr_i = r2 >= 1073741824.0 ? 1073741824 : (int)r2;   // 2^30 exceeds every int8 squared distance here
-        }
-    } else {
-        jp.thr_f = kind == SIMJOIN_L2 ? (float)(threshold * threshold) : (float)threshold;
-    }
+    set_thresholds(jp, i8, kind, threshold);
 
     const bool need_norms = kind != SIMJOIN_IP;
     if (need_norms) {
@@ -836,21 +840,8 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     const size_t es = elem_size(dtype);
     const int row_bytes = (int)(d * es);
     JoinParams jp;
-    std::memset(&jp, 0, sizeof jp);
-    jp.n = n;
-    jp.m = m;
-    jp.kc = (row_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES;
-    jp.last_ksteps = (row_bytes - (jp.kc - 1) * CHUNK_BYTES + 31) / 32;
-    jp.elems_per_chunk = (int)(CHUNK_BYTES / es);
-    jp.stationary = jp.kc <= MAX_STATIONARY_CHUNKS ? 1 : 0;
-    const int p_bytes = jp.stationary ? P_BUFS * jp.kc * A_CHUNK_BYTES : 0;
-    const int stage_bytes = B_CHUNK_BYTES + (jp.stationary ? 0 : A_CHUNK_BYTES);
-    int nstages = (nd.smem_optin - 1024 - CTRL_BYTES - STAGING_BYTES - p_bytes) / stage_bytes;
-    if (nstages > MAX_STAGES) nstages = MAX_STAGES;
-    if (nstages < 2) return SIMJOIN_ERR_UNSUPPORTED;
-    jp.nstages = nstages;
-    jp.epi_release = (jp.stationary && nstages >= 2 * jp.kc) ? 1 : 0;
-    const size_t smem = 1024 + (size_t)p_bytes + (size_t)nstages * stage_bytes + STAGING_BYTES + CTRL_BYTES;
+    size_t smem = 0;
+    if (!tile_geometry(&tmp, n, m, row_bytes, es, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
     jp.PB = (int)((n + P_ROWS - 1) / P_ROWS);
     jp.QT = (int)((m + TILE_N - 1) / TILE_N);
     jp.qpanel = q_panel_tiles(jp.QT, row_bytes);
@@ -859,15 +850,7 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     unsigned long long *ctrl = reinterpret_cast<unsigned long long *>(nd.scratch + NA_OFF_CTRL);
     jp.counter = ctrl;
     jp.status = reinterpret_cast<unsigned int *>(ctrl + 1);
-    if (i8) {
-        if (kind == SIMJOIN_IP) jp.thr_i = clamp_to_i32(std::ceil(threshold));
-        else {
-            const double r2 = std::floor(threshold * threshold);
-            jp.thr_i = r2 >= 1073741824.0 ? 1073741824 : (int)r2;
-        }
-    } else {
-        jp.thr_f = kind == SIMJOIN_L2 ? (float)(threshold * threshold) : (float)threshold;
-    }
+    set_thresholds(jp, i8, kind, threshold);
     jp.nx = nd.scratch + NA_OFF_NX;
     jp.ny = nd.scratch + NA_OFF_NY;
     jp.qstat = nd.scratch + NA_OFF_QSTAT;
