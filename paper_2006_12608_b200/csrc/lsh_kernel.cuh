@@ -47,6 +47,45 @@ __global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict_
     }
 }
 
+// The same keys for short rows (d <= LSH_KEYS_STAGED_MAX_D bytes): a block first copies its 64 rows into shared
+// memory with coalesced 16-byte loads (row pitch d + 4 bytes: an odd number of words, so the byte gathers of
+// different rows fall into different banks), then four threads per row split the repetitions.  The per-thread
+// gather of the kernel above touches 32 different cache lines with every load instruction.
+constexpr int LSH_KEYS_STAGED_MAX_D = 512;
+constexpr int LSH_KEYS_STAGED_ROWS = 64;
+__global__ void __launch_bounds__(256) lsh_keys_staged_kernel(const int8_t *__restrict__ X, long long rows, int d, int L_high, int L_low,
+                                                              int k, unsigned long long seed, uint16_t *__restrict__ rec, int stride) {
+    __shared__ int s_coord[LSH_MAX_REPS * LSH_MAX_BITS];
+    extern __shared__ uint32_t s_rows[];                       // LSH_KEYS_STAGED_ROWS x (d / 4 + 1) words
+    const int L = L_high + L_low;
+    for (int t = threadIdx.x; t < L * k; t += blockDim.x) {
+        const int l = t / k, b = t - l * k;
+        s_coord[t] = (int)(lsh_splitmix64(seed, (uint64_t)l * 64u + (uint64_t)b) % (uint64_t)d);
+    }
+    const long long row0 = (long long)blockIdx.x * LSH_KEYS_STAGED_ROWS;
+    const int g = d / 16, pitch = d / 4 + 1;
+    const uint4 *src = reinterpret_cast<const uint4 *>(X + row0 * d);
+    const long long avail = (rows - row0 < LSH_KEYS_STAGED_ROWS ? rows - row0 : LSH_KEYS_STAGED_ROWS) * g;
+    for (int t = threadIdx.x; t < LSH_KEYS_STAGED_ROWS * g; t += blockDim.x) {
+        if (t >= avail) break;
+        const uint4 q = __ldg(src + t);
+        const int r = t / g, c = t - r * g;
+        uint32_t *dst = s_rows + r * pitch + c * 4;
+        dst[0] = q.x; dst[1] = q.y; dst[2] = q.z; dst[3] = q.w;
+    }
+    __syncthreads();
+    const int r = threadIdx.x >> 2, part = threadIdx.x & 3;
+    const long long i = row0 + r;
+    if (i >= rows) return;
+    const int8_t *x = reinterpret_cast<const int8_t *>(s_rows + r * pitch);
+    for (int l = part; l < stride; l += 4) {
+        uint32_t key = 0;
+        const int bits = l < L_high ? k : (l < L ? k - 1 : 0);      // padding entries stay 0
+        for (int b = 0; b < bits; ++b) key |= (x[s_coord[l * k + b]] > 0 ? 1u : 0u) << b;
+        rec[i * stride + l] = (uint16_t)key;
+    }
+}
+
 // hist[key] += number of rows with that key (block-private histogram in shared memory first).
 // keys: the key of row i is keys[i * stride] (one column of the key records).
 __global__ void __launch_bounds__(LSH_SORT_THREADS) lsh_hist_kernel(const uint16_t *__restrict__ keys, int stride, long long rows,

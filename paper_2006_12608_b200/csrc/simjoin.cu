@@ -570,10 +570,18 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     const bool narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
 
     cudaEventRecord(ctx->ev[0], s);
-    lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p,
-                                                                stride);
-    lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q,
-                                                                stride);
+    if (d <= LSH_KEYS_STAGED_MAX_D) {
+        const size_t sm = (size_t)LSH_KEYS_STAGED_ROWS * (d / 4 + 1) * 4;
+        lsh_keys_staged_kernel<<<(unsigned)((n + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), 256, sm, s>>>(
+            reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p, stride);
+        lsh_keys_staged_kernel<<<(unsigned)((m + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), 256, sm, s>>>(
+            reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q, stride);
+    } else {
+        lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p,
+                                                                    stride);
+        lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q,
+                                                                    stride);
+    }
     if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
     cudaEventRecord(ctx->ev[1], s);
     const int g = d / 16;
