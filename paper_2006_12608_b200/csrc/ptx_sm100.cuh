@@ -1,6 +1,6 @@
 // Thin inline-PTX wrappers for the sm_100a features the join kernel uses:
 // mbarrier, TMA tiled loads, tcgen05 (TMEM allocation, UMMA issue/commit, TMEM loads).
-// Everything here is single-CTA (cta_group::1) and uses no cluster multicast.
+// Everything here is single-CTA (cta_group::1): every copy lands in the issuing CTA only.
 #pragma once
 #include <cuda.h>
 #include <cstdint>
