@@ -83,6 +83,7 @@ struct JoinParams {
     int epi_release;         // 1: the epilogue hands ring stages back (one commit per tile); needs nstages >= 2*kc
     int PB, QT;              // number of 256-row P tiles, 128-row Q tiles
     int qpanel;              // Q tiles per L2-resident panel
+    int wave_gq;             // > 0: two-dimensional waves, (gridDim / wave_gq) P tiles x wave_gq Q tiles at a time (very long rows)
     int thr_i;               // I8/IP: ceil(t);  I8/L2: floor(r*r); both clamped
     float thr_f;             // BF16: t (IP, COS) or r*r (L2)
     const void *nx;          // per-row term of P: int32 |x|^2 (I8/L2), fp32 |x| (COS) or |x|^2 (L2)
@@ -139,6 +140,23 @@ __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
         un.q0 = 0;
         un.q1 = (e.w + TILE_N - 1) / TILE_N;
         un.prow0 = e.x; un.prows = e.y; un.qrow0 = e.z; un.qrows = e.w;
+        return true;
+    }
+    if (p.wave_gq > 0) {
+        // Very long rows: 148 resident P tiles no longer fit in L2 next to a Q panel, and every tile would come
+        // from DRAM.  Instead a wave covers GP P tiles x GQ Q tiles, one pair per CTA; the Q index moves fastest
+        // from wave to wave, so the GP P tiles stay in L2 while Q streams through once per row of waves.
+        const int GQ = p.wave_gq, GP = G / GQ;
+        if (c >= GP * GQ) return false;                         // spare CTAs
+        const int a = c / GQ, b = c - a * GQ;
+        const int WQ = (p.QT + GQ - 1) / GQ, WP = (p.PB + GP - 1) / GP;
+        const int wp = u / WQ, wq = u - wp * WQ;
+        if (wp >= WP) return false;
+        const int pb = wp * GP + a, qt = wq * GQ + b;
+        const bool inside = pb < p.PB && qt < p.QT;             // the edges of the grid leave some pairs empty
+        un.pb = inside ? pb : 0;
+        un.q0 = inside ? qt : 0;
+        un.q1 = inside ? qt + 1 : 0;
         return true;
     }
     const int full = p.PB / G, rem = p.PB - full * G;
@@ -515,6 +533,65 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
     }
 }
 
+// Long rows (LONGK): 256 x 256 tiles with one accumulator buffer.  Nothing is resident: every ring stage
+// carries a 32 KiB chunk of the Q tile and a 32 KiB chunk of the P tile, and one warp issues 2 x 4 tcgen05.mma
+// of N = 256 per chunk (1024 tensor cycles), block s accumulating in TMEM columns s * 256 ...  Per unit of work
+// that is 64 KiB of operand traffic per 1024 tensor cycles instead of the 48 KiB per 552 of the streamed
+// 256 x 128 tile, and the accumulator hand-off is paid once per K loop.
+constexpr int LONG_TN = 2 * TILE_N;                           // rows of Q per long tile
+constexpr int LONG_Q_CHUNK_BYTES = LONG_TN * CHUNK_BYTES;     // 32 KiB
+constexpr int LONG_STAGE_BYTES = LONG_Q_CHUNK_BYTES + A_CHUNK_BYTES;
+constexpr int LONG_STAGES = 3;
+template <int DT>
+__device__ __forceinline__ void mma_issuer_long(const JoinParams &p, Ctrl *ctrl, uint8_t *smem_ring, const uint32_t tmem_base,
+                                                const int lane) {
+    constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, LONG_TN);
+    uint32_t stage = 0, phase = 0, accph = 0;
+    bool ok = true;
+    Unit un;
+    for (int u = 0; ok && get_unit<false>(p, u, un); ++u) {
+        if (un.q1 <= un.q0) continue;
+        for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
+            ok = wait_bar_warp(&ctrl->tempty[0], accph ^ 1, ctrl, p.status, 4);
+            if (!ok) break;
+            for (int c = 0; c < p.kc; ++c) {
+                ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
+                if (!ok) break;
+                tc_fence_after();
+                uint8_t *sb = smem_ring + (size_t)stage * LONG_STAGE_BYTES;
+                const uint64_t bdesc = umma_desc_sw128_kmajor(smem_u32(sb));
+                const uint64_t adesc = umma_desc_sw128_kmajor(smem_u32(sb + LONG_Q_CHUNK_BYTES));
+                const uint64_t adesc1 = umma_desc_sw128_kmajor(smem_u32(sb + LONG_Q_CHUNK_BYTES + A_SUB_BYTES));
+                const bool last_chunk = c == p.kc - 1;
+                const int ksteps = last_chunk ? p.last_ksteps : 4;
+                if (elect_one()) {
+                    umma_ss<DT == DT_I8>(tmem_base, adesc, bdesc, idesc, c != 0 ? 1u : 0u);
+                    if (ksteps > 1) umma_ss<DT == DT_I8>(tmem_base, adesc + 2, bdesc + 2, idesc, 1u);
+                    if (ksteps > 2) umma_ss<DT == DT_I8>(tmem_base, adesc + 4, bdesc + 4, idesc, 1u);
+                    if (ksteps > 3) umma_ss<DT == DT_I8>(tmem_base, adesc + 6, bdesc + 6, idesc, 1u);
+                    umma_ss<DT == DT_I8>(tmem_base + LONG_TN, adesc1, bdesc, idesc, c != 0 ? 1u : 0u);
+                    if (ksteps > 1) umma_ss<DT == DT_I8>(tmem_base + LONG_TN, adesc1 + 2, bdesc + 2, idesc, 1u);
+                    if (ksteps > 2) umma_ss<DT == DT_I8>(tmem_base + LONG_TN, adesc1 + 4, bdesc + 4, idesc, 1u);
+                    if (ksteps > 3) umma_ss<DT == DT_I8>(tmem_base + LONG_TN, adesc1 + 6, bdesc + 6, idesc, 1u);
+                    umma_commit(smem_u32(&ctrl->empty[stage]));
+                    if (last_chunk) umma_commit(smem_u32(&ctrl->tfull[0]));
+                }
+                __syncwarp();
+                if (++stage == (uint32_t)LONG_STAGES) { stage = 0; phase ^= 1; }
+            }
+            accph ^= 1;
+        }
+    }
+    if (!ok) {
+        if (lane == 0) {
+            umma_commit(smem_u32(&ctrl->drain[0]));
+            const long long t0 = clock64();
+            while (!mbar_try_wait(smem_u32(&ctrl->drain[0]), 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+        __syncwarp();
+    }
+}
+
 // NARROW (int8 only): the host has verified that every score fits in 16 bits, so the epilogue
 // loads the accumulator packed two columns per register and reduces it with packed 16-bit max --
 // half the registers and half the ALU work of the 32-bit path, which is what bounds short-K tiles.
@@ -527,10 +604,19 @@ __host__ __device__ constexpr int fast_nstages(int kc, int pbufs) {
                : (232448 - 1024 - CTRL_BYTES - STAGING_BYTES - pbufs * kc * A_CHUNK_BYTES) / B_CHUNK_BYTES;
 }
 // GROUPED: bucketed mode (int8 inner product only) -- see JoinParams::units.
-template <int DT, int KIND, bool NARROW = false, int KC = 0, bool GROUPED = false>
+// LONGK: the long-row geometry above (join kinds, brute-force schedule only); mapQ then has 256-row boxes.
+template <int DT, int KIND, bool NARROW = false, int KC = 0, bool GROUPED = false, bool LONGK = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ, const JoinParams p_in) {
+    static_assert(!LONGK || (KC == 0 && !GROUPED && KIND != KIND_STORE), "long-row mode: general join kinds only");
+    constexpr int TN = LONGK ? LONG_TN : TILE_N;          // rows of Q per tile
+    constexpr int NPASS = TN / EPI_COLS;                   // 128-column passes of an epilogue warp over its block
     JoinParams p = p_in;
+    if constexpr (LONGK) {
+        p.stationary = 0;
+        p.epi_release = 0;
+        p.nstages = LONG_STAGES;
+    }
     if constexpr (KC > 0) {
         p.kc = KC;
         p.stationary = 1;
@@ -548,7 +634,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kc = p.kc;
     const int p_bytes = p.stationary ? p_bufs(GROUPED, kc) * kc * A_CHUNK_BYTES : 0;
-    const int stage_bytes = B_CHUNK_BYTES + (p.stationary ? 0 : A_CHUNK_BYTES);
+    const int stage_bytes = LONGK ? LONG_STAGE_BYTES : B_CHUNK_BYTES + (p.stationary ? 0 : A_CHUNK_BYTES);
     uint8_t *smem_p = smem;
     uint8_t *smem_ring = smem + p_bytes;
     int2 *smem_staging = reinterpret_cast<int2 *>(smem_ring + (size_t)p.nstages * stage_bytes);
@@ -601,7 +687,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 if (++pbuf == (uint32_t)p_bufs(GROUPED, kc)) { pbuf = 0; pphase ^= 1; }
             }
             for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
-                const int q_row = (GROUPED ? un.qrow0 : 0) + tile_at<ALIGNED>(un, k) * TILE_N;
+                const int q_row = (GROUPED ? un.qrow0 : 0) + tile_at<ALIGNED>(un, k) * TN;
                 for (int c = 0; c < p.kc; ++c) {
                     ok = wait_bar_warp(&ctrl->empty[stage], phase ^ 1, ctrl, p.status, 2);
                     if (!ok) break;
@@ -611,7 +697,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         mbar_arrive_expect_tx(bar, (uint32_t)stage_bytes);
                         tma_load_2d(smem_u32(sb), &mapQ, bar, c * p.elems_per_chunk, q_row);
                         if (!p.stationary)
-                            tma_load_2d(smem_u32(sb + B_CHUNK_BYTES), &mapP, bar, c * p.elems_per_chunk, p_row);
+                            tma_load_2d(smem_u32(sb + (LONGK ? LONG_Q_CHUNK_BYTES : B_CHUNK_BYTES)), &mapP, bar, c * p.elems_per_chunk, p_row);
                     }
                     __syncwarp();
                     if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
@@ -638,7 +724,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         // In that case warp 1 issues every tile and warp 3 stays out.
         const bool fast = p.stationary && p.epi_release && p.last_ksteps == 4;
         constexpr bool OB = KIND == KIND_STORE;
-        if (fast && p.kc == 1) mma_issuer_role<DT, 1, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        if constexpr (LONGK) {
+            if (warp == 1) mma_issuer_long<DT>(p, ctrl, smem_ring, tmem_base, lane);
+        } else if (fast && p.kc == 1) mma_issuer_role<DT, 1, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
         else if (fast && p.kc == 2) mma_issuer_role<DT, 2, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
         else mma_issuer_role<DT, 0, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
     } else if (warp >= EPI_WARP0) {
@@ -676,23 +764,27 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 int fi = p.thr_i;
                 float ff = p.thr_f;
                 if constexpr (DT == DT_I8 && KIND == KIND_L2) {
-                    const int2 st = reinterpret_cast<const int2 *>(p.qstat)[qt / (QSTAT_ROWS / TILE_N)];
+                    const int2 st = reinterpret_cast<const int2 *>(p.qstat)[qt / (QSTAT_ROWS / TN)];
                     fi = (ri + st.x + 1) >> 1;                    // 2s >= |x|^2 - R + min|y|^2
                 }
                 if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
-                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt / (QSTAT_ROWS / TILE_N)];
+                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt / (QSTAT_ROWS / TN)];
                     ff = rf * (p.thr_f >= 0.f ? st.x : st.y);     // s >= t|x| * min|y| (max|y| when t < 0)
                 }
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
-                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt / (QSTAT_ROWS / TILE_N)];
+                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt / (QSTAT_ROWS / TN)];
                     ff = rf + st.x;                               // (|x|^2 + min|y|^2) - 2s <= r^2
                 }
                 // per-column terms of this warp's columns, 4 per lane, fetched while the tile is still
                 // being multiplied so that the exact test never waits on global memory
-                uint4 yq = make_uint4(0, 0, 0, 0);
-                if ((KIND == KIND_COS || KIND == KIND_L2) && lane < EPI_COLS / 4)
-                    yq = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint32_t *>(p.ny) +
-                                                               (long long)qt * TILE_N) + lane);
+                uint4 yq_pass[NPASS];
+#pragma unroll
+                for (int ps = 0; ps < NPASS; ++ps) {
+                    yq_pass[ps] = make_uint4(0, 0, 0, 0);
+                    if ((KIND == KIND_COS || KIND == KIND_L2) && lane < EPI_COLS / 4)
+                        yq_pass[ps] = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint32_t *>(p.ny) +
+                                                                            ((long long)qt * TN + ps * EPI_COLS)) + lane);
+                }
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
                 if (!ok) break;
                 tc_fence_after();
@@ -734,15 +826,20 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     if (acc == 0) accphase ^= 1;
                     continue;
                 }
-                // this warp's 128 columns of the tile, then hand the accumulator back to the MMA warp
+                // this warp's 128 columns of the tile (long rows: two passes of 128 over its block's 256), then hand
+                // the accumulator back to the MMA warp
                 constexpr int NV = NARROW ? EPI_COLS / 2 : EPI_COLS;      // accumulator words per thread
                 constexpr int GCOLS = 16, NG = EPI_COLS / GCOLS, GW = NV / NG;  // groups of 16 columns
                 constexpr int MODE = DT == DT_BF16 ? MAX_F32 : (NARROW ? MAX_S16X2 : MAX_S32);
+#pragma unroll
+                for (int ps = 0; ps < NPASS; ++ps) {
+                const uint4 yq = yq_pass[ps];
                 uint32_t v[NV];
-                tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TILE_N, v, std::integral_constant<bool, NARROW>{});
+                tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TN + ps * EPI_COLS, v,
+                              std::integral_constant<bool, NARROW>{});
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                if (ps == NPASS - 1 && lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
                 // level 0: the row maximum over this warp's 128 columns against the per-tile bound
                 // (a necessary condition of the exact test, in the same arithmetic)
                 auto bound_ok = [&](uint32_t word) -> bool {
@@ -762,7 +859,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
 #pragma unroll
                     for (int k = 0; k < NG; ++k) gm |= (bound_ok(TreeMax<GW, MODE>::run(v + k * GW)) ? 1u : 0u) << k;
                     if (!row_ok) gm = 0;
-                    const long long j0 = q_base + (long long)qt * TILE_N;
+                    const long long j0 = q_base + (long long)qt * TN + ps * EPI_COLS;
                     uint32_t mask[EPI_COLS / 32];
 #pragma unroll
                     for (int q = 0; q < EPI_COLS / 32; ++q) mask[q] = 0;
@@ -811,8 +908,13 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     }
                     emit_pairs<EPI_COLS / 32, GROUPED>(p, mask, lane, i, j0, stage_buf, stage_fill);
                 }
-                acc ^= 1;
-                if (acc == 0) accphase ^= 1;
+                }   // passes
+                if constexpr (LONGK) {
+                    accphase ^= 1;                      // one accumulator buffer
+                } else {
+                    acc ^= 1;
+                    if (acc == 0) accphase ^= 1;
+                }
             }
         }
         if (ok) flush_pairs<GROUPED>(p, stage_buf, stage_fill, lane);

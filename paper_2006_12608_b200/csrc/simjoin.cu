@@ -49,8 +49,9 @@ struct simjoin_ctx {
     float prepass_ms, join_ms;
     long long ioff, joff;
     bool attr_set[2][4][2][3][2];
-    // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
+    bool attr_set_long[2][3][2];
     DevBuf jl_a, jl_buf[2];             // JL transform: level matrix, ping-pong level outputs
+    // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
     DevBuf lsh_keys_p, lsh_keys_q, lsh_skeys_p, lsh_skeys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
 };
 
@@ -175,12 +176,32 @@ cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorM
     return launch_join_kc<DT, KIND, NARROW, 0, GROUPED>(ctx, mp, mq, jp, grid, smem);
 }
 
+// Chunks per row from which the join takes the long-row geometry.  Measured on B200 (n = m = 131 072, sustained,
+// fraction of nominal): 384-byte rows 0.70 resident-P vs 0.61 long; 512-byte rows 0.56 vs 0.64; longer rows cannot
+// keep P resident at all.
+#ifndef SIMJOIN_LONG_MIN_KC
+#define SIMJOIN_LONG_MIN_KC 4
+#endif
+// The long-row geometry (256 x 256 tiles, nothing resident, one accumulator buffer): general join kinds only.
+template <int DT, int KIND, bool NARROW>
+cudaError_t launch_join_long(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
+                             size_t smem) {
+    auto kern = join_kernel<DT, KIND, NARROW, 0, false, true>;
+    if (!ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
+        if (e != cudaSuccess) return e;
+        ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0] = true;
+    }
+    kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
+    return cudaGetLastError();
+}
+
 // Q tiles per panel.  A Q of up to 64 MiB is swept whole (it mostly stays in L2 and measured faster
 // that way); a larger one is cut into panels of about 32 MiB that stay resident in L2 while every P
 // block sweeps them (measured on a 128 MiB Q: 10.5 GB -> 0.74 GB of DRAM reads per launch).  Panels are
 // balanced so that the last one is not a sliver.
-int q_panel_tiles(int QT, int row_bytes) {
-    const long long tile_bytes = (long long)TILE_N * row_bytes;
+int q_panel_tiles(int QT, int row_bytes, int tile_rows = TILE_N) {
+    const long long tile_bytes = (long long)tile_rows * row_bytes;
     if ((long long)QT * tile_bytes <= (64LL << 20)) return QT;
     long long cap = (32LL << 20) / tile_bytes;
     if (cap < 8) cap = 8;
@@ -243,9 +264,21 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     JoinParams jp;
     size_t smem = 0;
     if (!tile_geometry(ctx, n, m, row_bytes, es, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
+    // rows of 512 bytes and more take the long-row geometry
+    const bool longk = jp.kc >= SIMJOIN_LONG_MIN_KC;
+    const int tn = longk ? LONG_TN : TILE_N;
+    if (longk) {
+        jp.stationary = 0;
+        jp.epi_release = 0;
+        jp.nstages = LONG_STAGES;
+        smem = 1024 + (size_t)LONG_STAGES * LONG_STAGE_BYTES + STAGING_BYTES + CTRL_BYTES;
+        if (smem > (size_t)ctx->max_smem_optin) return SIMJOIN_ERR_UNSUPPORTED;
+        // one P tile per CTA plus a Q panel must fit in L2 (126 MB) for the sweep schedule; beyond that, 2-D waves
+        if ((long long)ctx->num_sms * P_ROWS * row_bytes > (48LL << 20) && ctx->num_sms >= 8) jp.wave_gq = 4;
+    }
     jp.PB = (int)((n + P_ROWS - 1) / P_ROWS);
-    jp.QT = (int)((m + TILE_N - 1) / TILE_N);
-    jp.qpanel = q_panel_tiles(jp.QT, row_bytes);
+    jp.QT = (int)((m + tn - 1) / tn);
+    jp.qpanel = q_panel_tiles(jp.QT, row_bytes, tn);
     jp.out = reinterpret_cast<int2 *>(out_pairs);
     jp.capacity = capacity;
     jp.counter = ctx->d_ctrl;
@@ -258,7 +291,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     const bool need_norms = kind != SIMJOIN_IP;
     if (need_norms) {
         // ny is read in 16-entry groups up to the end of the last Q tile: pad it to whole tiles
-        if (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, (size_t)jp.QT * TILE_N * 4) || !grow(ctx->qstat, (size_t)jp.QT * 8))
+        if (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, (size_t)jp.QT * tn * 4) || !grow(ctx->qstat, (size_t)jp.QT * 8))
             return SIMJOIN_ERR_CUDA;
         jp.nx = ctx->nx.ptr;
         jp.ny = ctx->ny.ptr;
@@ -266,7 +299,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     }
 
     CUtensorMap mapP, mapQ;
-    if (!encode_rows_map(ctx, &mapP, P, n, d, P_ROWS) || !encode_rows_map(ctx, &mapQ, Q, m, d, TILE_N))
+    if (!encode_rows_map(ctx, &mapP, P, n, d, P_ROWS) || !encode_rows_map(ctx, &mapQ, Q, m, d, tn))
         return SIMJOIN_ERR_CUDA;
 
     cudaStream_t s = ctx->stream;
@@ -303,6 +336,15 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     cudaEventRecord(ctx->ev[1], s);
     const int grid = ctx->num_sms;
     cudaError_t e = cudaErrorInvalidValue;
+    if (longk) {
+        if (i8 && kind == SIMJOIN_IP && narrow) e = launch_join_long<DT_I8, KIND_IP, true>(ctx, mapP, mapQ, jp, grid, smem);
+        else if (i8 && kind == SIMJOIN_L2 && narrow) e = launch_join_long<DT_I8, KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
+        else if (i8 && kind == SIMJOIN_IP) e = launch_join_long<DT_I8, KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
+        else if (i8 && kind == SIMJOIN_L2) e = launch_join_long<DT_I8, KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
+        else if (!i8 && kind == SIMJOIN_IP) e = launch_join_long<DT_BF16, KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
+        else if (!i8 && kind == SIMJOIN_COS) e = launch_join_long<DT_BF16, KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem);
+        else if (!i8 && kind == SIMJOIN_L2) e = launch_join_long<DT_BF16, KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
+    } else
     if (i8 && kind == SIMJOIN_IP && narrow) e = launch_join<DT_I8, KIND_IP, true>(ctx, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_L2 && narrow) e = launch_join<DT_I8, KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_IP) e = launch_join<DT_I8, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
@@ -364,6 +406,7 @@ simjoin_status simjoin_create(simjoin_ctx **out, simjoin_dtype dtype, int device
     ctx->have_timing = false;
     ctx->ioff = ctx->joff = 0;
     std::memset(ctx->attr_set, 0, sizeof ctx->attr_set);
+    std::memset(ctx->attr_set_long, 0, sizeof ctx->attr_set_long);
     for (auto &e : ctx->ev) e = nullptr;
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
