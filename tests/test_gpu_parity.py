@@ -358,3 +358,44 @@ def test_repeated_runs_give_the_same_set(ctx_bf16):
     a, ca = gpu_join(ctx_bf16, w.P, w.Q, "l2", w.threshold, capacity=1 << 19)
     b, cb = gpu_join(ctx_bf16, w.P, w.Q, "l2", w.threshold, capacity=1 << 19)
     assert ca == cb and np.array_equal(np.sort(keys(a)), np.sort(keys(b)))
+
+
+# ------------------------------------------------------------------ long rows: 256 x 256 tiles, two epilogue passes
+@pytest.mark.parametrize("kind", ["ip", "l2"])
+@pytest.mark.parametrize("d,lo,hi", [(512, -3, 3), (656, -1, 1), (1024, -127, 127)])
+def test_i8_long_row_geometry(ctx_i8, kind, d, lo, hi):
+    """Rows of 512 bytes and more: whole chunks, a 16-byte last chunk (656), and values too wide for the packed
+    epilogue (1024); ragged row counts, hits in both column passes of a tile."""
+    P, Q = W.random_points("i8", 300 + 7, d, 81, lo=lo, hi=hi), W.random_points("i8", 1024 + 45, d, 82, lo=lo, hi=hi)
+    Q[5:260:3] = P[:85]                                  # planted equal rows, spread over both passes and several tiles
+    sd = (d * ((hi - lo + 1) ** 2 - 1) / 12.0)           # variance of one coordinate product sum, roughly
+    if kind == "ip":
+        t = 2.5 * (d * ((hi * (hi + 1)) / 3.0) ** 2) ** 0.5
+    else:
+        t = (2.0 * sd) ** 0.5 * 0.86                      # a little below the typical distance: the low tail passes
+    pairs, cnt = gpu_join(ctx_i8, P, Q, kind, t, capacity=1 << 20)
+    assert_exact(pairs, cnt, P, Q, kind, t)
+    assert cnt >= 85
+
+
+@pytest.mark.parametrize("kind", ["ip", "cos", "l2"])
+@pytest.mark.parametrize("d", [256, 264, 1040])
+def test_bf16_long_row_geometry(ctx_bf16, kind, d):
+    """bf16 rows of 512, 528 (16-byte last chunk) and 2080 bytes (the last also takes the two-dimensional waves)."""
+    P, Q = W.random_points("bf16", 260 + 3, d, 91), W.random_points("bf16", 800 + 31, d, 92)
+    Q[3:200:2] = P[:99]
+    t = {"ip": 3.0 * d ** 0.5, "cos": 0.12, "l2": (2.0 * d) ** 0.5 - 1.5}[kind]
+    pairs, cnt = gpu_join(ctx_bf16, P, Q, kind, t, capacity=1 << 20)
+    assert_band(pairs, cnt, P, Q, kind, t)
+    assert cnt >= 99
+
+
+def test_two_dimensional_waves_cover_every_tile_pair_once(ctx_i8):
+    """2 KiB rows switch to waves of 37 x 4 tile pairs: 39 P tiles x 6 Q tiles need two waves in each direction,
+    with partly empty ones at both edges."""
+    P, Q = W.random_points("i8", 38 * 256 + 17, 2048, 95, lo=-1, hi=1), W.random_points("i8", 5 * 256 + 40, 2048, 96, lo=-1, hi=1)
+    Q[::11] = P[:len(Q[::11])]
+    t = 3.6 * (2048 * 4.0 / 9.0) ** 0.5
+    pairs, cnt = gpu_join(ctx_i8, P, Q, "ip", t, capacity=1 << 20)
+    assert_exact(pairs, cnt, P, Q, "ip", t)
+    assert cnt >= len(Q[::11])
