@@ -50,6 +50,11 @@ constexpr int A_CHUNK_BYTES = P_ROWS * CHUNK_BYTES;   // 32 KiB: one K chunk of 
 constexpr int A_SUB_BYTES = TILE_M * CHUNK_BYTES;     // 16 KiB
 constexpr int B_CHUNK_BYTES = TILE_N * CHUNK_BYTES;   // 16 KiB
 constexpr int MAX_STAGES = 8;
+// long-row and wide-Q geometries (see join_kernel): 256 rows of Q per tile
+constexpr int LONG_TN = 2 * TILE_N;                           // rows of Q per long tile
+constexpr int LONG_Q_CHUNK_BYTES = LONG_TN * CHUNK_BYTES;     // 32 KiB
+constexpr int LONG_STAGE_BYTES = LONG_Q_CHUNK_BYTES + A_CHUNK_BYTES;
+constexpr int LONG_STAGES = 3;
 constexpr int MAX_STATIONARY_CHUNKS = 4;          // P block kept resident up to 512-byte rows
 #ifndef SIMJOIN_P_BUFS
 #define SIMJOIN_P_BUFS 1
@@ -446,11 +451,12 @@ __device__ __forceinline__ void store_tile_part(const JoinParams &p, uint32_t ta
 // operand-address select another ~25.  KC == 0 is the general path.
 // ONE_BLOCK_OK: a tile whose second P block lies wholly past the end of P skips that block's MMAs (the store
 // kind, whose resident operand often has <= 128 rows; the join kinds keep the branch out of their issue loop).
-template <int DT, int KC, bool GROUPED, bool ONE_BLOCK_OK>
+// WIDEQ: one resident block against 256 streamed rows (N = 256); the second block is never issued.
+template <int DT, int KC, bool GROUPED, bool ONE_BLOCK_OK, bool WIDEQ = false>
 __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl, uint8_t *smem_p, uint8_t *smem_ring,
                                                 const int stage_bytes_rt, const uint32_t tmem_base, const int warp, const int lane) {
     constexpr bool FAST = KC > 0;
-    constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, TILE_N);
+    constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, WIDEQ ? LONG_TN : TILE_N);
     const int kc = FAST ? KC : p.kc;
     const bool stationary = FAST ? true : p.stationary != 0;
     const bool epi_release = FAST ? true : p.epi_release != 0;
@@ -467,7 +473,7 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
             ok = wait_bar_warp(&ctrl->pfull[pbuf], pphase, ctrl, p.status, 3);
             if (!ok) break;
         }
-        const bool two = !ONE_BLOCK_OK || (GROUPED ? un.prows > TILE_M : (long long)un.pb * P_ROWS + TILE_M < p.n);
+        const bool two = !WIDEQ && (!ONE_BLOCK_OK || (GROUPED ? un.prows > TILE_M : (long long)un.pb * P_ROWS + TILE_M < p.n));
         for (int k = 0; ok && k < un.q1 - un.q0; ++k, tsel ^= 1) {
             if (dual && tsel != mid) {
                 // the other issuer's tile: step over its chunks in the ring
@@ -538,10 +544,6 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
 // of N = 256 per chunk (1024 tensor cycles), block s accumulating in TMEM columns s * 256 ...  Per unit of work
 // that is 64 KiB of operand traffic per 1024 tensor cycles instead of the 48 KiB per 552 of the streamed
 // 256 x 128 tile, and the accumulator hand-off is paid once per K loop.
-constexpr int LONG_TN = 2 * TILE_N;                           // rows of Q per long tile
-constexpr int LONG_Q_CHUNK_BYTES = LONG_TN * CHUNK_BYTES;     // 32 KiB
-constexpr int LONG_STAGE_BYTES = LONG_Q_CHUNK_BYTES + A_CHUNK_BYTES;
-constexpr int LONG_STAGES = 3;
 template <int DT>
 __device__ __forceinline__ void mma_issuer_long(const JoinParams &p, Ctrl *ctrl, uint8_t *smem_ring, const uint32_t tmem_base,
                                                 const int lane) {
@@ -604,12 +606,18 @@ __host__ __device__ constexpr int fast_nstages(int kc, int pbufs) {
                : (232448 - 1024 - CTRL_BYTES - STAGING_BYTES - pbufs * kc * A_CHUNK_BYTES) / B_CHUNK_BYTES;
 }
 // GROUPED: bucketed mode (int8 inner product only) -- see JoinParams::units.
-// LONGK: the long-row geometry above (join kinds, brute-force schedule only); mapQ then has 256-row boxes.
-template <int DT, int KIND, bool NARROW = false, int KC = 0, bool GROUPED = false, bool LONGK = false>
+// GEO selects the tile geometry.  GEO_LONG: the long-row geometry above (join kinds, brute-force schedule only).
+// GEO_WIDEQ (store kind, resident operand of at most 128 rows): one resident block against 256 streamed rows per
+// tile -- 4 MMAs of N = 256 per chunk into the 256 columns of an accumulator buffer, 32 KiB TMA transactions --
+// which this HBM-bound use prefers to two half-empty 128-column blocks.  In both, mapQ has 256-row boxes.
+constexpr int GEO_STD = 0, GEO_LONG = 1, GEO_WIDEQ = 2;
+template <int DT, int KIND, bool NARROW = false, int KC = 0, bool GROUPED = false, int GEO = GEO_STD>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ, const JoinParams p_in) {
+    constexpr bool LONGK = GEO == GEO_LONG, WIDEQ = GEO == GEO_WIDEQ;
     static_assert(!LONGK || (KC == 0 && !GROUPED && KIND != KIND_STORE), "long-row mode: general join kinds only");
-    constexpr int TN = LONGK ? LONG_TN : TILE_N;          // rows of Q per tile
+    static_assert(!WIDEQ || (KC == 0 && !GROUPED && KIND == KIND_STORE), "wide-Q mode: store kind only");
+    constexpr int TN = (LONGK || WIDEQ) ? LONG_TN : TILE_N;   // rows of Q per tile
     constexpr int NPASS = TN / EPI_COLS;                   // 128-column passes of an epilogue warp over its block
     JoinParams p = p_in;
     if constexpr (LONGK) {
@@ -634,7 +642,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kc = p.kc;
     const int p_bytes = p.stationary ? p_bufs(GROUPED, kc) * kc * A_CHUNK_BYTES : 0;
-    const int stage_bytes = LONGK ? LONG_STAGE_BYTES : B_CHUNK_BYTES + (p.stationary ? 0 : A_CHUNK_BYTES);
+    const int stage_bytes = LONGK ? LONG_STAGE_BYTES : (WIDEQ ? LONG_Q_CHUNK_BYTES : B_CHUNK_BYTES) + (p.stationary ? 0 : A_CHUNK_BYTES);
     uint8_t *smem_p = smem;
     uint8_t *smem_ring = smem + p_bytes;
     int2 *smem_staging = reinterpret_cast<int2 *>(smem_ring + (size_t)p.nstages * stage_bytes);
@@ -697,7 +705,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         mbar_arrive_expect_tx(bar, (uint32_t)stage_bytes);
                         tma_load_2d(smem_u32(sb), &mapQ, bar, c * p.elems_per_chunk, q_row);
                         if (!p.stationary)
-                            tma_load_2d(smem_u32(sb + (LONGK ? LONG_Q_CHUNK_BYTES : B_CHUNK_BYTES)), &mapP, bar, c * p.elems_per_chunk, p_row);
+                            tma_load_2d(smem_u32(sb + (TN == LONG_TN ? LONG_Q_CHUNK_BYTES : B_CHUNK_BYTES)), &mapP, bar, c * p.elems_per_chunk, p_row);
                     }
                     __syncwarp();
                     if (++stage == (uint32_t)p.nstages) { stage = 0; phase ^= 1; }
@@ -726,9 +734,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         constexpr bool OB = KIND == KIND_STORE;
         if constexpr (LONGK) {
             if (warp == 1) mma_issuer_long<DT>(p, ctrl, smem_ring, tmem_base, lane);
-        } else if (fast && p.kc == 1) mma_issuer_role<DT, 1, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
-        else if (fast && p.kc == 2) mma_issuer_role<DT, 2, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
-        else mma_issuer_role<DT, 0, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        } else if (fast && p.kc == 1 && !WIDEQ) mma_issuer_role<DT, 1, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        else if (fast && p.kc == 2 && !WIDEQ) mma_issuer_role<DT, 2, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        else mma_issuer_role<DT, 0, GROUPED, OB, WIDEQ>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
     } else if (warp >= EPI_WARP0) {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
@@ -814,11 +822,13 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     // lane <-> row of P (an output coordinate), columns <-> rows of Q (output rows).  With two P
                     // blocks in the tile this warp stores block `half`; with one, the two warps of a lane quarter
                     // split that block's 128 columns between them.
-                    const long long j0 = q_base + (long long)qt * TILE_N;
+                    const long long j0 = q_base + (long long)qt * TN;
                     uint16_t *sb = reinterpret_cast<uint16_t *>(stage_buf);          // [32 output rows][32 coordinates]
                     const int i_unit = (GROUPED ? un.prow0 : un.pb * P_ROWS) + quarter * 32;
                     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS;
-                    if (two_blocks)
+                    if constexpr (WIDEQ)        // one block, 256 streamed rows: this warp stores rows half * 128 ..
+                        store_tile_part<TILE_N>(p, t_lane + half * TILE_N, &ctrl->tempty[acc], lane, sb, j0 + half * TILE_N, q_end, i_unit);
+                    else if (two_blocks)
                         store_tile_part<TILE_N>(p, t_lane + half * TILE_N, &ctrl->tempty[acc], lane, sb, j0, q_end, i_unit + half * TILE_M);
                     else
                         store_tile_part<TILE_N / 2>(p, t_lane + half * (TILE_N / 2), &ctrl->tempty[acc], lane, sb, j0 + half * (TILE_N / 2), q_end, i_unit);

@@ -50,6 +50,7 @@ struct simjoin_ctx {
     long long ioff, joff;
     bool attr_set[2][4][2][3][2];
     bool attr_set_long[2][3][2];
+    bool attr_set_wideq;
     DevBuf jl_a, jl_buf[2];             // JL transform: level matrix, ping-pong level outputs
     // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
     DevBuf lsh_keys_p, lsh_keys_q, lsh_skeys_p, lsh_skeys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
@@ -186,11 +187,24 @@ cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorM
 template <int DT, int KIND, bool NARROW>
 cudaError_t launch_join_long(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
                              size_t smem) {
-    auto kern = join_kernel<DT, KIND, NARROW, 0, false, true>;
+    auto kern = join_kernel<DT, KIND, NARROW, 0, false, GEO_LONG>;
     if (!ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
         if (e != cudaSuccess) return e;
         ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0] = true;
+    }
+    kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
+    return cudaGetLastError();
+}
+
+// The wide-Q geometry of the store kind (one resident block of at most 128 rows against 256 streamed rows per tile).
+cudaError_t launch_store_wideq(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
+                               size_t smem) {
+    auto kern = join_kernel<DT_BF16, KIND_STORE, false, 0, false, GEO_WIDEQ>;
+    if (!ctx->attr_set_wideq) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
+        if (e != cudaSuccess) return e;
+        ctx->attr_set_wideq = true;
     }
     kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
     return cudaGetLastError();
@@ -407,6 +421,7 @@ simjoin_status simjoin_create(simjoin_ctx **out, simjoin_dtype dtype, int device
     ctx->ioff = ctx->joff = 0;
     std::memset(ctx->attr_set, 0, sizeof ctx->attr_set);
     std::memset(ctx->attr_set_long, 0, sizeof ctx->attr_set_long);
+    ctx->attr_set_wideq = false;
     for (auto &e : ctx->ev) e = nullptr;
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -720,8 +735,19 @@ simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, 
         JoinParams jp;
         size_t smem = 0;
         if (!tile_geometry(ctx, ki, rows, ci * 2, 2, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
+        // a level matrix of at most 128 rows and two chunks: 256 streamed rows per tile, 32 KiB ring stages
+        const bool wideq = ki <= TILE_M && jp.kc <= 2;
+        const int tn = wideq ? LONG_TN : TILE_N;
+        if (wideq) {
+            const int p_bytes = P_BUFS * jp.kc * A_CHUNK_BYTES;
+            int nstages = (ctx->max_smem_optin - 1024 - CTRL_BYTES - STAGING_BYTES - p_bytes) / LONG_Q_CHUNK_BYTES;
+            if (nstages > MAX_STAGES) nstages = MAX_STAGES;
+            jp.nstages = nstages;
+            jp.epi_release = nstages >= 2 * jp.kc ? 1 : 0;
+            smem = 1024 + (size_t)p_bytes + (size_t)nstages * LONG_Q_CHUNK_BYTES + STAGING_BYTES + CTRL_BYTES;
+        }
         jp.PB = (ki + P_ROWS - 1) / P_ROWS;
-        jp.QT = (int)((rows + TILE_N - 1) / TILE_N);
+        jp.QT = (int)((rows + tn - 1) / tn);
         jp.qpanel = jp.QT;                 // the blocks are read once: no L2 panels, one long sweep per CTA
         jp.counter = ctx->d_ctrl;
         jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
@@ -729,9 +755,11 @@ simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, 
         jp.store_ld = ki;
         jp.store_scale = (float)(1.0 / std::sqrt((double)ki));
         CUtensorMap mapA, mapX;
-        if (!encode_rows_map(ctx, &mapA, ctx->jl_a.ptr, ki, ci, P_ROWS) || !encode_rows_map(ctx, &mapX, src, rows, ci, TILE_N))
+        if (!encode_rows_map(ctx, &mapA, ctx->jl_a.ptr, ki, ci, P_ROWS) || !encode_rows_map(ctx, &mapX, src, rows, ci, tn))
             return SIMJOIN_ERR_CUDA;
-        if (launch_join<DT_BF16, KIND_STORE>(ctx, mapA, mapX, jp, ctx->num_sms, smem) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        const cudaError_t le = wideq ? launch_store_wideq(ctx, mapA, mapX, jp, ctx->num_sms, smem)
+                                     : launch_join<DT_BF16, KIND_STORE>(ctx, mapA, mapX, jp, ctx->num_sms, smem);
+        if (le != cudaSuccess) return SIMJOIN_ERR_CUDA;
         src = dst;
     }
     cudaEventRecord(ctx->ev[2], s);
