@@ -15,6 +15,10 @@ collective); the value is the ops of all ranks over the slowest rank's time.
 
 ``--impl reference`` times the CPU oracle (as it stands) on a bounded row slab of
 the same workload on the host cores.
+
+Two side modes time the widened entry points on synthetic data and say so in their line (they are not the
+headline metric): ``--lsh L,k[,L_low]`` the LSH-bucketed join (``simjoin_run_lsh``) on an int8 inner-product
+configuration, ``--jl n,d,k`` the JL transform (``simjoin_jl_transform``) with an HBM roofline.
 """
 from __future__ import annotations
 
