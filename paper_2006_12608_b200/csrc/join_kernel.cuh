@@ -56,20 +56,13 @@ constexpr int LONG_Q_CHUNK_BYTES = LONG_TN * CHUNK_BYTES;     // 32 KiB
 constexpr int LONG_STAGE_BYTES = LONG_Q_CHUNK_BYTES + A_CHUNK_BYTES;
 constexpr int LONG_STAGES = 3;
 constexpr int MAX_STATIONARY_CHUNKS = 4;          // P block kept resident up to 512-byte rows
-#ifndef SIMJOIN_P_BUFS
-#define SIMJOIN_P_BUFS 1
-#endif
-constexpr int P_BUFS = SIMJOIN_P_BUFS;            // resident P blocks: 1 (a short bubble per Q sweep) or 2
+constexpr int P_BUFS = 1;                         // resident P tiles of the sweep schedule (a short bubble per Q sweep)
 // Bucketed mode sweeps only a bucket's Q rows per P block (tens of tiles, not thousands): there the bubble
 // matters, and the next P block is fetched while the current one is still being multiplied (rows of up to
 // two chunks; longer rows would pay for the second block with ring depth).
 __host__ __device__ constexpr int p_bufs(bool grouped, int kc) { return grouped && kc <= 2 ? 2 : P_BUFS; }
 constexpr int EPI_WARP0 = 4;
-#ifndef SIMJOIN_EPI_WARPS
-#define SIMJOIN_EPI_WARPS 8
-#endif
-constexpr int NUM_EPI_WARPS = SIMJOIN_EPI_WARPS;               // 4 TMEM lane quarters x P_SUB blocks
-static_assert(NUM_EPI_WARPS == 4 * P_SUB, "one epilogue warp per TMEM lane quarter and P block");
+constexpr int NUM_EPI_WARPS = 4 * P_SUB;                       // one per TMEM lane quarter and P block
 constexpr int EPI_COLS = TILE_N;                               // accumulator columns per epilogue warp
 constexpr int NUM_THREADS = 32 * (EPI_WARP0 + NUM_EPI_WARPS);
 constexpr uint32_t TMEM_COLS = 512;
@@ -193,20 +186,13 @@ __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
 // The k-th tile a CTA visits in its unit.  Every CTA starts its sweep at a different offset and wraps
 // around, so that at any moment the CTAs read different Q tiles instead of all hitting the same L2
 // lines at once (measured: the aligned sweep is ~5 % slower on two-chunk tiles once Q is L2-resident).
-#ifndef SIMJOIN_ROTATE
-#define SIMJOIN_ROTATE 1
-#endif
 template <bool ALIGNED>
 __device__ __forceinline__ int tile_at(const Unit &un, int k) {
     if constexpr (ALIGNED) return un.q0 + k;
-#if SIMJOIN_ROTATE
     const int len = un.q1 - un.q0;
     int idx = k + (int)((long long)blockIdx.x * len / gridDim.x);
     if (idx >= len) idx -= len;
     return un.q0 + idx;
-#else
-    return un.q0 + k;
-#endif
 }
 
 // Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting.  The hot loop is a

@@ -180,9 +180,7 @@ cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorM
 // Chunks per row from which the join takes the long-row geometry.  Measured on B200 (n = m = 131 072, sustained,
 // fraction of nominal): 384-byte rows 0.70 resident-P vs 0.61 long; 512-byte rows 0.56 vs 0.64; longer rows cannot
 // keep P resident at all.
-#ifndef SIMJOIN_LONG_MIN_KC
-#define SIMJOIN_LONG_MIN_KC 4
-#endif
+constexpr int LONG_MIN_KC = 4;
 // The long-row geometry (256 x 256 tiles, nothing resident, one accumulator buffer): general join kinds only.
 template <int DT, int KIND, bool NARROW>
 cudaError_t launch_join_long(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
@@ -279,7 +277,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     size_t smem = 0;
     if (!tile_geometry(ctx, n, m, row_bytes, es, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
     // rows of 512 bytes and more take the long-row geometry
-    const bool longk = jp.kc >= SIMJOIN_LONG_MIN_KC;
+    const bool longk = jp.kc >= LONG_MIN_KC;
     const int tn = longk ? LONG_TN : TILE_N;
     if (longk) {
         jp.stationary = 0;
