@@ -110,7 +110,10 @@ simjoin_status simjoin_run(simjoin_ctx *ctx, const void *P, int64_t n, const voi
  * copies P and Q to device staging owned by the context, runs the join, and
  * copies min(*count, capacity) pairs back; all on the context's stream,
  * synchronised before return.  Pinned host memory makes the copies faster but
- * is not required.  Errors as simjoin_run (device pointers are rejected here).
+ * is not required.  A Q above 64 MiB is uploaded in slices of about 32 MiB on a second stream and every
+ * slice is joined as soon as it has landed, so that (with pinned memory) the copies of later slices hide
+ * behind the joins of earlier ones; the result is the union of the slices' results.
+ * Errors as simjoin_run (device pointers are rejected here).
  */
 simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n, const void *Q_host,
                                 int64_t m, int32_t d, simjoin_kind kind, double threshold,

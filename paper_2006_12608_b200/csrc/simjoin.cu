@@ -51,6 +51,8 @@ struct simjoin_ctx {
     bool attr_set[2][4][2][3][2];
     bool attr_set_long[2][3][2];
     bool attr_set_wideq;
+    cudaStream_t copy_stream;           // simjoin_run_host: uploads of Q slices overlap the joins of earlier slices
+    cudaEvent_t copy_ev[66];
     DevBuf jl_a, jl_buf[2];             // JL transform: level matrix, ping-pong level outputs
     // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
     DevBuf lsh_keys_p, lsh_keys_q, lsh_skeys_p, lsh_skeys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
@@ -420,6 +422,8 @@ simjoin_status simjoin_create(simjoin_ctx **out, simjoin_dtype dtype, int device
     std::memset(ctx->attr_set, 0, sizeof ctx->attr_set);
     std::memset(ctx->attr_set_long, 0, sizeof ctx->attr_set_long);
     ctx->attr_set_wideq = false;
+    ctx->copy_stream = nullptr;
+    for (auto &e : ctx->copy_ev) e = nullptr;
     for (auto &e : ctx->ev) e = nullptr;
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -460,6 +464,9 @@ simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
     release(ctx->lsh_sorted_p);
     release(ctx->lsh_sorted_q);
     release(ctx->lsh_misc);
+    for (auto &e : ctx->copy_ev)
+        if (e) cudaEventDestroy(e);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->d_ctrl) cudaFree(ctx->d_ctrl);
     if (ctx->h_ctrl) cudaFreeHost(ctx->h_ctrl);
     for (auto &e : ctx->ev)
@@ -503,12 +510,62 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
     const size_t pb = (size_t)n * d * es, qb = (size_t)m * d * es, ob = (size_t)capacity * 8;
     if (!grow(ctx->stage_p, pb) || !grow(ctx->stage_q, qb) || !grow(ctx->stage_out, ob ? ob : 8)) return SIMJOIN_ERR_CUDA;
     cudaStream_t s = ctx->stream;
-    if (cudaMemcpyAsync(ctx->stage_p.ptr, P_host, pb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(ctx->stage_q.ptr, Q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return SIMJOIN_ERR_CUDA;
-    st = run_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, kind, threshold,
-                    capacity ? reinterpret_cast<int32_t *>(ctx->stage_out.ptr) : nullptr, capacity, count);
-    if (st != SIMJOIN_OK && st != SIMJOIN_ERR_CAPACITY) return st;
+    // A large Q goes up in slices of about 32 MiB on a second stream, and each slice is joined (a call of its own,
+    // with the column offset of the slice) as soon as it has landed: the copies of the later slices hide behind
+    // the joins of the earlier ones.  The result is the union of the slices' results.
+    const size_t row_bytes = (size_t)d * es;
+    const int64_t slice_rows = qb > (64u << 20) ? (int64_t)(((32u << 20) / row_bytes + TILE_N - 1) / TILE_N * TILE_N) : m;
+    const int nslices = (int)((m + slice_rows - 1) / slice_rows);
+    if (nslices > 1 && nslices <= (int)(sizeof ctx->copy_ev / sizeof ctx->copy_ev[0])) {
+        if (!ctx->copy_stream && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        for (int q = 0; q <= nslices; ++q)
+            if (!ctx->copy_ev[q] && cudaEventCreateWithFlags(&ctx->copy_ev[q], cudaEventDisableTiming) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        cudaStream_t cs = ctx->copy_stream;
+        // the staging buffers may still be in use by earlier work on the context's stream
+        if (cudaEventRecord(ctx->copy_ev[nslices], s) != cudaSuccess || cudaStreamWaitEvent(cs, ctx->copy_ev[nslices], 0) != cudaSuccess)
+            return SIMJOIN_ERR_CUDA;
+        if (cudaMemcpyAsync(ctx->stage_p.ptr, P_host, pb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        for (int q = 0; q < nslices; ++q) {
+            const int64_t r0 = q * slice_rows, rows = (m - r0 < slice_rows) ? m - r0 : slice_rows;
+            if (cudaMemcpyAsync(static_cast<char *>(ctx->stage_q.ptr) + (size_t)r0 * row_bytes, static_cast<const char *>(Q_host) + (size_t)r0 * row_bytes,
+                                (size_t)rows * row_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+                cudaEventRecord(ctx->copy_ev[q], cs) != cudaSuccess)
+                return SIMJOIN_ERR_CUDA;
+        }
+        const long long joff0 = ctx->joff;
+        uint64_t total = 0;
+        float pre_ms = 0.f, join_ms = 0.f;
+        st = SIMJOIN_OK;
+        for (int q = 0; q < nslices && (st == SIMJOIN_OK || st == SIMJOIN_ERR_CAPACITY); ++q) {
+            const int64_t r0 = q * slice_rows, rows = (m - r0 < slice_rows) ? m - r0 : slice_rows;
+            if (cudaStreamWaitEvent(s, ctx->copy_ev[q], 0) != cudaSuccess) { st = SIMJOIN_ERR_CUDA; break; }
+            const uint64_t used = total < capacity ? total : capacity;
+            uint64_t cnt = 0;
+            ctx->joff = joff0 + r0;
+            const simjoin_status sq = run_device(ctx, ctx->stage_p.ptr, n, static_cast<char *>(ctx->stage_q.ptr) + (size_t)r0 * row_bytes, rows, d, kind,
+                                                 threshold, capacity > used ? reinterpret_cast<int32_t *>(ctx->stage_out.ptr) + 2 * used : nullptr,
+                                                 capacity - used, &cnt);
+            ctx->joff = joff0;
+            total += cnt;
+            if (sq != SIMJOIN_OK) st = sq;
+            if (ctx->have_timing) { pre_ms += ctx->prepass_ms; join_ms += ctx->join_ms; }
+        }
+        if (st != SIMJOIN_OK && st != SIMJOIN_ERR_CAPACITY) {
+            cudaStreamSynchronize(cs);
+            return st;
+        }
+        ctx->prepass_ms = pre_ms;
+        ctx->join_ms = join_ms;
+        *count = total;
+        st = total > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
+    } else {
+        if (cudaMemcpyAsync(ctx->stage_p.ptr, P_host, pb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+            cudaMemcpyAsync(ctx->stage_q.ptr, Q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return SIMJOIN_ERR_CUDA;
+        st = run_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, kind, threshold,
+                        capacity ? reinterpret_cast<int32_t *>(ctx->stage_out.ptr) : nullptr, capacity, count);
+        if (st != SIMJOIN_OK && st != SIMJOIN_ERR_CAPACITY) return st;
+    }
     const uint64_t wrote = *count < capacity ? *count : capacity;
     if (wrote > 0) {
         if (cudaMemcpyAsync(out_pairs_host, ctx->stage_out.ptr, (size_t)wrote * 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||

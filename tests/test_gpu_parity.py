@@ -271,6 +271,35 @@ def test_run_host_matches_device_path(ctx_i8):
     assert ctx_i8.simjoin_run_host(dP, w.n, w.Q, w.m, w.d, "ip", w.threshold, out, 10)[0] == B.SIMJOIN_ERR_ARG
 
 
+def test_run_host_uploads_a_large_q_in_slices(ctx_i8, ctx_bf16):
+    """A Q above 64 MiB goes up in ~32 MiB slices that are joined one by one while the next ones are still being
+    copied: the union of the slices' results, with their column offsets, must be the whole join; the capacity
+    is shared by the slices and the count stays the full one when it runs out."""
+    P, Q = W.random_points("i8", 200, 8192, 65), W.random_points("i8", 9000, 8192, 66)      # Q: 73.7 MB -> 3 slices of 4096 rows
+    t = 2.2 * (8192 * 16.0) ** 0.5
+    want, wcnt = O.join(P, Q, "ip", t, "i8")
+    assert wcnt > 1000 and len(np.unique(want[:, 1] // 4096)) == 3                          # hits in every slice
+    out = np.full((wcnt + 10, 2), -7, dtype=np.int32)
+    assert ctx_i8.simjoin_set_offsets(7, 100) == B.SIMJOIN_OK
+    try:
+        st, cnt = ctx_i8.simjoin_run_host(P, 200, Q, 9000, 8192, "ip", t, out, wcnt + 10)
+    finally:
+        ctx_i8.simjoin_set_offsets(0, 0)
+    assert (st, cnt) == (B.SIMJOIN_OK, wcnt)
+    assert np.array_equal(np.sort(keys(out[:cnt])), keys(want + np.array([7, 100]))) and np.all(out[cnt:] == -7)
+    small = np.full((wcnt // 2 + 4, 2), -7, dtype=np.int32)
+    st, cnt = ctx_i8.simjoin_run_host(P, 200, Q, 9000, 8192, "ip", t, small, wcnt // 2)
+    assert (st, cnt) == (B.SIMJOIN_ERR_CAPACITY, wcnt)
+    assert np.isin(keys(small[:wcnt // 2]), keys(want)).all() and np.all(small[wcnt // 2:] == -7)
+    assert len(np.unique(keys(small[:wcnt // 2]))) == wcnt // 2
+    # a norm kind through the same path (row terms are recomputed per slice)
+    Pb, Qb = W.random_points("bf16", 150, 4096, 67), W.random_points("bf16", 8500, 4096, 68)  # Q: 69.6 MB
+    outb = np.full((1 << 20, 2), -7, dtype=np.int32)
+    st, cnt = ctx_bf16.simjoin_run_host(Pb, 150, Qb, 8500, 4096, "cos", 0.03, outb, 1 << 20)
+    assert st == B.SIMJOIN_OK and cnt > 1000
+    assert_band(outb[:cnt], cnt, Pb, Qb, "cos", 0.03)
+
+
 def test_row_norms_prepass(ctx_i8, ctx_bf16):
     for rows, d in [(1, 16), (300, 64), (1000, 144), (513, 1024)]:
         X = W.random_points("i8", rows, d, 18, lo=-128, hi=127)
