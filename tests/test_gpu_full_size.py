@@ -170,3 +170,35 @@ def test_full_size_jl_transform_sampled_rows():
     err = np.abs(got - want)
     assert np.all(err <= bound[:, None]), (err.max(), bound.min())
     assert np.sqrt((err ** 2).mean()) <= 4.0 * np.sqrt(len(sh)) * 2.0 ** -9 * np.sqrt((want ** 2).mean()) / np.sqrt(3.0)
+
+
+def test_full_size_hamming_join():
+    """Hamming join on 1 048 576 x 1 048 576 bit-packed points of 128 bits, r = 14: every emitted pair is checked by
+    the oracle's bit count, every planted pair (8 flipped bits) is present, sampled rows are joined whole by the oracle.
+    Random pairs are at distance ~64 +- 5.7, so nothing but the planted pairs is expected within 14."""
+    n, d, r, k = 1 << 20, 128, 14, 50000
+    P = W.random_bits(n, d, 31)
+    Q = W.random_bits(n, d, 32, planted_from=P[:k], flips=8)
+    build.build()
+    cap = 4 * k
+    with B.Simjoin("i8", 0) as ctx:
+        dP, dQ = torch.from_numpy(P).cuda(), torch.from_numpy(Q).cuda()
+        out = torch.empty((cap, 2), dtype=torch.int32, device="cuda:0")
+        st, cnt = ctx.simjoin_run_hamming(dP, n, dQ, n, d, r, out, cap)
+        assert st == B.SIMJOIN_OK, B.strerror(st)
+        pairs = out[:cnt].cpu().numpy().astype(np.int64)
+    del dP, dQ, out
+    torch.cuda.empty_cache()
+    gk = keys(pairs)
+    assert len(np.unique(gk)) == cnt and cnt >= k
+    x = np.unpackbits(P[pairs[:, 0]] ^ Q[pairs[:, 1]], axis=1).sum(axis=1)       # independent popcount of the emitted pairs
+    assert np.all(x <= r)
+    assert all(O.hamming(P[i], Q[j], d) <= r for i, j in pairs[:: max(1, cnt // 64)])
+    planted = np.stack([np.arange(k), np.arange(k)], axis=1)
+    assert np.isin(keys(planted), gk).all()
+    rows = np.unique(np.concatenate([np.random.default_rng(9).choice(n, size=20, replace=False), [0, k - 1, k, n - 1]]))
+    want, _c = O.join_hamming(P[rows], Q, d, r)
+    want = want.astype(np.int64)
+    want[:, 0] = rows[want[:, 0]]
+    got = pairs[np.isin(pairs[:, 0], rows)]
+    assert np.array_equal(np.sort(keys(got)), np.sort(keys(want)))
