@@ -155,6 +155,18 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
                                int32_t *out_pairs, uint64_t capacity, uint64_t *count);
 
 /*
+ * LSH-bucketed Hamming join on bit-packed points: simjoin_run_hamming's operand transform followed by
+ * simjoin_run_lsh -- bit sampling is the LSH family of the Hamming distance, so bit b of the key of repetition l is
+ * simply coordinate splitmix64(seed, 64*l + b) mod d of the point.  The output is exactly
+ *     { (i, j) : Hamming(x_i, y_j) <= r  and  key_l(x_i) == key_l(y_j) for some repetition l }.
+ * Arguments as simjoin_run_hamming (P_bits, Q_bits, n, m, d, r) and simjoin_run_lsh (L, L_low, k, seed); errors
+ * as those two.  I8 contexts only.
+ */
+simjoin_status simjoin_run_hamming_lsh(simjoin_ctx *ctx, const void *P_bits, int64_t n, const void *Q_bits, int64_t m,
+                                       int32_t d, double r, int32_t L, int32_t L_low, int32_t k, uint64_t seed,
+                                       int32_t *out_pairs, uint64_t capacity, uint64_t *count);
+
+/*
  * JL transform (Section 3: the lemma that builds M = (I_{r_l} (x) A_l) ... (I_{r_1} (x) A_1) and computes M x
  * as l small dense products): out = X M^T for all n rows at once, reducing d coordinates to k, as a
  * pre-reduction before an (approximate) join on the k-dimensional rows.

@@ -184,6 +184,17 @@ def lsh_join(P: np.ndarray, Q: np.ndarray, threshold: float, L: int, k: int, see
         cap = int(cnt)
 
 
+def lsh_join_hamming(Pbits: np.ndarray, Qbits: np.ndarray, d: int, r: float, L: int, k: int, seed: int, threads: int = 0,
+                     L_low: int = 0):
+    """The LSH-bucketed Hamming join on bit-packed rows: the points are widened to +-1 rows (x -> 2x - 1, the operand
+    transform of the Hamming ip-distance), on which <x, y> = d - 2 Hamming(x, y) and the bit-sampling hash [x_c > 0] is
+    the sampled bit itself; then lsh_join with threshold d - 2 floor(r).  Returns (pairs, count)."""
+    def widen(b):
+        bits = np.unpackbits(np.ascontiguousarray(b), axis=1, bitorder="little")[:, :d]
+        return (2 * bits.astype(np.int8) - 1).astype(np.int8)
+    return lsh_join(widen(Pbits), widen(Qbits), float(d) - 2.0 * np.floor(r), L, k, seed, threads=threads, L_low=L_low)
+
+
 def lsh_keys(X: np.ndarray, L: int, k: int, seed: int, L_low: int = 0) -> np.ndarray:
     """(L + L_low, rows) uint32 hash keys of int8 rows."""
     lib = _load()

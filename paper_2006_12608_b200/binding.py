@@ -21,7 +21,7 @@ SIMJOIN_IP, SIMJOIN_COS, SIMJOIN_L2 = 0, 1, 2
 DTYPE = {"i8": SIMJOIN_I8, "bf16": SIMJOIN_BF16}
 KIND = {"ip": SIMJOIN_IP, "cos": SIMJOIN_COS, "l2": SIMJOIN_L2}
 
-EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_hamming", "simjoin_run_lsh", "simjoin_jl_transform", "simjoin_row_norms", "simjoin_set_offsets",
+EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_hamming", "simjoin_run_lsh", "simjoin_run_hamming_lsh", "simjoin_jl_transform", "simjoin_row_norms", "simjoin_set_offsets",
            "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_selftest_wait_timeout", "simjoin_destroy",
            "simjoin_strerror")
 SIMJOIN_NOALLOC_MAX_ROWS = 65536
@@ -56,6 +56,8 @@ def load() -> ctypes.CDLL:
     lib.simjoin_run_hamming.argtypes = [vp, vp, i64, vp, i64, i32, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_run_lsh.restype = c.c_int
     lib.simjoin_run_lsh.argtypes = [vp, vp, i64, vp, i64, i32, dbl, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
+    lib.simjoin_run_hamming_lsh.restype = c.c_int
+    lib.simjoin_run_hamming_lsh.argtypes = [vp, vp, i64, vp, i64, i32, dbl, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
     lib.simjoin_jl_transform.restype = c.c_int
     lib.simjoin_jl_transform.argtypes = [vp, vp, i64, i32, i32, u64, vp]
     lib.simjoin_run_noalloc.restype = c.c_int
@@ -147,6 +149,13 @@ class Simjoin:
         (pp, _a), (qp, _b), (op, _c) = _ptr(P), _ptr(Q), _ptr(out_pairs)
         st = load().simjoin_run_lsh(self._h, pp, n, qp, m, d, float(threshold), int(L), int(L_low), int(k), int(seed), op, capacity,
                                     ctypes.byref(cnt))
+        return st, cnt.value
+
+    def simjoin_run_hamming_lsh(self, P_bits, n, Q_bits, m, d, r, L, k, seed, out_pairs, capacity, L_low=0):
+        cnt = ctypes.c_uint64(0)
+        (pp, _a), (qp, _b), (op, _c) = _ptr(P_bits), _ptr(Q_bits), _ptr(out_pairs)
+        st = load().simjoin_run_hamming_lsh(self._h, pp, n, qp, m, d, float(r), int(L), int(L_low), int(k), int(seed), op,
+                                            capacity, ctypes.byref(cnt))
         return st, cnt.value
 
     def simjoin_jl_transform(self, X, n, d, k, seed, out):

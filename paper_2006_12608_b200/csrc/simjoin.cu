@@ -386,6 +386,173 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
 }
 
+// The LSH-bucketed join on device buffers of int8 rows.  Arguments were validated by the caller.
+simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, double threshold,
+                          int32_t L, int32_t L_low, int32_t k, uint64_t seed, int32_t *out_pairs, uint64_t capacity,
+                          uint64_t *count) {
+    *count = 0;
+    ctx->have_timing = false;
+    if (n == 0 || m == 0) return SIMJOIN_OK;
+
+    JoinParams jp;
+    size_t smem = 0;
+    if (!tile_geometry(ctx, n, m, d, 1, jp, smem, true)) return SIMJOIN_ERR_UNSUPPORTED;
+    const int nb_max = 1 << k;
+    const size_t max_units = (size_t)((n + P_ROWS - 1) / P_ROWS) + (size_t)nb_max;
+    // misc: hist_p | hist_q | cursor_p | cursor_q (nb words each) | nunits (padded to 16 B) | units
+    const size_t off_units = ((size_t)4 * nb_max * 4 + 16 + 15) & ~(size_t)15;
+    const int reps = L + L_low;
+    const int rec_words = (reps + 7) / 8, stride = rec_words * 8;   // key record of a row: 16-bit keys, padded to 16 bytes
+    const size_t rec_bytes = (size_t)rec_words * 16;
+    if (!grow(ctx->lsh_keys_p, n * rec_bytes) || !grow(ctx->lsh_keys_q, m * rec_bytes) ||
+        !grow(ctx->lsh_skeys_p, n * rec_bytes) || !grow(ctx->lsh_skeys_q, m * rec_bytes) ||
+        !grow(ctx->lsh_perm_p, (size_t)n * 4) || !grow(ctx->lsh_perm_q, (size_t)m * 4) ||
+        !grow(ctx->lsh_sorted_p, (size_t)n * d) || !grow(ctx->lsh_sorted_q, (size_t)m * d) ||
+        !grow(ctx->lsh_misc, off_units + max_units * 16))
+        return SIMJOIN_ERR_CUDA;
+    unsigned int *hist_p = reinterpret_cast<unsigned int *>(ctx->lsh_misc.ptr);
+    unsigned int *hist_q = hist_p + nb_max, *cursor_p = hist_q + nb_max, *cursor_q = cursor_p + nb_max, *nunits = cursor_q + nb_max;
+    int4 *units = reinterpret_cast<int4 *>(reinterpret_cast<unsigned char *>(ctx->lsh_misc.ptr) + off_units);
+    uint16_t *keys_p = reinterpret_cast<uint16_t *>(ctx->lsh_keys_p.ptr), *keys_q = reinterpret_cast<uint16_t *>(ctx->lsh_keys_q.ptr);
+    int *perm_p = reinterpret_cast<int *>(ctx->lsh_perm_p.ptr), *perm_q = reinterpret_cast<int *>(ctx->lsh_perm_q.ptr);
+
+    jp.out = reinterpret_cast<int2 *>(out_pairs);
+    jp.capacity = capacity;
+    jp.counter = ctx->d_ctrl;
+    jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
+    jp.ioff = (int)ctx->ioff;
+    jp.joff = (int)ctx->joff;
+    jp.thr_i = clamp_to_i32(std::ceil(threshold));
+    jp.units = units;
+    jp.nunits = nunits;
+    jp.perm_p = perm_p;
+    jp.perm_q = perm_q;
+    jp.rec_p = reinterpret_cast<const uint4 *>(ctx->lsh_skeys_p.ptr);
+    jp.rec_q = reinterpret_cast<const uint4 *>(ctx->lsh_skeys_q.ptr);
+    jp.rec_words = rec_words;
+
+    CUtensorMap mapP, mapQ;
+    if (!encode_rows_map(ctx, &mapP, ctx->lsh_sorted_p.ptr, n, d, P_ROWS) ||
+        !encode_rows_map(ctx, &mapQ, ctx->lsh_sorted_q.ptr, m, d, TILE_N))
+        return SIMJOIN_ERR_CUDA;
+
+    cudaStream_t s = ctx->stream;
+    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    // 16-bit epilogue when every score provably fits (as in the brute-force join)
+    unsigned int *d_max = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 2);
+    maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(P), (long long)n * d / 16, d_max);
+    maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(Q), (long long)m * d / 16, d_max + 1);
+    if (cudaGetLastError() != cudaSuccess ||
+        cudaMemcpyAsync(ctx->h_ctrl + 2, ctx->d_ctrl + 2, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    const unsigned int *h_max = reinterpret_cast<const unsigned int *>(ctx->h_ctrl + 2);
+    const bool narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
+
+    cudaEventRecord(ctx->ev[0], s);
+    if (d <= LSH_KEYS_STAGED_MAX_D) {
+        const size_t sm = (size_t)LSH_KEYS_STAGED_ROWS * (d / 4 + 1) * 4;
+        lsh_keys_staged_kernel<<<(unsigned)((n + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), 256, sm, s>>>(
+            reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p, stride);
+        lsh_keys_staged_kernel<<<(unsigned)((m + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), 256, sm, s>>>(
+            reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q, stride);
+    } else {
+        lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p,
+                                                                    stride);
+        lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q,
+                                                                    stride);
+    }
+    if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    cudaEventRecord(ctx->ev[1], s);
+    const int g = d / 16;
+    const unsigned hist_blocks = (unsigned)ctx->num_sms * 4;
+    const int rows_per_block = LSH_SORT_THREADS * LSH_SORT_ITEMS;
+    for (int l = 0; l < reps; ++l) {
+        const uint16_t *kp = keys_p + l, *kq = keys_q + l;          // column l of the key records
+        const int nb = l < L ? nb_max : nb_max / 2;          // buckets of this repetition
+        if (cudaMemsetAsync(hist_p, 0, (size_t)2 * nb_max * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kp, stride, n, nb, hist_p);
+        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kq, stride, m, nb, hist_q);
+        lsh_offsets_units_kernel<<<1, 1024, 0, s>>>(hist_p, hist_q, nb, cursor_p, cursor_q, units, nunits, P_ROWS);
+        lsh_scatter_kernel<<<(unsigned)((n + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kp, stride, n, nb,
+                                                                                                              cursor_p, perm_p);
+        lsh_scatter_kernel<<<(unsigned)((m + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kq, stride, m, nb,
+                                                                                                              cursor_q, perm_q);
+        lsh_gather_rows_kernel<<<(unsigned)(((long long)n * g + 255) / 256), 256, 0, s>>>(
+            reinterpret_cast<const uint4 *>(P), perm_p, n, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_p.ptr));
+        lsh_gather_rows_kernel<<<(unsigned)(((long long)m * g + 255) / 256), 256, 0, s>>>(
+            reinterpret_cast<const uint4 *>(Q), perm_q, m, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_q.ptr));
+        if (l > 0) {
+            // key records in regrouped order, for the duplicate check of the join's epilogue
+            lsh_gather_rows_kernel<<<(unsigned)(((long long)n * rec_words + 255) / 256), 256, 0, s>>>(
+                reinterpret_cast<const uint4 *>(keys_p), perm_p, n, rec_words, reinterpret_cast<uint4 *>(ctx->lsh_skeys_p.ptr));
+            lsh_gather_rows_kernel<<<(unsigned)(((long long)m * rec_words + 255) / 256), 256, 0, s>>>(
+                reinterpret_cast<const uint4 *>(keys_q), perm_q, m, rec_words, reinterpret_cast<uint4 *>(ctx->lsh_skeys_q.ptr));
+        }
+        if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        jp.rep = l;
+        const cudaError_t e = narrow ? launch_join<DT_I8, KIND_IP, true, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem)
+                                     : launch_join<DT_I8, KIND_IP, false, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem);
+        if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    }
+    cudaEventRecord(ctx->ev[2], s);
+    if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    if ((unsigned int)(ctx->h_ctrl[1] & 0xffffffffu) != 0) return SIMJOIN_ERR_TIMEOUT;
+    *count = ctx->h_ctrl[0];
+    float a = 0.f, b = 0.f;
+    if (cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess && cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
+        ctx->prepass_ms = a;       // hashing
+        ctx->join_ms = b;          // L x (regroup + bucketed join)
+        ctx->have_timing = true;
+    }
+    return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
+}
+
+simjoin_status check_lsh_args(int32_t L, int32_t L_low, int32_t k) {
+    if (L < 0 || L_low < 0 || L + L_low < 1 || L + L_low > LSH_MAX_REPS || k < 0 || (L_low > 0 && k < 1)) return SIMJOIN_ERR_ARG;
+    if (k > LSH_MAX_BITS) return SIMJOIN_ERR_UNSUPPORTED;
+    return SIMJOIN_OK;
+}
+
+simjoin_status check_hamming_args(const simjoin_ctx *ctx, const void *P_bits, int64_t n, const void *Q_bits, int64_t m, int32_t d,
+                                  double r, const int32_t *out_pairs, uint64_t capacity, const uint64_t *count) {
+    if (!ctx || !count || !P_bits || !Q_bits) return SIMJOIN_ERR_ARG;
+    if (ctx->dtype != SIMJOIN_I8) return SIMJOIN_ERR_UNSUPPORTED;
+    if (n < 0 || m < 0 || n >= SIMJOIN_MAX_ROWS || m >= SIMJOIN_MAX_ROWS || d <= 0) return SIMJOIN_ERR_ARG;
+    if (std::isnan(r) || r < 0) return SIMJOIN_ERR_ARG;
+    if (!out_pairs && capacity > 0) return SIMJOIN_ERR_ARG;
+    if (d % 128 != 0 || d > SIMJOIN_MAX_ROW_BYTES) return SIMJOIN_ERR_UNSUPPORTED;    // 16-byte packed rows
+    if ((reinterpret_cast<uintptr_t>(P_bits) & 15u) || (reinterpret_cast<uintptr_t>(Q_bits) & 15u)) return SIMJOIN_ERR_UNSUPPORTED;
+    if (n + ctx->ioff >= SIMJOIN_MAX_ROWS || m + ctx->joff >= SIMJOIN_MAX_ROWS) return SIMJOIN_ERR_ARG;
+    return SIMJOIN_OK;
+}
+
+// Operand transform of the Hamming joins: bits -> +-1 int8 rows in the context's staging buffers.  The device must be
+// current.  Leaves *count = 0.
+simjoin_status hamming_unpack(simjoin_ctx *ctx, const void *P_bits, int64_t n, const void *Q_bits, int64_t m, int32_t d,
+                              const int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+    if ((n > 0 && !is_device_ptr(P_bits, ctx->device)) || (m > 0 && !is_device_ptr(Q_bits, ctx->device))) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && !is_device_ptr(out_pairs, ctx->device)) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
+    *count = 0;
+    if (n == 0 || m == 0) return SIMJOIN_OK;
+    const size_t pb = (size_t)n * d, qb = (size_t)m * d;
+    if (!grow(ctx->stage_p, pb) || !grow(ctx->stage_q, qb)) return SIMJOIN_ERR_CUDA;
+    cudaStream_t s = ctx->stream;
+    const long long ph = (long long)n * d / 16, qh = (long long)m * d / 16;      // 16-bit groups
+    unpack_bits_pm1_kernel<<<(unsigned)((ph + 255) / 256), 256, 0, s>>>(reinterpret_cast<const uint16_t *>(P_bits), ph,
+                                                                         reinterpret_cast<uint4 *>(ctx->stage_p.ptr));
+    unpack_bits_pm1_kernel<<<(unsigned)((qh + 255) / 256), 256, 0, s>>>(reinterpret_cast<const uint16_t *>(Q_bits), qh,
+                                                                         reinterpret_cast<uint4 *>(ctx->stage_q.ptr));
+    return cudaGetLastError() == cudaSuccess ? SIMJOIN_OK : SIMJOIN_ERR_CUDA;
+}
+
 }  // namespace
 
 extern "C" {
@@ -579,30 +746,12 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
 
 simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t n, const void *Q_bits, int64_t m, int32_t d,
                                    double r, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
-    if (!ctx || !count || !P_bits || !Q_bits) return SIMJOIN_ERR_ARG;
-    if (ctx->dtype != SIMJOIN_I8) return SIMJOIN_ERR_UNSUPPORTED;
-    if (n < 0 || m < 0 || n >= SIMJOIN_MAX_ROWS || m >= SIMJOIN_MAX_ROWS || d <= 0) return SIMJOIN_ERR_ARG;
-    if (std::isnan(r) || r < 0) return SIMJOIN_ERR_ARG;
-    if (!out_pairs && capacity > 0) return SIMJOIN_ERR_ARG;
-    if (d % 128 != 0 || d > SIMJOIN_MAX_ROW_BYTES) return SIMJOIN_ERR_UNSUPPORTED;    // 16-byte packed rows
-    if ((reinterpret_cast<uintptr_t>(P_bits) & 15u) || (reinterpret_cast<uintptr_t>(Q_bits) & 15u)) return SIMJOIN_ERR_UNSUPPORTED;
-    if (n + ctx->ioff >= SIMJOIN_MAX_ROWS || m + ctx->joff >= SIMJOIN_MAX_ROWS) return SIMJOIN_ERR_ARG;
+    simjoin_status st = check_hamming_args(ctx, P_bits, n, Q_bits, m, d, r, out_pairs, capacity, count);
+    if (st != SIMJOIN_OK) return st;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SIMJOIN_ERR_CUDA;
-    if ((n > 0 && !is_device_ptr(P_bits, ctx->device)) || (m > 0 && !is_device_ptr(Q_bits, ctx->device))) return SIMJOIN_ERR_ARG;
-    if (capacity > 0 && !is_device_ptr(out_pairs, ctx->device)) return SIMJOIN_ERR_ARG;
-    if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
-    *count = 0;
-    if (n == 0 || m == 0) return SIMJOIN_OK;
-    const size_t pb = (size_t)n * d, qb = (size_t)m * d;
-    if (!grow(ctx->stage_p, pb) || !grow(ctx->stage_q, qb)) return SIMJOIN_ERR_CUDA;
-    cudaStream_t s = ctx->stream;
-    const long long ph = (long long)n * d / 16, qh = (long long)m * d / 16;      // 16-bit groups
-    unpack_bits_pm1_kernel<<<(unsigned)((ph + 255) / 256), 256, 0, s>>>(reinterpret_cast<const uint16_t *>(P_bits), ph,
-                                                                         reinterpret_cast<uint4 *>(ctx->stage_p.ptr));
-    unpack_bits_pm1_kernel<<<(unsigned)((qh + 255) / 256), 256, 0, s>>>(reinterpret_cast<const uint16_t *>(Q_bits), qh,
-                                                                         reinterpret_cast<uint4 *>(ctx->stage_q.ptr));
-    if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    st = hamming_unpack(ctx, P_bits, n, Q_bits, m, d, out_pairs, capacity, count);
+    if (st != SIMJOIN_OK || n == 0 || m == 0) return st;
     // Hamming <= r  <=>  Hamming <= floor(r)  <=>  d - 2*Hamming >= d - 2*floor(r)
     const double t = (double)d - 2.0 * std::floor(r);
     return run_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, SIMJOIN_IP, t, out_pairs, capacity, count);
@@ -614,135 +763,29 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     simjoin_status st = check_join_args(ctx, P, n, Q, m, d, SIMJOIN_IP, threshold, out_pairs, capacity, count);
     if (st != SIMJOIN_OK) return st;
     if (ctx->dtype != SIMJOIN_I8) return SIMJOIN_ERR_UNSUPPORTED;
-    if (L < 0 || L_low < 0 || L + L_low < 1 || L + L_low > LSH_MAX_REPS || k < 0 || (L_low > 0 && k < 1)) return SIMJOIN_ERR_ARG;
-    if (k > LSH_MAX_BITS) return SIMJOIN_ERR_UNSUPPORTED;
+    st = check_lsh_args(L, L_low, k);
+    if (st != SIMJOIN_OK) return st;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SIMJOIN_ERR_CUDA;
     if ((n > 0 && !is_device_ptr(P, ctx->device)) || (m > 0 && !is_device_ptr(Q, ctx->device))) return SIMJOIN_ERR_ARG;
     if (capacity > 0 && !is_device_ptr(out_pairs, ctx->device)) return SIMJOIN_ERR_ARG;
     if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
-    *count = 0;
-    ctx->have_timing = false;
-    if (n == 0 || m == 0) return SIMJOIN_OK;
+    return lsh_device(ctx, P, n, Q, m, d, threshold, L, L_low, k, seed, out_pairs, capacity, count);
+}
 
-    JoinParams jp;
-    size_t smem = 0;
-    if (!tile_geometry(ctx, n, m, d, 1, jp, smem, true)) return SIMJOIN_ERR_UNSUPPORTED;
-    const int nb_max = 1 << k;
-    const size_t max_units = (size_t)((n + P_ROWS - 1) / P_ROWS) + (size_t)nb_max;
-    // misc: hist_p | hist_q | cursor_p | cursor_q (nb words each) | nunits (padded to 16 B) | units
-    const size_t off_units = ((size_t)4 * nb_max * 4 + 16 + 15) & ~(size_t)15;
-    const int reps = L + L_low;
-    const int rec_words = (reps + 7) / 8, stride = rec_words * 8;   // key record of a row: 16-bit keys, padded to 16 bytes
-    const size_t rec_bytes = (size_t)rec_words * 16;
-    if (!grow(ctx->lsh_keys_p, n * rec_bytes) || !grow(ctx->lsh_keys_q, m * rec_bytes) ||
-        !grow(ctx->lsh_skeys_p, n * rec_bytes) || !grow(ctx->lsh_skeys_q, m * rec_bytes) ||
-        !grow(ctx->lsh_perm_p, (size_t)n * 4) || !grow(ctx->lsh_perm_q, (size_t)m * 4) ||
-        !grow(ctx->lsh_sorted_p, (size_t)n * d) || !grow(ctx->lsh_sorted_q, (size_t)m * d) ||
-        !grow(ctx->lsh_misc, off_units + max_units * 16))
-        return SIMJOIN_ERR_CUDA;
-    unsigned int *hist_p = reinterpret_cast<unsigned int *>(ctx->lsh_misc.ptr);
-    unsigned int *hist_q = hist_p + nb_max, *cursor_p = hist_q + nb_max, *cursor_q = cursor_p + nb_max, *nunits = cursor_q + nb_max;
-    int4 *units = reinterpret_cast<int4 *>(reinterpret_cast<unsigned char *>(ctx->lsh_misc.ptr) + off_units);
-    uint16_t *keys_p = reinterpret_cast<uint16_t *>(ctx->lsh_keys_p.ptr), *keys_q = reinterpret_cast<uint16_t *>(ctx->lsh_keys_q.ptr);
-    int *perm_p = reinterpret_cast<int *>(ctx->lsh_perm_p.ptr), *perm_q = reinterpret_cast<int *>(ctx->lsh_perm_q.ptr);
-
-    jp.out = reinterpret_cast<int2 *>(out_pairs);
-    jp.capacity = capacity;
-    jp.counter = ctx->d_ctrl;
-    jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
-    jp.ioff = (int)ctx->ioff;
-    jp.joff = (int)ctx->joff;
-    jp.thr_i = clamp_to_i32(std::ceil(threshold));
-    jp.units = units;
-    jp.nunits = nunits;
-    jp.perm_p = perm_p;
-    jp.perm_q = perm_q;
-    jp.rec_p = reinterpret_cast<const uint4 *>(ctx->lsh_skeys_p.ptr);
-    jp.rec_q = reinterpret_cast<const uint4 *>(ctx->lsh_skeys_q.ptr);
-    jp.rec_words = rec_words;
-
-    CUtensorMap mapP, mapQ;
-    if (!encode_rows_map(ctx, &mapP, ctx->lsh_sorted_p.ptr, n, d, P_ROWS) ||
-        !encode_rows_map(ctx, &mapQ, ctx->lsh_sorted_q.ptr, m, d, TILE_N))
-        return SIMJOIN_ERR_CUDA;
-
-    cudaStream_t s = ctx->stream;
-    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    // 16-bit epilogue when every score provably fits (as in the brute-force join)
-    unsigned int *d_max = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 2);
-    maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(P), (long long)n * d / 16, d_max);
-    maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(Q), (long long)m * d / 16, d_max + 1);
-    if (cudaGetLastError() != cudaSuccess ||
-        cudaMemcpyAsync(ctx->h_ctrl + 2, ctx->d_ctrl + 2, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaStreamSynchronize(s) != cudaSuccess) {
-        cudaGetLastError();
-        return SIMJOIN_ERR_CUDA;
-    }
-    const unsigned int *h_max = reinterpret_cast<const unsigned int *>(ctx->h_ctrl + 2);
-    const bool narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
-
-    cudaEventRecord(ctx->ev[0], s);
-    if (d <= LSH_KEYS_STAGED_MAX_D) {
-        const size_t sm = (size_t)LSH_KEYS_STAGED_ROWS * (d / 4 + 1) * 4;
-        lsh_keys_staged_kernel<<<(unsigned)((n + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), 256, sm, s>>>(
-            reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p, stride);
-        lsh_keys_staged_kernel<<<(unsigned)((m + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), 256, sm, s>>>(
-            reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q, stride);
-    } else {
-        lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p,
-                                                                    stride);
-        lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q,
-                                                                    stride);
-    }
-    if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    cudaEventRecord(ctx->ev[1], s);
-    const int g = d / 16;
-    const unsigned hist_blocks = (unsigned)ctx->num_sms * 4;
-    const int rows_per_block = LSH_SORT_THREADS * LSH_SORT_ITEMS;
-    for (int l = 0; l < reps; ++l) {
-        const uint16_t *kp = keys_p + l, *kq = keys_q + l;          // column l of the key records
-        const int nb = l < L ? nb_max : nb_max / 2;          // buckets of this repetition
-        if (cudaMemsetAsync(hist_p, 0, (size_t)2 * nb_max * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kp, stride, n, nb, hist_p);
-        lsh_hist_kernel<<<hist_blocks, LSH_SORT_THREADS, 0, s>>>(kq, stride, m, nb, hist_q);
-        lsh_offsets_units_kernel<<<1, 1024, 0, s>>>(hist_p, hist_q, nb, cursor_p, cursor_q, units, nunits, P_ROWS);
-        lsh_scatter_kernel<<<(unsigned)((n + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kp, stride, n, nb,
-                                                                                                              cursor_p, perm_p);
-        lsh_scatter_kernel<<<(unsigned)((m + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(kq, stride, m, nb,
-                                                                                                              cursor_q, perm_q);
-        lsh_gather_rows_kernel<<<(unsigned)(((long long)n * g + 255) / 256), 256, 0, s>>>(
-            reinterpret_cast<const uint4 *>(P), perm_p, n, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_p.ptr));
-        lsh_gather_rows_kernel<<<(unsigned)(((long long)m * g + 255) / 256), 256, 0, s>>>(
-            reinterpret_cast<const uint4 *>(Q), perm_q, m, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_q.ptr));
-        if (l > 0) {
-            // key records in regrouped order, for the duplicate check of the join's epilogue
-            lsh_gather_rows_kernel<<<(unsigned)(((long long)n * rec_words + 255) / 256), 256, 0, s>>>(
-                reinterpret_cast<const uint4 *>(keys_p), perm_p, n, rec_words, reinterpret_cast<uint4 *>(ctx->lsh_skeys_p.ptr));
-            lsh_gather_rows_kernel<<<(unsigned)(((long long)m * rec_words + 255) / 256), 256, 0, s>>>(
-                reinterpret_cast<const uint4 *>(keys_q), perm_q, m, rec_words, reinterpret_cast<uint4 *>(ctx->lsh_skeys_q.ptr));
-        }
-        if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
-        jp.rep = l;
-        const cudaError_t e = narrow ? launch_join<DT_I8, KIND_IP, true, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem)
-                                     : launch_join<DT_I8, KIND_IP, false, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem);
-        if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    }
-    cudaEventRecord(ctx->ev[2], s);
-    if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) {
-        cudaGetLastError();
-        return SIMJOIN_ERR_CUDA;
-    }
-    if ((unsigned int)(ctx->h_ctrl[1] & 0xffffffffu) != 0) return SIMJOIN_ERR_TIMEOUT;
-    *count = ctx->h_ctrl[0];
-    float a = 0.f, b = 0.f;
-    if (cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess && cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
-        ctx->prepass_ms = a;       // hashing
-        ctx->join_ms = b;          // L x (regroup + bucketed join)
-        ctx->have_timing = true;
-    }
-    return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
+simjoin_status simjoin_run_hamming_lsh(simjoin_ctx *ctx, const void *P_bits, int64_t n, const void *Q_bits, int64_t m, int32_t d,
+                                       double r, int32_t L, int32_t L_low, int32_t k, uint64_t seed, int32_t *out_pairs,
+                                       uint64_t capacity, uint64_t *count) {
+    simjoin_status st = check_hamming_args(ctx, P_bits, n, Q_bits, m, d, r, out_pairs, capacity, count);
+    if (st != SIMJOIN_OK) return st;
+    st = check_lsh_args(L, L_low, k);
+    if (st != SIMJOIN_OK) return st;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    st = hamming_unpack(ctx, P_bits, n, Q_bits, m, d, out_pairs, capacity, count);
+    if (st != SIMJOIN_OK || n == 0 || m == 0) return st;
+    const double t = (double)d - 2.0 * std::floor(r);
+    return lsh_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, t, L, L_low, k, seed, out_pairs, capacity, count);
 }
 
 simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, int32_t d, int32_t k, uint64_t seed, void *out) {

@@ -132,3 +132,22 @@ def test_lsh_offsets_capacity_and_errors(ctx):
     # the plain join still works on the same context afterwards
     got, cnt = ctx.join(dP, dQ, "ip", w.threshold, 1 << 16)
     assert cnt == O.join(w.P, w.Q, "ip", w.threshold, "i8")[1]
+
+
+@pytest.mark.parametrize("n,m,d,L,k", [(700, 900, 128, 4, 3), (3000, 2600, 256, 6, 5), (1200, 800, 1024, 3, 2)])
+def test_lsh_hamming_join_on_packed_bits(ctx, n, m, d, L, k):
+    """simjoin_run_hamming_lsh: bits -> +-1 operand transform, then the LSH-bucketed join; the sampled bit is the hash."""
+    Pb = W.random_bits(n, d, 51)
+    Qb = W.random_bits(m, d, 52, planted_from=Pb[: min(n, m, 200)], flips=d // 16)
+    dP, dQ = torch.from_numpy(Pb).cuda(), torch.from_numpy(Qb).cuda()
+    for r in (d // 16, 0.43 * d):
+        out = torch.full((1 << 20, 2), -5, dtype=torch.int32, device="cuda:0")
+        st, cnt = ctx.simjoin_run_hamming_lsh(dP, n, dQ, m, d, r, L, k, 77, out, 1 << 20, L_low=1)
+        assert st == B.SIMJOIN_OK, B.strerror(st)
+        want, wcnt = O.lsh_join_hamming(Pb, Qb, d, r, L, k, 77, L_low=1)
+        got = keys(out[:cnt].cpu().numpy())
+        assert cnt == wcnt and len(np.unique(got)) == cnt and np.array_equal(got, keys(want)), (n, m, d, r, cnt, wcnt)
+        assert cnt > 0
+    assert ctx.simjoin_run_hamming_lsh(dP, n, dQ, m, d, -1.0, L, k, 1, out, 8)[0] == B.SIMJOIN_ERR_ARG
+    assert ctx.simjoin_run_hamming_lsh(dP, n, dQ, m, d, 3.0, 0, k, 1, out, 8)[0] == B.SIMJOIN_ERR_ARG
+    assert ctx.simjoin_run_hamming_lsh(dP, n, dQ, m, d + 64, 3.0, L, k, 1, out, 8)[0] == B.SIMJOIN_ERR_UNSUPPORTED

@@ -124,6 +124,25 @@ def test_lsh_join_is_brute_force_restricted_to_colliding_pairs():
     assert as_set(all_pairs) == as_set(O.join(w.P, w.Q, "ip", 40.0, "i8")[0])
 
 
+def test_lsh_hamming_join_is_the_hamming_join_restricted_to_equal_sampled_bits():
+    # independent route: keys straight from the packed bits (the sampled bit is the hash), distances by XOR + popcount
+    d, L, k, seed = 128, 4, 5, 321
+    Pb = W.random_bits(500, d, 41)
+    Qb = W.random_bits(600, d, 42, planted_from=Pb[:60], flips=6)
+    coords = np.array([[_splitmix64(seed, l * 64 + b) % d for b in range(k)] for l in range(L)])
+    bp = np.unpackbits(Pb, axis=1, bitorder="little")[:, :d]
+    bq = np.unpackbits(Qb, axis=1, bitorder="little")[:, :d]
+    kp = (bp[:, coords].astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T
+    kq = (bq[:, coords].astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T
+    collide = (kp[:, :, None] == kq[:, None, :]).any(axis=0)
+    H = (bp[:, None, :] != bq[None, :, :]).sum(axis=2)
+    for r in (6, 40.5, 55):
+        ii, jj = np.nonzero(collide & (H <= r))
+        pairs, cnt = O.lsh_join_hamming(Pb, Qb, d, r, L, k, seed)
+        assert as_set(pairs) == set(zip(ii.tolist(), jj.tolist())) and cnt == len(ii)
+        assert as_set(pairs) <= as_set(O.join_hamming(Pb, Qb, d, r)[0])
+
+
 def test_lsh_recall_matches_the_collision_probability():
     # planted pairs differ in h = 8 of d = 128 coordinates: one k-bit sample collides with probability close
     # to (1 - h/d)^k, so the recall over L repetitions is about 1 - (1 - (1-h/d)^k)^L
