@@ -346,6 +346,9 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
             e2 = launch_norms<false>(ctx, Q, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
         }
         if (e1 != cudaSuccess || e2 != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        // the padding of ny up to whole tiles is read (and masked) by the epilogue: keep it defined
+        const size_t pad = (size_t)jp.QT * tn - (size_t)m;
+        if (pad > 0 && cudaMemsetAsync(static_cast<char *>(ctx->ny.ptr) + (size_t)m * 4, 0, pad * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     }
     cudaEventRecord(ctx->ev[1], s);
     const int grid = ctx->num_sms;
