@@ -126,7 +126,7 @@ struct Unit {
     int pb, q0, q1;
     int prow0, prows, qrow0, qrows;   // bucketed mode only
 };
-template <bool GROUPED>
+template <bool GROUPED, int TN = TILE_N>
 __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
     const int G = gridDim.x, c = blockIdx.x;
     if constexpr (GROUPED) {
@@ -136,7 +136,7 @@ __device__ __forceinline__ bool get_unit(const JoinParams &p, int u, Unit &un) {
         const int4 e = __ldg(p.units + idx);
         un.pb = 0;
         un.q0 = 0;
-        un.q1 = (e.w + TILE_N - 1) / TILE_N;
+        un.q1 = (e.w + TN - 1) / TN;
         un.prow0 = e.x; un.prows = e.y; un.qrow0 = e.z; un.qrows = e.w;
         return true;
     }
@@ -530,14 +530,14 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
 // of N = 256 per chunk (1024 tensor cycles), block s accumulating in TMEM columns s * 256 ...  Per unit of work
 // that is 64 KiB of operand traffic per 1024 tensor cycles instead of the 48 KiB per 552 of the streamed
 // 256 x 128 tile, and the accumulator hand-off is paid once per K loop.
-template <int DT>
+template <int DT, bool GROUPED>
 __device__ __forceinline__ void mma_issuer_long(const JoinParams &p, Ctrl *ctrl, uint8_t *smem_ring, const uint32_t tmem_base,
                                                 const int lane) {
     constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, LONG_TN);
     uint32_t stage = 0, phase = 0, accph = 0;
     bool ok = true;
     Unit un;
-    for (int u = 0; ok && get_unit<false>(p, u, un); ++u) {
+    for (int u = 0; ok && get_unit<GROUPED, LONG_TN>(p, u, un); ++u) {
         if (un.q1 <= un.q0) continue;
         for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
             ok = wait_bar_warp(&ctrl->tempty[0], accph ^ 1, ctrl, p.status, 4);
@@ -601,7 +601,7 @@ template <int DT, int KIND, bool NARROW = false, int KC = 0, bool GROUPED = fals
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ, const JoinParams p_in) {
     constexpr bool LONGK = GEO == GEO_LONG, WIDEQ = GEO == GEO_WIDEQ;
-    static_assert(!LONGK || (KC == 0 && !GROUPED && KIND != KIND_STORE), "long-row mode: general join kinds only");
+    static_assert(!LONGK || (KC == 0 && KIND != KIND_STORE), "long-row mode: general join kinds only");
     static_assert(!WIDEQ || (KC == 0 && !GROUPED && KIND == KIND_STORE), "wide-Q mode: store kind only");
     constexpr int TN = (LONGK || WIDEQ) ? LONG_TN : TILE_N;   // rows of Q per tile
     constexpr int NPASS = TN / EPI_COLS;                   // 128-column passes of an epilogue warp over its block
@@ -664,7 +664,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         uint32_t stage = 0, phase = 0, pbuf = 0, pphase = 0;
         bool ok = true;
         Unit un;
-        for (int u = 0; ok && get_unit<GROUPED>(p, u, un); ++u) {
+        for (int u = 0; ok && get_unit<GROUPED, TN>(p, u, un); ++u) {
             if (un.q1 <= un.q0) continue;            // nothing for this CTA in this wave (all roles skip it)
             const int p_row = GROUPED ? un.prow0 : un.pb * P_ROWS;
             if (p.stationary) {
@@ -719,7 +719,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         const bool fast = p.stationary && p.epi_release && p.last_ksteps == 4;
         constexpr bool OB = KIND == KIND_STORE;
         if constexpr (LONGK) {
-            if (warp == 1) mma_issuer_long<DT>(p, ctrl, smem_ring, tmem_base, lane);
+            if (warp == 1) mma_issuer_long<DT, GROUPED>(p, ctrl, smem_ring, tmem_base, lane);
         } else if (fast && p.kc == 1 && !WIDEQ) mma_issuer_role<DT, 1, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
         else if (fast && p.kc == 2 && !WIDEQ) mma_issuer_role<DT, 2, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
         else mma_issuer_role<DT, 0, GROUPED, OB, WIDEQ>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
@@ -733,7 +733,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         int stage_fill = 0;
         bool ok = true;
         Unit un;
-        for (int u = 0; ok && get_unit<GROUPED>(p, u, un); ++u) {
+        for (int u = 0; ok && get_unit<GROUPED, TN>(p, u, un); ++u) {
             if (un.q1 <= un.q0) continue;
             const long long i = GROUPED ? (long long)un.prow0 + row_in_tile : (long long)un.pb * P_ROWS + row_in_tile;
             const bool row_ok = GROUPED ? row_in_tile < un.prows : i < p.n;

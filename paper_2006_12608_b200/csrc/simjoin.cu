@@ -49,7 +49,7 @@ struct simjoin_ctx {
     float prepass_ms, join_ms;
     long long ioff, joff;
     bool attr_set[2][4][2][3][2];
-    bool attr_set_long[2][3][2];
+    bool attr_set_long[2][3][2][2];
     bool attr_set_wideq;
     cudaStream_t copy_stream;           // simjoin_run_host: uploads of Q slices overlap the joins of earlier slices
     cudaEvent_t copy_ev[66];
@@ -184,14 +184,14 @@ cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorM
 // keep P resident at all.
 constexpr int LONG_MIN_KC = 4;
 // The long-row geometry (256 x 256 tiles, nothing resident, one accumulator buffer): general join kinds only.
-template <int DT, int KIND, bool NARROW>
+template <int DT, int KIND, bool NARROW, bool GROUPED = false>
 cudaError_t launch_join_long(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
                              size_t smem) {
-    auto kern = join_kernel<DT, KIND, NARROW, 0, false, GEO_LONG>;
-    if (!ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0]) {
+    auto kern = join_kernel<DT, KIND, NARROW, 0, GROUPED, GEO_LONG>;
+    if (!ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0][GROUPED ? 1 : 0]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
         if (e != cudaSuccess) return e;
-        ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0] = true;
+        ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0][GROUPED ? 1 : 0] = true;
     }
     kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
     return cudaGetLastError();
@@ -400,6 +400,15 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     JoinParams jp;
     size_t smem = 0;
     if (!tile_geometry(ctx, n, m, d, 1, jp, smem, true)) return SIMJOIN_ERR_UNSUPPORTED;
+    // rows of 512 bytes and more: the long-row geometry inside the buckets too
+    const bool longk = jp.kc >= LONG_MIN_KC;
+    if (longk) {
+        jp.stationary = 0;
+        jp.epi_release = 0;
+        jp.nstages = LONG_STAGES;
+        smem = 1024 + (size_t)LONG_STAGES * LONG_STAGE_BYTES + STAGING_BYTES + CTRL_BYTES;
+        if (smem > (size_t)ctx->max_smem_optin) return SIMJOIN_ERR_UNSUPPORTED;
+    }
     const int nb_max = 1 << k;
     const size_t max_units = (size_t)((n + P_ROWS - 1) / P_ROWS) + (size_t)nb_max;
     // misc: hist_p | hist_q | cursor_p | cursor_q (nb words each) | nunits (padded to 16 B) | units
@@ -436,7 +445,7 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
 
     CUtensorMap mapP, mapQ;
     if (!encode_rows_map(ctx, &mapP, ctx->lsh_sorted_p.ptr, n, d, P_ROWS) ||
-        !encode_rows_map(ctx, &mapQ, ctx->lsh_sorted_q.ptr, m, d, TILE_N))
+        !encode_rows_map(ctx, &mapQ, ctx->lsh_sorted_q.ptr, m, d, longk ? LONG_TN : TILE_N))
         return SIMJOIN_ERR_CUDA;
 
     cudaStream_t s = ctx->stream;
@@ -496,8 +505,11 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         }
         if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
         jp.rep = l;
-        const cudaError_t e = narrow ? launch_join<DT_I8, KIND_IP, true, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem)
-                                     : launch_join<DT_I8, KIND_IP, false, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem);
+        const cudaError_t e =
+            longk ? (narrow ? launch_join_long<DT_I8, KIND_IP, true, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem)
+                            : launch_join_long<DT_I8, KIND_IP, false, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem))
+                  : (narrow ? launch_join<DT_I8, KIND_IP, true, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem)
+                            : launch_join<DT_I8, KIND_IP, false, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem));
         if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
     }
     cudaEventRecord(ctx->ev[2], s);
