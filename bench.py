@@ -240,6 +240,10 @@ def size_kw(args):
         kw["m"] = args.m
     if args.planted is not None and args.config != 5:
         kw["planted"] = args.planted
+    if args.d is not None:
+        kw["d"] = args.d
+    if args.threshold is not None:
+        kw["threshold"] = args.threshold
     return kw
 
 
@@ -255,6 +259,8 @@ def main():
     ap.add_argument("--n", type=int, default=None, help="override the row count of P (profiling / experiments)")
     ap.add_argument("--m", type=int, default=None, help="override the row count of Q")
     ap.add_argument("--planted", type=int, default=None)
+    ap.add_argument("--d", type=int, default=None, help="override the dimension (profiling other row lengths; give --threshold too)")
+    ap.add_argument("--threshold", type=float, default=None)
     ap.add_argument("--sigma-reading", default="radial")
     ap.add_argument("--lsh", default=None, metavar="L,k[,L_low]",
                     help="time the LSH-bucketed join (int8 inner-product configs) instead of the brute-force join: "
