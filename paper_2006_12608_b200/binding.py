@@ -192,6 +192,30 @@ class Simjoin:
             raise SimjoinError(st, "simjoin_run")
         return out[:min(cnt, capacity)], cnt
 
+    def join_lsh(self, P, Q, threshold: float, L: int, k: int, seed: int, capacity: int, L_low: int = 0, out=None):
+        """LSH-bucketed inner-product join of two int8 device tensors (simjoin_run_lsh).
+        Returns (pairs[min(count, capacity), 2] int32 device tensor, count)."""
+        import torch
+        n, d = P.shape
+        m = Q.shape[0]
+        if out is None:
+            out = torch.empty((max(int(capacity), 1), 2), dtype=torch.int32, device=P.device)
+        st, cnt = self.simjoin_run_lsh(P, n, Q, m, d, threshold, L, k, seed, out if capacity else None, capacity, L_low=L_low)
+        if st not in (SIMJOIN_OK, SIMJOIN_ERR_CAPACITY):
+            raise SimjoinError(st, "simjoin_run_lsh")
+        return out[:min(cnt, capacity)], cnt
+
+    def jl_transform(self, X, k: int, seed: int, out=None):
+        """JL transform of a bf16 device tensor (rows x d) to (rows x k) bf16 (simjoin_jl_transform)."""
+        import torch
+        n, d = X.shape
+        if out is None:
+            out = torch.empty((n, k), dtype=torch.bfloat16, device=X.device)
+        st = self.simjoin_jl_transform(X, n, d, k, seed, out)
+        if st != SIMJOIN_OK:
+            raise SimjoinError(st, "simjoin_jl_transform")
+        return out
+
     def close(self):
         if getattr(self, "_h", None) is not None and self._h.value:
             load().simjoin_destroy(self._h)

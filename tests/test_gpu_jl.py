@@ -94,3 +94,19 @@ def test_jl_argument_errors(ctx):
     assert ctx.simjoin_jl_transform(X, 0, 256, 64, 1, out) == B.SIMJOIN_OK
     with B.Simjoin("i8", 0) as ci:
         assert ci.simjoin_jl_transform(X, 64, 256, 64, 1, out) == B.SIMJOIN_ERR_UNSUPPORTED
+
+
+def test_binding_conveniences(ctx):
+    X = B.to_device(W.random_points("bf16", 500, 256, 3))
+    Y = ctx.jl_transform(X, 32, 9)
+    assert Y.shape == (500, 32) and Y.dtype == torch.bfloat16
+    want = O.jl_transform(W.random_points("bf16", 500, 256, 3), 32, 9)
+    assert np.abs(Y.float().cpu().numpy() - want).max() < 0.05 * np.abs(want).max()
+    with pytest.raises(B.SimjoinError):
+        ctx.jl_transform(X, 96, 9)
+    w = W.make_workload(4, n=1500, m=1200, planted=100)
+    with B.Simjoin("i8", 0) as ci:
+        pairs, cnt = ci.join_lsh(B.to_device(w.P), B.to_device(w.Q), w.threshold, 4, 3, 5, 1 << 16)
+        want_pairs, wcnt = O.lsh_join(w.P, w.Q, w.threshold, 4, 3, 5)
+        got = pairs.cpu().numpy().astype(np.int64)
+        assert cnt == wcnt and set(map(tuple, got)) == set(map(tuple, want_pairs.astype(np.int64)))
