@@ -308,6 +308,21 @@ void oracle_lsh_keys_i8(const int8_t *X, int64_t rows, int32_t d, int32_t L_high
         }
 }
 
+/* The same keys for bf16 rows: bit b = [x_{c(l,b)} > 0] on the value the 16-bit pattern denotes (+-0 -> 0).  For
+ * rows drawn from a rotation-invariant distribution this is the random-hyperplane hash of the angular distance with
+ * axis-aligned hyperplanes: two points at angle theta agree on a sampled sign with probability 1 - theta / pi. */
+void oracle_lsh_keys_bf16(const uint16_t *X, int64_t rows, int32_t d, int32_t L_high, int32_t L_low, int32_t k, uint64_t seed,
+                          uint32_t *keys) {
+    for (int32_t l = 0; l < L_high + L_low; ++l)
+        for (int64_t i = 0; i < rows; ++i) {
+            uint32_t key = 0;
+            const int32_t bits = l < L_high ? k : k - 1;
+            for (int32_t b = 0; b < bits; ++b)
+                if (oracle_bf16_to_f64(X[(size_t)i * d + oracle_lsh_coordinate(seed, l, b, d)]) > 0.0) key |= 1u << b;
+            keys[(size_t)l * rows + i] = key;
+        }
+}
+
 int64_t oracle_lsh_join_i8(const int8_t *P, int64_t n, const int8_t *Q, int64_t m, int32_t d, double threshold,
                            int32_t L_high, int32_t L_low, int32_t k, uint64_t seed, int32_t *out_pairs, int64_t capacity,
                            int32_t nthreads) {

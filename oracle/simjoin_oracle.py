@@ -74,6 +74,8 @@ def _load():
     lib.oracle_lsh_join_i8.argtypes = [vp, i64, vp, i64, i32, dbl, i32, i32, i32, c.c_uint64, vp, i64, i32]
     lib.oracle_lsh_keys_i8.restype = None
     lib.oracle_lsh_keys_i8.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, vp]
+    lib.oracle_lsh_keys_bf16.restype = None
+    lib.oracle_lsh_keys_bf16.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, vp]
     lib.oracle_lsh_coordinate.restype = i32
     lib.oracle_lsh_coordinate.argtypes = [c.c_uint64, i32, i32, i32]
     lib.oracle_jl_levels.restype = i32
@@ -195,13 +197,37 @@ def lsh_join_hamming(Pbits: np.ndarray, Qbits: np.ndarray, d: int, r: float, L: 
     return lsh_join(widen(Pbits), widen(Qbits), float(d) - 2.0 * np.floor(r), L, k, seed, threads=threads, L_low=L_low)
 
 
-def lsh_keys(X: np.ndarray, L: int, k: int, seed: int, L_low: int = 0) -> np.ndarray:
-    """(L + L_low, rows) uint32 hash keys of int8 rows."""
+def lsh_keys(X: np.ndarray, L: int, k: int, seed: int, L_low: int = 0, dtype: str = "i8") -> np.ndarray:
+    """(L + L_low, rows) uint32 hash keys of int8 rows (or bf16 bit patterns): bit b = [x_c > 0] at the sampled coordinate."""
     lib = _load()
-    X = _check(X, "i8")
+    X = _check(X, dtype)
     out = np.empty((L + L_low, X.shape[0]), dtype=np.uint32)
-    lib.oracle_lsh_keys_i8(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, out.ctypes.data)
+    fn = lib.oracle_lsh_keys_i8 if dtype == "i8" else lib.oracle_lsh_keys_bf16
+    fn(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, out.ctypes.data)
     return out
+
+
+def lsh_restrict(pairs: np.ndarray, P: np.ndarray, Q: np.ndarray, dtype: str, L: int, k: int, seed: int, L_low: int = 0) -> np.ndarray:
+    """The pairs of a (brute-force) join whose hash keys agree in at least one repetition: what the LSH-bucketed join of
+    any kind returns, since it runs the brute-force join inside the buckets of every repetition and takes the union."""
+    kp, kq = lsh_keys(P, L, k, seed, L_low, dtype), lsh_keys(Q, L, k, seed, L_low, dtype)
+    pairs = np.asarray(pairs).reshape(-1, 2)
+    if len(pairs) == 0:
+        return pairs
+    keep = (kp[:, pairs[:, 0]] == kq[:, pairs[:, 1]]).any(axis=0)
+    return pairs[keep]
+
+
+def lsh_join_kind(P, Q, kind: str, threshold: float, dtype: str, L: int, k: int, seed: int, L_low: int = 0, threads: int = 0):
+    """LSH-bucketed join of any kind and element type: the brute-force join restricted to colliding pairs."""
+    pairs, _c = join(P, Q, kind, threshold, dtype, threads=threads)
+    out = lsh_restrict(pairs, P, Q, dtype, L, k, seed, L_low)
+    return out, len(out)
+
+
+def lsh_band_sets(P, Q, kind: str, threshold: float, dtype: str, L: int, k: int, seed: int, L_low: int = 0, rel: float = 1e-2):
+    """band_sets restricted to colliding pairs: a floating-point LSH join G is accepted when S_strict <= G <= S_loose."""
+    return tuple(lsh_restrict(s, P, Q, dtype, L, k, seed, L_low) for s in band_sets(P, Q, kind, threshold, dtype, rel=rel))
 
 
 def lsh_coordinate(seed: int, rep: int, bit: int, d: int) -> int:

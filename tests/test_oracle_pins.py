@@ -143,6 +143,36 @@ def test_lsh_hamming_join_is_the_hamming_join_restricted_to_equal_sampled_bits()
         assert as_set(pairs) <= as_set(O.join_hamming(Pb, Qb, d, r)[0])
 
 
+def test_lsh_sign_keys_for_bf16_rows_and_joins_of_any_kind():
+    # keys re-derived in numpy from the decoded values; the restricted join equals the int8-specific oracle where both apply
+    L, k, seed, d = 4, 6, 55, 96
+    X = W.random_points("bf16", 300, d, 13)
+    X[0, :5] = [0x0000, 0x8000, 0x3f80, 0xbf80, 0x0001]                      # +0, -0, 1, -1, smallest subnormal
+    coords = np.array([[_splitmix64(seed, l * 64 + b) % d for b in range(k)] for l in range(L)])
+    vals = W.bf16_bits_to_f32(X).astype(np.float64)
+    want = ((vals[:, coords] > 0).astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T
+    assert np.array_equal(want, O.lsh_keys(X, L, k, seed, dtype="bf16"))
+    w = W.make_workload(4, n=400, m=500, planted=60)
+    a, ca = O.lsh_join(w.P, w.Q, 40.0, 3, 4, 9, L_low=1)
+    b, cb = O.lsh_join_kind(w.P, w.Q, "ip", 40.0, "i8", 3, 4, 9, L_low=1)
+    assert ca == cb and as_set(a) == as_set(b)
+    # an int8 Euclidean LSH join is a subset of the brute-force one, and everything at distance 0 with equal keys is in it
+    c, cc = O.lsh_join_kind(w.P, w.P, "l2", 3.0, "i8", 2, 5, 9)
+    assert {(i, i) for i in range(400)} <= as_set(c) <= as_set(O.join(w.P, w.P, "l2", 3.0, "i8")[0])
+
+
+def test_lsh_sign_hash_collision_probability_is_one_minus_theta_over_pi():
+    # unit Gaussian rows y = cos(theta) x + sin(theta) z: every sampled sign agrees with probability 1 - theta / pi
+    rng = np.random.default_rng(4)
+    n, d, theta = 3000, 256, 0.5
+    x = rng.standard_normal((n, d)); z = rng.standard_normal((n, d))
+    y = np.cos(theta) * x + np.sin(theta) * z
+    X, Y = W.f32_to_bf16_bits(x.astype(np.float32)), W.f32_to_bf16_bits(y.astype(np.float32))
+    kx, ky = O.lsh_keys(X, 8, 1, 3, dtype="bf16"), O.lsh_keys(Y, 8, 1, 3, dtype="bf16")     # 8 independent single-bit keys
+    agree = (kx == ky).mean()
+    assert abs(agree - (1 - theta / np.pi)) < 0.01, agree
+
+
 def test_lsh_recall_matches_the_collision_probability():
     # planted pairs differ in h = 8 of d = 128 coordinates: one k-bit sample collides with probability close
     # to (1 - h/d)^k, so the recall over L repetitions is about 1 - (1 - (1-h/d)^k)^L
