@@ -123,35 +123,39 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
 #define SIMJOIN_LSH_MAX_BITS 12
 
 /*
- * LSH-bucketed inner-product join (Section 4, the algorithm after the brute-force one): repetitions;
+ * LSH-bucketed join (Section 4, the algorithm after the brute-force one): repetitions;
  * in each, every point is hashed with a concatenation of base hashes from an LSH family, the points
  * are split into buckets by that hash, and the brute-force tile join runs inside each bucket; the
  * result is the union over the repetitions.  For a fractional number of base hashes the paper mixes
  * tables built from ceil(k) and floor(k) base hashes: here L repetitions use k bits and L_low more
  * use k - 1 (the same samples without the last).  The output is therefore exactly
- *     { (i, j) : <x_i, y_j> >= threshold  and  key_l(x_i) == key_l(y_j) for some repetition l },
- * a subset of simjoin_run's (precision 1; the recall is set by L, k and the data).
+ *     { (i, j) of simjoin_run(kind, threshold)  with  key_l(x_i) == key_l(y_j) for some repetition l },
+ * a subset of simjoin_run's (precision 1; the recall is set by L, k and the data; bf16: the same threshold band
+ * as simjoin_run).
  *
  *   Base hash     bit sampling: h(x) = [x_c > 0] for a sampled coordinate c -- the standard family for
- *                 Hamming distance, i.e. for +-1 rows such as simjoin_run_hamming builds.  Bit b of the
+ *                 Hamming distance, i.e. for +-1 rows such as simjoin_run_hamming builds; for bf16 rows the
+ *                 sign of the sampled coordinate, i.e. the random-hyperplane hash of the angular distance
+ *                 with axis-aligned hyperplanes (two rows of a rotation-invariant distribution at angle
+ *                 theta agree with probability 1 - theta/pi).  Bit b of the
  *                 key of repetition l samples coordinate splitmix64(seed, 64*l + b) mod d, where
  *                 splitmix64(seed, i): z = seed + (i+1)*0x9E3779B97F4A7C15; z = (z ^ z>>30)*0xBF58476D1CE4E5B9;
  *                 z = (z ^ z>>27)*0x94D049BB133111EB; z ^ z>>31  (all modulo 2^64).
- *   P, Q, n, m, d, threshold, out_pairs, capacity, count   as simjoin_run with kind = SIMJOIN_IP.
+ *   P, Q, n, m, d, kind, threshold, out_pairs, capacity, count   as simjoin_run (every dtype and kind it accepts).
  *   L, L_low      repetitions with k and with k - 1 bits; both >= 0, 1 <= L + L_low <= SIMJOIN_LSH_MAX_REPS,
  *                 L_low > 0 needs k >= 1 (ERR_ARG otherwise).
  *   k             key bits, 0..SIMJOIN_LSH_MAX_BITS (ERR_ARG if negative, ERR_UNSUPPORTED above);
  *                 k = 0 puts everything in one bucket and returns the brute-force result.
  *
- * I8 contexts only (ERR_UNSUPPORTED otherwise).  Every pair is reported once, whatever the number of
+ * Every pair is reported once, whatever the number of
  * repetitions it collides in; the order is unspecified.  The context keeps regrouped copies of P and Q
  * and two copies of a record of 16-bit keys per row as scratch:
- * (n+m) * (d + 4 + 32*ceil((L+L_low)/8)) bytes.  Hashing, regrouping, the work list and the bucketed
+ * (n+m) * (row bytes + 4 + 32*ceil((L+L_low)/8)) bytes (+ 4 per row for the norm kinds).  Hashing, regrouping, the work list and the bucketed
  * join all run on the device with no host round trip between repetitions.
  * simjoin_last_kernel_ms then reports (hashing, all repetitions).
  */
 simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
-                               double threshold, int32_t L, int32_t L_low, int32_t k, uint64_t seed,
+                               simjoin_kind kind, double threshold, int32_t L, int32_t L_low, int32_t k, uint64_t seed,
                                int32_t *out_pairs, uint64_t capacity, uint64_t *count);
 
 /*

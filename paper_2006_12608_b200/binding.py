@@ -55,7 +55,7 @@ def load() -> ctypes.CDLL:
     lib.simjoin_run_hamming.restype = c.c_int
     lib.simjoin_run_hamming.argtypes = [vp, vp, i64, vp, i64, i32, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_run_lsh.restype = c.c_int
-    lib.simjoin_run_lsh.argtypes = [vp, vp, i64, vp, i64, i32, dbl, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
+    lib.simjoin_run_lsh.argtypes = [vp, vp, i64, vp, i64, i32, c.c_int, dbl, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
     lib.simjoin_run_hamming_lsh.restype = c.c_int
     lib.simjoin_run_hamming_lsh.argtypes = [vp, vp, i64, vp, i64, i32, dbl, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
     lib.simjoin_jl_transform.restype = c.c_int
@@ -144,11 +144,11 @@ class Simjoin:
         st = load().simjoin_run_hamming(self._h, pp, n, qp, m, d, float(r), op, capacity, ctypes.byref(cnt))
         return st, cnt.value
 
-    def simjoin_run_lsh(self, P, n, Q, m, d, threshold, L, k, seed, out_pairs, capacity, L_low=0):
+    def simjoin_run_lsh(self, P, n, Q, m, d, threshold, L, k, seed, out_pairs, capacity, L_low=0, kind="ip"):
         cnt = ctypes.c_uint64(0)
         (pp, _a), (qp, _b), (op, _c) = _ptr(P), _ptr(Q), _ptr(out_pairs)
-        st = load().simjoin_run_lsh(self._h, pp, n, qp, m, d, float(threshold), int(L), int(L_low), int(k), int(seed), op, capacity,
-                                    ctypes.byref(cnt))
+        st = load().simjoin_run_lsh(self._h, pp, n, qp, m, d, KIND[kind] if isinstance(kind, str) else kind, float(threshold),
+                                    int(L), int(L_low), int(k), int(seed), op, capacity, ctypes.byref(cnt))
         return st, cnt.value
 
     def simjoin_run_hamming_lsh(self, P_bits, n, Q_bits, m, d, r, L, k, seed, out_pairs, capacity, L_low=0):
@@ -192,15 +192,15 @@ class Simjoin:
             raise SimjoinError(st, "simjoin_run")
         return out[:min(cnt, capacity)], cnt
 
-    def join_lsh(self, P, Q, threshold: float, L: int, k: int, seed: int, capacity: int, L_low: int = 0, out=None):
-        """LSH-bucketed inner-product join of two int8 device tensors (simjoin_run_lsh).
+    def join_lsh(self, P, Q, threshold: float, L: int, k: int, seed: int, capacity: int, L_low: int = 0, out=None, kind: str = "ip"):
+        """LSH-bucketed join of two device tensors (simjoin_run_lsh).
         Returns (pairs[min(count, capacity), 2] int32 device tensor, count)."""
         import torch
         n, d = P.shape
         m = Q.shape[0]
         if out is None:
             out = torch.empty((max(int(capacity), 1), 2), dtype=torch.int32, device=P.device)
-        st, cnt = self.simjoin_run_lsh(P, n, Q, m, d, threshold, L, k, seed, out if capacity else None, capacity, L_low=L_low)
+        st, cnt = self.simjoin_run_lsh(P, n, Q, m, d, threshold, L, k, seed, out if capacity else None, capacity, L_low=L_low, kind=kind)
         if st not in (SIMJOIN_OK, SIMJOIN_ERR_CAPACITY):
             raise SimjoinError(st, "simjoin_run_lsh")
         return out[:min(cnt, capacity)], cnt

@@ -757,17 +757,26 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 // per-tile filter bound: a necessary condition on max_j s_ij for row i to have any hit
                 int fi = p.thr_i;
                 float ff = p.thr_f;
+                // (min, max) of the per-column term over the tile's rows.  Bucketed mode: the tile starts at any row, so
+                // it takes the bounds of the one or two 256-row blocks it touches (wider, still necessary conditions).
+                int qb0 = qt / (QSTAT_ROWS / TN), qb1 = qb0;
+                if constexpr (GROUPED) {
+                    const long long w0 = q_base + (long long)qt * TN;
+                    const long long last = (p.m - 1) / QSTAT_ROWS;
+                    qb0 = (int)(w0 / QSTAT_ROWS);
+                    qb1 = (int)min((w0 + TN - 1) / QSTAT_ROWS, last);
+                }
                 if constexpr (DT == DT_I8 && KIND == KIND_L2) {
-                    const int2 st = reinterpret_cast<const int2 *>(p.qstat)[qt / (QSTAT_ROWS / TN)];
-                    fi = (ri + st.x + 1) >> 1;                    // 2s >= |x|^2 - R + min|y|^2
+                    const int2 s0 = reinterpret_cast<const int2 *>(p.qstat)[qb0], s1 = reinterpret_cast<const int2 *>(p.qstat)[qb1];
+                    fi = (ri + min(s0.x, s1.x) + 1) >> 1;         // 2s >= |x|^2 - R + min|y|^2
                 }
                 if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
-                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt / (QSTAT_ROWS / TN)];
-                    ff = rf * (p.thr_f >= 0.f ? st.x : st.y);     // s >= t|x| * min|y| (max|y| when t < 0)
+                    const float2 s0 = reinterpret_cast<const float2 *>(p.qstat)[qb0], s1 = reinterpret_cast<const float2 *>(p.qstat)[qb1];
+                    ff = rf * (p.thr_f >= 0.f ? fminf(s0.x, s1.x) : fmaxf(s0.y, s1.y));     // s >= t|x| * min|y| (max|y| when t < 0)
                 }
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
-                    const float2 st = reinterpret_cast<const float2 *>(p.qstat)[qt / (QSTAT_ROWS / TN)];
-                    ff = rf + st.x;                               // (|x|^2 + min|y|^2) - 2s <= r^2
+                    const float2 s0 = reinterpret_cast<const float2 *>(p.qstat)[qb0], s1 = reinterpret_cast<const float2 *>(p.qstat)[qb1];
+                    ff = rf + fminf(s0.x, s1.x);                  // (|x|^2 + min|y|^2) - 2s <= r^2
                 }
                 // per-column terms of this warp's columns, 4 per lane, fetched while the tile is still
                 // being multiplied so that the exact test never waits on global memory
@@ -775,9 +784,13 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
 #pragma unroll
                 for (int ps = 0; ps < NPASS; ++ps) {
                     yq_pass[ps] = make_uint4(0, 0, 0, 0);
-                    if ((KIND == KIND_COS || KIND == KIND_L2) && lane < EPI_COLS / 4)
-                        yq_pass[ps] = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint32_t *>(p.ny) +
-                                                                            ((long long)qt * TN + ps * EPI_COLS)) + lane);
+                    if ((KIND == KIND_COS || KIND == KIND_L2) && lane < EPI_COLS / 4) {
+                        const uint32_t *nyp = reinterpret_cast<const uint32_t *>(p.ny) + (q_base + (long long)qt * TN + ps * EPI_COLS) + 4 * lane;
+                        if constexpr (GROUPED)      // a bucket starts at any row: no 16-byte alignment
+                            yq_pass[ps] = make_uint4(__ldg(nyp), __ldg(nyp + 1), __ldg(nyp + 2), __ldg(nyp + 3));
+                        else
+                            yq_pass[ps] = __ldg(reinterpret_cast<const uint4 *>(nyp));
+                    }
                 }
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
                 if (!ok) break;

@@ -3,7 +3,9 @@
 // bucket is one contiguous row range, then list the (P row block, Q bucket) units the join kernel sweeps.
 //
 // Base hash: bit sampling, h(x) = [x_c > 0] for a sampled coordinate c -- the classic monotone family
-// for Hamming distance / +-1 data.  The coordinate of repetition l, bit b is
+// for Hamming distance / +-1 data, and for bf16 rows the sign of the sampled coordinate (the random-hyperplane
+// hash of the angular distance with axis-aligned hyperplanes; a bf16 value is positive exactly when its bit
+// pattern, read as int16, is).  The coordinate of repetition l, bit b is
 // splitmix64(seed, l * 64 + b) mod d, a counter-based generator, so nothing random is stored.
 #pragma once
 #include <cstdint>
@@ -27,7 +29,8 @@ __host__ __device__ inline uint64_t lsh_splitmix64(uint64_t seed, uint64_t idx) 
 // all keys of a row sit in one or two cache lines): k bits in the first L_high repetitions, k - 1 (the
 // same samples without the last) in the following L_low -- the paper's mix of tables for a fractional
 // number of base hashes.  One thread per row; the sampled coordinates are computed once per block.
-__global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict__ X, long long rows, int d, int L_high, int L_low,
+template <typename T>   // int8_t, or int16_t for bf16 bit patterns
+__global__ void __launch_bounds__(256) lsh_keys_kernel(const T *__restrict__ X, long long rows, int d, int L_high, int L_low,
                                                        int k, unsigned long long seed, uint16_t *__restrict__ rec, int stride) {
     __shared__ int s_coord[LSH_MAX_REPS * LSH_MAX_BITS];
     const int L = L_high + L_low;
@@ -38,7 +41,7 @@ __global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict_
     __syncthreads();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= rows) return;
-    const int8_t *x = X + i * d;
+    const T *x = X + i * d;
     for (int l = 0; l < stride; ++l) {
         uint32_t key = 0;
         const int bits = l < L_high ? k : (l < L ? k - 1 : 0);      // padding entries stay 0
@@ -47,23 +50,25 @@ __global__ void __launch_bounds__(256) lsh_keys_kernel(const int8_t *__restrict_
     }
 }
 
-// The same keys for short rows (d <= LSH_KEYS_STAGED_MAX_D bytes): a block first copies its 64 rows into shared
-// memory with coalesced 16-byte loads (row pitch d + 4 bytes: an odd number of words, so the byte gathers of
+// The same keys for short rows (at most LSH_KEYS_STAGED_MAX_D bytes): a block first copies its 64 rows into shared
+// memory with coalesced 16-byte loads (row pitch: row bytes + 4, an odd number of words, so the gathers of
 // different rows fall into different banks), then four threads per row split the repetitions.  The per-thread
 // gather of the kernel above touches 32 different cache lines with every load instruction.
 constexpr int LSH_KEYS_STAGED_MAX_D = 512;
 constexpr int LSH_KEYS_STAGED_ROWS = 64;
-__global__ void __launch_bounds__(256) lsh_keys_staged_kernel(const int8_t *__restrict__ X, long long rows, int d, int L_high, int L_low,
+template <typename T>
+__global__ void __launch_bounds__(256) lsh_keys_staged_kernel(const T *__restrict__ X, long long rows, int d, int L_high, int L_low,
                                                               int k, unsigned long long seed, uint16_t *__restrict__ rec, int stride) {
     __shared__ int s_coord[LSH_MAX_REPS * LSH_MAX_BITS];
-    extern __shared__ uint32_t s_rows[];                       // LSH_KEYS_STAGED_ROWS x (d / 4 + 1) words
+    extern __shared__ uint32_t s_rows[];                       // LSH_KEYS_STAGED_ROWS x (row bytes / 4 + 1) words
     const int L = L_high + L_low;
     for (int t = threadIdx.x; t < L * k; t += blockDim.x) {
         const int l = t / k, b = t - l * k;
         s_coord[t] = (int)(lsh_splitmix64(seed, (uint64_t)l * 64u + (uint64_t)b) % (uint64_t)d);
     }
     const long long row0 = (long long)blockIdx.x * LSH_KEYS_STAGED_ROWS;
-    const int g = d / 16, pitch = d / 4 + 1;
+    const int row_bytes = d * (int)sizeof(T);
+    const int g = row_bytes / 16, pitch = row_bytes / 4 + 1;
     const uint4 *src = reinterpret_cast<const uint4 *>(X + row0 * d);
     const long long avail = (rows - row0 < LSH_KEYS_STAGED_ROWS ? rows - row0 : LSH_KEYS_STAGED_ROWS) * g;
     for (int t = threadIdx.x; t < LSH_KEYS_STAGED_ROWS * g; t += blockDim.x) {
@@ -77,7 +82,7 @@ __global__ void __launch_bounds__(256) lsh_keys_staged_kernel(const int8_t *__re
     const int r = threadIdx.x >> 2, part = threadIdx.x & 3;
     const long long i = row0 + r;
     if (i >= rows) return;
-    const int8_t *x = reinterpret_cast<const int8_t *>(s_rows + r * pitch);
+    const T *x = reinterpret_cast<const T *>(s_rows + r * pitch);
     for (int l = part; l < stride; l += 4) {
         uint32_t key = 0;
         const int bits = l < L_high ? k : (l < L ? k - 1 : 0);      // padding entries stay 0

@@ -390,16 +390,38 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
 }
 
 // The LSH-bucketed join on device buffers of int8 rows.  Arguments were validated by the caller.
-simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, double threshold,
-                          int32_t L, int32_t L_low, int32_t k, uint64_t seed, int32_t *out_pairs, uint64_t capacity,
-                          uint64_t *count) {
+// One bucketed join launch: instantiation by element type, kind, epilogue width and geometry.
+cudaError_t launch_bucketed(simjoin_ctx *ctx, bool i8, simjoin_kind kind, bool narrow, bool longk, const CUtensorMap &mp,
+                            const CUtensorMap &mq, const JoinParams &jp, size_t smem) {
+    const int grid = ctx->num_sms;
+#define SJ_BUCKETED(DT, KIND, NARROW)                                                          \
+    return longk ? launch_join_long<DT, KIND, NARROW, true>(ctx, mp, mq, jp, grid, smem) \
+                 : launch_join<DT, KIND, NARROW, true>(ctx, mp, mq, jp, grid, smem)
+    if (i8 && kind == SIMJOIN_IP && narrow) { SJ_BUCKETED(DT_I8, KIND_IP, true); }
+    if (i8 && kind == SIMJOIN_IP) { SJ_BUCKETED(DT_I8, KIND_IP, false); }
+    if (i8 && kind == SIMJOIN_L2 && narrow) { SJ_BUCKETED(DT_I8, KIND_L2, true); }
+    if (i8 && kind == SIMJOIN_L2) { SJ_BUCKETED(DT_I8, KIND_L2, false); }
+    if (!i8 && kind == SIMJOIN_IP) { SJ_BUCKETED(DT_BF16, KIND_IP, false); }
+    if (!i8 && kind == SIMJOIN_COS) { SJ_BUCKETED(DT_BF16, KIND_COS, false); }
+    if (!i8 && kind == SIMJOIN_L2) { SJ_BUCKETED(DT_BF16, KIND_L2, false); }
+#undef SJ_BUCKETED
+    return cudaErrorInvalidValue;
+}
+
+simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, simjoin_kind kind,
+                          double threshold, int32_t L, int32_t L_low, int32_t k, uint64_t seed, int32_t *out_pairs,
+                          uint64_t capacity, uint64_t *count) {
     *count = 0;
     ctx->have_timing = false;
     if (n == 0 || m == 0) return SIMJOIN_OK;
+    const bool i8 = ctx->dtype == SIMJOIN_I8;
+    const size_t es = elem_size(ctx->dtype);
+    const int row_bytes = (int)(d * es);
+    const bool need_norms = kind != SIMJOIN_IP;
 
     JoinParams jp;
     size_t smem = 0;
-    if (!tile_geometry(ctx, n, m, d, 1, jp, smem, true)) return SIMJOIN_ERR_UNSUPPORTED;
+    if (!tile_geometry(ctx, n, m, row_bytes, es, jp, smem, true)) return SIMJOIN_ERR_UNSUPPORTED;
     // rows of 512 bytes and more: the long-row geometry inside the buckets too
     const bool longk = jp.kc >= LONG_MIN_KC;
     if (longk) {
@@ -419,8 +441,13 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     if (!grow(ctx->lsh_keys_p, n * rec_bytes) || !grow(ctx->lsh_keys_q, m * rec_bytes) ||
         !grow(ctx->lsh_skeys_p, n * rec_bytes) || !grow(ctx->lsh_skeys_q, m * rec_bytes) ||
         !grow(ctx->lsh_perm_p, (size_t)n * 4) || !grow(ctx->lsh_perm_q, (size_t)m * 4) ||
-        !grow(ctx->lsh_sorted_p, (size_t)n * d) || !grow(ctx->lsh_sorted_q, (size_t)m * d) ||
+        !grow(ctx->lsh_sorted_p, (size_t)n * row_bytes) || !grow(ctx->lsh_sorted_q, (size_t)m * row_bytes) ||
         !grow(ctx->lsh_misc, off_units + max_units * 16))
+        return SIMJOIN_ERR_CUDA;
+    // row terms of the regrouped rows (norm kinds); a bucket's last tile may read up to a tile past the end of ny
+    const size_t ny_entries = (size_t)m + LONG_TN + 8;
+    if (need_norms && (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, ny_entries * 4) ||
+                       !grow(ctx->qstat, (size_t)((m + NORM_TILE_ROWS - 1) / NORM_TILE_ROWS) * 8)))
         return SIMJOIN_ERR_CUDA;
     unsigned int *hist_p = reinterpret_cast<unsigned int *>(ctx->lsh_misc.ptr);
     unsigned int *hist_q = hist_p + nb_max, *cursor_p = hist_q + nb_max, *cursor_q = cursor_p + nb_max, *nunits = cursor_q + nb_max;
@@ -434,7 +461,12 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
     jp.ioff = (int)ctx->ioff;
     jp.joff = (int)ctx->joff;
-    jp.thr_i = clamp_to_i32(std::ceil(threshold));
+    set_thresholds(jp, i8, kind, threshold);
+    if (need_norms) {
+        jp.nx = ctx->nx.ptr;
+        jp.ny = ctx->ny.ptr;
+        jp.qstat = ctx->qstat.ptr;
+    }
     jp.units = units;
     jp.nunits = nunits;
     jp.perm_p = perm_p;
@@ -450,35 +482,52 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
 
     cudaStream_t s = ctx->stream;
     if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    // 16-bit epilogue when every score provably fits (as in the brute-force join)
-    unsigned int *d_max = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 2);
-    maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(P), (long long)n * d / 16, d_max);
-    maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(Q), (long long)m * d / 16, d_max + 1);
-    if (cudaGetLastError() != cudaSuccess ||
-        cudaMemcpyAsync(ctx->h_ctrl + 2, ctx->d_ctrl + 2, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaStreamSynchronize(s) != cudaSuccess) {
-        cudaGetLastError();
-        return SIMJOIN_ERR_CUDA;
+    // int8: 16-bit epilogue when every score provably fits (as in the brute-force join)
+    bool narrow = false;
+    if (i8) {
+        unsigned int *d_max = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 2);
+        maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(P), (long long)n * d / 16, d_max);
+        maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(Q), (long long)m * d / 16, d_max + 1);
+        if (cudaGetLastError() != cudaSuccess ||
+            cudaMemcpyAsync(ctx->h_ctrl + 2, ctx->d_ctrl + 2, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) {
+            cudaGetLastError();
+            return SIMJOIN_ERR_CUDA;
+        }
+        const unsigned int *h_max = reinterpret_cast<const unsigned int *>(ctx->h_ctrl + 2);
+        narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
     }
-    const unsigned int *h_max = reinterpret_cast<const unsigned int *>(ctx->h_ctrl + 2);
-    const bool narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
+    if (need_norms && cudaMemsetAsync(static_cast<char *>(ctx->ny.ptr) + (size_t)m * 4, 0, (ny_entries - (size_t)m) * 4, s) != cudaSuccess)
+        return SIMJOIN_ERR_CUDA;
 
     cudaEventRecord(ctx->ev[0], s);
-    if (d <= LSH_KEYS_STAGED_MAX_D) {
-        const size_t sm = (size_t)LSH_KEYS_STAGED_ROWS * (d / 4 + 1) * 4;
-        lsh_keys_staged_kernel<<<(unsigned)((n + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), 256, sm, s>>>(
-            reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p, stride);
-        lsh_keys_staged_kernel<<<(unsigned)((m + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), 256, sm, s>>>(
-            reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q, stride);
-    } else {
-        lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(P), n, d, L, L_low, k, seed, keys_p,
-                                                                    stride);
-        lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(reinterpret_cast<const int8_t *>(Q), m, d, L, L_low, k, seed, keys_q,
-                                                                    stride);
+    {
+        const unsigned bn = (unsigned)((n + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), bm = (unsigned)((m + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS);
+        const size_t sm = (size_t)LSH_KEYS_STAGED_ROWS * (row_bytes / 4 + 1) * 4;
+        const bool staged = row_bytes <= LSH_KEYS_STAGED_MAX_D;
+        if (i8) {
+            const int8_t *p8 = reinterpret_cast<const int8_t *>(P), *q8 = reinterpret_cast<const int8_t *>(Q);
+            if (staged) {
+                lsh_keys_staged_kernel<<<bn, 256, sm, s>>>(p8, n, d, L, L_low, k, seed, keys_p, stride);
+                lsh_keys_staged_kernel<<<bm, 256, sm, s>>>(q8, m, d, L, L_low, k, seed, keys_q, stride);
+            } else {
+                lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(p8, n, d, L, L_low, k, seed, keys_p, stride);
+                lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(q8, m, d, L, L_low, k, seed, keys_q, stride);
+            }
+        } else {
+            const int16_t *p16 = reinterpret_cast<const int16_t *>(P), *q16 = reinterpret_cast<const int16_t *>(Q);
+            if (staged) {
+                lsh_keys_staged_kernel<<<bn, 256, sm, s>>>(p16, n, d, L, L_low, k, seed, keys_p, stride);
+                lsh_keys_staged_kernel<<<bm, 256, sm, s>>>(q16, m, d, L, L_low, k, seed, keys_q, stride);
+            } else {
+                lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(p16, n, d, L, L_low, k, seed, keys_p, stride);
+                lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(q16, m, d, L, L_low, k, seed, keys_q, stride);
+            }
+        }
     }
     if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
     cudaEventRecord(ctx->ev[1], s);
-    const int g = d / 16;
+    const int g = row_bytes / 16;
     const unsigned hist_blocks = (unsigned)ctx->num_sms * 4;
     const int rows_per_block = LSH_SORT_THREADS * LSH_SORT_ITEMS;
     for (int l = 0; l < reps; ++l) {
@@ -503,14 +552,22 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
             lsh_gather_rows_kernel<<<(unsigned)(((long long)m * rec_words + 255) / 256), 256, 0, s>>>(
                 reinterpret_cast<const uint4 *>(keys_q), perm_q, m, rec_words, reinterpret_cast<uint4 *>(ctx->lsh_skeys_q.ptr));
         }
+        if (need_norms) {
+            // row terms and per-256-row bounds of the regrouped rows
+            const int sq = kind == SIMJOIN_COS ? 1 : 0;
+            cudaError_t e1, e2;
+            if (i8) {
+                e1 = launch_norms<true>(ctx, ctx->lsh_sorted_p.ptr, n, d, 0, ctx->nx.ptr, nullptr);
+                e2 = launch_norms<true>(ctx, ctx->lsh_sorted_q.ptr, m, d, 0, ctx->ny.ptr, ctx->qstat.ptr);
+            } else {
+                e1 = launch_norms<false>(ctx, ctx->lsh_sorted_p.ptr, n, d, sq, ctx->nx.ptr, nullptr);
+                e2 = launch_norms<false>(ctx, ctx->lsh_sorted_q.ptr, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
+            }
+            if (e1 != cudaSuccess || e2 != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        }
         if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
         jp.rep = l;
-        const cudaError_t e =
-            longk ? (narrow ? launch_join_long<DT_I8, KIND_IP, true, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem)
-                            : launch_join_long<DT_I8, KIND_IP, false, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem))
-                  : (narrow ? launch_join<DT_I8, KIND_IP, true, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem)
-                            : launch_join<DT_I8, KIND_IP, false, true>(ctx, mapP, mapQ, jp, ctx->num_sms, smem));
-        if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        if (launch_bucketed(ctx, i8, kind, narrow, longk, mapP, mapQ, jp, smem) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     }
     cudaEventRecord(ctx->ev[2], s);
     if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
@@ -772,12 +829,11 @@ simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t
     return run_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, SIMJOIN_IP, t, out_pairs, capacity, count);
 }
 
-simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, double threshold,
-                               int32_t L, int32_t L_low, int32_t k, uint64_t seed, int32_t *out_pairs, uint64_t capacity,
-                               uint64_t *count) {
-    simjoin_status st = check_join_args(ctx, P, n, Q, m, d, SIMJOIN_IP, threshold, out_pairs, capacity, count);
+simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
+                               simjoin_kind kind, double threshold, int32_t L, int32_t L_low, int32_t k, uint64_t seed,
+                               int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+    simjoin_status st = check_join_args(ctx, P, n, Q, m, d, kind, threshold, out_pairs, capacity, count);
     if (st != SIMJOIN_OK) return st;
-    if (ctx->dtype != SIMJOIN_I8) return SIMJOIN_ERR_UNSUPPORTED;
     st = check_lsh_args(L, L_low, k);
     if (st != SIMJOIN_OK) return st;
     DeviceGuard guard(ctx->device);
@@ -785,7 +841,7 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
     if ((n > 0 && !is_device_ptr(P, ctx->device)) || (m > 0 && !is_device_ptr(Q, ctx->device))) return SIMJOIN_ERR_ARG;
     if (capacity > 0 && !is_device_ptr(out_pairs, ctx->device)) return SIMJOIN_ERR_ARG;
     if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
-    return lsh_device(ctx, P, n, Q, m, d, threshold, L, L_low, k, seed, out_pairs, capacity, count);
+    return lsh_device(ctx, P, n, Q, m, d, kind, threshold, L, L_low, k, seed, out_pairs, capacity, count);
 }
 
 simjoin_status simjoin_run_hamming_lsh(simjoin_ctx *ctx, const void *P_bits, int64_t n, const void *Q_bits, int64_t m, int32_t d,
@@ -800,7 +856,7 @@ simjoin_status simjoin_run_hamming_lsh(simjoin_ctx *ctx, const void *P_bits, int
     st = hamming_unpack(ctx, P_bits, n, Q_bits, m, d, out_pairs, capacity, count);
     if (st != SIMJOIN_OK || n == 0 || m == 0) return st;
     const double t = (double)d - 2.0 * std::floor(r);
-    return lsh_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, t, L, L_low, k, seed, out_pairs, capacity, count);
+    return lsh_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, SIMJOIN_IP, t, L, L_low, k, seed, out_pairs, capacity, count);
 }
 
 simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, int32_t d, int32_t k, uint64_t seed, void *out) {

@@ -127,8 +127,7 @@ def test_lsh_offsets_capacity_and_errors(ctx):
     assert ctx.simjoin_run_lsh(*args, 2, 0, 1, out, 8, L_low=1)[0] == B.SIMJOIN_ERR_ARG          # k - 1 bits needs k >= 1
     assert ctx.simjoin_run_lsh(*args, 60, 3, 1, out, 8, L_low=5)[0] == B.SIMJOIN_ERR_ARG
     assert ctx.simjoin_run_lsh(dP, 0, dQ, 2000, 128, 100.0, 2, 3, 1, out, 8) == (B.SIMJOIN_OK, 0)
-    with B.Simjoin("bf16", 0) as cb:
-        assert cb.simjoin_run_lsh(*args, 2, 3, 1, out, 8)[0] == B.SIMJOIN_ERR_UNSUPPORTED
+    assert ctx.simjoin_run_lsh(*args, 2, 3, 1, out, 8, kind="cos")[0] == B.SIMJOIN_ERR_UNSUPPORTED     # int8 x cosine, as simjoin_run
     # the plain join still works on the same context afterwards
     got, cnt = ctx.join(dP, dQ, "ip", w.threshold, 1 << 16)
     assert cnt == O.join(w.P, w.Q, "ip", w.threshold, "i8")[1]
@@ -151,3 +150,51 @@ def test_lsh_hamming_join_on_packed_bits(ctx, n, m, d, L, k):
     assert ctx.simjoin_run_hamming_lsh(dP, n, dQ, m, d, -1.0, L, k, 1, out, 8)[0] == B.SIMJOIN_ERR_ARG
     assert ctx.simjoin_run_hamming_lsh(dP, n, dQ, m, d, 3.0, 0, k, 1, out, 8)[0] == B.SIMJOIN_ERR_ARG
     assert ctx.simjoin_run_hamming_lsh(dP, n, dQ, m, d + 64, 3.0, L, k, 1, out, 8)[0] == B.SIMJOIN_ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------ every kind and element type
+@pytest.fixture(scope="module")
+def ctx_bf16():
+    build.build()
+    c = B.Simjoin("bf16", 0)
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("d,L,k", [(128, 4, 3), (64, 3, 2), (256, 3, 4), (528, 2, 2)])
+def test_lsh_int8_euclidean_join(ctx, d, L, k):
+    """int8 rows, L2 kind: row norms and per-tile bounds are taken on the regrouped rows; exact pair set."""
+    P = W.random_points("i8", 1500 + 9, d, 61, lo=-2, hi=2)
+    Q = W.random_points("i8", 1900 + 5, d, 62, lo=-2, hi=2)
+    Q[7:600:3] = P[:198]
+    Q[8:600:3] = np.clip(P[200:398].astype(np.int16) + W.random_points("i8", 198, d, 63, lo=0, hi=1), -128, 127).astype(np.int8)
+    for r in (0.0, (0.3 * d) ** 0.5, (2.2 * d) ** 0.5):
+        dP, dQ = torch.from_numpy(P).cuda(), torch.from_numpy(Q).cuda()
+        out = torch.full((1 << 21, 2), -5, dtype=torch.int32, device="cuda:0")
+        st, cnt = ctx.simjoin_run_lsh(dP, len(P), dQ, len(Q), d, r, L, k, 19, out, 1 << 21, L_low=1, kind="l2")
+        assert st == B.SIMJOIN_OK, B.strerror(st)
+        want, wcnt = O.lsh_join_kind(P, Q, "l2", r, "i8", L, k, 19, L_low=1)
+        got = keys(out[:cnt].cpu().numpy())
+        assert cnt == wcnt and len(np.unique(got)) == cnt and np.array_equal(got, keys(want)), (d, r, cnt, wcnt)
+        assert cnt >= 100
+
+
+@pytest.mark.parametrize("kind", ["ip", "cos", "l2"])
+@pytest.mark.parametrize("d,L,k", [(128, 4, 3), (64, 3, 5), (264, 3, 2)])
+def test_lsh_bf16_sign_hash_join(ctx_bf16, kind, d, L, k):
+    """bf16 rows, the sign of a sampled coordinate as the hash: within the threshold band of the oracle's sets
+    restricted to colliding pairs; nothing twice."""
+    w = W.make_workload(2, n=1800 + 11, m=2100 + 3, d=d, planted=300)
+    t = {"ip": 0.85, "cos": 0.85, "l2": 0.55}[kind]
+    dP, dQ = B.to_device(w.P), B.to_device(w.Q)
+    out = torch.full((1 << 20, 2), -5, dtype=torch.int32, device="cuda:0")
+    st, cnt = ctx_bf16.simjoin_run_lsh(dP, w.n, dQ, w.m, d, t, L, k, 23, out, 1 << 20, L_low=1, kind=kind)
+    assert st == B.SIMJOIN_OK, B.strerror(st)
+    got = keys(out[:cnt].cpu().numpy())
+    assert len(np.unique(got)) == cnt
+    strict, exact, loose = O.lsh_band_sets(w.P, w.Q, kind, t, "bf16", L, k, 23, L_low=1)
+    assert np.isin(keys(strict), got).all() and np.isin(got, keys(loose)).all(), (kind, d, cnt, len(strict), len(loose))
+    assert len(strict) >= 50                                            # planted pairs that collide
+    # recall against the brute-force join: a planted pair at angle theta survives a k-bit table with (1 - theta/pi)^k
+    full = O.join(w.P, w.Q, kind, t, "bf16")[0]
+    assert len(exact) <= len(full) and len(exact) > 0.3 * len(full)
