@@ -1,0 +1,81 @@
+"""Randomised parity: a few hundred seeded cases over element type, kind, brute force / LSH, row length (all three tile
+geometries, partial chunks), ragged row counts and value ranges, each compared with the oracle (int8: the exact pair set;
+bf16: inside the threshold band).  Thresholds are taken from a sample of the oracle's scores so that every case has
+hits.  One ill-conditioned corner is left out on purpose: a bf16 Euclidean radius far below the rows' norms, where
+|x|^2 + |y|^2 - 2<x,y> cancels in fp32 beyond what a band relative to r can absorb."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import simjoin_oracle as O
+from paper_2006_12608_b200 import binding as B
+from paper_2006_12608_b200 import build
+from paper_2006_12608_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+ROW_BYTES = [16, 32, 48, 64, 96, 128, 144, 256, 272, 384, 400, 512, 528, 640, 1024, 1040, 2048, 2064, 4096]
+
+
+def keys(p):
+    p = np.asarray(p, dtype=np.int64).reshape(-1, 2)
+    return np.sort((p[:, 0] << 32) | p[:, 1])
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_cases_match_the_oracle(seed):
+    build.build()
+    rng = np.random.default_rng(seed)
+    ctxs = {"i8": B.Simjoin("i8", 0), "bf16": B.Simjoin("bf16", 0)}
+    cap = 1 << 21
+    out = torch.empty((cap + 2, 2), dtype=torch.int32, device="cuda:0")
+    try:
+        for case in range(130):
+            dtype = "i8" if rng.random() < 0.5 else "bf16"
+            kind = str(rng.choice(["ip", "l2"] if dtype == "i8" else ["ip", "cos", "l2"]))
+            d = int(rng.choice(ROW_BYTES)) // (1 if dtype == "i8" else 2)
+            n = int(rng.integers(1, 1200)) if rng.random() < 0.7 else int(rng.integers(1200, 40 * 256))
+            m = int(rng.integers(1, 3000))
+            if n * m * d > 2e9:
+                n = max(1, int(2e9 / (m * d)))
+            lsh = rng.random() < 0.35
+            s1, s2 = int(rng.integers(1 << 30)), int(rng.integers(1 << 30))
+            if dtype == "i8":
+                hi = int(rng.choice([1, 2, 5, 127]))
+                P, Q = W.random_points("i8", n, d, s1, lo=-hi, hi=hi), W.random_points("i8", m, d, s2, lo=-hi, hi=hi)
+            else:
+                P, Q = W.random_points("bf16", n, d, s1), W.random_points("bf16", m, d, s2)
+            kpl = min(n, m, 64)
+            Q[:kpl] = P[:kpl]                                   # equal rows: hits under every kind
+            smp = np.stack([rng.integers(0, n, 2000), rng.integers(0, m, 2000)], axis=1).astype(np.int32)
+            sc = O.scores(P, Q, kind, dtype, smp).astype(np.float64)
+            if kind == "l2":
+                dist = np.sqrt(np.maximum(sc, 0.0)) if dtype == "i8" else sc
+                t = float(np.quantile(dist, 0.002))
+                if dtype == "bf16":
+                    t = max(t, 0.6 * float(np.median(dist)))    # keep the radius well above the fp32 cancellation floor
+            else:
+                t = float(np.quantile(sc, 0.998))
+            ctx = ctxs[dtype]
+            dP, dQ = B.to_device(P), B.to_device(Q)
+            out.fill_(-5)
+            L = k = L_low = 0
+            if lsh:
+                L, k = int(rng.integers(1, 5)), int(rng.integers(0, 6))
+                L_low = int(rng.integers(0, 2)) if k >= 1 else 0
+                st, cnt = ctx.simjoin_run_lsh(dP, n, dQ, m, d, t, L, k, s1, out, cap, L_low=L_low, kind=kind)
+            else:
+                st, cnt = ctx.simjoin_run(dP, n, dQ, m, d, kind, t, out, cap)
+            what = dict(case=case, dtype=dtype, kind=kind, n=n, m=m, d=d, t=t, lsh=(L, k, L_low) if lsh else None, s1=s1, s2=s2)
+            assert st == B.SIMJOIN_OK, (B.strerror(st), what)
+            host = out.cpu().numpy()
+            got = keys(host[:cnt])
+            assert np.all(host[cnt:] == -5) and len(np.unique(got)) == cnt, what
+            if dtype == "i8":
+                want = O.lsh_join_kind(P, Q, kind, t, dtype, L, k, s1, L_low=L_low)[0] if lsh else O.join(P, Q, kind, t, dtype)[0]
+                assert np.array_equal(got, keys(want)), what
+            else:
+                sets = O.lsh_band_sets(P, Q, kind, t, dtype, L, k, s1, L_low=L_low) if lsh else O.band_sets(P, Q, kind, t, dtype)
+                assert np.isin(keys(sets[0]), got).all() and np.isin(got, keys(sets[2])).all(), what
+    finally:
+        for c in ctxs.values():
+            c.close()
