@@ -68,8 +68,10 @@ constexpr int NUM_THREADS = 32 * (EPI_WARP0 + NUM_EPI_WARPS);
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 constexpr int CTRL_BYTES = 256;
-constexpr int STAGE_PAIRS = 2048 / NUM_EPI_WARPS;                // per epilogue warp: pairs staged in shared memory
-constexpr int STAGING_BYTES = NUM_EPI_WARPS * STAGE_PAIRS * 8;  // 16 KiB
+constexpr int WARP_STAGE_BYTES = 2048;                           // per epilogue warp: staged pairs, then the column terms
+constexpr int COLTERM_BYTES = EPI_COLS * 4;                      // per-column terms of the 128 columns under test
+constexpr int STAGE_PAIRS = (WARP_STAGE_BYTES - COLTERM_BYTES) / 8;   // pairs staged in shared memory per warp
+constexpr int STAGING_BYTES = NUM_EPI_WARPS * WARP_STAGE_BYTES;  // 16 KiB
 
 struct JoinParams {
     long long n, m;          // rows of P, Q
@@ -338,14 +340,22 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     int cnt = 0;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) cnt += __popc(mask[q]);
-    int incl = cnt;
+    // prefix sum over the lanes.  Usual case, at most one hit per row: two votes instead of a chain of shuffles
+    int incl, total;
+    const uint32_t one = __ballot_sync(0xffffffffu, cnt != 0);
+    if (one == 0) return;
+    if (__ballot_sync(0xffffffffu, cnt > 1) == 0) {
+        incl = __popc(one & (0xffffffffu >> (31 - lane)));
+        total = __popc(one);
+    } else {
+        incl = cnt;
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += t;
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += t;
+        }
+        total = __shfl_sync(0xffffffffu, incl, 31);
     }
-    const int total = __shfl_sync(0xffffffffu, incl, 31);
-    if (total == 0) return;
     if (fill + total > STAGE_PAIRS) {
         flush_pairs<GROUPED>(p, buf, fill, lane);
         fill = 0;
@@ -729,7 +739,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         const int half = (warp - EPI_WARP0) >> 2;   // which of the tile's two P blocks (accumulator columns half * TILE_N ..)
         const int row_in_tile = half * TILE_M + quarter * 32 + lane;
         uint32_t acc = 0, accphase = 0, rstage = 0;   // rstage: next ring stage to hand back
-        int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * STAGE_PAIRS;
+        int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * (WARP_STAGE_BYTES / 8);
+        uint32_t *colterm = reinterpret_cast<uint32_t *>(stage_buf + STAGE_PAIRS);
         int stage_fill = 0;
         bool ok = true;
         Unit un;
@@ -741,7 +752,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             const long long q_base = GROUPED ? un.qrow0 : 0;                          // Q row of tile 0
             const long long q_end = GROUPED ? (long long)un.qrow0 + un.qrows : p.m;   // end of the Q rows of this unit
             int ri = 0;          // I8/L2: |x|^2 - floor(r^2)
-            float rf = 0.f;      // COS: t*|x|;  BF16/L2: |x|^2
+            float rf = 0.f;      // COS: t*|x|;  BF16/L2: (|x|^2 - r^2) / 2
             bool rzero = false;  // COS: x is the zero vector
             if (row_ok) {
                 if constexpr (DT == DT_I8 && KIND == KIND_L2) ri = reinterpret_cast<const int *>(p.nx)[i] - p.thr_i;
@@ -750,7 +761,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     rf = p.thr_f * nxr;
                     rzero = nxr == 0.f;
                 }
-                if constexpr (DT == DT_BF16 && KIND == KIND_L2) rf = reinterpret_cast<const float *>(p.nx)[i];
+                // BF16/L2 decides |x|^2 + |y|^2 - 2s <= r^2 as  s >= (|x|^2 - r^2)/2 + |y|^2/2:  one add per element
+                if constexpr (DT == DT_BF16 && KIND == KIND_L2) rf = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] - p.thr_f);
             }
             for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
                 const int qt = tile_at<ALIGNED>(un, k);
@@ -776,7 +788,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 }
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
                     const float2 s0 = reinterpret_cast<const float2 *>(p.qstat)[qb0], s1 = reinterpret_cast<const float2 *>(p.qstat)[qb1];
-                    ff = rf + fminf(s0.x, s1.x);                  // (|x|^2 + min|y|^2) - 2s <= r^2
+                    ff = rf + 0.5f * fminf(s0.x, s1.x);           // s >= (|x|^2 - r^2)/2 + min|y|^2/2
                 }
                 // per-column terms of this warp's columns, 4 per lane, fetched while the tile is still
                 // being multiplied so that the exact test never waits on global memory
@@ -838,7 +850,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 // this warp's 128 columns of the tile (long rows: two passes of 128 over its block's 256), then hand
                 // the accumulator back to the MMA warp
                 constexpr int NV = NARROW ? EPI_COLS / 2 : EPI_COLS;      // accumulator words per thread
-                constexpr int GCOLS = 16, NG = EPI_COLS / GCOLS, GW = NV / NG;  // groups of 16 columns
+                constexpr int GCOLS = 16, NG = EPI_COLS / GCOLS, GW = NV / NG;  // column groups of level 1
+                constexpr uint32_t GMASK = (1u << GCOLS) - 1u;
                 constexpr int MODE = DT == DT_BF16 ? MAX_F32 : (NARROW ? MAX_S16X2 : MAX_S32);
 #pragma unroll
                 for (int ps = 0; ps < NPASS; ++ps) {
@@ -855,41 +868,78 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     if constexpr (DT == DT_I8) {
                         const int mx = NARROW ? max((int)(short)(word & 0xffffu), (int)word >> 16) : (int)word;
                         return mx >= fi;
-                    } else if constexpr (KIND == KIND_L2) {
-                        return (ff - 2.f * __uint_as_float(word)) <= p.thr_f;
                     } else {
                         return __uint_as_float(word) >= ff;
                     }
                 };
-                bool hit = row_ok && bound_ok(TreeMax<NV, MODE>::run(v));
+                // bf16: taken over the maxima of the 16-column groups, which level 1 then has for free (dense
+                // outputs: -6 %); int8 keeps one flat tree, measured 5 % faster on the sparse headline join
+                constexpr bool GROUP_FIRST = DT == DT_BF16;
+                uint32_t gmax[NG];
+                bool hit;
+                if constexpr (GROUP_FIRST) {
+#pragma unroll
+                    for (int k = 0; k < NG; ++k) gmax[k] = TreeMax<GW, MODE>::run(v + k * GW);
+                    hit = row_ok && bound_ok(TreeMax<NG, MODE>::run(gmax));
+                } else {
+                    hit = row_ok && bound_ok(TreeMax<NV, MODE>::run(v));
+                }
                 if (__builtin_expect(__any_sync(0xffffffffu, hit) != 0, 0)) {   // rare for sparse joins: keep it out of line
                     // level 1: which 16-column groups can hold a hit for this row
                     uint32_t gm = 0;
 #pragma unroll
-                    for (int k = 0; k < NG; ++k) gm |= (bound_ok(TreeMax<GW, MODE>::run(v + k * GW)) ? 1u : 0u) << k;
+                    for (int k = 0; k < NG; ++k) {
+                        if constexpr (!GROUP_FIRST) gmax[k] = TreeMax<GW, MODE>::run(v + k * GW);
+                        gm |= (bound_ok(gmax[k]) ? 1u : 0u) << k;
+                    }
                     if (!row_ok) gm = 0;
                     const long long j0 = q_base + (long long)qt * TN + ps * EPI_COLS;
                     uint32_t mask[EPI_COLS / 32];
 #pragma unroll
                     for (int q = 0; q < EPI_COLS / 32; ++q) mask[q] = 0;
+                    if constexpr (KIND != KIND_IP) {
+                        // the per-column terms go through shared memory: level 2 reads 16 of them per group as four
+                        // broadcast loads (a shuffle per term cost four times the instructions)
+                        __syncwarp();
+                        reinterpret_cast<uint4 *>(colterm)[lane] = yq;
+                        __syncwarp();
+                    }
 #pragma unroll
                     for (int k = 0; k < NG; ++k) {
                         if (!__any_sync(0xffffffffu, (gm >> k) & 1u)) continue;
                         // level 2: the exact test on the 16 columns of group k
-                        const long long jg = j0 + k * GCOLS;
-                        const long long left = q_end - jg;                     // columns of this group inside Q (the bucket)
-                        const uint32_t valid = left >= GCOLS ? 0xffffu : (left <= 0 ? 0u : ((1u << (int)left) - 1u));
                         uint32_t yw[GCOLS];                                     // per-column term of Q (norm kinds)
                         if constexpr (KIND != KIND_IP) {
 #pragma unroll
-                            for (int t = 0; t < GCOLS / 4; ++t) {              // column k*16 + 4t + e lives in lane k*4 + t
-                                yw[4 * t] = __shfl_sync(0xffffffffu, yq.x, k * (GCOLS / 4) + t);
-                                yw[4 * t + 1] = __shfl_sync(0xffffffffu, yq.y, k * (GCOLS / 4) + t);
-                                yw[4 * t + 2] = __shfl_sync(0xffffffffu, yq.z, k * (GCOLS / 4) + t);
-                                yw[4 * t + 3] = __shfl_sync(0xffffffffu, yq.w, k * (GCOLS / 4) + t);
+                            for (int t = 0; t < GCOLS / 4; ++t) {
+                                const uint4 q4 = reinterpret_cast<const uint4 *>(colterm)[k * (GCOLS / 4) + t];
+                                yw[4 * t] = q4.x;
+                                yw[4 * t + 1] = q4.y;
+                                yw[4 * t + 2] = q4.z;
+                                yw[4 * t + 3] = q4.w;
                             }
                         }
                         uint32_t mk = 0;
+                        if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
+                            // The same decision as bound_ok, taken from a sign bit: fl(s - b) >= +0 exactly when
+                            // s >= b.  The adds run on the FMA pipe and one funnel shift collects the bit, where a
+                            // compare, a select and an OR would all queue on the half-rate ALU pipe (dense outputs).
+                            // Four independent chains of four columns.
+                            constexpr int NCH = GCOLS / 4;
+                            uint32_t fail[NCH];
+#pragma unroll
+                            for (int q = 0; q < NCH; ++q) fail[q] = 0;
+#pragma unroll
+                            for (int c = 0; c < GCOLS; ++c) {
+                                const float b = rf + 0.5f * __uint_as_float(yw[c]);
+                                fail[c >> 2] = __funnelshift_l(__float_as_uint(__uint_as_float(v[k * GCOLS + c]) - b), fail[c >> 2], 1);
+                            }
+                            // chain q holds columns 4q .. 4q+3 at bits 3 .. 0
+                            uint32_t fall = 0;                                  // column c -> bit GCOLS - 1 - c
+#pragma unroll
+                            for (int q = 0; q < NCH; ++q) fall |= fail[q] << (4 * (NCH - 1 - q));
+                            mk = (__brev(~fall) >> (32 - GCOLS)) & GMASK;
+                        } else {
 #pragma unroll
                         for (int c = 0; c < GCOLS; ++c) {
                             uint32_t x;
@@ -907,13 +957,20 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                                 const float nyr = __uint_as_float(yw[c]);
                                 pass = (rzero || nyr == 0.f) ? (p.thr_f <= 0.f) : (__uint_as_float(x) >= rf * nyr);
                             }
-                            if constexpr (DT == DT_BF16 && KIND == KIND_L2)
-                                pass = ((rf + __uint_as_float(yw[c])) - 2.f * __uint_as_float(x)) <= p.thr_f;
                             mk |= (pass ? 1u : 0u) << c;
                         }
-                        mk &= valid;
+                        }
                         if (!((gm >> k) & 1u)) mk = 0;       // the group bound is necessary: nothing can pass here
-                        mask[k >> 1] |= mk << ((k & 1) * 16);
+                        mask[(k * GCOLS) >> 5] |= mk << ((k * GCOLS) & 31);
+                    }
+                    // columns past the end of Q (of the bucket) were multiplied as zero rows: drop them
+                    const long long left = q_end - j0;
+                    if (left < EPI_COLS) {
+#pragma unroll
+                        for (int q = 0; q < EPI_COLS / 32; ++q) {
+                            const long long lq = left - 32 * q;
+                            mask[q] &= lq >= 32 ? 0xffffffffu : (lq <= 0 ? 0u : ((1u << (int)lq) - 1u));
+                        }
                     }
                     emit_pairs<EPI_COLS / 32, GROUPED>(p, mask, lane, i, j0, stage_buf, stage_fill);
                 }
