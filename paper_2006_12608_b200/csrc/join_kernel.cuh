@@ -920,7 +920,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             }
                         }
                         uint32_t mk = 0;
-                        if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
+                        if constexpr (DT == DT_BF16 && (KIND == KIND_L2 || KIND == KIND_IP)) {
                             // The same decision as bound_ok, taken from a sign bit: fl(s - b) >= +0 exactly when
                             // s >= b.  The adds run on the FMA pipe and one funnel shift collects the bit, where a
                             // compare, a select and an OR would all queue on the half-rate ALU pipe (dense outputs).
@@ -931,7 +931,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             for (int q = 0; q < NCH; ++q) fail[q] = 0;
 #pragma unroll
                             for (int c = 0; c < GCOLS; ++c) {
-                                const float b = rf + 0.5f * __uint_as_float(yw[c]);
+                                const float b = KIND == KIND_IP ? p.thr_f : rf + 0.5f * __uint_as_float(yw[c]);
                                 fail[c >> 2] = __funnelshift_l(__float_as_uint(__uint_as_float(v[k * GCOLS + c]) - b), fail[c >> 2], 1);
                             }
                             // chain q holds columns 4q .. 4q+3 at bits 3 .. 0

@@ -262,6 +262,8 @@ void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold
         }
     } else {
         jp.thr_f = kind == SIMJOIN_L2 ? (float)(threshold * threshold) : (float)threshold;
+        // the inner-product test reads the sign of s - t: with t = -0 a score of either zero gives +0 and passes
+        if (kind == SIMJOIN_IP && jp.thr_f == 0.f) jp.thr_f = -0.0f;
     }
 }
 

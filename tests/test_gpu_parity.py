@@ -139,6 +139,19 @@ def test_bf16_negative_threshold_and_zero_rows(ctx_bf16):
     assert_band(pairs, cnt, P, Q, "ip", -1.0)
 
 
+def test_bf16_inner_product_threshold_zero_counts_scores_of_either_zero(ctx_bf16):
+    """t = 0: a pair whose score is exactly zero passes, whichever zero the accumulator holds (a zero row against a row
+    of negative values sums products that are all -0)."""
+    P = W.f32_to_bf16_bits(np.zeros((40, 64), dtype=np.float32))
+    Q = W.f32_to_bf16_bits(-np.abs(np.random.default_rng(4).standard_normal((70, 64))).astype(np.float32) - 0.5)
+    P[1::2] = W.f32_to_bf16_bits(np.ones((20, 64), dtype=np.float32))          # odd rows: score < 0 against every Q row
+    for t in (0.0, -0.0):
+        pairs, cnt = gpu_join(ctx_bf16, P, Q, "ip", t)
+        want, wcnt = O.join(P, Q, "ip", t, "bf16")
+        assert cnt == wcnt == 20 * 70
+        assert set(map(tuple, pairs.tolist())) == set(map(tuple, want.tolist()))
+
+
 def test_i8_packed_16_bit_epilogue_boundary(ctx_i8):
     """int8 scores that provably fit in 16 bits take a packed epilogue; check both sides of that
     decision and scores at the very ends of the 16-bit range."""
