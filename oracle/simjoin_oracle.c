@@ -22,7 +22,12 @@
  *   - int8 inputs: exact integer arithmetic.  Inner product: pass iff
  *     s >= t over the reals (s is an integer below 2^53, so the double compare
  *     is exact).  Euclidean: pass iff the integer squared distance D satisfies
- *     (double)D <= r*r, r*r being the double product.
+ *     (double)D <= r*r, r*r being the double product.  Cosine: the three sums
+ *     <x,y>, |x|^2, |y|^2 are exact integers; the score is the fp64 quotient
+ *     <x,y> / (sqrt(|x|^2) * sqrt(|y|^2)) with each operation rounded once
+ *     (IEEE sqrt, product, quotient -- no fused operation), 0 for a zero
+ *     vector; pass iff score >= t.  The score is a floating-point number that
+ *     decides an integer result, so this exact sequence is part of the reading.
  *   - bf16 inputs: the 16-bit patterns are the inputs; each is widened exactly
  *     to fp64 and all sums run in fp64 with k ascending.
  *     cosine of a zero vector is defined as 0.
@@ -63,6 +68,14 @@ int64_t oracle_sqdist_i8(const int8_t *x, const int8_t *y, int32_t d) {
         s += e * e;
     }
     return s;
+}
+
+/* Cosine of two int8 rows: exact integer sums, then sqrt, product and quotient in fp64, each rounded once. */
+double oracle_cos_i8(const int8_t *x, const int8_t *y, int32_t d) {
+    int64_t s = oracle_ip_i8(x, y, d), nx = oracle_ip_i8(x, x, d), ny = oracle_ip_i8(y, y, d);
+    if (nx == 0 || ny == 0) return 0.0;
+    volatile double den = sqrt((double)nx) * sqrt((double)ny);   /* volatile: one rounding here, whatever the flags */
+    return (double)s / den;
 }
 
 /* The value a bfloat16 bit pattern denotes, as fp64 (exact). */
@@ -121,8 +134,8 @@ double oracle_score_bf16(const uint16_t *P, int64_t i, const uint16_t *Q, int64_
 }
 
 /* Scores of a list of pairs: out[p] = score(P[pairs[2p]], Q[pairs[2p+1]]).
- * int8: inner product (KIND_IP) or squared distance (KIND_L2) as int64 in out_i;
- * bf16: fp64 score in out_f. */
+ * int8: inner product (KIND_IP) or squared distance (KIND_L2) as int64 in out_i, cosine as fp64
+ * (oracle_scores_cos_i8); bf16: fp64 score in out_f. */
 int32_t oracle_scores_i8(const int8_t *P, const int8_t *Q, int32_t d, int32_t kind,
                          const int32_t *pairs, int64_t npairs, int64_t *out_i) {
     if (kind != KIND_IP && kind != KIND_L2) return -1;
@@ -130,6 +143,12 @@ int32_t oracle_scores_i8(const int8_t *P, const int8_t *Q, int32_t d, int32_t ki
         const int8_t *x = P + (size_t)pairs[2 * p] * d, *y = Q + (size_t)pairs[2 * p + 1] * d;
         out_i[p] = kind == KIND_IP ? oracle_ip_i8(x, y, d) : oracle_sqdist_i8(x, y, d);
     }
+    return 0;
+}
+
+int32_t oracle_scores_cos_i8(const int8_t *P, const int8_t *Q, int32_t d, const int32_t *pairs, int64_t npairs, double *out_f) {
+    for (int64_t p = 0; p < npairs; ++p)
+        out_f[p] = oracle_cos_i8(P + (size_t)pairs[2 * p] * d, Q + (size_t)pairs[2 * p + 1] * d, d);
     return 0;
 }
 
@@ -180,6 +199,7 @@ static void pb_push(pairbuf *b, int64_t i, int64_t j) {
 
 static int pass_i8(const int8_t *x, const int8_t *y, int32_t d, int kind, double thr) {
     if (kind == KIND_IP) return (double)oracle_ip_i8(x, y, d) >= thr;
+    if (kind == KIND_COS) return oracle_cos_i8(x, y, d) >= thr;
     return (double)oracle_sqdist_i8(x, y, d) <= thr * thr;
 }
 
@@ -223,7 +243,7 @@ int32_t oracle_max_threads(void) { return resolve_threads(0); }
 
 int64_t oracle_join_i8(const int8_t *P, int64_t n, const int8_t *Q, int64_t m, int32_t d, int32_t kind,
                        double threshold, int32_t *out_pairs, int64_t capacity, int32_t nthreads) {
-    if (n < 0 || m < 0 || d <= 0 || capacity < 0 || (kind != KIND_IP && kind != KIND_L2)) return -1;
+    if (n < 0 || m < 0 || d <= 0 || capacity < 0 || kind < KIND_IP || kind > KIND_L2) return -1;
     if (isnan(threshold) || (kind == KIND_L2 && threshold < 0)) return -1;
     if (n >= INT32_MAX || m >= INT32_MAX) return -1;
     int nt = resolve_threads(nthreads);

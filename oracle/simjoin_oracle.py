@@ -88,6 +88,8 @@ def _load():
     lib.oracle_jl_transform_bf16.argtypes = [vp, i64, i32, i32, c.c_uint64, vp]
     lib.oracle_scores_i8.restype = i32
     lib.oracle_scores_i8.argtypes = [vp, vp, i32, i32, vp, i64, vp]
+    lib.oracle_scores_cos_i8.restype = i32
+    lib.oracle_scores_cos_i8.argtypes = [vp, vp, i32, vp, i64, vp]
     lib.oracle_scores_bf16.restype = i32
     lib.oracle_scores_bf16.argtypes = [vp, vp, i32, i32, vp, i64, vp]
     lib.oracle_sq_norms_bf16.restype = None
@@ -282,7 +284,7 @@ def band_sets(P, Q, kind, threshold, dtype, rel: float = 1e-2, threads: int = 0)
 
 
 def scores(P, Q, kind: str, dtype: str, pairs: np.ndarray) -> np.ndarray:
-    """Score of each listed (i, j): int64 inner product / squared distance for
+    """Score of each listed (i, j): int64 inner product / squared distance and fp64 cosine for
     int8 rows, fp64 inner product / cosine / distance for bf16 rows."""
     lib = _load()
     P = _check(P, dtype)
@@ -291,7 +293,10 @@ def scores(P, Q, kind: str, dtype: str, pairs: np.ndarray) -> np.ndarray:
     d = P.shape[1]
     if len(pairs) and (pairs[:, 0].max() >= P.shape[0] or pairs[:, 1].max() >= Q.shape[0] or pairs.min() < 0):
         raise IndexError("pair index out of range")
-    if dtype == "i8":
+    if dtype == "i8" and kind == "cos":
+        out = np.empty(len(pairs), dtype=np.float64)
+        rc = lib.oracle_scores_cos_i8(P.ctypes.data, Q.ctypes.data, d, pairs.ctypes.data, len(pairs), out.ctypes.data)
+    elif dtype == "i8":
         out = np.empty(len(pairs), dtype=np.int64)
         rc = lib.oracle_scores_i8(P.ctypes.data, Q.ctypes.data, d, KIND[kind], pairs.ctypes.data, len(pairs), out.ctypes.data)
     else:

@@ -488,8 +488,7 @@ def test_empty_and_rejected_inputs():
         O.join(Q, Q, "l2", -1.0, "i8")
     with pytest.raises(ValueError):
         O.join(Q, Q, "ip", float("nan"), "i8")
-    with pytest.raises(ValueError):
-        O.join(Q, Q, "cos", 0.5, "i8")
+    assert O.join(Q, Q, "cos", 0.5, "i8")[1] == 16              # equal rows: cosine 1
 
 
 def test_planted_scores_match_the_recipes():
@@ -503,3 +502,66 @@ def test_planted_scores_match_the_recipes():
     w2 = W.make_workload(2, n=3000, m=2000, planted=100)
     c2 = O.scores(w2.P, w2.Q, "cos", "bf16", w2.planted)
     assert c2.min() > 0.93 and abs(c2.mean() - 1 / math.sqrt(1.09)) < 5e-3
+
+
+# ------------------------------------------------------------------ int8 cosine
+def _cos_passes_exactly(s: int, nx: int, ny: int, t: Fraction) -> bool:
+    """s / sqrt(nx * ny) >= t over the reals, decided in integers and rationals (0 for a zero vector)."""
+    if nx == 0 or ny == 0:
+        return 0 >= t
+    if s >= 0 and t < 0:
+        return True
+    if s < 0 and t >= 0:
+        return False
+    lhs, rhs = Fraction(s * s), t * t * nx * ny
+    return lhs >= rhs if s >= 0 else lhs <= rhs
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_int8_cosine_against_exact_rational_decisions(seed):
+    rng = np.random.default_rng(seed)
+    P = rng.integers(-127, 128, size=(23, 24)).astype(np.int8)
+    Q = rng.integers(-127, 128, size=(31, 24)).astype(np.int8)
+    P[5] = 0
+    Q[7] = 0
+    Q[9] = P[3]                                           # cosine exactly 1
+    Q[10] = -P[4]                                         # cosine exactly -1 (no -128 in range)
+    allp = np.array(list(itertools.product(range(len(P)), range(len(Q)))), dtype=np.int32)
+    sc = O.scores(P, Q, "cos", "i8", allp)
+    assert sc[3 * len(Q) + 9] == 1.0 and sc[4 * len(Q) + 10] == -1.0 and np.all(sc[5 * len(Q):6 * len(Q)] == 0.0)
+    Pi, Qi = P.astype(np.int64), Q.astype(np.int64)
+    for t in (0.3, 0.05, 0.0, -0.2, 1.0, -1.0, float(np.sort(sc)[-20]) + 1e-7):
+        if t not in (0.0, 1.0, -1.0):
+            assert np.abs(sc - t).min() > 1e-9             # away from every score: the fp64 rounding cannot matter
+        tq = Fraction(t)
+        want = {(i, j) for i in range(len(P)) for j in range(len(Q))
+                if _cos_passes_exactly(int(Pi[i] @ Qi[j]), int(Pi[i] @ Pi[i]), int(Qi[j] @ Qi[j]), tq)}
+        got, cnt = O.join(P, Q, "cos", t, "i8")
+        assert cnt == len(want) and as_set(got) == want, t
+
+
+def test_int8_cosine_equals_the_bf16_cosine_of_the_same_integers():
+    rng = np.random.default_rng(11)
+    P = rng.integers(-127, 128, size=(40, 32)).astype(np.int8)
+    Q = rng.integers(-127, 128, size=(50, 32)).astype(np.int8)
+    Pb, Qb = to_arr(P, "bf16"), to_arr(Q, "bf16")           # integers up to 127 are exact in bfloat16
+    allp = np.array(list(itertools.product(range(len(P)), range(len(Q)))), dtype=np.int32)
+    assert np.array_equal(O.scores(P, Q, "cos", "i8", allp), O.scores(Pb, Qb, "cos", "bf16", allp))
+    for t in (0.25, 0.0, -0.3):
+        a, ca = O.join(P, Q, "cos", t, "i8")
+        b, cb = O.join(Pb, Qb, "cos", t, "bf16")
+        assert ca == cb > 0 and np.array_equal(a, b)
+
+
+def test_int8_cosine_is_scale_invariant():
+    rng = np.random.default_rng(12)
+    P = rng.integers(-42, 43, size=(30, 16)).astype(np.int8)
+    Q = rng.integers(-63, 64, size=(35, 16)).astype(np.int8)
+    allp = np.array(list(itertools.product(range(len(P)), range(len(Q)))), dtype=np.int32)
+    sc = O.scores(P, Q, "cos", "i8", allp)
+    t = 0.2
+    assert np.abs(sc - t).min() > 1e-9
+    base, _ = O.join(P, Q, "cos", t, "i8")
+    assert len(base) > 0
+    assert np.array_equal(O.join((3 * P).astype(np.int8), (2 * Q).astype(np.int8), "cos", t, "i8")[0], base)
+    assert np.array_equal(O.join(Q, P, "cos", t, "i8")[0], np.array(sorted((j, i) for i, j in base.tolist()), dtype=np.int32))
