@@ -23,11 +23,12 @@
  *     s >= t over the reals (s is an integer below 2^53, so the double compare
  *     is exact).  Euclidean: pass iff the integer squared distance D satisfies
  *     (double)D <= r*r, r*r being the double product.  Cosine: the three sums
- *     <x,y>, |x|^2, |y|^2 are exact integers; the score is the fp64 quotient
- *     <x,y> / (sqrt(|x|^2) * sqrt(|y|^2)) with each operation rounded once
- *     (IEEE sqrt, product, quotient -- no fused operation), 0 for a zero
- *     vector; pass iff score >= t.  The score is a floating-point number that
- *     decides an integer result, so this exact sequence is part of the reading.
+ *     <x,y>, |x|^2, |y|^2 and the product |x|^2 |y|^2 are exact integers;
+ *     the score is the fp64 quotient <x,y> / sqrt(|x|^2 |y|^2) (conversion of
+ *     the product to double, IEEE sqrt, IEEE quotient: three roundings), 0 for
+ *     a zero vector; pass iff score >= t.  The score is a floating-point number
+ *     that decides an integer result, so this exact sequence is part of the
+ *     reading; with it parallel rows score exactly 1.
  *   - bf16 inputs: the 16-bit patterns are the inputs; each is widened exactly
  *     to fp64 and all sums run in fp64 with k ascending.
  *     cosine of a zero vector is defined as 0.
@@ -70,12 +71,13 @@ int64_t oracle_sqdist_i8(const int8_t *x, const int8_t *y, int32_t d) {
     return s;
 }
 
-/* Cosine of two int8 rows: exact integer sums, then sqrt, product and quotient in fp64, each rounded once. */
+/* Cosine of two int8 rows: <x,y>, |x|^2 and |y|^2 as exact integers, their product |x|^2 |y|^2 as an exact
+ * 64-bit integer (below 2^63 for rows of up to 2^17 coordinates), then three fp64 roundings: the integer to
+ * double, the square root, the quotient.  Parallel rows score exactly 1: the product is then a perfect square. */
 double oracle_cos_i8(const int8_t *x, const int8_t *y, int32_t d) {
     int64_t s = oracle_ip_i8(x, y, d), nx = oracle_ip_i8(x, x, d), ny = oracle_ip_i8(y, y, d);
     if (nx == 0 || ny == 0) return 0.0;
-    volatile double den = sqrt((double)nx) * sqrt((double)ny);   /* volatile: one rounding here, whatever the flags */
-    return (double)s / den;
+    return (double)s / sqrt((double)(nx * ny));
 }
 
 /* The value a bfloat16 bit pattern denotes, as fp64 (exact). */

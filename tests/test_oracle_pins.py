@@ -546,8 +546,10 @@ def test_int8_cosine_equals_the_bf16_cosine_of_the_same_integers():
     Q = rng.integers(-127, 128, size=(50, 32)).astype(np.int8)
     Pb, Qb = to_arr(P, "bf16"), to_arr(Q, "bf16")           # integers up to 127 are exact in bfloat16
     allp = np.array(list(itertools.product(range(len(P)), range(len(Q)))), dtype=np.int32)
-    assert np.array_equal(O.scores(P, Q, "cos", "i8", allp), O.scores(Pb, Qb, "cos", "bf16", allp))
+    si, sb = O.scores(P, Q, "cos", "i8", allp), O.scores(Pb, Qb, "cos", "bf16", allp)
+    np.testing.assert_allclose(si, sb, rtol=5e-16, atol=0)  # sqrt of the exact product vs product of two square roots
     for t in (0.25, 0.0, -0.3):
+        assert np.abs(si - t).min() > 1e-9
         a, ca = O.join(P, Q, "cos", t, "i8")
         b, cb = O.join(Pb, Qb, "cos", t, "bf16")
         assert ca == cb > 0 and np.array_equal(a, b)
@@ -565,3 +567,18 @@ def test_int8_cosine_is_scale_invariant():
     assert len(base) > 0
     assert np.array_equal(O.join((3 * P).astype(np.int8), (2 * Q).astype(np.int8), "cos", t, "i8")[0], base)
     assert np.array_equal(O.join(Q, P, "cos", t, "i8")[0], np.array(sorted((j, i) for i, j in base.tolist()), dtype=np.int32))
+
+
+def test_int8_cosine_of_parallel_rows_is_exactly_one_even_beyond_2_to_53():
+    rng = np.random.default_rng(13)
+    P = rng.integers(-63, 64, size=(6, 8192)).astype(np.int8)
+    P[0] = 63                                               # |x|^2 = 3.25e7, |x|^2 |2x|^2 = 4.2e15; rows 1..: ~1e7
+    P[1] = np.where(rng.random(8192) < 0.5, 63, -63)
+    Q = (2 * P).astype(np.int8)
+    Q[5] = -Q[5]
+    diag = np.array([[i, i] for i in range(6)], dtype=np.int32)
+    sc = O.scores(P, Q, "cos", "i8", diag)
+    assert np.array_equal(sc, [1, 1, 1, 1, 1, -1])
+    assert int(P[0].astype(np.int64) @ P[0]) * int(Q[0].astype(np.int64) @ Q[0]) > 2 ** 53
+    got, cnt = O.join(P, Q, "cos", 1.0, "i8")
+    assert got.tolist() == [[i, i] for i in range(5)]
