@@ -571,9 +571,9 @@ def test_int8_cosine_is_scale_invariant():
 
 def test_int8_cosine_of_parallel_rows_is_exactly_one_even_beyond_2_to_53():
     rng = np.random.default_rng(13)
-    P = rng.integers(-63, 64, size=(6, 8192)).astype(np.int8)
-    P[0] = 63                                               # |x|^2 = 3.25e7, |x|^2 |2x|^2 = 4.2e15; rows 1..: ~1e7
-    P[1] = np.where(rng.random(8192) < 0.5, 63, -63)
+    P = rng.integers(-63, 64, size=(6, 32768)).astype(np.int8)
+    P[0] = 63                                               # |x|^2 = 1.3e8, |x|^2 |2x|^2 = 6.8e16 > 2^53
+    P[1] = np.where(rng.random(32768) < 0.5, 63, -63)
     Q = (2 * P).astype(np.int8)
     Q[5] = -Q[5]
     diag = np.array([[i, i] for i in range(6)], dtype=np.int32)
