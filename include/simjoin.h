@@ -76,10 +76,14 @@ simjoin_status simjoin_create(simjoin_ctx **ctx, simjoin_dtype dtype, int device
  * The join (Section 4: join definition; brute-force product F_P * G_Q^T).
  *
  *   P, Q        device pointers, n x d and m x d, row-major, read-only.
- *   kind        see simjoin_kind.  Supported: I8 x {IP, L2}, BF16 x {IP, COS, L2}.
+ *   kind        see simjoin_kind.  Supported: {I8, BF16} x {IP, COS, L2}.
  *   threshold   t (IP, COS) or r (L2).  I8/IP passes when the integer score s
  *               satisfies s >= t over the reals; I8/L2 when the integer squared
- *               distance D satisfies D <= floor(r*r), r*r the double product.
+ *               distance D satisfies D <= floor(r*r), r*r the double product;
+ *               I8/COS when the fp64 quotient <x,y> / sqrt(|x|^2 |y|^2) is >= t
+ *               (exact integer sums and product; the conversion to double, the
+ *               square root and the quotient each rounded once; 0 for a zero
+ *               vector) -- int8 results are exact, with no tolerance band.
  *               BF16 kinds compare fp32 scores; pairs whose exact score lies
  *               within 1e-2*|threshold| of the threshold may fall on either side.
  *   out_pairs   device pointer to capacity x 2 int32, written as (i, j) rows.
@@ -97,7 +101,7 @@ simjoin_status simjoin_create(simjoin_ctx **ctx, simjoin_dtype dtype, int device
  * negative or >= 2^31, d <= 0, NaN threshold, L2 with threshold < 0, a host
  * pointer where a device pointer is required, out_pairs NULL with capacity > 0);
  * ERR_UNSUPPORTED (misaligned base pointer, d*sizeof(element) not a multiple
- * of 16 or above SIMJOIN_MAX_ROW_BYTES, I8 x COS).  After launch: ERR_CUDA,
+ * of 16 or above SIMJOIN_MAX_ROW_BYTES).  After launch: ERR_CUDA,
  * ERR_TIMEOUT (a wait in the kernel gave up; the context stays usable),
  * ERR_CAPACITY.
  */

@@ -86,7 +86,7 @@ struct JoinParams {
     int wave_gq;             // > 0: two-dimensional waves, (gridDim / wave_gq) P tiles x wave_gq Q tiles at a time (very long rows)
     int thr_i;               // I8/IP: ceil(t);  I8/L2: floor(r*r); both clamped
     float thr_f;             // BF16: t (IP, COS) or r*r (L2)
-    const void *nx;          // per-row term of P: int32 |x|^2 (I8/L2), fp32 |x| (COS) or |x|^2 (L2)
+    const void *nx;          // per-row term of P: int32 |x|^2 (I8/L2), fp32 |x| (COS, both element types) or |x|^2 (BF16/L2)
     const void *ny;          // same for Q
     const void *qstat;       // per 256 rows of Q (two tiles): (min, max) of ny over the valid rows
     int2 *out;               // capacity x (i, j)
@@ -102,6 +102,10 @@ struct JoinParams {
     const uint4 *rec_p, *rec_q;    // per regrouped position: the 16-bit hash keys of all repetitions, rec_words x 16 bytes
     int rec_words;
     int rep;                       // repetitions already joined: a pair whose keys agreed in one of them is not reported again
+    // I8/COS: candidates of the fp32 filter are decided exactly from the rows themselves when they leave the CTA
+    const void *rows_p, *rows_q;   // the row arrays the tensor maps cover
+    int row_bytes;
+    double thr_d;                  // t
     // KIND_STORE
     uint16_t *store_out;
     long long store_ld;
@@ -277,18 +281,53 @@ __device__ __forceinline__ bool already_reported(const JoinParams &p, long long 
     return seen;
 }
 
+// I8/COS: the exact decision for the pair of rows (li of P, lj of Q), from the rows themselves.  <x,y>, |x|^2,
+// |y|^2 are exact integers, the product |x|^2 |y|^2 an exact 64-bit integer; then three fp64 roundings -- the
+// integer to double, the square root, the quotient -- and the compare with t.  A zero vector scores 0.
+__device__ __forceinline__ bool cos_i8_passes(const JoinParams &p, long long li, long long lj) {
+    const int g = p.row_bytes >> 4;
+    const uint4 *x = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.rows_p) + li * p.row_bytes);
+    const uint4 *y = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.rows_q) + lj * p.row_bytes);
+    int s = 0, nx = 0, ny = 0;
+    for (int c = 0; c < g; ++c) {
+        const uint4 a = __ldg(x + c), b = __ldg(y + c);
+        s = __dp4a((int)a.x, (int)b.x, s);   nx = __dp4a((int)a.x, (int)a.x, nx);   ny = __dp4a((int)b.x, (int)b.x, ny);
+        s = __dp4a((int)a.y, (int)b.y, s);   nx = __dp4a((int)a.y, (int)a.y, nx);   ny = __dp4a((int)b.y, (int)b.y, ny);
+        s = __dp4a((int)a.z, (int)b.z, s);   nx = __dp4a((int)a.z, (int)a.z, nx);   ny = __dp4a((int)b.z, (int)b.z, ny);
+        s = __dp4a((int)a.w, (int)b.w, s);   nx = __dp4a((int)a.w, (int)a.w, nx);   ny = __dp4a((int)b.w, (int)b.w, ny);
+    }
+    if (nx == 0 || ny == 0) return 0.0 >= p.thr_d;
+    const double den = __dsqrt_rn(__ll2double_rn((long long)nx * (long long)ny));
+    return __ddiv_rn((double)s, den) >= p.thr_d;
+}
+
+// Is the staged pair dropped when it leaves the CTA?  Bucketed mode: reported by an earlier repetition.  VERIFY
+// (I8/COS): a candidate of the fp32 filter that fails the exact test.  Staged indices are regrouped positions in
+// bucketed mode, else row indices plus the caller's offsets.
+template <bool GROUPED, bool VERIFY>
+__device__ __forceinline__ bool drop_pair(const JoinParams &p, int i, int j) {
+    if constexpr (GROUPED) {
+        if (p.rep > 0 && already_reported(p, i, j)) return true;
+    }
+    if constexpr (VERIFY) {
+        if (!cos_i8_passes(p, GROUPED ? i : i - p.ioff, GROUPED ? j : j - p.joff)) return true;
+    }
+    return false;
+}
+
 template <bool GROUPED>
 __device__ __forceinline__ int2 final_pair(const JoinParams &p, int2 pr) {
     if constexpr (GROUPED) return make_int2(__ldg(p.perm_p + pr.x) + p.ioff, __ldg(p.perm_q + pr.y) + p.joff);
     return pr;
 }
-template <bool GROUPED>
+template <bool GROUPED, bool VERIFY = false>
 __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf, int fill, int lane) {
     if (fill == 0) return;
-    if constexpr (GROUPED) {
-        if (p.rep > 0) {
-            // Duplicates are dropped here, a whole buffer at a time (32 key-record lookups in flight per
-            // step), not when a hit is found: there the lookup's latency would stall the CTA's pipeline.
+    if constexpr (GROUPED || VERIFY) {
+        if (VERIFY || p.rep > 0) {
+            // Duplicates (and, for I8/COS, candidates that fail the exact test) are dropped here, a whole buffer
+            // at a time (32 lookups in flight per step), not when a hit is found: there the lookup's latency
+            // would stall the CTA's pipeline.
             int2 *wbuf = const_cast<int2 *>(buf);
             int kept = 0;
             for (int k0 = 0; k0 < fill; k0 += 32) {
@@ -296,7 +335,7 @@ __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf
                 bool keep = false;
                 if (k < fill) {
                     const int2 pr = wbuf[k];
-                    keep = !already_reported(p, pr.x, pr.y);
+                    keep = !drop_pair<GROUPED, VERIFY>(p, pr.x, pr.y);
                     if (!keep) wbuf[k].x = -1;
                 }
                 kept += __popc(__ballot_sync(0xffffffffu, keep));
@@ -334,7 +373,7 @@ __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf
 // prefix over the warp, then into the warp's shared-memory staging buffer, which is flushed with
 // one global atomic per ~STAGE_PAIRS pairs.  A block with more hits than the buffer holds goes
 // straight to global memory.  `fill` (warp-uniform) is the number of pairs staged so far.
-template <int NQ, bool GROUPED>
+template <int NQ, bool GROUPED, bool VERIFY = false>
 __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (&mask)[NQ], int lane, long long i, long long j0,
                                            int2 *buf, int &fill) {
     int cnt = 0;
@@ -357,15 +396,15 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
         total = __shfl_sync(0xffffffffu, incl, 31);
     }
     if (fill + total > STAGE_PAIRS) {
-        flush_pairs<GROUPED>(p, buf, fill, lane);
+        flush_pairs<GROUPED, VERIFY>(p, buf, fill, lane);
         fill = 0;
     }
     // bucketed mode stages regrouped positions; they become original rows when they leave the CTA
     const int ii = (int)(i + (GROUPED ? 0 : p.ioff));
     const int jj = (int)(j0 + (GROUPED ? 0 : p.joff));
     if (total > STAGE_PAIRS) {
-        if constexpr (GROUPED) {
-            if (p.rep > 0) {
+        if constexpr (GROUPED || VERIFY) {
+            if (VERIFY || p.rep > 0) {
                 // more hits in one block than the buffer holds (rare): check and write them one by one
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
@@ -373,7 +412,7 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
                     while (mk) {
                         const int c = __ffs(mk) - 1;
                         mk &= mk - 1;
-                        if (already_reported(p, ii, jj + 32 * q + c)) continue;
+                        if (drop_pair<GROUPED, VERIFY>(p, ii, jj + 32 * q + c)) continue;
                         const unsigned long long slot = atomicAdd(p.counter, 1ULL);
                         if (slot < p.capacity) p.out[slot] = final_pair<GROUPED>(p, make_int2(ii, jj + 32 * q + c));
                     }
@@ -739,6 +778,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         const int half = (warp - EPI_WARP0) >> 2;   // which of the tile's two P blocks (accumulator columns half * TILE_N ..)
         const int row_in_tile = half * TILE_M + quarter * 32 + lane;
         uint32_t acc = 0, accphase = 0, rstage = 0;   // rstage: next ring stage to hand back
+        constexpr bool VERIFY = DT == DT_I8 && KIND == KIND_COS;     // candidates are decided exactly at flush time
         int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * (WARP_STAGE_BYTES / 8);
         uint32_t *colterm = reinterpret_cast<uint32_t *>(stage_buf + STAGE_PAIRS);
         int stage_fill = 0;
@@ -760,6 +800,14 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     const float nxr = reinterpret_cast<const float *>(p.nx)[i];
                     rf = p.thr_f * nxr;
                     rzero = nxr == 0.f;
+                }
+                if constexpr (DT == DT_I8 && KIND == KIND_COS) {
+                    // fp32 filter for s >= t |x| |y|, lowered by 2^-18 relative (the fp32 roundings of t, the two norms,
+                    // the products and of s itself add up to under 2^-21): a necessary condition of the exact test,
+                    // which decides the surviving candidates when they leave the CTA.  t > 0: the norm of a zero
+                    // vector is stored as +inf, so that nothing involving it becomes a candidate.
+                    const float b = p.thr_f * reinterpret_cast<const float *>(p.nx)[i];
+                    rf = b >= 0.f ? b * (1.f - 0x1p-18f) : b * (1.f + 0x1p-18f);
                 }
                 // BF16/L2 decides |x|^2 + |y|^2 - 2s <= r^2 as  s >= (|x|^2 - r^2)/2 + |y|^2/2:  one add per element
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) rf = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] - p.thr_f);
@@ -786,12 +834,19 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     const float2 s0 = reinterpret_cast<const float2 *>(p.qstat)[qb0], s1 = reinterpret_cast<const float2 *>(p.qstat)[qb1];
                     ff = rf * (p.thr_f >= 0.f ? fminf(s0.x, s1.x) : fmaxf(s0.y, s1.y));     // s >= t|x| * min|y| (max|y| when t < 0)
                 }
+                if constexpr (DT == DT_I8 && KIND == KIND_COS) {
+                    const float2 s0 = reinterpret_cast<const float2 *>(p.qstat)[qb0], s1 = reinterpret_cast<const float2 *>(p.qstat)[qb1];
+                    // compared with the row maximum converted to fp32, as the element test converts the scores: the
+                    // conversion is monotone, so the bound stays a necessary condition of that test
+                    ff = rf * (p.thr_f >= 0.f ? fminf(s0.x, s1.x) : fmaxf(s0.y, s1.y));
+                }
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
                     const float2 s0 = reinterpret_cast<const float2 *>(p.qstat)[qb0], s1 = reinterpret_cast<const float2 *>(p.qstat)[qb1];
                     ff = rf + 0.5f * fminf(s0.x, s1.x);           // s >= (|x|^2 - r^2)/2 + min|y|^2/2
                 }
                 // per-column terms of this warp's columns, 4 per lane, fetched while the tile is still
-                // being multiplied so that the exact test never waits on global memory
+                // being multiplied so that the exact test never waits on global memory (fetching them only when a
+                // candidate shows up was measured: no gain for sparse joins, 5 % slower dense ones)
                 uint4 yq_pass[NPASS];
 #pragma unroll
                 for (int ps = 0; ps < NPASS; ++ps) {
@@ -867,6 +922,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 auto bound_ok = [&](uint32_t word) -> bool {
                     if constexpr (DT == DT_I8) {
                         const int mx = NARROW ? max((int)(short)(word & 0xffffu), (int)word >> 16) : (int)word;
+                        if constexpr (KIND == KIND_COS) return (float)mx >= ff;
                         return mx >= fi;
                     } else {
                         return __uint_as_float(word) >= ff;
@@ -953,6 +1009,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             if constexpr (DT == DT_I8 && KIND == KIND_IP) pass = (int)x >= p.thr_i;
                             if constexpr (DT == DT_I8 && KIND == KIND_L2) pass = 2 * (int)x - (int)yw[c] >= ri;
                             if constexpr (DT == DT_BF16 && KIND == KIND_IP) pass = __uint_as_float(x) >= p.thr_f;
+                            if constexpr (DT == DT_I8 && KIND == KIND_COS) pass = (float)(int)x >= rf * __uint_as_float(yw[c]);
                             if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
                                 const float nyr = __uint_as_float(yw[c]);
                                 pass = (rzero || nyr == 0.f) ? (p.thr_f <= 0.f) : (__uint_as_float(x) >= rf * nyr);
@@ -972,7 +1029,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             mask[q] &= lq >= 32 ? 0xffffffffu : (lq <= 0 ? 0u : ((1u << (int)lq) - 1u));
                         }
                     }
-                    emit_pairs<EPI_COLS / 32, GROUPED>(p, mask, lane, i, j0, stage_buf, stage_fill);
+                    emit_pairs<EPI_COLS / 32, GROUPED, VERIFY>(p, mask, lane, i, j0, stage_buf, stage_fill);
                 }
                 }   // passes
                 if constexpr (LONGK) {
@@ -983,7 +1040,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 }
             }
         }
-        if (ok) flush_pairs<GROUPED>(p, stage_buf, stage_fill, lane);
+        if (ok) flush_pairs<GROUPED, VERIFY>(p, stage_buf, stage_fill, lane);
     }
 
     tc_fence_before();

@@ -125,7 +125,6 @@ simjoin_status check_join_args(const simjoin_ctx *ctx, const void *P, int64_t n,
     }
     if (st != SIMJOIN_OK) return st;
     if (n + ctx->ioff >= SIMJOIN_MAX_ROWS || m + ctx->joff >= SIMJOIN_MAX_ROWS) return SIMJOIN_ERR_ARG;
-    if (ctx->dtype == SIMJOIN_I8 && kind == SIMJOIN_COS) return SIMJOIN_ERR_UNSUPPORTED;
     return SIMJOIN_OK;
 }
 
@@ -254,8 +253,10 @@ bool tile_geometry(const simjoin_ctx *ctx, int64_t n, int64_t m, int row_bytes, 
 
 // Thresholds in the precision each path decides in.
 void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold) {
+    jp.thr_d = threshold;
     if (i8) {
         if (kind == SIMJOIN_IP) jp.thr_i = clamp_to_i32(std::ceil(threshold));
+        else if (kind == SIMJOIN_COS) jp.thr_f = (float)threshold;      // fp32 filter; the exact test takes thr_d
         else {
             const double r2 = std::floor(threshold * threshold);
             jp.thr_i = r2 >= 1073741824.0 ? 1073741824 : (int)r2;   // 2^30 exceeds every int8 squared distance here
@@ -265,6 +266,13 @@ void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold
         // the inner-product test reads the sign of s - t: with t = -0 a score of either zero gives +0 and passes
         if (kind == SIMJOIN_IP && jp.thr_f == 0.f) jp.thr_f = -0.0f;
     }
+}
+
+// What the norm pre-pass stores per row.  0: |x|^2; 1: |x| in fp32 (cosine); 2: the same with +inf for a zero
+// vector -- int8 cosine with t > 0, where a zero vector passes nothing and must not raise candidates.
+int norm_mode(bool i8, simjoin_kind kind, double threshold) {
+    if (kind != SIMJOIN_COS) return 0;
+    return i8 && threshold > 0 ? 2 : 1;
 }
 
 // The join on device buffers.  Arguments were validated by the caller.
@@ -303,6 +311,9 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.joff = (int)ctx->joff;
 
     set_thresholds(jp, i8, kind, threshold);
+    jp.rows_p = P;
+    jp.rows_q = Q;
+    jp.row_bytes = row_bytes;
 
     const bool need_norms = kind != SIMJOIN_IP;
     if (need_norms) {
@@ -338,11 +349,11 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     }
     cudaEventRecord(ctx->ev[0], s);
     if (need_norms) {
-        const int sq = kind == SIMJOIN_COS ? 1 : 0;
+        const int sq = norm_mode(i8, kind, threshold);
         cudaError_t e1, e2;
         if (i8) {
-            e1 = launch_norms<true>(ctx, P, n, d, 0, ctx->nx.ptr, nullptr);
-            e2 = launch_norms<true>(ctx, Q, m, d, 0, ctx->ny.ptr, ctx->qstat.ptr);
+            e1 = launch_norms<true>(ctx, P, n, d, sq, ctx->nx.ptr, nullptr);
+            e2 = launch_norms<true>(ctx, Q, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
         } else {
             e1 = launch_norms<false>(ctx, P, n, d, sq, ctx->nx.ptr, nullptr);
             e2 = launch_norms<false>(ctx, Q, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
@@ -358,6 +369,8 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     if (longk) {
         if (i8 && kind == SIMJOIN_IP && narrow) e = launch_join_long<DT_I8, KIND_IP, true>(ctx, mapP, mapQ, jp, grid, smem);
         else if (i8 && kind == SIMJOIN_L2 && narrow) e = launch_join_long<DT_I8, KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
+        else if (i8 && kind == SIMJOIN_COS && narrow) e = launch_join_long<DT_I8, KIND_COS, true>(ctx, mapP, mapQ, jp, grid, smem);
+        else if (i8 && kind == SIMJOIN_COS) e = launch_join_long<DT_I8, KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem);
         else if (i8 && kind == SIMJOIN_IP) e = launch_join_long<DT_I8, KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
         else if (i8 && kind == SIMJOIN_L2) e = launch_join_long<DT_I8, KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
         else if (!i8 && kind == SIMJOIN_IP) e = launch_join_long<DT_BF16, KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
@@ -366,6 +379,8 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     } else
     if (i8 && kind == SIMJOIN_IP && narrow) e = launch_join<DT_I8, KIND_IP, true>(ctx, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_L2 && narrow) e = launch_join<DT_I8, KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
+    else if (i8 && kind == SIMJOIN_COS && narrow) e = launch_join<DT_I8, KIND_COS, true>(ctx, mapP, mapQ, jp, grid, smem);
+    else if (i8 && kind == SIMJOIN_COS) e = launch_join<DT_I8, KIND_COS>(ctx, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_IP) e = launch_join<DT_I8, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_L2) e = launch_join<DT_I8, KIND_L2>(ctx, mapP, mapQ, jp, grid, smem);
     else if (!i8 && kind == SIMJOIN_IP) e = launch_join<DT_BF16, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
@@ -403,6 +418,8 @@ cudaError_t launch_bucketed(simjoin_ctx *ctx, bool i8, simjoin_kind kind, bool n
     if (i8 && kind == SIMJOIN_IP) { SJ_BUCKETED(DT_I8, KIND_IP, false); }
     if (i8 && kind == SIMJOIN_L2 && narrow) { SJ_BUCKETED(DT_I8, KIND_L2, true); }
     if (i8 && kind == SIMJOIN_L2) { SJ_BUCKETED(DT_I8, KIND_L2, false); }
+    if (i8 && kind == SIMJOIN_COS && narrow) { SJ_BUCKETED(DT_I8, KIND_COS, true); }
+    if (i8 && kind == SIMJOIN_COS) { SJ_BUCKETED(DT_I8, KIND_COS, false); }
     if (!i8 && kind == SIMJOIN_IP) { SJ_BUCKETED(DT_BF16, KIND_IP, false); }
     if (!i8 && kind == SIMJOIN_COS) { SJ_BUCKETED(DT_BF16, KIND_COS, false); }
     if (!i8 && kind == SIMJOIN_L2) { SJ_BUCKETED(DT_BF16, KIND_L2, false); }
@@ -464,6 +481,9 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.ioff = (int)ctx->ioff;
     jp.joff = (int)ctx->joff;
     set_thresholds(jp, i8, kind, threshold);
+    jp.rows_p = ctx->lsh_sorted_p.ptr;      // the regrouped rows, addressed by regrouped position
+    jp.rows_q = ctx->lsh_sorted_q.ptr;
+    jp.row_bytes = row_bytes;
     if (need_norms) {
         jp.nx = ctx->nx.ptr;
         jp.ny = ctx->ny.ptr;
@@ -556,11 +576,11 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         }
         if (need_norms) {
             // row terms and per-256-row bounds of the regrouped rows
-            const int sq = kind == SIMJOIN_COS ? 1 : 0;
+            const int sq = norm_mode(i8, kind, threshold);
             cudaError_t e1, e2;
             if (i8) {
-                e1 = launch_norms<true>(ctx, ctx->lsh_sorted_p.ptr, n, d, 0, ctx->nx.ptr, nullptr);
-                e2 = launch_norms<true>(ctx, ctx->lsh_sorted_q.ptr, m, d, 0, ctx->ny.ptr, ctx->qstat.ptr);
+                e1 = launch_norms<true>(ctx, ctx->lsh_sorted_p.ptr, n, d, sq, ctx->nx.ptr, nullptr);
+                e2 = launch_norms<true>(ctx, ctx->lsh_sorted_q.ptr, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
             } else {
                 e1 = launch_norms<false>(ctx, ctx->lsh_sorted_p.ptr, n, d, sq, ctx->nx.ptr, nullptr);
                 e2 = launch_norms<false>(ctx, ctx->lsh_sorted_q.ptr, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
@@ -1101,6 +1121,9 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     jp.counter = ctrl;
     jp.status = reinterpret_cast<unsigned int *>(ctrl + 1);
     set_thresholds(jp, i8, kind, threshold);
+    jp.rows_p = P;
+    jp.rows_q = Q;
+    jp.row_bytes = row_bytes;
     jp.nx = nd.scratch + NA_OFF_NX;
     jp.ny = nd.scratch + NA_OFF_NY;
     jp.qstat = nd.scratch + NA_OFF_QSTAT;
@@ -1112,11 +1135,11 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     // the array keeps the previous call's contents: the counter / status block must start at zero
     if (cudaMemsetAsync(ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     if (kind != SIMJOIN_IP) {
-        const int sq = kind == SIMJOIN_COS ? 1 : 0;
+        const int sq = norm_mode(i8, kind, threshold);
         cudaError_t e1, e2;
         if (i8) {
-            e1 = launch_norms<true>(&tmp, P, n, d, 0, const_cast<void *>(jp.nx), nullptr);
-            e2 = launch_norms<true>(&tmp, Q, m, d, 0, const_cast<void *>(jp.ny), const_cast<void *>(jp.qstat));
+            e1 = launch_norms<true>(&tmp, P, n, d, sq, const_cast<void *>(jp.nx), nullptr);
+            e2 = launch_norms<true>(&tmp, Q, m, d, sq, const_cast<void *>(jp.ny), const_cast<void *>(jp.qstat));
         } else {
             e1 = launch_norms<false>(&tmp, P, n, d, sq, const_cast<void *>(jp.nx), nullptr);
             e2 = launch_norms<false>(&tmp, Q, m, d, sq, const_cast<void *>(jp.ny), const_cast<void *>(jp.qstat));
@@ -1126,6 +1149,7 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     cudaError_t e = cudaErrorInvalidValue;
     if (i8 && kind == SIMJOIN_IP) e = launch_join<DT_I8, KIND_IP>(&tmp, mapP, mapQ, jp, nd.sms, smem);
     else if (i8 && kind == SIMJOIN_L2) e = launch_join<DT_I8, KIND_L2>(&tmp, mapP, mapQ, jp, nd.sms, smem);
+    else if (i8 && kind == SIMJOIN_COS) e = launch_join<DT_I8, KIND_COS>(&tmp, mapP, mapQ, jp, nd.sms, smem);
     else if (!i8 && kind == SIMJOIN_IP) e = launch_join<DT_BF16, KIND_IP>(&tmp, mapP, mapQ, jp, nd.sms, smem);
     else if (!i8 && kind == SIMJOIN_COS) e = launch_join<DT_BF16, KIND_COS>(&tmp, mapP, mapQ, jp, nd.sms, smem);
     else if (!i8 && kind == SIMJOIN_L2) e = launch_join<DT_BF16, KIND_L2>(&tmp, mapP, mapQ, jp, nd.sms, smem);

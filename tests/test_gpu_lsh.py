@@ -127,7 +127,6 @@ def test_lsh_offsets_capacity_and_errors(ctx):
     assert ctx.simjoin_run_lsh(*args, 2, 0, 1, out, 8, L_low=1)[0] == B.SIMJOIN_ERR_ARG          # k - 1 bits needs k >= 1
     assert ctx.simjoin_run_lsh(*args, 60, 3, 1, out, 8, L_low=5)[0] == B.SIMJOIN_ERR_ARG
     assert ctx.simjoin_run_lsh(dP, 0, dQ, 2000, 128, 100.0, 2, 3, 1, out, 8) == (B.SIMJOIN_OK, 0)
-    assert ctx.simjoin_run_lsh(*args, 2, 3, 1, out, 8, kind="cos")[0] == B.SIMJOIN_ERR_UNSUPPORTED     # int8 x cosine, as simjoin_run
     # the plain join still works on the same context afterwards
     got, cnt = ctx.join(dP, dQ, "ip", w.threshold, 1 << 16)
     assert cnt == O.join(w.P, w.Q, "ip", w.threshold, "i8")[1]
@@ -177,6 +176,26 @@ def test_lsh_int8_euclidean_join(ctx, d, L, k):
         got = keys(out[:cnt].cpu().numpy())
         assert cnt == wcnt and len(np.unique(got)) == cnt and np.array_equal(got, keys(want)), (d, r, cnt, wcnt)
         assert cnt >= 100
+
+
+@pytest.mark.parametrize("d,L,k,hi", [(128, 4, 3, 2), (64, 3, 2, 127), (256, 3, 4, 127), (528, 2, 2, 40)])
+def test_lsh_int8_cosine_join(ctx, d, L, k, hi):
+    """int8 rows, cosine: the fp32 filter's candidates are decided exactly on the regrouped rows; exact pair set."""
+    P = W.random_points("i8", 1500 + 9, d, 71, lo=-hi, hi=hi)
+    Q = W.random_points("i8", 1900 + 5, d, 72, lo=-hi, hi=hi)
+    Q[7:600:3] = P[:198]
+    Q[8:600:3] = np.clip(P[200:398].astype(np.int16) + W.random_points("i8", 198, d, 73, lo=-1, hi=1), -127, 127).astype(np.int8)
+    P[1400] = 0
+    Q[1700] = 0
+    for t in (1.0, 0.8, 0.0):
+        dP, dQ = torch.from_numpy(P).cuda(), torch.from_numpy(Q).cuda()
+        out = torch.full((1 << 22, 2), -5, dtype=torch.int32, device="cuda:0")
+        st, cnt = ctx.simjoin_run_lsh(dP, len(P), dQ, len(Q), d, t, L, k, 23, out, 1 << 22, L_low=1, kind="cos")
+        assert st == B.SIMJOIN_OK, B.strerror(st)
+        want, wcnt = O.lsh_join_kind(P, Q, "cos", t, "i8", L, k, 23, L_low=1)
+        got = out[:cnt].cpu().numpy()
+        assert cnt == wcnt > 0 and np.array_equal(np.sort(keys(got)), np.sort(keys(want)))
+        assert np.all(out[cnt:].cpu().numpy() == -5)
 
 
 @pytest.mark.parametrize("kind", ["ip", "cos", "l2"])

@@ -257,7 +257,6 @@ def test_bad_arguments_are_rejected_before_launch(ctx_i8, ctx_bf16):
     U = B.SIMJOIN_ERR_UNSUPPORTED
     assert ctx_i8.simjoin_run(P, 64, P, 64, 24, "ip", 0.0, out, 8)[0] == U                   # 24 B rows
     assert ctx_i8.simjoin_run(P.data_ptr() + 1, 32, P, 64, 64, "ip", 0.0, out, 8)[0] == U    # misaligned
-    assert ctx_i8.simjoin_run(P, 64, P, 64, 64, "cos", 0.5, out, 8)[0] == U
     assert ctx_i8.simjoin_run(P, 1, P, 1, 16384, "ip", 0.0, out, 8)[0] == U                  # row too long
     assert ctx_i8.simjoin_last_kernel_ms()[0] in (B.SIMJOIN_OK, B.SIMJOIN_ERR_ARG)
     # the context is still usable afterwards
@@ -441,3 +440,51 @@ def test_two_dimensional_waves_cover_every_tile_pair_once(ctx_i8):
     pairs, cnt = gpu_join(ctx_i8, P, Q, "ip", t, capacity=1 << 20)
     assert_exact(pairs, cnt, P, Q, "ip", t)
     assert cnt >= len(Q[::11])
+
+
+# ------------------------------------------------------------------ int8 cosine (exact, as every int8 kind)
+def int8_cos_case(ctx_i8, P, Q, t, cap=1 << 20):
+    pairs, cnt = gpu_join(ctx_i8, P, Q, "cos", t, cap)
+    want, wcnt = O.join(P, Q, "cos", t, "i8")
+    assert cnt == wcnt, (cnt, wcnt, t)
+    got = np.asarray(pairs, dtype=np.int64).reshape(-1, 2)
+    assert len(np.unique((got[:, 0] << 32) | got[:, 1])) == cnt
+    assert set(map(tuple, got.tolist())) == set(map(tuple, want.tolist()))
+    return cnt
+
+
+@pytest.mark.parametrize("n,m,d,hi", [(300, 500, 64, 127), (1000, 777, 128, 3), (513, 1025, 48, 127), (700, 900, 272, 127),
+                                      (600, 400, 640, 5), (300, 700, 1040, 127), (260, 300, 2064, 127)])
+@pytest.mark.parametrize("t", [0.35, 0.0, -0.2])
+def test_i8_cosine_matches_oracle(ctx_i8, n, m, d, hi, t):
+    """Both epilogue widths (hi = 3, 5: scores fit 16 bits), every tile geometry, positive / zero / negative t."""
+    P, Q = W.random_points("i8", n, d, 51, lo=-hi, hi=hi), W.random_points("i8", m, d, 52, lo=-hi, hi=hi)
+    P[3] = 0
+    Q[7] = 0
+    Q[11] = P[5]                                              # cosine exactly 1
+    if t > 0:
+        allp = np.stack([np.repeat(np.arange(40), 50), np.tile(np.arange(50), 40)], axis=1).astype(np.int32)
+        t = float(np.quantile(O.scores(P, Q, "cos", "i8", allp), 0.995))   # a threshold that has hits at every d
+    assert int8_cos_case(ctx_i8, P, Q, t, cap=1 << 21) > 0
+
+
+def test_i8_cosine_threshold_one_and_ties(ctx_i8):
+    """Parallel rows score exactly 1 and pass t = 1; thresholds equal to attained scores are inclusive."""
+    rng = np.random.default_rng(5)
+    P = rng.integers(-60, 61, size=(400, 128)).astype(np.int8)
+    Q = rng.integers(-60, 61, size=(600, 128)).astype(np.int8)
+    Q[:100] = 2 * P[:100]
+    Q[100:150] = -P[100:150]
+    assert int8_cos_case(ctx_i8, P, Q, 1.0) == 100
+    assert int8_cos_case(ctx_i8, P, Q, -1.0) == 400 * 600
+    allp = np.stack([np.repeat(np.arange(400), 600), np.tile(np.arange(600), 400)], axis=1).astype(np.int32)
+    sc = np.sort(O.scores(P, Q, "cos", "i8", allp))
+    for t in (sc[-150], sc[-1000], np.nextafter(sc[-150], 2.0), np.nextafter(sc[-1000], -2.0)):
+        int8_cos_case(ctx_i8, P, Q, float(t))
+
+
+def test_i8_cosine_planted_pairs_at_scale(ctx_i8):
+    w = W.make_workload(4, n=20000, m=30000, planted=300)          # +-1 rows: cosine = <x,y> / d
+    t = w.threshold / w.d
+    cnt = int8_cos_case(ctx_i8, w.P, w.Q, t)
+    assert cnt >= 300 and cnt == O.join(w.P, w.Q, "ip", w.threshold, "i8")[1]
