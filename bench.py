@@ -261,6 +261,8 @@ def main():
     ap.add_argument("--planted", type=int, default=None)
     ap.add_argument("--d", type=int, default=None, help="override the dimension (profiling other row lengths; give --threshold too)")
     ap.add_argument("--threshold", type=float, default=None)
+    ap.add_argument("--kind", default=None, choices=["ip", "cos", "l2"],
+                    help="join kind to run on the configuration's points instead of its own (give --threshold too)")
     ap.add_argument("--sigma-reading", default="radial")
     ap.add_argument("--lsh", default=None, metavar="L,k[,L_low]",
                     help="time the LSH-bucketed join (int8 inner-product configs) instead of the brute-force join: "
@@ -288,6 +290,8 @@ def main():
 
     if args.impl == "reference":
         w = W.make_workload(args.config, sigma_reading=args.sigma_reading, **size_kw(args)) if rank == 0 else None
+        if w is not None and args.kind:
+            w.kind = args.kind
         run_reference(args, w)
         return
 
@@ -308,6 +312,8 @@ def main():
 
     # Each rank owns one row block of a (world * n)-row P and a full copy of Q.
     w = W.make_workload(args.config, seed=rank, sigma_reading=args.sigma_reading, **size_kw(args))
+    if args.kind:
+        w.kind = args.kind
     if world > 1:
         w.Q = W.make_workload(args.config, seed=0, sigma_reading=args.sigma_reading, **size_kw(args)).Q if rank else w.Q
         w.planted = w.planted if rank == 0 else np.zeros((0, 2), np.int64)
