@@ -77,6 +77,19 @@ def test_full_size_int8(cfg):
     check_sampled_rows(w, pairs, sample_rows(w, pairs), exact=True)
 
 
+def test_full_size_int8_cosine_on_the_config_4_points():
+    """The cosine join of int8 points at full size: the config-4 points, t = threshold / d (unit-modulus rows)."""
+    w = W.make_workload(4)
+    assert np.all(np.abs(w.P[:64]) == 1)                # +-1 rows: cosine = <x,y> / d
+    w.kind, w.threshold = "cos", w.threshold / w.d
+    pairs, cnt = run_full(w, capacity=4 * len(w.planted))
+    k = keys(pairs)
+    assert len(np.unique(k)) == cnt == len(w.planted)
+    assert np.isin(keys(w.planted), k).all()
+    assert np.all(O.scores(w.P, w.Q, "cos", "i8", pairs) >= w.threshold)
+    check_sampled_rows(w, pairs, sample_rows(w, pairs), exact=True)
+
+
 def test_full_size_cfg2_cosine():
     w = W.make_workload(2)
     pairs, cnt = run_full(w, capacity=1 << 16)
