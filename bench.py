@@ -23,6 +23,7 @@ configuration, ``--jl n,d,k`` the JL transform (``simjoin_jl_transform``) with a
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -466,7 +467,10 @@ def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32" if w.dtype == "i8" else "f32", "data": "synthetic",
             "config": {"workload": w.name, "n": w.n, "m": w.m, "d": w.d, "kind": w.kind, "in_dtype": w.dtype,
-                       "threshold": w.threshold, "pairs_found": int(cnt), "l2": "inputs (P+Q) larger than L2; no flush",
+                       "threshold": w.threshold, "pairs_found": int(cnt),
+                       "l2": ("inputs (P+Q) larger than L2; no flush" if w.P.nbytes + w.Q.nbytes > 126e6
+                              else "inputs (P+Q) fit in L2 and are not flushed between steps: not a headline number"),
+                       "inputs_sha256": {"P": hashlib.sha256(w.P).hexdigest(), "Q": hashlib.sha256(w.Q).hexdigest()},
                        "sharding": f"P row blocks x{world}, Q replicated" if world > 1 else "single GPU",
                        "note": w.note},
             "clocks": clocks,

@@ -51,3 +51,27 @@ def test_full_size_parameters_match_the_benchmark_table():
     assert (c[3]["n"], c[3]["d"], c[3]["threshold"], c[3]["planted"]) == (262144, 256, 3000.0, 10000)
     assert (c[4]["n"], c[4]["d"], c[4]["threshold"], c[4]["planted"]) == (1048576, 128, 100.0, 100000)
     assert (c[5]["n"], c[5]["d"], c[5]["threshold"], c[5]["centers"]) == (524288, 64, 0.25, 1024)
+
+
+# sha256 of the generated arrays (the bits every report's `inputs_sha256` names): guards the recipe against drift.
+# Written from the generator itself; these are inputs, not results.
+INPUT_SHA256 = {
+    1: ("cc9e8c4d39b49eb4c8cf9f6e01a01ded4d4eedc5dc2df9230e9b522874e58c77",
+        "0a4938c48a5f227fc5e45409c4087bee9ac569b0be4d7c6ba7daf800f06810e9"),
+    2: ("42199fde961e89aa19e75611b773b392cb36065f437aa282f5e3a17643efcd93",
+        "aec654e9d5d0adb86f0889852e8726f3f843342232ba2644f2b3d8ffbf716e5b"),
+    3: ("615a900578b4d996839c4928cdcaaf400a55adedab8bba587e82da141721b549",
+        "69ad8faef9a3425802989835650910d1406a9d2b52a407232d54c8252d1e4e32"),
+    4: ("6b25980a41b34306e72f85aa50340e9b80c765df6112c6c81fb9165942c6d371",
+        "823e1aca23c611d05517b00a278a3169fcdb7701fe3eb433d9fed01838d02b3d"),
+    5: ("38545e49488b86ae623b11f7dde58b7cc309cbcfa8fa311a16564ebecf742e1d",
+        "6092bca46ff31113246b175073696d709d362fb2aa4bd5055e7aa2bdac1e9537"),
+}
+SHA_SIZES = {1: {}, 2: {}, 3: dict(n=4096, m=4096, planted=64), 4: dict(n=4096, m=4096, planted=64), 5: dict(n=4096, m=4096)}
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_generated_inputs_have_the_recorded_hashes(cfg):
+    import hashlib
+    w = W.make_workload(cfg, **SHA_SIZES[cfg])
+    assert (hashlib.sha256(w.P).hexdigest(), hashlib.sha256(w.Q).hexdigest()) == INPUT_SHA256[cfg]
