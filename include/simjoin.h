@@ -116,7 +116,9 @@ simjoin_status simjoin_run(simjoin_ctx *ctx, const void *P, int64_t n, const voi
  * synchronised before return.  Pinned host memory makes the copies faster but
  * is not required.  A Q above 64 MiB is uploaded in slices of about 32 MiB on a second stream and every
  * slice is joined as soon as it has landed, so that (with pinned memory) the copies of later slices hide
- * behind the joins of earlier ones; the result is the union of the slices' results.
+ * behind the joins of earlier ones; the result is the union of the slices' results.  With room for 64 MiB of
+ * pairs or more (capacity >= 2^23) Q is cut into eight slices whatever its size, and the pairs of a slice are
+ * copied to out_pairs_host while the next slice is joined (dense results: the download hides behind the joins).
  * Errors as simjoin_run (device pointers are rejected here).
  */
 simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n, const void *Q_host,

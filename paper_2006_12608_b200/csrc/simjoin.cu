@@ -773,9 +773,13 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
     cudaStream_t s = ctx->stream;
     // A large Q goes up in slices of about 32 MiB on a second stream, and each slice is joined (a call of its own,
     // with the column offset of the slice) as soon as it has landed: the copies of the later slices hide behind
-    // the joins of the earlier ones.  The result is the union of the slices' results.
+    // the joins of the earlier ones.  The result is the union of the slices' results.  A caller that provides room
+    // for a large output (64 MiB of pairs and more) gets slices too, eight of them: the pairs of a slice travel back
+    // to the host on the second stream while the next slice is joined.
     const size_t row_bytes = (size_t)d * es;
-    const int64_t slice_rows = qb > (64u << 20) ? (int64_t)(((32u << 20) / row_bytes + TILE_N - 1) / TILE_N * TILE_N) : m;
+    int64_t slice_rows = m;
+    if (qb > (64u << 20)) slice_rows = (int64_t)(((32u << 20) / row_bytes + TILE_N - 1) / TILE_N * TILE_N);
+    else if (ob >= (64u << 20) && m >= 8 * 4096) slice_rows = ((m + 7) / 8 + LONG_TN - 1) / LONG_TN * LONG_TN;
     const int nslices = (int)((m + slice_rows - 1) / slice_rows);
     if (nslices > 1 && nslices <= (int)(sizeof ctx->copy_ev / sizeof ctx->copy_ev[0])) {
         if (!ctx->copy_stream && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return SIMJOIN_ERR_CUDA;
@@ -810,15 +814,22 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
             total += cnt;
             if (sq != SIMJOIN_OK) st = sq;
             if (ctx->have_timing) { pre_ms += ctx->prepass_ms; join_ms += ctx->join_ms; }
+            // the slice's join has finished (run_device synchronises): its pairs go home behind the next slice's join
+            const uint64_t now = total < capacity ? total : capacity;
+            if ((sq == SIMJOIN_OK || sq == SIMJOIN_ERR_CAPACITY) && now > used &&
+                cudaMemcpyAsync(out_pairs_host + 2 * used, reinterpret_cast<int32_t *>(ctx->stage_out.ptr) + 2 * used,
+                                (size_t)(now - used) * 8, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+                st = SIMJOIN_ERR_CUDA;
         }
-        if (st != SIMJOIN_OK && st != SIMJOIN_ERR_CAPACITY) {
-            cudaStreamSynchronize(cs);
-            return st;
+        if (cudaStreamSynchronize(cs) != cudaSuccess) {
+            cudaGetLastError();
+            return SIMJOIN_ERR_CUDA;
         }
+        if (st != SIMJOIN_OK && st != SIMJOIN_ERR_CAPACITY) return st;
         ctx->prepass_ms = pre_ms;
         ctx->join_ms = join_ms;
         *count = total;
-        st = total > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
+        return total > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
     } else {
         if (cudaMemcpyAsync(ctx->stage_p.ptr, P_host, pb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
             cudaMemcpyAsync(ctx->stage_q.ptr, Q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess)

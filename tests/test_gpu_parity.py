@@ -312,6 +312,28 @@ def test_run_host_uploads_a_large_q_in_slices(ctx_i8, ctx_bf16):
     assert_band(outb[:cnt], cnt, Pb, Qb, "cos", 0.03)
 
 
+def test_run_host_downloads_a_dense_result_slice_by_slice(ctx_i8):
+    """Room for 2^23 pairs and more: Q is joined in eight slices and every slice's pairs travel to the host while the
+    next slice is joined.  Result and overflow behaviour are those of the one-piece call."""
+    P, Q = W.random_points("i8", 300, 64, 75, lo=-3, hi=3), W.random_points("i8", 40000 + 37, 64, 76, lo=-3, hi=3)
+    t = 4.0
+    want, wcnt = O.join(P, Q, "ip", t, "i8")
+    assert wcnt > 3_000_000
+    cap = 1 << 23
+    out = np.full((cap + 4, 2), -7, dtype=np.int32)
+    st, cnt = ctx_i8.simjoin_run_host(P, len(P), Q, len(Q), 64, "ip", t, out, cap)
+    assert (st, cnt) == (B.SIMJOIN_OK, wcnt)
+    assert np.array_equal(np.sort(keys(out[:cnt])), keys(want)) and np.all(out[cnt:] == -7)
+    # more pairs than room: capacity is shared by the slices, the count stays the full one
+    P2 = W.random_points("i8", 900, 64, 77, lo=-3, hi=3)
+    want2, wcnt2 = O.join(P2, Q, "ip", t, "i8")
+    assert wcnt2 > cap
+    st, cnt = ctx_i8.simjoin_run_host(P2, len(P2), Q, len(Q), 64, "ip", t, out, cap)
+    assert (st, cnt) == (B.SIMJOIN_ERR_CAPACITY, wcnt2)
+    got = keys(out[:cap])
+    assert len(np.unique(got)) == cap and np.isin(got, keys(want2)).all() and np.all(out[cap:] == -7)
+
+
 def test_row_norms_prepass(ctx_i8, ctx_bf16):
     for rows, d in [(1, 16), (300, 64), (1000, 144), (513, 1024)]:
         X = W.random_points("i8", rows, d, 18, lo=-128, hi=127)
