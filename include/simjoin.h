@@ -218,6 +218,46 @@ simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t
                                    int32_t d, double r, int32_t *out_pairs, uint64_t capacity, uint64_t *count);
 
 /*
+ * Candidate filter (Section 4's join definition applied to a list of pairs instead of all of P x Q): keeps the
+ * listed pairs (i, j) for which (row i of P, row j of Q) passes `kind` at `threshold`, and drops the others.
+ *
+ *   P, Q, n, m, d, kind, threshold   as simjoin_run.
+ *   pairs       device pointer to count_in x 2 int32, 8-byte aligned: indices as the joins of this context emit them
+ *               (row offsets of simjoin_set_offsets included).  Compacted in place; the order of the kept pairs is
+ *               unspecified.  An index outside [0, n) x [0, m) makes the call return ERR_ARG (the list is then
+ *               unspecified, nothing outside it is touched).
+ *   count_out   HOST pointer; number of pairs kept.
+ *
+ * Arithmetic: I8 exact (the decisions simjoin_run takes); BF16 in fp32 -- inner product and cosine as sums over
+ * the row, the Euclidean distance in the difference form sum (x - y)^2 <= r^2 (no cancellation of large norms);
+ * a pair whose exact score lies within 1e-2*|threshold| of the threshold may fall on either side.
+ * One warp per pair, two rows read per pair.  Synchronises the stream.  Scratch: count_in x 8 bytes.
+ */
+simjoin_status simjoin_filter_pairs(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
+                                    simjoin_kind kind, double threshold, int32_t *pairs, uint64_t count_in,
+                                    uint64_t *count_out);
+
+/*
+ * Euclidean join behind a JL pre-reduction (Section 3's transform used as the paper introduces it: reduce the
+ * dimension, then search): both point sets are reduced from d to k coordinates with the same matrix M
+ * (simjoin_jl_transform, same seed), the reduced points are joined with the radius widened to r * (1 + slack),
+ * and the candidates are decided on the original rows (simjoin_filter_pairs, radius r).  The result is a subset
+ * of the exact join { (i, j) : |x_i - y_j| <= r } (band rule of simjoin_filter_pairs): a true pair is missed only
+ * when M stretches its distance by more than 1 + slack.  With random-sign levels the relative spread of |M z| / |z|
+ * is about 1 / sqrt(2k) per level; slack = 0.3 at k = 64 loses well under 1 % of the pairs.
+ *
+ *   P, Q        device pointers, n x d and m x d bf16.  d, k, seed: as simjoin_jl_transform.  slack >= 0.
+ *   out_pairs, capacity, count: as simjoin_run; the capacity must hold the CANDIDATES (when it does not, the call
+ *               returns ERR_CAPACITY with *count = the number of candidates and out_pairs unspecified).
+ *
+ * BF16 contexts only.  Scratch: the two reduced sets ((n + m) x k bf16) plus that of the calls above.
+ * simjoin_last_kernel_ms then reports (both transforms, reduced join + filter).
+ */
+simjoin_status simjoin_run_jl_l2(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, double r,
+                                 int32_t k, uint64_t seed, double slack, int32_t *out_pairs, uint64_t capacity,
+                                 uint64_t *count);
+
+/*
  * Row squared norms, the pre-pass behind the |x|^2 and |y|^2 terms of the
  * squared-L2 and cosine ip-distances (Section 4).  X: device pointer, rows x d.
  * out: device pointer to `rows` values -- int32 (exact) for I8 contexts, fp32

@@ -307,6 +307,17 @@ def scores(P, Q, kind: str, dtype: str, pairs: np.ndarray) -> np.ndarray:
     return out
 
 
+def filter_pairs(P, Q, kind: str, threshold: float, dtype: str, pairs: np.ndarray) -> np.ndarray:
+    """The listed pairs that pass: Section 4's join predicate applied pair by pair (same decisions as `join`)."""
+    pairs = np.ascontiguousarray(pairs, dtype=np.int32).reshape(-1, 2)
+    sc = scores(P, Q, kind, dtype, pairs)
+    if kind == "l2":
+        keep = sc.astype(np.float64) <= (float(threshold) * float(threshold) if dtype == "i8" else float(threshold))
+    else:
+        keep = sc.astype(np.float64) >= float(threshold)
+    return pairs[keep]
+
+
 def sq_norms(X: np.ndarray, dtype: str) -> np.ndarray:
     """Row squared norms: exact int64 (int8 rows) or fp64 (bf16 rows)."""
     lib = _load()

@@ -21,7 +21,7 @@ SIMJOIN_IP, SIMJOIN_COS, SIMJOIN_L2 = 0, 1, 2
 DTYPE = {"i8": SIMJOIN_I8, "bf16": SIMJOIN_BF16}
 KIND = {"ip": SIMJOIN_IP, "cos": SIMJOIN_COS, "l2": SIMJOIN_L2}
 
-EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_hamming", "simjoin_run_lsh", "simjoin_run_hamming_lsh", "simjoin_jl_transform", "simjoin_row_norms", "simjoin_set_offsets",
+EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_hamming", "simjoin_run_lsh", "simjoin_run_hamming_lsh", "simjoin_jl_transform", "simjoin_filter_pairs", "simjoin_run_jl_l2", "simjoin_row_norms", "simjoin_set_offsets",
            "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_selftest_wait_timeout", "simjoin_destroy",
            "simjoin_strerror")
 SIMJOIN_NOALLOC_MAX_ROWS = 65536
@@ -60,6 +60,10 @@ def load() -> ctypes.CDLL:
     lib.simjoin_run_hamming_lsh.argtypes = [vp, vp, i64, vp, i64, i32, dbl, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
     lib.simjoin_jl_transform.restype = c.c_int
     lib.simjoin_jl_transform.argtypes = [vp, vp, i64, i32, i32, u64, vp]
+    lib.simjoin_filter_pairs.restype = c.c_int
+    lib.simjoin_filter_pairs.argtypes = [vp, vp, i64, vp, i64, i32, c.c_int, dbl, vp, u64, c.POINTER(u64)]
+    lib.simjoin_run_jl_l2.restype = c.c_int
+    lib.simjoin_run_jl_l2.argtypes = [vp, vp, i64, vp, i64, i32, dbl, i32, u64, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_run_noalloc.restype = c.c_int
     lib.simjoin_run_noalloc.argtypes = [c.c_int, vp, c.c_int, vp, i64, vp, i64, i32, c.c_int, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_row_norms.restype = c.c_int
@@ -161,6 +165,20 @@ class Simjoin:
     def simjoin_jl_transform(self, X, n, d, k, seed, out):
         (xp, _a), (op, _b) = _ptr(X), _ptr(out)
         return load().simjoin_jl_transform(self._h, xp, n, d, k, int(seed), op)
+
+    def simjoin_filter_pairs(self, P, n, Q, m, d, kind, threshold, pairs, count_in):
+        cnt = ctypes.c_uint64(0)
+        (pp, _a), (qp, _b), (lp, _c) = _ptr(P), _ptr(Q), _ptr(pairs)
+        st = load().simjoin_filter_pairs(self._h, pp, n, qp, m, d, KIND[kind] if isinstance(kind, str) else kind,
+                                         float(threshold), lp, count_in, ctypes.byref(cnt))
+        return st, cnt.value
+
+    def simjoin_run_jl_l2(self, P, n, Q, m, d, r, k, seed, slack, out_pairs, capacity):
+        cnt = ctypes.c_uint64(0)
+        (pp, _a), (qp, _b), (op, _c) = _ptr(P), _ptr(Q), _ptr(out_pairs)
+        st = load().simjoin_run_jl_l2(self._h, pp, n, qp, m, d, float(r), k, int(seed), float(slack), op, capacity,
+                                      ctypes.byref(cnt))
+        return st, cnt.value
 
     def simjoin_row_norms(self, X, rows, d, out):
         (xp, _a), (op, _b) = _ptr(X), _ptr(out)

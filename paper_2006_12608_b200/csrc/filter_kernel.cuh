@@ -1,0 +1,102 @@
+// Candidate filter: given a list of index pairs (i, j), keep those whose rows pass the join's predicate
+// (Section 4's definition, applied to listed pairs instead of all of P x Q).  It closes the approximate pipeline
+// "reduce with the JL transform of Section 3, join the short rows with some slack, decide the candidates on the
+// original rows": whatever distortion the reduction adds, only true pairs leave.
+// One warp per pair: the lanes stride over the 16-byte groups of the two rows, three running sums are reduced with
+// shuffles, lane 0 decides and appends the pair to the output list (one atomic per kept pair; order unspecified).
+// HBM/L2-bound: 2 rows per candidate.  A listed index outside the point sets raises a status bit and is skipped.
+#pragma once
+#include <cstdint>
+
+namespace sj {
+
+constexpr int FILTER_THREADS = 256;
+
+// int8 rows: exact integer sums.  IP: s >= ceil(t) (thr_i);  L2: sum (x-y)^2 <= floor(r^2) (thr_i), taken as
+// |x|^2 + |y|^2 - 2s in integers;  COS: the fp64 sequence of the join's exact test (thr_d).
+// bf16 rows: fp32 sums.  IP: s >= t;  COS: s >= t |x| |y|, a zero vector scoring 0;  L2: the difference form
+// sum (x-y)^2 <= r^2, which does not cancel like the norm expansion of the tile epilogue.
+template <int DT, int KIND>
+__global__ void __launch_bounds__(FILTER_THREADS)
+filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__restrict__ Q, long long m, int g,
+                    const int2 *__restrict__ in, unsigned long long count_in, int ioff, int joff, int thr_i, float thr_f,
+                    double thr_d, int2 *__restrict__ out, unsigned long long *__restrict__ counter,
+                    unsigned int *__restrict__ status) {
+    const int lane = threadIdx.x & 31;
+    const unsigned long long warp = ((unsigned long long)blockIdx.x * FILTER_THREADS + threadIdx.x) >> 5;
+    const unsigned long long nwarps = ((unsigned long long)gridDim.x * FILTER_THREADS) >> 5;
+    for (unsigned long long k = warp; k < count_in; k += nwarps) {
+        const int2 pr = in[k];
+        const long long li = (long long)pr.x - ioff, lj = (long long)pr.y - joff;
+        if (li < 0 || li >= n || lj < 0 || lj >= m) {      // not a pair of these point sets: flag it, touch nothing
+            if (lane == 0) atomicOr(status, 0x20000000u);
+            continue;
+        }
+        const uint4 *x = P + li * g, *y = Q + lj * g;
+        bool pass = false;
+        if constexpr (DT == DT_I8) {
+            int s = 0, nx = 0, ny = 0;
+            for (int c = lane; c < g; c += 32) {
+                const uint4 a = __ldg(x + c), b = __ldg(y + c);
+                const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    s = __dp4a((int)aw[t], (int)bw[t], s);
+                    nx = __dp4a((int)aw[t], (int)aw[t], nx);
+                    ny = __dp4a((int)bw[t], (int)bw[t], ny);
+                }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                s += __shfl_xor_sync(0xffffffffu, s, off);
+                nx += __shfl_xor_sync(0xffffffffu, nx, off);
+                ny += __shfl_xor_sync(0xffffffffu, ny, off);
+            }
+            if constexpr (KIND == KIND_IP) pass = s >= thr_i;
+            if constexpr (KIND == KIND_L2) pass = (long long)nx + ny - 2LL * s <= (long long)thr_i;
+            if constexpr (KIND == KIND_COS) {
+                if (nx == 0 || ny == 0) pass = 0.0 >= thr_d;
+                else pass = __ddiv_rn((double)s, __dsqrt_rn(__ll2double_rn((long long)nx * (long long)ny))) >= thr_d;
+            }
+        } else {
+            float s = 0.f, nx = 0.f, ny = 0.f;       // L2: s accumulates the squared differences
+            for (int c = lane; c < g; c += 32) {
+                const uint4 a = __ldg(x + c), b = __ldg(y + c);
+                const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float x0 = __uint_as_float(aw[t] << 16), x1 = __uint_as_float(aw[t] & 0xffff0000u);
+                    const float y0 = __uint_as_float(bw[t] << 16), y1 = __uint_as_float(bw[t] & 0xffff0000u);
+                    if constexpr (KIND == KIND_L2) {
+                        const float e0 = x0 - y0, e1 = x1 - y1;
+                        s = fmaf(e0, e0, s);
+                        s = fmaf(e1, e1, s);
+                    } else {
+                        s = fmaf(x0, y0, s);
+                        s = fmaf(x1, y1, s);
+                    }
+                    if constexpr (KIND == KIND_COS) {
+                        nx = fmaf(x0, x0, nx);
+                        nx = fmaf(x1, x1, nx);
+                        ny = fmaf(y0, y0, ny);
+                        ny = fmaf(y1, y1, ny);
+                    }
+                }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                s += __shfl_xor_sync(0xffffffffu, s, off);
+                if constexpr (KIND == KIND_COS) {
+                    nx += __shfl_xor_sync(0xffffffffu, nx, off);
+                    ny += __shfl_xor_sync(0xffffffffu, ny, off);
+                }
+            }
+            if constexpr (KIND == KIND_IP) pass = s >= thr_f;
+            if constexpr (KIND == KIND_L2) pass = s <= thr_f;
+            if constexpr (KIND == KIND_COS) pass = (nx == 0.f || ny == 0.f) ? thr_f <= 0.f : s >= thr_f * sqrtf(nx) * sqrtf(ny);
+        }
+        if (lane == 0 && pass) out[atomicAdd(counter, 1ULL)] = pr;
+    }
+}
+
+}  // namespace sj

@@ -12,6 +12,7 @@
 #include <new>
 
 #include "join_kernel.cuh"
+#include "filter_kernel.cuh"
 #include "jl_kernel.cuh"
 #include "lsh_kernel.cuh"
 #include "prepass_kernel.cuh"
@@ -54,6 +55,8 @@ struct simjoin_ctx {
     cudaStream_t copy_stream;           // simjoin_run_host: uploads of Q slices overlap the joins of earlier slices
     cudaEvent_t copy_ev[66];
     DevBuf jl_a, jl_buf[2];             // JL transform: level matrix, ping-pong level outputs
+    DevBuf jl_p, jl_q;                  // simjoin_run_jl_l2: the reduced point sets
+    DevBuf filter_out;                  // simjoin_filter_pairs: the kept pairs before they replace the list
     // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
     DevBuf lsh_keys_p, lsh_keys_q, lsh_skeys_p, lsh_skeys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
 };
@@ -647,6 +650,54 @@ simjoin_status hamming_unpack(simjoin_ctx *ctx, const void *P_bits, int64_t n, c
     return cudaGetLastError() == cudaSuccess ? SIMJOIN_OK : SIMJOIN_ERR_CUDA;
 }
 
+// Keep the listed pairs whose rows pass the predicate; the list is compacted in place (order unspecified).
+simjoin_status filter_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, simjoin_kind kind,
+                             double threshold, int32_t *pairs, uint64_t count_in, uint64_t *count_out) {
+    *count_out = 0;
+    if (count_in == 0) return SIMJOIN_OK;
+    const bool i8 = ctx->dtype == SIMJOIN_I8;
+    const int g = (int)((size_t)d * elem_size(ctx->dtype) / 16);
+    if (!grow(ctx->filter_out, (size_t)count_in * 8)) return SIMJOIN_ERR_CUDA;
+    JoinParams jp;
+    std::memset(&jp, 0, sizeof jp);
+    set_thresholds(jp, i8, kind, threshold);
+    cudaStream_t s = ctx->stream;
+    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    // one warp per pair, at most 16 blocks per SM (the warps then stride over the list)
+    const unsigned long long want_blocks = (count_in * 32 + FILTER_THREADS - 1) / FILTER_THREADS;
+    const unsigned long long max_blocks = (unsigned long long)ctx->num_sms * 16;
+    const unsigned blocks = (unsigned)(want_blocks < max_blocks ? want_blocks : max_blocks);
+    const uint4 *p4 = reinterpret_cast<const uint4 *>(P), *q4 = reinterpret_cast<const uint4 *>(Q);
+    const int2 *in = reinterpret_cast<const int2 *>(pairs);
+    int2 *out = reinterpret_cast<int2 *>(ctx->filter_out.ptr);
+    unsigned int *status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
+#define SJ_FILTER(DT, KIND)                                                                                              \
+    filter_pairs_kernel<DT, KIND><<<blocks, FILTER_THREADS, 0, s>>>(p4, n, q4, m, g, in, count_in, (int)ctx->ioff, (int)ctx->joff, \
+                                                                    jp.thr_i, jp.thr_f, jp.thr_d, out, ctx->d_ctrl, status)
+    if (i8 && kind == SIMJOIN_IP) SJ_FILTER(DT_I8, KIND_IP);
+    else if (i8 && kind == SIMJOIN_COS) SJ_FILTER(DT_I8, KIND_COS);
+    else if (i8) SJ_FILTER(DT_I8, KIND_L2);
+    else if (kind == SIMJOIN_IP) SJ_FILTER(DT_BF16, KIND_IP);
+    else if (kind == SIMJOIN_COS) SJ_FILTER(DT_BF16, KIND_COS);
+    else SJ_FILTER(DT_BF16, KIND_L2);
+#undef SJ_FILTER
+    if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    if ((ctx->h_ctrl[1] & 0xffffffffu) != 0) return SIMJOIN_ERR_ARG;        // an index outside the point sets
+    const uint64_t kept = ctx->h_ctrl[0];
+    if (kept > 0 && (cudaMemcpyAsync(pairs, out, (size_t)kept * 8, cudaMemcpyDeviceToDevice, s) != cudaSuccess ||
+                     cudaStreamSynchronize(s) != cudaSuccess)) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    *count_out = kept;
+    return SIMJOIN_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -716,6 +767,9 @@ simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
     release(ctx->jl_a);
     release(ctx->jl_buf[0]);
     release(ctx->jl_buf[1]);
+    release(ctx->jl_p);
+    release(ctx->jl_q);
+    release(ctx->filter_out);
     release(ctx->lsh_keys_p);
     release(ctx->lsh_keys_q);
     release(ctx->lsh_skeys_p);
@@ -978,6 +1032,65 @@ simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, 
         ctx->have_timing = true;
     }
     return SIMJOIN_OK;
+}
+
+simjoin_status simjoin_filter_pairs(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
+                                    simjoin_kind kind, double threshold, int32_t *pairs, uint64_t count_in, uint64_t *count_out) {
+    if (!count_out) return SIMJOIN_ERR_ARG;
+    simjoin_status st = check_join_args(ctx, P, n, Q, m, d, kind, threshold, pairs, count_in, count_out);
+    if (st != SIMJOIN_OK) return st;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    *count_out = 0;
+    if (count_in == 0) return SIMJOIN_OK;
+    if (n == 0 || m == 0) return SIMJOIN_ERR_ARG;                        // a listed pair cannot exist
+    if (!is_device_ptr(P, ctx->device) || !is_device_ptr(Q, ctx->device) || !is_device_ptr(pairs, ctx->device)) return SIMJOIN_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
+    ctx->have_timing = false;
+    return filter_device(ctx, P, n, Q, m, d, kind, threshold, pairs, count_in, count_out);
+}
+
+simjoin_status simjoin_run_jl_l2(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, double r,
+                                 int32_t k, uint64_t seed, double slack, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+    simjoin_status st = check_join_args(ctx, P, n, Q, m, d, SIMJOIN_L2, r, out_pairs, capacity, count);
+    if (st != SIMJOIN_OK) return st;
+    if (ctx->dtype != SIMJOIN_BF16) return SIMJOIN_ERR_UNSUPPORTED;
+    if (std::isnan(slack) || slack < 0 || std::isinf(slack)) return SIMJOIN_ERR_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    if ((n > 0 && !is_device_ptr(P, ctx->device)) || (m > 0 && !is_device_ptr(Q, ctx->device))) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && !is_device_ptr(out_pairs, ctx->device)) return SIMJOIN_ERR_ARG;
+    if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
+    *count = 0;
+    if (n == 0 || m == 0) return simjoin_jl_transform(ctx, P, 0, d, k, seed, const_cast<void *>(P));   // shape rules only
+    if (!grow(ctx->jl_p, (size_t)n * k * 2 + 16) || !grow(ctx->jl_q, (size_t)m * k * 2 + 16)) return SIMJOIN_ERR_CUDA;
+    // the same M for both sets: |M x - M y| = |M (x - y)| is within a factor 1 +- eps of |x - y|
+    st = simjoin_jl_transform(ctx, P, n, d, k, seed, ctx->jl_p.ptr);
+    if (st != SIMJOIN_OK) return st;
+    float jl_ms = ctx->have_timing ? ctx->join_ms : 0.f;
+    st = simjoin_jl_transform(ctx, Q, m, d, k, seed, ctx->jl_q.ptr);
+    if (st != SIMJOIN_OK) return st;
+    jl_ms += ctx->have_timing ? ctx->join_ms : 0.f;
+    // candidates: the join of the reduced points with the radius widened by the slack
+    uint64_t cand = 0;
+    st = run_device(ctx, ctx->jl_p.ptr, n, ctx->jl_q.ptr, m, k, SIMJOIN_L2, r * (1.0 + slack), out_pairs, capacity, &cand);
+    const float join_ms = ctx->have_timing ? ctx->prepass_ms + ctx->join_ms : 0.f;
+    if (st == SIMJOIN_ERR_CAPACITY) {
+        *count = cand;                  // more candidates than room: nothing can be decided
+        return st;
+    }
+    if (st != SIMJOIN_OK) return st;
+    cudaStream_t s = ctx->stream;
+    cudaEventRecord(ctx->ev[0], s);
+    st = filter_device(ctx, P, n, Q, m, d, SIMJOIN_L2, r, out_pairs, cand, count);
+    cudaEventRecord(ctx->ev[1], s);
+    float f_ms = 0.f;
+    if (st == SIMJOIN_OK && cudaEventSynchronize(ctx->ev[1]) == cudaSuccess && cudaEventElapsedTime(&f_ms, ctx->ev[0], ctx->ev[1]) == cudaSuccess) {
+        ctx->prepass_ms = jl_ms;
+        ctx->join_ms = join_ms + f_ms;
+        ctx->have_timing = true;
+    }
+    return st;
 }
 
 simjoin_status simjoin_row_norms(simjoin_ctx *ctx, const void *X, int64_t rows, int32_t d, void *out) {

@@ -582,3 +582,22 @@ def test_int8_cosine_of_parallel_rows_is_exactly_one_even_beyond_2_to_53():
     assert int(P[0].astype(np.int64) @ P[0]) * int(Q[0].astype(np.int64) @ Q[0]) > 2 ** 53
     got, cnt = O.join(P, Q, "cos", 1.0, "i8")
     assert got.tolist() == [[i, i] for i in range(5)]
+
+
+# ------------------------------------------------------------------ the pair filter
+@pytest.mark.parametrize("dtype,kind,t", [("i8", "ip", 30.0), ("i8", "l2", 14.5), ("i8", "cos", 0.2),
+                                          ("bf16", "ip", 2.0), ("bf16", "cos", 0.25), ("bf16", "l2", 5.0)])
+def test_filter_of_every_pair_is_the_join(dtype, kind, t):
+    if dtype == "i8":
+        P, Q = W.random_points("i8", 37, 24, 5, lo=-4, hi=4), W.random_points("i8", 41, 24, 6, lo=-4, hi=4)
+    else:
+        P, Q = W.random_points("bf16", 37, 24, 5), W.random_points("bf16", 41, 24, 6)
+    allp = np.array(list(itertools.product(range(len(P)), range(len(Q)))), dtype=np.int32)
+    want, cnt = O.join(P, Q, kind, t, dtype)
+    assert 0 < cnt < len(allp)
+    assert np.array_equal(O.filter_pairs(P, Q, kind, t, dtype, allp), want)
+    rng = np.random.default_rng(3)
+    some = allp[rng.permutation(len(allp))[:400]]
+    kept = O.filter_pairs(P, Q, kind, t, dtype, some)
+    assert as_set(kept) == as_set(want) & as_set(some)
+    assert [tuple(p) for p in kept.tolist()] == [tuple(p) for p in some.tolist() if tuple(p) in as_set(want)]   # order kept
