@@ -233,6 +233,65 @@ def run_jl(args):
     print(json.dumps(line), flush=True)
 
 
+def run_jl_join(args):
+    """--jl-join n,d,k[,slack]: the Euclidean join behind a JL pre-reduction (simjoin_run_jl_l2) on the config-2 recipe
+    at dimension d (unit rows, 5000 planted near pairs, r = 0.45), timed beside the direct join of the same points."""
+    import torch
+    from paper_2006_12608_b200 import binding as B
+    from paper_2006_12608_b200 import build
+    n, d, k = (int(x) for x in args.jl_join[:3])
+    slack = float(args.jl_join[3]) if len(args.jl_join) > 3 else 0.3
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the join has no CPU path")
+    if not os.path.exists(B.LIB_PATH):
+        build.build()
+    torch.cuda.set_device(0)
+    w = W.make_workload(2, n=n, m=n, d=d, planted=5000)
+    r = 0.45
+    ctx = B.Simjoin("bf16", 0)
+    dP, dQ = B.to_device(w.P), B.to_device(w.Q)
+    cap = 1 << 22
+    out = torch.empty((cap, 2), dtype=torch.int32, device="cuda:0")
+
+    def timed(fn):
+        ts = []
+        for it in range(args.warmup + args.steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            st, cnt = fn()
+            e1.record()
+            torch.cuda.synchronize()
+            if st != B.SIMJOIN_OK:
+                raise RuntimeError(B.strerror(st))
+            if it >= args.warmup:
+                ts.append(e0.elapsed_time(e1))
+        got = out[:cnt].cpu().numpy().astype(np.int64)
+        return statistics.mean(ts), (got[:, 0] << 32) | got[:, 1]
+
+    direct_ms, exact = timed(lambda: ctx.simjoin_run(dP, n, dQ, n, d, "l2", r, out, cap))
+    sampler = ClockSampler(0)
+    sampler.start()
+    ms, got = timed(lambda: ctx.simjoin_run_jl_l2(dP, n, dQ, n, d, r, k, 2006, slack, out, cap))
+    clocks = sampler.stop()
+    _st, jl_ms, rest_ms = ctx.simjoin_last_kernel_ms()
+    ctx.close()
+    ops = 2.0 * n * n * d
+    line = {"metric": METRIC, "value": ops / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"cfg2 recipe at d={d}, {n} x {n}, l2 r={r}", "n": n, "m": n, "d": d, "kind": "l2",
+                       "threshold": r, "pairs_found": int(len(got))},
+            "clocks": clocks, "e2e": None, "gpu_launches": None, "roofline": None,
+            "algorithm": {"name": "JL pre-reduction + join + candidate filter (simjoin_run_jl_l2)", "k": k, "slack": slack,
+                          "jl_ms": jl_ms, "reduced_join_and_filter_ms": rest_ms, "direct_join_ms": direct_ms,
+                          "speedup_over_direct_join": direct_ms / ms,
+                          "recall_of_the_direct_join": float(np.isin(exact, got).mean()) if len(exact) else None,
+                          "false_pairs": int((~np.isin(got, exact)).sum()),
+                          "note": "value = 2*n*m*d of the ORIGINAL dimension over the pipeline's time: the brute-force-"
+                                  "equivalent rate of an approximate join, not the headline metric"}}
+    print(json.dumps(line), flush=True)
+
+
 def size_kw(args):
     kw = {}
     if args.n is not None:
@@ -271,7 +330,17 @@ def main():
     ap.add_argument("--jl", default=None, metavar="n,d,k",
                     help="time the JL transform (simjoin_jl_transform) of n bf16 points from d to k coordinates instead "
                          "of the join; HBM-bound, reported in algorithmic GB/s; not the headline metric")
+    ap.add_argument("--jl-join", default=None, metavar="n,d,k[,slack]",
+                    help="time the Euclidean join behind a JL pre-reduction (simjoin_run_jl_l2) beside the direct join; "
+                         "reports speedup and recall; not the headline metric")
     args = ap.parse_args()
+    if args.jl_join:
+        args.jl_join = args.jl_join.split(",")
+        if args.warmup < 3:
+            args.warmup = 3
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_jl_join(args)
+        return
     if args.jl:
         args.jl = tuple(int(x) for x in args.jl.split(","))
         if args.warmup < 3:
