@@ -650,6 +650,95 @@ simjoin_status hamming_unpack(simjoin_ctx *ctx, const void *P_bits, int64_t n, c
     return cudaGetLastError() == cudaSuccess ? SIMJOIN_OK : SIMJOIN_ERR_CUDA;
 }
 
+// The JL transform (Section 3) of n rows; row r of the result starts at out + r * out_ld (out_ld >= k, a multiple of 8).
+simjoin_status jl_device(simjoin_ctx *ctx, const void *X, int64_t n, int32_t d, int32_t k, uint64_t seed, void *out, int64_t out_ld) {
+    if (!ctx || !X || !out || n < 0 || d <= 0 || k <= 0) return SIMJOIN_ERR_ARG;
+    if (ctx->dtype != SIMJOIN_BF16) return SIMJOIN_ERR_UNSUPPORTED;
+    if (d % k != 0) return SIMJOIN_ERR_ARG;
+    int levels = 0;
+    for (int q = d / k; q > 1; q /= 2, ++levels)
+        if (q % 2 != 0) return SIMJOIN_ERR_ARG;                       // zeta = 2: d / k must be a power of two
+    if (levels < 1) return SIMJOIN_ERR_ARG;
+    if (k % 8 != 0) return SIMJOIN_ERR_UNSUPPORTED;                   // 16-byte rows at every level
+    const int c_max = levels == 1 ? 2 * k : 2 * (levels - 1) * k;     // widest block: the last level's
+    if ((size_t)c_max * 2 > SIMJOIN_MAX_ROW_BYTES || (size_t)d * 2 > SIMJOIN_MAX_ROW_BYTES) return SIMJOIN_ERR_UNSUPPORTED;
+    if (n * (int64_t)(d / (2 * k)) >= SIMJOIN_MAX_ROWS) return SIMJOIN_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(X) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) return SIMJOIN_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SIMJOIN_ERR_CUDA;
+    ctx->have_timing = false;
+    if (n == 0) return SIMJOIN_OK;
+    if (!is_device_ptr(X, ctx->device) || !is_device_ptr(out, ctx->device)) return SIMJOIN_ERR_ARG;
+    // ping-pong level outputs (at most d/2 coordinates per point) and the largest level matrix
+    size_t a_elems = 0, mid_elems = 0;
+    for (int i = 1; i <= levels; ++i) {
+        const size_t ki = i < levels ? (size_t)i * k : (size_t)k, ci = i == 1 ? (size_t)2 * k : (size_t)2 * (i - 1) * k;
+        const size_t ri = (size_t)1 << (levels - i);
+        if (ki * ci > a_elems) a_elems = ki * ci;
+        if (i < levels && ri * ki > mid_elems) mid_elems = ri * ki;
+    }
+    if (!grow(ctx->jl_a, a_elems * 2) || (levels > 1 && (!grow(ctx->jl_buf[0], (size_t)n * mid_elems * 2) ||
+                                                          (levels > 2 && !grow(ctx->jl_buf[1], (size_t)n * mid_elems * 2)))))
+        return SIMJOIN_ERR_CUDA;
+    cudaStream_t s = ctx->stream;
+    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    cudaEventRecord(ctx->ev[0], s);
+    cudaEventRecord(ctx->ev[1], s);
+    const void *src = X;
+    for (int i = 1; i <= levels; ++i) {
+        const int ki = i < levels ? i * k : k, ci = i == 1 ? 2 * k : 2 * (i - 1) * k;
+        const int64_t rows = n * ((int64_t)1 << (levels - i));        // n * r_i blocks of c_i coordinates
+        void *dst = i == levels ? out : ctx->jl_buf[(i - 1) & 1].ptr;
+        jl_sign_matrix_kernel<<<(unsigned)(((long long)ki * ci + 255) / 256), 256, 0, s>>>(seed, i, ki, ci,
+                                                                                         reinterpret_cast<uint16_t *>(ctx->jl_a.ptr));
+        if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        // the tile kernel with the level matrix as the resident operand and the blocks as the streamed one
+        JoinParams jp;
+        size_t smem = 0;
+        if (!tile_geometry(ctx, ki, rows, ci * 2, 2, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
+        // a level matrix of at most 128 rows and two chunks: 256 streamed rows per tile, 32 KiB ring stages
+        const bool wideq = ki <= TILE_M && jp.kc <= 2;
+        const int tn = wideq ? LONG_TN : TILE_N;
+        if (wideq) {
+            const int p_bytes = P_BUFS * jp.kc * A_CHUNK_BYTES;
+            int nstages = (ctx->max_smem_optin - 1024 - CTRL_BYTES - STAGING_BYTES - p_bytes) / LONG_Q_CHUNK_BYTES;
+            if (nstages > MAX_STAGES) nstages = MAX_STAGES;
+            jp.nstages = nstages;
+            jp.epi_release = nstages >= 2 * jp.kc ? 1 : 0;
+            smem = 1024 + (size_t)p_bytes + (size_t)nstages * LONG_Q_CHUNK_BYTES + STAGING_BYTES + CTRL_BYTES;
+        }
+        jp.PB = (ki + P_ROWS - 1) / P_ROWS;
+        jp.QT = (int)((rows + tn - 1) / tn);
+        jp.qpanel = jp.QT;                 // the blocks are read once: no L2 panels, one long sweep per CTA
+        jp.counter = ctx->d_ctrl;
+        jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
+        jp.store_out = reinterpret_cast<uint16_t *>(dst);
+        jp.store_ld = i == levels ? out_ld : ki;
+        jp.store_scale = (float)(1.0 / std::sqrt((double)ki));
+        CUtensorMap mapA, mapX;
+        if (!encode_rows_map(ctx, &mapA, ctx->jl_a.ptr, ki, ci, P_ROWS) || !encode_rows_map(ctx, &mapX, src, rows, ci, tn))
+            return SIMJOIN_ERR_CUDA;
+        const cudaError_t le = wideq ? launch_store_wideq(ctx, mapA, mapX, jp, ctx->num_sms, smem)
+                                     : launch_join<DT_BF16, KIND_STORE>(ctx, mapA, mapX, jp, ctx->num_sms, smem);
+        if (le != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        src = dst;
+    }
+    cudaEventRecord(ctx->ev[2], s);
+    if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
+    }
+    if ((unsigned int)(ctx->h_ctrl[1] & 0xffffffffu) != 0) return SIMJOIN_ERR_TIMEOUT;
+    float b = 0.f;
+    if (cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
+        ctx->prepass_ms = 0.f;
+        ctx->join_ms = b;          // all levels
+        ctx->have_timing = true;
+    }
+    return SIMJOIN_OK;
+}
+
 // Keep the listed pairs whose rows pass the predicate; the list is compacted in place (order unspecified).
 simjoin_status filter_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, simjoin_kind kind,
                              double threshold, int32_t *pairs, uint64_t count_in, uint64_t *count_out) {
@@ -947,91 +1036,7 @@ simjoin_status simjoin_run_hamming_lsh(simjoin_ctx *ctx, const void *P_bits, int
 }
 
 simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, int32_t d, int32_t k, uint64_t seed, void *out) {
-    if (!ctx || !X || !out || n < 0 || d <= 0 || k <= 0) return SIMJOIN_ERR_ARG;
-    if (ctx->dtype != SIMJOIN_BF16) return SIMJOIN_ERR_UNSUPPORTED;
-    if (d % k != 0) return SIMJOIN_ERR_ARG;
-    int levels = 0;
-    for (int q = d / k; q > 1; q /= 2, ++levels)
-        if (q % 2 != 0) return SIMJOIN_ERR_ARG;                       // zeta = 2: d / k must be a power of two
-    if (levels < 1) return SIMJOIN_ERR_ARG;
-    if (k % 8 != 0) return SIMJOIN_ERR_UNSUPPORTED;                   // 16-byte rows at every level
-    const int c_max = levels == 1 ? 2 * k : 2 * (levels - 1) * k;     // widest block: the last level's
-    if ((size_t)c_max * 2 > SIMJOIN_MAX_ROW_BYTES || (size_t)d * 2 > SIMJOIN_MAX_ROW_BYTES) return SIMJOIN_ERR_UNSUPPORTED;
-    if (n * (int64_t)(d / (2 * k)) >= SIMJOIN_MAX_ROWS) return SIMJOIN_ERR_ARG;
-    if ((reinterpret_cast<uintptr_t>(X) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) return SIMJOIN_ERR_UNSUPPORTED;
-    DeviceGuard guard(ctx->device);
-    if (!guard.ok) return SIMJOIN_ERR_CUDA;
-    ctx->have_timing = false;
-    if (n == 0) return SIMJOIN_OK;
-    if (!is_device_ptr(X, ctx->device) || !is_device_ptr(out, ctx->device)) return SIMJOIN_ERR_ARG;
-    // ping-pong level outputs (at most d/2 coordinates per point) and the largest level matrix
-    size_t a_elems = 0, mid_elems = 0;
-    for (int i = 1; i <= levels; ++i) {
-        const size_t ki = i < levels ? (size_t)i * k : (size_t)k, ci = i == 1 ? (size_t)2 * k : (size_t)2 * (i - 1) * k;
-        const size_t ri = (size_t)1 << (levels - i);
-        if (ki * ci > a_elems) a_elems = ki * ci;
-        if (i < levels && ri * ki > mid_elems) mid_elems = ri * ki;
-    }
-    if (!grow(ctx->jl_a, a_elems * 2) || (levels > 1 && (!grow(ctx->jl_buf[0], (size_t)n * mid_elems * 2) ||
-                                                          (levels > 2 && !grow(ctx->jl_buf[1], (size_t)n * mid_elems * 2)))))
-        return SIMJOIN_ERR_CUDA;
-    cudaStream_t s = ctx->stream;
-    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    cudaEventRecord(ctx->ev[0], s);
-    cudaEventRecord(ctx->ev[1], s);
-    const void *src = X;
-    for (int i = 1; i <= levels; ++i) {
-        const int ki = i < levels ? i * k : k, ci = i == 1 ? 2 * k : 2 * (i - 1) * k;
-        const int64_t rows = n * ((int64_t)1 << (levels - i));        // n * r_i blocks of c_i coordinates
-        void *dst = i == levels ? out : ctx->jl_buf[(i - 1) & 1].ptr;
-        jl_sign_matrix_kernel<<<(unsigned)(((long long)ki * ci + 255) / 256), 256, 0, s>>>(seed, i, ki, ci,
-                                                                                         reinterpret_cast<uint16_t *>(ctx->jl_a.ptr));
-        if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
-        // the tile kernel with the level matrix as the resident operand and the blocks as the streamed one
-        JoinParams jp;
-        size_t smem = 0;
-        if (!tile_geometry(ctx, ki, rows, ci * 2, 2, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
-        // a level matrix of at most 128 rows and two chunks: 256 streamed rows per tile, 32 KiB ring stages
-        const bool wideq = ki <= TILE_M && jp.kc <= 2;
-        const int tn = wideq ? LONG_TN : TILE_N;
-        if (wideq) {
-            const int p_bytes = P_BUFS * jp.kc * A_CHUNK_BYTES;
-            int nstages = (ctx->max_smem_optin - 1024 - CTRL_BYTES - STAGING_BYTES - p_bytes) / LONG_Q_CHUNK_BYTES;
-            if (nstages > MAX_STAGES) nstages = MAX_STAGES;
-            jp.nstages = nstages;
-            jp.epi_release = nstages >= 2 * jp.kc ? 1 : 0;
-            smem = 1024 + (size_t)p_bytes + (size_t)nstages * LONG_Q_CHUNK_BYTES + STAGING_BYTES + CTRL_BYTES;
-        }
-        jp.PB = (ki + P_ROWS - 1) / P_ROWS;
-        jp.QT = (int)((rows + tn - 1) / tn);
-        jp.qpanel = jp.QT;                 // the blocks are read once: no L2 panels, one long sweep per CTA
-        jp.counter = ctx->d_ctrl;
-        jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
-        jp.store_out = reinterpret_cast<uint16_t *>(dst);
-        jp.store_ld = ki;
-        jp.store_scale = (float)(1.0 / std::sqrt((double)ki));
-        CUtensorMap mapA, mapX;
-        if (!encode_rows_map(ctx, &mapA, ctx->jl_a.ptr, ki, ci, P_ROWS) || !encode_rows_map(ctx, &mapX, src, rows, ci, tn))
-            return SIMJOIN_ERR_CUDA;
-        const cudaError_t le = wideq ? launch_store_wideq(ctx, mapA, mapX, jp, ctx->num_sms, smem)
-                                     : launch_join<DT_BF16, KIND_STORE>(ctx, mapA, mapX, jp, ctx->num_sms, smem);
-        if (le != cudaSuccess) return SIMJOIN_ERR_CUDA;
-        src = dst;
-    }
-    cudaEventRecord(ctx->ev[2], s);
-    if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) {
-        cudaGetLastError();
-        return SIMJOIN_ERR_CUDA;
-    }
-    if ((unsigned int)(ctx->h_ctrl[1] & 0xffffffffu) != 0) return SIMJOIN_ERR_TIMEOUT;
-    float b = 0.f;
-    if (cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
-        ctx->prepass_ms = 0.f;
-        ctx->join_ms = b;          // all levels
-        ctx->have_timing = true;
-    }
-    return SIMJOIN_OK;
+    return jl_device(ctx, X, n, d, k, seed, out, k);
 }
 
 simjoin_status simjoin_filter_pairs(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
@@ -1063,12 +1068,17 @@ simjoin_status simjoin_run_jl_l2(simjoin_ctx *ctx, const void *P, int64_t n, con
     if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
     *count = 0;
     if (n == 0 || m == 0) return simjoin_jl_transform(ctx, P, 0, d, k, seed, const_cast<void *>(P));   // shape rules only
-    if (!grow(ctx->jl_p, (size_t)n * k * 2 + 16) || !grow(ctx->jl_q, (size_t)m * k * 2 + 16)) return SIMJOIN_ERR_CUDA;
+    // The reduced points are joined as they are, by the Euclidean kind.  Section 4's squared-L2 embedding -- 8 appended
+    // coordinates (x, -|x|^2/2, 1) . (y, 1, -|y|^2/2) = -|x - y|^2 / 2, an inner-product join with a constant threshold
+    // and an exact row-maximum filter -- was measured and dropped: the 16 extra bytes per row open a second (third)
+    // chunk with a short tail, and the reduced join took 15.9 ms instead of 11.8 (k = 128; 3.35 against 3.2-3.3 at k = 64).
+    if (!grow(ctx->jl_p, (size_t)n * k * 2) || !grow(ctx->jl_q, (size_t)m * k * 2)) return SIMJOIN_ERR_CUDA;
+    cudaStream_t s = ctx->stream;
     // the same M for both sets: |M x - M y| = |M (x - y)| is within a factor 1 +- eps of |x - y|
-    st = simjoin_jl_transform(ctx, P, n, d, k, seed, ctx->jl_p.ptr);
+    st = jl_device(ctx, P, n, d, k, seed, ctx->jl_p.ptr, k);
     if (st != SIMJOIN_OK) return st;
     float jl_ms = ctx->have_timing ? ctx->join_ms : 0.f;
-    st = simjoin_jl_transform(ctx, Q, m, d, k, seed, ctx->jl_q.ptr);
+    st = jl_device(ctx, Q, m, d, k, seed, ctx->jl_q.ptr, k);
     if (st != SIMJOIN_OK) return st;
     jl_ms += ctx->have_timing ? ctx->join_ms : 0.f;
     // candidates: the join of the reduced points with the radius widened by the slack
@@ -1080,7 +1090,6 @@ simjoin_status simjoin_run_jl_l2(simjoin_ctx *ctx, const void *P, int64_t n, con
         return st;
     }
     if (st != SIMJOIN_OK) return st;
-    cudaStream_t s = ctx->stream;
     cudaEventRecord(ctx->ev[0], s);
     st = filter_device(ctx, P, n, Q, m, d, SIMJOIN_L2, r, out_pairs, cand, count);
     cudaEventRecord(ctx->ev[1], s);
