@@ -847,17 +847,22 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 // per-column terms of this warp's columns, 4 per lane, fetched while the tile is still
                 // being multiplied so that the exact test never waits on global memory (fetching them only when a
                 // candidate shows up was measured: no gain for sparse joins, 5 % slower dense ones)
+                // int8 kinds fetch them only when a candidate shows up: measured -1.6 % (cosine) and -2.6 % (Euclidean) on a
+                // sparse 262 144^2 join, +0.5-1 % on a dense one (the adaptive form -- prefetch while the previous tile
+                // had candidates -- lost on both)
+                constexpr bool LAZY_COLTERMS = DT == DT_I8;
+                auto load_colterms = [&](int ps) -> uint4 {
+                    const uint32_t *nyp = reinterpret_cast<const uint32_t *>(p.ny) + (q_base + (long long)qt * TN + ps * EPI_COLS) + 4 * lane;
+                    if constexpr (GROUPED)          // a bucket starts at any row: no 16-byte alignment
+                        return make_uint4(__ldg(nyp), __ldg(nyp + 1), __ldg(nyp + 2), __ldg(nyp + 3));
+                    else
+                        return __ldg(reinterpret_cast<const uint4 *>(nyp));
+                };
                 uint4 yq_pass[NPASS];
 #pragma unroll
                 for (int ps = 0; ps < NPASS; ++ps) {
                     yq_pass[ps] = make_uint4(0, 0, 0, 0);
-                    if ((KIND == KIND_COS || KIND == KIND_L2) && lane < EPI_COLS / 4) {
-                        const uint32_t *nyp = reinterpret_cast<const uint32_t *>(p.ny) + (q_base + (long long)qt * TN + ps * EPI_COLS) + 4 * lane;
-                        if constexpr (GROUPED)      // a bucket starts at any row: no 16-byte alignment
-                            yq_pass[ps] = make_uint4(__ldg(nyp), __ldg(nyp + 1), __ldg(nyp + 2), __ldg(nyp + 3));
-                        else
-                            yq_pass[ps] = __ldg(reinterpret_cast<const uint4 *>(nyp));
-                    }
+                    if constexpr ((KIND == KIND_COS || KIND == KIND_L2) && !LAZY_COLTERMS) yq_pass[ps] = load_colterms(ps);
                 }
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
                 if (!ok) break;
@@ -910,7 +915,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 constexpr int MODE = DT == DT_BF16 ? MAX_F32 : (NARROW ? MAX_S16X2 : MAX_S32);
 #pragma unroll
                 for (int ps = 0; ps < NPASS; ++ps) {
-                const uint4 yq = yq_pass[ps];
+                uint4 yq = yq_pass[ps];
                 uint32_t v[NV];
                 tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TN + ps * EPI_COLS, v,
                               std::integral_constant<bool, NARROW>{});
@@ -956,6 +961,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     if constexpr (KIND != KIND_IP) {
                         // the per-column terms go through shared memory: level 2 reads 16 of them per group as four
                         // broadcast loads (a shuffle per term cost four times the instructions)
+                        if constexpr (LAZY_COLTERMS) yq = load_colterms(ps);
                         __syncwarp();
                         reinterpret_cast<uint4 *>(colterm)[lane] = yq;
                         __syncwarp();
