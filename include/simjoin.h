@@ -240,7 +240,8 @@ simjoin_status simjoin_filter_pairs(simjoin_ctx *ctx, const void *P, int64_t n, 
 /*
  * Euclidean join behind a JL pre-reduction (Section 3's transform used as the paper introduces it: reduce the
  * dimension, then search): both point sets are reduced from d to k coordinates with the same matrix M
- * (simjoin_jl_transform, same seed), the reduced points are joined with the radius widened to r * (1 + slack),
+ * (simjoin_jl_transform, same seed), the reduced points are joined with the radius widened to r * (1 + slack)
+ * (the reduced rows of Q ordered by norm first, which keeps the join's per-block bounds tight),
  * and the candidates are decided on the original rows (simjoin_filter_pairs, radius r).  The result is a subset
  * of the exact join { (i, j) : |x_i - y_j| <= r } (band rule of simjoin_filter_pairs): a true pair is missed only
  * when M stretches its distance by more than 1 + slack.  With random-sign levels the relative spread of |M z| / |z|

@@ -8,6 +8,8 @@
 #pragma once
 #include <cstdint>
 
+#include "lsh_kernel.cuh"   // block_scan4 and the counting-sort kernels
+
 namespace sj {
 
 constexpr int FILTER_THREADS = 256;
@@ -97,6 +99,60 @@ filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__res
         }
         if (lane == 0 && pass) out[atomicAdd(counter, 1ULL)] = pr;
     }
+}
+
+// ---- ordering rows by norm (the reduced join of simjoin_run_jl_l2) ----
+// The tile epilogue prunes with a bound built from the smallest |y|^2 of a 256-row block of Q.  Reduced rows have
+// norms that spread by +-1/sqrt(k/2) around the original ones, which loosens that bound; with the rows of Q ordered
+// by norm every block is nearly constant.  A counting sort on a 12-bit quantisation of the norm is enough.
+
+// range[0] = min, range[1] = max of the (non-negative) norms, as float bits (whose integer order is the floats').
+__global__ void __launch_bounds__(256) norm_range_kernel(const float *__restrict__ ny, long long m, unsigned int *range) {
+    unsigned int mn = 0x7f7f7f7fu, mx = 0u;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (long long)gridDim.x * blockDim.x) {
+        const unsigned int b = __float_as_uint(ny[i]);
+        mn = min(mn, b);
+        mx = max(mx, b);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, off));
+        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicMin(range, mn);
+        atomicMax(range + 1, mx);
+    }
+}
+
+// key[i] in [0, nb): the position of ny[i] between the smallest and the largest norm.
+__global__ void __launch_bounds__(256) norm_keys_kernel(const float *__restrict__ ny, long long m, const unsigned int *__restrict__ range,
+                                                        int nb, uint16_t *__restrict__ keys) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= m) return;
+    const float lo = __uint_as_float(range[0]), hi = __uint_as_float(range[1]);
+    const float span = hi - lo;
+    int key = span > 0.f ? (int)((ny[i] - lo) / span * (float)nb) : 0;
+    keys[i] = (uint16_t)min(max(key, 0), nb - 1);
+}
+
+// cursor[b] = number of rows with a key below b (one block; nb <= 4096).
+__global__ void __launch_bounds__(1024) hist_offsets_kernel(const unsigned int *__restrict__ hist, int nb, unsigned int *__restrict__ cursor) {
+    __shared__ unsigned int s_warp[33];
+    unsigned int v[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) v[t] = threadIdx.x * 4 + t < nb ? hist[threadIdx.x * 4 + t] : 0u;
+    block_scan4(v, s_warp);
+#pragma unroll
+    for (int t = 0; t < 4; ++t)
+        if (threadIdx.x * 4 + t < nb) cursor[threadIdx.x * 4 + t] = v[t];
+}
+
+// pairs[t].y: position in the ordered copy (+ joff) -> original row (+ joff).
+__global__ void __launch_bounds__(256) remap_second_index_kernel(int2 *__restrict__ pairs, unsigned long long count,
+                                                                 const int *__restrict__ perm, int joff) {
+    const unsigned long long t = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < count) pairs[t].y = perm[pairs[t].y - joff] + joff;
 }
 
 }  // namespace sj

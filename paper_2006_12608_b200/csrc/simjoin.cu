@@ -1081,9 +1081,37 @@ simjoin_status simjoin_run_jl_l2(simjoin_ctx *ctx, const void *P, int64_t n, con
     st = jl_device(ctx, Q, m, d, k, seed, ctx->jl_q.ptr, k);
     if (st != SIMJOIN_OK) return st;
     jl_ms += ctx->have_timing ? ctx->join_ms : 0.f;
+    // Order the reduced rows of Q by norm (counting sort on 12 bits of the norm): the join's per-tile bound is built
+    // from the smallest |y|^2 of each 256-row block, and the reduced norms spread (measured at k = 64: the join of
+    // the unordered rows 2.46 ms, 7 % of the warp blocks entering the exact test for nothing).
+    const int nb = LSH_MAX_BUCKETS;
+    const int g = k * 2 / 16;
+    if (!grow(ctx->nx, (size_t)m * 4) || !grow(ctx->lsh_keys_q, (size_t)m * 2) || !grow(ctx->lsh_perm_q, (size_t)m * 4) ||
+        !grow(ctx->lsh_misc, (size_t)2 * nb * 4 + 16) || !grow(ctx->lsh_sorted_q, (size_t)m * k * 2))
+        return SIMJOIN_ERR_CUDA;
+    {
+        float *ny = reinterpret_cast<float *>(ctx->nx.ptr);
+        uint16_t *keys = reinterpret_cast<uint16_t *>(ctx->lsh_keys_q.ptr);
+        int *perm = reinterpret_cast<int *>(ctx->lsh_perm_q.ptr);
+        unsigned int *hist = reinterpret_cast<unsigned int *>(ctx->lsh_misc.ptr), *cursor = hist + nb, *range = cursor + nb;
+        // running minimum starts at 0x7f7f7f7f (3.4e38, above every norm), running maximum at 0
+        if (launch_norms<false>(ctx, ctx->jl_q.ptr, m, k, 0, ny, nullptr) != cudaSuccess ||
+            cudaMemsetAsync(hist, 0, (size_t)nb * 4, s) != cudaSuccess ||
+            cudaMemsetAsync(range, 0x7f, 4, s) != cudaSuccess || cudaMemsetAsync(range + 1, 0, 4, s) != cudaSuccess)
+            return SIMJOIN_ERR_CUDA;
+        const int rows_per_block = LSH_SORT_THREADS * LSH_SORT_ITEMS;
+        norm_range_kernel<<<ctx->num_sms * 4, 256, 0, s>>>(ny, m, range);
+        norm_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(ny, m, range, nb, keys);
+        lsh_hist_kernel<<<(unsigned)ctx->num_sms * 4, LSH_SORT_THREADS, 0, s>>>(keys, 1, m, nb, hist);
+        hist_offsets_kernel<<<1, 1024, 0, s>>>(hist, nb, cursor);
+        lsh_scatter_kernel<<<(unsigned)((m + rows_per_block - 1) / rows_per_block), LSH_SORT_THREADS, 0, s>>>(keys, 1, m, nb, cursor, perm);
+        lsh_gather_rows_kernel<<<(unsigned)(((long long)m * g + 255) / 256), 256, 0, s>>>(
+            reinterpret_cast<const uint4 *>(ctx->jl_q.ptr), perm, m, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_q.ptr));
+        if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    }
     // candidates: the join of the reduced points with the radius widened by the slack
     uint64_t cand = 0;
-    st = run_device(ctx, ctx->jl_p.ptr, n, ctx->jl_q.ptr, m, k, SIMJOIN_L2, r * (1.0 + slack), out_pairs, capacity, &cand);
+    st = run_device(ctx, ctx->jl_p.ptr, n, ctx->lsh_sorted_q.ptr, m, k, SIMJOIN_L2, r * (1.0 + slack), out_pairs, capacity, &cand);
     const float join_ms = ctx->have_timing ? ctx->prepass_ms + ctx->join_ms : 0.f;
     if (st == SIMJOIN_ERR_CAPACITY) {
         *count = cand;                  // more candidates than room: nothing can be decided
@@ -1091,6 +1119,11 @@ simjoin_status simjoin_run_jl_l2(simjoin_ctx *ctx, const void *P, int64_t n, con
     }
     if (st != SIMJOIN_OK) return st;
     cudaEventRecord(ctx->ev[0], s);
+    if (cand > 0) {
+        remap_second_index_kernel<<<(unsigned)((cand + 255) / 256), 256, 0, s>>>(reinterpret_cast<int2 *>(out_pairs), cand,
+                                                                               reinterpret_cast<const int *>(ctx->lsh_perm_q.ptr), (int)ctx->joff);
+        if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    }
     st = filter_device(ctx, P, n, Q, m, d, SIMJOIN_L2, r, out_pairs, cand, count);
     cudaEventRecord(ctx->ev[1], s);
     float f_ms = 0.f;
