@@ -1,6 +1,6 @@
 """Randomised parity: a few hundred seeded cases over element type, kind, brute force / LSH, row length (all three tile
 geometries, partial chunks), ragged row counts and value ranges, each compared with the oracle (int8: the exact pair set;
-bf16: inside the threshold band).  Thresholds are taken from a sample of the oracle's scores so that every case has
+bf16: inside the threshold band); half of the cases also run the pair filter on a random candidate list.  Thresholds are taken from a sample of the oracle's scores so that every case has
 hits.  One ill-conditioned corner is left out on purpose: a bf16 Euclidean radius far below the rows' norms, where
 |x|^2 + |y|^2 - 2<x,y> cancels in fp32 beyond what a band relative to r can absorb."""
 import numpy as np
@@ -76,6 +76,21 @@ def test_random_cases_match_the_oracle(seed):
             else:
                 sets = O.lsh_band_sets(P, Q, kind, t, dtype, L, k, s1, L_low=L_low) if lsh else O.band_sets(P, Q, kind, t, dtype)
                 assert np.isin(keys(sets[0]), got).all() and np.isin(got, keys(sets[2])).all(), what
+            # the pair filter on a random candidate list of the same points (plus some reported pairs)
+            if rng.random() < 0.5:
+                nc = int(rng.integers(1, 2000))
+                cand = np.stack([rng.integers(0, n, nc), rng.integers(0, m, nc)], axis=1).astype(np.int32)
+                cand = np.concatenate([cand, host[:min(cnt, 300)]])
+                lst = torch.from_numpy(np.ascontiguousarray(cand)).cuda()
+                st2, kc = ctx.simjoin_filter_pairs(dP, n, dQ, m, d, kind, t, lst, len(cand))
+                assert st2 == B.SIMJOIN_OK, (B.strerror(st2), what)
+                kept = keys(lst[:kc].cpu().numpy())
+                if dtype == "i8":
+                    assert np.array_equal(kept, keys(O.filter_pairs(P, Q, kind, t, dtype, cand))), what
+                else:
+                    t_loose, t_strict = (t * 1.01, t * 0.99) if kind == "l2" else (t - 0.01 * abs(t), t + 0.01 * abs(t))
+                    assert np.isin(keys(O.filter_pairs(P, Q, kind, t_strict, dtype, cand)), kept).all(), what
+                    assert np.isin(kept, keys(O.filter_pairs(P, Q, kind, t_loose, dtype, cand))).all(), what
     finally:
         for c in ctxs.values():
             c.close()
