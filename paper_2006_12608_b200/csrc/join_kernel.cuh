@@ -793,13 +793,17 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             const long long q_end = GROUPED ? (long long)un.qrow0 + un.qrows : p.m;   // end of the Q rows of this unit
             int ri = 0;          // I8/L2: |x|^2 - floor(r^2)
             float rf = 0.f;      // COS: t*|x|;  BF16/L2: (|x|^2 - r^2) / 2
-            bool rzero = false;  // COS: x is the zero vector
             if (row_ok) {
                 if constexpr (DT == DT_I8 && KIND == KIND_L2) ri = reinterpret_cast<const int *>(p.nx)[i] - p.thr_i;
                 if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
-                    const float nxr = reinterpret_cast<const float *>(p.nx)[i];
-                    rf = p.thr_f * nxr;
-                    rzero = nxr == 0.f;
+                    // s >= (t |x|) |y|, read off the sign of s - b like the other bf16 kinds.  The cosine with a zero
+                    // vector counts as 0 (passes iff t <= 0), and the stored norms make the products say so:
+                    //   t > 0: the pre-pass stores +inf for a zero vector, so b = +inf and nothing passes (a row
+                    //          term that underflows to 0 becomes the smallest denormal: 0 * inf would be NaN);
+                    //   t <= 0 (a zero t is passed as -0): b = -0 whenever a zero vector is involved, and
+                    //          s - (-0) = +0 for a score of either zero.
+                    rf = p.thr_f * reinterpret_cast<const float *>(p.nx)[i];
+                    if (p.thr_f > 0.f && rf == 0.f) rf = 1.401298464e-45f;
                 }
                 if constexpr (DT == DT_I8 && KIND == KIND_COS) {
                     // fp32 filter for s >= t |x| |y|, lowered by 2^-18 relative (the fp32 roundings of t, the two norms,
@@ -982,7 +986,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             }
                         }
                         uint32_t mk = 0;
-                        if constexpr (DT == DT_BF16 && (KIND == KIND_L2 || KIND == KIND_IP)) {
+                        if constexpr (DT == DT_BF16) {
                             // The same decision as bound_ok, taken from a sign bit: fl(s - b) >= +0 exactly when
                             // s >= b.  The adds run on the FMA pipe and one funnel shift collects the bit, where a
                             // compare, a select and an OR would all queue on the half-rate ALU pipe (dense outputs).
@@ -993,7 +997,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             for (int q = 0; q < NCH; ++q) fail[q] = 0;
 #pragma unroll
                             for (int c = 0; c < GCOLS; ++c) {
-                                const float b = KIND == KIND_IP ? p.thr_f : rf + 0.5f * __uint_as_float(yw[c]);
+                                const float b = KIND == KIND_IP    ? p.thr_f
+                                                : KIND == KIND_COS ? __fmul_rn(rf, __uint_as_float(yw[c]))   // as level 0 rounds it
+                                                                   : rf + 0.5f * __uint_as_float(yw[c]);
                                 fail[c >> 2] = __funnelshift_l(__float_as_uint(__uint_as_float(v[k * GCOLS + c]) - b), fail[c >> 2], 1);
                             }
                             // chain q holds columns 4q .. 4q+3 at bits 3 .. 0
@@ -1014,12 +1020,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             bool pass = false;
                             if constexpr (DT == DT_I8 && KIND == KIND_IP) pass = (int)x >= p.thr_i;
                             if constexpr (DT == DT_I8 && KIND == KIND_L2) pass = 2 * (int)x - (int)yw[c] >= ri;
-                            if constexpr (DT == DT_BF16 && KIND == KIND_IP) pass = __uint_as_float(x) >= p.thr_f;
                             if constexpr (DT == DT_I8 && KIND == KIND_COS) pass = (float)(int)x >= rf * __uint_as_float(yw[c]);
-                            if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
-                                const float nyr = __uint_as_float(yw[c]);
-                                pass = (rzero || nyr == 0.f) ? (p.thr_f <= 0.f) : (__uint_as_float(x) >= rf * nyr);
-                            }
                             mk |= (pass ? 1u : 0u) << c;
                         }
                         }

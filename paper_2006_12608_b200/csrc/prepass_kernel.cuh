@@ -68,8 +68,8 @@ __device__ __forceinline__ void warp_rows_pow2(const uint4 *__restrict__ X, long
 }
 
 // X: rows x (g * 16 bytes).  norms[r] = sum of squares of row r; with sqrt_out its square root in fp32 (int8
-// rows too: the bits of the float in the int32 array, whose order is the floats' order; sqrt_out == 2 stores
-// +inf for a zero row).  tile_minmax[b] = (min, max) of norms over the valid rows of tile b (may be null).
+// rows too: the bits of the float in the int32 array, whose order is the floats' order); sqrt_out == 2 stores
+// +inf for a zero row.  tile_minmax[b] = (min, max) of norms over the valid rows of tile b (may be null).
 template <bool kInt8>
 __global__ void __launch_bounds__(NORM_THREADS)
 row_norms_kernel(const uint4 *__restrict__ X, long long rows, int g, int sqrt_out,
@@ -104,7 +104,9 @@ row_norms_kernel(const uint4 *__restrict__ X, long long rows, int g, int sqrt_ou
     __syncthreads();
     const long long r = (long long)blockIdx.x * NORM_TILE_ROWS + threadIdx.x;
     T v = s_val[threadIdx.x];
-    if constexpr (!kInt8) { if (sqrt_out) v = sqrtf(v); }
+    if constexpr (!kInt8) {
+        if (sqrt_out) v = (v == 0.f && sqrt_out == 2) ? __int_as_float(0x7f800000) : sqrtf(v);
+    }
     if constexpr (kInt8) {
         if (sqrt_out) v = __float_as_int(v == 0 && sqrt_out == 2 ? __int_as_float(0x7f800000) : sqrtf((float)v));
     }

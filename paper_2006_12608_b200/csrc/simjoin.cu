@@ -266,16 +266,16 @@ void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold
         }
     } else {
         jp.thr_f = kind == SIMJOIN_L2 ? (float)(threshold * threshold) : (float)threshold;
-        // the inner-product test reads the sign of s - t: with t = -0 a score of either zero gives +0 and passes
-        if (kind == SIMJOIN_IP && jp.thr_f == 0.f) jp.thr_f = -0.0f;
+        // the inner-product and cosine tests read the sign of s - b: with t = -0 a score of either zero gives +0 and passes
+        if (kind != SIMJOIN_L2 && jp.thr_f == 0.f) jp.thr_f = -0.0f;
     }
 }
 
 // What the norm pre-pass stores per row.  0: |x|^2; 1: |x| in fp32 (cosine); 2: the same with +inf for a zero
-// vector -- int8 cosine with t > 0, where a zero vector passes nothing and must not raise candidates.
-int norm_mode(bool i8, simjoin_kind kind, double threshold) {
+// vector -- cosine with t > 0, where a zero vector passes nothing: the epilogue's products t |x| |y| are then +inf.
+int norm_mode(bool /*i8*/, simjoin_kind kind, double threshold) {
     if (kind != SIMJOIN_COS) return 0;
-    return i8 && threshold > 0 ? 2 : 1;
+    return (float)threshold > 0.f ? 2 : 1;        // decided on the fp32 threshold the epilogue uses
 }
 
 // The join on device buffers.  Arguments were validated by the caller.

@@ -152,6 +152,26 @@ def test_bf16_inner_product_threshold_zero_counts_scores_of_either_zero(ctx_bf16
         assert set(map(tuple, pairs.tolist())) == set(map(tuple, want.tolist()))
 
 
+def test_bf16_cosine_zero_vectors_and_scores_of_either_zero(ctx_bf16):
+    """Cosine with a zero vector counts as 0: it passes t <= 0 and fails t > 0, also when the accumulator holds -0
+    (a zero row against rows of negative values) and next to rows and columns that do pass."""
+    rng = np.random.default_rng(6)
+    P = W.random_points("bf16", 70, 64, 91)
+    Q = W.f32_to_bf16_bits(-np.abs(rng.standard_normal((90, 64))).astype(np.float32) - 0.25)      # all negative
+    P[::7] = 0
+    Q[5] = 0
+    Q[40:44] = 0
+    Q[60] = P[3]
+    for t in (0.0, -0.0, -0.3, 1e-3, 0.4, 1e-42):
+        pairs, cnt = gpu_join(ctx_bf16, P, Q, "cos", t)
+        want, wcnt = O.join(P, Q, "cos", t, "bf16")
+        zero = lambda s: {(i, j) for (i, j) in s if i % 7 == 0 or j in (5, 40, 41, 42, 43)}
+        got = set(map(tuple, pairs.tolist()))
+        assert zero(got) == zero(set(map(tuple, want.tolist()))), t
+        if t not in (0.0, -0.0, 1e-42):
+            assert_band(pairs, cnt, P, Q, "cos", t)
+
+
 def test_i8_packed_16_bit_epilogue_boundary(ctx_i8):
     """int8 scores that provably fit in 16 bits take a packed epilogue; check both sides of that
     decision and scores at the very ends of the 16-bit range."""
