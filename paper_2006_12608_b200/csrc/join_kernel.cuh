@@ -917,15 +917,30 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 constexpr int GCOLS = 16, NG = EPI_COLS / GCOLS, GW = NV / NG;  // column groups of level 1
                 constexpr uint32_t GMASK = (1u << GCOLS) - 1u;
                 constexpr int MODE = DT == DT_BF16 ? MAX_F32 : (NARROW ? MAX_S16X2 : MAX_S32);
+                // Long rows with the packed epilogue: both passes' words fit in registers (2 x 64), so the single
+                // accumulator goes back to the MMA warp before any test runs instead of after the first pass's.
+                constexpr bool LOAD_ALL = LONGK && NARROW;
+                uint32_t vall[LOAD_ALL ? NPASS : 1][NV];
+                if constexpr (LOAD_ALL) {
+#pragma unroll
+                    for (int ps = 0; ps < NPASS; ++ps)
+                        tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TN + ps * EPI_COLS, vall[ps],
+                                      std::integral_constant<bool, NARROW>{});
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                }
 #pragma unroll
                 for (int ps = 0; ps < NPASS; ++ps) {
                 uint4 yq = yq_pass[ps];
-                uint32_t v[NV];
-                tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TN + ps * EPI_COLS, v,
-                              std::integral_constant<bool, NARROW>{});
-                tc_fence_before();
-                __syncwarp();
-                if (ps == NPASS - 1 && lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                uint32_t (&v)[NV] = vall[LOAD_ALL ? ps : 0];
+                if constexpr (!LOAD_ALL) {
+                    tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TN + ps * EPI_COLS, v,
+                                  std::integral_constant<bool, NARROW>{});
+                    tc_fence_before();
+                    __syncwarp();
+                    if (ps == NPASS - 1 && lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                }
                 // level 0: the row maximum over this warp's 128 columns against the per-tile bound
                 // (a necessary condition of the exact test, in the same arithmetic)
                 auto bound_ok = [&](uint32_t word) -> bool {
