@@ -231,7 +231,7 @@ simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t
  * Arithmetic: I8 exact (the decisions simjoin_run takes); BF16 in fp32 -- inner product and cosine as sums over
  * the row, the Euclidean distance in the difference form sum (x - y)^2 <= r^2 (no cancellation of large norms);
  * a pair whose exact score lies within 1e-2*|threshold| of the threshold may fall on either side.
- * One warp per pair, two rows read per pair.  Synchronises the stream.  Scratch: count_in x 8 bytes.
+ * A group of lanes per pair (sized to the row), two rows read per pair.  Synchronises the stream.  Scratch: count_in x 8 bytes.
  */
 simjoin_status simjoin_filter_pairs(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
                                     simjoin_kind kind, double threshold, int32_t *pairs, uint64_t count_in,

@@ -2,9 +2,10 @@
 // (Section 4's definition, applied to listed pairs instead of all of P x Q).  It closes the approximate pipeline
 // "reduce with the JL transform of Section 3, join the short rows with some slack, decide the candidates on the
 // original rows": whatever distortion the reduction adds, only true pairs leave.
-// One warp per pair: the lanes stride over the 16-byte groups of the two rows, three running sums are reduced with
-// shuffles, lane 0 decides and appends the pair to the output list (one atomic per kept pair; order unspecified).
-// HBM/L2-bound: 2 rows per candidate.  A listed index outside the point sets raises a status bit and is skipped.
+// A group of G lanes per pair (G = the power of two covering the row's 16-byte words, at most 32: a warp takes
+// 32 / G pairs at a time, so that short rows keep all lanes loading): the lanes stride over the words of the two rows,
+// three running sums are reduced with shuffles inside the group, its first lane decides and appends the pair to the
+// output list (one atomic per kept pair; order unspecified).  HBM/L2-bound: 2 rows per candidate.  A listed index outside the point sets raises a status bit and is skipped.
 #pragma once
 #include <cstdint>
 
@@ -23,22 +24,29 @@ __global__ void __launch_bounds__(FILTER_THREADS)
 filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__restrict__ Q, long long m, int g,
                     const int2 *__restrict__ in, unsigned long long count_in, int ioff, int joff, int thr_i, float thr_f,
                     double thr_d, int2 *__restrict__ out, unsigned long long *__restrict__ counter,
-                    unsigned int *__restrict__ status) {
-    const int lane = threadIdx.x & 31;
+                    unsigned int *__restrict__ status, int G) {
+    const int wlane = threadIdx.x & 31;
+    const int lane = wlane & (G - 1), sub = wlane / G, ppw = 32 / G;      // lane within the pair's group; pairs per warp
     const unsigned long long warp = ((unsigned long long)blockIdx.x * FILTER_THREADS + threadIdx.x) >> 5;
     const unsigned long long nwarps = ((unsigned long long)gridDim.x * FILTER_THREADS) >> 5;
-    for (unsigned long long k = warp; k < count_in; k += nwarps) {
-        const int2 pr = in[k];
-        const long long li = (long long)pr.x - ioff, lj = (long long)pr.y - joff;
-        if (li < 0 || li >= n || lj < 0 || lj >= m) {      // not a pair of these point sets: flag it, touch nothing
-            if (lane == 0) atomicOr(status, 0x20000000u);
-            continue;
+    for (unsigned long long k0 = warp * ppw; k0 < count_in; k0 += nwarps * ppw) {      // warp-uniform trip count
+        const unsigned long long k = k0 + sub;
+        int2 pr = make_int2(0, 0);
+        bool live = k < count_in;
+        if (live) {
+            pr = in[k];
+            const long long li = (long long)pr.x - ioff, lj = (long long)pr.y - joff;
+            if (li < 0 || li >= n || lj < 0 || lj >= m) {  // not a pair of these point sets: flag it, touch nothing
+                if (lane == 0) atomicOr(status, 0x20000000u);
+                live = false;
+            }
         }
-        const uint4 *x = P + li * g, *y = Q + lj * g;
+        const uint4 *x = P + (live ? (long long)pr.x - ioff : 0) * g, *y = Q + (live ? (long long)pr.y - joff : 0) * g;
+        const int gl = live ? g : 0;                       // a dead group loads nothing but keeps shuffling
         bool pass = false;
         if constexpr (DT == DT_I8) {
             int s = 0, nx = 0, ny = 0;
-            for (int c = lane; c < g; c += 32) {
+            for (int c = lane; c < gl; c += G) {
                 const uint4 a = __ldg(x + c), b = __ldg(y + c);
                 const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
@@ -48,8 +56,7 @@ filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__res
                     ny = __dp4a((int)bw[t], (int)bw[t], ny);
                 }
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
+            for (int off = G >> 1; off > 0; off >>= 1) {
                 s += __shfl_xor_sync(0xffffffffu, s, off);
                 nx += __shfl_xor_sync(0xffffffffu, nx, off);
                 ny += __shfl_xor_sync(0xffffffffu, ny, off);
@@ -62,7 +69,7 @@ filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__res
             }
         } else {
             float s = 0.f, nx = 0.f, ny = 0.f;       // L2: s accumulates the squared differences
-            for (int c = lane; c < g; c += 32) {
+            for (int c = lane; c < gl; c += G) {
                 const uint4 a = __ldg(x + c), b = __ldg(y + c);
                 const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
@@ -85,8 +92,7 @@ filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__res
                     }
                 }
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
+            for (int off = G >> 1; off > 0; off >>= 1) {
                 s += __shfl_xor_sync(0xffffffffu, s, off);
                 if constexpr (KIND == KIND_COS) {
                     nx += __shfl_xor_sync(0xffffffffu, nx, off);
@@ -97,7 +103,7 @@ filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__res
             if constexpr (KIND == KIND_L2) pass = s <= thr_f;
             if constexpr (KIND == KIND_COS) pass = (nx == 0.f || ny == 0.f) ? thr_f <= 0.f : s >= thr_f * sqrtf(nx) * sqrtf(ny);
         }
-        if (lane == 0 && pass) out[atomicAdd(counter, 1ULL)] = pr;
+        if (live && lane == 0 && pass) out[atomicAdd(counter, 1ULL)] = pr;
     }
 }
 

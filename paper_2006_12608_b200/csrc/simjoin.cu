@@ -752,8 +752,11 @@ simjoin_status filter_device(simjoin_ctx *ctx, const void *P, int64_t n, const v
     set_thresholds(jp, i8, kind, threshold);
     cudaStream_t s = ctx->stream;
     if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    // one warp per pair, at most 16 blocks per SM (the warps then stride over the list)
-    const unsigned long long want_blocks = (count_in * 32 + FILTER_THREADS - 1) / FILTER_THREADS;
+    // G lanes per pair (the power of two covering the row's 16-byte words), at most 16 blocks per SM (the warps then
+    // stride over the list)
+    int G = 1;
+    while (G < g && G < 32) G *= 2;
+    const unsigned long long want_blocks = (count_in * G + FILTER_THREADS - 1) / FILTER_THREADS;
     const unsigned long long max_blocks = (unsigned long long)ctx->num_sms * 16;
     const unsigned blocks = (unsigned)(want_blocks < max_blocks ? want_blocks : max_blocks);
     const uint4 *p4 = reinterpret_cast<const uint4 *>(P), *q4 = reinterpret_cast<const uint4 *>(Q);
@@ -762,7 +765,7 @@ simjoin_status filter_device(simjoin_ctx *ctx, const void *P, int64_t n, const v
     unsigned int *status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
 #define SJ_FILTER(DT, KIND)                                                                                              \
     filter_pairs_kernel<DT, KIND><<<blocks, FILTER_THREADS, 0, s>>>(p4, n, q4, m, g, in, count_in, (int)ctx->ioff, (int)ctx->joff, \
-                                                                    jp.thr_i, jp.thr_f, jp.thr_d, out, ctx->d_ctrl, status)
+                                                                    jp.thr_i, jp.thr_f, jp.thr_d, out, ctx->d_ctrl, status, G)
     if (i8 && kind == SIMJOIN_IP) SJ_FILTER(DT_I8, KIND_IP);
     else if (i8 && kind == SIMJOIN_COS) SJ_FILTER(DT_I8, KIND_COS);
     else if (i8) SJ_FILTER(DT_I8, KIND_L2);
