@@ -312,22 +312,44 @@ static uint64_t splitmix64_at(uint64_t seed, uint64_t idx) {
     return z ^ (z >> 31);
 }
 
+/* The coordinates sampled by the bits of repetition `rep`: bit b takes the first of
+ *     splitmix64(seed, 64 rep + b + 4096 a) mod d,   a = 0, 1, 2, ...
+ * that no earlier bit of the repetition took -- bit sampling without replacement, so that a repetition of k bits
+ * really has 2^k buckets (sampled with replacement, k = 7 of d = 128 coordinates repeat one in 15 % of the
+ * repetitions).  From bit d on every coordinate is taken and a = 0 is used as it comes. */
+static void lsh_rep_coordinates(uint64_t seed, int32_t rep, int32_t bits, int32_t d, int32_t *coord) {
+    for (int32_t b = 0; b < bits; ++b) {
+        for (uint64_t a = 0;; ++a) {
+            int32_t c = (int32_t)(splitmix64_at(seed, (uint64_t)rep * 64u + (uint64_t)b + 4096u * a) % (uint64_t)d);
+            int taken = 0;
+            for (int32_t e = 0; e < b && b < d; ++e) taken |= coord[e] == c;
+            if (!taken) { coord[b] = c; break; }
+        }
+    }
+}
+
 int32_t oracle_lsh_coordinate(uint64_t seed, int32_t rep, int32_t bit, int32_t d) {
-    return (int32_t)(splitmix64_at(seed, (uint64_t)rep * 64u + (uint64_t)bit) % (uint64_t)d);
+    int32_t coord[64];
+    if (bit < 0 || bit >= 64) return -1;
+    lsh_rep_coordinates(seed, rep, bit + 1, d, coord);
+    return coord[bit];
 }
 
 /* keys[l * rows + i] = the hash of row i in repetition l (bit b = [x_{c(l,b)} > 0]); k bits in the
  * first L_high repetitions, k - 1 in the next L_low. */
 void oracle_lsh_keys_i8(const int8_t *X, int64_t rows, int32_t d, int32_t L_high, int32_t L_low, int32_t k, uint64_t seed,
                         uint32_t *keys) {
-    for (int32_t l = 0; l < L_high + L_low; ++l)
+    for (int32_t l = 0; l < L_high + L_low; ++l) {
+        int32_t coord[64];
+        const int32_t bits = l < L_high ? k : k - 1;
+        lsh_rep_coordinates(seed, l, bits, d, coord);
         for (int64_t i = 0; i < rows; ++i) {
             uint32_t key = 0;
-            const int32_t bits = l < L_high ? k : k - 1;
             for (int32_t b = 0; b < bits; ++b)
-                if (X[(size_t)i * d + oracle_lsh_coordinate(seed, l, b, d)] > 0) key |= 1u << b;
+                if (X[(size_t)i * d + coord[b]] > 0) key |= 1u << b;
             keys[(size_t)l * rows + i] = key;
         }
+    }
 }
 
 /* The same keys for bf16 rows: bit b = [x_{c(l,b)} > 0] on the value the 16-bit pattern denotes (+-0 -> 0).  For
@@ -335,14 +357,17 @@ void oracle_lsh_keys_i8(const int8_t *X, int64_t rows, int32_t d, int32_t L_high
  * axis-aligned hyperplanes: two points at angle theta agree on a sampled sign with probability 1 - theta / pi. */
 void oracle_lsh_keys_bf16(const uint16_t *X, int64_t rows, int32_t d, int32_t L_high, int32_t L_low, int32_t k, uint64_t seed,
                           uint32_t *keys) {
-    for (int32_t l = 0; l < L_high + L_low; ++l)
+    for (int32_t l = 0; l < L_high + L_low; ++l) {
+        int32_t coord[64];
+        const int32_t bits = l < L_high ? k : k - 1;
+        lsh_rep_coordinates(seed, l, bits, d, coord);
         for (int64_t i = 0; i < rows; ++i) {
             uint32_t key = 0;
-            const int32_t bits = l < L_high ? k : k - 1;
             for (int32_t b = 0; b < bits; ++b)
-                if (oracle_bf16_to_f64(X[(size_t)i * d + oracle_lsh_coordinate(seed, l, b, d)]) > 0.0) key |= 1u << b;
+                if (oracle_bf16_to_f64(X[(size_t)i * d + coord[b]]) > 0.0) key |= 1u << b;
             keys[(size_t)l * rows + i] = key;
         }
+    }
 }
 
 int64_t oracle_lsh_join_i8(const int8_t *P, int64_t n, const int8_t *Q, int64_t m, int32_t d, double threshold,

@@ -95,11 +95,40 @@ def _splitmix64(seed, idx):
     return z ^ (z >> 31)
 
 
+def _lsh_coords(seed, L, k, d):
+    """Bit b of repetition l samples the first of splitmix64(seed, 64 l + b + 4096 a) mod d, a = 0, 1, ..., that no
+    earlier bit of the repetition took (sampling without replacement)."""
+    out = []
+    for l in range(L):
+        row = []
+        for b in range(k):
+            a = 0
+            while True:
+                c = _splitmix64(seed, l * 64 + b + 4096 * a) % d
+                if b >= d or c not in row:
+                    row.append(c)
+                    break
+                a += 1
+        out.append(row)
+    return np.array(out).reshape(L, k)
+
+
+def test_lsh_coordinates_are_distinct_within_a_repetition():
+    for seed, L, k, d in [(2006, 8, 7, 128), (1, 64, 12, 16), (7, 5, 12, 8)]:
+        c = _lsh_coords(seed, L, k, d)
+        assert all(O.lsh_coordinate(seed, l, b, d) == c[l, b] for l in range(L) for b in range(k))
+        assert all(len(set(c[l, :min(k, d)])) == min(k, d) for l in range(L))
+        assert all(c[l, 0] == _splitmix64(seed, l * 64) % d for l in range(L))     # the first bit is the plain sample
+    # the plain samples of seed 2006 repeat a coordinate in repetitions 0 and 4 (6 and 5 distinct of 7)
+    plain = [[_splitmix64(2006, l * 64 + b) % 128 for b in range(7)] for l in range(8)]
+    assert [len(set(r)) for r in plain] == [6, 7, 7, 7, 5, 7, 7, 7]
+
+
 def test_lsh_join_is_brute_force_restricted_to_colliding_pairs():
     # independent route: python-int splitmix64 for the sampled coordinates, numpy for keys and scores
     w = W.make_workload(4, n=700, m=600, planted=80)
     L, k, seed, d = 5, 4, 1234, w.d
-    coords = np.array([[_splitmix64(seed, l * 64 + b) % d for b in range(k)] for l in range(L)])
+    coords = _lsh_coords(seed, L, k, d)
     assert all(O.lsh_coordinate(seed, l, b, d) == coords[l, b] for l in range(L) for b in range(k))
     kp = ((w.P[:, coords] > 0).astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T      # (L, n)
     kq = ((w.Q[:, coords] > 0).astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T
@@ -129,7 +158,7 @@ def test_lsh_hamming_join_is_the_hamming_join_restricted_to_equal_sampled_bits()
     d, L, k, seed = 128, 4, 5, 321
     Pb = W.random_bits(500, d, 41)
     Qb = W.random_bits(600, d, 42, planted_from=Pb[:60], flips=6)
-    coords = np.array([[_splitmix64(seed, l * 64 + b) % d for b in range(k)] for l in range(L)])
+    coords = _lsh_coords(seed, L, k, d)
     bp = np.unpackbits(Pb, axis=1, bitorder="little")[:, :d]
     bq = np.unpackbits(Qb, axis=1, bitorder="little")[:, :d]
     kp = (bp[:, coords].astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T
@@ -148,7 +177,7 @@ def test_lsh_sign_keys_for_bf16_rows_and_joins_of_any_kind():
     L, k, seed, d = 4, 6, 55, 96
     X = W.random_points("bf16", 300, d, 13)
     X[0, :5] = [0x0000, 0x8000, 0x3f80, 0xbf80, 0x0001]                      # +0, -0, 1, -1, smallest subnormal
-    coords = np.array([[_splitmix64(seed, l * 64 + b) % d for b in range(k)] for l in range(L)])
+    coords = _lsh_coords(seed, L, k, d)
     vals = W.bf16_bits_to_f32(X).astype(np.float64)
     want = ((vals[:, coords] > 0).astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T
     assert np.array_equal(want, O.lsh_keys(X, L, k, seed, dtype="bf16"))
@@ -174,13 +203,13 @@ def test_lsh_sign_hash_collision_probability_is_one_minus_theta_over_pi():
 
 
 def test_lsh_recall_matches_the_collision_probability():
-    # planted pairs differ in h = 8 of d = 128 coordinates: one k-bit sample collides with probability close
-    # to (1 - h/d)^k, so the recall over L repetitions is about 1 - (1 - (1-h/d)^k)^L
+    # planted pairs differ in h = 8 of d = 128 coordinates: a repetition of k distinct sampled coordinates collides
+    # with probability C(d-h, k) / C(d, k), so the recall over L repetitions is about 1 - (1 - that)^L
     w = W.make_workload(4, n=4000, m=4000, planted=2000)
     L, k = 4, 8
     pairs, _c = O.lsh_join(w.P, w.Q, w.threshold, L, k, 99)
     found = np.isin(O.pairs_to_set(w.planted), O.pairs_to_set(pairs)).mean()
-    p1 = (1 - 8 / 128) ** k
+    p1 = math.comb(128 - 8, k) / math.comb(128, k)
     expect = 1 - (1 - p1) ** L
     assert abs(found - expect) < 0.04, (found, expect)
     with pytest.raises(ValueError):
