@@ -143,8 +143,10 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
  *                 Hamming distance, i.e. for +-1 rows such as simjoin_run_hamming builds; for bf16 rows the
  *                 sign of the sampled coordinate, i.e. the random-hyperplane hash of the angular distance
  *                 with axis-aligned hyperplanes (two rows of a rotation-invariant distribution at angle
- *                 theta agree with probability 1 - theta/pi).  Bit b of the
- *                 key of repetition l samples coordinate splitmix64(seed, 64*l + b) mod d, where
+ *                 theta agree with probability 1 - theta/pi).  The k bits of a repetition sample k DISTINCT
+ *                 coordinates (without replacement, so that the repetition has 2^k buckets): bit b of
+ *                 repetition l takes the first of splitmix64(seed, 64*l + b + 4096*a) mod d, a = 0, 1, ...,
+ *                 that no earlier bit of the repetition took (from bit d on, a = 0 as it comes), where
  *                 splitmix64(seed, i): z = seed + (i+1)*0x9E3779B97F4A7C15; z = (z ^ z>>30)*0xBF58476D1CE4E5B9;
  *                 z = (z ^ z>>27)*0x94D049BB133111EB; z ^ z>>31  (all modulo 2^64).
  *   P, Q, n, m, d, kind, threshold, out_pairs, capacity, count   as simjoin_run (every dtype and kind it accepts).
@@ -167,7 +169,7 @@ simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const
 /*
  * LSH-bucketed Hamming join on bit-packed points: simjoin_run_hamming's operand transform followed by
  * simjoin_run_lsh -- bit sampling is the LSH family of the Hamming distance, so bit b of the key of repetition l is
- * simply coordinate splitmix64(seed, 64*l + b) mod d of the point.  The output is exactly
+ * simply the coordinate of the point that simjoin_run_lsh samples for that bit.  The output is exactly
  *     { (i, j) : Hamming(x_i, y_j) <= r  and  key_l(x_i) == key_l(y_j) for some repetition l }.
  * Arguments as simjoin_run_hamming (P_bits, Q_bits, n, m, d, r) and simjoin_run_lsh (L, L_low, k, seed); errors
  * as those two.  I8 contexts only.

@@ -25,19 +25,38 @@ __host__ __device__ inline uint64_t lsh_splitmix64(uint64_t seed, uint64_t idx) 
     return z ^ (z >> 31);
 }
 
+// s_coord[l * k + b] = the coordinate bit b of repetition l samples: the first of
+//     splitmix64(seed, 64 l + b + 4096 a) mod d,   a = 0, 1, 2, ...
+// that no earlier bit of the repetition took (bit sampling without replacement: k bits give 2^k buckets; from bit d
+// on, when every coordinate is taken, a = 0 is used as it comes).  One thread per repetition, one block, once per
+// call: the key kernels read the table from global memory.
+__global__ void __launch_bounds__(64) lsh_coordinates_kernel(unsigned long long seed, int L, int k, int d, int *__restrict__ coords) {
+    for (int l = threadIdx.x; l < L; l += blockDim.x) {
+        int *coord = coords + l * k;
+        for (int b = 0; b < k; ++b) {
+            for (uint64_t a = 0;; ++a) {
+                const int c = (int)(lsh_splitmix64(seed, (uint64_t)l * 64u + (uint64_t)b + 4096u * a) % (uint64_t)d);
+                bool taken = false;
+                for (int e = 0; e < b && b < d; ++e) taken = taken || coord[e] == c;
+                if (!taken) { coord[b] = c; break; }
+            }
+        }
+    }
+}
+__device__ __forceinline__ void lsh_load_coordinates(const int *__restrict__ coords, int L, int k, int *s_coord) {
+    for (int t = threadIdx.x; t < L * k; t += blockDim.x) s_coord[t] = coords[t];
+}
+
 // rec[i * stride + l] = key of row i in repetition l (one record of `stride` 16-bit keys per row, so that
 // all keys of a row sit in one or two cache lines): k bits in the first L_high repetitions, k - 1 (the
 // same samples without the last) in the following L_low -- the paper's mix of tables for a fractional
 // number of base hashes.  One thread per row; the sampled coordinates are computed once per block.
 template <typename T>   // int8_t, or int16_t for bf16 bit patterns
 __global__ void __launch_bounds__(256) lsh_keys_kernel(const T *__restrict__ X, long long rows, int d, int L_high, int L_low,
-                                                       int k, unsigned long long seed, uint16_t *__restrict__ rec, int stride) {
+                                                       int k, const int *__restrict__ coords, uint16_t *__restrict__ rec, int stride) {
     __shared__ int s_coord[LSH_MAX_REPS * LSH_MAX_BITS];
     const int L = L_high + L_low;
-    for (int t = threadIdx.x; t < L * k; t += blockDim.x) {
-        const int l = t / k, b = t - l * k;
-        s_coord[t] = (int)(lsh_splitmix64(seed, (uint64_t)l * 64u + (uint64_t)b) % (uint64_t)d);
-    }
+    lsh_load_coordinates(coords, L, k, s_coord);
     __syncthreads();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= rows) return;
@@ -58,14 +77,11 @@ constexpr int LSH_KEYS_STAGED_MAX_D = 512;
 constexpr int LSH_KEYS_STAGED_ROWS = 64;
 template <typename T>
 __global__ void __launch_bounds__(256) lsh_keys_staged_kernel(const T *__restrict__ X, long long rows, int d, int L_high, int L_low,
-                                                              int k, unsigned long long seed, uint16_t *__restrict__ rec, int stride) {
+                                                              int k, const int *__restrict__ coords, uint16_t *__restrict__ rec, int stride) {
     __shared__ int s_coord[LSH_MAX_REPS * LSH_MAX_BITS];
     extern __shared__ uint32_t s_rows[];                       // LSH_KEYS_STAGED_ROWS x (row bytes / 4 + 1) words
     const int L = L_high + L_low;
-    for (int t = threadIdx.x; t < L * k; t += blockDim.x) {
-        const int l = t / k, b = t - l * k;
-        s_coord[t] = (int)(lsh_splitmix64(seed, (uint64_t)l * 64u + (uint64_t)b) % (uint64_t)d);
-    }
+    lsh_load_coordinates(coords, L, k, s_coord);
     const long long row0 = (long long)blockIdx.x * LSH_KEYS_STAGED_ROWS;
     const int row_bytes = d * (int)sizeof(T);
     const int g = row_bytes / 16, pitch = row_bytes / 4 + 1;

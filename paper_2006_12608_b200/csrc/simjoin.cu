@@ -456,7 +456,8 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     const int nb_max = 1 << k;
     const size_t max_units = (size_t)((n + P_ROWS - 1) / P_ROWS) + (size_t)nb_max;
     // misc: hist_p | hist_q | cursor_p | cursor_q (nb words each) | nunits (padded to 16 B) | units
-    const size_t off_units = ((size_t)4 * nb_max * 4 + 16 + 15) & ~(size_t)15;
+    const size_t off_coords = ((size_t)4 * nb_max * 4 + 16 + 15) & ~(size_t)15;       // sampled coordinates: reps x k ints
+    const size_t off_units = (off_coords + (size_t)LSH_MAX_REPS * LSH_MAX_BITS * 4 + 15) & ~(size_t)15;
     const int reps = L + L_low;
     const int rec_words = (reps + 7) / 8, stride = rec_words * 8;   // key record of a row: 16-bit keys, padded to 16 bytes
     const size_t rec_bytes = (size_t)rec_words * 16;
@@ -474,6 +475,7 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     unsigned int *hist_p = reinterpret_cast<unsigned int *>(ctx->lsh_misc.ptr);
     unsigned int *hist_q = hist_p + nb_max, *cursor_p = hist_q + nb_max, *cursor_q = cursor_p + nb_max, *nunits = cursor_q + nb_max;
     int4 *units = reinterpret_cast<int4 *>(reinterpret_cast<unsigned char *>(ctx->lsh_misc.ptr) + off_units);
+    int *coords = reinterpret_cast<int *>(reinterpret_cast<unsigned char *>(ctx->lsh_misc.ptr) + off_coords);
     uint16_t *keys_p = reinterpret_cast<uint16_t *>(ctx->lsh_keys_p.ptr), *keys_q = reinterpret_cast<uint16_t *>(ctx->lsh_keys_q.ptr);
     int *perm_p = reinterpret_cast<int *>(ctx->lsh_perm_p.ptr), *perm_q = reinterpret_cast<int *>(ctx->lsh_perm_q.ptr);
 
@@ -530,23 +532,24 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         const unsigned bn = (unsigned)((n + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), bm = (unsigned)((m + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS);
         const size_t sm = (size_t)LSH_KEYS_STAGED_ROWS * (row_bytes / 4 + 1) * 4;
         const bool staged = row_bytes <= LSH_KEYS_STAGED_MAX_D;
+        lsh_coordinates_kernel<<<1, 64, 0, s>>>(seed, L + L_low, k, d, coords);
         if (i8) {
             const int8_t *p8 = reinterpret_cast<const int8_t *>(P), *q8 = reinterpret_cast<const int8_t *>(Q);
             if (staged) {
-                lsh_keys_staged_kernel<<<bn, 256, sm, s>>>(p8, n, d, L, L_low, k, seed, keys_p, stride);
-                lsh_keys_staged_kernel<<<bm, 256, sm, s>>>(q8, m, d, L, L_low, k, seed, keys_q, stride);
+                lsh_keys_staged_kernel<<<bn, 256, sm, s>>>(p8, n, d, L, L_low, k, coords, keys_p, stride);
+                lsh_keys_staged_kernel<<<bm, 256, sm, s>>>(q8, m, d, L, L_low, k, coords, keys_q, stride);
             } else {
-                lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(p8, n, d, L, L_low, k, seed, keys_p, stride);
-                lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(q8, m, d, L, L_low, k, seed, keys_q, stride);
+                lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(p8, n, d, L, L_low, k, coords, keys_p, stride);
+                lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(q8, m, d, L, L_low, k, coords, keys_q, stride);
             }
         } else {
             const int16_t *p16 = reinterpret_cast<const int16_t *>(P), *q16 = reinterpret_cast<const int16_t *>(Q);
             if (staged) {
-                lsh_keys_staged_kernel<<<bn, 256, sm, s>>>(p16, n, d, L, L_low, k, seed, keys_p, stride);
-                lsh_keys_staged_kernel<<<bm, 256, sm, s>>>(q16, m, d, L, L_low, k, seed, keys_q, stride);
+                lsh_keys_staged_kernel<<<bn, 256, sm, s>>>(p16, n, d, L, L_low, k, coords, keys_p, stride);
+                lsh_keys_staged_kernel<<<bm, 256, sm, s>>>(q16, m, d, L, L_low, k, coords, keys_q, stride);
             } else {
-                lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(p16, n, d, L, L_low, k, seed, keys_p, stride);
-                lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(q16, m, d, L, L_low, k, seed, keys_q, stride);
+                lsh_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(p16, n, d, L, L_low, k, coords, keys_p, stride);
+                lsh_keys_kernel<<<(unsigned)((m + 255) / 256), 256, 0, s>>>(q16, m, d, L, L_low, k, coords, keys_q, stride);
             }
         }
     }
