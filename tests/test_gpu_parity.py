@@ -530,3 +530,25 @@ def test_i8_cosine_planted_pairs_at_scale(ctx_i8):
     t = w.threshold / w.d
     cnt = int8_cos_case(ctx_i8, w.P, w.Q, t)
     assert cnt >= 300 and cnt == O.join(w.P, w.Q, "ip", w.threshold, "i8")[1]
+
+
+def test_repeated_calls_give_the_same_set(ctx_i8, ctx_bf16):
+    """The output order is unspecified (atomics), the set is not: repeated calls on one context, other calls in
+    between, return the same pairs -- also for bf16, where in-band pairs could fall on either side but the arithmetic
+    of a given launch configuration is fixed."""
+    w = W.make_workload(4, n=5000, m=7000, planted=300)
+    wb = W.make_workload(2, n=4000, m=3000, planted=300)
+    Pb, Qb = W.random_points("bf16", 2000, 64, 95), W.random_points("bf16", 2500, 64, 96)
+    first = {}
+    for rep in range(3):
+        runs = {"i8": gpu_join(ctx_i8, w.P, w.Q, "ip", 40.0, 1 << 22)[0],
+                "cos": gpu_join(ctx_bf16, wb.P, wb.Q, "cos", 0.2, 1 << 22)[0],
+                "l2": gpu_join(ctx_bf16, Pb, Qb, "l2", 9.0, 1 << 22)[0]}
+        for name, pairs in runs.items():
+            k = np.sort(keys(pairs))
+            assert len(k) > 1000
+            if rep == 0:
+                first[name] = k
+            else:
+                assert np.array_equal(first[name], k), name
+
