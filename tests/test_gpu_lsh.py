@@ -217,3 +217,24 @@ def test_lsh_bf16_sign_hash_join(ctx_bf16, kind, d, L, k):
     # recall against the brute-force join: a planted pair at angle theta survives a k-bit table with (1 - theta/pi)^k
     full = O.join(w.P, w.Q, kind, t, "bf16")[0]
     assert len(exact) <= len(full) and len(exact) > 0.3 * len(full)
+
+
+def test_lsh_more_key_bits_than_coordinates(ctx_bf16, ctx):
+    """k > d: the first d bits take every coordinate once, the later ones sample as they come.  8-coordinate bf16
+    rows (16 bytes) with 12 key bits, and 16-coordinate int8 rows with 12 of 16 coordinates taken."""
+    rng = np.random.default_rng(8)
+    Pb = W.f32_to_bf16_bits(rng.standard_normal((900, 8)).astype(np.float32))
+    Qb = W.f32_to_bf16_bits(rng.standard_normal((1100, 8)).astype(np.float32))
+    Qb[:300] = Pb[:300]
+    out = torch.full((1 << 20, 2), -5, dtype=torch.int32, device="cuda:0")
+    st, cnt = ctx_bf16.simjoin_run_lsh(B.to_device(Pb), 900, B.to_device(Qb), 1100, 8, 0.5, 3, 12, 7, out, 1 << 20, L_low=2, kind="l2")
+    assert st == B.SIMJOIN_OK, B.strerror(st)
+    got = keys(out[:cnt].cpu().numpy())
+    strict, exact, loose = O.lsh_band_sets(Pb, Qb, "l2", 0.5, "bf16", 3, 12, 7, L_low=2)
+    assert len(np.unique(got)) == cnt and np.isin(keys(strict), got).all() and np.isin(got, keys(loose)).all()
+    assert len(strict) >= 300
+    Pi = W.random_points("i8", 700, 16, 97, lo=-1, hi=1)
+    Qi = W.random_points("i8", 800, 16, 98, lo=-1, hi=1)
+    Qi[:200] = Pi[:200]
+    assert check(ctx, Pi, Qi, 6.0, 4, 12, 3) >= 200
+
