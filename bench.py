@@ -528,9 +528,9 @@ def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks
     launches_per_step = 1 + (2 if w.kind != "ip" else 0) + (2 if w.dtype == "i8" else 0)   # join + norms + max|x|
     if args.lsh:
         # max|x| x2, sampled coordinates, keys x2, then per table: 2 histograms, offsets + work list, 2 scatters, 2 row
-        # gathers, the join, and from the second table on 2 gathers of the key records
+        # gathers, the join
         tables = args.lsh[0] + (args.lsh[2] if len(args.lsh) > 2 else 0)
-        launches_per_step = 5 + 8 * tables + 2 * (tables - 1)
+        launches_per_step = 5 + 8 * tables
         roofline = None
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",

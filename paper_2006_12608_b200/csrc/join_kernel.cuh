@@ -99,7 +99,7 @@ struct JoinParams {
     const int4 *units;             // per unit: first P row, P rows (<= 128), first Q row, Q rows
     const unsigned int *nunits;    // number of units (written by the kernel that builds the list)
     const int *perm_p, *perm_q;    // regrouped position -> original row
-    const uint4 *rec_p, *rec_q;    // per regrouped position: the 16-bit hash keys of all repetitions, rec_words x 16 bytes
+    const uint4 *rec_p, *rec_q;    // per ORIGINAL row: the 16-bit hash keys of all repetitions, rec_words x 16 bytes
     int rec_words;
     int rep;                       // repetitions already joined: a pair whose keys agreed in one of them is not reported again
     // I8/COS: candidates of the fp32 filter are decided exactly from the rows themselves when they leave the CTA
@@ -265,9 +265,10 @@ struct TreeMax<1, MODE> {
 // stores are coalesced.
 // Bucketed mode, repetition > 0: did the hash keys of regrouped rows (i, j) already agree in an earlier
 // repetition?  Then that repetition found and reported the pair (Section 4's union over repetitions).
-// Both key records are addressed by regrouped position, so the loads of a pair go out together.
+// The key records stay in the rows' original order and are reached through the regrouping permutation: one more
+// dependent load per staged pair, against two gathers of all key records per repetition.
 __device__ __forceinline__ bool already_reported(const JoinParams &p, long long i, long long j) {
-    const uint4 *rp = p.rec_p + i * p.rec_words, *rq = p.rec_q + j * p.rec_words;
+    const uint4 *rp = p.rec_p + (long long)__ldg(p.perm_p + i) * p.rec_words, *rq = p.rec_q + (long long)__ldg(p.perm_q + j) * p.rec_words;
     bool seen = false;
     for (int w = 0; w * 8 < p.rep; ++w) {
         const uint4 a = __ldg(rp + w), b = __ldg(rq + w);

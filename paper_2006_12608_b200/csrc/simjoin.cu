@@ -58,7 +58,7 @@ struct simjoin_ctx {
     DevBuf jl_p, jl_q;                  // simjoin_run_jl_l2: the reduced point sets
     DevBuf filter_out;                  // simjoin_filter_pairs: the kept pairs before they replace the list
     // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
-    DevBuf lsh_keys_p, lsh_keys_q, lsh_skeys_p, lsh_skeys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
+    DevBuf lsh_keys_p, lsh_keys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
 };
 
 namespace {
@@ -462,7 +462,6 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     const int rec_words = (reps + 7) / 8, stride = rec_words * 8;   // key record of a row: 16-bit keys, padded to 16 bytes
     const size_t rec_bytes = (size_t)rec_words * 16;
     if (!grow(ctx->lsh_keys_p, n * rec_bytes) || !grow(ctx->lsh_keys_q, m * rec_bytes) ||
-        !grow(ctx->lsh_skeys_p, n * rec_bytes) || !grow(ctx->lsh_skeys_q, m * rec_bytes) ||
         !grow(ctx->lsh_perm_p, (size_t)n * 4) || !grow(ctx->lsh_perm_q, (size_t)m * 4) ||
         !grow(ctx->lsh_sorted_p, (size_t)n * row_bytes) || !grow(ctx->lsh_sorted_q, (size_t)m * row_bytes) ||
         !grow(ctx->lsh_misc, off_units + max_units * 16))
@@ -498,8 +497,8 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.nunits = nunits;
     jp.perm_p = perm_p;
     jp.perm_q = perm_q;
-    jp.rec_p = reinterpret_cast<const uint4 *>(ctx->lsh_skeys_p.ptr);
-    jp.rec_q = reinterpret_cast<const uint4 *>(ctx->lsh_skeys_q.ptr);
+    jp.rec_p = reinterpret_cast<const uint4 *>(ctx->lsh_keys_p.ptr);      // in the rows' original order
+    jp.rec_q = reinterpret_cast<const uint4 *>(ctx->lsh_keys_q.ptr);
     jp.rec_words = rec_words;
 
     CUtensorMap mapP, mapQ;
@@ -573,13 +572,6 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
             reinterpret_cast<const uint4 *>(P), perm_p, n, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_p.ptr));
         lsh_gather_rows_kernel<<<(unsigned)(((long long)m * g + 255) / 256), 256, 0, s>>>(
             reinterpret_cast<const uint4 *>(Q), perm_q, m, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_q.ptr));
-        if (l > 0) {
-            // key records in regrouped order, for the duplicate check of the join's epilogue
-            lsh_gather_rows_kernel<<<(unsigned)(((long long)n * rec_words + 255) / 256), 256, 0, s>>>(
-                reinterpret_cast<const uint4 *>(keys_p), perm_p, n, rec_words, reinterpret_cast<uint4 *>(ctx->lsh_skeys_p.ptr));
-            lsh_gather_rows_kernel<<<(unsigned)(((long long)m * rec_words + 255) / 256), 256, 0, s>>>(
-                reinterpret_cast<const uint4 *>(keys_q), perm_q, m, rec_words, reinterpret_cast<uint4 *>(ctx->lsh_skeys_q.ptr));
-        }
         if (need_norms) {
             // row terms and per-256-row bounds of the regrouped rows
             const int sq = norm_mode(i8, kind, threshold);
@@ -867,8 +859,6 @@ simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
     release(ctx->filter_out);
     release(ctx->lsh_keys_p);
     release(ctx->lsh_keys_q);
-    release(ctx->lsh_skeys_p);
-    release(ctx->lsh_skeys_q);
     release(ctx->lsh_perm_p);
     release(ctx->lsh_perm_q);
     release(ctx->lsh_sorted_p);
