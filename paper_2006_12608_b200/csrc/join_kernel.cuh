@@ -96,7 +96,7 @@ struct JoinParams {
     int ioff, joff;          // added to emitted indices
     // Bucketed mode (the LSH join): the rows of P and Q have been regrouped so that each bucket is a
     // contiguous row range, and the work list names (P row range, Q row range) units instead of the grid.
-    const int4 *units;             // per unit: first P row, P rows (<= 128), first Q row, Q rows
+    const int4 *units;             // per unit: first P row, P rows (<= P_ROWS = 256), first Q row, Q rows
     const unsigned int *nunits;    // number of units (written by the kernel that builds the list)
     const int *perm_p, *perm_q;    // regrouped position -> original row
     const uint4 *rec_p, *rec_q;    // per ORIGINAL row: the 16-bit hash keys of all repetitions, rec_words x 16 bytes
@@ -106,11 +106,33 @@ struct JoinParams {
     const void *rows_p, *rows_q;   // the row arrays the tensor maps cover
     int row_bytes;
     double thr_d;                  // t
+    // Variant selection on the device.  With sel_mode != 0 the host launches the plain and the ALT instantiation
+    // back to back and each decides from the same two device words whether it is the one to run; the other returns
+    // at once.  The host therefore needs no round trip between the pre-pass that writes the words and the join.
+    //   SEL_I8_RANGE   words = max|P|, max|Q| over all int8 coordinates: ALT (16-bit epilogue) iff d * max * max <= 32767
+    //   SEL_L2_RADIUS  words = float bits of max |x|^2, max |y|^2: ALT (candidates decided from the rows) iff the rounding
+    //                  error of the norm expansion, sel_coef * (max|x|^2 + max|y|^2), exceeds 1.9 % of r^2
+    const unsigned int *sel_words;
+    int sel_mode;
+    float sel_coef;
+    // BF16/L2, ALT: the tile test is a filter  s >= (l2_xscale |x|^2 - l2_thr_filter) / 2 + l2_ycoef |y|^2, lowered by the
+    // error bound so that every pair the difference form accepts is a candidate
+    float l2_xscale, l2_ycoef, l2_thr_filter;
     // KIND_STORE
     uint16_t *store_out;
     long long store_ld;
     float store_scale;
 };
+
+constexpr int SEL_NONE = 0, SEL_I8_RANGE = 1, SEL_L2_RADIUS = 2;
+// Share of r^2 that the norm expansion's rounding error may reach before the Euclidean join switches to deciding
+// candidates from the rows: the tolerance is |distance - r| <= 1e-2 r, i.e. 1.99 % of r^2 on the squared scale.
+constexpr float L2_BAND_SHARE = 0.019f;
+__device__ __forceinline__ bool alt_selected(const JoinParams &p) {
+    const unsigned int a = __ldg(p.sel_words), b = __ldg(p.sel_words + 1);
+    if (p.sel_mode == SEL_I8_RANGE) return (unsigned long long)p.row_bytes * a * b <= 32767ull;
+    return p.sel_coef * (__uint_as_float(a) + __uint_as_float(b)) > L2_BAND_SHARE * p.thr_f;
+}
 
 struct Ctrl {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES];
@@ -302,16 +324,43 @@ __device__ __forceinline__ bool cos_i8_passes(const JoinParams &p, long long li,
     return __ddiv_rn((double)s, den) >= p.thr_d;
 }
 
-// Is the staged pair dropped when it leaves the CTA?  Bucketed mode: reported by an earlier repetition.  VERIFY
-// (I8/COS): a candidate of the fp32 filter that fails the exact test.  Staged indices are regrouped positions in
-// bucketed mode, else row indices plus the caller's offsets.
-template <bool GROUPED, bool VERIFY>
+// BF16/L2, small radii: the decision for the pair of rows (li of P, lj of Q) in the difference form
+// sum (x_k - y_k)^2 <= r^2, fp32, which does not cancel the way |x|^2 + |y|^2 - 2<x,y> does when r^2 is far
+// below the norms (relative error about d * 2^-24 whatever the radius).
+__device__ __forceinline__ bool l2_bf16_passes(const JoinParams &p, long long li, long long lj) {
+    const int g = p.row_bytes >> 4;
+    const uint4 *x = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.rows_p) + li * p.row_bytes);
+    const uint4 *y = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.rows_q) + lj * p.row_bytes);
+    float s[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int c = 0; c < g; ++c) {
+        const uint4 a = __ldg(x + c), b = __ldg(y + c);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const float e0 = __uint_as_float(aw[t] << 16) - __uint_as_float(bw[t] << 16);
+            const float e1 = __uint_as_float(aw[t] & 0xffff0000u) - __uint_as_float(bw[t] & 0xffff0000u);
+            s[t] = fmaf(e0, e0, s[t]);
+            s[t] = fmaf(e1, e1, s[t]);
+        }
+    }
+    return (s[0] + s[1]) + (s[2] + s[3]) <= p.thr_f;
+}
+
+// Is the staged pair dropped when it leaves the CTA?  Bucketed mode: reported by an earlier repetition.  VERIFY:
+// the pair is a candidate of a tile-level filter and fails the decision taken from its two rows (VERIFY_COS_I8: the
+// exact int8 cosine; VERIFY_L2_BF16: the difference-form Euclidean test).  Staged indices are regrouped positions
+// in bucketed mode, else row indices plus the caller's offsets.
+constexpr int VERIFY_NONE = 0, VERIFY_COS_I8 = 1, VERIFY_L2_BF16 = 2;
+template <bool GROUPED, int VERIFY>
 __device__ __forceinline__ bool drop_pair(const JoinParams &p, int i, int j) {
     if constexpr (GROUPED) {
         if (p.rep > 0 && already_reported(p, i, j)) return true;
     }
-    if constexpr (VERIFY) {
+    if constexpr (VERIFY == VERIFY_COS_I8) {
         if (!cos_i8_passes(p, GROUPED ? i : i - p.ioff, GROUPED ? j : j - p.joff)) return true;
+    }
+    if constexpr (VERIFY == VERIFY_L2_BF16) {
+        if (!l2_bf16_passes(p, GROUPED ? i : i - p.ioff, GROUPED ? j : j - p.joff)) return true;
     }
     return false;
 }
@@ -321,12 +370,12 @@ __device__ __forceinline__ int2 final_pair(const JoinParams &p, int2 pr) {
     if constexpr (GROUPED) return make_int2(__ldg(p.perm_p + pr.x) + p.ioff, __ldg(p.perm_q + pr.y) + p.joff);
     return pr;
 }
-template <bool GROUPED, bool VERIFY = false>
+template <bool GROUPED, int VERIFY = VERIFY_NONE>
 __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf, int fill, int lane) {
     if (fill == 0) return;
-    if constexpr (GROUPED || VERIFY) {
-        if (VERIFY || p.rep > 0) {
-            // Duplicates (and, for I8/COS, candidates that fail the exact test) are dropped here, a whole buffer
+    if constexpr (GROUPED || VERIFY != VERIFY_NONE) {
+        if (VERIFY != VERIFY_NONE || p.rep > 0) {
+            // Duplicates (and, for the filtered kinds, candidates that fail the exact test) are dropped here, a whole buffer
             // at a time (32 lookups in flight per step), not when a hit is found: there the lookup's latency
             // would stall the CTA's pipeline.
             int2 *wbuf = const_cast<int2 *>(buf);
@@ -374,7 +423,7 @@ __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf
 // prefix over the warp, then into the warp's shared-memory staging buffer, which is flushed with
 // one global atomic per ~STAGE_PAIRS pairs.  A block with more hits than the buffer holds goes
 // straight to global memory.  `fill` (warp-uniform) is the number of pairs staged so far.
-template <int NQ, bool GROUPED, bool VERIFY = false>
+template <int NQ, bool GROUPED, int VERIFY = VERIFY_NONE>
 __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (&mask)[NQ], int lane, long long i, long long j0,
                                            int2 *buf, int &fill) {
     int cnt = 0;
@@ -404,8 +453,8 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     const int ii = (int)(i + (GROUPED ? 0 : p.ioff));
     const int jj = (int)(j0 + (GROUPED ? 0 : p.joff));
     if (total > STAGE_PAIRS) {
-        if constexpr (GROUPED || VERIFY) {
-            if (VERIFY || p.rep > 0) {
+        if constexpr (GROUPED || VERIFY != VERIFY_NONE) {
+            if (VERIFY != VERIFY_NONE || p.rep > 0) {
                 // more hits in one block than the buffer holds (rare): check and write them one by one
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
@@ -630,9 +679,14 @@ __device__ __forceinline__ void mma_issuer_long(const JoinParams &p, Ctrl *ctrl,
     }
 }
 
-// NARROW (int8 only): the host has verified that every score fits in 16 bits, so the epilogue
-// loads the accumulator packed two columns per register and reduces it with packed 16-bit max --
-// half the registers and half the ALU work of the 32-bit path, which is what bounds short-K tiles.
+// ALT selects the second instantiation of a (element type, kind) pair; which of the two runs is decided on the
+// device (JoinParams::sel_mode), or by the host where no selection is in force.
+//   int8 (NARROW): every score provably fits in 16 bits, so the epilogue loads the accumulator packed two columns per
+//     register and reduces it with packed 16-bit max -- half the registers and half the ALU work of the 32-bit path,
+//     which is what bounds short-K tiles.
+//   bf16 Euclidean: the radius is too small for the norm expansion |x|^2 + |y|^2 - 2<x,y> in fp32 (its rounding error
+//     exceeds the stated tolerance on r): the tile test becomes a filter, lowered by the error bound, and every
+//     candidate is decided in the difference form from its two rows when it leaves the CTA.
 // KC > 0 (1 or 2): the chunks per tile, and with them the resident-P mode, the ring depth and the
 // epilogue hand-back, are compile-time constants -- the host selects these instantiations when the
 // run-time values agree.  Measured on B200: -6 % on the one-chunk int8 join.  KC == 0: all run-time.
@@ -641,16 +695,22 @@ __host__ __device__ constexpr int fast_nstages(int kc, int pbufs) {
                ? MAX_STAGES
                : (232448 - 1024 - CTRL_BYTES - STAGING_BYTES - pbufs * kc * A_CHUNK_BYTES) / B_CHUNK_BYTES;
 }
-// GROUPED: bucketed mode (int8 inner product only) -- see JoinParams::units.
+// GROUPED: bucketed mode (every element type and kind) -- see JoinParams::units.
 // GEO selects the tile geometry.  GEO_LONG: the long-row geometry above (join kinds, brute-force schedule only).
 // GEO_WIDEQ (store kind, resident operand of at most 128 rows): one resident block against 256 streamed rows per
 // tile -- 4 MMAs of N = 256 per chunk into the 256 columns of an accumulator buffer, 32 KiB TMA transactions --
 // which this HBM-bound use prefers to two half-empty 128-column blocks.  In both, mapQ has 256-row boxes.
 constexpr int GEO_STD = 0, GEO_LONG = 1, GEO_WIDEQ = 2;
-template <int DT, int KIND, bool NARROW = false, int KC = 0, bool GROUPED = false, int GEO = GEO_STD>
+template <int DT, int KIND, bool ALT = false, int KC = 0, bool GROUPED = false, int GEO = GEO_STD>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ, const JoinParams p_in) {
     constexpr bool LONGK = GEO == GEO_LONG, WIDEQ = GEO == GEO_WIDEQ;
+    constexpr bool NARROW = DT == DT_I8 && ALT;
+    constexpr bool L2_FILTER = DT == DT_BF16 && KIND == KIND_L2 && ALT;
+    static_assert(DT == DT_I8 || !ALT || KIND == KIND_L2, "bf16: only the Euclidean kind has a second variant");
+    // not the variant the data calls for: the other launch does the work (uniform over the grid, before any barrier
+    // or tensor-memory allocation exists)
+    if (p_in.sel_mode != SEL_NONE && alt_selected(p_in) != ALT) return;
     static_assert(!LONGK || (KC == 0 && KIND != KIND_STORE), "long-row mode: general join kinds only");
     static_assert(!WIDEQ || (KC == 0 && !GROUPED && KIND == KIND_STORE), "wide-Q mode: store kind only");
     constexpr int TN = (LONGK || WIDEQ) ? LONG_TN : TILE_N;   // rows of Q per tile
@@ -749,8 +809,23 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             }
         }
         if (!ok && lane == 0) {
-            // aborting: give copies already in flight time to land before shared memory is released
-            for (int t = 0; t < 200; ++t) __nanosleep(1000);
+            // aborting: shared memory may be released only after the copies already in flight have landed.  Stage s was
+            // last armed in this trip round the ring (s < stage) or in the previous one; a `full` barrier that was never
+            // armed reads as complete for the previous trip's parity.  Every wait is bounded (~1 ms each).
+            const long long lim = 2000000LL;
+            for (uint32_t s = 0; s < (uint32_t)p.nstages; ++s) {
+                const uint32_t par = s < stage ? phase : phase ^ 1u;
+                const long long t0 = clock64();
+                while (!mbar_try_wait(smem_u32(&ctrl->full[s]), par) && clock64() - t0 < lim) {}
+            }
+            if (p.stationary) {
+                const uint32_t nb = (uint32_t)p_bufs(GROUPED, kc);
+                for (uint32_t b = 0; b < nb; ++b) {
+                    const uint32_t par = b < pbuf ? pphase : pphase ^ 1u;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(smem_u32(&ctrl->pfull[b]), par) && clock64() - t0 < lim) {}
+                }
+            }
         }
         __syncwarp();
     } else if (warp == 1 || warp == 3) {
@@ -779,7 +854,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         const int half = (warp - EPI_WARP0) >> 2;   // which of the tile's two P blocks (accumulator columns half * TILE_N ..)
         const int row_in_tile = half * TILE_M + quarter * 32 + lane;
         uint32_t acc = 0, accphase = 0, rstage = 0;   // rstage: next ring stage to hand back
-        constexpr bool VERIFY = DT == DT_I8 && KIND == KIND_COS;     // candidates are decided exactly at flush time
+        // candidates of a filter are decided from their rows at flush time
+        constexpr int VERIFY = (DT == DT_I8 && KIND == KIND_COS) ? VERIFY_COS_I8 : (L2_FILTER ? VERIFY_L2_BF16 : VERIFY_NONE);
         int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * (WARP_STAGE_BYTES / 8);
         uint32_t *colterm = reinterpret_cast<uint32_t *>(stage_buf + STAGE_PAIRS);
         int stage_fill = 0;
@@ -815,7 +891,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     rf = b >= 0.f ? b * (1.f - 0x1p-18f) : b * (1.f + 0x1p-18f);
                 }
                 // BF16/L2 decides |x|^2 + |y|^2 - 2s <= r^2 as  s >= (|x|^2 - r^2)/2 + |y|^2/2:  one add per element
-                if constexpr (DT == DT_BF16 && KIND == KIND_L2) rf = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] - p.thr_f);
+                if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
+                    if constexpr (L2_FILTER) rf = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] * p.l2_xscale - p.l2_thr_filter);
+                    else rf = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] - p.thr_f);
+                }
             }
             for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
                 const int qt = tile_at<ALIGNED>(un, k);
@@ -847,7 +926,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 }
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
                     const float2 s0 = reinterpret_cast<const float2 *>(p.qstat)[qb0], s1 = reinterpret_cast<const float2 *>(p.qstat)[qb1];
-                    ff = rf + 0.5f * fminf(s0.x, s1.x);           // s >= (|x|^2 - r^2)/2 + min|y|^2/2
+                    // s >= (|x|^2 - r^2)/2 + min|y|^2/2; the filter form rounds exactly as its element test does
+                    if constexpr (L2_FILTER) ff = __fmaf_rn(p.l2_ycoef, fminf(s0.x, s1.x), rf);
+                    else ff = rf + 0.5f * fminf(s0.x, s1.x);
                 }
                 // per-column terms of this warp's columns, 4 per lane, fetched while the tile is still
                 // being multiplied so that the exact test never waits on global memory (fetching them only when a
@@ -1015,6 +1096,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             for (int c = 0; c < GCOLS; ++c) {
                                 const float b = KIND == KIND_IP    ? p.thr_f
                                                 : KIND == KIND_COS ? __fmul_rn(rf, __uint_as_float(yw[c]))   // as level 0 rounds it
+                                                : L2_FILTER        ? __fmaf_rn(p.l2_ycoef, __uint_as_float(yw[c]), rf)
                                                                    : rf + 0.5f * __uint_as_float(yw[c]);
                                 fail[c >> 2] = __funnelshift_l(__float_as_uint(__uint_as_float(v[k * GCOLS + c]) - b), fail[c >> 2], 1);
                             }

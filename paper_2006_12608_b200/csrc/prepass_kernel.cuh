@@ -70,11 +70,13 @@ __device__ __forceinline__ void warp_rows_pow2(const uint4 *__restrict__ X, long
 // X: rows x (g * 16 bytes).  norms[r] = sum of squares of row r; with sqrt_out its square root in fp32 (int8
 // rows too: the bits of the float in the int32 array, whose order is the floats' order); sqrt_out == 2 stores
 // +inf for a zero row.  tile_minmax[b] = (min, max) of norms over the valid rows of tile b (may be null).
+// all_max (may be null): the largest stored value of the whole launch, folded in with one atomicMax per block on
+// its bit pattern (stored values are non-negative, so the patterns order like the values).
 template <bool kInt8>
 __global__ void __launch_bounds__(NORM_THREADS)
 row_norms_kernel(const uint4 *__restrict__ X, long long rows, int g, int sqrt_out,
                  typename NormAcc<kInt8>::type *__restrict__ norms,
-                 typename NormAcc<kInt8>::type *__restrict__ tile_minmax) {
+                 typename NormAcc<kInt8>::type *__restrict__ tile_minmax, unsigned int *__restrict__ all_max) {
     using T = typename NormAcc<kInt8>::type;
     __shared__ T s_val[NORM_TILE_ROWS];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -112,7 +114,7 @@ row_norms_kernel(const uint4 *__restrict__ X, long long rows, int g, int sqrt_ou
     }
     const bool valid = r < rows;
     if (valid) norms[r] = v;
-    if (tile_minmax == nullptr) return;
+    if (tile_minmax == nullptr && all_max == nullptr) return;
     // block min / max over valid rows (row 0 of a launched tile is always valid)
     __syncthreads();
     s_val[threadIdx.x] = v;
@@ -132,22 +134,37 @@ row_norms_kernel(const uint4 *__restrict__ X, long long rows, int g, int sqrt_ou
             mn = s_mn[w] < mn ? s_mn[w] : mn;
             mx = s_mx[w] > mx ? s_mx[w] : mx;
         }
-        tile_minmax[2 * (long long)blockIdx.x] = mn;
-        tile_minmax[2 * (long long)blockIdx.x + 1] = mx;
+        if (tile_minmax != nullptr) {
+            tile_minmax[2 * (long long)blockIdx.x] = mn;
+            tile_minmax[2 * (long long)blockIdx.x + 1] = mx;
+        }
+        if (all_max != nullptr) {
+            unsigned int bits;
+            if constexpr (kInt8) bits = (unsigned int)mx;
+            else bits = __float_as_uint(mx);
+            atomicMax(all_max, bits);
+        }
     }
 }
 
-// max |x| over an int8 buffer of n16 16-byte words, folded into *out with atomicMax.  The host
-// uses it to prove that d * max|P| * max|Q| fits in 16 bits before choosing the packed epilogue.
-__global__ void __launch_bounds__(256) maxabs_i8_kernel(const uint4 *__restrict__ X, long long n16, unsigned int *out) {
+// max |x| over two int8 buffers of nP16 and nQ16 16-byte words, folded into out[0] (P) and out[1] (Q) with
+// atomicMax; the first half of the grid reads P, the second Q.  The join kernel proves from these two words that
+// d * max|P| * max|Q| fits in 16 bits before it takes the packed epilogue.
+__global__ void __launch_bounds__(256) maxabs_i8_kernel(const uint4 *__restrict__ P, long long nP16, const uint4 *__restrict__ Q,
+                                                        long long nQ16, unsigned int *out) {
+    const unsigned int half = gridDim.x >> 1;
+    const bool second = blockIdx.x >= half;
+    const uint4 *X = second ? Q : P;
+    const long long n16 = second ? nQ16 : nP16;
+    const unsigned int blk = second ? blockIdx.x - half : blockIdx.x, nblk = second ? gridDim.x - half : half;
     unsigned int m = 0;   // four unsigned byte maxima
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (long long)gridDim.x * blockDim.x) {
+    for (long long i = (long long)blk * blockDim.x + threadIdx.x; i < n16; i += (long long)nblk * blockDim.x) {
         const uint4 q = __ldg(X + i);
         m = __vmaxu4(m, __vmaxu4(__vmaxu4(__vabs4(q.x), __vabs4(q.y)), __vmaxu4(__vabs4(q.z), __vabs4(q.w))));
     }
     unsigned int v = max(max(m & 0xffu, (m >> 8) & 0xffu), max((m >> 16) & 0xffu, m >> 24));
     v = __reduce_max_sync(0xffffffffu, v);
-    if ((threadIdx.x & 31) == 0 && v > 0) atomicMax(out, v);
+    if ((threadIdx.x & 31) == 0 && v > 0) atomicMax(out + (second ? 1 : 0), v);
 }
 
 // Operand transform for the Hamming ip-distance (Section 4): bit-packed {0,1} coordinates -> +-1 int8

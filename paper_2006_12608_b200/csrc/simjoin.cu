@@ -32,6 +32,17 @@ struct DevBuf {
     size_t bytes = 0;
 };
 
+constexpr int MAX_HOST_SLICES = 66;     // simjoin_run_host: a Q of more slices than this goes up in one piece
+
+// Device-side working memory of one join call, and the host words its result lands in.  simjoin_run takes it from the
+// context's buffers (grown on demand); the allocation-free entry point points it at a fixed array.
+struct JoinScratch {
+    void *nx, *ny, *qstat;        // row terms of P (n entries) and Q (whole tiles), (min, max) of ny per 256 rows of Q
+    unsigned long long *d_ctrl;   // 64 bytes: [0] pair counter, [1] status word, [2] max|P|, max|Q| (two 32-bit words, int8),
+                                  // [3] bit patterns of max|x|^2, max|y|^2 (two 32-bit words, bf16 Euclidean)
+    unsigned long long *h_ctrl;   // host copy of words [0] and [1]
+};
+
 }  // namespace
 
 struct simjoin_ctx {
@@ -53,7 +64,7 @@ struct simjoin_ctx {
     bool attr_set_long[2][3][2][2];
     bool attr_set_wideq;
     cudaStream_t copy_stream;           // simjoin_run_host: uploads of Q slices overlap the joins of earlier slices
-    cudaEvent_t copy_ev[66];
+    cudaEvent_t copy_ev[MAX_HOST_SLICES + 1];   // one per slice, plus one that orders the copy stream behind earlier work
     DevBuf jl_a, jl_buf[2];             // JL transform: level matrix, ping-pong level outputs
     DevBuf jl_p, jl_q;                  // simjoin_run_jl_l2: the reduced point sets
     DevBuf filter_out;                  // simjoin_filter_pairs: the kept pairs before they replace the list
@@ -146,39 +157,39 @@ bool encode_rows_map(const simjoin_ctx *ctx, CUtensorMap *map, const void *X, in
 
 template <bool kInt8>
 cudaError_t launch_norms(const simjoin_ctx *ctx, const void *X, int64_t rows, int32_t d, int sqrt_out, void *norms,
-                         void *minmax) {
+                         void *minmax, unsigned int *all_max = nullptr) {
     using T = typename NormAcc<kInt8>::type;
     if (rows == 0) return cudaSuccess;
     const int g = (int)((size_t)d * elem_size(ctx->dtype) / 16);
     const unsigned blocks = (unsigned)((rows + NORM_TILE_ROWS - 1) / NORM_TILE_ROWS);
     row_norms_kernel<kInt8><<<blocks, NORM_THREADS, 0, ctx->stream>>>(reinterpret_cast<const uint4 *>(X), rows, g, sqrt_out,
-                                                                     reinterpret_cast<T *>(norms), reinterpret_cast<T *>(minmax));
+                                                                     reinterpret_cast<T *>(norms), reinterpret_cast<T *>(minmax), all_max);
     return cudaGetLastError();
 }
 
-template <int DT, int KIND, bool NARROW, int KC, bool GROUPED>
+template <int DT, int KIND, bool ALT, int KC, bool GROUPED>
 cudaError_t launch_join_kc(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
                            size_t smem) {
-    auto kern = join_kernel<DT, KIND, NARROW, KC, GROUPED>;
-    if (!ctx->attr_set[DT][KIND][NARROW ? 1 : 0][KC][GROUPED ? 1 : 0]) {
+    auto kern = join_kernel<DT, KIND, ALT, KC, GROUPED>;
+    if (!ctx->attr_set[DT][KIND][ALT ? 1 : 0][KC][GROUPED ? 1 : 0]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
         if (e != cudaSuccess) return e;
-        ctx->attr_set[DT][KIND][NARROW ? 1 : 0][KC][GROUPED ? 1 : 0] = true;
+        ctx->attr_set[DT][KIND][ALT ? 1 : 0][KC][GROUPED ? 1 : 0] = true;
     }
     kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
     return cudaGetLastError();
 }
 
 // Picks the instantiation with compile-time chunk count when the run-time parameters match it.
-template <int DT, int KIND, bool NARROW = false, bool GROUPED = false>
+template <int DT, int KIND, bool ALT = false, bool GROUPED = false>
 cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
                         size_t smem) {
     const bool fast = jp.stationary && jp.epi_release && jp.last_ksteps == 4;
     if (fast && jp.kc == 1 && jp.nstages == fast_nstages(1, p_bufs(GROUPED, 1)))
-        return launch_join_kc<DT, KIND, NARROW, 1, GROUPED>(ctx, mp, mq, jp, grid, smem);
+        return launch_join_kc<DT, KIND, ALT, 1, GROUPED>(ctx, mp, mq, jp, grid, smem);
     if (fast && jp.kc == 2 && jp.nstages == fast_nstages(2, p_bufs(GROUPED, 2)))
-        return launch_join_kc<DT, KIND, NARROW, 2, GROUPED>(ctx, mp, mq, jp, grid, smem);
-    return launch_join_kc<DT, KIND, NARROW, 0, GROUPED>(ctx, mp, mq, jp, grid, smem);
+        return launch_join_kc<DT, KIND, ALT, 2, GROUPED>(ctx, mp, mq, jp, grid, smem);
+    return launch_join_kc<DT, KIND, ALT, 0, GROUPED>(ctx, mp, mq, jp, grid, smem);
 }
 
 // Chunks per row from which the join takes the long-row geometry.  Measured on B200 (n = m = 131 072, sustained,
@@ -186,14 +197,14 @@ cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorM
 // keep P resident at all.
 constexpr int LONG_MIN_KC = 4;
 // The long-row geometry (256 x 256 tiles, nothing resident, one accumulator buffer): general join kinds only.
-template <int DT, int KIND, bool NARROW, bool GROUPED = false>
+template <int DT, int KIND, bool ALT, bool GROUPED = false>
 cudaError_t launch_join_long(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
                              size_t smem) {
-    auto kern = join_kernel<DT, KIND, NARROW, 0, GROUPED, GEO_LONG>;
-    if (!ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0][GROUPED ? 1 : 0]) {
+    auto kern = join_kernel<DT, KIND, ALT, 0, GROUPED, GEO_LONG>;
+    if (!ctx->attr_set_long[DT][KIND][ALT ? 1 : 0][GROUPED ? 1 : 0]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
         if (e != cudaSuccess) return e;
-        ctx->attr_set_long[DT][KIND][NARROW ? 1 : 0][GROUPED ? 1 : 0] = true;
+        ctx->attr_set_long[DT][KIND][ALT ? 1 : 0][GROUPED ? 1 : 0] = true;
     }
     kern<<<grid, NUM_THREADS, smem, ctx->stream>>>(mp, mq, jp);
     return cudaGetLastError();
@@ -255,7 +266,7 @@ bool tile_geometry(const simjoin_ctx *ctx, int64_t n, int64_t m, int row_bytes, 
 }
 
 // Thresholds in the precision each path decides in.
-void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold) {
+void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold, int32_t d = 0) {
     jp.thr_d = threshold;
     if (i8) {
         if (kind == SIMJOIN_IP) jp.thr_i = clamp_to_i32(std::ceil(threshold));
@@ -268,6 +279,22 @@ void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold
         jp.thr_f = kind == SIMJOIN_L2 ? (float)(threshold * threshold) : (float)threshold;
         // the inner-product and cosine tests read the sign of s - b: with t = -0 a score of either zero gives +0 and passes
         if (kind != SIMJOIN_L2 && jp.thr_f == 0.f) jp.thr_f = -0.0f;
+        if (kind == SIMJOIN_L2 && d > 0) {
+            // Rounding error of the norm expansion |x|^2 + |y|^2 - 2<x,y> as the tile epilogue evaluates it, relative to
+            // |x|^2 + |y|^2, counted in fp32 roundings of at most 2^-24 each: the pre-pass adds a row's squares in at
+            // most 8 ceil(g / 32) + 5 steps (g = 16-byte words per row); the tensor core is charged two roundings of
+            // 2^-23 per 16-coordinate step on sum |x_k y_k| <= (|x|^2 + |y|^2) / 2, twice over (2<x,y>) and doubled once
+            // more for what is not known of its internal order: d / 2; the epilogue's own operations and the
+            // filter's coefficients: 16.  Measured errors are about a tenth of this.
+            const int g = d * 2 / 16;
+            const double roundings = 8.0 * ((g + 31) / 32) + 5.0 + 0.5 * d + 16.0;
+            const double eps = std::ldexp(roundings, -24);
+            jp.sel_coef = (float)eps;
+            jp.l2_xscale = (float)(1.0 - eps);
+            jp.l2_ycoef = (float)(0.5 * (1.0 - eps));
+            // the difference form's own error (about d 2^-24 relative) is far inside the 2^-10 added here
+            jp.l2_thr_filter = std::nextafterf((float)(threshold * threshold * (1.0 + 1.0 / 1024.0)), INFINITY);
+        }
     }
 }
 
@@ -278,9 +305,45 @@ int norm_mode(bool /*i8*/, simjoin_kind kind, double threshold) {
     return (float)threshold > 0.f ? 2 : 1;        // decided on the fp32 threshold the epilogue uses
 }
 
-// The join on device buffers.  Arguments were validated by the caller.
+// One launch of the brute-force join kernel in the geometry the rows call for.
+template <int DT, int KIND, bool ALT>
+cudaError_t launch_geo(simjoin_ctx *ctx, bool longk, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
+                       size_t smem) {
+    return longk ? launch_join_long<DT, KIND, ALT>(ctx, mp, mq, jp, grid, smem) : launch_join<DT, KIND, ALT>(ctx, mp, mq, jp, grid, smem);
+}
+// Both variants back to back: each reads the selection words and only the one they call for does the work.
+template <int DT, int KIND>
+cudaError_t launch_both(simjoin_ctx *ctx, bool longk, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
+                        size_t smem) {
+    const cudaError_t e = launch_geo<DT, KIND, false>(ctx, longk, mp, mq, jp, grid, smem);
+    return e != cudaSuccess ? e : launch_geo<DT, KIND, true>(ctx, longk, mp, mq, jp, grid, smem);
+}
+
+// Which variant of the join kernel runs is decided on the device from two words of the control block that a pre-pass
+// fills: int8 -- max|P|, max|Q| (the 16-bit epilogue when every score provably fits); bf16 Euclidean -- the largest
+// squared norms (candidates decided from the rows when r^2 is below what the norm expansion resolves).
+void set_selection(JoinParams &jp, bool i8, simjoin_kind kind, unsigned long long *d_ctrl) {
+    if (i8) {
+        jp.sel_mode = SEL_I8_RANGE;
+        jp.sel_words = reinterpret_cast<const unsigned int *>(d_ctrl + 2);
+    } else if (kind == SIMJOIN_L2) {
+        jp.sel_mode = SEL_L2_RADIUS;
+        jp.sel_words = reinterpret_cast<const unsigned int *>(d_ctrl + 3);
+    }
+}
+
+cudaError_t launch_maxabs(const simjoin_ctx *ctx, const void *P, long long p16, const void *Q, long long q16, unsigned long long *d_ctrl) {
+    maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(reinterpret_cast<const uint4 *>(P), p16, reinterpret_cast<const uint4 *>(Q), q16,
+                                                                 reinterpret_cast<unsigned int *>(d_ctrl + 2));
+    return cudaGetLastError();
+}
+
+// The join on device buffers.  Arguments were validated by the caller.  `fixed`: working memory provided by the caller
+// (the allocation-free entry point); otherwise the context's buffers are grown to fit.  No host round trip happens
+// between the pre-passes and the join: one stream synchronisation at the end.
 simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
-                          simjoin_kind kind, double threshold, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+                          simjoin_kind kind, double threshold, int32_t *out_pairs, uint64_t capacity, uint64_t *count,
+                          const JoinScratch *fixed = nullptr) {
     *count = 0;
     ctx->have_timing = false;
     if (n == 0 || m == 0) return SIMJOIN_OK;
@@ -308,99 +371,81 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.qpanel = q_panel_tiles(jp.QT, row_bytes, tn);
     jp.out = reinterpret_cast<int2 *>(out_pairs);
     jp.capacity = capacity;
-    jp.counter = ctx->d_ctrl;
-    jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
     jp.ioff = (int)ctx->ioff;
     jp.joff = (int)ctx->joff;
 
-    set_thresholds(jp, i8, kind, threshold);
+    set_thresholds(jp, i8, kind, threshold, d);
     jp.rows_p = P;
     jp.rows_q = Q;
     jp.row_bytes = row_bytes;
 
     const bool need_norms = kind != SIMJOIN_IP;
-    if (need_norms) {
+    JoinScratch scr;
+    if (fixed) {
+        scr = *fixed;
+    } else {
         // ny is read in 16-entry groups up to the end of the last Q tile: pad it to whole tiles
-        if (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, (size_t)jp.QT * tn * 4) || !grow(ctx->qstat, (size_t)jp.QT * 8))
+        if (need_norms && (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, (size_t)jp.QT * tn * 4) || !grow(ctx->qstat, (size_t)jp.QT * 8)))
             return SIMJOIN_ERR_CUDA;
-        jp.nx = ctx->nx.ptr;
-        jp.ny = ctx->ny.ptr;
-        jp.qstat = ctx->qstat.ptr;
+        scr = JoinScratch{ctx->nx.ptr, ctx->ny.ptr, ctx->qstat.ptr, ctx->d_ctrl, ctx->h_ctrl};
     }
+    jp.counter = scr.d_ctrl;
+    jp.status = reinterpret_cast<unsigned int *>(scr.d_ctrl + 1);
+    if (need_norms) {
+        jp.nx = scr.nx;
+        jp.ny = scr.ny;
+        jp.qstat = scr.qstat;
+    }
+    set_selection(jp, i8, kind, scr.d_ctrl);
 
     CUtensorMap mapP, mapQ;
     if (!encode_rows_map(ctx, &mapP, P, n, d, P_ROWS) || !encode_rows_map(ctx, &mapQ, Q, m, d, tn))
         return SIMJOIN_ERR_CUDA;
 
     cudaStream_t s = ctx->stream;
-    if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    // int8: if d * max|P| * max|Q| fits in 16 bits, every score does, and the packed epilogue applies
-    bool narrow = false;
-    if (i8) {
-        unsigned int *d_max = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 2);
-        const int blocks = ctx->num_sms * 8;
-        maxabs_i8_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const uint4 *>(P), (long long)n * row_bytes / 16, d_max);
-        maxabs_i8_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const uint4 *>(Q), (long long)m * row_bytes / 16, d_max + 1);
-        if (cudaGetLastError() != cudaSuccess ||
-            cudaMemcpyAsync(ctx->h_ctrl + 2, ctx->d_ctrl + 2, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-            cudaStreamSynchronize(s) != cudaSuccess) {
-            cudaGetLastError();
-            return SIMJOIN_ERR_CUDA;
-        }
-        const unsigned int *h_max = reinterpret_cast<const unsigned int *>(ctx->h_ctrl + 2);
-        narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
-    }
-    cudaEventRecord(ctx->ev[0], s);
+    const bool timed = ctx->ev[0] != nullptr;
+    // the control block keeps the previous call's contents: counter, status and selection words start at zero
+    if (cudaMemsetAsync(scr.d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (i8 && launch_maxabs(ctx, P, (long long)n * row_bytes / 16, Q, (long long)m * row_bytes / 16, scr.d_ctrl) != cudaSuccess)
+        return SIMJOIN_ERR_CUDA;
+    if (timed) cudaEventRecord(ctx->ev[0], s);
     if (need_norms) {
         const int sq = norm_mode(i8, kind, threshold);
+        unsigned int *nmax = (!i8 && kind == SIMJOIN_L2) ? reinterpret_cast<unsigned int *>(scr.d_ctrl + 3) : nullptr;
         cudaError_t e1, e2;
         if (i8) {
-            e1 = launch_norms<true>(ctx, P, n, d, sq, ctx->nx.ptr, nullptr);
-            e2 = launch_norms<true>(ctx, Q, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
+            e1 = launch_norms<true>(ctx, P, n, d, sq, scr.nx, nullptr);
+            e2 = launch_norms<true>(ctx, Q, m, d, sq, scr.ny, scr.qstat);
         } else {
-            e1 = launch_norms<false>(ctx, P, n, d, sq, ctx->nx.ptr, nullptr);
-            e2 = launch_norms<false>(ctx, Q, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
+            e1 = launch_norms<false>(ctx, P, n, d, sq, scr.nx, nullptr, nmax);
+            e2 = launch_norms<false>(ctx, Q, m, d, sq, scr.ny, scr.qstat, nmax ? nmax + 1 : nullptr);
         }
         if (e1 != cudaSuccess || e2 != cudaSuccess) return SIMJOIN_ERR_CUDA;
         // the padding of ny up to whole tiles is read (and masked) by the epilogue: keep it defined
         const size_t pad = (size_t)jp.QT * tn - (size_t)m;
-        if (pad > 0 && cudaMemsetAsync(static_cast<char *>(ctx->ny.ptr) + (size_t)m * 4, 0, pad * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        if (pad > 0 && cudaMemsetAsync(static_cast<char *>(scr.ny) + (size_t)m * 4, 0, pad * 4, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     }
-    cudaEventRecord(ctx->ev[1], s);
+    if (timed) cudaEventRecord(ctx->ev[1], s);
     const int grid = ctx->num_sms;
     cudaError_t e = cudaErrorInvalidValue;
-    if (longk) {
-        if (i8 && kind == SIMJOIN_IP && narrow) e = launch_join_long<DT_I8, KIND_IP, true>(ctx, mapP, mapQ, jp, grid, smem);
-        else if (i8 && kind == SIMJOIN_L2 && narrow) e = launch_join_long<DT_I8, KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
-        else if (i8 && kind == SIMJOIN_COS && narrow) e = launch_join_long<DT_I8, KIND_COS, true>(ctx, mapP, mapQ, jp, grid, smem);
-        else if (i8 && kind == SIMJOIN_COS) e = launch_join_long<DT_I8, KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem);
-        else if (i8 && kind == SIMJOIN_IP) e = launch_join_long<DT_I8, KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
-        else if (i8 && kind == SIMJOIN_L2) e = launch_join_long<DT_I8, KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
-        else if (!i8 && kind == SIMJOIN_IP) e = launch_join_long<DT_BF16, KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
-        else if (!i8 && kind == SIMJOIN_COS) e = launch_join_long<DT_BF16, KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem);
-        else if (!i8 && kind == SIMJOIN_L2) e = launch_join_long<DT_BF16, KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
-    } else
-    if (i8 && kind == SIMJOIN_IP && narrow) e = launch_join<DT_I8, KIND_IP, true>(ctx, mapP, mapQ, jp, grid, smem);
-    else if (i8 && kind == SIMJOIN_L2 && narrow) e = launch_join<DT_I8, KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
-    else if (i8 && kind == SIMJOIN_COS && narrow) e = launch_join<DT_I8, KIND_COS, true>(ctx, mapP, mapQ, jp, grid, smem);
-    else if (i8 && kind == SIMJOIN_COS) e = launch_join<DT_I8, KIND_COS>(ctx, mapP, mapQ, jp, grid, smem);
-    else if (i8 && kind == SIMJOIN_IP) e = launch_join<DT_I8, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
-    else if (i8 && kind == SIMJOIN_L2) e = launch_join<DT_I8, KIND_L2>(ctx, mapP, mapQ, jp, grid, smem);
-    else if (!i8 && kind == SIMJOIN_IP) e = launch_join<DT_BF16, KIND_IP>(ctx, mapP, mapQ, jp, grid, smem);
-    else if (!i8 && kind == SIMJOIN_COS) e = launch_join<DT_BF16, KIND_COS>(ctx, mapP, mapQ, jp, grid, smem);
-    else if (!i8 && kind == SIMJOIN_L2) e = launch_join<DT_BF16, KIND_L2>(ctx, mapP, mapQ, jp, grid, smem);
+    if (i8 && kind == SIMJOIN_IP) e = launch_both<DT_I8, KIND_IP>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    else if (i8 && kind == SIMJOIN_L2) e = launch_both<DT_I8, KIND_L2>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    else if (i8 && kind == SIMJOIN_COS) e = launch_both<DT_I8, KIND_COS>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    else if (!i8 && kind == SIMJOIN_IP) e = launch_geo<DT_BF16, KIND_IP, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    else if (!i8 && kind == SIMJOIN_COS) e = launch_geo<DT_BF16, KIND_COS, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    else if (!i8 && kind == SIMJOIN_L2) e = launch_both<DT_BF16, KIND_L2>(ctx, longk, mapP, mapQ, jp, grid, smem);
     if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    cudaEventRecord(ctx->ev[2], s);
-    if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (timed) cudaEventRecord(ctx->ev[2], s);
+    if (cudaMemcpyAsync(scr.h_ctrl, scr.d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) {
         cudaGetLastError();
         return SIMJOIN_ERR_CUDA;
     }
-    const unsigned int kstatus = (unsigned int)(ctx->h_ctrl[1] & 0xffffffffu);
+    const unsigned int kstatus = (unsigned int)(scr.h_ctrl[1] & 0xffffffffu);
     if (kstatus != 0) return SIMJOIN_ERR_TIMEOUT;
-    *count = ctx->h_ctrl[0];
+    *count = scr.h_ctrl[0];
     float a = 0.f, b = 0.f;
-    if (cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess &&
+    if (timed && cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess &&
         cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
         ctx->prepass_ms = need_norms ? a : 0.f;
         ctx->join_ms = b;
@@ -409,23 +454,26 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
 }
 
-// The LSH-bucketed join on device buffers of int8 rows.  Arguments were validated by the caller.
-// One bucketed join launch: instantiation by element type, kind, epilogue width and geometry.
-cudaError_t launch_bucketed(simjoin_ctx *ctx, bool i8, simjoin_kind kind, bool narrow, bool longk, const CUtensorMap &mp,
+// One bucketed join launch: instantiation by element type, kind, variant and geometry.
+cudaError_t launch_bucketed(simjoin_ctx *ctx, bool i8, simjoin_kind kind, bool longk, const CUtensorMap &mp,
                             const CUtensorMap &mq, const JoinParams &jp, size_t smem) {
     const int grid = ctx->num_sms;
-#define SJ_BUCKETED(DT, KIND, NARROW)                                                          \
-    return longk ? launch_join_long<DT, KIND, NARROW, true>(ctx, mp, mq, jp, grid, smem) \
-                 : launch_join<DT, KIND, NARROW, true>(ctx, mp, mq, jp, grid, smem)
-    if (i8 && kind == SIMJOIN_IP && narrow) { SJ_BUCKETED(DT_I8, KIND_IP, true); }
-    if (i8 && kind == SIMJOIN_IP) { SJ_BUCKETED(DT_I8, KIND_IP, false); }
-    if (i8 && kind == SIMJOIN_L2 && narrow) { SJ_BUCKETED(DT_I8, KIND_L2, true); }
-    if (i8 && kind == SIMJOIN_L2) { SJ_BUCKETED(DT_I8, KIND_L2, false); }
-    if (i8 && kind == SIMJOIN_COS && narrow) { SJ_BUCKETED(DT_I8, KIND_COS, true); }
-    if (i8 && kind == SIMJOIN_COS) { SJ_BUCKETED(DT_I8, KIND_COS, false); }
-    if (!i8 && kind == SIMJOIN_IP) { SJ_BUCKETED(DT_BF16, KIND_IP, false); }
-    if (!i8 && kind == SIMJOIN_COS) { SJ_BUCKETED(DT_BF16, KIND_COS, false); }
-    if (!i8 && kind == SIMJOIN_L2) { SJ_BUCKETED(DT_BF16, KIND_L2, false); }
+#define SJ_BUCKETED(DT, KIND, ALT)                                                          \
+    (longk ? launch_join_long<DT, KIND, ALT, true>(ctx, mp, mq, jp, grid, smem) \
+           : launch_join<DT, KIND, ALT, true>(ctx, mp, mq, jp, grid, smem))
+    // where the device selects the variant (int8; bf16 Euclidean) both are launched and one returns at once
+#define SJ_BUCKETED_BOTH(DT, KIND)                                   \
+    {                                                                \
+        const cudaError_t e = SJ_BUCKETED(DT, KIND, false);          \
+        return e != cudaSuccess ? e : SJ_BUCKETED(DT, KIND, true);   \
+    }
+    if (i8 && kind == SIMJOIN_IP) SJ_BUCKETED_BOTH(DT_I8, KIND_IP)
+    if (i8 && kind == SIMJOIN_L2) SJ_BUCKETED_BOTH(DT_I8, KIND_L2)
+    if (i8 && kind == SIMJOIN_COS) SJ_BUCKETED_BOTH(DT_I8, KIND_COS)
+    if (!i8 && kind == SIMJOIN_IP) return SJ_BUCKETED(DT_BF16, KIND_IP, false);
+    if (!i8 && kind == SIMJOIN_COS) return SJ_BUCKETED(DT_BF16, KIND_COS, false);
+    if (!i8 && kind == SIMJOIN_L2) SJ_BUCKETED_BOTH(DT_BF16, KIND_L2)
+#undef SJ_BUCKETED_BOTH
 #undef SJ_BUCKETED
     return cudaErrorInvalidValue;
 }
@@ -484,7 +532,8 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
     jp.ioff = (int)ctx->ioff;
     jp.joff = (int)ctx->joff;
-    set_thresholds(jp, i8, kind, threshold);
+    set_thresholds(jp, i8, kind, threshold, d);
+    set_selection(jp, i8, kind, ctx->d_ctrl);
     jp.rows_p = ctx->lsh_sorted_p.ptr;      // the regrouped rows, addressed by regrouped position
     jp.rows_q = ctx->lsh_sorted_q.ptr;
     jp.row_bytes = row_bytes;
@@ -508,21 +557,10 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
 
     cudaStream_t s = ctx->stream;
     if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    // int8: 16-bit epilogue when every score provably fits (as in the brute-force join)
-    bool narrow = false;
-    if (i8) {
-        unsigned int *d_max = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 2);
-        maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(P), (long long)n * d / 16, d_max);
-        maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, s>>>(reinterpret_cast<const uint4 *>(Q), (long long)m * d / 16, d_max + 1);
-        if (cudaGetLastError() != cudaSuccess ||
-            cudaMemcpyAsync(ctx->h_ctrl + 2, ctx->d_ctrl + 2, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-            cudaStreamSynchronize(s) != cudaSuccess) {
-            cudaGetLastError();
-            return SIMJOIN_ERR_CUDA;
-        }
-        const unsigned int *h_max = reinterpret_cast<const unsigned int *>(ctx->h_ctrl + 2);
-        narrow = (double)d * (double)h_max[0] * (double)h_max[1] <= 32767.0;
-    }
+    // the variant (16-bit epilogue for int8, row-decided candidates for small bf16 radii) is selected on the device, as in
+    // the brute-force join; the norm kinds' pre-pass runs once per repetition on the regrouped rows and folds the same
+    // maxima into the selection words every time
+    if (i8 && launch_maxabs(ctx, P, (long long)n * d / 16, Q, (long long)m * d / 16, ctx->d_ctrl) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     if (need_norms && cudaMemsetAsync(static_cast<char *>(ctx->ny.ptr) + (size_t)m * 4, 0, (ny_entries - (size_t)m) * 4, s) != cudaSuccess)
         return SIMJOIN_ERR_CUDA;
 
@@ -580,14 +618,15 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
                 e1 = launch_norms<true>(ctx, ctx->lsh_sorted_p.ptr, n, d, sq, ctx->nx.ptr, nullptr);
                 e2 = launch_norms<true>(ctx, ctx->lsh_sorted_q.ptr, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
             } else {
-                e1 = launch_norms<false>(ctx, ctx->lsh_sorted_p.ptr, n, d, sq, ctx->nx.ptr, nullptr);
-                e2 = launch_norms<false>(ctx, ctx->lsh_sorted_q.ptr, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
+                unsigned int *nmax = kind == SIMJOIN_L2 ? reinterpret_cast<unsigned int *>(ctx->d_ctrl + 3) : nullptr;
+                e1 = launch_norms<false>(ctx, ctx->lsh_sorted_p.ptr, n, d, sq, ctx->nx.ptr, nullptr, nmax);
+                e2 = launch_norms<false>(ctx, ctx->lsh_sorted_q.ptr, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr, nmax ? nmax + 1 : nullptr);
             }
             if (e1 != cudaSuccess || e2 != cudaSuccess) return SIMJOIN_ERR_CUDA;
         }
         if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
         jp.rep = l;
-        if (launch_bucketed(ctx, i8, kind, narrow, longk, mapP, mapQ, jp, smem) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        if (launch_bucketed(ctx, i8, kind, longk, mapP, mapQ, jp, smem) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     }
     cudaEventRecord(ctx->ev[2], s);
     if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
@@ -920,21 +959,29 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
     if (qb > (64u << 20)) slice_rows = (int64_t)(((32u << 20) / row_bytes + TILE_N - 1) / TILE_N * TILE_N);
     else if (ob >= (64u << 20) && m >= 8 * 4096) slice_rows = ((m + 7) / 8 + LONG_TN - 1) / LONG_TN * LONG_TN;
     const int nslices = (int)((m + slice_rows - 1) / slice_rows);
-    if (nslices > 1 && nslices <= (int)(sizeof ctx->copy_ev / sizeof ctx->copy_ev[0])) {
+    static_assert(sizeof(((simjoin_ctx *)nullptr)->copy_ev) / sizeof(cudaEvent_t) == MAX_HOST_SLICES + 1, "one event per slice and one more");
+    if (nslices > 1 && nslices <= MAX_HOST_SLICES) {
         if (!ctx->copy_stream && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return SIMJOIN_ERR_CUDA;
         for (int q = 0; q <= nslices; ++q)
             if (!ctx->copy_ev[q] && cudaEventCreateWithFlags(&ctx->copy_ev[q], cudaEventDisableTiming) != cudaSuccess) return SIMJOIN_ERR_CUDA;
         cudaStream_t cs = ctx->copy_stream;
+        // Nothing the caller passes may be in use after the call returns: an error exit waits for the copies
+        // already enqueued from the caller's buffers.
+        auto fail = [&](simjoin_status code) {
+            cudaStreamSynchronize(cs);
+            cudaGetLastError();
+            return code;
+        };
         // the staging buffers may still be in use by earlier work on the context's stream
         if (cudaEventRecord(ctx->copy_ev[nslices], s) != cudaSuccess || cudaStreamWaitEvent(cs, ctx->copy_ev[nslices], 0) != cudaSuccess)
-            return SIMJOIN_ERR_CUDA;
-        if (cudaMemcpyAsync(ctx->stage_p.ptr, P_host, pb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+            return fail(SIMJOIN_ERR_CUDA);
+        if (cudaMemcpyAsync(ctx->stage_p.ptr, P_host, pb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return fail(SIMJOIN_ERR_CUDA);
         for (int q = 0; q < nslices; ++q) {
             const int64_t r0 = q * slice_rows, rows = (m - r0 < slice_rows) ? m - r0 : slice_rows;
             if (cudaMemcpyAsync(static_cast<char *>(ctx->stage_q.ptr) + (size_t)r0 * row_bytes, static_cast<const char *>(Q_host) + (size_t)r0 * row_bytes,
                                 (size_t)rows * row_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
                 cudaEventRecord(ctx->copy_ev[q], cs) != cudaSuccess)
-                return SIMJOIN_ERR_CUDA;
+                return fail(SIMJOIN_ERR_CUDA);
         }
         const long long joff0 = ctx->joff;
         uint64_t total = 0;
@@ -1192,33 +1239,30 @@ constexpr int NA_MAX_DEVICES = 64;
 struct NoAllocDevice {
     bool ready;
     unsigned char *scratch;   // device address of g_noalloc_scratch on this device
-    int sms, smem_optin;
-    bool attr_set[2][4][2][3][2];
+    // A context that owns nothing (no buffers, no events, no second stream): it carries the device's limits and the
+    // "kernel attribute already set" flags from call to call; dtype and stream are filled in per call.
+    simjoin_ctx ctx;
 };
 NoAllocDevice g_na_dev[NA_MAX_DEVICES];
-EncodeTiledFn g_na_encode = nullptr;
 
 // Once per device, with that device current.
 simjoin_status noalloc_setup(int device) {
     NoAllocDevice &nd = g_na_dev[device];
     if (nd.ready) return SIMJOIN_OK;
-    int major = 0;
+    int major = 0, sms = 0, smem = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
-        cudaDeviceGetAttribute(&nd.sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
-        cudaDeviceGetAttribute(&nd.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
         cudaGetLastError();
         return SIMJOIN_ERR_CUDA;
     }
     if (major != 10) return SIMJOIN_ERR_ARCH;
-    if (!g_na_encode) {
-        void *fn = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess || !fn) {
-            cudaGetLastError();
-            return SIMJOIN_ERR_CUDA;
-        }
-        g_na_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn) {
+        cudaGetLastError();
+        return SIMJOIN_ERR_CUDA;
     }
     void *ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
@@ -1226,7 +1270,11 @@ simjoin_status noalloc_setup(int device) {
         return SIMJOIN_ERR_CUDA;
     }
     nd.scratch = static_cast<unsigned char *>(ptr);
-    std::memset(nd.attr_set, 0, sizeof nd.attr_set);
+    nd.ctx = simjoin_ctx{};
+    nd.ctx.device = device;
+    nd.ctx.num_sms = sms;
+    nd.ctx.max_smem_optin = smem;
+    nd.ctx.encode = reinterpret_cast<EncodeTiledFn>(fn);
     nd.ready = true;
     return SIMJOIN_OK;
 }
@@ -1238,14 +1286,12 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
                                    int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
     if (dtype != SIMJOIN_I8 && dtype != SIMJOIN_BF16) return SIMJOIN_ERR_ARG;
     if (device < 0 || device >= NA_MAX_DEVICES) return SIMJOIN_ERR_ARG;
-    // a stack context carries dtype / stream / limits to the helpers; it owns nothing
-    simjoin_ctx tmp{};
-    tmp.dtype = dtype;
-    tmp.device = device;
-    tmp.stream = static_cast<cudaStream_t>(cuda_stream);
-    tmp.ioff = tmp.joff = 0;
-    simjoin_status st = check_join_args(&tmp, P, n, Q, m, d, kind, threshold, out_pairs, capacity, count);
-    if (st != SIMJOIN_OK) return st;
+    {
+        simjoin_ctx probe{};       // argument checks only need the element type (offsets are zero)
+        probe.dtype = dtype;
+        const simjoin_status st = check_join_args(&probe, P, n, Q, m, d, kind, threshold, out_pairs, capacity, count);
+        if (st != SIMJOIN_OK) return st;
+    }
     if ((uint64_t)n > NA_ROWS || (uint64_t)m > NA_ROWS) return SIMJOIN_ERR_UNSUPPORTED;   // beyond the static scratch
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
@@ -1255,77 +1301,21 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     if (device >= ndev) return SIMJOIN_ERR_ARG;
     DeviceGuard guard(device);
     if (!guard.ok) return SIMJOIN_ERR_CUDA;
-    st = noalloc_setup(device);
+    simjoin_status st = noalloc_setup(device);
     if (st != SIMJOIN_OK) return st;
     NoAllocDevice &nd = g_na_dev[device];
     if ((n > 0 && !is_device_ptr(P, device)) || (m > 0 && !is_device_ptr(Q, device))) return SIMJOIN_ERR_ARG;
     if (capacity > 0 && !is_device_ptr(out_pairs, device)) return SIMJOIN_ERR_ARG;
     if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
-    *count = 0;
-    if (n == 0 || m == 0) return SIMJOIN_OK;
-    tmp.num_sms = nd.sms;
-    tmp.max_smem_optin = nd.smem_optin;
-    tmp.encode = g_na_encode;
-    std::memcpy(tmp.attr_set, nd.attr_set, sizeof nd.attr_set);
-
-    const bool i8 = dtype == SIMJOIN_I8;
-    const size_t es = elem_size(dtype);
-    const int row_bytes = (int)(d * es);
-    JoinParams jp;
-    size_t smem = 0;
-    if (!tile_geometry(&tmp, n, m, row_bytes, es, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
-    jp.PB = (int)((n + P_ROWS - 1) / P_ROWS);
-    jp.QT = (int)((m + TILE_N - 1) / TILE_N);
-    jp.qpanel = q_panel_tiles(jp.QT, row_bytes);
-    jp.out = reinterpret_cast<int2 *>(out_pairs);
-    jp.capacity = capacity;
-    unsigned long long *ctrl = reinterpret_cast<unsigned long long *>(nd.scratch + NA_OFF_CTRL);
-    jp.counter = ctrl;
-    jp.status = reinterpret_cast<unsigned int *>(ctrl + 1);
-    set_thresholds(jp, i8, kind, threshold);
-    jp.rows_p = P;
-    jp.rows_q = Q;
-    jp.row_bytes = row_bytes;
-    jp.nx = nd.scratch + NA_OFF_NX;
-    jp.ny = nd.scratch + NA_OFF_NY;
-    jp.qstat = nd.scratch + NA_OFF_QSTAT;
-
-    CUtensorMap mapP, mapQ;
-    if (!encode_rows_map(&tmp, &mapP, P, n, d, P_ROWS) || !encode_rows_map(&tmp, &mapQ, Q, m, d, TILE_N))
-        return SIMJOIN_ERR_CUDA;
-    cudaStream_t s = tmp.stream;
-    // the array keeps the previous call's contents: the counter / status block must start at zero
-    if (cudaMemsetAsync(ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    if (kind != SIMJOIN_IP) {
-        const int sq = norm_mode(i8, kind, threshold);
-        cudaError_t e1, e2;
-        if (i8) {
-            e1 = launch_norms<true>(&tmp, P, n, d, sq, const_cast<void *>(jp.nx), nullptr);
-            e2 = launch_norms<true>(&tmp, Q, m, d, sq, const_cast<void *>(jp.ny), const_cast<void *>(jp.qstat));
-        } else {
-            e1 = launch_norms<false>(&tmp, P, n, d, sq, const_cast<void *>(jp.nx), nullptr);
-            e2 = launch_norms<false>(&tmp, Q, m, d, sq, const_cast<void *>(jp.ny), const_cast<void *>(jp.qstat));
-        }
-        if (e1 != cudaSuccess || e2 != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    }
-    cudaError_t e = cudaErrorInvalidValue;
-    if (i8 && kind == SIMJOIN_IP) e = launch_join<DT_I8, KIND_IP>(&tmp, mapP, mapQ, jp, nd.sms, smem);
-    else if (i8 && kind == SIMJOIN_L2) e = launch_join<DT_I8, KIND_L2>(&tmp, mapP, mapQ, jp, nd.sms, smem);
-    else if (i8 && kind == SIMJOIN_COS) e = launch_join<DT_I8, KIND_COS>(&tmp, mapP, mapQ, jp, nd.sms, smem);
-    else if (!i8 && kind == SIMJOIN_IP) e = launch_join<DT_BF16, KIND_IP>(&tmp, mapP, mapQ, jp, nd.sms, smem);
-    else if (!i8 && kind == SIMJOIN_COS) e = launch_join<DT_BF16, KIND_COS>(&tmp, mapP, mapQ, jp, nd.sms, smem);
-    else if (!i8 && kind == SIMJOIN_L2) e = launch_join<DT_BF16, KIND_L2>(&tmp, mapP, mapQ, jp, nd.sms, smem);
-    std::memcpy(nd.attr_set, tmp.attr_set, sizeof nd.attr_set);
-    if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    nd.ctx.dtype = dtype;
+    nd.ctx.stream = static_cast<cudaStream_t>(cuda_stream);
+    // The same code path as simjoin_run from here on -- same geometry choice, pre-passes and kernel instantiations --
+    // with its working memory in the fixed array (n, m <= NA_ROWS: whole tiles of Q never pass the end of ny) and the
+    // counter read back into two words on this stack.
     unsigned long long host_ctrl[2] = {0, 0};
-    if (cudaMemcpyAsync(host_ctrl, ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaStreamSynchronize(s) != cudaSuccess) {
-        cudaGetLastError();
-        return SIMJOIN_ERR_CUDA;
-    }
-    if ((host_ctrl[1] & 0xffffffffu) != 0) return SIMJOIN_ERR_TIMEOUT;
-    *count = host_ctrl[0];
-    return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
+    const JoinScratch scr{nd.scratch + NA_OFF_NX, nd.scratch + NA_OFF_NY, nd.scratch + NA_OFF_QSTAT,
+                          reinterpret_cast<unsigned long long *>(nd.scratch + NA_OFF_CTRL), host_ctrl};
+    return run_device(&nd.ctx, P, n, Q, m, d, kind, threshold, out_pairs, capacity, count, &scr);
 }
 
 const char *simjoin_strerror(simjoin_status status) {

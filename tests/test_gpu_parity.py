@@ -13,7 +13,7 @@ from paper_2006_12608_b200 import build
 from paper_2006_12608_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
-BAND_REL = 1e-2      # the band half-width relative to |threshold| (spec tolerance)
+BAND_REL = 1e-2      # the band half-width relative to |threshold| (the stated tolerance)
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -262,6 +262,34 @@ def test_offsets_shift_emitted_indices(ctx_i8):
     assert ctx_i8.simjoin_set_offsets(-1, 0) == B.SIMJOIN_ERR_ARG
 
 
+@pytest.mark.parametrize("world", [2, 3, 8])
+def test_row_block_shards_on_the_gpu_union_to_the_whole_join(ctx_i8, ctx_bf16, world):
+    """Theorem 1's block decomposition through the CUDA path: the row blocks of `sharding.row_block`, joined one after
+    another with simjoin_set_offsets(start, 0) -- what each rank of a sharded run does on its own GPU -- concatenate to
+    the oracle's whole join (int8 exact, bf16 inside the band), ragged n."""
+    from paper_2006_12608_b200 import sharding
+    w = W.make_workload(4, n=3001, m=1700, planted=400)
+    wb = W.make_workload(2, n=2003, m=1500, planted=300)
+    for ctx, wl, exact in ((ctx_i8, w, True), (ctx_bf16, wb, False)):
+        parts, total = [], 0
+        try:
+            for rank in range(world):
+                start, rows = sharding.row_block(wl.n, world, rank)
+                assert ctx.simjoin_set_offsets(start, 0) == B.SIMJOIN_OK
+                pairs, cnt = gpu_join(ctx, wl.P[start:start + rows], wl.Q, wl.kind, wl.threshold)
+                assert len(pairs) == cnt and (cnt == 0 or (pairs[:, 0].min() >= start and pairs[:, 0].max() < start + rows))
+                parts.append(pairs)
+                total += cnt
+        finally:
+            assert ctx.simjoin_set_offsets(0, 0) == B.SIMJOIN_OK
+        allp = np.concatenate(parts)
+        if exact:
+            assert_exact(allp, total, wl.P, wl.Q, wl.kind, wl.threshold)
+        else:
+            assert_band(allp, total, wl.P, wl.Q, wl.kind, wl.threshold)
+        assert np.isin(keys(wl.planted), keys(allp)).all()
+
+
 def test_bad_arguments_are_rejected_before_launch(ctx_i8, ctx_bf16):
     P = B.to_device(W.random_points("i8", 64, 64, 17))
     out = torch.zeros((8, 2), dtype=torch.int32, device="cuda:0")
@@ -434,6 +462,32 @@ def test_cfg5_reduced(ctx_bf16, reading):
         assert np.all(w.labels_p[pairs[:, 0]] == w.labels_q[pairs[:, 1]])
     else:
         assert cnt == 0
+
+
+@pytest.mark.parametrize("d", [64, 1024, 2048])
+@pytest.mark.parametrize("r", [0.05, 0.0, 2.0])
+def test_bf16_l2_radius_far_below_the_norms(ctx_bf16, d, r):
+    """N(0,1) rows (|x|^2 about d) with planted equal and near-equal rows, and radii whose square is far below what
+    |x|^2 + |y|^2 - 2<x,y> resolves in fp32: the join must still be inside the band of the oracle's difference-form
+    distances (equal rows at r = 0; rows one or two bf16 steps apart in a single coordinate, 0.016 to 0.031, at
+    r = 0.05).  d = 64 at r = 2 stays on the norm-expansion path, the others are decided from the rows."""
+    rng = np.random.default_rng(d)
+    n, m = 700 + 13, 900 + 5
+    Pf = rng.standard_normal((n, d)).astype(np.float32)
+    Qf = rng.standard_normal((m, d)).astype(np.float32)
+    P, Q = W.f32_to_bf16_bits(Pf), W.f32_to_bf16_bits(Qf)
+    Q[3:603:3] = P[:200]                                   # equal rows
+    # near-equal rows: one coordinate of value v moved by one or two bf16 steps (2^-8 |v| each: 0.004 .. 0.03 apart)
+    for t, (i, j) in enumerate(zip(range(200, 400), range(4, 604, 3))):
+        row = P[i].copy()
+        c = int(np.argmax(W.bf16_bits_to_f32(row) * (1 if t % 2 else -1)))
+        row[c] += 1 + (t % 3 == 0)
+        Q[j] = row
+    pairs, cnt = gpu_join(ctx_bf16, P, Q, "l2", r, capacity=1 << 20)
+    assert_band(pairs, cnt, P, Q, "l2", r)
+    assert cnt >= 200
+    got = set(map(tuple, pairs.tolist()))
+    assert all((i, 3 + 3 * i) in got for i in range(200)), "an equal pair is missing"
 
 
 def test_repeated_runs_give_the_same_set(ctx_bf16):

@@ -1,8 +1,9 @@
 """Randomised parity: a few hundred seeded cases over element type, kind, brute force / LSH, row length (all three tile
 geometries, partial chunks), ragged row counts and value ranges, each compared with the oracle (int8: the exact pair set;
-bf16: inside the threshold band); half of the cases also run the pair filter on a random candidate list.  Thresholds are taken from a sample of the oracle's scores so that every case has
-hits.  One ill-conditioned corner is left out on purpose: a bf16 Euclidean radius far below the rows' norms, where
-|x|^2 + |y|^2 - 2<x,y> cancels in fp32 beyond what a band relative to r can absorb."""
+bf16: inside the threshold band); half of the cases also run the pair filter on a random candidate list.  Thresholds are
+taken from a sample of the oracle's scores so that every case has hits; bf16 Euclidean radii go down to whatever the
+sample's low tail gives, including radii far below the rows' norms (small point sets, where the sample meets the planted
+equal rows), which the join decides from the rows in the difference form."""
 import numpy as np
 import pytest
 import torch
@@ -51,8 +52,8 @@ def test_random_cases_match_the_oracle(seed):
             if kind == "l2":
                 dist = np.sqrt(np.maximum(sc, 0.0)) if dtype == "i8" else sc
                 t = float(np.quantile(dist, 0.002))
-                if dtype == "bf16":
-                    t = max(t, 0.6 * float(np.median(dist)))    # keep the radius well above the fp32 cancellation floor
+                if dtype == "bf16" and rng.random() < 0.25:
+                    t = float(rng.choice([0.0, 1e-3, 0.05, 0.3]))   # radii far below the norms: equal and near-equal rows only
             else:
                 t = float(np.quantile(sc, 0.998))
             ctx = ctxs[dtype]
