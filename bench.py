@@ -77,18 +77,29 @@ class ClockSampler:
             pass
         self.proc = None
         self.lines = []
+        self.first = 0
         self.thread = None
 
-    def start(self):
+    def start(self, wait_first: float = 3.0):
+        """Start sampling every 50 ms and wait (at most `wait_first` seconds) for the first sample, so that a short
+        timed region is not over before nvidia-smi has come up; samples taken before mark() are dropped."""
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
         self.thread = threading.Thread(target=self._read, daemon=True)
         self.thread.start()
+        t0 = time.perf_counter()
+        while not self.lines and time.perf_counter() - t0 < wait_first:
+            time.sleep(0.01)
+        self.mark()
+
+    def mark(self):
+        """The timed region starts now: forget what was sampled before."""
+        self.first = len(self.lines)
 
     def _read(self):
         for line in self.proc.stdout:
@@ -106,7 +117,7 @@ class ClockSampler:
             self.thread.join(timeout=2)
         sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.lines:
+        for line in self.lines[self.first:]:
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 6:
                 continue
@@ -316,6 +327,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="skip the per_config block (configurations 1, 2, 3, 5 at full size) and the int8 library peak")
+    ap.add_argument("--per-config-seconds", type=float, default=0.6, help="length of each per_config timed region")
     ap.add_argument("--n", type=int, default=None, help="override the row count of P (profiling / experiments)")
     ap.add_argument("--m", type=int, default=None, help="override the row count of Q")
     ap.add_argument("--planted", type=int, default=None)
@@ -484,7 +498,7 @@ def measure_e2e(args, ctx, w, capacity, cnt, world, dev, sync_all):
     hP = torch.from_numpy(w.P.view(np.int16) if w.P.dtype == np.uint16 else w.P).pin_memory()
     hQ = torch.from_numpy(w.Q.view(np.int16) if w.Q.dtype == np.uint16 else w.Q).pin_memory()
     hout = torch.empty((capacity, 2), dtype=torch.int32).pin_memory()
-    e2e_steps = max(1, min(args.steps, 5))
+    e2e_steps = getattr(args, "e2e_steps", None) or max(1, min(args.steps, 5))
 
     def e2e_step():
         st, c = ctx.simjoin_run_host(hP, w.n, hQ, w.m, w.d, w.kind, w.threshold, hout, capacity)
@@ -509,23 +523,155 @@ def measure_e2e(args, ctx, w, capacity, cnt, world, dev, sync_all):
             "d2h_bytes_per_step": int(cnt * 8 + 16), "steps": e2e_steps}
 
 
+def roofline_of(w, kernel_ms, region_ms, clocks, peaks, int8_peak=None):
+    """Roofline entry of the join kernel for workload w.  `frac` follows the measured-peak rule: the measured cuBLAS
+    bf16 rate (sustained for a timed region of a quarter second and more, which runs at the power cap; burst below),
+    times the nominal 2:1 ratio for int8.  That denominator is a library's rate, not the chip's ceiling, so three
+    other readings go beside it: the share of the nominal dense peak, of the ceiling at the SM clock actually sampled
+    (148 SMs x 8192 int8 (4096 bf16) multiply-adds per clock), and of an int8 library GEMM measured in this run."""
+    achieved = w.ops / (kernel_ms * 1e-3) / 1e12
+    ratio = 2.0 if w.dtype == "i8" else 1.0
+    sustained = region_ms >= 250.0
+    peak_key = "bf16_tflops_sustained" if sustained else "bf16_tflops"
+    peak = peaks[peak_key] * ratio
+    r = {"bound": "tensor", "kernel": "join_kernel", "achieved": achieved, "peak": peak, "unit": "TOP/s",
+         "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.cfg_id) if (w.n, w.m) == (W.CONFIGS[w.cfg_id]["n"], W.CONFIGS[w.cfg_id]["m"]) else None,
+         "peak_source": f"{peaks['source']}: cuBLAS bf16 {'sustained' if sustained else 'burst'} {peaks[peak_key]} TFLOP/s"
+                        + (" x 2 (nominal int8:bf16 ratio)" if ratio == 2.0 else ""),
+         "frac_of_nominal": achieved / NOMINAL_TOPS[w.dtype], "kernel_ms": kernel_ms}
+    r["traffic_source"] = ("one-pass ncu capture of the full-size launch, profiles/join_kernel_dram_traffic_cfg4_full.md "
+                           "(a constant of this file, not observed by this run)") if r["traffic"] else None
+    if clocks.get("sm_mhz"):
+        per_clk = 148 * (8192 if w.dtype == "i8" else 4096) * 2
+        r["frac_of_clock_ceiling"] = achieved / (per_clk * clocks["sm_mhz"] * 1e6 / 1e12)
+    if int8_peak and "burst_tops" in int8_peak and w.dtype == "i8":
+        r["frac_of_int8_library_peak"] = achieved / int8_peak["sustained_tops" if sustained else "burst_tops"]
+    return r
+
+
+def measure_int8_library_peak(seconds: float = 4.0):
+    """An int8 library GEMM on this GPU, measured the way the bf16 peaks were: torch._int_mm on 8192^3 ternary data,
+    best of 10 single calls (burst) and back-to-back calls for `seconds` (sustained, at the power cap)."""
+    import torch
+    try:
+        N = 8192
+        gen = torch.Generator(device="cuda").manual_seed(7)
+        a = torch.randint(-1, 2, (N, N), generator=gen, device="cuda", dtype=torch.int8)
+        b = torch.randint(-1, 2, (N, N), generator=gen, device="cuda", dtype=torch.int8)
+        ops = 2.0 * N * N * N
+        for _ in range(3):
+            torch._int_mm(a, b)
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch._int_mm(a, b)
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        reps = max(10, int(seconds * 1e3 / best))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            torch._int_mm(a, b)
+        e1.record()
+        torch.cuda.synchronize()
+        return {"burst_tops": ops / (best * 1e-3) / 1e12, "sustained_tops": ops * reps / (e0.elapsed_time(e1) * 1e-3) / 1e12,
+                "how": f"torch._int_mm {N}^3, ternary int8 data: best of 10 calls; {reps} calls back to back"}
+    except Exception as exc:                       # the library call is context, never a reason to lose the line
+        return {"unavailable": f"{type(exc).__name__}: {exc}"}
+
+
+def measure_side_config(cfg_id, args, peaks, int8_peak, min_seconds):
+    """One of the other configurations at full size, measured like the headline one: warm-up, a result check, a timed
+    region of at least `min_seconds` (so that the clock sampler sees it), the kernel's own CUDA-event time, and a short
+    end-to-end leg through simjoin_run_host."""
+    import torch
+    from paper_2006_12608_b200 import binding as B
+    w = W.make_workload(cfg_id, sigma_reading=args.sigma_reading)
+    dev = torch.device("cuda", 0)
+    dP, dQ = B.to_device(w.P, dev), B.to_device(w.Q, dev)
+    same_cluster = None
+    if w.cfg_id == 5 and args.sigma_reading == "radial":
+        ncl = int(max(w.labels_p.max(), w.labels_q.max())) + 1
+        same_cluster = int(np.sum(np.bincount(w.labels_p, minlength=ncl).astype(np.int64)
+                                  * np.bincount(w.labels_q, minlength=ncl).astype(np.int64)))
+    capacity = int(same_cluster * 1.05) if same_cluster else max(4 * len(w.planted), 1 << 20)
+    out = torch.empty((capacity, 2), dtype=torch.int32, device=dev)
+    ctx = B.Simjoin(w.dtype, 0)
+
+    def step():
+        st, c = ctx.simjoin_run(dP, w.n, dQ, w.m, w.d, w.kind, w.threshold, out, capacity)
+        if st != B.SIMJOIN_OK:
+            raise RuntimeError(f"simjoin_run (config {cfg_id}): {B.strerror(st)}")
+        return c
+
+    cnt = 0
+    for _ in range(3):
+        cnt = step()
+    # step time after the warm-up (first calls allocate and set kernel attributes), for sizing the timed region
+    reps, t0 = 0, time.perf_counter()
+    while reps < 2 or (time.perf_counter() - t0 < 0.02 and reps < 2000):
+        step()
+        reps += 1
+    est = (time.perf_counter() - t0) / reps
+    got = out[:cnt].cpu().numpy().astype(np.int64)
+    keys = (got[:, 0] << 32) | got[:, 1]
+    if cnt <= (1 << 24):
+        assert len(np.unique(keys)) == cnt, "duplicate pairs in the join output"
+    if len(w.planted):
+        assert np.isin((w.planted[:, 0] << 32) | w.planted[:, 1], keys).all(), "a planted pair is missing"
+    if same_cluster is not None:
+        assert cnt == same_cluster and np.all(w.labels_p[got[:, 0]] == w.labels_q[got[:, 1]])
+    del got, keys
+    steps = max(5, int(np.ceil(min_seconds / max(est, 1e-6))))
+    sampler = ClockSampler(0)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    join_ms, pre_ms = 0.0, 0.0
+    e0.record()
+    for _ in range(steps):
+        step()
+        _st, a, b = ctx.simjoin_last_kernel_ms()
+        pre_ms += a
+        join_ms += b
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    region_ms = e0.elapsed_time(e1)
+    ms_per_step = region_ms / steps
+    args_e2e = argparse.Namespace(steps=3, e2e_steps=int(min(2000, max(3, np.ceil(0.2 / max(est, 1e-6))))))
+    e2e = measure_e2e(args_e2e, ctx, w, capacity, cnt, 1, dev, torch.cuda.synchronize)
+    ctx.close()
+    entry = {"workload": w.name, "n": w.n, "m": w.m, "d": w.d, "kind": w.kind, "in_dtype": w.dtype, "threshold": w.threshold,
+             "steps": steps, "ms_per_step": ms_per_step, "kernel_ms": join_ms / steps, "prepass_ms": pre_ms / steps,
+             "value": w.ops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "pairs_found": int(cnt), "e2e": e2e, "clocks": clocks,
+             "l2": ("inputs (P+Q) larger than L2; no flush" if w.P.nbytes + w.Q.nbytes > 126e6
+                    else "inputs (P+Q) fit in L2 and are not flushed between steps")}
+    if cfg_id == 1:
+        entry["note"] = "latency-bound: one partial wave of tiles; its time is the figure, not a fraction of a peak"
+    else:
+        r = roofline_of(w, join_ms / steps, region_ms, clocks, peaks, int8_peak)
+        entry.update({k: r[k] for k in ("frac", "frac_of_nominal", "peak", "peak_source") if k in r})
+        for k in ("frac_of_clock_ceiling", "frac_of_int8_library_peak"):
+            if k in r:
+                entry[k] = r[k]
+    del dP, dQ, out
+    torch.cuda.empty_cache()
+    return entry
+
+
 def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks, e2e):
     peaks = measured_peaks()
     jm = statistics.mean(join_ms)
-    achieved = w.ops / (jm * 1e-3) / 1e12
-    ratio = 2.0 if w.dtype == "i8" else 1.0          # nominal dense int8 : bf16 rate
-    # a timed region of back-to-back launches lasting a good fraction of a second runs at the power cap:
-    # sustained peak; a few milliseconds of launches run at burst clocks: burst peak
-    sustained = ms_per_step * args.steps >= 250.0
-    peak_key = "bf16_tflops_sustained" if sustained else "bf16_tflops"
-    peak = peaks[peak_key] * ratio
-    roofline = {"bound": "tensor", "kernel": "join_kernel", "achieved": achieved, "peak": peak, "unit": "TOP/s",
-                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.cfg_id),
-                "peak_source": f"{peaks['source']}: cuBLAS bf16 {'sustained' if sustained else 'burst'} {peaks[peak_key]} TFLOP/s"
-                               + (" x 2 (nominal int8:bf16 ratio)" if ratio == 2.0 else ""),
-                "frac_of_nominal": achieved / NOMINAL_TOPS[w.dtype], "kernel_ms": jm,
-                "prepass_ms": statistics.mean(pre_ms)}
-    launches_per_step = 1 + (2 if w.kind != "ip" else 0) + (2 if w.dtype == "i8" else 0)   # join + norms + max|x|
+    side = world == 1 and not args.lsh and not args.no_per_config
+    int8_peak = measure_int8_library_peak() if side else None
+    roofline = roofline_of(w, jm, ms_per_step * args.steps, clocks, peaks, int8_peak)
+    roofline["prepass_ms"] = statistics.mean(pre_ms)
+    # the join (int8 and bf16 Euclidean: both variants are launched, one returns at once), the norm pre-pass, max|x|
+    launches_per_step = (2 if (w.dtype == "i8" or w.kind == "l2") else 1) + (2 if w.kind != "ip" else 0) + (1 if w.dtype == "i8" else 0)
     if args.lsh:
         # max|x| x2, sampled coordinates, keys x2, then per table: 2 histograms, offsets + work list, 2 scatters, 2 row
         # gathers, the join
@@ -552,6 +698,11 @@ def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks
                              "hash_ms": statistics.mean(pre_ms), "tables_ms": jm,
                              "note": "value = 2*n*m*d over the step time: the brute-force-equivalent rate of an approximate "
                                      "join, not the headline metric; precision is 1, recall as given"}
+    if int8_peak is not None:
+        line["int8_library_peak"] = int8_peak
+    if side and args.config == 4 and not size_kw(args) and not args.kind:
+        # the other four configurations at full size, each with its own clock record (the headline stays config 4)
+        line["per_config"] = {str(c): measure_side_config(c, args, peaks, int8_peak, args.per_config_seconds) for c in (1, 2, 3, 5)}
     if not args.no_cpu_baseline and world == 1 and not args.lsh:
         rows = slab_rows_for(w, 12.0)
         dt, _c, threads = oracle_slab(w, rows)

@@ -44,7 +44,9 @@ typedef enum {
     SIMJOIN_COS = 1, /* keep (i,j) when <x_i, y_j>/(|x_i| |y_j|)    >= threshold;
                         the cosine with a zero vector counts as 0                */
     SIMJOIN_L2 = 2   /* keep (i,j) when |x_i - y_j| <= threshold (threshold >= 0),
-                        evaluated as |x|^2 + |y|^2 - 2<x,y> <= threshold^2       */
+                        evaluated as |x|^2 + |y|^2 - 2<x,y> <= threshold^2; bf16
+                        radii too small for that form in fp32 are decided from
+                        the rows as sum (x - y)^2 <= threshold^2                 */
 } simjoin_kind;
 
 typedef enum {
@@ -85,7 +87,13 @@ simjoin_status simjoin_create(simjoin_ctx **ctx, simjoin_dtype dtype, int device
  *               square root and the quotient each rounded once; 0 for a zero
  *               vector) -- int8 results are exact, with no tolerance band.
  *               BF16 kinds compare fp32 scores; pairs whose exact score lies
- *               within 1e-2*|threshold| of the threshold may fall on either side.
+ *               within 1e-2*|threshold| of the threshold may fall on either side,
+ *               and only those -- at every threshold the call accepts.  (BF16/L2:
+ *               the norm expansion's fp32 rounding error, bounded from the largest
+ *               norms the pre-pass meets, is compared with 1.9 % of r^2 on the
+ *               device; when it is larger the tile test only raises candidates,
+ *               lowered by that bound, and each is decided in the difference
+ *               form from its two rows.  r = 0 returns exactly the equal rows.)
  *   out_pairs   device pointer to capacity x 2 int32, written as (i, j) rows.
  *               May be NULL when capacity == 0 (count-only mode).
  *   count       HOST pointer; receives the total number of passing pairs, even
@@ -95,7 +103,9 @@ simjoin_status simjoin_create(simjoin_ctx **ctx, simjoin_dtype dtype, int device
  * pair at most once, in unspecified order.  When *count > capacity the written
  * subset is arbitrary but valid and the call returns ERR_CAPACITY.
  * The call enqueues on the context's stream and synchronises that stream
- * before it returns.  n == 0 or m == 0 gives OK with *count = 0.
+ * once, before it returns (no host round trip in between: which variant of
+ * the kernel runs -- 16- or 32-bit int8 epilogue, BF16/L2 small-radius form --
+ * is decided on the device).  n == 0 or m == 0 gives OK with *count = 0.
  *
  * Errors, all detected before any launch: ERR_ARG (null ctx/P/Q/count, n or m
  * negative or >= 2^31, d <= 0, NaN threshold, L2 with threshold < 0, a host
@@ -279,6 +289,21 @@ simjoin_status simjoin_row_norms(simjoin_ctx *ctx, const void *X, int64_t rows, 
 simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64_t row_offset_q);
 
 /*
+ * Tuning knobs of a context; none of them changes a result.
+ *
+ *   SIMJOIN_OPT_SELECT_MIN_OPS   int8 joins of at least this many operations (2 n m d) run the max|x| pre-pass and let
+ *                                the device choose the 16-bit packed epilogue when every score provably fits 16 bits;
+ *                                smaller joins take the 32-bit epilogue unasked, which saves two steps of launch latency
+ *                                (default 2e11; 0 = always ask).  value >= 0.
+ *   SIMJOIN_OPT_KERNEL_TIMING    1 (default): simjoin_run records CUDA events around its pre-pass and its join kernel
+ *                                for simjoin_last_kernel_ms; 0: it records none (three stream operations less per call,
+ *                                which shows on joins of a few microseconds) and simjoin_last_kernel_ms reports ERR_ARG.
+ * Errors: ERR_ARG (null ctx, unknown option, NaN or out-of-range value).
+ */
+typedef enum { SIMJOIN_OPT_SELECT_MIN_OPS = 0, SIMJOIN_OPT_KERNEL_TIMING = 1 } simjoin_option;
+simjoin_status simjoin_set_option(simjoin_ctx *ctx, simjoin_option option, double value);
+
+/*
  * Device time of the kernels of the last successful simjoin_run /
  * simjoin_run_host on this context, in milliseconds, measured with CUDA events
  * on the context's stream: the norm pre-pass (0 when the kind needs none) and
@@ -306,10 +331,13 @@ simjoin_status simjoin_selftest_wait_timeout(simjoin_ctx *ctx);
  * framework owning all device memory, code on a path where an out-of-memory failure is not
  * an option.  simjoin_create / simjoin_run grow scratch with cudaMalloc; this call does not.
  * It calls no cudaMalloc, cudaFree, cudaMallocHost, event or stream creation, nor any other
- * allocating routine: the scratch of the norm pre-pass and of the join kernel (row norms,
- * per-tile norm bounds, the counter / status block) lives in a fixed array inside the
- * library's device image, about 0.5 MiB that every GPU loading the library holds until the
- * process exits.  There is no context: device, stream and dtype are arguments.
+ * allocating routine: the scratch of the pre-passes and of the join kernel (row norms,
+ * per-tile norm bounds, the counter / status / selection block) lives in a fixed array inside
+ * the library's device image, about 0.5 MiB that every GPU loading the library holds until the
+ * process exits.  There is no context: device, stream and dtype are arguments.  From the
+ * choice of the tile geometry on it is simjoin_run's own code path -- the same pre-passes,
+ * the same kernel instantiations for every row length, the same device-side choice of
+ * variant -- only the working memory differs.
  *
  * Same semantics, supported kinds and error codes as simjoin_run, with these differences:
  *   - n and m must not exceed SIMJOIN_NOALLOC_MAX_ROWS; larger inputs are rejected with

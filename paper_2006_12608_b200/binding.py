@@ -21,10 +21,11 @@ SIMJOIN_IP, SIMJOIN_COS, SIMJOIN_L2 = 0, 1, 2
 DTYPE = {"i8": SIMJOIN_I8, "bf16": SIMJOIN_BF16}
 KIND = {"ip": SIMJOIN_IP, "cos": SIMJOIN_COS, "l2": SIMJOIN_L2}
 
-EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_hamming", "simjoin_run_lsh", "simjoin_run_hamming_lsh", "simjoin_jl_transform", "simjoin_filter_pairs", "simjoin_run_jl_l2", "simjoin_row_norms", "simjoin_set_offsets",
+EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_hamming", "simjoin_run_lsh", "simjoin_run_hamming_lsh", "simjoin_jl_transform", "simjoin_filter_pairs", "simjoin_run_jl_l2", "simjoin_row_norms", "simjoin_set_offsets", "simjoin_set_option",
            "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_selftest_wait_timeout", "simjoin_destroy",
            "simjoin_strerror")
 SIMJOIN_NOALLOC_MAX_ROWS = 65536
+SIMJOIN_OPT_SELECT_MIN_OPS, SIMJOIN_OPT_KERNEL_TIMING = 0, 1
 
 _lib = None
 
@@ -70,6 +71,8 @@ def load() -> ctypes.CDLL:
     lib.simjoin_row_norms.argtypes = [vp, vp, i64, i32, vp]
     lib.simjoin_set_offsets.restype = c.c_int
     lib.simjoin_set_offsets.argtypes = [vp, i64, i64]
+    lib.simjoin_set_option.restype = c.c_int
+    lib.simjoin_set_option.argtypes = [vp, c.c_int, dbl]
     lib.simjoin_last_kernel_ms.restype = c.c_int
     lib.simjoin_last_kernel_ms.argtypes = [vp, c.POINTER(c.c_float), c.POINTER(c.c_float)]
     lib.simjoin_selftest_wait_timeout.restype = c.c_int
@@ -186,6 +189,9 @@ class Simjoin:
 
     def simjoin_set_offsets(self, row_offset_p: int, row_offset_q: int):
         return load().simjoin_set_offsets(self._h, row_offset_p, row_offset_q)
+
+    def simjoin_set_option(self, option: int, value: float):
+        return load().simjoin_set_option(self._h, int(option), float(value))
 
     def simjoin_selftest_wait_timeout(self):
         return load().simjoin_selftest_wait_timeout(self._h)

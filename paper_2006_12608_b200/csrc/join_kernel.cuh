@@ -115,6 +115,14 @@ struct JoinParams {
     const unsigned int *sel_words;
     int sel_mode;
     float sel_coef;
+    // When not null: a 64-byte control block that no launch of this call reads or writes.  The kernel zeroes it, so
+    // that the caller's next join finds its counter, status and selection words cleared without a memset of its own.
+    unsigned long long *zero_next;
+    // When not null: two words of pinned host memory that the device can write.  The last CTA to finish (a ticket in
+    // done_ticket, a zeroed word of the control block) stores the pair count and the status word there, which saves
+    // the device-to-host copy that would otherwise follow the kernel in the stream.
+    unsigned long long *host_result;
+    unsigned int *done_ticket;
     // BF16/L2, ALT: the tile test is a filter  s >= (l2_xscale |x|^2 - l2_thr_filter) / 2 + l2_ycoef |y|^2, lowered by the
     // error bound so that every pair the difference form accepts is a candidate
     float l2_xscale, l2_ycoef, l2_thr_filter;
@@ -710,6 +718,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     static_assert(DT == DT_I8 || !ALT || KIND == KIND_L2, "bf16: only the Euclidean kind has a second variant");
     // not the variant the data calls for: the other launch does the work (uniform over the grid, before any barrier
     // or tensor-memory allocation exists)
+    if (p_in.zero_next != nullptr && blockIdx.x == 0 && threadIdx.x < 8) p_in.zero_next[threadIdx.x] = 0ull;
     if (p_in.sel_mode != SEL_NONE && alt_selected(p_in) != ALT) return;
     static_assert(!LONGK || (KC == 0 && KIND != KIND_STORE), "long-row mode: general join kinds only");
     static_assert(!WIDEQ || (KC == 0 && !GROUPED && KIND == KIND_STORE), "wide-Q mode: store kind only");
@@ -1153,6 +1162,16 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     if (warp == 2) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+    if (p.host_result != nullptr && threadIdx.x == 0) {
+        // every pair of this CTA has been counted (the epilogue warps flushed before the barrier above)
+        __threadfence();
+        if (atomicAdd(p.done_ticket, 1u) == gridDim.x - 1) {
+            __threadfence();
+            p.host_result[0] = atomicAdd(p.counter, 0ull);
+            p.host_result[1] = (unsigned long long)atomicOr(p.status, 0u);
+            __threadfence_system();
+        }
     }
 }
 

@@ -32,6 +32,10 @@ struct DevBuf {
     size_t bytes = 0;
 };
 
+// Joins of fewer operations (2 n m d) than this run the 32-bit int8 epilogue without asking whether the 16-bit one
+// applies: the max|x| pre-pass and the second launch cost two more steps in the stream's dependent chain (about 13 us
+// measured on B200), which the packed epilogue's ~15 % only wins back on joins of ~90 us and more.
+constexpr double DEFAULT_SELECT_MIN_OPS = 2.0e11;
 constexpr int MAX_HOST_SLICES = 66;     // simjoin_run_host: a Q of more slices than this goes up in one piece
 
 // Device-side working memory of one join call, and the host words its result lands in.  simjoin_run takes it from the
@@ -39,8 +43,10 @@ constexpr int MAX_HOST_SLICES = 66;     // simjoin_run_host: a Q of more slices 
 struct JoinScratch {
     void *nx, *ny, *qstat;        // row terms of P (n entries) and Q (whole tiles), (min, max) of ny per 256 rows of Q
     unsigned long long *d_ctrl;   // 64 bytes: [0] pair counter, [1] status word, [2] max|P|, max|Q| (two 32-bit words, int8),
-                                  // [3] bit patterns of max|x|^2, max|y|^2 (two 32-bit words, bf16 Euclidean)
+                                  // [3] bit patterns of max|x|^2, max|y|^2 (two 32-bit words, bf16 Euclidean),
+                                  // [4] low word: ticket of finished CTAs
     unsigned long long *h_ctrl;   // host copy of words [0] and [1]
+    bool h_ctrl_mapped;           // h_ctrl is pinned memory the device can write: the kernel stores the result there
 };
 
 }  // namespace
@@ -54,8 +60,11 @@ struct simjoin_ctx {
     EncodeTiledFn encode;
     DevBuf nx, ny, qstat, pstat;        // row terms and per-tile bounds
     DevBuf stage_p, stage_q, stage_out; // device staging of simjoin_run_host
-    unsigned long long *d_ctrl;         // [0] pair counter, [1] status word (low 32 bits)
+    unsigned long long *d_ctrl;         // two 64-byte control blocks (layout: JoinScratch::d_ctrl)
     unsigned long long *h_ctrl;         // pinned mirror
+    int ctrl_clean;                     // the block that the last simjoin_run's kernel left zeroed for the next one, or -1
+    double select_min_ops;              // SIMJOIN_OPT_SELECT_MIN_OPS
+    bool kernel_timing;                 // SIMJOIN_OPT_KERNEL_TIMING
     cudaEvent_t ev[4];
     bool have_timing;
     float prepass_ms, join_ms;
@@ -387,28 +396,49 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         // ny is read in 16-entry groups up to the end of the last Q tile: pad it to whole tiles
         if (need_norms && (!grow(ctx->nx, (size_t)n * 4) || !grow(ctx->ny, (size_t)jp.QT * tn * 4) || !grow(ctx->qstat, (size_t)jp.QT * 8)))
             return SIMJOIN_ERR_CUDA;
-        scr = JoinScratch{ctx->nx.ptr, ctx->ny.ptr, ctx->qstat.ptr, ctx->d_ctrl, ctx->h_ctrl};
+        scr = JoinScratch{ctx->nx.ptr, ctx->ny.ptr, ctx->qstat.ptr, ctx->d_ctrl, ctx->h_ctrl, true};
+    }
+    // The context owns two control blocks and alternates between them: the join kernel of one call zeroes the block of
+    // the next, which then starts without a memset (one step less in the stream's dependent chain; it shows on small
+    // joins).  A call that fails, or any other entry point that uses the control block, breaks the chain, and the next
+    // call clears its block itself.
+    bool need_clear = true;
+    int cur = 0;
+    if (!fixed) {
+        if (ctx->ctrl_clean >= 0) {
+            cur = ctx->ctrl_clean;
+            need_clear = false;
+        }
+        scr.d_ctrl = ctx->d_ctrl + 8 * cur;
+        jp.zero_next = ctx->d_ctrl + 8 * (cur ^ 1);
+        ctx->ctrl_clean = -1;
     }
     jp.counter = scr.d_ctrl;
     jp.status = reinterpret_cast<unsigned int *>(scr.d_ctrl + 1);
+    if (scr.h_ctrl_mapped) {
+        jp.host_result = scr.h_ctrl;
+        jp.done_ticket = reinterpret_cast<unsigned int *>(scr.d_ctrl + 4);
+    }
     if (need_norms) {
         jp.nx = scr.nx;
         jp.ny = scr.ny;
         jp.qstat = scr.qstat;
     }
-    set_selection(jp, i8, kind, scr.d_ctrl);
+    // small int8 joins take the 32-bit epilogue unasked (see DEFAULT_SELECT_MIN_OPS)
+    const bool select_i8 = i8 && 2.0 * (double)n * (double)m * (double)d >= ctx->select_min_ops;
+    if (!i8 || select_i8) set_selection(jp, i8, kind, scr.d_ctrl);
 
     CUtensorMap mapP, mapQ;
     if (!encode_rows_map(ctx, &mapP, P, n, d, P_ROWS) || !encode_rows_map(ctx, &mapQ, Q, m, d, tn))
         return SIMJOIN_ERR_CUDA;
 
     cudaStream_t s = ctx->stream;
-    const bool timed = ctx->ev[0] != nullptr;
+    const bool timed = ctx->ev[0] != nullptr && ctx->kernel_timing;
     // the control block keeps the previous call's contents: counter, status and selection words start at zero
-    if (cudaMemsetAsync(scr.d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
-    if (i8 && launch_maxabs(ctx, P, (long long)n * row_bytes / 16, Q, (long long)m * row_bytes / 16, scr.d_ctrl) != cudaSuccess)
+    if (need_clear && cudaMemsetAsync(scr.d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (select_i8 && launch_maxabs(ctx, P, (long long)n * row_bytes / 16, Q, (long long)m * row_bytes / 16, scr.d_ctrl) != cudaSuccess)
         return SIMJOIN_ERR_CUDA;
-    if (timed) cudaEventRecord(ctx->ev[0], s);
+    if (timed && need_norms) cudaEventRecord(ctx->ev[0], s);      // (every event is a step in the stream: none without a pre-pass)
     if (need_norms) {
         const int sq = norm_mode(i8, kind, threshold);
         unsigned int *nmax = (!i8 && kind == SIMJOIN_L2) ? reinterpret_cast<unsigned int *>(scr.d_ctrl + 3) : nullptr;
@@ -428,7 +458,11 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     if (timed) cudaEventRecord(ctx->ev[1], s);
     const int grid = ctx->num_sms;
     cudaError_t e = cudaErrorInvalidValue;
-    if (i8 && kind == SIMJOIN_IP) e = launch_both<DT_I8, KIND_IP>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    if (i8 && !select_i8) {
+        if (kind == SIMJOIN_IP) e = launch_geo<DT_I8, KIND_IP, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
+        else if (kind == SIMJOIN_L2) e = launch_geo<DT_I8, KIND_L2, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
+        else e = launch_geo<DT_I8, KIND_COS, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    } else if (i8 && kind == SIMJOIN_IP) e = launch_both<DT_I8, KIND_IP>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_L2) e = launch_both<DT_I8, KIND_L2>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_COS) e = launch_both<DT_I8, KIND_COS>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (!i8 && kind == SIMJOIN_IP) e = launch_geo<DT_BF16, KIND_IP, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
@@ -436,16 +470,17 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     else if (!i8 && kind == SIMJOIN_L2) e = launch_both<DT_BF16, KIND_L2>(ctx, longk, mapP, mapQ, jp, grid, smem);
     if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
     if (timed) cudaEventRecord(ctx->ev[2], s);
-    if (cudaMemcpyAsync(scr.h_ctrl, scr.d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    if (!scr.h_ctrl_mapped && cudaMemcpyAsync(scr.h_ctrl, scr.d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) {
         cudaGetLastError();
         return SIMJOIN_ERR_CUDA;
     }
     const unsigned int kstatus = (unsigned int)(scr.h_ctrl[1] & 0xffffffffu);
     if (kstatus != 0) return SIMJOIN_ERR_TIMEOUT;
+    if (!fixed) ctx->ctrl_clean = cur ^ 1;        // the kernel has zeroed the other block
     *count = scr.h_ctrl[0];
     float a = 0.f, b = 0.f;
-    if (timed && cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess &&
+    if (timed && (!need_norms || cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess) &&
         cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
         ctx->prepass_ms = need_norms ? a : 0.f;
         ctx->join_ms = b;
@@ -556,6 +591,7 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         return SIMJOIN_ERR_CUDA;
 
     cudaStream_t s = ctx->stream;
+    ctx->ctrl_clean = -1;                         // this call uses the first control block and leaves it dirty
     if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     // the variant (16-bit epilogue for int8, row-decided candidates for small bf16 radii) is selected on the device, as in
     // the brute-force join; the norm kinds' pre-pass runs once per repetition on the regrouped rows and folds the same
@@ -715,6 +751,7 @@ simjoin_status jl_device(simjoin_ctx *ctx, const void *X, int64_t n, int32_t d, 
                                                           (levels > 2 && !grow(ctx->jl_buf[1], (size_t)n * mid_elems * 2)))))
         return SIMJOIN_ERR_CUDA;
     cudaStream_t s = ctx->stream;
+    ctx->ctrl_clean = -1;                         // this call uses the first control block and leaves it dirty
     if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     cudaEventRecord(ctx->ev[0], s);
     cudaEventRecord(ctx->ev[1], s);
@@ -785,6 +822,7 @@ simjoin_status filter_device(simjoin_ctx *ctx, const void *P, int64_t n, const v
     std::memset(&jp, 0, sizeof jp);
     set_thresholds(jp, i8, kind, threshold);
     cudaStream_t s = ctx->stream;
+    ctx->ctrl_clean = -1;                         // this call uses the first control block and leaves it dirty
     if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     // G lanes per pair (the power of two covering the row's 16-byte words), at most 16 blocks per SM (the warps then
     // stride over the list)
@@ -857,6 +895,9 @@ simjoin_status simjoin_create(simjoin_ctx **out, simjoin_dtype dtype, int device
     ctx->h_ctrl = nullptr;
     ctx->have_timing = false;
     ctx->ioff = ctx->joff = 0;
+    ctx->ctrl_clean = -1;
+    ctx->select_min_ops = DEFAULT_SELECT_MIN_OPS;
+    ctx->kernel_timing = true;
     std::memset(ctx->attr_set, 0, sizeof ctx->attr_set);
     std::memset(ctx->attr_set_long, 0, sizeof ctx->attr_set_long);
     ctx->attr_set_wideq = false;
@@ -920,6 +961,21 @@ simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64
     ctx->ioff = row_offset_p;
     ctx->joff = row_offset_q;
     return SIMJOIN_OK;
+}
+
+simjoin_status simjoin_set_option(simjoin_ctx *ctx, simjoin_option option, double value) {
+    if (!ctx || std::isnan(value)) return SIMJOIN_ERR_ARG;
+    switch (option) {
+        case SIMJOIN_OPT_SELECT_MIN_OPS:
+            if (value < 0) return SIMJOIN_ERR_ARG;
+            ctx->select_min_ops = value;
+            return SIMJOIN_OK;
+        case SIMJOIN_OPT_KERNEL_TIMING:
+            if (value != 0.0 && value != 1.0) return SIMJOIN_ERR_ARG;
+            ctx->kernel_timing = value != 0.0;
+            return SIMJOIN_OK;
+    }
+    return SIMJOIN_ERR_ARG;
 }
 
 simjoin_status simjoin_run(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
@@ -1200,6 +1256,7 @@ simjoin_status simjoin_selftest_wait_timeout(simjoin_ctx *ctx) {
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SIMJOIN_ERR_CUDA;
     cudaStream_t s = ctx->stream;
+    ctx->ctrl_clean = -1;                         // this call uses the first control block and leaves it dirty
     if (cudaMemsetAsync(ctx->d_ctrl, 0, 64, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1), 2000000LL);   // ~1 ms
     if (cudaGetLastError() != cudaSuccess ||
@@ -1314,7 +1371,7 @@ simjoin_status simjoin_run_noalloc(int device, void *cuda_stream, simjoin_dtype 
     // counter read back into two words on this stack.
     unsigned long long host_ctrl[2] = {0, 0};
     const JoinScratch scr{nd.scratch + NA_OFF_NX, nd.scratch + NA_OFF_NY, nd.scratch + NA_OFF_QSTAT,
-                          reinterpret_cast<unsigned long long *>(nd.scratch + NA_OFF_CTRL), host_ctrl};
+                          reinterpret_cast<unsigned long long *>(nd.scratch + NA_OFF_CTRL), host_ctrl, false};
     return run_device(&nd.ctx, P, n, Q, m, d, kind, threshold, out_pairs, capacity, count, &scr);
 }
 

@@ -25,7 +25,11 @@ def _built():
 
 @pytest.fixture(scope="module")
 def ctx_i8():
+    """An int8 context that asks the device for the epilogue width on every join, however small, so that the small
+    shapes below reach the max|x| pre-pass, the device-side choice and both epilogues (the default skips them on
+    joins this small: test_small_int8_joins_skip_the_epilogue_choice)."""
     c = B.Simjoin("i8", 0)
+    assert c.simjoin_set_option(B.SIMJOIN_OPT_SELECT_MIN_OPS, 0.0) == B.SIMJOIN_OK
     yield c
     c.close()
 
@@ -191,6 +195,23 @@ def test_i8_packed_16_bit_epilogue_boundary(ctx_i8):
             pairs, cnt = gpu_join(ctx_i8, P, Q, kind, t)
             assert_exact(pairs, cnt, P, Q, kind, t)
         assert (d * amp * amp <= 32767) == narrow
+
+
+def test_small_int8_joins_skip_the_epilogue_choice():
+    """The default context takes the 32-bit epilogue unasked on small joins (two launches less) and the device's
+    choice from SIMJOIN_OPT_SELECT_MIN_OPS operations on; the pair set is the oracle's either way, also when calls
+    of both sorts alternate on one context (they share the two control blocks)."""
+    P, Q = W.random_points("i8", 900, 64, 33, lo=-3, hi=3), W.random_points("i8", 1300, 64, 34, lo=-3, hi=3)
+    with B.Simjoin("i8", 0) as ctx:
+        assert ctx.simjoin_set_option(99, 1.0) == B.SIMJOIN_ERR_ARG
+        assert ctx.simjoin_set_option(B.SIMJOIN_OPT_SELECT_MIN_OPS, -1.0) == B.SIMJOIN_ERR_ARG
+        for min_ops in (None, 0.0, 1e18, 0.0, 2e11):
+            if min_ops is not None:
+                assert ctx.simjoin_set_option(B.SIMJOIN_OPT_SELECT_MIN_OPS, min_ops) == B.SIMJOIN_OK
+            for kind, t in (("ip", 30.0), ("l2", 19.0), ("cos", 0.4)):
+                pairs, cnt = gpu_join(ctx, P, Q, kind, t)
+                assert_exact(pairs, cnt, P, Q, kind, t)
+                assert cnt > 0
 
 
 def test_staged_compaction_flush_paths(ctx_i8, ctx_bf16):
