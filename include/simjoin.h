@@ -298,9 +298,17 @@ simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64
  *   SIMJOIN_OPT_KERNEL_TIMING    1 (default): simjoin_run records CUDA events around its pre-pass and its join kernel
  *                                for simjoin_last_kernel_ms; 0: it records none (three stream operations less per call,
  *                                which shows on joins of a few microseconds) and simjoin_last_kernel_ms reports ERR_ARG.
+ *   SIMJOIN_OPT_DENSE_EPILOGUE   which epilogue layout bf16 joins over rows of one or two whole 128-byte chunks run
+ *                                (d = 64 or 128): 0 = always 8 epilogue warps of 128 columns (best when pairs are rare:
+ *                                the work is row maxima); 1 = always 16 warps of 64 columns (best when most 32 x 128
+ *                                blocks of scores hold a pair: the work is element tests, bound by dependent-issue
+ *                                latency, which twice the warps hide; measured 77.5 -> 70.8 ms on 2.7e8 pairs out of
+ *                                524 288^2, +2 % on a join with 1000 pairs out of 65 536^2); 2 (default) = by the
+ *                                previous simjoin_run of the context: 16 warps after a join with at least one pair per
+ *                                two such blocks.  Other joins ignore it.
  * Errors: ERR_ARG (null ctx, unknown option, NaN or out-of-range value).
  */
-typedef enum { SIMJOIN_OPT_SELECT_MIN_OPS = 0, SIMJOIN_OPT_KERNEL_TIMING = 1 } simjoin_option;
+typedef enum { SIMJOIN_OPT_SELECT_MIN_OPS = 0, SIMJOIN_OPT_KERNEL_TIMING = 1, SIMJOIN_OPT_DENSE_EPILOGUE = 2 } simjoin_option;
 simjoin_status simjoin_set_option(simjoin_ctx *ctx, simjoin_option option, double value);
 
 /*

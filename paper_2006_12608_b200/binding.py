@@ -25,7 +25,7 @@ EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_ham
            "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_selftest_wait_timeout", "simjoin_destroy",
            "simjoin_strerror")
 SIMJOIN_NOALLOC_MAX_ROWS = 65536
-SIMJOIN_OPT_SELECT_MIN_OPS, SIMJOIN_OPT_KERNEL_TIMING = 0, 1
+SIMJOIN_OPT_SELECT_MIN_OPS, SIMJOIN_OPT_KERNEL_TIMING, SIMJOIN_OPT_DENSE_EPILOGUE = 0, 1, 2
 
 _lib = None
 

@@ -72,6 +72,15 @@ constexpr int WARP_STAGE_BYTES = 2048;                           // per epilogue
 constexpr int COLTERM_BYTES = EPI_COLS * 4;                      // per-column terms of the 128 columns under test
 constexpr int STAGE_PAIRS = (WARP_STAGE_BYTES - COLTERM_BYTES) / 8;   // pairs staged in shared memory per warp
 constexpr int STAGING_BYTES = NUM_EPI_WARPS * WARP_STAGE_BYTES;  // 16 KiB
+// The dense-output instantiations run 16 epilogue warps (EW = 16): four per TMEM lane quarter, each taking 64 of a P
+// block's 128 columns, on the same 16 KiB of staging (1 KiB per warp).  A join whose every 32 x 128 block holds hits is
+// bound by the dependent-issue latency of the element tests, which twice the warps hide; a sparse join is bound by the
+// throughput of the row maxima and is faster with 8 warps of 128 columns (fewer, longer trees).
+__host__ __device__ constexpr int epi_cols(int ew) { return TILE_N * NUM_EPI_WARPS / ew; }
+__host__ __device__ constexpr int warp_stage_bytes(int ew) { return STAGING_BYTES / ew; }
+__host__ __device__ constexpr int stage_pairs(int ew) { return (warp_stage_bytes(ew) - epi_cols(ew) * 4) / 8; }
+__host__ __device__ constexpr int num_threads(int ew) { return 32 * (EPI_WARP0 + ew); }
+static_assert(stage_pairs(NUM_EPI_WARPS) == STAGE_PAIRS && num_threads(NUM_EPI_WARPS) == NUM_THREADS, "");
 
 struct JoinParams {
     long long n, m;          // rows of P, Q
@@ -431,7 +440,7 @@ __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf
 // prefix over the warp, then into the warp's shared-memory staging buffer, which is flushed with
 // one global atomic per ~STAGE_PAIRS pairs.  A block with more hits than the buffer holds goes
 // straight to global memory.  `fill` (warp-uniform) is the number of pairs staged so far.
-template <int NQ, bool GROUPED, int VERIFY = VERIFY_NONE>
+template <int NQ, bool GROUPED, int VERIFY = VERIFY_NONE, int SP = STAGE_PAIRS>
 __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (&mask)[NQ], int lane, long long i, long long j0,
                                            int2 *buf, int &fill) {
     int cnt = 0;
@@ -441,7 +450,8 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
     int incl, total;
     const uint32_t one = __ballot_sync(0xffffffffu, cnt != 0);
     if (one == 0) return;
-    if (__ballot_sync(0xffffffffu, cnt > 1) == 0) {
+    const bool single = __ballot_sync(0xffffffffu, cnt > 1) == 0;
+    if (single) {
         incl = __popc(one & (0xffffffffu >> (31 - lane)));
         total = __popc(one);
     } else {
@@ -453,14 +463,14 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
         }
         total = __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (fill + total > STAGE_PAIRS) {
+    if (fill + total > SP) {
         flush_pairs<GROUPED, VERIFY>(p, buf, fill, lane);
         fill = 0;
     }
     // bucketed mode stages regrouped positions; they become original rows when they leave the CTA
     const int ii = (int)(i + (GROUPED ? 0 : p.ioff));
     const int jj = (int)(j0 + (GROUPED ? 0 : p.joff));
-    if (total > STAGE_PAIRS) {
+    if (total > SP) {
         if constexpr (GROUPED || VERIFY != VERIFY_NONE) {
             if (VERIFY != VERIFY_NONE || p.rep > 0) {
                 // more hits in one block than the buffer holds (rare): check and write them one by one
@@ -492,6 +502,19 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
                 ++slot;
             }
         }
+        return;
+    }
+    if (single) {
+        // one hit per row at most (total <= 32 fits): every hit lane finds its one column without a loop
+        if (cnt != 0) {
+            int col = 0;
+#pragma unroll
+            for (int q = 0; q < NQ; ++q)
+                if (mask[q] != 0) col = 32 * q + __ffs(mask[q]) - 1;
+            buf[fill + incl - 1] = make_int2(ii, jj + col);
+        }
+        fill += total;
+        __syncwarp();
         return;
     }
     int pos = fill + incl - cnt;
@@ -709,8 +732,8 @@ __host__ __device__ constexpr int fast_nstages(int kc, int pbufs) {
 // tile -- 4 MMAs of N = 256 per chunk into the 256 columns of an accumulator buffer, 32 KiB TMA transactions --
 // which this HBM-bound use prefers to two half-empty 128-column blocks.  In both, mapQ has 256-row boxes.
 constexpr int GEO_STD = 0, GEO_LONG = 1, GEO_WIDEQ = 2;
-template <int DT, int KIND, bool ALT = false, int KC = 0, bool GROUPED = false, int GEO = GEO_STD>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <int DT, int KIND, bool ALT = false, int KC = 0, bool GROUPED = false, int GEO = GEO_STD, int EW = NUM_EPI_WARPS>
+__global__ void __launch_bounds__(num_threads(EW), 1)
 join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ, const JoinParams p_in) {
     constexpr bool LONGK = GEO == GEO_LONG, WIDEQ = GEO == GEO_WIDEQ;
     constexpr bool NARROW = DT == DT_I8 && ALT;
@@ -722,8 +745,11 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     if (p_in.sel_mode != SEL_NONE && alt_selected(p_in) != ALT) return;
     static_assert(!LONGK || (KC == 0 && KIND != KIND_STORE), "long-row mode: general join kinds only");
     static_assert(!WIDEQ || (KC == 0 && !GROUPED && KIND == KIND_STORE), "wide-Q mode: store kind only");
+    static_assert(EW == NUM_EPI_WARPS || (EW == 2 * NUM_EPI_WARPS && GEO == GEO_STD && KIND != KIND_STORE), "16 epilogue warps: join kinds, standard geometry");
     constexpr int TN = (LONGK || WIDEQ) ? LONG_TN : TILE_N;   // rows of Q per tile
-    constexpr int NPASS = TN / EPI_COLS;                   // 128-column passes of an epilogue warp over its block
+    constexpr int NPASS = TN / TILE_N;                     // 128-column passes of the epilogue over a P block's columns
+    constexpr int ECOLS = epi_cols(EW);                    // accumulator columns per epilogue warp and pass
+    constexpr int SPAIRS = stage_pairs(EW);                // pairs a warp stages before it flushes
     JoinParams p = p_in;
     if constexpr (LONGK) {
         p.stationary = 0;
@@ -759,7 +785,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             mbar_init(smem_u32(&ctrl->pfull[b]), 1);
             mbar_init(smem_u32(&ctrl->pempty[b]), p.epi_release ? 2 : 1);   // one commit per issuing warp
             mbar_init(smem_u32(&ctrl->tfull[b]), 1);
-            mbar_init(smem_u32(&ctrl->tempty[b]), NUM_EPI_WARPS);
+            mbar_init(smem_u32(&ctrl->tempty[b]), EW);
         }
         mbar_init(smem_u32(&ctrl->drain[0]), 1);
         mbar_init(smem_u32(&ctrl->drain[1]), 1);
@@ -860,13 +886,14 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     } else if (warp >= EPI_WARP0) {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
-        const int half = (warp - EPI_WARP0) >> 2;   // which of the tile's two P blocks (accumulator columns half * TILE_N ..)
+        const int half = ((warp - EPI_WARP0) >> 2) & 1;   // which of the tile's two P blocks (accumulator columns half * TILE_N ..)
+        const int coff = ((warp - EPI_WARP0) >> 3) * ECOLS;   // 16 warps: first column of this warp within a 128-column pass
         const int row_in_tile = half * TILE_M + quarter * 32 + lane;
         uint32_t acc = 0, accphase = 0, rstage = 0;   // rstage: next ring stage to hand back
         // candidates of a filter are decided from their rows at flush time
         constexpr int VERIFY = (DT == DT_I8 && KIND == KIND_COS) ? VERIFY_COS_I8 : (L2_FILTER ? VERIFY_L2_BF16 : VERIFY_NONE);
-        int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * (WARP_STAGE_BYTES / 8);
-        uint32_t *colterm = reinterpret_cast<uint32_t *>(stage_buf + STAGE_PAIRS);
+        int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * (warp_stage_bytes(EW) / 8);
+        uint32_t *colterm = reinterpret_cast<uint32_t *>(stage_buf + SPAIRS);
         int stage_fill = 0;
         bool ok = true;
         Unit un;
@@ -946,9 +973,14 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 // sparse 262 144^2 join, +0.5-1 % on a dense one (the adaptive form -- prefetch while the previous tile
                 // had candidates -- lost on both)
                 constexpr bool LAZY_COLTERMS = DT == DT_I8;
+                constexpr int CPL = ECOLS / 32;           // per-column terms per lane: 4, or 2 with 16 epilogue warps
                 auto load_colterms = [&](int ps) -> uint4 {
-                    const uint32_t *nyp = reinterpret_cast<const uint32_t *>(p.ny) + (q_base + (long long)qt * TN + ps * EPI_COLS) + 4 * lane;
-                    if constexpr (GROUPED)          // a bucket starts at any row: no 16-byte alignment
+                    const uint32_t *nyp = reinterpret_cast<const uint32_t *>(p.ny) + (q_base + (long long)qt * TN + ps * TILE_N + coff) + CPL * lane;
+                    if constexpr (CPL == 2) {
+                        if constexpr (GROUPED) return make_uint4(__ldg(nyp), __ldg(nyp + 1), 0u, 0u);
+                        const uint2 t2 = __ldg(reinterpret_cast<const uint2 *>(nyp));
+                        return make_uint4(t2.x, t2.y, 0u, 0u);
+                    } else if constexpr (GROUPED)   // a bucket starts at any row: no 16-byte alignment
                         return make_uint4(__ldg(nyp), __ldg(nyp + 1), __ldg(nyp + 2), __ldg(nyp + 3));
                     else
                         return __ldg(reinterpret_cast<const uint4 *>(nyp));
@@ -1004,8 +1036,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 }
                 // this warp's 128 columns of the tile (long rows: two passes of 128 over its block's 256), then hand
                 // the accumulator back to the MMA warp
-                constexpr int NV = NARROW ? EPI_COLS / 2 : EPI_COLS;      // accumulator words per thread
-                constexpr int GCOLS = 16, NG = EPI_COLS / GCOLS, GW = NV / NG;  // column groups of level 1
+                constexpr int NV = NARROW ? ECOLS / 2 : ECOLS;            // accumulator words per thread
+                constexpr int GCOLS = 16, NG = ECOLS / GCOLS, GW = NV / NG;     // column groups of level 1
                 constexpr uint32_t GMASK = (1u << GCOLS) - 1u;
                 constexpr int MODE = DT == DT_BF16 ? MAX_F32 : (NARROW ? MAX_S16X2 : MAX_S32);
                 // Long rows with the packed epilogue: both passes' words fit in registers (2 x 64), so the single
@@ -1015,7 +1047,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 if constexpr (LOAD_ALL) {
 #pragma unroll
                     for (int ps = 0; ps < NPASS; ++ps)
-                        tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TN + ps * EPI_COLS, vall[ps],
+                        tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TN + ps * TILE_N + coff, vall[ps],
                                       std::integral_constant<bool, NARROW>{});
                     tc_fence_before();
                     __syncwarp();
@@ -1026,7 +1058,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 uint4 yq = yq_pass[ps];
                 uint32_t (&v)[NV] = vall[LOAD_ALL ? ps : 0];
                 if constexpr (!LOAD_ALL) {
-                    tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TN + ps * EPI_COLS, v,
+                    tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TN + ps * TILE_N + coff, v,
                                   std::integral_constant<bool, NARROW>{});
                     tc_fence_before();
                     __syncwarp();
@@ -1064,16 +1096,17 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         gm |= (bound_ok(gmax[k]) ? 1u : 0u) << k;
                     }
                     if (!row_ok) gm = 0;
-                    const long long j0 = q_base + (long long)qt * TN + ps * EPI_COLS;
-                    uint32_t mask[EPI_COLS / 32];
+                    const long long j0 = q_base + (long long)qt * TN + ps * TILE_N + coff;
+                    uint32_t mask[ECOLS / 32];
 #pragma unroll
-                    for (int q = 0; q < EPI_COLS / 32; ++q) mask[q] = 0;
+                    for (int q = 0; q < ECOLS / 32; ++q) mask[q] = 0;
                     if constexpr (KIND != KIND_IP) {
                         // the per-column terms go through shared memory: level 2 reads 16 of them per group as four
                         // broadcast loads (a shuffle per term cost four times the instructions)
                         if constexpr (LAZY_COLTERMS) yq = load_colterms(ps);
                         __syncwarp();
-                        reinterpret_cast<uint4 *>(colterm)[lane] = yq;
+                        if constexpr (CPL == 2) reinterpret_cast<uint2 *>(colterm)[lane] = make_uint2(yq.x, yq.y);
+                        else reinterpret_cast<uint4 *>(colterm)[lane] = yq;
                         __syncwarp();
                     }
 #pragma unroll
@@ -1136,14 +1169,14 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     }
                     // columns past the end of Q (of the bucket) were multiplied as zero rows: drop them
                     const long long left = q_end - j0;
-                    if (left < EPI_COLS) {
+                    if (left < ECOLS) {
 #pragma unroll
-                        for (int q = 0; q < EPI_COLS / 32; ++q) {
+                        for (int q = 0; q < ECOLS / 32; ++q) {
                             const long long lq = left - 32 * q;
                             mask[q] &= lq >= 32 ? 0xffffffffu : (lq <= 0 ? 0u : ((1u << (int)lq) - 1u));
                         }
                     }
-                    emit_pairs<EPI_COLS / 32, GROUPED, VERIFY>(p, mask, lane, i, j0, stage_buf, stage_fill);
+                    emit_pairs<ECOLS / 32, GROUPED, VERIFY, SPAIRS>(p, mask, lane, i, j0, stage_buf, stage_fill);
                 }
                 }   // passes
                 if constexpr (LONGK) {

@@ -36,6 +36,8 @@ struct DevBuf {
 // applies: the max|x| pre-pass and the second launch cost two more steps in the stream's dependent chain (about 13 us
 // measured on B200), which the packed epilogue's ~15 % only wins back on joins of ~90 us and more.
 constexpr double DEFAULT_SELECT_MIN_OPS = 2.0e11;
+// Pairs per 32 x 128 block of scores from which a join counts as dense (its next run takes 16 epilogue warps).
+constexpr double DENSE_MIN_PAIRS_PER_BLOCK = 0.5;
 constexpr int MAX_HOST_SLICES = 66;     // simjoin_run_host: a Q of more slices than this goes up in one piece
 
 // Device-side working memory of one join call, and the host words its result lands in.  simjoin_run takes it from the
@@ -72,6 +74,9 @@ struct simjoin_ctx {
     bool attr_set[2][4][2][3][2];
     bool attr_set_long[2][3][2][2];
     bool attr_set_wideq;
+    bool attr_set_dense[3][2][3];
+    int dense_mode;                     // SIMJOIN_OPT_DENSE_EPILOGUE: 0 never, 1 always (where instantiated), 2 by the last join's density
+    double last_density;                // pairs per 32 x 128 block of scores in the last successful simjoin_run (-1: none yet)
     cudaStream_t copy_stream;           // simjoin_run_host: uploads of Q slices overlap the joins of earlier slices
     cudaEvent_t copy_ev[MAX_HOST_SLICES + 1];   // one per slice, plus one that orders the copy stream behind earlier work
     DevBuf jl_a, jl_buf[2];             // JL transform: level matrix, ping-pong level outputs
@@ -199,6 +204,30 @@ cudaError_t launch_join(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorM
     if (fast && jp.kc == 2 && jp.nstages == fast_nstages(2, p_bufs(GROUPED, 2)))
         return launch_join_kc<DT, KIND, ALT, 2, GROUPED>(ctx, mp, mq, jp, grid, smem);
     return launch_join_kc<DT, KIND, ALT, 0, GROUPED>(ctx, mp, mq, jp, grid, smem);
+}
+
+// The 16-epilogue-warp instantiations (dense outputs): bf16 kinds, rows of one or two whole chunks, brute-force schedule.
+template <int DT, int KIND, bool ALT, int KC>
+cudaError_t launch_join_dense_kc(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid, size_t smem) {
+    constexpr int EW = 2 * NUM_EPI_WARPS;
+    auto kern = join_kernel<DT, KIND, ALT, KC, false, GEO_STD, EW>;
+    if (!ctx->attr_set_dense[KIND][ALT ? 1 : 0][KC]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
+        if (e != cudaSuccess) return e;
+        ctx->attr_set_dense[KIND][ALT ? 1 : 0][KC] = true;
+    }
+    kern<<<grid, num_threads(EW), smem, ctx->stream>>>(mp, mq, jp);
+    return cudaGetLastError();
+}
+// Is there a dense instantiation for this geometry?
+bool dense_available(bool i8, const JoinParams &jp) {
+    const bool fast = jp.stationary && jp.epi_release && jp.last_ksteps == 4;
+    return !i8 && fast && (jp.kc == 1 || jp.kc == 2) && jp.nstages == fast_nstages(jp.kc, p_bufs(false, jp.kc));
+}
+template <int KIND, bool ALT>
+cudaError_t launch_join_dense(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid, size_t smem) {
+    return jp.kc == 1 ? launch_join_dense_kc<DT_BF16, KIND, ALT, 1>(ctx, mp, mq, jp, grid, smem)
+                      : launch_join_dense_kc<DT_BF16, KIND, ALT, 2>(ctx, mp, mq, jp, grid, smem);
 }
 
 // Chunks per row from which the join takes the long-row geometry.  Measured on B200 (n = m = 131 072, sustained,
@@ -465,6 +494,16 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     } else if (i8 && kind == SIMJOIN_IP) e = launch_both<DT_I8, KIND_IP>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_L2) e = launch_both<DT_I8, KIND_L2>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_COS) e = launch_both<DT_I8, KIND_COS>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    else if (!i8 && dense_available(i8, jp) && !longk &&
+             (ctx->dense_mode == 1 || (ctx->dense_mode == 2 && ctx->last_density >= DENSE_MIN_PAIRS_PER_BLOCK))) {
+        // the last join on this context was dense: the 16-epilogue-warp instantiation of the same kind
+        if (kind == SIMJOIN_IP) e = launch_join_dense<KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
+        else if (kind == SIMJOIN_COS) e = launch_join_dense<KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem);
+        else {
+            e = launch_join_dense<KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
+            if (e == cudaSuccess) e = launch_join_dense<KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
+        }
+    }
     else if (!i8 && kind == SIMJOIN_IP) e = launch_geo<DT_BF16, KIND_IP, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (!i8 && kind == SIMJOIN_COS) e = launch_geo<DT_BF16, KIND_COS, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (!i8 && kind == SIMJOIN_L2) e = launch_both<DT_BF16, KIND_L2>(ctx, longk, mapP, mapQ, jp, grid, smem);
@@ -479,6 +518,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     if (kstatus != 0) return SIMJOIN_ERR_TIMEOUT;
     if (!fixed) ctx->ctrl_clean = cur ^ 1;        // the kernel has zeroed the other block
     *count = scr.h_ctrl[0];
+    ctx->last_density = (double)*count / ((double)((n + 31) / 32) * (double)((m + 127) / 128));
     float a = 0.f, b = 0.f;
     if (timed && (!need_norms || cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess) &&
         cudaEventElapsedTime(&b, ctx->ev[1], ctx->ev[2]) == cudaSuccess) {
@@ -901,6 +941,9 @@ simjoin_status simjoin_create(simjoin_ctx **out, simjoin_dtype dtype, int device
     std::memset(ctx->attr_set, 0, sizeof ctx->attr_set);
     std::memset(ctx->attr_set_long, 0, sizeof ctx->attr_set_long);
     ctx->attr_set_wideq = false;
+    std::memset(ctx->attr_set_dense, 0, sizeof ctx->attr_set_dense);
+    ctx->dense_mode = 2;
+    ctx->last_density = -1.0;
     ctx->copy_stream = nullptr;
     for (auto &e : ctx->copy_ev) e = nullptr;
     for (auto &e : ctx->ev) e = nullptr;
@@ -969,6 +1012,10 @@ simjoin_status simjoin_set_option(simjoin_ctx *ctx, simjoin_option option, doubl
         case SIMJOIN_OPT_SELECT_MIN_OPS:
             if (value < 0) return SIMJOIN_ERR_ARG;
             ctx->select_min_ops = value;
+            return SIMJOIN_OK;
+        case SIMJOIN_OPT_DENSE_EPILOGUE:
+            if (value != 0.0 && value != 1.0 && value != 2.0) return SIMJOIN_ERR_ARG;
+            ctx->dense_mode = (int)value;
             return SIMJOIN_OK;
         case SIMJOIN_OPT_KERNEL_TIMING:
             if (value != 0.0 && value != 1.0) return SIMJOIN_ERR_ARG;

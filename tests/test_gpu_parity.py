@@ -511,6 +511,26 @@ def test_bf16_l2_radius_far_below_the_norms(ctx_bf16, d, r):
     assert all((i, 3 + 3 * i) in got for i in range(200)), "an equal pair is missing"
 
 
+@pytest.mark.parametrize("kind", ["ip", "cos", "l2"])
+@pytest.mark.parametrize("n,m,d", [(129, 257, 64), (700, 1300, 64), (513, 1000, 128), (300, 2100, 128), (140, 300, 72)])
+def test_bf16_dense_epilogue_matches_the_oracle(kind, n, m, d):
+    """The 16-epilogue-warp instantiations (rows of one or two whole chunks), forced on: sparse and dense outputs, ragged
+    tiles, hits in both 64-column halves of a block; other row lengths fall back to the regular kernel.  Then the default
+    mode, where a context switches to them after a dense join and back after a sparse one: same sets."""
+    P, Q = W.random_points("bf16", n, d, 15), W.random_points("bf16", m, d, 16)
+    Q[1:m:7][:n] = P[:len(Q[1:m:7][:n])]
+    sparse = {"ip": 1.5 * d ** 0.5, "cos": 1.5 / d ** 0.5, "l2": (2 * d) ** 0.5 - 1.2}[kind]
+    dense = {"ip": -0.3 * d ** 0.5, "cos": -0.3 / d ** 0.5, "l2": (2 * d) ** 0.5 + 0.4}[kind]
+    with B.Simjoin("bf16", 0) as ctx:
+        assert ctx.simjoin_set_option(B.SIMJOIN_OPT_DENSE_EPILOGUE, 3.0) == B.SIMJOIN_ERR_ARG
+        for mode in (1.0, 2.0):
+            assert ctx.simjoin_set_option(B.SIMJOIN_OPT_DENSE_EPILOGUE, mode) == B.SIMJOIN_OK
+            for t in (sparse, dense, dense, sparse, sparse):
+                pairs, cnt = gpu_join(ctx, P, Q, kind, t, capacity=1 << 22)
+                assert_band(pairs, cnt, P, Q, kind, t)
+                assert cnt > 0
+
+
 def test_repeated_runs_give_the_same_set(ctx_bf16):
     w = W.make_workload(5, n=3000, m=3000, centers=30)
     a, ca = gpu_join(ctx_bf16, w.P, w.Q, "l2", w.threshold, capacity=1 << 19)
