@@ -299,9 +299,11 @@ int64_t oracle_join_hamming_bits(const uint8_t *P, int64_t n, const uint8_t *Q, 
  * each bucket; the result is the union over the repetitions.  With a fixed hash family the result is
  * therefore exactly { (i, j) in the brute-force join : the hashes of x_i and y_j agree in at least
  * one repetition } -- which is what this oracle enumerates, with no buckets at all.
- * Base hash (bit sampling, the classic monotone LSH for Hamming / +-1 data): h(x) = [x_c > 0] for a
- * sampled coordinate c.  Coordinate of repetition l, bit b: splitmix64(seed, l*64 + b) mod d -- a
- * counter-based generator that the CUDA library implements on its own.
+ * Base hash, family 0 (bit sampling, the classic monotone LSH for Hamming / +-1 data): h(x) = [x_c > 0] for a
+ * sampled coordinate c; the k bits of a repetition sample k distinct coordinates (lsh_rep_coordinates below) from
+ * a counter-based generator that the CUDA library implements on its own.
+ * Base hash, family 1 (random hyperplanes, the LSH of the angular distance): h(x) = [<a, x> > 0] for a vector a of
+ * independent random signs (oracle_lsh_hp_sign below); a projection of exactly zero gives bit 0.
  * When the number of base hashes the analysis asks for is not an integer, the paper builds L_high
  * tables from ceil(k) base hashes and L_low tables from floor(k): here the first L_high repetitions
  * use k bits and the following L_low use k - 1. */
@@ -367,6 +369,59 @@ void oracle_lsh_keys_bf16(const uint16_t *X, int64_t rows, int32_t d, int32_t L_
                 if (oracle_bf16_to_f64(X[(size_t)i * d + coord[b]]) > 0.0) key |= 1u << b;
             keys[(size_t)l * rows + i] = key;
         }
+    }
+}
+
+/* ---- family 1: sign random projections ----
+ * Hyperplane of repetition `rep`, bit `bit`: a vector of d independent random signs, coordinate c being +1 when bit 0
+ * of splitmix64(seed, 2^60 + (64 rep + bit) 2^20 + c) is set and -1 otherwise (rows of at most 2^20 coordinates).
+ * Random-sign vectors have the angular collision law of Gaussian ones in the limit of many coordinates of
+ * comparable size: two points at angle theta agree on a bit with probability 1 - theta / pi, whatever the
+ * distribution of the data (no rotation invariance needed, unlike the sampled-coordinate sign). */
+int32_t oracle_lsh_hp_sign(uint64_t seed, int32_t rep, int32_t bit, int32_t c) {
+    const uint64_t idx = (1ULL << 60) + (((uint64_t)rep * 64u + (uint64_t)bit) << 20) + (uint64_t)c;
+    return (splitmix64_at(seed, idx) & 1u) ? 1 : -1;
+}
+
+/* keys[l * rows + i]: bit b = [ sum_c a_{l,b,c} x_{i,c} > 0 ], the sum an exact integer; k bits in the first L_high
+ * repetitions, k - 1 (the same hyperplanes without the last) in the next L_low. */
+void oracle_lsh_keys_hp_i8(const int8_t *X, int64_t rows, int32_t d, int32_t L_high, int32_t L_low, int32_t k, uint64_t seed,
+                           uint32_t *keys) {
+    for (int32_t l = 0; l < L_high + L_low; ++l) {
+        const int32_t bits = l < L_high ? k : k - 1;
+        for (int64_t i = 0; i < rows; ++i) keys[(size_t)l * rows + i] = 0;
+        for (int32_t b = 0; b < bits; ++b)
+            for (int64_t i = 0; i < rows; ++i) {
+                int64_t proj = 0;
+                for (int32_t c = 0; c < d; ++c) proj += (int64_t)oracle_lsh_hp_sign(seed, l, b, c) * (int64_t)X[(size_t)i * d + c];
+                if (proj > 0) keys[(size_t)l * rows + i] |= 1u << b;
+            }
+    }
+}
+
+/* The same for bf16 rows, projections summed in fp64 with c ascending.  A floating-point sign decides a bit here, and
+ * an implementation that accumulates in fp32 may decide a projection close to zero the other way: `unsure` (may be
+ * NULL) gets, per repetition and row, the mask of the bits with |projection| <= tol * sum_c |x_c|; a comparison of
+ * hash keys leaves those bits free. */
+void oracle_lsh_keys_hp_bf16(const uint16_t *X, int64_t rows, int32_t d, int32_t L_high, int32_t L_low, int32_t k, uint64_t seed,
+                             double tol, uint32_t *keys, uint32_t *unsure) {
+    for (int32_t l = 0; l < L_high + L_low; ++l) {
+        const int32_t bits = l < L_high ? k : k - 1;
+        for (int64_t i = 0; i < rows; ++i) {
+            keys[(size_t)l * rows + i] = 0;
+            if (unsure) unsure[(size_t)l * rows + i] = 0;
+        }
+        for (int32_t b = 0; b < bits; ++b)
+            for (int64_t i = 0; i < rows; ++i) {
+                double proj = 0.0, mass = 0.0;
+                for (int32_t c = 0; c < d; ++c) {
+                    const double v = oracle_bf16_to_f64(X[(size_t)i * d + c]);
+                    proj += (double)oracle_lsh_hp_sign(seed, l, b, c) * v;
+                    mass += fabs(v);
+                }
+                if (proj > 0.0) keys[(size_t)l * rows + i] |= 1u << b;
+                if (unsure && fabs(proj) <= tol * mass) unsure[(size_t)l * rows + i] |= 1u << b;
+            }
     }
 }
 

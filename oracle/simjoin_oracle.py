@@ -76,6 +76,12 @@ def _load():
     lib.oracle_lsh_keys_i8.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, vp]
     lib.oracle_lsh_keys_bf16.restype = None
     lib.oracle_lsh_keys_bf16.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, vp]
+    lib.oracle_lsh_hp_sign.restype = i32
+    lib.oracle_lsh_hp_sign.argtypes = [c.c_uint64, i32, i32, i32]
+    lib.oracle_lsh_keys_hp_i8.restype = None
+    lib.oracle_lsh_keys_hp_i8.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, vp]
+    lib.oracle_lsh_keys_hp_bf16.restype = None
+    lib.oracle_lsh_keys_hp_bf16.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, dbl, vp, vp]
     lib.oracle_lsh_coordinate.restype = i32
     lib.oracle_lsh_coordinate.argtypes = [c.c_uint64, i32, i32, i32]
     lib.oracle_jl_levels.restype = i32
@@ -199,37 +205,94 @@ def lsh_join_hamming(Pbits: np.ndarray, Qbits: np.ndarray, d: int, r: float, L: 
     return lsh_join(widen(Pbits), widen(Qbits), float(d) - 2.0 * np.floor(r), L, k, seed, threads=threads, L_low=L_low)
 
 
-def lsh_keys(X: np.ndarray, L: int, k: int, seed: int, L_low: int = 0, dtype: str = "i8") -> np.ndarray:
-    """(L + L_low, rows) uint32 hash keys of int8 rows (or bf16 bit patterns): bit b = [x_c > 0] at the sampled coordinate."""
+FAMILIES = ("bits", "hyperplanes")
+
+
+def hp_tolerance(d: int) -> float:
+    """Relative size (to sum |x_c|) below which an fp32 accumulation of d exact products, in any order and with the
+    tensor core's internal truncation, may decide the sign of a hyperplane projection differently from fp64."""
+    return (d + 64) * 2.0 ** -23
+
+
+def lsh_keys(X: np.ndarray, L: int, k: int, seed: int, L_low: int = 0, dtype: str = "i8", family: str = "bits") -> np.ndarray:
+    """(L + L_low, rows) uint32 hash keys.  family "bits": bit b = [x_c > 0] at the sampled coordinate (int8 rows or
+    bf16 bit patterns); family "hyperplanes": bit b = [<a, x> > 0] for a random-sign vector a."""
     lib = _load()
     X = _check(X, dtype)
     out = np.empty((L + L_low, X.shape[0]), dtype=np.uint32)
-    fn = lib.oracle_lsh_keys_i8 if dtype == "i8" else lib.oracle_lsh_keys_bf16
-    fn(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, out.ctypes.data)
+    if family == "bits":
+        fn = lib.oracle_lsh_keys_i8 if dtype == "i8" else lib.oracle_lsh_keys_bf16
+        fn(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, out.ctypes.data)
+    elif family == "hyperplanes":
+        if dtype == "i8":
+            lib.oracle_lsh_keys_hp_i8(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, out.ctypes.data)
+        else:
+            lib.oracle_lsh_keys_hp_bf16(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, 0.0, out.ctypes.data, None)
+    else:
+        raise ValueError(family)
     return out
 
 
-def lsh_restrict(pairs: np.ndarray, P: np.ndarray, Q: np.ndarray, dtype: str, L: int, k: int, seed: int, L_low: int = 0) -> np.ndarray:
+def lsh_keys_unsure(X: np.ndarray, L: int, k: int, seed: int, L_low: int = 0, tol: float | None = None):
+    """Hyperplane keys of bf16 rows and, per repetition and row, the mask of the bits whose projection is within
+    tol * sum |x_c| of zero (default tol: hp_tolerance(d)): (keys, unsure), both (L + L_low, rows) uint32."""
+    lib = _load()
+    X = _check(X, "bf16")
+    keys = np.empty((L + L_low, X.shape[0]), dtype=np.uint32)
+    unsure = np.empty_like(keys)
+    lib.oracle_lsh_keys_hp_bf16(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed,
+                                hp_tolerance(X.shape[1]) if tol is None else float(tol), keys.ctypes.data, unsure.ctypes.data)
+    return keys, unsure
+
+
+def hp_sign(seed: int, rep: int, bit: int, c: int) -> int:
+    return int(_load().oracle_lsh_hp_sign(seed, rep, bit, c))
+
+
+def lsh_restrict(pairs: np.ndarray, P: np.ndarray, Q: np.ndarray, dtype: str, L: int, k: int, seed: int, L_low: int = 0,
+                 family: str = "bits", unsure: str | None = None) -> np.ndarray:
     """The pairs of a (brute-force) join whose hash keys agree in at least one repetition: what the LSH-bucketed join of
-    any kind returns, since it runs the brute-force join inside the buckets of every repetition and takes the union."""
-    kp, kq = lsh_keys(P, L, k, seed, L_low, dtype), lsh_keys(Q, L, k, seed, L_low, dtype)
+    any kind returns, since it runs the brute-force join inside the buckets of every repetition and takes the union.
+    bf16 hyperplane keys depend on floating-point signs: unsure="strict" keeps a pair only if some repetition's keys
+    agree with no bit of either point in doubt, unsure="loose" if some repetition's keys agree on every bit that is
+    not in doubt -- any correct fp32 implementation returns a set between the two."""
     pairs = np.asarray(pairs).reshape(-1, 2)
     if len(pairs) == 0:
         return pairs
-    keep = (kp[:, pairs[:, 0]] == kq[:, pairs[:, 1]]).any(axis=0)
+    if unsure is None or family != "hyperplanes" or dtype != "bf16":
+        kp, kq = lsh_keys(P, L, k, seed, L_low, dtype, family), lsh_keys(Q, L, k, seed, L_low, dtype, family)
+        keep = (kp[:, pairs[:, 0]] == kq[:, pairs[:, 1]]).any(axis=0)
+        return pairs[keep]
+    (kp, up), (kq, uq) = lsh_keys_unsure(P, L, k, seed, L_low), lsh_keys_unsure(Q, L, k, seed, L_low)
+    diff = kp[:, pairs[:, 0]] ^ kq[:, pairs[:, 1]]
+    free = up[:, pairs[:, 0]] | uq[:, pairs[:, 1]]
+    if unsure == "strict":
+        keep = ((diff == 0) & (free == 0)).any(axis=0)
+    elif unsure == "loose":
+        keep = ((diff & ~free) == 0).any(axis=0)
+    else:
+        raise ValueError(unsure)
     return pairs[keep]
 
 
-def lsh_join_kind(P, Q, kind: str, threshold: float, dtype: str, L: int, k: int, seed: int, L_low: int = 0, threads: int = 0):
-    """LSH-bucketed join of any kind and element type: the brute-force join restricted to colliding pairs."""
+def lsh_join_kind(P, Q, kind: str, threshold: float, dtype: str, L: int, k: int, seed: int, L_low: int = 0, threads: int = 0,
+                  family: str = "bits"):
+    """LSH-bucketed join of any kind, element type and hash family: the brute-force join restricted to colliding pairs."""
     pairs, _c = join(P, Q, kind, threshold, dtype, threads=threads)
-    out = lsh_restrict(pairs, P, Q, dtype, L, k, seed, L_low)
+    out = lsh_restrict(pairs, P, Q, dtype, L, k, seed, L_low, family)
     return out, len(out)
 
 
-def lsh_band_sets(P, Q, kind: str, threshold: float, dtype: str, L: int, k: int, seed: int, L_low: int = 0, rel: float = 1e-2):
-    """band_sets restricted to colliding pairs: a floating-point LSH join G is accepted when S_strict <= G <= S_loose."""
-    return tuple(lsh_restrict(s, P, Q, dtype, L, k, seed, L_low) for s in band_sets(P, Q, kind, threshold, dtype, rel=rel))
+def lsh_band_sets(P, Q, kind: str, threshold: float, dtype: str, L: int, k: int, seed: int, L_low: int = 0, rel: float = 1e-2,
+                  family: str = "bits"):
+    """band_sets restricted to colliding pairs: a floating-point LSH join G is accepted when S_strict <= G <= S_loose
+    (hyperplane keys of bf16 rows: the strict set also needs a collision with no bit in doubt, the loose set accepts
+    one on the bits that are not in doubt)."""
+    s_strict, s_exact, s_loose = band_sets(P, Q, kind, threshold, dtype, rel=rel)
+    hp = family == "hyperplanes" and dtype == "bf16"
+    return (lsh_restrict(s_strict, P, Q, dtype, L, k, seed, L_low, family, "strict" if hp else None),
+            lsh_restrict(s_exact, P, Q, dtype, L, k, seed, L_low, family),
+            lsh_restrict(s_loose, P, Q, dtype, L, k, seed, L_low, family, "loose" if hp else None))
 
 
 def lsh_coordinate(seed: int, rep: int, bit: int, d: int) -> int:

@@ -31,7 +31,7 @@ def to_arr(rows, dtype):
 
 # ------------------------------------------------------------------ hand-worked
 GOLDEN = sorted(g for g in glob.glob(os.path.join(os.path.dirname(__file__), "golden", "*.json"))
-                if not os.path.basename(g).startswith("hamming"))
+                if not os.path.basename(g).startswith(("hamming", "lsh_")))
 
 
 @pytest.mark.parametrize("path", GOLDEN, ids=[os.path.basename(p) for p in GOLDEN])
@@ -630,3 +630,106 @@ def test_filter_of_every_pair_is_the_join(dtype, kind, t):
     kept = O.filter_pairs(P, Q, kind, t, dtype, some)
     assert as_set(kept) == as_set(want) & as_set(some)
     assert [tuple(p) for p in kept.tolist()] == [tuple(p) for p in some.tolist() if tuple(p) in as_set(want)]   # order kept
+
+
+# ------------------------------------------------------------------ hyperplane (sign random projection) LSH family
+def _hp_signs(seed, L, k, d):
+    """(L, k, d) array of +-1: coordinate c of the hyperplane of repetition l, bit b -- Python integers."""
+    return np.array([[[1 if _splitmix64(seed, (1 << 60) + ((l * 64 + b) << 20) + c) & 1 else -1 for c in range(d)]
+                      for b in range(k)] for l in range(L)], dtype=np.int64)
+
+
+def test_lsh_hyperplane_keys_golden(golden_dir):
+    g = json.load(open(os.path.join(golden_dir, "lsh_hyperplane_d8.json")))
+    X = np.array(g["points"], dtype=np.int8)
+    keys = O.lsh_keys(X, g["L"], g["k"], g["seed"], L_low=g["L_low"], family="hyperplanes")
+    assert keys.tolist() == g["keys"]
+    planes = np.array(g["hyperplanes"])
+    assert all(O.hp_sign(g["seed"], l, b, c) == planes[l, b, c] for l in range(3) for b in range(3) for c in range(8))
+    # the same integer points as bf16 rows (exact in bf16) hash alike, and none of their projections is in doubt except 0
+    Xb = W.f32_to_bf16_bits(X.astype(np.float32))
+    kb, unsure = O.lsh_keys_unsure(Xb, g["L"], g["k"], g["seed"], L_low=g["L_low"])
+    assert kb.tolist() == g["keys"]
+    proj = g["projections"]
+    for l in range(3):
+        for i in range(len(X)):
+            zero_bits = sum(1 << b for b, v in enumerate(proj[l][i]) if v == 0)
+            assert unsure[l, i] == zero_bits
+
+
+def test_lsh_hyperplane_keys_against_python_int_signs_and_numpy_products():
+    seed, L, L_low, k, d = 77, 3, 2, 5, 48
+    R = _hp_signs(seed, L + L_low, k, d)
+    X = W.random_points("i8", 300, d, 5, lo=-128, hi=127)
+    proj = np.einsum("lbc,ic->lib", R, X.astype(np.int64))                      # exact integers
+    want = ((proj > 0).astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).astype(np.uint32)
+    want[L:] &= (1 << (k - 1)) - 1                                             # L_low tables: the same planes without the last
+    assert np.array_equal(want, O.lsh_keys(X, L, k, seed, L_low=L_low, family="hyperplanes"))
+    # bf16 rows: fp64 products of the widened values; bits agree wherever the projection is not in doubt
+    Xb = W.random_points("bf16", 300, d, 6)
+    projf = np.einsum("lbc,ic->lib", R.astype(np.float64), W.bf16_bits_to_f32(Xb).astype(np.float64))
+    wantb = ((projf > 0).astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).astype(np.uint32)
+    wantb[L:] &= (1 << (k - 1)) - 1
+    kb, unsure = O.lsh_keys_unsure(Xb, L, k, seed, L_low=L_low)
+    assert np.array_equal(wantb & ~unsure, kb & ~unsure) and (unsure != 0).mean() < 0.01
+    assert np.array_equal(kb, O.lsh_keys(Xb, L, k, seed, L_low=L_low, dtype="bf16", family="hyperplanes"))
+
+
+def test_lsh_hyperplane_key_symmetries():
+    seed, L, k, d = 5, 4, 6, 64
+    X = W.random_points("i8", 200, d, 9, lo=-60, hi=60)
+    keys = O.lsh_keys(X, L, k, seed, family="hyperplanes")
+    assert np.array_equal(keys, O.lsh_keys((2 * X).astype(np.int8), L, k, seed, family="hyperplanes"))          # scale invariant
+    R = _hp_signs(seed, L, k, d)
+    nonzero = (np.einsum("lbc,ic->lib", R, X.astype(np.int64)) != 0).all(axis=2)       # (L, rows)
+    flipped = O.lsh_keys((-X).astype(np.int8), L, k, seed, family="hyperplanes")
+    assert np.array_equal(flipped[nonzero], (~keys & ((1 << k) - 1))[nonzero])           # -x lies on the other side of every plane
+    assert not O.lsh_keys(np.zeros((3, d), np.int8), L, k, seed, family="hyperplanes").any()                   # sign(0) := bit 0
+    # permuting the rows permutes the keys; a different seed gives different planes
+    perm = np.random.default_rng(0).permutation(len(X))
+    assert np.array_equal(keys[:, perm], O.lsh_keys(X[perm], L, k, seed, family="hyperplanes"))
+    assert not np.array_equal(keys, O.lsh_keys(X, L, k, seed + 1, family="hyperplanes"))
+
+
+def test_lsh_hyperplane_collision_law_holds_on_anisotropic_data_where_coordinate_signs_fail():
+    """Pairs at a known angle theta collide on a hyperplane bit with probability 1 - theta / pi whatever the shape of
+    the data; the sampled-coordinate sign only has that law for rotation-invariant data.  Data: 16 of 128 coordinates
+    are five times larger than the rest and carry all of the difference between the two points of a pair, so the
+    angle is set by coordinates that a sampled-coordinate hash rarely looks at."""
+    rng = np.random.default_rng(21)
+    d, npairs, big = 128, 400, 16
+    scale = np.ones(d)
+    scale[:big] = 5.0
+    base = rng.standard_normal((npairs, d)) * scale
+    other = base.copy()
+    other[:, :big] += 0.8 * 5.0 * rng.standard_normal((npairs, big))
+    X, Y = W.f32_to_bf16_bits(base.astype(np.float32)), W.f32_to_bf16_bits(other.astype(np.float32))
+    xf, yf = W.bf16_bits_to_f32(X).astype(np.float64), W.bf16_bits_to_f32(Y).astype(np.float64)
+    cos = (xf * yf).sum(axis=1) / np.sqrt((xf * xf).sum(axis=1) * (yf * yf).sum(axis=1))
+    expect = float(np.mean(1.0 - np.arccos(np.clip(cos, -1, 1)) / np.pi))           # about 0.81
+    L = 64
+    kx, ky = (O.lsh_keys(Z, L, 1, 3, dtype="bf16", family="hyperplanes") for Z in (X, Y))      # 64 single-bit keys
+    agree_hp = float((kx == ky).mean())
+    assert abs(agree_hp - expect) < 0.01, (agree_hp, expect)                        # 25 600 bits: sigma = 0.0025
+    bx, by = (O.lsh_keys(Z, L, 1, 3, dtype="bf16", family="bits") for Z in (X, Y))
+    agree_bits = float((bx == by).mean())
+    assert agree_bits > expect + 0.1, (agree_bits, expect)      # seven sampled coordinates in eight are equal in x and y
+
+
+def test_lsh_hyperplane_join_is_the_join_restricted_to_colliding_pairs():
+    w = W.make_workload(3, n=500, m=400, planted=60)
+    L, k, seed = 4, 5, 11
+    pairs, cnt = O.lsh_join_kind(w.P, w.Q, "ip", w.threshold, "i8", L, k, seed, family="hyperplanes")
+    R = _hp_signs(seed, L, k, w.d)
+    kp = ((np.einsum("lbc,ic->lib", R, w.P.astype(np.int64)) > 0) << np.arange(k)).sum(axis=2)
+    kq = ((np.einsum("lbc,ic->lib", R, w.Q.astype(np.int64)) > 0) << np.arange(k)).sum(axis=2)
+    full, _c = O.join(w.P, w.Q, "ip", w.threshold, "i8")
+    keep = (kp[:, full[:, 0]] == kq[:, full[:, 1]]).any(axis=0)
+    assert cnt == int(keep.sum()) and np.array_equal(pairs, full[keep]) and 0 < cnt
+    everything, c0 = O.lsh_join_kind(w.P, w.Q, "ip", w.threshold, "i8", 1, 0, seed, family="hyperplanes")          # k = 0: one bucket
+    assert c0 == len(full)
+    # bf16: the strict / loose collision sets bracket the plain one
+    wb = W.make_workload(2, n=400, m=300, planted=80)
+    s, e, lo = O.lsh_band_sets(wb.P, wb.Q, "cos", wb.threshold, "bf16", 6, 4, 5, family="hyperplanes")
+    ks, ke, kl = (O.pairs_to_set(z) for z in (s, e, lo))
+    assert np.isin(ks, kl).all() and len(ke) > 0 and len(kl) >= len(ks)
