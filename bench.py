@@ -341,6 +341,8 @@ def main():
     ap.add_argument("--lsh", default=None, metavar="L,k[,L_low]",
                     help="time the LSH-bucketed join (int8 inner-product configs) instead of the brute-force join: "
                          "L tables of k bits (+ L_low of k-1); not the headline metric, the line says so")
+    ap.add_argument("--lsh-family", default="bits", choices=["bits", "hyperplanes"],
+                    help="hash family of --lsh: sampled coordinates, or random hyperplanes (keys computed on the tensor cores)")
     ap.add_argument("--jl", default=None, metavar="n,d,k",
                     help="time the JL transform (simjoin_jl_transform) of n bf16 points from d to k coordinates instead "
                          "of the join; HBM-bound, reported in algorithmic GB/s; not the headline metric")
@@ -420,7 +422,7 @@ def main():
         if args.lsh:
             L, k = args.lsh[0], args.lsh[1]
             st, cnt = ctx.simjoin_run_lsh(dP, w.n, dQ, w.m, w.d, w.threshold, L, k, 2006, out, capacity,
-                                          L_low=args.lsh[2] if len(args.lsh) > 2 else 0)
+                                          L_low=args.lsh[2] if len(args.lsh) > 2 else 0, family=args.lsh_family)
         else:
             st, cnt = ctx.simjoin_run(dP, w.n, dQ, w.m, w.d, w.kind, w.threshold, out, capacity)
         if st != B.SIMJOIN_OK:
@@ -693,7 +695,7 @@ def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline}
     if args.lsh:
-        line["algorithm"] = {"name": "lsh-bucketed join (simjoin_run_lsh)", "L": args.lsh[0], "k": args.lsh[1],
+        line["algorithm"] = {"name": "lsh-bucketed join (simjoin_run_lsh)", "family": args.lsh_family, "L": args.lsh[0], "k": args.lsh[1],
                              "L_low": args.lsh[2] if len(args.lsh) > 2 else 0, "recall_on_planted_pairs": args.recall,
                              "hash_ms": statistics.mean(pre_ms), "tables_ms": jm,
                              "note": "value = 2*n*m*d over the step time: the brute-force-equivalent rate of an approximate "

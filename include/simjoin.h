@@ -149,7 +149,8 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
  * a subset of simjoin_run's (precision 1; the recall is set by L, k and the data; bf16: the same threshold band
  * as simjoin_run).
  *
- *   Base hash     bit sampling: h(x) = [x_c > 0] for a sampled coordinate c -- the standard family for
+ *   family        the LSH family (the paper takes it as a black box: "an (r, cr, p1, p2)-sensitive monotone LSH").
+ *     SIMJOIN_LSH_BITS         bit sampling: h(x) = [x_c > 0] for a sampled coordinate c -- the standard family for
  *                 Hamming distance, i.e. for +-1 rows such as simjoin_run_hamming builds; for bf16 rows the
  *                 sign of the sampled coordinate, i.e. the random-hyperplane hash of the angular distance
  *                 with axis-aligned hyperplanes (two rows of a rotation-invariant distribution at angle
@@ -159,9 +160,19 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
  *                 that no earlier bit of the repetition took (from bit d on, a = 0 as it comes), where
  *                 splitmix64(seed, i): z = seed + (i+1)*0x9E3779B97F4A7C15; z = (z ^ z>>30)*0xBF58476D1CE4E5B9;
  *                 z = (z ^ z>>27)*0x94D049BB133111EB; z ^ z>>31  (all modulo 2^64).
+ *     SIMJOIN_LSH_HYPERPLANES  random hyperplanes (sign random projections), the LSH of the angular distance for data of
+ *                 any shape: h(x) = [<a, x> > 0], a projection of exactly zero giving 0; a is a vector of random signs,
+ *                 coordinate c of the hyperplane of repetition l, bit b being +1 when bit 0 of
+ *                 splitmix64(seed, 2^60 + (64 l + b) 2^20 + c) is set and -1 otherwise.  Two points at angle theta agree
+ *                 on a bit with probability 1 - theta/pi.  The projections of all points onto all hyperplanes are one
+ *                 dense product, computed by the tile kernel on the tensor cores (16 hyperplane rows per repetition,
+ *                 a sign-collecting epilogue that writes the key records).  int8: the projections are exact integers
+ *                 and the keys exact; bf16: fp32 accumulation, so a projection within about (d + 64) 2^-23 sum |x_c| of
+ *                 zero may hash to either side (such a point may land in either of two buckets of that repetition).
  *   P, Q, n, m, d, kind, threshold, out_pairs, capacity, count   as simjoin_run (every dtype and kind it accepts).
- *   L, L_low      repetitions with k and with k - 1 bits; both >= 0, 1 <= L + L_low <= SIMJOIN_LSH_MAX_REPS,
- *                 L_low > 0 needs k >= 1 (ERR_ARG otherwise).
+ *   L, L_low      repetitions with k and with k - 1 bits (the first k - 1 samples / hyperplanes of their k); both >= 0,
+ *                 1 <= L + L_low <= SIMJOIN_LSH_MAX_REPS, L_low > 0 needs k >= 1 (ERR_ARG otherwise; also for an
+ *                 unknown family).
  *   k             key bits, 0..SIMJOIN_LSH_MAX_BITS (ERR_ARG if negative, ERR_UNSUPPORTED above);
  *                 k = 0 puts everything in one bucket and returns the brute-force result.
  *
@@ -172,9 +183,10 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
  * join all run on the device with no host round trip between repetitions.
  * simjoin_last_kernel_ms then reports (hashing, all repetitions).
  */
+typedef enum { SIMJOIN_LSH_BITS = 0, SIMJOIN_LSH_HYPERPLANES = 1 } simjoin_lsh_family;
 simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
-                               simjoin_kind kind, double threshold, int32_t L, int32_t L_low, int32_t k, uint64_t seed,
-                               int32_t *out_pairs, uint64_t capacity, uint64_t *count);
+                               simjoin_kind kind, double threshold, simjoin_lsh_family family, int32_t L, int32_t L_low,
+                               int32_t k, uint64_t seed, int32_t *out_pairs, uint64_t capacity, uint64_t *count);
 
 /*
  * LSH-bucketed Hamming join on bit-packed points: simjoin_run_hamming's operand transform followed by

@@ -20,6 +20,8 @@ SIMJOIN_IP, SIMJOIN_COS, SIMJOIN_L2 = 0, 1, 2
  SIMJOIN_ERR_TIMEOUT, SIMJOIN_ERR_ARCH) = range(7)
 DTYPE = {"i8": SIMJOIN_I8, "bf16": SIMJOIN_BF16}
 KIND = {"ip": SIMJOIN_IP, "cos": SIMJOIN_COS, "l2": SIMJOIN_L2}
+SIMJOIN_LSH_BITS, SIMJOIN_LSH_HYPERPLANES = 0, 1
+LSH_FAMILY = {"bits": SIMJOIN_LSH_BITS, "hyperplanes": SIMJOIN_LSH_HYPERPLANES}
 
 EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_hamming", "simjoin_run_lsh", "simjoin_run_hamming_lsh", "simjoin_jl_transform", "simjoin_filter_pairs", "simjoin_run_jl_l2", "simjoin_row_norms", "simjoin_set_offsets", "simjoin_set_option",
            "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_selftest_wait_timeout", "simjoin_destroy",
@@ -56,7 +58,7 @@ def load() -> ctypes.CDLL:
     lib.simjoin_run_hamming.restype = c.c_int
     lib.simjoin_run_hamming.argtypes = [vp, vp, i64, vp, i64, i32, dbl, vp, u64, c.POINTER(u64)]
     lib.simjoin_run_lsh.restype = c.c_int
-    lib.simjoin_run_lsh.argtypes = [vp, vp, i64, vp, i64, i32, c.c_int, dbl, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
+    lib.simjoin_run_lsh.argtypes = [vp, vp, i64, vp, i64, i32, c.c_int, dbl, c.c_int, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
     lib.simjoin_run_hamming_lsh.restype = c.c_int
     lib.simjoin_run_hamming_lsh.argtypes = [vp, vp, i64, vp, i64, i32, dbl, i32, i32, i32, u64, vp, u64, c.POINTER(u64)]
     lib.simjoin_jl_transform.restype = c.c_int
@@ -151,10 +153,11 @@ class Simjoin:
         st = load().simjoin_run_hamming(self._h, pp, n, qp, m, d, float(r), op, capacity, ctypes.byref(cnt))
         return st, cnt.value
 
-    def simjoin_run_lsh(self, P, n, Q, m, d, threshold, L, k, seed, out_pairs, capacity, L_low=0, kind="ip"):
+    def simjoin_run_lsh(self, P, n, Q, m, d, threshold, L, k, seed, out_pairs, capacity, L_low=0, kind="ip", family="bits"):
         cnt = ctypes.c_uint64(0)
         (pp, _a), (qp, _b), (op, _c) = _ptr(P), _ptr(Q), _ptr(out_pairs)
         st = load().simjoin_run_lsh(self._h, pp, n, qp, m, d, KIND[kind] if isinstance(kind, str) else kind, float(threshold),
+                                    LSH_FAMILY[family] if isinstance(family, str) else int(family),
                                     int(L), int(L_low), int(k), int(seed), op, capacity, ctypes.byref(cnt))
         return st, cnt.value
 
@@ -216,7 +219,8 @@ class Simjoin:
             raise SimjoinError(st, "simjoin_run")
         return out[:min(cnt, capacity)], cnt
 
-    def join_lsh(self, P, Q, threshold: float, L: int, k: int, seed: int, capacity: int, L_low: int = 0, out=None, kind: str = "ip"):
+    def join_lsh(self, P, Q, threshold: float, L: int, k: int, seed: int, capacity: int, L_low: int = 0, out=None, kind: str = "ip",
+                 family: str = "bits"):
         """LSH-bucketed join of two device tensors (simjoin_run_lsh).
         Returns (pairs[min(count, capacity), 2] int32 device tensor, count)."""
         import torch
@@ -224,7 +228,8 @@ class Simjoin:
         m = Q.shape[0]
         if out is None:
             out = torch.empty((max(int(capacity), 1), 2), dtype=torch.int32, device=P.device)
-        st, cnt = self.simjoin_run_lsh(P, n, Q, m, d, threshold, L, k, seed, out if capacity else None, capacity, L_low=L_low, kind=kind)
+        st, cnt = self.simjoin_run_lsh(P, n, Q, m, d, threshold, L, k, seed, out if capacity else None, capacity, L_low=L_low, kind=kind,
+                                       family=family)
         if st not in (SIMJOIN_OK, SIMJOIN_ERR_CAPACITY):
             raise SimjoinError(st, "simjoin_run_lsh")
         return out[:min(cnt, capacity)], cnt

@@ -31,6 +31,12 @@ constexpr int KIND_IP = 0, KIND_COS = 1, KIND_L2 = 2;
 // out[j * store_ld + i] = bf16(store_scale * <P_i, Q_j>).  This is the dense product Q * P^T with P the
 // small, resident operand: one level of the JL transform of Section 3.
 constexpr int KIND_STORE = 3;
+// KIND_SIGN (both element types): no predicate either -- the signs of the score tile are written out as hash keys.
+// P holds hyperplanes, 16 rows per repetition of the LSH join (unused rows are zero), Q the points: the 32 signs
+// [<P_i, Q_j> > 0] of the rows 32 w .. 32 w + 31 form word w of point j's key record, i.e. the 16-bit keys of
+// repetitions 2 w and 2 w + 1:  key_out[j * key_ld + w].  This is the random-hyperplane LSH of Section 4's LSH join
+// computed as the dense product it is; int8 projections are exact integers.
+constexpr int KIND_SIGN = 4;
 
 // One tile is 256 rows of P (two 128-row MMA blocks, both resident in shared memory) against 128 rows of Q.
 // Every Q chunk that arrives is multiplied with both P blocks, so a tile needs half the L2 -> shared-memory
@@ -135,6 +141,9 @@ struct JoinParams {
     // BF16/L2, ALT: the tile test is a filter  s >= (l2_xscale |x|^2 - l2_thr_filter) / 2 + l2_ycoef |y|^2, lowered by the
     // error bound so that every pair the difference form accepts is a candidate
     float l2_xscale, l2_ycoef, l2_thr_filter;
+    // KIND_SIGN
+    uint32_t *key_out;
+    long long key_ld;              // 32-bit words per key record
     // KIND_STORE
     uint16_t *store_out;
     long long store_ld;
@@ -743,9 +752,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     // or tensor-memory allocation exists)
     if (p_in.zero_next != nullptr && blockIdx.x == 0 && threadIdx.x < 8) p_in.zero_next[threadIdx.x] = 0ull;
     if (p_in.sel_mode != SEL_NONE && alt_selected(p_in) != ALT) return;
-    static_assert(!LONGK || (KC == 0 && KIND != KIND_STORE), "long-row mode: general join kinds only");
+    static_assert(!LONGK || (KC == 0 && KIND != KIND_STORE && KIND != KIND_SIGN), "long-row mode: general join kinds only");
+    static_assert(KIND != KIND_SIGN || (KC == 0 && !GROUPED && GEO == GEO_STD && !ALT), "hash keys: general path only");
     static_assert(!WIDEQ || (KC == 0 && !GROUPED && KIND == KIND_STORE), "wide-Q mode: store kind only");
-    static_assert(EW == NUM_EPI_WARPS || (EW == 2 * NUM_EPI_WARPS && GEO == GEO_STD && KIND != KIND_STORE), "16 epilogue warps: join kinds, standard geometry");
+    static_assert(EW == NUM_EPI_WARPS || (EW == 2 * NUM_EPI_WARPS && GEO == GEO_STD && KIND != KIND_STORE && KIND != KIND_SIGN), "16 epilogue warps: join kinds, standard geometry");
     constexpr int TN = (LONGK || WIDEQ) ? LONG_TN : TILE_N;   // rows of Q per tile
     constexpr int NPASS = TN / TILE_N;                     // 128-column passes of the epilogue over a P block's columns
     constexpr int ECOLS = epi_cols(EW);                    // accumulator columns per epilogue warp and pass
@@ -766,7 +776,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     // Aligned sweeps (no per-CTA rotation): bucketed units are short, and the store kind reads the streamed
     // operand once per 256-row tile of the resident one -- the CTAs that share a segment then walk it in
     // step, so that the second reader finds the tile in L2 (measured: rotated, that level read its input twice).
-    constexpr bool ALIGNED = GROUPED || KIND == KIND_STORE;
+    constexpr bool ALIGNED = GROUPED || KIND == KIND_STORE || KIND == KIND_SIGN;
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128-byte swizzle pattern repeats every 1024 bytes.
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -877,7 +887,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         // barrier that is still one phase behind, and a parity wait cannot tell phases two apart.
         // In that case warp 1 issues every tile and warp 3 stays out.
         const bool fast = p.stationary && p.epi_release && p.last_ksteps == 4;
-        constexpr bool OB = KIND == KIND_STORE;
+        constexpr bool OB = KIND == KIND_STORE || KIND == KIND_SIGN;
         if constexpr (LONGK) {
             if (warp == 1) mma_issuer_long<DT, GROUPED>(p, ctrl, smem_ring, tmem_base, lane);
         } else if (fast && p.kc == 1 && !WIDEQ) mma_issuer_role<DT, 1, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
@@ -1015,6 +1025,36 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                         }
                     }
                     __syncwarp();
+                }
+                if constexpr (KIND == KIND_SIGN) {
+                    // lane <-> hyperplane (row of P), columns <-> points (rows of Q).  One vote per column collects the
+                    // signs of this warp's 32 hyperplanes for that point; lane c keeps the words of columns c, c + 32, ...
+                    // and stores them into the points' key records.
+                    const long long j0 = q_base + (long long)qt * TN;
+                    const int plane0 = un.pb * P_ROWS + half * TILE_M + quarter * 32;      // first hyperplane of this warp
+                    const bool have = plane0 < (int)p.n && (half == 0 || two_blocks);
+                    uint32_t v[TILE_N];
+                    if (have) tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TILE_N, v, std::false_type{});
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                    if (have) {
+                        uint32_t keep[TILE_N / 32] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                        for (int c = 0; c < TILE_N; ++c) {
+                            const bool pos = DT == DT_I8 ? (int)v[c] > 0 : __uint_as_float(v[c]) > 0.f;
+                            const uint32_t word = __ballot_sync(0xffffffffu, pos);
+                            if ((c & 31) == lane) keep[c >> 5] = word;
+                        }
+#pragma unroll
+                        for (int q = 0; q < TILE_N / 32; ++q) {
+                            const long long j = j0 + 32 * q + lane;
+                            if (j < q_end) p.key_out[j * p.key_ld + (plane0 >> 5)] = keep[q];
+                        }
+                    }
+                    acc ^= 1;
+                    if (acc == 0) accphase ^= 1;
+                    continue;
                 }
                 if constexpr (KIND == KIND_STORE) {
                     // lane <-> row of P (an output coordinate), columns <-> rows of Q (output rows).  With two P

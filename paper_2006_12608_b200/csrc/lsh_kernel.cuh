@@ -2,11 +2,14 @@
 // concatenation of k base hashes, and for each repetition regroup the rows of P and Q so that every
 // bucket is one contiguous row range, then list the (P row block, Q bucket) units the join kernel sweeps.
 //
-// Base hash: bit sampling, h(x) = [x_c > 0] for a sampled coordinate c -- the classic monotone family
+// Base hash, first family: bit sampling, h(x) = [x_c > 0] for a sampled coordinate c -- the classic monotone family
 // for Hamming distance / +-1 data, and for bf16 rows the sign of the sampled coordinate (the random-hyperplane
 // hash of the angular distance with axis-aligned hyperplanes; a bf16 value is positive exactly when its bit
-// pattern, read as int16, is).  The coordinate of repetition l, bit b is
-// splitmix64(seed, l * 64 + b) mod d, a counter-based generator, so nothing random is stored.
+// pattern, read as int16, is).  The k bits of a repetition sample k distinct coordinates, drawn from a counter-based
+// generator (lsh_coordinates_kernel), so nothing random is stored.
+// Second family: random hyperplanes, h(x) = [<a, x> > 0] with a a vector of random signs from the same generator
+// (lsh_hyperplanes_kernel); the projections of all points onto all hyperplanes are one dense product, which the
+// tile kernel computes with a sign-collecting epilogue (KIND_SIGN).
 #pragma once
 #include <cstdint>
 
@@ -43,6 +46,26 @@ __global__ void __launch_bounds__(64) lsh_coordinates_kernel(unsigned long long 
         }
     }
 }
+// The hyperplanes of the second family as a matrix for the tile kernel: 16 rows per repetition, row 16 l + b the
+// hyperplane of repetition l, bit b -- coordinate c is +1 when bit 0 of splitmix64(seed, 2^60 + (64 l + b) 2^20 + c) is
+// set and -1 otherwise -- and zero rows for the bits a repetition does not use (b >= k, or k - 1 in the last L_low
+// repetitions) and for the padding repetitions up to `reps_padded`.  T: int8_t, or uint16_t holding bf16 bit patterns.
+template <typename T>
+__global__ void __launch_bounds__(256) lsh_hyperplanes_kernel(unsigned long long seed, int L_high, int L_low, int k, int d,
+                                                              int reps_padded, T *__restrict__ planes) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (long long)reps_padded * 16 * d) return;
+    const int c = (int)(t % d), row = (int)(t / d), l = row >> 4, b = row & 15;
+    const int bits = l < L_high ? k : (l < L_high + L_low ? k - 1 : 0);
+    T val = 0;
+    if (b < bits) {
+        const bool plus = lsh_splitmix64(seed, (1ULL << 60) + (((uint64_t)l * 64u + (uint64_t)b) << 20) + (uint64_t)c) & 1u;
+        if constexpr (sizeof(T) == 1) val = plus ? (T)1 : (T)-1;
+        else val = plus ? (T)0x3F80 : (T)0xBF80;            // +-1.0 in bf16
+    }
+    planes[t] = val;
+}
+
 __device__ __forceinline__ void lsh_load_coordinates(const int *__restrict__ coords, int L, int k, int *s_coord) {
     for (int t = threadIdx.x; t < L * k; t += blockDim.x) s_coord[t] = coords[t];
 }

@@ -84,6 +84,8 @@ struct simjoin_ctx {
     DevBuf filter_out;                  // simjoin_filter_pairs: the kept pairs before they replace the list
     // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
     DevBuf lsh_keys_p, lsh_keys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
+    DevBuf lsh_planes;                  // hyperplane family: 16 rows per repetition
+    bool attr_set_sign[2];
 };
 
 namespace {
@@ -529,6 +531,33 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
 }
 
+// Hash keys of the hyperplane family for all rows of X: the tile kernel with the hyperplane matrix as the resident
+// operand, the points as the streamed one and the sign-collecting epilogue; writes the key records.
+template <int DT>
+simjoin_status hyperplane_keys(simjoin_ctx *ctx, const void *planes, int plane_rows, const void *X, int64_t rows, int32_t d,
+                               void *rec, int rec_words) {
+    const size_t es = elem_size(ctx->dtype);
+    JoinParams jp;
+    size_t smem = 0;
+    if (!tile_geometry(ctx, plane_rows, rows, (int)(d * es), es, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
+    jp.PB = (plane_rows + P_ROWS - 1) / P_ROWS;
+    jp.QT = (int)((rows + TILE_N - 1) / TILE_N);
+    jp.qpanel = jp.QT;                 // the points are read once per 256 hyperplanes: one long sweep per CTA
+    jp.counter = ctx->d_ctrl;
+    jp.status = reinterpret_cast<unsigned int *>(ctx->d_ctrl + 1);
+    jp.key_out = reinterpret_cast<uint32_t *>(rec);
+    jp.key_ld = (long long)rec_words * 4;
+    CUtensorMap mapA, mapX;
+    if (!encode_rows_map(ctx, &mapA, planes, plane_rows, d, P_ROWS) || !encode_rows_map(ctx, &mapX, X, rows, d, TILE_N)) return SIMJOIN_ERR_CUDA;
+    auto kern = join_kernel<DT, KIND_SIGN, false, 0, false, GEO_STD>;
+    if (!ctx->attr_set_sign[DT]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        ctx->attr_set_sign[DT] = true;
+    }
+    kern<<<ctx->num_sms, NUM_THREADS, smem, ctx->stream>>>(mapA, mapX, jp);
+    return cudaGetLastError() == cudaSuccess ? SIMJOIN_OK : SIMJOIN_ERR_CUDA;
+}
+
 // One bucketed join launch: instantiation by element type, kind, variant and geometry.
 cudaError_t launch_bucketed(simjoin_ctx *ctx, bool i8, simjoin_kind kind, bool longk, const CUtensorMap &mp,
                             const CUtensorMap &mq, const JoinParams &jp, size_t smem) {
@@ -554,8 +583,8 @@ cudaError_t launch_bucketed(simjoin_ctx *ctx, bool i8, simjoin_kind kind, bool l
 }
 
 simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d, simjoin_kind kind,
-                          double threshold, int32_t L, int32_t L_low, int32_t k, uint64_t seed, int32_t *out_pairs,
-                          uint64_t capacity, uint64_t *count) {
+                          double threshold, simjoin_lsh_family family, int32_t L, int32_t L_low, int32_t k, uint64_t seed,
+                          int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
     *count = 0;
     ctx->have_timing = false;
     if (n == 0 || m == 0) return SIMJOIN_OK;
@@ -641,7 +670,23 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         return SIMJOIN_ERR_CUDA;
 
     cudaEventRecord(ctx->ev[0], s);
-    {
+    if (family == SIMJOIN_LSH_HYPERPLANES) {
+        // all projections of all points at once: (points) x (16 rows per repetition, padded to whole key words)
+        const int plane_rows = stride * 16;
+        if (!grow(ctx->lsh_planes, (size_t)plane_rows * row_bytes)) return SIMJOIN_ERR_CUDA;
+        const unsigned pblocks = (unsigned)(((long long)plane_rows * d + 255) / 256);
+        simjoin_status hs;
+        if (i8) {
+            lsh_hyperplanes_kernel<<<pblocks, 256, 0, s>>>(seed, L, L_low, k, d, stride, reinterpret_cast<int8_t *>(ctx->lsh_planes.ptr));
+            hs = hyperplane_keys<DT_I8>(ctx, ctx->lsh_planes.ptr, plane_rows, P, n, d, keys_p, rec_words);
+            if (hs == SIMJOIN_OK) hs = hyperplane_keys<DT_I8>(ctx, ctx->lsh_planes.ptr, plane_rows, Q, m, d, keys_q, rec_words);
+        } else {
+            lsh_hyperplanes_kernel<<<pblocks, 256, 0, s>>>(seed, L, L_low, k, d, stride, reinterpret_cast<uint16_t *>(ctx->lsh_planes.ptr));
+            hs = hyperplane_keys<DT_BF16>(ctx, ctx->lsh_planes.ptr, plane_rows, P, n, d, keys_p, rec_words);
+            if (hs == SIMJOIN_OK) hs = hyperplane_keys<DT_BF16>(ctx, ctx->lsh_planes.ptr, plane_rows, Q, m, d, keys_q, rec_words);
+        }
+        if (hs != SIMJOIN_OK) return hs;
+    } else {
         const unsigned bn = (unsigned)((n + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), bm = (unsigned)((m + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS);
         const size_t sm = (size_t)LSH_KEYS_STAGED_ROWS * (row_bytes / 4 + 1) * 4;
         const bool staged = row_bytes <= LSH_KEYS_STAGED_MAX_D;
@@ -721,7 +766,8 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     return *count > capacity ? SIMJOIN_ERR_CAPACITY : SIMJOIN_OK;
 }
 
-simjoin_status check_lsh_args(int32_t L, int32_t L_low, int32_t k) {
+simjoin_status check_lsh_args(int32_t L, int32_t L_low, int32_t k, simjoin_lsh_family family = SIMJOIN_LSH_BITS) {
+    if (family != SIMJOIN_LSH_BITS && family != SIMJOIN_LSH_HYPERPLANES) return SIMJOIN_ERR_ARG;
     if (L < 0 || L_low < 0 || L + L_low < 1 || L + L_low > LSH_MAX_REPS || k < 0 || (L_low > 0 && k < 1)) return SIMJOIN_ERR_ARG;
     if (k > LSH_MAX_BITS) return SIMJOIN_ERR_UNSUPPORTED;
     return SIMJOIN_OK;
@@ -942,6 +988,7 @@ simjoin_status simjoin_create(simjoin_ctx **out, simjoin_dtype dtype, int device
     std::memset(ctx->attr_set_long, 0, sizeof ctx->attr_set_long);
     ctx->attr_set_wideq = false;
     std::memset(ctx->attr_set_dense, 0, sizeof ctx->attr_set_dense);
+    ctx->attr_set_sign[0] = ctx->attr_set_sign[1] = false;
     ctx->dense_mode = 2;
     ctx->last_density = -1.0;
     ctx->copy_stream = nullptr;
@@ -987,6 +1034,7 @@ simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
     release(ctx->lsh_sorted_p);
     release(ctx->lsh_sorted_q);
     release(ctx->lsh_misc);
+    release(ctx->lsh_planes);
     for (auto &e : ctx->copy_ev)
         if (e) cudaEventDestroy(e);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -1152,18 +1200,18 @@ simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t
 }
 
 simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
-                               simjoin_kind kind, double threshold, int32_t L, int32_t L_low, int32_t k, uint64_t seed,
-                               int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
+                               simjoin_kind kind, double threshold, simjoin_lsh_family family, int32_t L, int32_t L_low, int32_t k,
+                               uint64_t seed, int32_t *out_pairs, uint64_t capacity, uint64_t *count) {
     simjoin_status st = check_join_args(ctx, P, n, Q, m, d, kind, threshold, out_pairs, capacity, count);
     if (st != SIMJOIN_OK) return st;
-    st = check_lsh_args(L, L_low, k);
+    st = check_lsh_args(L, L_low, k, family);
     if (st != SIMJOIN_OK) return st;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SIMJOIN_ERR_CUDA;
     if ((n > 0 && !is_device_ptr(P, ctx->device)) || (m > 0 && !is_device_ptr(Q, ctx->device))) return SIMJOIN_ERR_ARG;
     if (capacity > 0 && !is_device_ptr(out_pairs, ctx->device)) return SIMJOIN_ERR_ARG;
     if (capacity > 0 && (reinterpret_cast<uintptr_t>(out_pairs) & 7u) != 0) return SIMJOIN_ERR_UNSUPPORTED;
-    return lsh_device(ctx, P, n, Q, m, d, kind, threshold, L, L_low, k, seed, out_pairs, capacity, count);
+    return lsh_device(ctx, P, n, Q, m, d, kind, threshold, family, L, L_low, k, seed, out_pairs, capacity, count);
 }
 
 simjoin_status simjoin_run_hamming_lsh(simjoin_ctx *ctx, const void *P_bits, int64_t n, const void *Q_bits, int64_t m, int32_t d,
@@ -1178,7 +1226,7 @@ simjoin_status simjoin_run_hamming_lsh(simjoin_ctx *ctx, const void *P_bits, int
     st = hamming_unpack(ctx, P_bits, n, Q_bits, m, d, out_pairs, capacity, count);
     if (st != SIMJOIN_OK || n == 0 || m == 0) return st;
     const double t = (double)d - 2.0 * std::floor(r);
-    return lsh_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, SIMJOIN_IP, t, L, L_low, k, seed, out_pairs, capacity, count);
+    return lsh_device(ctx, ctx->stage_p.ptr, n, ctx->stage_q.ptr, m, d, SIMJOIN_IP, t, SIMJOIN_LSH_BITS, L, L_low, k, seed, out_pairs, capacity, count);
 }
 
 simjoin_status simjoin_jl_transform(simjoin_ctx *ctx, const void *X, int64_t n, int32_t d, int32_t k, uint64_t seed, void *out) {

@@ -238,3 +238,82 @@ def test_lsh_more_key_bits_than_coordinates(ctx_bf16, ctx):
     Qi[:200] = Pi[:200]
     assert check(ctx, Pi, Qi, 6.0, 4, 12, 3) >= 200
 
+
+
+# ------------------------------------------------------------------ the random-hyperplane family (keys on the tensor cores)
+def run_family(ctx, P, Q, kind, t, L, k, seed, L_low=0, cap=1 << 21, family="hyperplanes"):
+    dP, dQ = B.to_device(P), B.to_device(Q)
+    out = torch.full((cap + 2, 2), -5, dtype=torch.int32, device="cuda:0")
+    st, cnt = ctx.simjoin_run_lsh(dP, P.shape[0], dQ, Q.shape[0], P.shape[1], t, L, k, seed, out, cap, L_low=L_low, kind=kind, family=family)
+    assert st == B.SIMJOIN_OK, B.strerror(st)
+    host = out.cpu().numpy()
+    assert np.all(host[cnt:] == -5)
+    got = keys(host[:cnt])
+    assert len(np.unique(got)) == cnt, "a pair was reported twice"
+    return got
+
+
+@pytest.mark.parametrize("kind", ["ip", "cos", "l2"])
+@pytest.mark.parametrize("n,m,d,L,L_low,k,hi", [(700, 600, 128, 5, 0, 4, 1), (129, 257, 64, 3, 2, 1, 3), (5000, 7000, 144, 4, 1, 6, 127),
+                                               (3000, 2500, 16, 2, 0, 12, 5), (900, 1100, 640, 17, 0, 3, 3), (600, 500, 2064, 3, 1, 5, 127),
+                                               (1500, 1800, 256, 33, 2, 2, 2)])
+def test_hyperplane_lsh_join_int8_is_exact(ctx, kind, n, m, d, L, L_low, k, hi):
+    """int8 projections are exact integers, so the keys -- and with them the result -- equal the oracle's bit for bit:
+    one and several key words per record (L + L_low up to 35: three P tiles of hyperplanes), partial chunks, rows that
+    stream both operands, values up to +-127 (projections up to 2^18)."""
+    P, Q = W.random_points("i8", n, d, 201, lo=-hi, hi=hi), W.random_points("i8", m, d, 202, lo=-hi, hi=hi)
+    kp = min(n, m, 200) // 2
+    Q[:kp] = P[:kp]
+    Q[kp:2 * kp:2] = -P[kp:2 * kp:2]                      # opposite points: every bit differs
+    P[7] = 0                                              # projections of exactly zero hash to bit 0
+    smp = np.stack([np.arange(kp), np.arange(kp)], axis=1).astype(np.int32)
+    sc = O.scores(P, Q, kind, "i8", smp).astype(np.float64)
+    t = {"ip": float(np.quantile(sc, 0.3)), "cos": 0.95, "l2": 0.5}[kind]
+    got = run_family(ctx, P, Q, kind, t, L, k, 4242 + k, L_low=L_low)
+    want, wcnt = O.lsh_join_kind(P, Q, kind, t, "i8", L, k, 4242 + k, L_low=L_low, family="hyperplanes")
+    assert len(got) == wcnt and np.array_equal(got, keys(want)) and wcnt > 0
+
+
+@pytest.mark.parametrize("kind", ["ip", "cos", "l2"])
+@pytest.mark.parametrize("d,L,k", [(128, 4, 3), (64, 3, 5), (264, 3, 2), (1040, 2, 4)])
+def test_hyperplane_lsh_join_bf16_within_the_band(ctx_bf16, kind, d, L, k):
+    """bf16: the threshold band of the join, and a band on the hash as well -- a projection too close to zero for fp32
+    accumulation to decide may put the point on either side, so the result lies between the strict and the loose
+    collision sets of the oracle."""
+    w = W.make_workload(2, n=1800 + 11, m=2100 + 3, d=d, planted=300)
+    t = {"ip": 0.85, "cos": 0.85, "l2": 0.55}[kind]
+    got = run_family(ctx_bf16, w.P, w.Q, kind, t, L, k, 23, L_low=1)
+    strict, exact, loose = O.lsh_band_sets(w.P, w.Q, kind, t, "bf16", L, k, 23, L_low=1, family="hyperplanes")
+    assert np.isin(keys(strict), got).all() and np.isin(got, keys(loose)).all(), (kind, d, len(got), len(strict), len(loose))
+    assert len(strict) >= 50 and len(loose) - len(strict) <= max(3, len(loose) // 50)
+
+
+def test_hyperplane_lsh_recall_on_anisotropic_data_beats_coordinate_signs(ctx_bf16):
+    """16 of 128 coordinates are five times larger than the rest and carry the difference inside a near pair, as in the
+    oracle's collision-law pin: sampled-coordinate signs see mostly the 112 small, equal coordinates, so near and
+    far-but-equal-on-the-small-coordinates pairs collide alike; hyperplanes follow the angle."""
+    rng = np.random.default_rng(5)
+    n, d, big = 4000, 128, 16
+    scale = np.ones(d, dtype=np.float32)
+    scale[:big] = 5.0
+    Pf = rng.standard_normal((n, d)).astype(np.float32) * scale
+    Qf = rng.standard_normal((n, d)).astype(np.float32) * scale
+    Qf[:400] = Pf[:400]
+    Qf[:400, :big] += 0.25 * 5.0 * rng.standard_normal((400, big)).astype(np.float32)        # near pairs, cosine about 0.97
+    P, Q = W.f32_to_bf16_bits(Pf), W.f32_to_bf16_bits(Qf)
+    t = 0.93
+    full = keys(O.join(P, Q, "cos", t, "bf16")[0])
+    assert 380 <= len(full) <= 420
+    L, k = 6, 8
+    hp = run_family(ctx_bf16, P, Q, "cos", t, L, k, 9)
+    recall_hp = np.isin(full, hp).mean()
+    want = 1.0 - (1.0 - (1.0 - np.arccos(0.97) / np.pi) ** k) ** L
+    assert abs(recall_hp - want) < 0.08, (recall_hp, want)
+
+
+def test_hyperplane_lsh_argument_checks(ctx):
+    X = B.to_device(W.random_points("i8", 64, 64, 1))
+    out = torch.zeros((8, 2), dtype=torch.int32, device="cuda:0")
+    assert ctx.simjoin_run_lsh(X, 64, X, 64, 64, 10.0, 2, 3, 1, out, 8, family=7)[0] == B.SIMJOIN_ERR_ARG
+    assert ctx.simjoin_run_lsh(X, 64, X, 64, 64, 10.0, 2, 13, 1, out, 8, family="hyperplanes")[0] == B.SIMJOIN_ERR_UNSUPPORTED
+    assert ctx.simjoin_run_lsh(X, 0, X, 64, 64, 10.0, 2, 3, 1, out, 8, family="hyperplanes") == (B.SIMJOIN_OK, 0)
