@@ -45,7 +45,7 @@ UNIT = "TOPS"
 NOMINAL_TOPS = {"i8": 4500.0, "bf16": 2250.0}          # dense, per GPU (context only)
 # DRAM bytes per join-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum), from a one-pass ncu
 # capture of the full-size launch (profiles/join_kernel_dram_traffic_cfg4_full.md).
-NCU_TRAFFIC_BYTES = {4: 699.35e6 + 5.83e6}
+NCU_TRAFFIC_BYTES = {4: 690.11e6 + 5.89e6}
 # the same for all levels of one JL transform call, keyed by (n, d, k) (profiles/jl_transform_*.md)
 # captured at n = 262144 (1.2956e9 read + 0.6277e9 written); the 1 048 576-point entry is that x 4 (every level's
 # traffic is proportional to n)
