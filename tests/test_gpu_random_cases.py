@@ -14,7 +14,7 @@ from paper_2006_12608_b200 import build
 from paper_2006_12608_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
-ROW_BYTES = [16, 32, 48, 64, 96, 128, 144, 256, 272, 384, 400, 512, 528, 640, 1024, 1040, 2048, 2064, 4096]
+ROW_BYTES = [16, 32, 48, 64, 96, 128, 128, 144, 256, 256, 272, 384, 400, 512, 528, 640, 1024, 1040, 2048, 2064, 4096]
 
 
 def keys(p):
@@ -59,25 +59,29 @@ def test_random_cases_match_the_oracle(seed):
             ctx = ctxs[dtype]
             if dtype == "i8":     # small joins: the device's choice of the epilogue width, or the 32-bit one unasked
                 assert ctx.simjoin_set_option(B.SIMJOIN_OPT_SELECT_MIN_OPS, 0.0 if rng.random() < 0.7 else 2e11) == B.SIMJOIN_OK
+            else:                 # 8 or 16 epilogue warps (where both exist), or by the previous call's density
+                assert ctx.simjoin_set_option(B.SIMJOIN_OPT_DENSE_EPILOGUE, float(rng.integers(0, 3))) == B.SIMJOIN_OK
             dP, dQ = B.to_device(P), B.to_device(Q)
             out.fill_(-5)
             L = k = L_low = 0
+            family = "bits"
             if lsh:
                 L, k = int(rng.integers(1, 5)), int(rng.integers(0, 6))
                 L_low = int(rng.integers(0, 2)) if k >= 1 else 0
-                st, cnt = ctx.simjoin_run_lsh(dP, n, dQ, m, d, t, L, k, s1, out, cap, L_low=L_low, kind=kind)
+                family = "hyperplanes" if rng.random() < 0.4 else "bits"
+                st, cnt = ctx.simjoin_run_lsh(dP, n, dQ, m, d, t, L, k, s1, out, cap, L_low=L_low, kind=kind, family=family)
             else:
                 st, cnt = ctx.simjoin_run(dP, n, dQ, m, d, kind, t, out, cap)
-            what = dict(case=case, dtype=dtype, kind=kind, n=n, m=m, d=d, t=t, lsh=(L, k, L_low) if lsh else None, s1=s1, s2=s2)
+            what = dict(case=case, dtype=dtype, kind=kind, n=n, m=m, d=d, t=t, lsh=(L, k, L_low, family) if lsh else None, s1=s1, s2=s2)
             assert st == B.SIMJOIN_OK, (B.strerror(st), what)
             host = out.cpu().numpy()
             got = keys(host[:cnt])
             assert np.all(host[cnt:] == -5) and len(np.unique(got)) == cnt, what
             if dtype == "i8":
-                want = O.lsh_join_kind(P, Q, kind, t, dtype, L, k, s1, L_low=L_low)[0] if lsh else O.join(P, Q, kind, t, dtype)[0]
+                want = O.lsh_join_kind(P, Q, kind, t, dtype, L, k, s1, L_low=L_low, family=family)[0] if lsh else O.join(P, Q, kind, t, dtype)[0]
                 assert np.array_equal(got, keys(want)), what
             else:
-                sets = O.lsh_band_sets(P, Q, kind, t, dtype, L, k, s1, L_low=L_low) if lsh else O.band_sets(P, Q, kind, t, dtype)
+                sets = O.lsh_band_sets(P, Q, kind, t, dtype, L, k, s1, L_low=L_low, family=family) if lsh else O.band_sets(P, Q, kind, t, dtype)
                 assert np.isin(keys(sets[0]), got).all() and np.isin(got, keys(sets[2])).all(), what
             # the pair filter on a random candidate list of the same points (plus some reported pairs)
             if rng.random() < 0.5:
