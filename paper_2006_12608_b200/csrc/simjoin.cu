@@ -60,7 +60,7 @@ struct simjoin_ctx {
     int num_sms;
     int max_smem_optin;
     EncodeTiledFn encode;
-    DevBuf nx, ny, qstat, pstat;        // row terms and per-tile bounds
+    DevBuf nx, ny, qstat;               // row terms and per-tile bounds
     DevBuf stage_p, stage_q, stage_out; // device staging of simjoin_run_host
     unsigned long long *d_ctrl;         // two 64-byte control blocks (layout: JoinScratch::d_ctrl)
     unsigned long long *h_ctrl;         // pinned mirror
@@ -1017,7 +1017,6 @@ simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
     release(ctx->nx);
     release(ctx->ny);
     release(ctx->qstat);
-    release(ctx->pstat);
     release(ctx->stage_p);
     release(ctx->stage_q);
     release(ctx->stage_out);
