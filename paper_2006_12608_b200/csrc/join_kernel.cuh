@@ -130,6 +130,7 @@ struct JoinParams {
     const unsigned int *sel_words;
     int sel_mode;
     float sel_coef;
+    float sel_r2;                  // SEL_L2_RADIUS: r^2 (the kernel's own threshold differs when it runs on transformed operands)
     // When not null: a 64-byte control block that no launch of this call reads or writes.  The kernel zeroes it, so
     // that the caller's next join finds its counter, status and selection words cleared without a memset of its own.
     unsigned long long *zero_next;
@@ -157,7 +158,7 @@ constexpr float L2_BAND_SHARE = 0.019f;
 __device__ __forceinline__ bool alt_selected(const JoinParams &p) {
     const unsigned int a = __ldg(p.sel_words), b = __ldg(p.sel_words + 1);
     if (p.sel_mode == SEL_I8_RANGE) return (unsigned long long)p.row_bytes * a * b <= 32767ull;
-    return p.sel_coef * (__uint_as_float(a) + __uint_as_float(b)) > L2_BAND_SHARE * p.thr_f;
+    return p.sel_coef * (__uint_as_float(a) + __uint_as_float(b)) > L2_BAND_SHARE * p.sel_r2;
 }
 
 struct Ctrl {

@@ -85,6 +85,7 @@ struct simjoin_ctx {
     // LSH join scratch: hash keys, regrouping permutations, regrouped copies of P and Q, histograms + work list
     DevBuf lsh_keys_p, lsh_keys_q, lsh_perm_p, lsh_perm_q, lsh_sorted_p, lsh_sorted_q, lsh_misc;
     DevBuf lsh_planes;                  // hyperplane family: 16 rows per repetition
+    DevBuf emb_p, emb_q;                // dense Euclidean joins: the point sets with the squared-L2 embedding coordinates appended
     bool attr_set_sign[2];
 };
 
@@ -345,6 +346,50 @@ int norm_mode(bool /*i8*/, simjoin_kind kind, double threshold) {
     return (float)threshold > 0.f ? 2 : 1;        // decided on the fp32 threshold the epilogue uses
 }
 
+// The plain form of a dense bf16 Euclidean join through the operand transform of l2_embed_rows_kernel: both point sets are
+// copied with 8 coordinates appended (context-owned buffers), and the 16-epilogue-warp inner-product kernel runs on the
+// copies with the constant threshold -r^2/2.  The copies' rows are padded with zeros to whole 128-byte chunks, so the
+// whole-chunk instantiations apply and every box row is an aligned line.  Returns ERR_UNSUPPORTED (nothing launched)
+// when the transformed rows do not fit two chunks.  `jp_l2`: the Euclidean join's parameters (norms already computed).
+simjoin_status launch_l2_embedded(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
+                                  const JoinScratch &scr, const JoinParams &jp_l2, int grid) {
+    if ((d + 8) * 2 > 2 * CHUNK_BYTES) return SIMJOIN_ERR_UNSUPPORTED;
+    const int row_bytes = ((d + 8) * 2 + CHUNK_BYTES - 1) / CHUNK_BYTES * CHUNK_BYTES, de = row_bytes / 2;      // whole chunks
+    JoinParams jp;
+    size_t smem = 0;
+    if (!tile_geometry(ctx, n, m, row_bytes, 2, jp, smem)) return SIMJOIN_ERR_UNSUPPORTED;
+    if (!dense_available(false, jp)) return SIMJOIN_ERR_UNSUPPORTED;
+    if (!grow(ctx->emb_p, (size_t)n * row_bytes) || !grow(ctx->emb_q, (size_t)m * row_bytes)) return SIMJOIN_ERR_CUDA;
+    const int g = d * 2 / 16, gout = row_bytes / 16;
+    l2_embed_rows_kernel<<<(unsigned)(((long long)n * gout + 255) / 256), 256, 0, ctx->stream>>>(
+        reinterpret_cast<const uint4 *>(P), reinterpret_cast<const float *>(scr.nx), n, g, gout, 0, reinterpret_cast<uint4 *>(ctx->emb_p.ptr));
+    l2_embed_rows_kernel<<<(unsigned)(((long long)m * gout + 255) / 256), 256, 0, ctx->stream>>>(
+        reinterpret_cast<const uint4 *>(Q), reinterpret_cast<const float *>(scr.ny), m, g, gout, 1, reinterpret_cast<uint4 *>(ctx->emb_q.ptr));
+    if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
+    jp.PB = jp_l2.PB;
+    jp.QT = jp_l2.QT;
+    jp.qpanel = q_panel_tiles(jp.QT, row_bytes, TILE_N);
+    jp.out = jp_l2.out;
+    jp.capacity = jp_l2.capacity;
+    jp.counter = jp_l2.counter;
+    jp.status = jp_l2.status;
+    jp.ioff = jp_l2.ioff;
+    jp.joff = jp_l2.joff;
+    jp.zero_next = jp_l2.zero_next;
+    jp.host_result = jp_l2.host_result;
+    jp.done_ticket = jp_l2.done_ticket;
+    jp.sel_mode = jp_l2.sel_mode;               // runs only when the selection words call for the plain form
+    jp.sel_words = jp_l2.sel_words;
+    jp.sel_coef = jp_l2.sel_coef;
+    jp.sel_r2 = jp_l2.sel_r2;
+    jp.thr_f = -0.5f * jp_l2.thr_f;             // <x', y'> = -|x - y|^2 / 2 >= -r^2 / 2
+    jp.thr_d = -0.5 * (double)jp_l2.thr_f;
+    CUtensorMap mapP, mapQ;
+    if (!encode_rows_map(ctx, &mapP, ctx->emb_p.ptr, n, de, P_ROWS) || !encode_rows_map(ctx, &mapQ, ctx->emb_q.ptr, m, de, TILE_N))
+        return SIMJOIN_ERR_CUDA;
+    return launch_join_dense<KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem) == cudaSuccess ? SIMJOIN_OK : SIMJOIN_ERR_CUDA;
+}
+
 // One launch of the brute-force join kernel in the geometry the rows call for.
 template <int DT, int KIND, bool ALT>
 cudaError_t launch_geo(simjoin_ctx *ctx, bool longk, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid,
@@ -369,6 +414,7 @@ void set_selection(JoinParams &jp, bool i8, simjoin_kind kind, unsigned long lon
     } else if (kind == SIMJOIN_L2) {
         jp.sel_mode = SEL_L2_RADIUS;
         jp.sel_words = reinterpret_cast<const unsigned int *>(d_ctrl + 3);
+        jp.sel_r2 = jp.thr_f;
     }
 }
 
@@ -502,7 +548,13 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         if (kind == SIMJOIN_IP) e = launch_join_dense<KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
         else if (kind == SIMJOIN_COS) e = launch_join_dense<KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem);
         else {
-            e = launch_join_dense<KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
+            // The plain form of the dense Euclidean join runs as an inner-product join on transformed operands where the
+            // transformed rows still fit two chunks (Section 4's squared-L2 embedding: l2_embed_rows_kernel); the
+            // small-radius form stays on the points themselves.  Whichever the selection words call for does the work.
+            const simjoin_status es2 = fixed ? SIMJOIN_ERR_UNSUPPORTED
+                                             : launch_l2_embedded(ctx, P, n, Q, m, d, scr, jp, grid);
+            if (es2 == SIMJOIN_ERR_CUDA) return SIMJOIN_ERR_CUDA;
+            e = es2 == SIMJOIN_OK ? cudaSuccess : launch_join_dense<KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
             if (e == cudaSuccess) e = launch_join_dense<KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
         }
     }
@@ -1034,6 +1086,8 @@ simjoin_status simjoin_destroy(simjoin_ctx *ctx) {
     release(ctx->lsh_sorted_q);
     release(ctx->lsh_misc);
     release(ctx->lsh_planes);
+    release(ctx->emb_p);
+    release(ctx->emb_q);
     for (auto &e : ctx->copy_ev)
         if (e) cudaEventDestroy(e);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);

@@ -514,8 +514,9 @@ def test_bf16_l2_radius_far_below_the_norms(ctx_bf16, d, r):
 @pytest.mark.parametrize("kind", ["ip", "cos", "l2"])
 @pytest.mark.parametrize("n,m,d", [(129, 257, 64), (700, 1300, 64), (513, 1000, 128), (300, 2100, 128), (140, 300, 72)])
 def test_bf16_dense_epilogue_matches_the_oracle(kind, n, m, d):
-    """The 16-epilogue-warp instantiations (rows of one or two whole chunks), forced on: sparse and dense outputs, ragged
-    tiles, hits in both 64-column halves of a block; other row lengths fall back to the regular kernel.  Then the default
+    """The 16-epilogue-warp instantiations (rows of one or two whole chunks; Euclidean joins of rows up to 240 bytes through
+    the operand transform), forced on: sparse and dense outputs, ragged tiles, hits in both 64-column halves of a block;
+    other row lengths fall back to the regular kernel.  Then the default
     mode, where a context switches to them after a dense join and back after a sparse one: same sets."""
     P, Q = W.random_points("bf16", n, d, 15), W.random_points("bf16", m, d, 16)
     Q[1:m:7][:n] = P[:len(Q[1:m:7][:n])]
@@ -529,6 +530,14 @@ def test_bf16_dense_epilogue_matches_the_oracle(kind, n, m, d):
                 pairs, cnt = gpu_join(ctx, P, Q, kind, t, capacity=1 << 22)
                 assert_band(pairs, cnt, P, Q, kind, t)
                 assert cnt > 0
+            if kind == "l2":
+                # A Euclidean join in the 16-warp layout runs on transformed operands (the squared-L2 embedding appended
+                # to copies of the rows) where those fit two chunks; a radius far below the norms must still select the
+                # form that decides candidates from the original rows: only the planted equal rows are that close.
+                for t in (0.01, 0.0):
+                    pairs, cnt = gpu_join(ctx, P, Q, kind, t, capacity=1 << 22)
+                    assert_band(pairs, cnt, P, Q, kind, t)
+                    assert cnt == len(Q[1:m:7][:n])
 
 
 def test_repeated_runs_give_the_same_set(ctx_bf16):
