@@ -338,6 +338,7 @@ def main():
     ap.add_argument("--kind", default=None, choices=["ip", "cos", "l2"],
                     help="join kind to run on the configuration's points instead of its own (give --threshold too)")
     ap.add_argument("--sigma-reading", default="radial")
+    ap.add_argument("--seed", type=int, default=0, help="seed of the synthetic inputs (rank r of a sharded run draws its P block with seed + r)")
     ap.add_argument("--lsh", default=None, metavar="L,k[,L_low]",
                     help="time the LSH-bucketed join of the configuration instead of the brute-force join: "
                          "L tables of k bits (+ L_low of k-1); not the headline metric, the line says so")
@@ -375,7 +376,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
     if args.impl == "reference":
-        w = W.make_workload(args.config, sigma_reading=args.sigma_reading, **size_kw(args)) if rank == 0 else None
+        w = W.make_workload(args.config, seed=args.seed, sigma_reading=args.sigma_reading, **size_kw(args)) if rank == 0 else None
         if w is not None and args.kind:
             w.kind = args.kind
         run_reference(args, w)
@@ -397,11 +398,11 @@ def main():
     B.load()
 
     # Each rank owns one row block of a (world * n)-row P and a full copy of Q.
-    w = W.make_workload(args.config, seed=rank, sigma_reading=args.sigma_reading, **size_kw(args))
+    w = W.make_workload(args.config, seed=args.seed + rank, sigma_reading=args.sigma_reading, **size_kw(args))
     if args.kind:
         w.kind = args.kind
     if world > 1:
-        w.Q = W.make_workload(args.config, seed=0, sigma_reading=args.sigma_reading, **size_kw(args)).Q if rank else w.Q
+        w.Q = W.make_workload(args.config, seed=args.seed, sigma_reading=args.sigma_reading, **size_kw(args)).Q if rank else w.Q
         w.planted = w.planted if rank == 0 else np.zeros((0, 2), np.int64)
     dev = torch.device("cuda", local_rank)
     dP, dQ = B.to_device(w.P, dev), B.to_device(w.Q, dev)
@@ -684,7 +685,7 @@ def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32" if w.dtype == "i8" else "f32", "data": "synthetic",
             "config": {"workload": w.name, "n": w.n, "m": w.m, "d": w.d, "kind": w.kind, "in_dtype": w.dtype,
-                       "threshold": w.threshold, "pairs_found": int(cnt),
+                       "threshold": w.threshold, "pairs_found": int(cnt), "seed": args.seed,
                        "l2": ("inputs (P+Q) larger than L2; no flush" if w.P.nbytes + w.Q.nbytes > 126e6
                               else "inputs (P+Q) fit in L2 and are not flushed between steps: not a headline number"),
                        "inputs_sha256": {"P": hashlib.sha256(w.P).hexdigest(), "Q": hashlib.sha256(w.Q).hexdigest()},

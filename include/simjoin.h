@@ -20,7 +20,8 @@
  *     columns otherwise: zero columns change no score).
  *   - Nothing the caller passes is freed or retained after a call returns.
  *     P and Q are only read.
- *   - No function throws, prints or exits; every failure is a status code.
+ *   - No function throws, prints or exits; every failure is a status code.  (With SIMJOIN_DEBUG=1 in the
+ *     environment simjoin_run writes one line per join to stderr: sizes, geometry, variant choice, count.)
  *   - A context is not thread-safe; use one per host thread / stream.
  */
 #ifndef SIMJOIN_H_

@@ -7,6 +7,7 @@
 
 #include <cmath>
 #include <cstdint>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -101,6 +102,15 @@ struct DeviceGuard {
         if (prev >= 0) cudaSetDevice(prev);
     }
 };
+
+// The library prints nothing unless the environment holds SIMJOIN_DEBUG=1: then one line per join on stderr.
+bool debug_log() {
+    static const bool on = [] {
+        const char *v = std::getenv("SIMJOIN_DEBUG");
+        return v && v[0] == '1';
+    }();
+    return on;
+}
 
 bool grow(DevBuf &b, size_t bytes) {
     if (bytes <= b.bytes) return true;
@@ -572,6 +582,13 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     if (kstatus != 0) return SIMJOIN_ERR_TIMEOUT;
     if (!fixed) ctx->ctrl_clean = cur ^ 1;        // the kernel has zeroed the other block
     *count = scr.h_ctrl[0];
+    if (debug_log())
+        std::fprintf(stderr, "[simjoin] run dtype=%s kind=%d n=%lld m=%lld d=%d t=%g: %d chunk(s) per row, %s geometry, %d ring stages, "
+                             "%s, pairs=%llu capacity=%llu\n",
+                     i8 ? "i8" : "bf16", (int)kind, (long long)n, (long long)m, (int)d, threshold, jp.kc,
+                     longk ? (jp.wave_gq ? "long-row (2-D waves)" : "long-row") : (jp.stationary ? "resident-P" : "streamed"), jp.nstages,
+                     jp.sel_mode == SEL_NONE ? "one variant" : (jp.sel_mode == SEL_I8_RANGE ? "epilogue width chosen on the device" : "Euclidean form chosen on the device"),
+                     (unsigned long long)*count, (unsigned long long)capacity);
     ctx->last_density = (double)*count / ((double)((n + 31) / 32) * (double)((m + 127) / 128));
     float a = 0.f, b = 0.f;
     if (timed && (!need_norms || cudaEventElapsedTime(&a, ctx->ev[0], ctx->ev[1]) == cudaSuccess) &&
