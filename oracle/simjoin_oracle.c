@@ -319,12 +319,19 @@ static uint64_t splitmix64_at(uint64_t seed, uint64_t idx) {
  * that no earlier bit of the repetition took -- bit sampling without replacement, so that a repetition of k bits
  * really has 2^k buckets (sampled with replacement, k = 7 of d = 128 coordinates repeat one in 15 % of the
  * repetitions).  From bit d on every coordinate is taken and a = 0 is used as it comes. */
+static int lsh_iid_sampling = 0;      /* 1: the k bits of a repetition are k independent samples (a coordinate may repeat) */
+
+/* Chooses between the two bit-sampling rules for the calls that follow: distinct coordinates within a repetition (0, the
+ * default) or the paper's plain concatenation of k independent base hashes (1), for which a pair at Hamming distance h
+ * collides in a repetition with probability exactly (1 - h/d)^k. */
+void oracle_lsh_set_iid_sampling(int32_t on) { lsh_iid_sampling = on != 0; }
+
 static void lsh_rep_coordinates(uint64_t seed, int32_t rep, int32_t bits, int32_t d, int32_t *coord) {
     for (int32_t b = 0; b < bits; ++b) {
         for (uint64_t a = 0;; ++a) {
             int32_t c = (int32_t)(splitmix64_at(seed, (uint64_t)rep * 64u + (uint64_t)b + 4096u * a) % (uint64_t)d);
             int taken = 0;
-            for (int32_t e = 0; e < b && b < d; ++e) taken |= coord[e] == c;
+            for (int32_t e = 0; e < b && b < d && !lsh_iid_sampling; ++e) taken |= coord[e] == c;
             if (!taken) { coord[b] = c; break; }
         }
     }

@@ -82,6 +82,8 @@ def _load():
     lib.oracle_lsh_keys_hp_i8.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, vp]
     lib.oracle_lsh_keys_hp_bf16.restype = None
     lib.oracle_lsh_keys_hp_bf16.argtypes = [vp, i64, i32, i32, i32, i32, c.c_uint64, dbl, vp, vp]
+    lib.oracle_lsh_set_iid_sampling.restype = None
+    lib.oracle_lsh_set_iid_sampling.argtypes = [i32]
     lib.oracle_lsh_coordinate.restype = i32
     lib.oracle_lsh_coordinate.argtypes = [c.c_uint64, i32, i32, i32]
     lib.oracle_jl_levels.restype = i32
@@ -205,7 +207,7 @@ def lsh_join_hamming(Pbits: np.ndarray, Qbits: np.ndarray, d: int, r: float, L: 
     return lsh_join(widen(Pbits), widen(Qbits), float(d) - 2.0 * np.floor(r), L, k, seed, threads=threads, L_low=L_low)
 
 
-FAMILIES = ("bits", "hyperplanes")
+FAMILIES = ("bits", "hyperplanes", "bits_iid")
 
 
 def hp_tolerance(d: int) -> float:
@@ -216,13 +218,18 @@ def hp_tolerance(d: int) -> float:
 
 def lsh_keys(X: np.ndarray, L: int, k: int, seed: int, L_low: int = 0, dtype: str = "i8", family: str = "bits") -> np.ndarray:
     """(L + L_low, rows) uint32 hash keys.  family "bits": bit b = [x_c > 0] at the sampled coordinate (int8 rows or
-    bf16 bit patterns); family "hyperplanes": bit b = [<a, x> > 0] for a random-sign vector a."""
+    bf16 bit patterns), the k coordinates of a repetition distinct; "bits_iid": the same with k independent samples
+    (the paper's plain concatenation of base hashes); "hyperplanes": bit b = [<a, x> > 0] for a random-sign vector a."""
     lib = _load()
     X = _check(X, dtype)
     out = np.empty((L + L_low, X.shape[0]), dtype=np.uint32)
-    if family == "bits":
+    if family in ("bits", "bits_iid"):
         fn = lib.oracle_lsh_keys_i8 if dtype == "i8" else lib.oracle_lsh_keys_bf16
-        fn(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, out.ctypes.data)
+        lib.oracle_lsh_set_iid_sampling(1 if family == "bits_iid" else 0)       # k independent samples, or k distinct ones
+        try:
+            fn(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, out.ctypes.data)
+        finally:
+            lib.oracle_lsh_set_iid_sampling(0)
     elif family == "hyperplanes":
         if dtype == "i8":
             lib.oracle_lsh_keys_hp_i8(X.ctypes.data, X.shape[0], X.shape[1], L, L_low, k, seed, out.ctypes.data)

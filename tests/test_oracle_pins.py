@@ -733,3 +733,39 @@ def test_lsh_hyperplane_join_is_the_join_restricted_to_colliding_pairs():
     s, e, lo = O.lsh_band_sets(wb.P, wb.Q, "cos", wb.threshold, "bf16", 6, 4, 5, family="hyperplanes")
     ks, ke, kl = (O.pairs_to_set(z) for z in (s, e, lo))
     assert np.isin(ks, kl).all() and len(ke) > 0 and len(kl) >= len(ks)
+
+
+def test_lsh_iid_bit_sampling_is_the_plain_concatenation_of_independent_samples():
+    """family "bits_iid": bit b of repetition l reads coordinate splitmix64(seed, 64 l + b) mod d whether or not an earlier
+    bit took it -- the paper's concatenation of k independent base hashes, whose collision probability for a pair at
+    Hamming distance h is exactly (1 - h/d)^k."""
+    seed, L, k, d = 2006, 8, 7, 128
+    coords = np.array([[_splitmix64(seed, l * 64 + b) % d for b in range(k)] for l in range(L)])
+    assert [len(set(r)) for r in coords.tolist()] == [6, 7, 7, 7, 5, 7, 7, 7]       # repetitions 0 and 4 repeat a coordinate
+    X = W.random_points("i8", 500, d, 3, lo=-1, hi=1)
+    want = ((X[:, coords] > 0).astype(np.uint32) << np.arange(k, dtype=np.uint32)).sum(axis=2).T
+    got = O.lsh_keys(X, L, k, seed, family="bits_iid")
+    assert np.array_equal(want, got)
+    assert not np.array_equal(got, O.lsh_keys(X, L, k, seed))                        # the distinct-coordinate family differs there
+    assert np.array_equal(O.lsh_keys(X, L, k, seed), O.lsh_keys(X, L, k, seed, family="bits"))      # and the default is unchanged
+    # collision law on +-1 rows at Hamming distance h: 64 repetitions x 3000 pairs
+    rng = np.random.default_rng(4)
+    h, kk, reps = 16, 5, 64
+    A = (rng.integers(0, 2, size=(3000, d), dtype=np.int8) * 2 - 1).astype(np.int8)
+    Bm = A.copy()
+    flip = np.argsort(rng.random((3000, d)), axis=1)[:, :h]
+    Bm[np.repeat(np.arange(3000), h), flip.ravel()] *= -1
+    ka, kb = O.lsh_keys(A, reps, kk, 9, family="bits_iid"), O.lsh_keys(Bm, reps, kk, 9, family="bits_iid")
+    assert abs((ka == kb).mean() - (1 - h / d) ** kk) < 0.004                        # 0.5129; sigma = 0.0011
+    kd, ke = O.lsh_keys(A, reps, kk, 9), O.lsh_keys(Bm, reps, kk, 9)
+    hyper = math.comb(d - h, kk) / math.comb(d, kk)                                 # distinct coordinates: hypergeometric, 0.5090
+    assert abs((kd == ke).mean() - hyper) < 0.004
+    # the join of the family is the join restricted to its collisions
+    w = W.make_workload(4, n=600, m=500, planted=100)
+    pairs, cnt = O.lsh_join_kind(w.P, w.Q, "ip", 40.0, "i8", 3, 6, seed, family="bits_iid")
+    full, _c = O.join(w.P, w.Q, "ip", 40.0, "i8")
+    cp = np.array([[_splitmix64(seed, l * 64 + b) % w.d for b in range(6)] for l in range(3)])
+    kp = ((w.P[:, cp] > 0).astype(np.uint32) << np.arange(6, dtype=np.uint32)).sum(axis=2).T
+    kq = ((w.Q[:, cp] > 0).astype(np.uint32) << np.arange(6, dtype=np.uint32)).sum(axis=2).T
+    keep = (kp[:, full[:, 0]] == kq[:, full[:, 1]]).any(axis=0)
+    assert np.array_equal(pairs, full[keep]) and cnt == int(keep.sum()) > 0
