@@ -161,6 +161,10 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
  *                 that no earlier bit of the repetition took (from bit d on, a = 0 as it comes), where
  *                 splitmix64(seed, i): z = seed + (i+1)*0x9E3779B97F4A7C15; z = (z ^ z>>30)*0xBF58476D1CE4E5B9;
  *                 z = (z ^ z>>27)*0x94D049BB133111EB; z ^ z>>31  (all modulo 2^64).
+ *     SIMJOIN_LSH_BITS_IID     bit sampling as the paper states it, "a concatenation of k independent base hashes": bit b of
+ *                 repetition l samples splitmix64(seed, 64*l + b) mod d whether or not an earlier bit took that coordinate
+ *                 (a repetition with a repeated coordinate has fewer, larger buckets).  A pair at Hamming distance h then
+ *                 collides in a repetition with probability exactly (1 - h/d)^k, the p1^k of the paper's analysis.
  *     SIMJOIN_LSH_HYPERPLANES  random hyperplanes (sign random projections), the LSH of the angular distance for data of
  *                 any shape: h(x) = [<a, x> > 0], a projection of exactly zero giving 0; a is a vector of random signs,
  *                 coordinate c of the hyperplane of repetition l, bit b being +1 when bit 0 of
@@ -184,7 +188,7 @@ simjoin_status simjoin_run_host(simjoin_ctx *ctx, const void *P_host, int64_t n,
  * join all run on the device with no host round trip between repetitions.
  * simjoin_last_kernel_ms then reports (hashing, all repetitions).
  */
-typedef enum { SIMJOIN_LSH_BITS = 0, SIMJOIN_LSH_HYPERPLANES = 1 } simjoin_lsh_family;
+typedef enum { SIMJOIN_LSH_BITS = 0, SIMJOIN_LSH_HYPERPLANES = 1, SIMJOIN_LSH_BITS_IID = 2 } simjoin_lsh_family;
 simjoin_status simjoin_run_lsh(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
                                simjoin_kind kind, double threshold, simjoin_lsh_family family, int32_t L, int32_t L_low,
                                int32_t k, uint64_t seed, int32_t *out_pairs, uint64_t capacity, uint64_t *count);

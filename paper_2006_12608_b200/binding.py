@@ -20,8 +20,8 @@ SIMJOIN_IP, SIMJOIN_COS, SIMJOIN_L2 = 0, 1, 2
  SIMJOIN_ERR_TIMEOUT, SIMJOIN_ERR_ARCH) = range(7)
 DTYPE = {"i8": SIMJOIN_I8, "bf16": SIMJOIN_BF16}
 KIND = {"ip": SIMJOIN_IP, "cos": SIMJOIN_COS, "l2": SIMJOIN_L2}
-SIMJOIN_LSH_BITS, SIMJOIN_LSH_HYPERPLANES = 0, 1
-LSH_FAMILY = {"bits": SIMJOIN_LSH_BITS, "hyperplanes": SIMJOIN_LSH_HYPERPLANES}
+SIMJOIN_LSH_BITS, SIMJOIN_LSH_HYPERPLANES, SIMJOIN_LSH_BITS_IID = 0, 1, 2
+LSH_FAMILY = {"bits": SIMJOIN_LSH_BITS, "hyperplanes": SIMJOIN_LSH_HYPERPLANES, "bits_iid": SIMJOIN_LSH_BITS_IID}
 
 EXPORTS = ("simjoin_create", "simjoin_run", "simjoin_run_host", "simjoin_run_hamming", "simjoin_run_lsh", "simjoin_run_hamming_lsh", "simjoin_jl_transform", "simjoin_filter_pairs", "simjoin_run_jl_l2", "simjoin_row_norms", "simjoin_set_offsets", "simjoin_set_option",
            "simjoin_last_kernel_ms", "simjoin_run_noalloc", "simjoin_selftest_wait_timeout", "simjoin_destroy",

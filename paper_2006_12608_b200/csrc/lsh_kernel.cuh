@@ -33,14 +33,15 @@ __host__ __device__ inline uint64_t lsh_splitmix64(uint64_t seed, uint64_t idx) 
 // that no earlier bit of the repetition took (bit sampling without replacement: k bits give 2^k buckets; from bit d
 // on, when every coordinate is taken, a = 0 is used as it comes).  One thread per repetition, one block, once per
 // call: the key kernels read the table from global memory.
-__global__ void __launch_bounds__(64) lsh_coordinates_kernel(unsigned long long seed, int L, int k, int d, int *__restrict__ coords) {
+// `distinct` == 0: the k bits are k independent samples (a = 0 always; a coordinate may repeat within a repetition).
+__global__ void __launch_bounds__(64) lsh_coordinates_kernel(unsigned long long seed, int L, int k, int d, int distinct, int *__restrict__ coords) {
     for (int l = threadIdx.x; l < L; l += blockDim.x) {
         int *coord = coords + l * k;
         for (int b = 0; b < k; ++b) {
             for (uint64_t a = 0;; ++a) {
                 const int c = (int)(lsh_splitmix64(seed, (uint64_t)l * 64u + (uint64_t)b + 4096u * a) % (uint64_t)d);
                 bool taken = false;
-                for (int e = 0; e < b && b < d; ++e) taken = taken || coord[e] == c;
+                for (int e = 0; e < b && b < d && distinct; ++e) taken = taken || coord[e] == c;
                 if (!taken) { coord[b] = c; break; }
             }
         }

@@ -759,7 +759,7 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         const unsigned bn = (unsigned)((n + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS), bm = (unsigned)((m + LSH_KEYS_STAGED_ROWS - 1) / LSH_KEYS_STAGED_ROWS);
         const size_t sm = (size_t)LSH_KEYS_STAGED_ROWS * (row_bytes / 4 + 1) * 4;
         const bool staged = row_bytes <= LSH_KEYS_STAGED_MAX_D;
-        lsh_coordinates_kernel<<<1, 64, 0, s>>>(seed, L + L_low, k, d, coords);
+        lsh_coordinates_kernel<<<1, 64, 0, s>>>(seed, L + L_low, k, d, family == SIMJOIN_LSH_BITS ? 1 : 0, coords);
         if (i8) {
             const int8_t *p8 = reinterpret_cast<const int8_t *>(P), *q8 = reinterpret_cast<const int8_t *>(Q);
             if (staged) {
@@ -836,7 +836,7 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
 }
 
 simjoin_status check_lsh_args(int32_t L, int32_t L_low, int32_t k, simjoin_lsh_family family = SIMJOIN_LSH_BITS) {
-    if (family != SIMJOIN_LSH_BITS && family != SIMJOIN_LSH_HYPERPLANES) return SIMJOIN_ERR_ARG;
+    if (family != SIMJOIN_LSH_BITS && family != SIMJOIN_LSH_HYPERPLANES && family != SIMJOIN_LSH_BITS_IID) return SIMJOIN_ERR_ARG;
     if (L < 0 || L_low < 0 || L + L_low < 1 || L + L_low > LSH_MAX_REPS || k < 0 || (L_low > 0 && k < 1)) return SIMJOIN_ERR_ARG;
     if (k > LSH_MAX_BITS) return SIMJOIN_ERR_UNSUPPORTED;
     return SIMJOIN_OK;

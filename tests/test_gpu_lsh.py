@@ -317,3 +317,16 @@ def test_hyperplane_lsh_argument_checks(ctx):
     assert ctx.simjoin_run_lsh(X, 64, X, 64, 64, 10.0, 2, 3, 1, out, 8, family=7)[0] == B.SIMJOIN_ERR_ARG
     assert ctx.simjoin_run_lsh(X, 64, X, 64, 64, 10.0, 2, 13, 1, out, 8, family="hyperplanes")[0] == B.SIMJOIN_ERR_UNSUPPORTED
     assert ctx.simjoin_run_lsh(X, 0, X, 64, 64, 10.0, 2, 3, 1, out, 8, family="hyperplanes") == (B.SIMJOIN_OK, 0)
+
+
+@pytest.mark.parametrize("kind", ["ip", "l2"])
+def test_iid_bit_sampling_family_matches_the_oracle(ctx, kind):
+    """SIMJOIN_LSH_BITS_IID: the k bits of a repetition are independent samples.  With seed 2006 two of eight 7-bit repetitions
+    repeat a coordinate (half the buckets there), which the distinct-coordinate family avoids; both are exact on int8 rows."""
+    w = W.make_workload(4, n=5000, m=6000, planted=400)
+    t = {"ip": 40.0, "l2": 9.5}[kind]
+    got = run_family(ctx, w.P, w.Q, kind, t, 8, 7, 2006, L_low=1, family="bits_iid")
+    want, wcnt = O.lsh_join_kind(w.P, w.Q, kind, t, "i8", 8, 7, 2006, L_low=1, family="bits_iid")
+    assert len(got) == wcnt > 0 and np.array_equal(got, keys(want))
+    if kind == "ip":      # enough pairs of middling score that the two families' collisions differ
+        assert not np.array_equal(got, run_family(ctx, w.P, w.Q, kind, t, 8, 7, 2006, L_low=1, family="bits"))

@@ -68,7 +68,7 @@ def test_random_cases_match_the_oracle(seed):
             if lsh:
                 L, k = int(rng.integers(1, 5)), int(rng.integers(0, 6))
                 L_low = int(rng.integers(0, 2)) if k >= 1 else 0
-                family = "hyperplanes" if rng.random() < 0.4 else "bits"
+                family = str(rng.choice(["bits", "bits", "hyperplanes", "hyperplanes", "bits_iid"]))
                 st, cnt = ctx.simjoin_run_lsh(dP, n, dQ, m, d, t, L, k, s1, out, cap, L_low=L_low, kind=kind, family=family)
             else:
                 st, cnt = ctx.simjoin_run(dP, n, dQ, m, d, kind, t, out, cap)
