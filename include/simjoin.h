@@ -125,7 +125,7 @@ simjoin_status simjoin_run(simjoin_ctx *ctx, const void *P, int64_t n, const voi
  * copies P and Q to device staging owned by the context, runs the join, and
  * copies min(*count, capacity) pairs back; all on the context's stream,
  * synchronised before return.  Pinned host memory makes the copies faster but
- * is not required.  A Q above 64 MiB is uploaded in slices of about 32 MiB on a second stream and every
+ * is not required.  A Q above 64 MiB is uploaded in slices of about 32 MiB (one of 32 to 64 MiB in four slices) on a second stream and every
  * slice is joined as soon as it has landed, so that (with pinned memory) the copies of later slices hide
  * behind the joins of earlier ones; the result is the union of the slices' results.  With room for 64 MiB of
  * pairs or more (capacity >= 2^23) Q is cut into eight slices whatever its size, and the pairs of a slice are
