@@ -381,6 +381,19 @@ def test_run_host_uploads_a_large_q_in_slices(ctx_i8, ctx_bf16):
     assert_band(outb[:cnt], cnt, Pb, Qb, "cos", 0.03)
 
 
+def test_run_host_uploads_a_mid_size_q_in_four_slices(ctx_i8):
+    """A Q of 32 to 64 MiB (here 33 000 rows of 1 KiB) is joined in four slices of 8448 rows; hits in every slice, ragged last one."""
+    P, Q = W.random_points("i8", 150, 1024, 85), W.random_points("i8", 33000, 1024, 86)
+    Q[::1100] = P[:30]
+    t = 3.3 * (1024 * 16.0) ** 0.5
+    want, wcnt = O.join(P, Q, "ip", t, "i8")
+    assert wcnt >= 30 and len(np.unique(want[:, 1] // 8448)) == 4
+    out = np.full((wcnt + 10, 2), -7, dtype=np.int32)
+    st, cnt = ctx_i8.simjoin_run_host(P, 150, Q, 33000, 1024, "ip", t, out, wcnt + 10)
+    assert (st, cnt) == (B.SIMJOIN_OK, wcnt)
+    assert np.array_equal(np.sort(keys(out[:cnt])), keys(want)) and np.all(out[cnt:] == -7)
+
+
 def test_run_host_downloads_a_dense_result_slice_by_slice(ctx_i8):
     """Room for 2^23 pairs and more: Q is joined in eight slices and every slice's pairs travel to the host while the
     next slice is joined.  Result and overflow behaviour are those of the one-piece call."""
