@@ -68,9 +68,10 @@ typedef enum {
  * Create a context for joins over `dtype` points on CUDA device `device`,
  * enqueueing on `cuda_stream` (a cudaStream_t; NULL = the legacy default
  * stream).  The stream stays owned by the caller and must outlive the context.
- * The context owns its scratch (row norms, per-tile norm bounds, a 64-byte
- * counter/status block, staging buffers of simjoin_run_host), grown on demand
- * with cudaMalloc and released by simjoin_destroy.
+ * The context owns its scratch (row norms, per-tile norm bounds, two 64-byte
+ * control blocks and a pinned host mirror that the kernel writes its result to,
+ * staging buffers of simjoin_run_host, the buffers of the widened entry points),
+ * grown on demand with cudaMalloc and released by simjoin_destroy.
  * Errors: ERR_ARG (null ctx, unknown dtype, bad device), ERR_ARCH, ERR_CUDA.
  */
 simjoin_status simjoin_create(simjoin_ctx **ctx, simjoin_dtype dtype, int device, void *cuda_stream);
