@@ -397,12 +397,17 @@ void oracle_lsh_keys_hp_i8(const int8_t *X, int64_t rows, int32_t d, int32_t L_h
     for (int32_t l = 0; l < L_high + L_low; ++l) {
         const int32_t bits = l < L_high ? k : k - 1;
         for (int64_t i = 0; i < rows; ++i) keys[(size_t)l * rows + i] = 0;
-        for (int32_t b = 0; b < bits; ++b)
+        for (int32_t b = 0; b < bits; ++b) {
+            int32_t *a = (int32_t *)malloc(sizeof(int32_t) * (size_t)d);           /* the hyperplane, written out once */
+            if (!a) return;
+            for (int32_t c = 0; c < d; ++c) a[c] = oracle_lsh_hp_sign(seed, l, b, c);
             for (int64_t i = 0; i < rows; ++i) {
                 int64_t proj = 0;
-                for (int32_t c = 0; c < d; ++c) proj += (int64_t)oracle_lsh_hp_sign(seed, l, b, c) * (int64_t)X[(size_t)i * d + c];
+                for (int32_t c = 0; c < d; ++c) proj += (int64_t)a[c] * (int64_t)X[(size_t)i * d + c];
                 if (proj > 0) keys[(size_t)l * rows + i] |= 1u << b;
             }
+            free(a);
+        }
     }
 }
 
@@ -418,17 +423,22 @@ void oracle_lsh_keys_hp_bf16(const uint16_t *X, int64_t rows, int32_t d, int32_t
             keys[(size_t)l * rows + i] = 0;
             if (unsure) unsure[(size_t)l * rows + i] = 0;
         }
-        for (int32_t b = 0; b < bits; ++b)
+        for (int32_t b = 0; b < bits; ++b) {
+            double *a = (double *)malloc(sizeof(double) * (size_t)d);              /* the hyperplane, written out once */
+            if (!a) return;
+            for (int32_t c = 0; c < d; ++c) a[c] = (double)oracle_lsh_hp_sign(seed, l, b, c);
             for (int64_t i = 0; i < rows; ++i) {
                 double proj = 0.0, mass = 0.0;
                 for (int32_t c = 0; c < d; ++c) {
                     const double v = oracle_bf16_to_f64(X[(size_t)i * d + c]);
-                    proj += (double)oracle_lsh_hp_sign(seed, l, b, c) * v;
+                    proj += a[c] * v;
                     mass += fabs(v);
                 }
                 if (proj > 0.0) keys[(size_t)l * rows + i] |= 1u << b;
                 if (unsure && fabs(proj) <= tol * mass) unsure[(size_t)l * rows + i] |= 1u << b;
             }
+            free(a);
+        }
     }
 }
 

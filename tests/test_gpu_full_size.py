@@ -124,9 +124,10 @@ def test_full_size_cfg5_literal_sigma_is_empty():
     assert cnt == 0
 
 
-def test_full_size_lsh_join_cfg4():
+@pytest.mark.parametrize("family", ["bits", "hyperplanes"])
+def test_full_size_lsh_join_cfg4(family):
     """The LSH-bucketed join at the headline size (1 048 576 x 1 048 576, 8 tables of 7 bits), as `bench.py --lsh 8,7`
-    times it.  The result is the set {brute-force pairs whose keys agree in some table}: every emitted pair is scored
+    (`--lsh-family hyperplanes`) times it, for both hash families (int8: hyperplane keys are exact integers' signs).  The result is the set {brute-force pairs whose keys agree in some table}: every emitted pair is scored
     by the oracle and its keys (the oracle's) agree in a table; nothing is emitted twice; every planted pair whose
     oracle keys agree in a table is present, and only those; sampled rows are joined whole by the oracle."""
     L, k, seed = 8, 7, 2006
@@ -136,7 +137,7 @@ def test_full_size_lsh_join_cfg4():
     with B.Simjoin("i8", 0) as ctx:
         dP, dQ = B.to_device(w.P), B.to_device(w.Q)
         out = torch.empty((cap, 2), dtype=torch.int32, device="cuda:0")
-        st, cnt = ctx.simjoin_run_lsh(dP, w.n, dQ, w.m, w.d, w.threshold, L, k, seed, out, cap)
+        st, cnt = ctx.simjoin_run_lsh(dP, w.n, dQ, w.m, w.d, w.threshold, L, k, seed, out, cap, family=family)
         assert st == B.SIMJOIN_OK, B.strerror(st)
         pairs = out[:cnt].cpu().numpy().astype(np.int64)
     del dP, dQ, out
@@ -144,12 +145,13 @@ def test_full_size_lsh_join_cfg4():
     gk = keys(pairs)
     assert len(np.unique(gk)) == cnt
     assert np.all(O.scores(w.P, w.Q, "ip", "i8", pairs.astype(np.int32)) >= w.threshold)
-    kp, kq = O.lsh_keys(w.P, L, k, seed), O.lsh_keys(w.Q, L, k, seed)          # (L, rows)
+    kp, kq = O.lsh_keys(w.P, L, k, seed, family=family), O.lsh_keys(w.Q, L, k, seed, family=family)          # (L, rows)
     assert np.all((kp[:, pairs[:, 0]] == kq[:, pairs[:, 1]]).any(axis=0))      # every emitted pair collides in a table
     pl = w.planted
     collide = (kp[:, pl[:, 0]] == kq[:, pl[:, 1]]).any(axis=0)
     assert np.array_equal(np.isin(keys(pl), gk), collide)                      # planted pairs: present iff they collide
-    assert collide.mean() > 0.999                                              # closed form: 1 - (1 - (120/128)^7)^8 = 0.9997
+    # closed forms: bit sampling 1 - (1 - (120/128)^7)^8 = 0.9997; hyperplanes at angle acos(0.875): 1 - (1 - 0.839^7)^8 = 0.938
+    assert collide.mean() > (0.999 if family == "bits" else 0.92)
     rows = sample_rows(w, pairs, k=24)
     sub_keys = kp[:, rows]
     want, _c = O.join(w.P[rows], w.Q, "ip", w.threshold, "i8")                 # brute force on the sampled rows ...
