@@ -25,9 +25,13 @@ def keys(p):
     return (p[:, 0] << 32) | p[:, 1]
 
 
-def run_full(w, capacity):
+def run_full(w, capacity, dense_epilogue=None):
+    """One join at full size, in the launch configuration `bench.py` times.  dense_epilogue: SIMJOIN_OPT_DENSE_EPILOGUE
+    (None: the default, under which the first call of a context runs the 8-warp layout)."""
     build.build()
     with B.Simjoin(w.dtype, 0) as ctx:
+        if dense_epilogue is not None:
+            assert ctx.simjoin_set_option(B.SIMJOIN_OPT_DENSE_EPILOGUE, float(dense_epilogue)) == B.SIMJOIN_OK
         dP, dQ = B.to_device(w.P), B.to_device(w.Q)
         out = torch.empty((capacity, 2), dtype=torch.int32, device="cuda:0")
         st, cnt = ctx.simjoin_run(dP, w.n, dQ, w.m, w.d, w.kind, w.threshold, out, capacity)
@@ -101,12 +105,15 @@ def test_full_size_cfg2_cosine():
     check_sampled_rows(w, pairs, sample_rows(w, pairs), exact=False)
 
 
-def test_full_size_cfg5_mixture_dense():
+@pytest.mark.parametrize("dense_epilogue", [0, 1])
+def test_full_size_cfg5_mixture_dense(dense_epilogue):
+    """Both layouts the bench's calls go through: 8 epilogue warps on the points themselves (a context's first call), and 16
+    warps on the operands with the squared-L2 embedding appended (every later call of a dense join)."""
     w = W.make_workload(5)
     per_p = np.bincount(w.labels_p, minlength=1024).astype(np.int64)
     per_q = np.bincount(w.labels_q, minlength=1024).astype(np.int64)
     same_cluster = int(np.sum(per_p * per_q))
-    pairs, cnt = run_full(w, capacity=int(same_cluster * 1.02))
+    pairs, cnt = run_full(w, capacity=int(same_cluster * 1.02), dense_epilogue=dense_epilogue)
     assert cnt == same_cluster                         # independent pin: the join is the same-cluster relation
     assert np.all(w.labels_p[pairs[:, 0]] == w.labels_q[pairs[:, 1]])
     k = keys(pairs)
