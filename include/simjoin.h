@@ -324,7 +324,8 @@ simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64
  *                                524 288^2, +2 % on a join with 1000 pairs out of 65 536^2); 2 (default) = by the
  *                                previous simjoin_run of the context: 16 warps after a join with at least one pair per
  *                                two such blocks.  A Euclidean join in the 16-warp layout whose rows are at most 240 bytes
- *                                long runs as an inner-product join on transformed operands -- Section 4's squared-L2
+ *                                long (under 2: after a join with at least one pair per block) runs as an inner-product
+ *                                join on transformed operands -- Section 4's squared-L2
  *                                embedding: 8 coordinates carrying -|x|^2/2 and -|y|^2/2 in three bf16 pieces each, appended
  *                                to context-owned copies of both point sets ((n + m) x 128 or 256 bytes of scratch) -- with
  *                                the constant threshold -r^2/2 (70.8 -> 63.3 ms on the same join); radii too small for the

@@ -39,6 +39,10 @@ struct DevBuf {
 constexpr double DEFAULT_SELECT_MIN_OPS = 2.0e11;
 // Pairs per 32 x 128 block of scores from which a join counts as dense (its next run takes 16 epilogue warps).
 constexpr double DENSE_MIN_PAIRS_PER_BLOCK = 0.5;
+// ... and from which a Euclidean join in that layout also runs on transformed operands.  Measured on 262 144^2 mixtures, d = 64,
+// 16 against 8 warps: cosine 0.87 / 0.91 / 0.93 / 1.00 of the time at 8 / 2 / 0.5 / 0.125 pairs per block; Euclidean with the
+// transform 0.72 / 0.84 / 1.04 / 1.27.
+constexpr double EMBED_MIN_PAIRS_PER_BLOCK = 1.0;
 constexpr int MAX_HOST_SLICES = 66;     // simjoin_run_host: a Q of more slices than this goes up in one piece
 
 // Device-side working memory of one join call, and the host words its result lands in.  simjoin_run takes it from the
@@ -561,8 +565,8 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
             // The plain form of the dense Euclidean join runs as an inner-product join on transformed operands where the
             // transformed rows still fit two chunks (Section 4's squared-L2 embedding: l2_embed_rows_kernel); the
             // small-radius form stays on the points themselves.  Whichever the selection words call for does the work.
-            const simjoin_status es2 = fixed ? SIMJOIN_ERR_UNSUPPORTED
-                                             : launch_l2_embedded(ctx, P, n, Q, m, d, scr, jp, grid);
+            const bool embed = !fixed && (ctx->dense_mode == 1 || ctx->last_density >= EMBED_MIN_PAIRS_PER_BLOCK);
+            const simjoin_status es2 = embed ? launch_l2_embedded(ctx, P, n, Q, m, d, scr, jp, grid) : SIMJOIN_ERR_UNSUPPORTED;
             if (es2 == SIMJOIN_ERR_CUDA) return SIMJOIN_ERR_CUDA;
             e = es2 == SIMJOIN_OK ? cudaSuccess : launch_join_dense<KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
             if (e == cudaSuccess) e = launch_join_dense<KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
