@@ -68,3 +68,17 @@ def test_product_path_does_not_touch_the_oracle():
                 with open(os.path.join(dirpath, f)) as fh:
                     src = fh.read()
                 assert not re.search(r"^\s*(from|import)\s+oracle|simjoin_oracle|liboracle|oracle/", src, flags=re.M), f
+
+
+def test_argument_checks_that_need_no_gpu(lib):
+    """Null handles and unknown enumerators are rejected before any CUDA call is made."""
+    c = ctypes
+    assert lib.simjoin_create(None, 0, 0, None) == binding.SIMJOIN_ERR_ARG
+    assert lib.simjoin_set_option(None, binding.SIMJOIN_OPT_SELECT_MIN_OPS, 1.0) == binding.SIMJOIN_ERR_ARG
+    assert lib.simjoin_set_offsets(None, 0, 0) == binding.SIMJOIN_ERR_ARG
+    assert lib.simjoin_last_kernel_ms(None, None, None) == binding.SIMJOIN_ERR_ARG
+    assert lib.simjoin_destroy(None) == binding.SIMJOIN_OK
+    cnt = c.c_uint64(7)
+    assert lib.simjoin_run(None, None, 0, None, 0, 16, 0, 0.0, None, 0, c.byref(cnt)) == binding.SIMJOIN_ERR_ARG
+    assert lib.simjoin_run_noalloc(0, None, 5, None, 0, None, 0, 16, 0, 0.0, None, 0, c.byref(cnt)) == binding.SIMJOIN_ERR_ARG   # dtype
+    assert lib.simjoin_run_noalloc(-1, None, 0, None, 0, None, 0, 16, 0, 0.0, None, 0, c.byref(cnt)) == binding.SIMJOIN_ERR_ARG  # device
