@@ -33,3 +33,23 @@ def test_reference_arm_kind_override_and_silent_ranks():
     d = json.loads(run(["--kind", "cos", "--threshold", "0.6"])[0])
     assert d["config"]["kind"] == "cos" and d["config"]["threshold"] == 0.6
     assert run([], env={"RANK": "1", "WORLD_SIZE": "2", "LOCAL_RANK": "1"}) == []
+
+
+def test_roofline_arithmetic_of_the_bench_line():
+    """The fractions in the bench line are plain ratios of the kernel's rate: check them on made-up numbers."""
+    import bench
+    from paper_2006_12608_b200 import workloads as W
+    w = W.make_workload(4, n=1024, m=2048, planted=0)
+    peaks = {"hbm_gbs": 6000.0, "bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0, "source": "test"}
+    ops = 2 * 1024 * 2048 * 128
+    r = bench.roofline_of(w, kernel_ms=1.0, region_ms=1000.0, clocks={"sm_mhz": 1500.0}, peaks=peaks,
+                          int8_peak={"burst_tops": 3000.0, "sustained_tops": 2500.0})
+    achieved = ops / 1e-3 / 1e12
+    assert abs(r["achieved"] - achieved) < 1e-12 and r["peak"] == 2800.0 and abs(r["frac"] - achieved / 2800.0) < 1e-15
+    assert abs(r["frac_of_nominal"] - achieved / 4500.0) < 1e-15
+    assert abs(r["frac_of_clock_ceiling"] - achieved / (148 * 8192 * 2 * 1.5e9 / 1e12)) < 1e-15
+    assert abs(r["frac_of_int8_library_peak"] - achieved / 2500.0) < 1e-15
+    assert r["traffic"] is None and r["traffic_source"] is None            # not the captured size
+    burst = bench.roofline_of(w, 1.0, 100.0, {"sm_mhz": None}, peaks)
+    assert burst["peak"] == 3200.0 and "frac_of_clock_ceiling" not in burst and "frac_of_int8_library_peak" not in burst
+    assert bench.jl_level_dims(1024, 64) == [1024, 512, 512, 384, 64]
