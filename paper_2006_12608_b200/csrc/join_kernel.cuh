@@ -468,8 +468,8 @@ __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf
 
 // Compact the pairs (i, j0 + 32*q + c), c in mask[q], of the 32 rows this warp owns: popcount
 // prefix over the warp, then into the warp's shared-memory staging buffer, which is flushed with
-// one global atomic per ~STAGE_PAIRS pairs.  A block with more hits than the buffer holds goes
-// straight to global memory.  `fill` (warp-uniform) is the number of pairs staged so far.
+// one global atomic per ~STAGE_PAIRS pairs.  A block with more hits than the buffer holds leaves in
+// rounds through the same buffer.  `fill` (warp-uniform) is the number of pairs staged so far.
 template <int NQ, bool GROUPED, int VERIFY = VERIFY_NONE, int SP = STAGE_PAIRS>
 __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (&mask)[NQ], int lane, long long i, long long j0,
                                            int2 *buf, int &fill) {
@@ -505,9 +505,9 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
         // join on clustered data, where a quarter of all scores can pass).  The block leaves in rounds through the
         // (empty) staging buffer: every lane contributes up to SP / 32 of its remaining hits per round, and the round is
         // written out by all 32 lanes together -- coalesced stores, the position -> row lookups of bucketed mode 32 in
-        // flight -- instead of every lane walking its own hits with one dependent lookup and one 8-byte store each
-        // (measured on the bucketed dense join: 3.5 ms of a 3.8 ms call).  Where nothing can be dropped the whole
-        // block's slots are reserved with one atomic up front; otherwise every round goes through flush_pairs.
+        // flight -- instead of every lane walking its own hits with one dependent lookup and one 8-byte store each, and
+        // one atomic per pair where pairs can be dropped.  Where nothing can be dropped the whole block's slots are
+        // reserved with one atomic up front; otherwise every round goes through flush_pairs.
         constexpr int PER_LANE = SP / 32;
         bool plain = true;
         if constexpr (GROUPED || VERIFY != VERIFY_NONE) plain = !(VERIFY != VERIFY_NONE || p.rep > 0);
