@@ -311,6 +311,33 @@ def test_row_block_shards_on_the_gpu_union_to_the_whole_join(ctx_i8, ctx_bf16, w
         assert np.isin(keys(wl.planted), keys(allp)).all()
 
 
+def test_context_on_a_stream_of_its_own():
+    """A context bound to a non-default stream: every launch, the selection words, the control-block hand-over between
+    consecutive calls and the result the kernel stores to host memory follow that stream."""
+    w = W.make_workload(3, n=2500, m=1900, planted=150)
+    wb = W.make_workload(5, n=1200, m=1500, centers=15)
+    dP, dQ, bP, bQ = B.to_device(w.P), B.to_device(w.Q), B.to_device(wb.P), B.to_device(wb.Q)
+    out = torch.full((1 << 18, 2), -7, dtype=torch.int32, device="cuda:0")
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream(device=0)
+    ci, cb = B.Simjoin("i8", 0, stream=stream.cuda_stream), B.Simjoin("bf16", 0, stream=stream.cuda_stream)
+    try:
+        assert ci.simjoin_set_option(B.SIMJOIN_OPT_SELECT_MIN_OPS, 0.0) == B.SIMJOIN_OK
+        want, wcnt = O.join(w.P, w.Q, "ip", w.threshold, "i8")
+        for _ in range(3):
+            st, cnt = ci.simjoin_run(dP, w.n, dQ, w.m, w.d, "ip", w.threshold, out, 1 << 18)
+            assert (st, cnt) == (B.SIMJOIN_OK, wcnt)
+            stream.synchronize()
+            assert np.array_equal(np.sort(keys(out[:cnt].cpu().numpy())), keys(want))
+        for _ in range(3):                      # dense: the second and third call take the 16-warp layout
+            st, cnt = cb.simjoin_run(bP, wb.n, bQ, wb.m, wb.d, "l2", wb.threshold, out, 1 << 18)
+            assert st == B.SIMJOIN_OK
+            assert_band(out[:cnt].cpu().numpy(), cnt, wb.P, wb.Q, "l2", wb.threshold)
+    finally:
+        ci.close()
+        cb.close()
+
+
 def test_bad_arguments_are_rejected_before_launch(ctx_i8, ctx_bf16):
     P = B.to_device(W.random_points("i8", 64, 64, 17))
     out = torch.zeros((8, 2), dtype=torch.int32, device="cuda:0")
