@@ -619,7 +619,10 @@ __device__ __forceinline__ void store_tile_part(const JoinParams &p, uint32_t ta
 // ONE_BLOCK_OK: a tile whose second P block lies wholly past the end of P skips that block's MMAs (the store
 // kind, whose resident operand often has <= 128 rows; the join kinds keep the branch out of their issue loop).
 // WIDEQ: one resident block against 256 streamed rows (N = 256); the second block is never issued.
-template <int DT, int KC, bool GROUPED, bool ONE_BLOCK_OK, bool WIDEQ = false>
+// LASTK (fast path only): 32-byte K steps issued for a tile's last chunk -- 4 for rows of whole chunks; fewer where the
+// rest of the chunk is known to be zero (the transformed operands of dense Euclidean joins end 16 bytes into their
+// last chunk), which saves the tensor work and the energy of multiplying zeros.
+template <int DT, int KC, bool GROUPED, bool ONE_BLOCK_OK, bool WIDEQ = false, int LASTK = 4>
 __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl, uint8_t *smem_p, uint8_t *smem_ring,
                                                 const int stage_bytes_rt, const uint32_t tmem_base, const int warp, const int lane) {
     constexpr bool FAST = KC > 0;
@@ -666,7 +669,7 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
                 const uint64_t adesc1 = umma_desc_sw128_kmajor(a_addr + A_SUB_BYTES);        // P block 1
                 const uint64_t bdesc = umma_desc_sw128_kmajor(smem_u32(sb));
                 const bool last_chunk = c == kc - 1;
-                const int ksteps = FAST ? 4 : (last_chunk ? p.last_ksteps : 4);
+                const int ksteps = FAST ? ((KC > 0 && c == KC - 1) ? LASTK : 4) : (last_chunk ? p.last_ksteps : 4);
                 if (elect_one()) {
                     // the Q chunk against both resident P blocks: block s accumulates in columns s * TILE_N ..
                     umma_ss<DT == DT_I8>(d_tmem, adesc, bdesc, idesc, c != 0 ? 1u : 0u);
@@ -783,7 +786,7 @@ __host__ __device__ constexpr int fast_nstages(int kc, int pbufs) {
 // tile -- 4 MMAs of N = 256 per chunk into the 256 columns of an accumulator buffer, 32 KiB TMA transactions --
 // which this HBM-bound use prefers to two half-empty 128-column blocks.  In both, mapQ has 256-row boxes.
 constexpr int GEO_STD = 0, GEO_LONG = 1, GEO_WIDEQ = 2;
-template <int DT, int KIND, bool ALT = false, int KC = 0, bool GROUPED = false, int GEO = GEO_STD, int EW = NUM_EPI_WARPS>
+template <int DT, int KIND, bool ALT = false, int KC = 0, bool GROUPED = false, int GEO = GEO_STD, int EW = NUM_EPI_WARPS, int LASTK = 4>
 __global__ void __launch_bounds__(num_threads(EW), 1)
 join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ, const JoinParams p_in) {
     constexpr bool LONGK = GEO == GEO_LONG, WIDEQ = GEO == GEO_WIDEQ;
@@ -797,6 +800,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     static_assert(!LONGK || (KC == 0 && KIND != KIND_STORE && KIND != KIND_SIGN), "long-row mode: general join kinds only");
     static_assert(KIND != KIND_SIGN || (KC == 0 && !GROUPED && GEO == GEO_STD && !ALT), "hash keys: general path only");
     static_assert(!WIDEQ || (KC == 0 && !GROUPED && KIND == KIND_STORE), "wide-Q mode: store kind only");
+    static_assert(LASTK == 4 || (KC > 0 && LASTK >= 1 && LASTK < 4), "a short last chunk: compile-time chunk counts only");
     static_assert(EW == NUM_EPI_WARPS || (EW == 2 * NUM_EPI_WARPS && GEO == GEO_STD && KIND != KIND_STORE && KIND != KIND_SIGN), "16 epilogue warps: join kinds, standard geometry");
     constexpr int TN = (LONGK || WIDEQ) ? LONG_TN : TILE_N;   // rows of Q per tile
     constexpr int NPASS = TN / TILE_N;                     // 128-column passes of the epilogue over a P block's columns
@@ -813,7 +817,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         p.stationary = 1;
         p.epi_release = 1;
         p.nstages = fast_nstages(KC, p_bufs(GROUPED, KC));
-        p.last_ksteps = 4;
+        p.last_ksteps = 4;        // (the issuers of a LASTK < 4 instantiation stop short of the chunk's zero-filled rest)
     }
     // Aligned sweeps (no per-CTA rotation): bucketed units are short, and the store kind reads the streamed
     // operand once per 256-row tile of the resident one -- the CTAs that share a segment then walk it in
@@ -932,8 +936,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         constexpr bool OB = KIND == KIND_STORE || KIND == KIND_SIGN;
         if constexpr (LONGK) {
             if (warp == 1) mma_issuer_long<DT, GROUPED>(p, ctrl, smem_ring, tmem_base, lane);
-        } else if (fast && p.kc == 1 && !WIDEQ) mma_issuer_role<DT, 1, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
-        else if (fast && p.kc == 2 && !WIDEQ) mma_issuer_role<DT, 2, GROUPED, OB>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        } else if (fast && p.kc == 1 && !WIDEQ) mma_issuer_role<DT, 1, GROUPED, OB, false, KC == 1 ? LASTK : 4>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
+        else if (fast && p.kc == 2 && !WIDEQ) mma_issuer_role<DT, 2, GROUPED, OB, false, KC == 2 ? LASTK : 4>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
         else mma_issuer_role<DT, 0, GROUPED, OB, WIDEQ>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
     } else if (warp >= EPI_WARP0) {
         // ------------------------------------------------------------------ epilogue

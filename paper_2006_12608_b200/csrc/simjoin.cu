@@ -80,6 +80,7 @@ struct simjoin_ctx {
     bool attr_set_long[2][3][2][2];
     bool attr_set_wideq;
     bool attr_set_dense[3][2][3];
+    bool attr_set_embed[3][5];
     int dense_mode;                     // SIMJOIN_OPT_DENSE_EPILOGUE: 0 never, 1 always (where instantiated), 2 by the last join's density
     double last_density;                // pairs per 32 x 128 block of scores in the last successful simjoin_run (-1: none yet)
     cudaStream_t copy_stream;           // simjoin_run_host: uploads of Q slices overlap the joins of earlier slices
@@ -360,6 +361,20 @@ int norm_mode(bool /*i8*/, simjoin_kind kind, double threshold) {
     return (float)threshold > 0.f ? 2 : 1;        // decided on the fp32 threshold the epilogue uses
 }
 
+// The inner-product kernel of launch_l2_embedded: 16 epilogue warps, KC chunks per row, LASTK K steps in the last one.
+template <int KC, int LASTK>
+cudaError_t launch_embedded_kc(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid, size_t smem) {
+    constexpr int EW = 2 * NUM_EPI_WARPS;
+    auto kern = join_kernel<DT_BF16, KIND_IP, false, KC, false, GEO_STD, EW, LASTK>;
+    if (!ctx->attr_set_embed[KC][LASTK]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
+        if (e != cudaSuccess) return e;
+        ctx->attr_set_embed[KC][LASTK] = true;
+    }
+    kern<<<grid, num_threads(EW), smem, ctx->stream>>>(mp, mq, jp);
+    return cudaGetLastError();
+}
+
 // The plain form of a dense bf16 Euclidean join through the operand transform of l2_embed_rows_kernel: both point sets are
 // copied with 8 coordinates appended (context-owned buffers), and the 16-epilogue-warp inner-product kernel runs on the
 // copies with the constant threshold -r^2/2.  The copies' rows are padded with zeros to whole 128-byte chunks, so the
@@ -401,7 +416,14 @@ simjoin_status launch_l2_embedded(simjoin_ctx *ctx, const void *P, int64_t n, co
     CUtensorMap mapP, mapQ;
     if (!encode_rows_map(ctx, &mapP, ctx->emb_p.ptr, n, de, P_ROWS) || !encode_rows_map(ctx, &mapQ, ctx->emb_q.ptr, m, de, TILE_N))
         return SIMJOIN_ERR_CUDA;
-    return launch_join_dense<KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem) == cudaSuccess ? SIMJOIN_OK : SIMJOIN_ERR_CUDA;
+    // 32-byte K steps that the d + 8 coordinates reach into the last chunk: the issuers stop there
+    const int lastk = ((d + 8) * 2 - (jp.kc - 1) * CHUNK_BYTES + 31) / 32;
+    cudaError_t e = cudaErrorInvalidValue;
+#define SJ_EMBED(KC_, LK_) e = launch_embedded_kc<KC_, LK_>(ctx, mapP, mapQ, jp, grid, smem)
+    if (jp.kc == 1) { if (lastk == 1) SJ_EMBED(1, 1); else if (lastk == 2) SJ_EMBED(1, 2); else if (lastk == 3) SJ_EMBED(1, 3); else SJ_EMBED(1, 4); }
+    else { if (lastk == 1) SJ_EMBED(2, 1); else if (lastk == 2) SJ_EMBED(2, 2); else if (lastk == 3) SJ_EMBED(2, 3); else SJ_EMBED(2, 4); }
+#undef SJ_EMBED
+    return e == cudaSuccess ? SIMJOIN_OK : SIMJOIN_ERR_CUDA;
 }
 
 // One launch of the brute-force join kernel in the geometry the rows call for.
@@ -1061,6 +1083,7 @@ simjoin_status simjoin_create(simjoin_ctx **out, simjoin_dtype dtype, int device
     std::memset(ctx->attr_set_long, 0, sizeof ctx->attr_set_long);
     ctx->attr_set_wideq = false;
     std::memset(ctx->attr_set_dense, 0, sizeof ctx->attr_set_dense);
+    std::memset(ctx->attr_set_embed, 0, sizeof ctx->attr_set_embed);
     ctx->attr_set_sign[0] = ctx->attr_set_sign[1] = false;
     ctx->dense_mode = 2;
     ctx->last_density = -1.0;
