@@ -326,9 +326,9 @@ simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64
  *                                two such blocks.  A Euclidean join in the 16-warp layout whose rows are at most 240 bytes
  *                                long (under 2: after a join with at least one pair per block) runs as an inner-product
  *                                join on transformed operands -- Section 4's squared-L2
- *                                embedding: 8 coordinates carrying -|x|^2/2 and -|y|^2/2 in three bf16 pieces each, appended
+ *                                embedding: 8 coordinates carrying (r^2 - |x|^2)/2 and -|y|^2/2 in three bf16 pieces each, appended
  *                                to context-owned copies of both point sets ((n + m) x 128 or 256 bytes of scratch) -- with
- *                                the constant threshold -r^2/2 (70.8 -> 58.0 ms on the same join); radii too small for the
+ *                                the threshold folded into them as well, <x', y'> >= 0 (70.8 -> 56.8 ms on the same join); radii too small for the
  *                                fp32 norm expansion still take the row-deciding form on the points themselves.  Other
  *                                joins ignore the option.
  * Errors: ERR_ARG (null ctx, unknown option, NaN or out-of-range value).

@@ -792,11 +792,16 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     constexpr bool LONGK = GEO == GEO_LONG, WIDEQ = GEO == GEO_WIDEQ;
     constexpr bool NARROW = DT == DT_I8 && ALT;
     constexpr bool L2_FILTER = DT == DT_BF16 && KIND == KIND_L2 && ALT;
-    static_assert(DT == DT_I8 || !ALT || KIND == KIND_L2, "bf16: only the Euclidean kind has a second variant");
+    // bf16 inner product, ALT: the threshold is zero and folded into the operands (the transformed Euclidean join), so a
+    // score passes when its sign bit is clear -- the element test is one funnel shift, no add.  In the device-side choice
+    // between the two Euclidean forms this kernel stands for the plain one.
+    constexpr bool IP_SIGN = DT == DT_BF16 && KIND == KIND_IP && ALT;
+    constexpr bool SEL_ALT = ALT && !IP_SIGN;
+    static_assert(DT == DT_I8 || !ALT || KIND == KIND_L2 || KIND == KIND_IP, "bf16: the Euclidean and inner-product kinds have a second variant");
     // not the variant the data calls for: the other launch does the work (uniform over the grid, before any barrier
     // or tensor-memory allocation exists)
     if (p_in.zero_next != nullptr && blockIdx.x == 0 && threadIdx.x < 8) p_in.zero_next[threadIdx.x] = 0ull;
-    if (p_in.sel_mode != SEL_NONE && alt_selected(p_in) != ALT) return;
+    if (p_in.sel_mode != SEL_NONE && alt_selected(p_in) != SEL_ALT) return;
     static_assert(!LONGK || (KC == 0 && KIND != KIND_STORE && KIND != KIND_SIGN), "long-row mode: general join kinds only");
     static_assert(KIND != KIND_SIGN || (KC == 0 && !GROUPED && GEO == GEO_STD && !ALT), "hash keys: general path only");
     static_assert(!WIDEQ || (KC == 0 && !GROUPED && KIND == KIND_STORE), "wide-Q mode: store kind only");
@@ -1226,7 +1231,8 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                                                 : KIND == KIND_COS ? __fmul_rn(rf, __uint_as_float(yw[c]))   // as level 0 rounds it
                                                 : L2_FILTER        ? __fmaf_rn(p.l2_ycoef, __uint_as_float(yw[c]), rf)
                                                                    : rf + 0.5f * __uint_as_float(yw[c]);
-                                fail[c >> 2] = __funnelshift_l(__float_as_uint(__uint_as_float(v[k * GCOLS + c]) - b), fail[c >> 2], 1);
+                                if constexpr (IP_SIGN) fail[c >> 2] = __funnelshift_l(v[k * GCOLS + c], fail[c >> 2], 1);
+                                else fail[c >> 2] = __funnelshift_l(__float_as_uint(__uint_as_float(v[k * GCOLS + c]) - b), fail[c >> 2], 1);
                             }
                             // chain q holds columns 4q .. 4q+3 at bits 3 .. 0
                             uint32_t fall = 0;                                  // column c -> bit GCOLS - 1 - c

@@ -188,14 +188,16 @@ __global__ void __launch_bounds__(256) unpack_bits_pm1_kernel(const uint16_t *__
 // Operand transform for the squared Euclidean ip-distance (Section 4 lists f(x) = (x_k^2, 1, -2 x_k)_k, g(y) = (1, y_k^2, y_k)_k;
 // the same inner product with the squares summed up front): 8 coordinates appended to every bf16 row,
 //     P side:  (x, a1, a2, a3, 1, 1, 1, 0, 0)        Q side:  (y, 1, 1, 1, b1, b2, b3, 0, 0)
-// with a1 + a2 + a3 = -|x|^2 / 2 and b1 + b2 + b3 = -|y|^2 / 2 exactly (an fp32 value splits into three bf16 pieces of 8
-// significant bits each), so that <x', y'> = <x, y> - |x|^2/2 - |y|^2/2 = -|x - y|^2 / 2 and the Euclidean join becomes an
-// inner-product join with the constant threshold -r^2/2: no per-column term in the tile epilogue, an exact row-maximum
-// filter.  norms: |x|^2 per row in fp32, as the norm pre-pass left it.  Output rows are gout >= g + 1 16-byte words long
+// with a1 + a2 + a3 = (shift - |x|^2) / 2 and b1 + b2 + b3 = -|y|^2 / 2 exactly (an fp32 value splits into three bf16 pieces
+// of 8 significant bits each), so that <x', y'> = <x, y> + (shift - |x|^2 - |y|^2) / 2 = (shift - |x - y|^2) / 2.  With
+// shift = r^2 the Euclidean join becomes the inner-product join <x', y'> >= 0: no per-column term in the tile epilogue, an
+// exact row-maximum filter, the element test a sign bit.  norms: |x|^2 per row in fp32, as the norm pre-pass left it.  Output rows are gout >= g + 1 16-byte words long
 // (whole 128-byte chunks, so that every row of a TMA box is one aligned line; measured 65.1 -> 62 ms on the dense
 // 524 288^2 join against rows of exactly g + 1 words), zero past the appended coordinates.  One thread per output word.
+// shift (P side): added to -|x|^2/2 before the split -- r^2/2, which moves the threshold into the operands: the join is
+// then <x', y'> >= 0.
 __global__ void __launch_bounds__(256) l2_embed_rows_kernel(const uint4 *__restrict__ X, const float *__restrict__ norms, long long rows,
-                                                            int g, int gout, int q_side, uint4 *__restrict__ out) {
+                                                            int g, int gout, int q_side, float shift, uint4 *__restrict__ out) {
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= rows * gout) return;
     const long long r = t / gout;
@@ -204,7 +206,7 @@ __global__ void __launch_bounds__(256) l2_embed_rows_kernel(const uint4 *__restr
         out[t] = c < g ? __ldg(X + r * g + c) : make_uint4(0u, 0u, 0u, 0u);
         return;
     }
-    const float h = -0.5f * norms[r];
+    const float h = 0.5f * (shift - norms[r]);        // Q side: shift = 0
     const uint32_t hb = __float_as_uint(h);
     const float p1 = __uint_as_float(hb & 0xffff0000u);                  // truncation keeps the remainder exact
     const float r1 = h - p1;

@@ -365,7 +365,7 @@ int norm_mode(bool /*i8*/, simjoin_kind kind, double threshold) {
 template <int KC, int LASTK>
 cudaError_t launch_embedded_kc(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid, size_t smem) {
     constexpr int EW = 2 * NUM_EPI_WARPS;
-    auto kern = join_kernel<DT_BF16, KIND_IP, false, KC, false, GEO_STD, EW, LASTK>;
+    auto kern = join_kernel<DT_BF16, KIND_IP, true, KC, false, GEO_STD, EW, LASTK>;      // threshold 0: sign test
     if (!ctx->attr_set_embed[KC][LASTK]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin);
         if (e != cudaSuccess) return e;
@@ -391,9 +391,9 @@ simjoin_status launch_l2_embedded(simjoin_ctx *ctx, const void *P, int64_t n, co
     if (!grow(ctx->emb_p, (size_t)n * row_bytes) || !grow(ctx->emb_q, (size_t)m * row_bytes)) return SIMJOIN_ERR_CUDA;
     const int g = d * 2 / 16, gout = row_bytes / 16;
     l2_embed_rows_kernel<<<(unsigned)(((long long)n * gout + 255) / 256), 256, 0, ctx->stream>>>(
-        reinterpret_cast<const uint4 *>(P), reinterpret_cast<const float *>(scr.nx), n, g, gout, 0, reinterpret_cast<uint4 *>(ctx->emb_p.ptr));
+        reinterpret_cast<const uint4 *>(P), reinterpret_cast<const float *>(scr.nx), n, g, gout, 0, jp_l2.thr_f, reinterpret_cast<uint4 *>(ctx->emb_p.ptr));
     l2_embed_rows_kernel<<<(unsigned)(((long long)m * gout + 255) / 256), 256, 0, ctx->stream>>>(
-        reinterpret_cast<const uint4 *>(Q), reinterpret_cast<const float *>(scr.ny), m, g, gout, 1, reinterpret_cast<uint4 *>(ctx->emb_q.ptr));
+        reinterpret_cast<const uint4 *>(Q), reinterpret_cast<const float *>(scr.ny), m, g, gout, 1, 0.f, reinterpret_cast<uint4 *>(ctx->emb_q.ptr));
     if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
     jp.PB = jp_l2.PB;
     jp.QT = jp_l2.QT;
@@ -411,8 +411,8 @@ simjoin_status launch_l2_embedded(simjoin_ctx *ctx, const void *P, int64_t n, co
     jp.sel_words = jp_l2.sel_words;
     jp.sel_coef = jp_l2.sel_coef;
     jp.sel_r2 = jp_l2.sel_r2;
-    jp.thr_f = -0.5f * jp_l2.thr_f;             // <x', y'> = -|x - y|^2 / 2 >= -r^2 / 2
-    jp.thr_d = -0.5 * (double)jp_l2.thr_f;
+    jp.thr_f = -0.0f;                           // <x', y'> = (r^2 - |x - y|^2) / 2 >= 0: a score of either zero passes the bounds
+    jp.thr_d = 0.0;
     CUtensorMap mapP, mapQ;
     if (!encode_rows_map(ctx, &mapP, ctx->emb_p.ptr, n, de, P_ROWS) || !encode_rows_map(ctx, &mapQ, ctx->emb_q.ptr, m, de, TILE_N))
         return SIMJOIN_ERR_CUDA;
