@@ -194,8 +194,7 @@ __global__ void __launch_bounds__(256) unpack_bits_pm1_kernel(const uint16_t *__
 // exact row-maximum filter, the element test a sign bit.  norms: |x|^2 per row in fp32, as the norm pre-pass left it.  Output rows are gout >= g + 1 16-byte words long
 // (whole 128-byte chunks, so that every row of a TMA box is one aligned line; measured 65.1 -> 62 ms on the dense
 // 524 288^2 join against rows of exactly g + 1 words), zero past the appended coordinates.  One thread per output word.
-// shift (P side): added to -|x|^2/2 before the split -- r^2/2, which moves the threshold into the operands: the join is
-// then <x', y'> >= 0.
+// shift: r^2 on the P side (which moves the threshold into the operands), 0 on the Q side.
 __global__ void __launch_bounds__(256) l2_embed_rows_kernel(const uint4 *__restrict__ X, const float *__restrict__ norms, long long rows,
                                                             int g, int gout, int q_side, float shift, uint4 *__restrict__ out) {
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
