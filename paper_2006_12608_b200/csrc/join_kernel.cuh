@@ -1155,19 +1155,20 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     __syncwarp();
                     if (ps == NPASS - 1 && lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
                 }
-                if constexpr (IP_SIGN && EW == 2 * NUM_EPI_WARPS) {
+                if constexpr (IP_SIGN) {
                     // Dense output with the test "sign bit clear": no filter levels at all.  One funnel shift per column
-                    // collects the sign bits of the lane's 64 scores (8 independent chains of 8), which costs less than
+                    // collects the sign bits of the lane's scores (independent chains of 8), which costs less than
                     // the maxima, votes and branches of the hierarchy when most blocks hold hits anyway.
-                    static_assert(ECOLS == 64 && NPASS == 1, "the flat test is written for 64 columns per warp");
-                    uint32_t ch[8];
+                    static_assert(NPASS == 1 && !NARROW, "the flat test: standard geometry, 32-bit words");
+                    constexpr int NCHAIN = ECOLS / 8, NW = ECOLS / 32;
+                    uint32_t ch[NCHAIN];
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) ch[q] = 0;
+                    for (int q = 0; q < NCHAIN; ++q) ch[q] = 0;
 #pragma unroll
-                    for (int c = 0; c < 64; ++c) ch[c >> 3] = __funnelshift_l(v[c], ch[c >> 3], 1);     // column 8q + t -> bit 7 - t of chain q
-                    uint32_t mask[2];
+                    for (int c = 0; c < ECOLS; ++c) ch[c >> 3] = __funnelshift_l(v[c], ch[c >> 3], 1);     // column 8q + t -> bit 7 - t of chain q
+                    uint32_t mask[NW];
 #pragma unroll
-                    for (int w = 0; w < 2; ++w) {
+                    for (int w = 0; w < NW; ++w) {
                         const uint32_t neg = (ch[4 * w] << 24) | (ch[4 * w + 1] << 16) | (ch[4 * w + 2] << 8) | ch[4 * w + 3];   // column 32w + c -> bit 31 - c
                         mask[w] = row_ok ? __brev(~neg) : 0u;
                     }
@@ -1175,12 +1176,12 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     const long long left = q_end - j0;
                     if (left < ECOLS) {
 #pragma unroll
-                        for (int q = 0; q < 2; ++q) {
+                        for (int q = 0; q < NW; ++q) {
                             const long long lq = left - 32 * q;
                             mask[q] &= lq >= 32 ? 0xffffffffu : (lq <= 0 ? 0u : ((1u << (int)lq) - 1u));
                         }
                     }
-                    emit_pairs<2, GROUPED, VERIFY, SPAIRS>(p, mask, lane, i, j0, stage_buf, stage_fill);
+                    emit_pairs<NW, GROUPED, VERIFY, SPAIRS>(p, mask, lane, i, j0, stage_buf, stage_fill);
                     continue;
                 }
                 // level 0: the row maximum over this warp's 128 columns against the per-tile bound
