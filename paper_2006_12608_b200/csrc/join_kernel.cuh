@@ -797,6 +797,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     // between the two Euclidean forms this kernel stands for the plain one.
     constexpr bool IP_SIGN = DT == DT_BF16 && KIND == KIND_IP && ALT;
     constexpr bool SEL_ALT = ALT && !IP_SIGN;
+    // The sign test with 16 epilogue warps: the two groups of eight take alternate tiles (group g owns accumulator g), and
+    // every warp tests all 128 columns of its 32 rows in two loads of 64, so the per-tile work of a warp (barrier wait,
+    // hand-back, tail mask, compaction) is paid once per 128 columns instead of once per 64.
+    constexpr bool TWO_TILE = IP_SIGN && EW == 2 * NUM_EPI_WARPS;
     static_assert(DT == DT_I8 || !ALT || KIND == KIND_L2 || KIND == KIND_IP, "bf16: the Euclidean and inner-product kinds have a second variant");
     // not the variant the data calls for: the other launch does the work (uniform over the grid, before any barrier
     // or tensor-memory allocation exists)
@@ -846,7 +850,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             mbar_init(smem_u32(&ctrl->pfull[b]), 1);
             mbar_init(smem_u32(&ctrl->pempty[b]), p.epi_release ? 2 : 1);   // one commit per issuing warp
             mbar_init(smem_u32(&ctrl->tfull[b]), 1);
-            mbar_init(smem_u32(&ctrl->tempty[b]), EW);
+            mbar_init(smem_u32(&ctrl->tempty[b]), TWO_TILE ? EW / 2 : EW);
         }
         mbar_init(smem_u32(&ctrl->drain[0]), 1);
         mbar_init(smem_u32(&ctrl->drain[1]), 1);
@@ -948,9 +952,12 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
         const int half = ((warp - EPI_WARP0) >> 2) & 1;   // which of the tile's two P blocks (accumulator columns half * TILE_N ..)
-        const int coff = ((warp - EPI_WARP0) >> 3) * ECOLS;   // 16 warps: first column of this warp within a 128-column pass
+        const int group = (warp - EPI_WARP0) >> 3;        // 16 warps: which half of a 128-column pass, or (TWO_TILE) which tiles
+        const int coff = TWO_TILE ? 0 : group * ECOLS;    // first column of this warp within a 128-column pass
         const int row_in_tile = half * TILE_M + quarter * 32 + lane;
-        uint32_t acc = 0, accphase = 0, rstage = 0;   // rstage: next ring stage to hand back
+        uint32_t acc = TWO_TILE ? group : 0, accphase = 0;
+        uint32_t rstage = TWO_TILE ? group * p.kc : 0;    // next ring stage to hand back
+        uint32_t tile_parity = 0;                         // TWO_TILE: parity of the number of tiles before this unit
         // candidates of a filter are decided from their rows at flush time
         constexpr int VERIFY = (DT == DT_I8 && KIND == KIND_COS) ? VERIFY_COS_I8 : (L2_FILTER ? VERIFY_L2_BF16 : VERIFY_NONE);
         int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * (warp_stage_bytes(EW) / 8);
@@ -993,7 +1000,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     else rf = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] - p.thr_f);
                 }
             }
-            for (int k = 0; ok && k < un.q1 - un.q0; ++k) {
+            const int k_first = TWO_TILE ? (int)((group ^ tile_parity) & 1u) : 0;
+            tile_parity ^= (uint32_t)(un.q1 - un.q0) & 1u;
+            for (int k = k_first; ok && k < un.q1 - un.q0; k += TWO_TILE ? 2 : 1) {
                 const int qt = tile_at<ALIGNED>(un, k);
                 // per-tile filter bound: a necessary condition on max_j s_ij for row i to have any hit
                 int fi = p.thr_i;
@@ -1055,7 +1064,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 ok = wait_bar_warp(&ctrl->tfull[acc], accphase, ctrl, p.status, 6);
                 if (!ok) break;
                 tc_fence_after();
-                if (p.epi_release && warp == EPI_WARP0) {
+                if (p.epi_release && (TWO_TILE ? ((warp - EPI_WARP0) & 7) == 0 : warp == EPI_WARP0)) {
                     // the tile's MMAs have retired: its ring stages are free again
                     // (straight-line for one or two chunks: this sits on the accumulator hand-back path
                     // of the whole CTA, and a loop with a run-time trip count costs ~40 cycles per tile)
@@ -1075,7 +1084,51 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             if (++rstage == (uint32_t)p.nstages) rstage = 0;
                         }
                     }
+                    if constexpr (TWO_TILE) {       // the other group hands back the next tile's stages (nstages >= 2 kc here)
+                        rstage += (uint32_t)p.kc;
+                        if (rstage >= (uint32_t)p.nstages) rstage -= (uint32_t)p.nstages;
+                    }
                     __syncwarp();
+                }
+                if constexpr (TWO_TILE) {
+                    // Dense output with the test "sign bit clear": no filter levels at all.  One funnel shift per column
+                    // collects the sign bits of the lane's scores, 32 columns to a chain, which costs less than the
+                    // maxima, votes and branches of the hierarchy when most blocks hold hits anyway.
+                    static_assert(!LONGK && !NARROW && ECOLS == 64, "the flat test: standard geometry, 32-bit words");
+                    uint32_t mask[4];
+                    uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0;
+#pragma unroll 1
+                    for (int ps = 0; ps < 2; ++ps) {
+                        uint32_t v[ECOLS];
+                        tmem_ld_words(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS + half * TILE_N + ps * ECOLS, v, std::false_type{});
+                        if (ps == 1) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                        }
+                        uint32_t c0 = 0, c1 = 0;            // column 32w + c -> bit 31 - c of chain w
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            c0 = __funnelshift_l(v[c], c0, 1);
+                            c1 = __funnelshift_l(v[32 + c], c1, 1);
+                        }
+                        c0 = row_ok ? __brev(~c0) : 0u;
+                        c1 = row_ok ? __brev(~c1) : 0u;
+                        if (ps == 0) { m0 = c0; m1 = c1; } else { m2 = c0; m3 = c1; }
+                    }
+                    mask[0] = m0; mask[1] = m1; mask[2] = m2; mask[3] = m3;
+                    const long long j0 = q_base + (long long)qt * TN;
+                    const long long left = q_end - j0;
+                    if (left < TILE_N) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const long long lq = left - 32 * q;
+                            mask[q] &= lq >= 32 ? 0xffffffffu : (lq <= 0 ? 0u : ((1u << (int)lq) - 1u));
+                        }
+                    }
+                    emit_pairs<4, GROUPED, VERIFY, SPAIRS>(p, mask, lane, i, j0, stage_buf, stage_fill);
+                    accphase ^= 1;                      // this group's one accumulator
+                    continue;
                 }
                 if constexpr (KIND == KIND_SIGN) {
                     // lane <-> hyperplane (row of P), columns <-> points (rows of Q).  One vote per column collects the
@@ -1154,35 +1207,6 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     tc_fence_before();
                     __syncwarp();
                     if (ps == NPASS - 1 && lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
-                }
-                if constexpr (IP_SIGN) {
-                    // Dense output with the test "sign bit clear": no filter levels at all.  One funnel shift per column
-                    // collects the sign bits of the lane's scores (independent chains of 8), which costs less than
-                    // the maxima, votes and branches of the hierarchy when most blocks hold hits anyway.
-                    static_assert(NPASS == 1 && !NARROW, "the flat test: standard geometry, 32-bit words");
-                    constexpr int NCHAIN = ECOLS / 8, NW = ECOLS / 32;
-                    uint32_t ch[NCHAIN];
-#pragma unroll
-                    for (int q = 0; q < NCHAIN; ++q) ch[q] = 0;
-#pragma unroll
-                    for (int c = 0; c < ECOLS; ++c) ch[c >> 3] = __funnelshift_l(v[c], ch[c >> 3], 1);     // column 8q + t -> bit 7 - t of chain q
-                    uint32_t mask[NW];
-#pragma unroll
-                    for (int w = 0; w < NW; ++w) {
-                        const uint32_t neg = (ch[4 * w] << 24) | (ch[4 * w + 1] << 16) | (ch[4 * w + 2] << 8) | ch[4 * w + 3];   // column 32w + c -> bit 31 - c
-                        mask[w] = row_ok ? __brev(~neg) : 0u;
-                    }
-                    const long long j0 = q_base + (long long)qt * TN + coff;
-                    const long long left = q_end - j0;
-                    if (left < ECOLS) {
-#pragma unroll
-                        for (int q = 0; q < NW; ++q) {
-                            const long long lq = left - 32 * q;
-                            mask[q] &= lq >= 32 ? 0xffffffffu : (lq <= 0 ? 0u : ((1u << (int)lq) - 1u));
-                        }
-                    }
-                    emit_pairs<NW, GROUPED, VERIFY, SPAIRS>(p, mask, lane, i, j0, stage_buf, stage_fill);
-                    continue;
                 }
                 // level 0: the row maximum over this warp's 128 columns against the per-tile bound
                 // (a necessary condition of the exact test, in the same arithmetic)

@@ -5,8 +5,15 @@ The oracle cannot enumerate 10^12 pairs in a test, so at full size the checks ar
   - no pair is emitted twice,
   - for a sample of P rows the oracle's whole row join equals the emitted pairs of those rows
     (no false negative), within the band rule for bf16,
-  - every planted pair is found; the count matches what the generator's structure fixes.
+  - every planted pair is found; the count matches what the generator's structure fixes,
+  - the WHOLE sorted pair set equals the one the oracle's plain double loop produced over all n x m pairs, compared
+    through the digest tests/golden/make_full_size_digests.py stored (that oracle run takes up to an hour of host
+    time per configuration, so it is not repeated here).
 """
+import hashlib
+import json
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -123,6 +130,34 @@ def test_full_size_cfg5_mixture_dense(dense_epilogue):
     d = O.scores(w.P, w.Q, "l2", "bf16", sub)
     assert np.all(d <= w.threshold * (1 + BAND_REL))
     check_sampled_rows(w, pairs, sample_rows(w, pairs, k=24), exact=False)
+
+
+def stored_digests():
+    with open(os.path.join(os.path.dirname(__file__), "golden", "full_size_digests.json")) as f:
+        return json.load(f)
+
+
+@pytest.mark.parametrize("cfg", [2, 3, 4, 5])
+def test_full_size_whole_join_equals_the_oracles(cfg):
+    """The complete result at full size against the oracle's complete result (stored as a digest of the sorted pair
+    keys).  int8: the two sets are equal.  bf16: the result minus the oracle's 1 % band equals the oracle's strict set."""
+    g = stored_digests()[str(cfg)]
+    w = W.make_workload(cfg)
+    assert (w.n, w.m, w.d, w.kind, w.dtype, w.threshold) == (g["n"], g["m"], g["d"], g["kind"], g["dtype"], g["threshold"])
+    assert hashlib.sha256(w.P.tobytes()).hexdigest() == g["inputs_sha256"]["P"]
+    assert hashlib.sha256(w.Q.tobytes()).hexdigest() == g["inputs_sha256"]["Q"]
+    want = g["count"] if w.dtype == "i8" else g["loose_count"]
+    pairs, cnt = run_full(w, capacity=int(want * 1.02) + 1024)
+    k = np.sort(keys(pairs))
+    assert len(k) == cnt and np.all(k[1:] != k[:-1])
+    if w.dtype == "i8":
+        assert cnt == g["count"]
+        assert hashlib.sha256(k.astype("<i8").tobytes()).hexdigest() == g["sorted_keys_sha256"]
+    else:
+        band = keys(np.asarray(g["band_pairs"], dtype=np.int64).reshape(-1, 2))
+        k = k[~np.isin(k, band)]
+        assert len(k) == g["strict_count"]
+        assert hashlib.sha256(k.astype("<i8").tobytes()).hexdigest() == g["strict_sorted_keys_sha256"]
 
 
 def test_full_size_cfg5_literal_sigma_is_empty():

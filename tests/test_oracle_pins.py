@@ -31,7 +31,7 @@ def to_arr(rows, dtype):
 
 # ------------------------------------------------------------------ hand-worked
 GOLDEN = sorted(g for g in glob.glob(os.path.join(os.path.dirname(__file__), "golden", "*.json"))
-                if not os.path.basename(g).startswith(("hamming", "lsh_")))
+                if not os.path.basename(g).startswith(("hamming", "lsh_", "full_size_")))
 
 
 @pytest.mark.parametrize("path", GOLDEN, ids=[os.path.basename(p) for p in GOLDEN])
