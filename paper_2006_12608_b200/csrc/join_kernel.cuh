@@ -622,10 +622,15 @@ __device__ __forceinline__ void store_tile_part(const JoinParams &p, uint32_t ta
 // LASTK (fast path only): 32-byte K steps issued for a tile's last chunk -- 4 for rows of whole chunks; fewer where the
 // rest of the chunk is known to be zero (the transformed operands of dense Euclidean joins end 16 bytes into their
 // last chunk), which saves the tensor work and the energy of multiplying zeros.
-template <int DT, int KC, bool GROUPED, bool ONE_BLOCK_OK, bool WIDEQ = false, int LASTK = 4>
+// SPLIT (fast path only): both issuing warps work on every tile, warp 1 on P block 0 and warp 3 on P block 1, and wait
+// for the tile's operand chunks before they wait for the accumulator.  The time from an accumulator's hand-back to its
+// next commit then holds one barrier wait and half a tile's issues instead of three waits and a whole tile's -- for the
+// epilogue whose warp groups own one accumulator each, where that time is not hidden behind another tile's tests.
+template <int DT, int KC, bool GROUPED, bool ONE_BLOCK_OK, bool WIDEQ = false, int LASTK = 4, bool SPLIT = false>
 __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl, uint8_t *smem_p, uint8_t *smem_ring,
                                                 const int stage_bytes_rt, const uint32_t tmem_base, const int warp, const int lane) {
     constexpr bool FAST = KC > 0;
+    static_assert(!SPLIT || (FAST && !WIDEQ), "split issue: compile-time chunk count, standard geometry");
     constexpr uint32_t idesc = umma_idesc(DT == DT_I8 ? 2u : 1u, 1u, TILE_M, WIDEQ ? LONG_TN : TILE_N);
     const int kc = FAST ? KC : p.kc;
     const bool stationary = FAST ? true : p.stationary != 0;
@@ -645,7 +650,7 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
         }
         const bool two = !WIDEQ && (!ONE_BLOCK_OK || (GROUPED ? un.prows > TILE_M : (long long)un.pb * P_ROWS + TILE_M < p.n));
         for (int k = 0; ok && k < un.q1 - un.q0; ++k, tsel ^= 1) {
-            if (dual && tsel != mid) {
+            if (!SPLIT && dual && tsel != mid) {
                 // the other issuer's tile: step over its chunks in the ring
                 stage += (uint32_t)kc;
                 while (stage >= (uint32_t)p.nstages) { stage -= (uint32_t)p.nstages; phase ^= 1; }
@@ -653,12 +658,23 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
             }
             const uint32_t a = tsel;                       // accumulator of this tile
             const uint32_t d_tmem = tmem_base + a * ACC_COLS;
+            if constexpr (SPLIT) {
+                uint32_t st = stage, ph = phase;
+#pragma unroll
+                for (int c = 0; c < KC; ++c) {
+                    ok = ok && wait_bar_warp(&ctrl->full[st], ph, ctrl, p.status, 5);
+                    if (++st == (uint32_t)p.nstages) { st = 0; ph ^= 1; }
+                }
+                if (!ok) break;
+            }
             ok = wait_bar_warp(&ctrl->tempty[a], (a ? accph1 : accph0) ^ 1, ctrl, p.status, 4);
             if (!ok) break;
 #pragma unroll
             for (int c = 0; c < (FAST ? KC : kc); ++c) {
-                ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
-                if (!ok) break;
+                if constexpr (!SPLIT) {
+                    ok = wait_bar_warp(&ctrl->full[stage], phase, ctrl, p.status, 5);
+                    if (!ok) break;
+                }
                 tc_fence_after();
                 // operands are computed by the whole (converged) warp so that they stay warp-uniform;
                 // the four K steps are unrolled: a loop around single tcgen05.mma issues is slow
@@ -672,11 +688,13 @@ __device__ __forceinline__ void mma_issuer_role(const JoinParams &p, Ctrl *ctrl,
                 const int ksteps = FAST ? ((KC > 0 && c == KC - 1) ? LASTK : 4) : (last_chunk ? p.last_ksteps : 4);
                 if (elect_one()) {
                     // the Q chunk against both resident P blocks: block s accumulates in columns s * TILE_N ..
-                    umma_ss<DT == DT_I8>(d_tmem, adesc, bdesc, idesc, c != 0 ? 1u : 0u);
-                    if (ksteps > 1) umma_ss<DT == DT_I8>(d_tmem, adesc + 2, bdesc + 2, idesc, 1u);
-                    if (ksteps > 2) umma_ss<DT == DT_I8>(d_tmem, adesc + 4, bdesc + 4, idesc, 1u);
-                    if (ksteps > 3) umma_ss<DT == DT_I8>(d_tmem, adesc + 6, bdesc + 6, idesc, 1u);
-                    if (two) {
+                    if (!SPLIT || mid == 0) {
+                        umma_ss<DT == DT_I8>(d_tmem, adesc, bdesc, idesc, c != 0 ? 1u : 0u);
+                        if (ksteps > 1) umma_ss<DT == DT_I8>(d_tmem, adesc + 2, bdesc + 2, idesc, 1u);
+                        if (ksteps > 2) umma_ss<DT == DT_I8>(d_tmem, adesc + 4, bdesc + 4, idesc, 1u);
+                        if (ksteps > 3) umma_ss<DT == DT_I8>(d_tmem, adesc + 6, bdesc + 6, idesc, 1u);
+                    }
+                    if (two && (!SPLIT || mid == 1)) {
                         umma_ss<DT == DT_I8>(d_tmem + TILE_N, adesc1, bdesc, idesc, c != 0 ? 1u : 0u);
                         if (ksteps > 1) umma_ss<DT == DT_I8>(d_tmem + TILE_N, adesc1 + 2, bdesc + 2, idesc, 1u);
                         if (ksteps > 2) umma_ss<DT == DT_I8>(d_tmem + TILE_N, adesc1 + 4, bdesc + 4, idesc, 1u);
@@ -849,7 +867,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctrl->pfull[b]), 1);
             mbar_init(smem_u32(&ctrl->pempty[b]), p.epi_release ? 2 : 1);   // one commit per issuing warp
-            mbar_init(smem_u32(&ctrl->tfull[b]), 1);
+            mbar_init(smem_u32(&ctrl->tfull[b]), TWO_TILE ? 2 : 1);      // split issue: one commit per issuing warp
             mbar_init(smem_u32(&ctrl->tempty[b]), TWO_TILE ? EW / 2 : EW);
         }
         mbar_init(smem_u32(&ctrl->drain[0]), 1);
@@ -945,6 +963,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         constexpr bool OB = KIND == KIND_STORE || KIND == KIND_SIGN;
         if constexpr (LONGK) {
             if (warp == 1) mma_issuer_long<DT, GROUPED>(p, ctrl, smem_ring, tmem_base, lane);
+        } else if constexpr (TWO_TILE) {
+            // (the host launches these instantiations only where the fast path's conditions hold)
+            static_assert(KC == 1 || KC == 2, "alternate-tile epilogue: rows of one or two chunks");
+            mma_issuer_role<DT, KC, GROUPED, OB, false, LASTK, true>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
         } else if (fast && p.kc == 1 && !WIDEQ) mma_issuer_role<DT, 1, GROUPED, OB, false, KC == 1 ? LASTK : 4>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
         else if (fast && p.kc == 2 && !WIDEQ) mma_issuer_role<DT, 2, GROUPED, OB, false, KC == 2 ? LASTK : 4>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
         else mma_issuer_role<DT, 0, GROUPED, OB, WIDEQ>(p, ctrl, smem_p, smem_ring, stage_bytes, tmem_base, warp, lane);
