@@ -323,14 +323,17 @@ simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64
  *                                latency, which twice the warps hide; measured 77.5 -> 70.8 ms on 2.7e8 pairs out of
  *                                524 288^2, +2 % on a join with 1000 pairs out of 65 536^2); 2 (default) = by the
  *                                previous simjoin_run of the context: 16 warps after a join with at least one pair per
- *                                two such blocks.  A Euclidean join in the 16-warp layout whose rows are at most 240 bytes
- *                                long (under 2: after a join with at least one pair per block) runs as an inner-product
- *                                join on transformed operands -- Section 4's squared-L2
- *                                embedding: 8 coordinates carrying (r^2 - |x|^2)/2 and -|y|^2/2 in three bf16 pieces each, appended
- *                                to context-owned copies of both point sets ((n + m) x 128 or 256 bytes of scratch) -- with
- *                                the threshold folded into them as well, <x', y'> >= 0, tested flat on every score's sign bit (70.8 -> 48.4 ms on the same join); radii too small for the
- *                                fp32 norm expansion still take the row-deciding form on the points themselves.  Other
- *                                joins ignore the option.
+ *                                two such blocks.  A join in the 16-warp layout whose rows are at most 240 bytes long
+ *                                (under 2: after a join with at least one pair per block) runs as the sign test of one
+ *                                inner product on transformed operands -- Section 4's ip-distance embeddings with the
+ *                                threshold folded in: 8 coordinates appended to context-owned copies of both point sets
+ *                                ((n + m) x 128 or 256 bytes of scratch) so that <x', y'> >= 0 exactly when the pair
+ *                                passes.  Euclidean: (r^2 - |x|^2)/2 and -|y|^2/2 in three bf16 pieces each against ones
+ *                                (70.8 -> 42.3 ms on the same join); inner product: -t in three pieces against ones;
+ *                                cosine: the six largest piece products of (-t |x|) |y| and two flags for zero vectors
+ *                                (18.3 -> 10.4 ms on 6.7e7 pairs out of 262 144^2, d = 64).  Euclidean radii too small for
+ *                                the fp32 norm expansion still take the row-deciding form on the points themselves.
+ *                                Other joins ignore the option.
  * Errors: ERR_ARG (null ctx, unknown option, NaN or out-of-range value).
  */
 typedef enum { SIMJOIN_OPT_SELECT_MIN_OPS = 0, SIMJOIN_OPT_KERNEL_TIMING = 1, SIMJOIN_OPT_DENSE_EPILOGUE = 2 } simjoin_option;

@@ -15,6 +15,8 @@
 //   warps 4-11  epilogue: warp w reads TMEM lanes 32*(w%4).. of P block (w-4)/4; row max vs a
 //               per-tile bound, then 16-column group maxima, then the exact test; passing pairs go
 //               through a per-warp shared-memory staging buffer to the output list
+// Dense outputs (bf16, rows of one or two chunks) run with 16 epilogue warps (EW = 16, 640 threads): two warps share a
+// block of rows and split its 128 columns -- or, for the sign test on transformed operands, take alternate tiles.
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word and drains.
 #pragma once
 #include <cuda_bf16.h>

@@ -185,18 +185,38 @@ __global__ void __launch_bounds__(256) unpack_bits_pm1_kernel(const uint16_t *__
     out[t] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// Operand transform for the squared Euclidean ip-distance (Section 4 lists f(x) = (x_k^2, 1, -2 x_k)_k, g(y) = (1, y_k^2, y_k)_k;
-// the same inner product with the squares summed up front): 8 coordinates appended to every bf16 row,
-//     P side:  (x, a1, a2, a3, 1, 1, 1, 0, 0)        Q side:  (y, 1, 1, 1, b1, b2, b3, 0, 0)
-// with a1 + a2 + a3 = (shift - |x|^2) / 2 and b1 + b2 + b3 = -|y|^2 / 2 exactly (an fp32 value splits into three bf16 pieces
-// of 8 significant bits each), so that <x', y'> = <x, y> + (shift - |x|^2 - |y|^2) / 2 = (shift - |x - y|^2) / 2.  With
-// shift = r^2 the Euclidean join becomes the inner-product join <x', y'> >= 0: no per-column term in the tile epilogue, an
-// exact row-maximum filter, the element test a sign bit.  norms: |x|^2 per row in fp32, as the norm pre-pass left it.  Output rows are gout >= g + 1 16-byte words long
-// (whole 128-byte chunks, so that every row of a TMA box is one aligned line; measured 65.1 -> 62 ms on the dense
-// 524 288^2 join against rows of exactly g + 1 words), zero past the appended coordinates.  One thread per output word.
-// shift: r^2 on the P side (which moves the threshold into the operands), 0 on the Q side.
-__global__ void __launch_bounds__(256) l2_embed_rows_kernel(const uint4 *__restrict__ X, const float *__restrict__ norms, long long rows,
-                                                            int g, int gout, int q_side, float shift, uint4 *__restrict__ out) {
+// An fp32 value as three bf16 pieces of 8 significant bits each (truncation keeps every remainder exact): h = p1 + p2 + p3.
+__device__ __forceinline__ void split3_bf16(float h, uint32_t &b1, uint32_t &b2, uint32_t &b3) {
+    const float p1 = __uint_as_float(__float_as_uint(h) & 0xffff0000u);
+    const float r1 = h - p1;
+    const float p2 = __uint_as_float(__float_as_uint(r1) & 0xffff0000u);
+    const float p3 = r1 - p2;                                            // at most 8 significant bits are left
+    b1 = __float_as_uint(p1) >> 16;
+    b2 = __float_as_uint(p2) >> 16;
+    b3 = __float_as_uint(p3) >> 16;
+}
+
+// Operand transforms that turn a thresholded ip-distance of Section 4 into the sign of one inner product: 8 coordinates are
+// appended to every bf16 row so that <x', y'> >= 0 exactly when the pair passes.  The tile epilogue then needs no per-row or
+// per-column term and its element test is the score's sign bit.
+//   EMBED_L2  (Section 4 lists f(x) = (x_k^2, 1, -2 x_k)_k, g(y) = (1, y_k^2, y_k)_k; the same inner product with the
+//             squares summed up front):
+//                 P side (x, a1, a2, a3, 1, 1, 1, 0, 0)      Q side (y, 1, 1, 1, b1, b2, b3, 0, 0)
+//             a1 + a2 + a3 = (r^2 - |x|^2) / 2 and b1 + b2 + b3 = -|y|^2 / 2 exactly, so <x', y'> = (r^2 - |x - y|^2) / 2.
+//             norms: |x|^2 in fp32 as the norm pre-pass left it; shift: r^2 on the P side, 0 on the Q side.
+//   EMBED_IP  <x, y> >= t:   P side (x, c1, c2, c3, 0, ...) with c1 + c2 + c3 = -t (shift = t), Q side (y, 1, 1, 1, 0, ...).
+//   EMBED_COS <x, y> >= t |x| |y| (f = g = x / |x| of Section 4, cleared of the division): with u = -t |x| and v = |y| split
+//             into pieces, the product u v is the sum of the nine piece products, of which the six largest are kept (the
+//             rest is below 2^-23 of it):
+//                 P side (x, u1, u1, u1, u2, u2, u3, zx, 1)    Q side (y, v1, v2, v3, v1, v2, v1, 1, zy)
+//             norms: |x| in fp32; a zero vector is stored as +inf when t > 0 (it passes nothing): its pieces are zero and its
+//             flag zx (zy) is -1, which makes every score it takes part in negative.  shift = t on the P side.
+// Output rows are gout >= g + 1 16-byte words long (whole 128-byte chunks, so that every row of a TMA box is one aligned
+// line; measured 65.1 -> 62 ms on the dense 524 288^2 Euclidean join against rows of exactly g + 1 words), zero past the
+// appended coordinates.  One thread per output word.
+constexpr int EMBED_L2 = 0, EMBED_IP = 1, EMBED_COS = 2;
+__global__ void __launch_bounds__(256) embed_rows_kernel(const uint4 *__restrict__ X, const float *__restrict__ norms, long long rows,
+                                                         int g, int gout, int mode, int q_side, float shift, uint4 *__restrict__ out) {
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= rows * gout) return;
     const long long r = t / gout;
@@ -205,17 +225,27 @@ __global__ void __launch_bounds__(256) l2_embed_rows_kernel(const uint4 *__restr
         out[t] = c < g ? __ldg(X + r * g + c) : make_uint4(0u, 0u, 0u, 0u);
         return;
     }
-    const float h = 0.5f * (shift - norms[r]);        // Q side: shift = 0
-    const uint32_t hb = __float_as_uint(h);
-    const float p1 = __uint_as_float(hb & 0xffff0000u);                  // truncation keeps the remainder exact
-    const float r1 = h - p1;
-    const float p2 = __uint_as_float(__float_as_uint(r1) & 0xffff0000u);
-    const float p3 = (r1 - p2);                                          // at most 8 significant bits are left
-    const uint32_t b1 = __float_as_uint(p1) >> 16, b2 = __float_as_uint(p2) >> 16, b3 = __float_as_uint(p3) >> 16;
-    const uint32_t one = 0x3F80u;
+    const uint32_t one = 0x3F80u, minus_one = 0xBF80u;
+    uint32_t b1, b2, b3;
     // eight bf16 values, low half of a word first
-    if (q_side) out[t] = make_uint4(one | (one << 16), one | (b1 << 16), b2 | (b3 << 16), 0u);
-    else out[t] = make_uint4(b1 | (b2 << 16), b3 | (one << 16), one | (one << 16), 0u);
+    if (mode == EMBED_L2) {
+        split3_bf16(0.5f * (shift - norms[r]), b1, b2, b3);
+        if (q_side) out[t] = make_uint4(one | (one << 16), one | (b1 << 16), b2 | (b3 << 16), 0u);
+        else out[t] = make_uint4(b1 | (b2 << 16), b3 | (one << 16), one | (one << 16), 0u);
+    } else if (mode == EMBED_IP) {
+        if (q_side) out[t] = make_uint4(one | (one << 16), one, 0u, 0u);
+        else {
+            split3_bf16(-shift, b1, b2, b3);
+            out[t] = make_uint4(b1 | (b2 << 16), b3, 0u, 0u);
+        }
+    } else {
+        const float nr = norms[r];
+        const bool none = nr == __int_as_float(0x7f800000);        // a zero vector under t > 0
+        split3_bf16(none ? 0.f : (q_side ? nr : -shift * nr), b1, b2, b3);
+        const uint32_t z = none ? minus_one : 0u;
+        if (q_side) out[t] = make_uint4(b1 | (b2 << 16), b3 | (b1 << 16), b2 | (b1 << 16), one | (z << 16));
+        else out[t] = make_uint4(b1 | (b1 << 16), b1 | (b2 << 16), b2 | (b3 << 16), z | (one << 16));
+    }
 }
 
 }  // namespace sj

@@ -333,6 +333,9 @@ void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold
         }
     } else {
         jp.thr_f = kind == SIMJOIN_L2 ? (float)(threshold * threshold) : (float)threshold;
+        // a cosine lies in [-1, 1]: thresholds beyond +-2 decide like +-2, and the products t |x| |y| stay finite
+        // (t = -inf times the norm 0 of a zero vector would be NaN, and its pairs would be lost)
+        if (kind == SIMJOIN_COS) jp.thr_f = fminf(fmaxf(jp.thr_f, -2.f), 2.f);
         // the inner-product and cosine tests read the sign of s - b: with t = -0 a score of either zero gives +0 and passes
         if (kind != SIMJOIN_L2 && jp.thr_f == 0.f) jp.thr_f = -0.0f;
         if (kind == SIMJOIN_L2 && d > 0) {
@@ -361,7 +364,7 @@ int norm_mode(bool /*i8*/, simjoin_kind kind, double threshold) {
     return (float)threshold > 0.f ? 2 : 1;        // decided on the fp32 threshold the epilogue uses
 }
 
-// The inner-product kernel of launch_l2_embedded: 16 epilogue warps, KC chunks per row, LASTK K steps in the last one.
+// The inner-product kernel of launch_embedded: 16 epilogue warps, KC chunks per row, LASTK K steps in the last one.
 template <int KC, int LASTK>
 cudaError_t launch_embedded_kc(simjoin_ctx *ctx, const CUtensorMap &mp, const CUtensorMap &mq, const JoinParams &jp, int grid, size_t smem) {
     constexpr int EW = 2 * NUM_EPI_WARPS;
@@ -375,14 +378,15 @@ cudaError_t launch_embedded_kc(simjoin_ctx *ctx, const CUtensorMap &mp, const CU
     return cudaGetLastError();
 }
 
-// The plain form of a dense bf16 Euclidean join through the operand transform of l2_embed_rows_kernel: both point sets are
-// copied with 8 coordinates appended (context-owned buffers), and the 16-epilogue-warp inner-product kernel runs on the
-// copies with the constant threshold -r^2/2.  The copies' rows are padded with zeros to whole 128-byte chunks, so the
-// whole-chunk instantiations apply and every box row is an aligned line.  Returns ERR_UNSUPPORTED (nothing launched)
-// when the transformed rows do not fit two chunks.  `jp_l2`: the Euclidean join's parameters (norms already computed).
-simjoin_status launch_l2_embedded(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
-                                  const JoinScratch &scr, const JoinParams &jp_l2, int grid) {
-    if ((d + 8) * 2 > 2 * CHUNK_BYTES) return SIMJOIN_ERR_UNSUPPORTED;
+// A dense bf16 join through the operand transforms of embed_rows_kernel: both point sets are copied with 8 coordinates
+// appended (context-owned buffers), and the 16-epilogue-warp sign-test kernel runs on the copies: <x', y'> >= 0.  For the
+// Euclidean kind this is the plain form (the small-radius form stays on the points themselves; the selection words
+// decide).  The copies' rows are padded with zeros to whole 128-byte chunks, so the whole-chunk instantiations apply and
+// every box row is an aligned line.  Returns ERR_UNSUPPORTED (nothing launched) when the transformed rows do not fit
+// two chunks or the threshold is not finite.  `jp_l2`: the join's own parameters (norms already computed).
+simjoin_status launch_embedded(simjoin_ctx *ctx, simjoin_kind kind, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,
+                               const JoinScratch &scr, const JoinParams &jp_l2, int grid) {
+    if ((d + 8) * 2 > 2 * CHUNK_BYTES || !std::isfinite(jp_l2.thr_f)) return SIMJOIN_ERR_UNSUPPORTED;
     const int row_bytes = ((d + 8) * 2 + CHUNK_BYTES - 1) / CHUNK_BYTES * CHUNK_BYTES, de = row_bytes / 2;      // whole chunks
     JoinParams jp;
     size_t smem = 0;
@@ -390,10 +394,11 @@ simjoin_status launch_l2_embedded(simjoin_ctx *ctx, const void *P, int64_t n, co
     if (!dense_available(false, jp)) return SIMJOIN_ERR_UNSUPPORTED;
     if (!grow(ctx->emb_p, (size_t)n * row_bytes) || !grow(ctx->emb_q, (size_t)m * row_bytes)) return SIMJOIN_ERR_CUDA;
     const int g = d * 2 / 16, gout = row_bytes / 16;
-    l2_embed_rows_kernel<<<(unsigned)(((long long)n * gout + 255) / 256), 256, 0, ctx->stream>>>(
-        reinterpret_cast<const uint4 *>(P), reinterpret_cast<const float *>(scr.nx), n, g, gout, 0, jp_l2.thr_f, reinterpret_cast<uint4 *>(ctx->emb_p.ptr));
-    l2_embed_rows_kernel<<<(unsigned)(((long long)m * gout + 255) / 256), 256, 0, ctx->stream>>>(
-        reinterpret_cast<const uint4 *>(Q), reinterpret_cast<const float *>(scr.ny), m, g, gout, 1, 0.f, reinterpret_cast<uint4 *>(ctx->emb_q.ptr));
+    const int mode = kind == SIMJOIN_L2 ? EMBED_L2 : (kind == SIMJOIN_IP ? EMBED_IP : EMBED_COS);
+    embed_rows_kernel<<<(unsigned)(((long long)n * gout + 255) / 256), 256, 0, ctx->stream>>>(
+        reinterpret_cast<const uint4 *>(P), reinterpret_cast<const float *>(scr.nx), n, g, gout, mode, 0, jp_l2.thr_f, reinterpret_cast<uint4 *>(ctx->emb_p.ptr));
+    embed_rows_kernel<<<(unsigned)(((long long)m * gout + 255) / 256), 256, 0, ctx->stream>>>(
+        reinterpret_cast<const uint4 *>(Q), reinterpret_cast<const float *>(scr.ny), m, g, gout, mode, 1, 0.f, reinterpret_cast<uint4 *>(ctx->emb_q.ptr));
     if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
     jp.PB = jp_l2.PB;
     jp.QT = jp_l2.QT;
@@ -411,7 +416,7 @@ simjoin_status launch_l2_embedded(simjoin_ctx *ctx, const void *P, int64_t n, co
     jp.sel_words = jp_l2.sel_words;
     jp.sel_coef = jp_l2.sel_coef;
     jp.sel_r2 = jp_l2.sel_r2;
-    jp.thr_f = -0.0f;                           // <x', y'> = (r^2 - |x - y|^2) / 2 >= 0: a score of either zero passes the bounds
+    jp.thr_f = -0.0f;                           // <x', y'> >= 0 (Euclidean: (r^2 - |x - y|^2) / 2): a score of either zero passes
     jp.thr_d = 0.0;
     CUtensorMap mapP, mapQ;
     if (!encode_rows_map(ctx, &mapP, ctx->emb_p.ptr, n, de, P_ROWS) || !encode_rows_map(ctx, &mapQ, ctx->emb_q.ptr, m, de, TILE_N))
@@ -580,17 +585,18 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     else if (i8 && kind == SIMJOIN_COS) e = launch_both<DT_I8, KIND_COS>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (!i8 && dense_available(i8, jp) && !longk &&
              (ctx->dense_mode == 1 || (ctx->dense_mode == 2 && ctx->last_density >= DENSE_MIN_PAIRS_PER_BLOCK))) {
-        // the last join on this context was dense: the 16-epilogue-warp instantiation of the same kind
-        if (kind == SIMJOIN_IP) e = launch_join_dense<KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
-        else if (kind == SIMJOIN_COS) e = launch_join_dense<KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem);
+        // The last join on this context was dense: the 16-epilogue-warp instantiation of the same kind -- or, where the
+        // transformed rows still fit two chunks, the sign test on transformed operands (Section 4's ip-distance
+        // embeddings: embed_rows_kernel).  Euclidean joins: that is the plain form; the small-radius form stays on
+        // the points themselves, and whichever the selection words call for does the work.
+        const bool embed = !fixed && (ctx->dense_mode == 1 || ctx->last_density >= EMBED_MIN_PAIRS_PER_BLOCK);
+        const simjoin_status es2 = embed ? launch_embedded(ctx, kind, P, n, Q, m, d, scr, jp, grid) : SIMJOIN_ERR_UNSUPPORTED;
+        if (es2 == SIMJOIN_ERR_CUDA) return SIMJOIN_ERR_CUDA;
+        e = cudaSuccess;
+        if (kind == SIMJOIN_IP) { if (es2 != SIMJOIN_OK) e = launch_join_dense<KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem); }
+        else if (kind == SIMJOIN_COS) { if (es2 != SIMJOIN_OK) e = launch_join_dense<KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem); }
         else {
-            // The plain form of the dense Euclidean join runs as an inner-product join on transformed operands where the
-            // transformed rows still fit two chunks (Section 4's squared-L2 embedding: l2_embed_rows_kernel); the
-            // small-radius form stays on the points themselves.  Whichever the selection words call for does the work.
-            const bool embed = !fixed && (ctx->dense_mode == 1 || ctx->last_density >= EMBED_MIN_PAIRS_PER_BLOCK);
-            const simjoin_status es2 = embed ? launch_l2_embedded(ctx, P, n, Q, m, d, scr, jp, grid) : SIMJOIN_ERR_UNSUPPORTED;
-            if (es2 == SIMJOIN_ERR_CUDA) return SIMJOIN_ERR_CUDA;
-            e = es2 == SIMJOIN_OK ? cudaSuccess : launch_join_dense<KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
+            if (es2 != SIMJOIN_OK) e = launch_join_dense<KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
             if (e == cudaSuccess) e = launch_join_dense<KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
         }
     }

@@ -580,6 +580,44 @@ def test_bf16_dense_epilogue_matches_the_oracle(kind, n, m, d):
                     assert cnt == len(Q[1:m:7][:n])
 
 
+@pytest.mark.parametrize("kind", ["ip", "cos"])
+@pytest.mark.parametrize("d", [24, 64, 112])
+def test_bf16_dense_sign_test_handles_zero_vectors_and_every_threshold(kind, d):
+    """Dense inner-product and cosine joins of rows up to 240 bytes run as the sign of one inner product on transformed
+    operands (the threshold, and for the cosine the norms, travel as appended coordinates).  Zero vectors on both sides
+    (their cosine counts as 0: they pass iff t <= 0), equal and opposite rows, thresholds of both signs, zero, tiny, huge
+    and infinite; the exact set outside the band, everything at +-inf."""
+    n, m = 300, 700
+    P, Q = W.random_points("bf16", n, d, 31), W.random_points("bf16", m, d, 32)
+    P[5] = 0
+    P[130] = 0
+    Q[7] = 0
+    Q[300:303] = 0
+    Q[11:311:3] = P[:100]
+    Q[12] = P[1] ^ np.uint16(0x8000)                     # the opposite row
+    Q[13] = W.f32_to_bf16_bits(W.bf16_bits_to_f32(P[2]) * 2.0 ** -60)      # a tiny multiple: cosine 1, inner product ~0
+    scale = d ** 0.5 if kind == "ip" else 1.0 / d ** 0.5
+    with B.Simjoin("bf16", 0) as ctx:
+        assert ctx.simjoin_set_option(B.SIMJOIN_OPT_DENSE_EPILOGUE, 1.0) == B.SIMJOIN_OK
+        for t in (0.0, -0.0, 1e-30, -1e-30, 0.2 * scale, -0.2 * scale, 1.7 * scale, -2.5 * scale, 0.999 if kind == "cos" else 3.0 * d,
+                  1.0 if kind == "cos" else 1e30, -1.0 if kind == "cos" else -1e30):
+            pairs, cnt = gpu_join(ctx, P, Q, kind, t, capacity=n * m + 8)
+            assert_band(pairs, cnt, P, Q, kind, t)
+        pairs, cnt = gpu_join(ctx, P, Q, kind, float("inf"), capacity=n * m + 8)
+        assert cnt == 0
+        pairs, cnt = gpu_join(ctx, P, Q, kind, float("-inf"), capacity=n * m + 8)
+        assert cnt == n * m
+    with B.Simjoin("bf16", 0) as ctx:                        # the same on the points themselves (8-warp layout)
+        assert ctx.simjoin_set_option(B.SIMJOIN_OPT_DENSE_EPILOGUE, 0.0) == B.SIMJOIN_OK
+        pairs, cnt = gpu_join(ctx, P, Q, kind, float("-inf"), capacity=n * m + 8)
+        assert cnt == n * m
+        pairs, cnt = gpu_join(ctx, P, Q, kind, float("inf"), capacity=n * m + 8)
+        assert cnt == 0
+        for t in (0.0, 1e-30, -1e-30):
+            pairs, cnt = gpu_join(ctx, P, Q, kind, t, capacity=n * m + 8)
+            assert_band(pairs, cnt, P, Q, kind, t)
+
+
 def test_repeated_runs_give_the_same_set(ctx_bf16):
     w = W.make_workload(5, n=3000, m=3000, centers=30)
     a, ca = gpu_join(ctx_bf16, w.P, w.Q, "l2", w.threshold, capacity=1 << 19)
