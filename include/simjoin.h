@@ -323,7 +323,9 @@ simjoin_status simjoin_set_offsets(simjoin_ctx *ctx, int64_t row_offset_p, int64
  *                                latency, which twice the warps hide; measured 77.5 -> 70.8 ms on 2.7e8 pairs out of
  *                                524 288^2, +2 % on a join with 1000 pairs out of 65 536^2); 2 (default) = by the
  *                                previous simjoin_run of the context: 16 warps after a join with at least one pair per
- *                                two such blocks.  A join in the 16-warp layout whose rows are at most 240 bytes long
+ *                                two such blocks; a context that has run no join yet counts the pairs of a sample first
+ *                                (its first 256 rows of P against 128 rows of Q per SM) when the join has at least
+ *                                1e12 operations.  A join in the 16-warp layout whose rows are at most 240 bytes long
  *                                (under 2: after a join with at least one pair per block) runs as the sign test of one
  *                                inner product on transformed operands -- Section 4's ip-distance embeddings with the
  *                                threshold folded in: 8 coordinates appended to context-owned copies of both point sets

@@ -43,6 +43,9 @@ constexpr double DENSE_MIN_PAIRS_PER_BLOCK = 0.5;
 // 16 against 8 warps: cosine 0.87 / 0.91 / 0.93 / 1.00 of the time at 8 / 2 / 0.5 / 0.125 pairs per block; Euclidean with the
 // transform 0.72 / 0.84 / 1.04 / 1.27.
 constexpr double EMBED_MIN_PAIRS_PER_BLOCK = 1.0;
+// Joins of at least this many operations (2 n m d) sample their output density when the context has no history: below
+// it the sample's launch and synchronisation (tens of microseconds) are not worth what the better layout saves.
+constexpr double DENSITY_SAMPLE_MIN_OPS = 1e12;
 constexpr int MAX_HOST_SLICES = 66;     // simjoin_run_host: a Q of more slices than this goes up in one piece
 
 // Device-side working memory of one join call, and the host words its result lands in.  simjoin_run takes it from the
@@ -493,6 +496,18 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         // one P tile per CTA plus a Q panel must fit in L2 (126 MB) for the sweep schedule; beyond that, 2-D waves
         if ((long long)ctx->num_sms * P_ROWS * row_bytes > (48LL << 20) && ctx->num_sms >= 8) jp.wave_gq = 4;
     }
+    // A context without history (no join yet) that is about to run a large bf16 join which has a dense layout first
+    // counts the pairs of a sample -- the first P tile against one Q tile per SM, a few microseconds -- so that its
+    // first join already runs in the layout its output density calls for (the count sets last_density).
+    if (!fixed && !i8 && !longk && ctx->dense_mode == 2 && ctx->last_density < 0.0 && dense_available(i8, jp) &&
+        2.0 * (double)n * (double)m * (double)d >= DENSITY_SAMPLE_MIN_OPS) {
+        ctx->last_density = 0.0;                // the sample itself runs sparse
+        uint64_t sampled = 0;
+        const simjoin_status ss = run_device(ctx, P, std::min<int64_t>(n, P_ROWS), Q, std::min<int64_t>(m, (int64_t)ctx->num_sms * TILE_N), d, kind,
+                                             threshold, nullptr, 0, &sampled);
+        if (ss != SIMJOIN_OK && ss != SIMJOIN_ERR_CAPACITY) return ss;
+        ctx->have_timing = false;
+    }
     jp.PB = (int)((n + P_ROWS - 1) / P_ROWS);
     jp.QT = (int)((m + tn - 1) / tn);
     jp.qpanel = q_panel_tiles(jp.QT, row_bytes, tn);
@@ -576,6 +591,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     if (timed) cudaEventRecord(ctx->ev[1], s);
     const int grid = ctx->num_sms;
     cudaError_t e = cudaErrorInvalidValue;
+    const char *layout = "8 epilogue warps";
     if (i8 && !select_i8) {
         if (kind == SIMJOIN_IP) e = launch_geo<DT_I8, KIND_IP, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
         else if (kind == SIMJOIN_L2) e = launch_geo<DT_I8, KIND_L2, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
@@ -592,6 +608,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         const bool embed = !fixed && (ctx->dense_mode == 1 || ctx->last_density >= EMBED_MIN_PAIRS_PER_BLOCK);
         const simjoin_status es2 = embed ? launch_embedded(ctx, kind, P, n, Q, m, d, scr, jp, grid) : SIMJOIN_ERR_UNSUPPORTED;
         if (es2 == SIMJOIN_ERR_CUDA) return SIMJOIN_ERR_CUDA;
+        layout = es2 == SIMJOIN_OK ? "16 epilogue warps on transformed operands" : "16 epilogue warps";
         e = cudaSuccess;
         if (kind == SIMJOIN_IP) { if (es2 != SIMJOIN_OK) e = launch_join_dense<KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem); }
         else if (kind == SIMJOIN_COS) { if (es2 != SIMJOIN_OK) e = launch_join_dense<KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem); }
@@ -615,10 +632,10 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     if (!fixed) ctx->ctrl_clean = cur ^ 1;        // the kernel has zeroed the other block
     *count = scr.h_ctrl[0];
     if (debug_log())
-        std::fprintf(stderr, "[simjoin] run dtype=%s kind=%d n=%lld m=%lld d=%d t=%g: %d chunk(s) per row, %s geometry, %d ring stages, "
+        std::fprintf(stderr, "[simjoin] run dtype=%s kind=%d n=%lld m=%lld d=%d t=%g: %d chunk(s) per row, %s geometry, %d ring stages, %s, "
                              "%s, pairs=%llu capacity=%llu\n",
                      i8 ? "i8" : "bf16", (int)kind, (long long)n, (long long)m, (int)d, threshold, jp.kc,
-                     longk ? (jp.wave_gq ? "long-row (2-D waves)" : "long-row") : (jp.stationary ? "resident-P" : "streamed"), jp.nstages,
+                     longk ? (jp.wave_gq ? "long-row (2-D waves)" : "long-row") : (jp.stationary ? "resident-P" : "streamed"), jp.nstages, layout,
                      jp.sel_mode == SEL_NONE ? "one variant" : (jp.sel_mode == SEL_I8_RANGE ? "epilogue width chosen on the device" : "Euclidean form chosen on the device"),
                      (unsigned long long)*count, (unsigned long long)capacity);
     ctx->last_density = (double)*count / ((double)((n + 31) / 32) * (double)((m + 127) / 128));

@@ -31,6 +31,7 @@ from paper_2006_12608_b200 import workloads as W            # noqa: E402
 
 OUT = os.path.join(os.path.dirname(os.path.abspath(__file__)), "full_size_digests.json")
 BAND_REL = 1e-2
+CAPACITY = 300_000_000          # one pass of the oracle: room for the densest configuration (2.7e8 pairs, 2.4 GB)
 
 
 def keys(pairs):
@@ -48,7 +49,8 @@ def one_config(cfg, threads):
              "inputs_sha256": {"P": hashlib.sha256(w.P.tobytes()).hexdigest(), "Q": hashlib.sha256(w.Q.tobytes()).hexdigest()}}
     t0 = time.time()
     if w.dtype == "i8":
-        pairs, count = O.join(w.P, w.Q, w.kind, w.threshold, w.dtype, threads=threads)
+        pairs, count = O.join(w.P, w.Q, w.kind, w.threshold, w.dtype, capacity=CAPACITY, threads=threads)
+        assert count <= CAPACITY
         entry["oracle_seconds"] = round(time.time() - t0, 1)
         k = np.sort(keys(pairs))
         assert len(k) == count and (len(k) < 2 or (np.diff(k) > 0).all())
@@ -57,7 +59,8 @@ def one_config(cfg, threads):
         t = float(w.threshold)
         delta = BAND_REL * abs(t)
         strict_t, loose_t = (t - delta, t + delta) if w.kind == "l2" else (t + delta, t - delta)
-        loose, _ = O.join(w.P, w.Q, w.kind, loose_t, w.dtype, threads=threads)
+        loose, count = O.join(w.P, w.Q, w.kind, loose_t, w.dtype, capacity=CAPACITY, threads=threads)
+        assert count <= CAPACITY
         entry["oracle_seconds"] = round(time.time() - t0, 1)
         # split the loose set by the oracle's own scores (one pass over its pairs instead of two more joins)
         s = O.scores(w.P, w.Q, w.kind, w.dtype, loose)

@@ -34,7 +34,7 @@ def keys(p):
 
 def run_full(w, capacity, dense_epilogue=None):
     """One join at full size, in the launch configuration `bench.py` times.  dense_epilogue: SIMJOIN_OPT_DENSE_EPILOGUE
-    (None: the default, under which the first call of a context runs the 8-warp layout)."""
+    (None: the default, under which a context picks the layout from a sample's pair count or from its previous join)."""
     build.build()
     with B.Simjoin(w.dtype, 0) as ctx:
         if dense_epilogue is not None:
@@ -114,7 +114,7 @@ def test_full_size_cfg2_cosine():
 
 @pytest.mark.parametrize("dense_epilogue", [0, 1])
 def test_full_size_cfg5_mixture_dense(dense_epilogue):
-    """Both layouts the bench's calls go through: 8 epilogue warps on the points themselves (a context's first call), and 16
+    """Both layouts, each forced: 8 epilogue warps on the points themselves, and 16
     warps on the operands with the squared-L2 embedding appended (every later call of a dense join)."""
     w = W.make_workload(5)
     per_p = np.bincount(w.labels_p, minlength=1024).astype(np.int64)

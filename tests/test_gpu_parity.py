@@ -3,6 +3,8 @@
 int8 joins must equal the oracle's sorted pair set bit for bit.  bf16 joins must lie
 between the oracle's strict and loose band sets (scores within 1e-2*|t| of the
 threshold may fall on either side); in-band disagreements are reported."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -616,6 +618,47 @@ def test_bf16_dense_sign_test_handles_zero_vectors_and_every_threshold(kind, d):
         for t in (0.0, 1e-30, -1e-30):
             pairs, cnt = gpu_join(ctx, P, Q, kind, t, capacity=n * m + 8)
             assert_band(pairs, cnt, P, Q, kind, t)
+
+
+def test_first_large_join_of_a_context_samples_its_density():
+    """A fresh context in the default mode counts a sample's pairs before a join of 1e12 operations or more and picks the
+    layout from that: the dense mixture then runs on transformed operands at once, a sparse join of the same size does not;
+    either way the result is the one the forced 8-warp layout gives."""
+    w = W.make_workload(5, n=98304, m=98304, centers=1024)
+    cap = 12_000_000
+    per_p = np.bincount(w.labels_p, minlength=1024).astype(np.int64)
+    per_q = np.bincount(w.labels_q, minlength=1024).astype(np.int64)
+    for t in (w.threshold, 0.01):
+        sets = []
+        for mode in (2.0, 0.0):
+            with B.Simjoin("bf16", 0) as ctx:
+                assert ctx.simjoin_set_option(B.SIMJOIN_OPT_DENSE_EPILOGUE, mode) == B.SIMJOIN_OK
+                pairs, cnt = gpu_join(ctx, w.P, w.Q, "l2", t, capacity=cap)
+                sets.append(np.sort(keys(pairs)))
+        assert np.array_equal(sets[0], sets[1])
+        if t == w.threshold:
+            assert len(sets[0]) == int(np.sum(per_p * per_q))
+
+
+def test_debug_log_names_the_layout_the_sample_chose():
+    """SIMJOIN_DEBUG=1: the sample's line, then the join's own line with the dense layout, on a context's very first call."""
+    import subprocess
+    import sys
+    code = (
+        "import torch\n"
+        "from paper_2006_12608_b200 import binding as B, workloads as W\n"
+        "w = W.make_workload(5, n=98304, m=98304, centers=1024)\n"
+        "out = torch.empty((12_000_000, 2), dtype=torch.int32, device='cuda:0')\n"
+        "with B.Simjoin('bf16', 0) as ctx:\n"
+        "    st, cnt = ctx.simjoin_run(B.to_device(w.P), w.n, B.to_device(w.Q), w.m, w.d, 'l2', w.threshold, out, 12_000_000)\n"
+        "    assert st == 0, st\n")
+    env = dict(os.environ, SIMJOIN_DEBUG="1")
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, cwd=os.path.dirname(os.path.dirname(__file__)), timeout=600)
+    assert r.returncode == 0, r.stderr
+    lines = [ln for ln in r.stderr.splitlines() if ln.startswith("[simjoin] run")]
+    assert len(lines) == 2
+    assert "n=256 " in lines[0] and "capacity=0" in lines[0] and "8 epilogue warps" in lines[0]
+    assert "n=98304 " in lines[1] and "16 epilogue warps on transformed operands" in lines[1]
 
 
 def test_repeated_runs_give_the_same_set(ctx_bf16):
