@@ -812,10 +812,11 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     constexpr bool LONGK = GEO == GEO_LONG, WIDEQ = GEO == GEO_WIDEQ;
     constexpr bool NARROW = DT == DT_I8 && ALT;
     constexpr bool L2_FILTER = DT == DT_BF16 && KIND == KIND_L2 && ALT;
-    // bf16 inner product, ALT: the threshold is zero and folded into the operands (the transformed Euclidean join), so a
-    // score passes when its sign bit is clear -- the element test is one funnel shift, no add.  In the device-side choice
-    // between the two Euclidean forms this kernel stands for the plain one.
+    // bf16 inner product, ALT: the threshold is zero and folded into the operands (dense joins of every kind on transformed
+    // operands), so a score passes when its sign bit is clear -- the element test is one funnel shift, no add.  In the
+    // device-side choice between the two Euclidean forms this kernel stands for the plain one.
     constexpr bool IP_SIGN = DT == DT_BF16 && KIND == KIND_IP && ALT;
+    static_assert(!IP_SIGN || EW == 2 * NUM_EPI_WARPS, "the sign test is built for the 16-warp layout only");
     constexpr bool SEL_ALT = ALT && !IP_SIGN;
     // The sign test with 16 epilogue warps: the two groups of eight take alternate tiles (group g owns accumulator g), and
     // every warp tests all 128 columns of its 32 rows in two loads of 64, so the per-tile work of a warp (barrier wait,
@@ -1308,8 +1309,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                                                 : KIND == KIND_COS ? __fmul_rn(rf, __uint_as_float(yw[c]))   // as level 0 rounds it
                                                 : L2_FILTER        ? __fmaf_rn(p.l2_ycoef, __uint_as_float(yw[c]), rf)
                                                                    : rf + 0.5f * __uint_as_float(yw[c]);
-                                if constexpr (IP_SIGN) fail[c >> 2] = __funnelshift_l(v[k * GCOLS + c], fail[c >> 2], 1);
-                                else fail[c >> 2] = __funnelshift_l(__float_as_uint(__uint_as_float(v[k * GCOLS + c]) - b), fail[c >> 2], 1);
+                                fail[c >> 2] = __funnelshift_l(__float_as_uint(__uint_as_float(v[k * GCOLS + c]) - b), fail[c >> 2], 1);
                             }
                             // chain q holds columns 4q .. 4q+3 at bits 3 .. 0
                             uint32_t fall = 0;                                  // column c -> bit GCOLS - 1 - c
