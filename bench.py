@@ -675,6 +675,10 @@ def finish(args, ctx, w, world, cnt, value, ms_per_step, join_ms, pre_ms, clocks
     roofline["prepass_ms"] = statistics.mean(pre_ms)
     # the join (int8 and bf16 Euclidean: both variants are launched, one returns at once), the norm pre-pass, max|x|
     launches_per_step = (2 if (w.dtype == "i8" or w.kind == "l2") else 1) + (2 if w.kind != "ip" else 0) + (1 if w.dtype == "i8" else 0)
+    # dense bf16 joins of short rows run on transformed copies of both point sets: two more launches
+    blocks = -(-w.n // 32) * -(-w.m // 128)
+    if w.dtype == "bf16" and (w.d + 8) * 2 <= 256 and cnt / blocks >= 1.0:
+        launches_per_step += 2
     if args.lsh:
         # max|x| x2, sampled coordinates, keys x2, then per table: 2 histograms, offsets + work list, 2 scatters, 2 row
         # gathers, the join
