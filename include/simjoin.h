@@ -95,7 +95,16 @@ simjoin_status simjoin_create(simjoin_ctx **ctx, simjoin_dtype dtype, int device
  *               norms the pre-pass meets, is compared with 1.9 % of r^2 on the
  *               device; when it is larger the tile test only raises candidates,
  *               lowered by that bound, and each is decided in the difference
- *               form from its two rows.  r = 0 returns exactly the equal rows.)
+ *               form from its two rows.  r = 0 returns exactly the equal rows.
+ *               BF16/IP and BF16/COS: where the band is narrower than the fp32
+ *               accumulation error of the tile product -- t = 0 above all, where
+ *               it is empty -- the tile test likewise only raises candidates and
+ *               each is decided from its two rows in fp64, products exact, sums
+ *               over k ascending: the exact decision.  Cosine: chosen by the
+ *               host, |t| below ~200 error bounds; inner product: chosen on
+ *               the device from the largest norms, for which every BF16/IP join
+ *               runs the norm pre-pass.  A BF16 cosine threshold beyond +-2
+ *               decides like +-2.)
  *   out_pairs   device pointer to capacity x 2 int32, written as (i, j) rows.
  *               May be NULL when capacity == 0 (count-only mode).
  *   count       HOST pointer; receives the total number of passing pairs, even
@@ -260,7 +269,9 @@ simjoin_status simjoin_run_hamming(simjoin_ctx *ctx, const void *P_bits, int64_t
  *
  * Arithmetic: I8 exact (the decisions simjoin_run takes); BF16 in fp32 -- inner product and cosine as sums over
  * the row, the Euclidean distance in the difference form sum (x - y)^2 <= r^2 (no cancellation of large norms);
- * a pair whose exact score lies within 1e-2*|threshold| of the threshold may fall on either side.
+ * a pair whose exact score lies within 1e-2*|threshold| of the threshold may fall on either side.  An inner product or
+ * cosine whose fp32 value lies within the sums' rounding error of the threshold is decided again in fp64 (exact
+ * products, k ascending), so thresholds at or next to zero, whose band is empty, are decided exactly too.
  * A group of lanes per pair (sized to the row), two rows read per pair.  Synchronises the stream.  Scratch: count_in x 8 bytes.
  */
 simjoin_status simjoin_filter_pairs(simjoin_ctx *ctx, const void *P, int64_t n, const void *Q, int64_t m, int32_t d,

@@ -18,7 +18,10 @@ constexpr int FILTER_THREADS = 256;
 // int8 rows: exact integer sums.  IP: s >= ceil(t) (thr_i);  L2: sum (x-y)^2 <= floor(r^2) (thr_i), taken as
 // |x|^2 + |y|^2 - 2s in integers;  COS: the fp64 sequence of the join's exact test (thr_d).
 // bf16 rows: fp32 sums.  IP: s >= t;  COS: s >= t |x| |y|, a zero vector scoring 0;  L2: the difference form
-// sum (x-y)^2 <= r^2, which does not cancel like the norm expansion of the tile epilogue.
+// sum (x-y)^2 <= r^2, which does not cancel like the norm expansion of the tile epilogue.  An inner product or cosine
+// whose fp32 value lies within the sums' rounding error ((d + 32) 2^-23 |x| |y|) of the threshold is decided again in
+// fp64 (exact products, k ascending, the fp64 threshold): whatever the threshold -- zero included, where the tolerance
+// band 1e-2 |t| is empty -- the decision is the one exact arithmetic takes.
 template <int DT, int KIND>
 __global__ void __launch_bounds__(FILTER_THREADS)
 filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__restrict__ Q, long long m, int g,
@@ -84,7 +87,7 @@ filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__res
                         s = fmaf(x0, y0, s);
                         s = fmaf(x1, y1, s);
                     }
-                    if constexpr (KIND == KIND_COS) {
+                    if constexpr (KIND != KIND_L2) {
                         nx = fmaf(x0, x0, nx);
                         nx = fmaf(x1, x1, nx);
                         ny = fmaf(y0, y0, ny);
@@ -94,14 +97,39 @@ filter_pairs_kernel(const uint4 *__restrict__ P, long long n, const uint4 *__res
             }
             for (int off = G >> 1; off > 0; off >>= 1) {
                 s += __shfl_xor_sync(0xffffffffu, s, off);
-                if constexpr (KIND == KIND_COS) {
+                if constexpr (KIND != KIND_L2) {
                     nx += __shfl_xor_sync(0xffffffffu, nx, off);
                     ny += __shfl_xor_sync(0xffffffffu, ny, off);
                 }
             }
-            if constexpr (KIND == KIND_IP) pass = s >= thr_f;
             if constexpr (KIND == KIND_L2) pass = s <= thr_f;
-            if constexpr (KIND == KIND_COS) pass = (nx == 0.f || ny == 0.f) ? thr_f <= 0.f : s >= thr_f * sqrtf(nx) * sqrtf(ny);
+            if constexpr (KIND != KIND_L2) {
+                const float nn = sqrtf(nx) * sqrtf(ny);
+                const float b = KIND == KIND_IP ? thr_f : thr_f * nn;
+                pass = s >= b;
+                const float margin = (float)(g * 8 + 32) * 0x1p-23f * nn;
+                // (a comparison that is false for a NaN or infinite margin also takes the slow path)
+                if (live && lane == 0 && !(fabsf(s - b) > margin)) {
+                    double s2 = 0.0, nx2 = 0.0, ny2 = 0.0;
+                    for (int c = 0; c < g; ++c) {
+                        const uint4 a = __ldg(x + c), bb = __ldg(y + c);
+                        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const double x0 = (double)__uint_as_float(aw[t] << 16), x1 = (double)__uint_as_float(aw[t] & 0xffff0000u);
+                            const double y0 = (double)__uint_as_float(bw[t] << 16), y1 = (double)__uint_as_float(bw[t] & 0xffff0000u);
+                            s2 = __dadd_rn(s2, __dmul_rn(x0, y0));
+                            s2 = __dadd_rn(s2, __dmul_rn(x1, y1));
+                            nx2 = __dadd_rn(nx2, __dmul_rn(x0, x0));
+                            nx2 = __dadd_rn(nx2, __dmul_rn(x1, x1));
+                            ny2 = __dadd_rn(ny2, __dmul_rn(y0, y0));
+                            ny2 = __dadd_rn(ny2, __dmul_rn(y1, y1));
+                        }
+                    }
+                    if constexpr (KIND == KIND_IP) pass = s2 >= thr_d;
+                    else pass = (nx2 == 0.0 || ny2 == 0.0) ? 0.0 >= thr_d : __ddiv_rn(s2, __dmul_rn(__dsqrt_rn(nx2), __dsqrt_rn(ny2))) >= thr_d;
+                }
+            }
         }
         if (live && lane == 0 && pass) out[atomicAdd(counter, 1ULL)] = pr;
     }

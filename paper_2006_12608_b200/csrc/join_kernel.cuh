@@ -153,13 +153,20 @@ struct JoinParams {
     float store_scale;
 };
 
-constexpr int SEL_NONE = 0, SEL_I8_RANGE = 1, SEL_L2_RADIUS = 2;
+constexpr int SEL_NONE = 0, SEL_I8_RANGE = 1, SEL_L2_RADIUS = 2, SEL_IP_SMALL = 3;
 // Share of r^2 that the norm expansion's rounding error may reach before the Euclidean join switches to deciding
 // candidates from the rows: the tolerance is |distance - r| <= 1e-2 r, i.e. 1.99 % of r^2 on the squared scale.
 constexpr float L2_BAND_SHARE = 0.019f;
+// Share of the tolerance band 1e-2 |t| that the fp32 accumulation error of an inner product (at most sel_coef |x| |y|)
+// may reach before a bf16 inner-product or cosine join switches to deciding candidates from the rows in fp64.
+constexpr float IPCOS_BAND_SHARE = 0.5e-2f;
+// How far below the threshold that form's tile filter sits, in units of the error bound.
+constexpr float IPCOS_FILTER_MARGIN = 1.25f;
 __device__ __forceinline__ bool alt_selected(const JoinParams &p) {
     const unsigned int a = __ldg(p.sel_words), b = __ldg(p.sel_words + 1);
     if (p.sel_mode == SEL_I8_RANGE) return (unsigned long long)p.row_bytes * a * b <= 32767ull;
+    // SEL_IP_SMALL: the words hold max |x|^2 and max |y|^2, sel_r2 the threshold t
+    if (p.sel_mode == SEL_IP_SMALL) return p.sel_coef * (sqrtf(__uint_as_float(a)) * sqrtf(__uint_as_float(b))) > IPCOS_BAND_SHARE * fabsf(p.sel_r2);
     return p.sel_coef * (__uint_as_float(a) + __uint_as_float(b)) > L2_BAND_SHARE * p.sel_r2;
 }
 
@@ -375,11 +382,45 @@ __device__ __forceinline__ bool l2_bf16_passes(const JoinParams &p, long long li
     return (s[0] + s[1]) + (s[2] + s[3]) <= p.thr_f;
 }
 
+// BF16 inner product / cosine, thresholds so close to zero that the tolerance band is narrower than the fp32 accumulation
+// error: the decision for the pair of rows (li of P, lj of Q) in fp64 -- products of bf16 values are exact in fp64, the
+// sums run over k ascending, the cosine is <x,y> / (sqrt(|x|^2) sqrt(|y|^2)) and 0 for a zero vector; the compare takes
+// the fp64 threshold.
+template <bool COS>
+__device__ __forceinline__ bool ipcos_bf16_passes(const JoinParams &p, long long li, long long lj) {
+    const int g = p.row_bytes >> 4;
+    const uint4 *x = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.rows_p) + li * p.row_bytes);
+    const uint4 *y = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.rows_q) + lj * p.row_bytes);
+    double s = 0.0, nx = 0.0, ny = 0.0;
+    for (int c = 0; c < g; ++c) {
+        const uint4 a = __ldg(x + c), b = __ldg(y + c);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const double x0 = (double)__uint_as_float(aw[t] << 16), x1 = (double)__uint_as_float(aw[t] & 0xffff0000u);
+            const double y0 = (double)__uint_as_float(bw[t] << 16), y1 = (double)__uint_as_float(bw[t] & 0xffff0000u);
+            s = __dadd_rn(s, __dmul_rn(x0, y0));
+            s = __dadd_rn(s, __dmul_rn(x1, y1));
+            if constexpr (COS) {
+                nx = __dadd_rn(nx, __dmul_rn(x0, x0));
+                nx = __dadd_rn(nx, __dmul_rn(x1, x1));
+                ny = __dadd_rn(ny, __dmul_rn(y0, y0));
+                ny = __dadd_rn(ny, __dmul_rn(y1, y1));
+            }
+        }
+    }
+    if constexpr (COS) {
+        if (nx == 0.0 || ny == 0.0) return 0.0 >= p.thr_d;
+        return __ddiv_rn(s, __dmul_rn(__dsqrt_rn(nx), __dsqrt_rn(ny))) >= p.thr_d;
+    }
+    return s >= p.thr_d;
+}
+
 // Is the staged pair dropped when it leaves the CTA?  Bucketed mode: reported by an earlier repetition.  VERIFY:
 // the pair is a candidate of a tile-level filter and fails the decision taken from its two rows (VERIFY_COS_I8: the
 // exact int8 cosine; VERIFY_L2_BF16: the difference-form Euclidean test).  Staged indices are regrouped positions
 // in bucketed mode, else row indices plus the caller's offsets.
-constexpr int VERIFY_NONE = 0, VERIFY_COS_I8 = 1, VERIFY_L2_BF16 = 2;
+constexpr int VERIFY_NONE = 0, VERIFY_COS_I8 = 1, VERIFY_L2_BF16 = 2, VERIFY_IP_BF16 = 3, VERIFY_COS_BF16 = 4;
 template <bool GROUPED, int VERIFY>
 __device__ __forceinline__ bool drop_pair(const JoinParams &p, int i, int j) {
     if constexpr (GROUPED) {
@@ -390,6 +431,9 @@ __device__ __forceinline__ bool drop_pair(const JoinParams &p, int i, int j) {
     }
     if constexpr (VERIFY == VERIFY_L2_BF16) {
         if (!l2_bf16_passes(p, GROUPED ? i : i - p.ioff, GROUPED ? j : j - p.joff)) return true;
+    }
+    if constexpr (VERIFY == VERIFY_IP_BF16 || VERIFY == VERIFY_COS_BF16) {
+        if (!ipcos_bf16_passes<VERIFY == VERIFY_COS_BF16>(p, GROUPED ? i : i - p.ioff, GROUPED ? j : j - p.joff)) return true;
     }
     return false;
 }
@@ -815,14 +859,17 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     // bf16 inner product, ALT: the threshold is zero and folded into the operands (dense joins of every kind on transformed
     // operands), so a score passes when its sign bit is clear -- the element test is one funnel shift, no add.  In the
     // device-side choice between the two Euclidean forms this kernel stands for the plain one.
-    constexpr bool IP_SIGN = DT == DT_BF16 && KIND == KIND_IP && ALT;
-    static_assert(!IP_SIGN || EW == 2 * NUM_EPI_WARPS, "the sign test is built for the 16-warp layout only");
+    constexpr bool IP_SIGN = DT == DT_BF16 && KIND == KIND_IP && ALT && EW == 2 * NUM_EPI_WARPS;
+    // bf16 inner product (8 epilogue warps) and cosine, ALT: the tile test is a filter lowered by the fp32 accumulation error
+    // bound, and every candidate is decided from its rows in fp64 when the warp's staging buffer is flushed -- for
+    // thresholds whose tolerance band 1e-2 |t| is narrower than that error (t = 0 above all).
+    constexpr bool IPCOS_FILTER = DT == DT_BF16 && ALT && ((KIND == KIND_IP && EW == NUM_EPI_WARPS) || KIND == KIND_COS);
     constexpr bool SEL_ALT = ALT && !IP_SIGN;
     // The sign test with 16 epilogue warps: the two groups of eight take alternate tiles (group g owns accumulator g), and
     // every warp tests all 128 columns of its 32 rows in two loads of 64, so the per-tile work of a warp (barrier wait,
     // hand-back, tail mask, compaction) is paid once per 128 columns instead of once per 64.
     constexpr bool TWO_TILE = IP_SIGN && EW == 2 * NUM_EPI_WARPS;
-    static_assert(DT == DT_I8 || !ALT || KIND == KIND_L2 || KIND == KIND_IP, "bf16: the Euclidean and inner-product kinds have a second variant");
+    static_assert(DT == DT_I8 || !ALT || KIND == KIND_L2 || KIND == KIND_IP || KIND == KIND_COS, "bf16: the join kinds have a second variant");
     // not the variant the data calls for: the other launch does the work (uniform over the grid, before any barrier
     // or tensor-memory allocation exists)
     if (p_in.zero_next != nullptr && blockIdx.x == 0 && threadIdx.x < 8) p_in.zero_next[threadIdx.x] = 0ull;
@@ -837,6 +884,11 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     constexpr int ECOLS = epi_cols(EW);                    // accumulator columns per epilogue warp and pass
     constexpr int SPAIRS = stage_pairs(EW);                // pairs a warp stages before it flushes
     JoinParams p = p_in;
+    if constexpr (IPCOS_FILTER && KIND == KIND_IP) {
+        // the filter threshold: t lowered by the error bound at the largest norms (the words hold max |x|^2, max |y|^2)
+        const float mx = sqrtf(__uint_as_float(__ldg(p.sel_words))), my = sqrtf(__uint_as_float(__ldg(p.sel_words + 1)));
+        p.thr_f = __fsub_rd(p.thr_f, __fmul_ru(IPCOS_FILTER_MARGIN * p.sel_coef, __fmul_ru(mx, my)));
+    }
     if constexpr (LONGK) {
         p.stationary = 0;
         p.epi_release = 0;
@@ -984,7 +1036,11 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
         uint32_t rstage = TWO_TILE ? group * p.kc : 0;    // next ring stage to hand back
         uint32_t tile_parity = 0;                         // TWO_TILE: parity of the number of tiles before this unit
         // candidates of a filter are decided from their rows at flush time
-        constexpr int VERIFY = (DT == DT_I8 && KIND == KIND_COS) ? VERIFY_COS_I8 : (L2_FILTER ? VERIFY_L2_BF16 : VERIFY_NONE);
+        constexpr int VERIFY = (DT == DT_I8 && KIND == KIND_COS) ? VERIFY_COS_I8
+                               : L2_FILTER                      ? VERIFY_L2_BF16
+                               : !IPCOS_FILTER                  ? VERIFY_NONE
+                               : KIND == KIND_IP                ? VERIFY_IP_BF16
+                                                                : VERIFY_COS_BF16;
         int2 *stage_buf = smem_staging + (warp - EPI_WARP0) * (warp_stage_bytes(EW) / 8);
         uint32_t *colterm = reinterpret_cast<uint32_t *>(stage_buf + SPAIRS);
         int stage_fill = 0;

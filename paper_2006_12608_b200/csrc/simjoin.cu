@@ -341,6 +341,14 @@ void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold
         if (kind == SIMJOIN_COS) jp.thr_f = fminf(fmaxf(jp.thr_f, -2.f), 2.f);
         // the inner-product and cosine tests read the sign of s - b: with t = -0 a score of either zero gives +0 and passes
         if (kind != SIMJOIN_L2 && jp.thr_f == 0.f) jp.thr_f = -0.0f;
+        if (kind != SIMJOIN_L2 && d > 0) {
+            // Rounding error of the fp32-accumulated inner product relative to |x| |y| (sum |x_k y_k| is at most that),
+            // charged like the Euclidean form below: d / 2 roundings of 2^-24 for the tensor core, 8 ceil(g / 32) + 5
+            // for the norms the cosine test multiplies with, 16 for the epilogue's own operations.  Where this exceeds
+            // half the tolerance band 1e-2 |t| the join decides its candidates from the rows in fp64 (see run_device).
+            const int g = d * 2 / 16;
+            jp.sel_coef = (float)std::ldexp(8.0 * ((g + 31) / 32) + 5.0 + 0.5 * d + 16.0, -24);
+        }
         if (kind == SIMJOIN_L2 && d > 0) {
             // Rounding error of the norm expansion |x|^2 + |y|^2 - 2<x,y> as the tile epilogue evaluates it, relative to
             // |x|^2 + |y|^2, counted in fp32 roundings of at most 2^-24 each: the pre-pass adds a row's squares in at
@@ -362,9 +370,9 @@ void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold
 
 // What the norm pre-pass stores per row.  0: |x|^2; 1: |x| in fp32 (cosine); 2: the same with +inf for a zero
 // vector -- cosine with t > 0, where a zero vector passes nothing: the epilogue's products t |x| |y| are then +inf.
-int norm_mode(bool /*i8*/, simjoin_kind kind, double threshold) {
+int norm_mode(bool /*i8*/, simjoin_kind kind, float thr_f) {
     if (kind != SIMJOIN_COS) return 0;
-    return (float)threshold > 0.f ? 2 : 1;        // decided on the fp32 threshold the epilogue uses
+    return thr_f > 0.f ? 2 : 1;                   // decided on the fp32 threshold the epilogue uses
 }
 
 // The inner-product kernel of launch_embedded: 16 epilogue warps, KC chunks per row, LASTK K steps in the last one.
@@ -462,6 +470,28 @@ void set_selection(JoinParams &jp, bool i8, simjoin_kind kind, unsigned long lon
     }
 }
 
+// bf16 inner-product and cosine joins whose threshold sits so close to zero that the tolerance band 1e-2 |t| is narrower
+// than the fp32 accumulation error of the tile product decide their candidates from the rows in fp64.
+// Cosine: relative to |x| |y| both sides of the comparison scale alike, so the host can tell -- returns true and lowers the
+// tile test's threshold to the filter's.
+bool cos_row_form(JoinParams &jp, bool i8, simjoin_kind kind) {
+    if (i8 || kind != SIMJOIN_COS) return false;
+    const bool rows = jp.sel_coef > IPCOS_BAND_SHARE * std::fabs(jp.thr_f);
+    if (rows) {
+        jp.thr_f = std::nextafterf(jp.thr_f - IPCOS_FILTER_MARGIN * jp.sel_coef, -INFINITY);
+        if (jp.thr_f == 0.f) jp.thr_f = -0.0f;
+    }
+    return rows;
+}
+// Inner product: it depends on the largest norms, which the norm pre-pass leaves in the control block: the device chooses
+// between the two forms (both are launched).
+void ip_form_selection(JoinParams &jp, bool i8, simjoin_kind kind, unsigned long long *d_ctrl) {
+    if (i8 || kind != SIMJOIN_IP) return;
+    jp.sel_mode = SEL_IP_SMALL;
+    jp.sel_words = reinterpret_cast<const unsigned int *>(d_ctrl + 3);
+    jp.sel_r2 = jp.thr_f;
+}
+
 cudaError_t launch_maxabs(const simjoin_ctx *ctx, const void *P, long long p16, const void *Q, long long q16, unsigned long long *d_ctrl) {
     maxabs_i8_kernel<<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(reinterpret_cast<const uint4 *>(P), p16, reinterpret_cast<const uint4 *>(Q), q16,
                                                                  reinterpret_cast<unsigned int *>(d_ctrl + 2));
@@ -521,7 +551,13 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.rows_q = Q;
     jp.row_bytes = row_bytes;
 
-    const bool need_norms = kind != SIMJOIN_IP;
+    // bf16 inner-product joins run the norm pre-pass for its maxima: they tell whether the threshold's tolerance band is
+    // wider than the fp32 accumulation error (decided on the device, like the Euclidean form)
+    const bool need_norms = kind != SIMJOIN_IP || !i8;
+    // bf16 cosine with a threshold that close to zero: the tile test becomes a filter lowered by the error bound and every
+    // candidate is decided from its rows in fp64 (relative to |x| |y| both sides of the comparison scale alike, so the
+    // host can tell)
+    const bool cos_rows = cos_row_form(jp, i8, kind);
     JoinScratch scr;
     if (fixed) {
         scr = *fixed;
@@ -560,6 +596,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     // small int8 joins take the 32-bit epilogue unasked (see DEFAULT_SELECT_MIN_OPS)
     const bool select_i8 = i8 && 2.0 * (double)n * (double)m * (double)d >= ctx->select_min_ops;
     if (!i8 || select_i8) set_selection(jp, i8, kind, scr.d_ctrl);
+    ip_form_selection(jp, i8, kind, scr.d_ctrl);
 
     CUtensorMap mapP, mapQ;
     if (!encode_rows_map(ctx, &mapP, P, n, d, P_ROWS) || !encode_rows_map(ctx, &mapQ, Q, m, d, tn))
@@ -573,8 +610,8 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         return SIMJOIN_ERR_CUDA;
     if (timed && need_norms) cudaEventRecord(ctx->ev[0], s);      // (every event is a step in the stream: none without a pre-pass)
     if (need_norms) {
-        const int sq = norm_mode(i8, kind, threshold);
-        unsigned int *nmax = (!i8 && kind == SIMJOIN_L2) ? reinterpret_cast<unsigned int *>(scr.d_ctrl + 3) : nullptr;
+        const int sq = norm_mode(i8, kind, i8 ? (float)threshold : jp.thr_f);
+        unsigned int *nmax = (!i8 && kind != SIMJOIN_COS) ? reinterpret_cast<unsigned int *>(scr.d_ctrl + 3) : nullptr;
         cudaError_t e1, e2;
         if (i8) {
             e1 = launch_norms<true>(ctx, P, n, d, sq, scr.nx, nullptr);
@@ -599,6 +636,7 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     } else if (i8 && kind == SIMJOIN_IP) e = launch_both<DT_I8, KIND_IP>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_L2) e = launch_both<DT_I8, KIND_L2>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (i8 && kind == SIMJOIN_COS) e = launch_both<DT_I8, KIND_COS>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    else if (cos_rows) e = launch_geo<DT_BF16, KIND_COS, true>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (!i8 && dense_available(i8, jp) && !longk &&
              (ctx->dense_mode == 1 || (ctx->dense_mode == 2 && ctx->last_density >= DENSE_MIN_PAIRS_PER_BLOCK))) {
         // The last join on this context was dense: the 16-epilogue-warp instantiation of the same kind -- or, where the
@@ -610,14 +648,18 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         if (es2 == SIMJOIN_ERR_CUDA) return SIMJOIN_ERR_CUDA;
         layout = es2 == SIMJOIN_OK ? "16 epilogue warps on transformed operands" : "16 epilogue warps";
         e = cudaSuccess;
-        if (kind == SIMJOIN_IP) { if (es2 != SIMJOIN_OK) e = launch_join_dense<KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem); }
+        if (kind == SIMJOIN_IP) {
+            if (es2 != SIMJOIN_OK) e = launch_join_dense<KIND_IP, false>(ctx, mapP, mapQ, jp, grid, smem);
+            // (the row-deciding form of the inner-product join has one layout: 8 epilogue warps)
+            if (e == cudaSuccess) e = launch_geo<DT_BF16, KIND_IP, true>(ctx, false, mapP, mapQ, jp, grid, smem);
+        }
         else if (kind == SIMJOIN_COS) { if (es2 != SIMJOIN_OK) e = launch_join_dense<KIND_COS, false>(ctx, mapP, mapQ, jp, grid, smem); }
         else {
             if (es2 != SIMJOIN_OK) e = launch_join_dense<KIND_L2, false>(ctx, mapP, mapQ, jp, grid, smem);
             if (e == cudaSuccess) e = launch_join_dense<KIND_L2, true>(ctx, mapP, mapQ, jp, grid, smem);
         }
     }
-    else if (!i8 && kind == SIMJOIN_IP) e = launch_geo<DT_BF16, KIND_IP, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
+    else if (!i8 && kind == SIMJOIN_IP) e = launch_both<DT_BF16, KIND_IP>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (!i8 && kind == SIMJOIN_COS) e = launch_geo<DT_BF16, KIND_COS, false>(ctx, longk, mapP, mapQ, jp, grid, smem);
     else if (!i8 && kind == SIMJOIN_L2) e = launch_both<DT_BF16, KIND_L2>(ctx, longk, mapP, mapQ, jp, grid, smem);
     if (e != cudaSuccess) return SIMJOIN_ERR_CUDA;
@@ -636,7 +678,11 @@ simjoin_status run_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
                              "%s, pairs=%llu capacity=%llu\n",
                      i8 ? "i8" : "bf16", (int)kind, (long long)n, (long long)m, (int)d, threshold, jp.kc,
                      longk ? (jp.wave_gq ? "long-row (2-D waves)" : "long-row") : (jp.stationary ? "resident-P" : "streamed"), jp.nstages, layout,
-                     jp.sel_mode == SEL_NONE ? "one variant" : (jp.sel_mode == SEL_I8_RANGE ? "epilogue width chosen on the device" : "Euclidean form chosen on the device"),
+                     cos_rows ? "candidates decided from the rows (threshold near zero)"
+                     : jp.sel_mode == SEL_NONE ? "one variant"
+                     : jp.sel_mode == SEL_I8_RANGE ? "epilogue width chosen on the device"
+                     : jp.sel_mode == SEL_IP_SMALL ? "plain or row-deciding form chosen on the device"
+                                                   : "Euclidean form chosen on the device",
                      (unsigned long long)*count, (unsigned long long)capacity);
     ctx->last_density = (double)*count / ((double)((n + 31) / 32) * (double)((m + 127) / 128));
     float a = 0.f, b = 0.f;
@@ -678,12 +724,13 @@ simjoin_status hyperplane_keys(simjoin_ctx *ctx, const void *planes, int plane_r
 
 // One bucketed join launch: instantiation by element type, kind, variant and geometry.
 cudaError_t launch_bucketed(simjoin_ctx *ctx, bool i8, simjoin_kind kind, bool longk, const CUtensorMap &mp,
-                            const CUtensorMap &mq, const JoinParams &jp, size_t smem) {
+                            const CUtensorMap &mq, const JoinParams &jp, size_t smem, bool cos_rows) {
     const int grid = ctx->num_sms;
 #define SJ_BUCKETED(DT, KIND, ALT)                                                          \
     (longk ? launch_join_long<DT, KIND, ALT, true>(ctx, mp, mq, jp, grid, smem) \
            : launch_join<DT, KIND, ALT, true>(ctx, mp, mq, jp, grid, smem))
-    // where the device selects the variant (int8; bf16 Euclidean) both are launched and one returns at once
+    // where the device selects the variant (int8; bf16 Euclidean and inner product) both are launched and one returns at
+    // once; the row-deciding form of the bf16 cosine join is the host's choice (cos_rows)
 #define SJ_BUCKETED_BOTH(DT, KIND)                                   \
     {                                                                \
         const cudaError_t e = SJ_BUCKETED(DT, KIND, false);          \
@@ -692,8 +739,8 @@ cudaError_t launch_bucketed(simjoin_ctx *ctx, bool i8, simjoin_kind kind, bool l
     if (i8 && kind == SIMJOIN_IP) SJ_BUCKETED_BOTH(DT_I8, KIND_IP)
     if (i8 && kind == SIMJOIN_L2) SJ_BUCKETED_BOTH(DT_I8, KIND_L2)
     if (i8 && kind == SIMJOIN_COS) SJ_BUCKETED_BOTH(DT_I8, KIND_COS)
-    if (!i8 && kind == SIMJOIN_IP) return SJ_BUCKETED(DT_BF16, KIND_IP, false);
-    if (!i8 && kind == SIMJOIN_COS) return SJ_BUCKETED(DT_BF16, KIND_COS, false);
+    if (!i8 && kind == SIMJOIN_IP) SJ_BUCKETED_BOTH(DT_BF16, KIND_IP)
+    if (!i8 && kind == SIMJOIN_COS) return cos_rows ? SJ_BUCKETED(DT_BF16, KIND_COS, true) : SJ_BUCKETED(DT_BF16, KIND_COS, false);
     if (!i8 && kind == SIMJOIN_L2) SJ_BUCKETED_BOTH(DT_BF16, KIND_L2)
 #undef SJ_BUCKETED_BOTH
 #undef SJ_BUCKETED
@@ -709,7 +756,7 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     const bool i8 = ctx->dtype == SIMJOIN_I8;
     const size_t es = elem_size(ctx->dtype);
     const int row_bytes = (int)(d * es);
-    const bool need_norms = kind != SIMJOIN_IP;
+    const bool need_norms = kind != SIMJOIN_IP || !i8;       // (bf16 inner product: for the maxima, as in run_device)
 
     JoinParams jp;
     size_t smem = 0;
@@ -756,6 +803,8 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
     jp.joff = (int)ctx->joff;
     set_thresholds(jp, i8, kind, threshold, d);
     set_selection(jp, i8, kind, ctx->d_ctrl);
+    const bool cos_rows = cos_row_form(jp, i8, kind);
+    ip_form_selection(jp, i8, kind, ctx->d_ctrl);
     jp.rows_p = ctx->lsh_sorted_p.ptr;      // the regrouped rows, addressed by regrouped position
     jp.rows_q = ctx->lsh_sorted_q.ptr;
     jp.row_bytes = row_bytes;
@@ -851,13 +900,13 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
             reinterpret_cast<const uint4 *>(Q), perm_q, m, g, reinterpret_cast<uint4 *>(ctx->lsh_sorted_q.ptr));
         if (need_norms) {
             // row terms and per-256-row bounds of the regrouped rows
-            const int sq = norm_mode(i8, kind, threshold);
+            const int sq = norm_mode(i8, kind, i8 ? (float)threshold : jp.thr_f);
             cudaError_t e1, e2;
             if (i8) {
                 e1 = launch_norms<true>(ctx, ctx->lsh_sorted_p.ptr, n, d, sq, ctx->nx.ptr, nullptr);
                 e2 = launch_norms<true>(ctx, ctx->lsh_sorted_q.ptr, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr);
             } else {
-                unsigned int *nmax = kind == SIMJOIN_L2 ? reinterpret_cast<unsigned int *>(ctx->d_ctrl + 3) : nullptr;
+                unsigned int *nmax = kind != SIMJOIN_COS ? reinterpret_cast<unsigned int *>(ctx->d_ctrl + 3) : nullptr;
                 e1 = launch_norms<false>(ctx, ctx->lsh_sorted_p.ptr, n, d, sq, ctx->nx.ptr, nullptr, nmax);
                 e2 = launch_norms<false>(ctx, ctx->lsh_sorted_q.ptr, m, d, sq, ctx->ny.ptr, ctx->qstat.ptr, nmax ? nmax + 1 : nullptr);
             }
@@ -865,7 +914,7 @@ simjoin_status lsh_device(simjoin_ctx *ctx, const void *P, int64_t n, const void
         }
         if (cudaGetLastError() != cudaSuccess) return SIMJOIN_ERR_CUDA;
         jp.rep = l;
-        if (launch_bucketed(ctx, i8, kind, longk, mapP, mapQ, jp, smem) != cudaSuccess) return SIMJOIN_ERR_CUDA;
+        if (launch_bucketed(ctx, i8, kind, longk, mapP, mapQ, jp, smem, cos_rows) != cudaSuccess) return SIMJOIN_ERR_CUDA;
     }
     cudaEventRecord(ctx->ev[2], s);
     if (cudaMemcpyAsync(ctx->h_ctrl, ctx->d_ctrl, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SIMJOIN_ERR_CUDA;

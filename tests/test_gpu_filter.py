@@ -86,6 +86,34 @@ def test_filter_bf16_within_the_band(ctxs, kind, t, d):
     assert np.array_equal(kcnts, cnts[np.searchsorted(ck, kk)])                           # a kept pair keeps every copy
 
 
+@pytest.mark.parametrize("kind", ["ip", "cos"])
+@pytest.mark.parametrize("d", [64, 264, 1024])
+def test_filter_bf16_inner_products_at_the_threshold_are_decided_exactly(ctxs, kind, d):
+    """Gaussian coordinates (inexact fp32 sums), thresholds at zero, next to zero and equal to the exact score of listed
+    pairs: a pair whose fp32 score lies within the sums' rounding error of the threshold is decided again in fp64, so the
+    kept list is the oracle's, copy for copy, with no band."""
+    rng = np.random.default_rng(d + 5)
+    P = W.f32_to_bf16_bits(rng.standard_normal((500, d)).astype(np.float32))
+    Q = W.f32_to_bf16_bits(rng.standard_normal((700, d)).astype(np.float32))
+    P[4] = 0
+    Q[6] = 0
+    Q[8] = P[9]
+    cand = np.stack([rng.integers(0, 500, 60000), rng.integers(0, 700, 60000)], axis=1).astype(np.int32)
+    cand[:700, 0], cand[:700, 1] = 4, np.arange(700)
+    sc = O.scores(P, Q, kind, "bf16", cand)
+    near = [float(sc[k]) for k in np.argsort(np.abs(sc)) if sc[k] != 0.0][:6]
+    for t in [0.0, -0.0, 1e-30, -1e-30] + near + [float(np.quantile(sc, 0.9)), float(sc[17])]:
+        kept = gpu_filter(ctxs["bf16"], P, Q, kind, t, cand)
+        want = O.filter_pairs(P, Q, kind, t, "bf16", cand)
+        if abs(t) < 1e-3 * (d if kind == "ip" else 1):
+            assert np.array_equal(np.sort(keys(kept)), np.sort(keys(want))), (kind, d, t)
+        else:
+            # a threshold equal to a pair's score in fp64 need not be a float: the plain band rule applies
+            lo = O.filter_pairs(P, Q, kind, t + REL * abs(t), "bf16", cand)
+            hi = O.filter_pairs(P, Q, kind, t - REL * abs(t), "bf16", cand)
+            assert np.isin(keys(lo), keys(kept)).all() and np.isin(keys(kept), keys(hi)).all()
+
+
 def test_filter_small_radius_on_long_rows_does_not_cancel(ctxs):
     """The difference form resolves radii far below the rows' norms (where the tile epilogue's norm expansion cannot)."""
     d = 2048

@@ -219,6 +219,33 @@ def test_lsh_bf16_sign_hash_join(ctx_bf16, kind, d, L, k):
     assert len(exact) <= len(full) and len(exact) > 0.3 * len(full)
 
 
+@pytest.mark.parametrize("kind", ["ip", "cos"])
+@pytest.mark.parametrize("d,L,k", [(64, 3, 2), (128, 2, 1), (520, 2, 1)])
+def test_lsh_bf16_thresholds_near_zero_are_decided_from_the_rows(ctx_bf16, kind, d, L, k):
+    """The bucketed join of bf16 points at inner-product / cosine thresholds with an empty tolerance band (zero, next to
+    zero, the exact score of a colliding pair): candidates are decided from the regrouped rows in fp64, so the result is
+    the oracle's exact set restricted to colliding pairs, bit for bit (the sampled-sign keys are exact)."""
+    rng = np.random.default_rng(d + L)
+    n, m = 900, 1100
+    P = W.f32_to_bf16_bits(rng.standard_normal((n, d)).astype(np.float32))
+    Q = W.f32_to_bf16_bits(rng.standard_normal((m, d)).astype(np.float32))
+    P[2] = 0
+    Q[3] = 0
+    dP, dQ = B.to_device(P), B.to_device(Q)
+    cap = n * m + 8
+    out = torch.full((cap, 2), -5, dtype=torch.int32, device="cuda:0")
+    coll = O.lsh_join_kind(P, Q, kind, float("-inf"), "bf16", L, k, 29)[0]        # every colliding pair
+    sc = O.scores(P, Q, kind, "bf16", coll)
+    near = [float(sc[i]) for i in np.argsort(np.abs(sc)) if sc[i] != 0.0][:5]
+    for t in [0.0, 1e-30, -1e-30] + near:
+        st, cnt = ctx_bf16.simjoin_run_lsh(dP, n, dQ, m, d, t, L, k, 29, out, cap, kind=kind)
+        assert st == B.SIMJOIN_OK, B.strerror(st)
+        got = keys(out[:cnt].cpu().numpy())
+        want = keys(O.lsh_join_kind(P, Q, kind, t, "bf16", L, k, 29)[0])
+        assert len(np.unique(got)) == cnt
+        assert np.array_equal(np.sort(got), np.sort(want)), (kind, d, t, cnt, len(want))
+
+
 def test_lsh_more_key_bits_than_coordinates(ctx_bf16, ctx):
     """k > d: the first d bits take every coordinate once, the later ones sample as they come.  8-coordinate bf16
     rows (16 bytes) with 12 key bits, and 16-coordinate int8 rows with 12 of 16 coordinates taken."""

@@ -620,6 +620,45 @@ def test_bf16_dense_sign_test_handles_zero_vectors_and_every_threshold(kind, d):
             assert_band(pairs, cnt, P, Q, kind, t)
 
 
+@pytest.mark.parametrize("kind", ["ip", "cos"])
+@pytest.mark.parametrize("n,m,d", [(300, 700, 64), (513, 1000, 128), (200, 600, 72), (150, 700, 520)])
+@pytest.mark.parametrize("dense", [0.0, 1.0])
+def test_bf16_thresholds_near_zero_are_decided_from_the_rows(kind, n, m, d, dense):
+    """An inner-product or cosine threshold at or near zero leaves no tolerance band (1e-2 |t|) for the fp32 accumulation
+    error of the tile product.  There the tile test is a filter and every candidate is decided from its rows in fp64, in the
+    oracle's order of operations: the result is the oracle's exact set, bit for bit -- Gaussian coordinates (inexact sums),
+    zero vectors, opposite rows, short, two-chunk and long rows, both epilogue layouts asked for.  Thresholds whose band
+    is wide enough keep the plain test (band rule)."""
+    rng = np.random.default_rng(d + n)
+    P = W.f32_to_bf16_bits(rng.standard_normal((n, d)).astype(np.float32))
+    Q = W.f32_to_bf16_bits(rng.standard_normal((m, d)).astype(np.float32))
+    P[3] = 0
+    Q[5] = 0
+    Q[9] = P[7] ^ np.uint16(0x8000)
+    Q[11] = P[8]
+    scale = float(d) if kind == "ip" else 1.0
+    with B.Simjoin("bf16", 0) as ctx:
+        assert ctx.simjoin_set_option(B.SIMJOIN_OPT_DENSE_EPILOGUE, dense) == B.SIMJOIN_OK
+        for t in (0.0, -0.0, 1e-30, -1e-30, 1e-7 * scale, -1e-7 * scale, 3e-5 * scale, -2e-4 * scale):
+            pairs, cnt = gpu_join(ctx, P, Q, kind, t, capacity=n * m + 8)
+            assert_exact(pairs, cnt, P, Q, kind, t, dtype="bf16")
+        for t in (0.05 * scale ** 0.5, -0.05 * scale ** 0.5, 0.2 * scale ** 0.5):
+            pairs, cnt = gpu_join(ctx, P, Q, kind, t, capacity=n * m + 8)
+            assert_band(pairs, cnt, P, Q, kind, t)
+        if d == 64:
+            # thresholds equal to the exact score of a pair whose score is nearly zero: that pair passes by equality, which
+            # an fp32-accumulated score gets right only by chance
+            cand = np.stack(np.meshgrid(np.arange(64), np.arange(m), indexing="ij"), axis=-1).reshape(-1, 2).astype(np.int32)
+            sc = O.scores(P, Q, kind, "bf16", cand)
+            order = np.argsort(np.abs(sc))
+            picked = [k for k in order if sc[k] != 0.0][:12]
+            for k in picked:
+                t = float(sc[k])
+                pairs, cnt = gpu_join(ctx, P, Q, kind, t, capacity=n * m + 8)
+                assert_exact(pairs, cnt, P, Q, kind, t, dtype="bf16")
+                assert tuple(cand[k]) in set(map(tuple, pairs.tolist()))
+
+
 def test_first_large_join_of_a_context_samples_its_density():
     """A fresh context in the default mode counts a sample's pairs before a join of 1e12 operations or more and picks the
     layout from that: the dense mixture then runs on transformed operands at once, a sparse join of the same size does not;
