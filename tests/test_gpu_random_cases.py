@@ -3,7 +3,9 @@ geometries, partial chunks), ragged row counts and value ranges, each compared w
 bf16: inside the threshold band); half of the cases also run the pair filter on a random candidate list.  Thresholds are
 taken from a sample of the oracle's scores so that every case has hits; bf16 Euclidean radii go down to whatever the
 sample's low tail gives, including radii far below the rows' norms (small point sets, where the sample meets the planted
-equal rows), which the join decides from the rows in the difference form."""
+equal rows), which the join decides from the rows in the difference form.  bf16 points are small integers (exact sums) or
+Gaussian (inexact ones); a fifth of the inner-product and cosine cases take a threshold at or next to zero -- or equal to a
+sampled pair's exact score -- where the band is empty and the join decides its candidates from the rows in fp64."""
 import numpy as np
 import pytest
 import torch
@@ -38,13 +40,23 @@ def test_random_cases_match_the_oracle(seed):
             m = int(rng.integers(1, 3000))
             if n * m * d > 2e9:
                 n = max(1, int(2e9 / (m * d)))
+            # thresholds at or next to zero (inner product, cosine): half of all pairs pass, and the tolerance band is empty
+            near_zero = kind != "l2" and rng.random() < 0.2
+            if near_zero:
+                n, m = min(n, 1000), min(m, 2000)
             lsh = rng.random() < 0.35
             s1, s2 = int(rng.integers(1 << 30)), int(rng.integers(1 << 30))
+            small_ints = False
             if dtype == "i8":
                 hi = int(rng.choice([1, 2, 5, 127]))
                 P, Q = W.random_points("i8", n, d, s1, lo=-hi, hi=hi), W.random_points("i8", m, d, s2, lo=-hi, hi=hi)
-            else:
+            elif rng.random() < 0.6:
                 P, Q = W.random_points("bf16", n, d, s1), W.random_points("bf16", m, d, s2)
+                small_ints = True
+            else:   # Gaussian coordinates: sums that fp32 does not hold exactly
+                g = np.random.default_rng(s1)
+                P = W.f32_to_bf16_bits(g.standard_normal((n, d)).astype(np.float32) * float(rng.choice([1e-3, 1.0, 50.0])))
+                Q = W.f32_to_bf16_bits(g.standard_normal((m, d)).astype(np.float32) * float(rng.choice([1e-3, 1.0, 50.0])))
             kpl = min(n, m, 64)
             Q[:kpl] = P[:kpl]                                   # equal rows: hits under every kind
             smp = np.stack([rng.integers(0, n, 2000), rng.integers(0, m, 2000)], axis=1).astype(np.int32)
@@ -52,10 +64,13 @@ def test_random_cases_match_the_oracle(seed):
             if kind == "l2":
                 dist = np.sqrt(np.maximum(sc, 0.0)) if dtype == "i8" else sc
                 t = float(np.quantile(dist, 0.002))
-                if dtype == "bf16" and rng.random() < 0.25:
+                if dtype == "bf16" and small_ints and rng.random() < 0.25:
                     t = float(rng.choice([0.0, 1e-3, 0.05, 0.3]))   # radii far below the norms: equal and near-equal rows only
             else:
                 t = float(np.quantile(sc, 0.998))
+            if near_zero:
+                nz = sc[sc != 0.0]
+                t = float(rng.choice([0.0, -0.0, 1e-30, -1e-30, float(nz[np.argmin(np.abs(nz))]) if len(nz) else 0.0]))
             ctx = ctxs[dtype]
             if dtype == "i8":     # small joins: the device's choice of the epilogue width, or the 32-bit one unasked
                 assert ctx.simjoin_set_option(B.SIMJOIN_OPT_SELECT_MIN_OPS, 0.0 if rng.random() < 0.7 else 2e11) == B.SIMJOIN_OK
