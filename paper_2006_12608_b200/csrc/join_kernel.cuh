@@ -132,6 +132,7 @@ struct JoinParams {
     const unsigned int *sel_words;
     int sel_mode;
     float sel_coef;
+    float thr_hi;                  // row-deciding inner-product / cosine forms: scores above this threshold pass without a look at the rows
     float sel_r2;                  // SEL_L2_RADIUS: r^2 (the kernel's own threshold differs when it runs on transformed operands)
     // When not null: a 64-byte control block that no launch of this call reads or writes.  The kernel zeroes it, so
     // that the caller's next join finds its counter, status and selection words cleared without a memset of its own.
@@ -421,11 +422,15 @@ __device__ __forceinline__ bool ipcos_bf16_passes(const JoinParams &p, long long
 // exact int8 cosine; VERIFY_L2_BF16: the difference-form Euclidean test).  Staged indices are regrouped positions
 // in bucketed mode, else row indices plus the caller's offsets.
 constexpr int VERIFY_NONE = 0, VERIFY_COS_I8 = 1, VERIFY_L2_BF16 = 2, VERIFY_IP_BF16 = 3, VERIFY_COS_BF16 = 4;
+// VERIFY_IP_BF16 / VERIFY_COS_BF16 stage a candidate with bit 31 of j set and a pair that is sure to pass with the bit
+// clear: only candidates are decided from their rows (`candidate`; the other kinds decide every staged pair).
+__host__ __device__ constexpr bool verify_flags(int verify) { return verify == 3 || verify == 4; }
 template <bool GROUPED, int VERIFY>
-__device__ __forceinline__ bool drop_pair(const JoinParams &p, int i, int j) {
+__device__ __forceinline__ bool drop_pair(const JoinParams &p, int i, int j, bool candidate = true) {
     if constexpr (GROUPED) {
         if (p.rep > 0 && already_reported(p, i, j)) return true;
     }
+    if (verify_flags(VERIFY) && !candidate) return false;
     if constexpr (VERIFY == VERIFY_COS_I8) {
         if (!cos_i8_passes(p, GROUPED ? i : i - p.ioff, GROUPED ? j : j - p.joff)) return true;
     }
@@ -480,8 +485,14 @@ __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf
                 const int k = k0 + lane;
                 bool keep = false;
                 if (k < fill) {
-                    const int2 pr = wbuf[k];
-                    keep = !drop_pair<GROUPED, VERIFY>(p, pr.x, pr.y);
+                    int2 pr = wbuf[k];
+                    bool candidate = true;
+                    if constexpr (verify_flags(VERIFY)) {
+                        candidate = pr.y < 0;
+                        pr.y &= 0x7fffffff;
+                        wbuf[k].y = pr.y;
+                    }
+                    keep = !drop_pair<GROUPED, VERIFY>(p, pr.x, pr.y, candidate);
                     if (!keep) wbuf[k].x = -1;
                 }
                 kept += __popc(__ballot_sync(0xffffffffu, keep));
@@ -516,9 +527,12 @@ __device__ __forceinline__ void flush_pairs(const JoinParams &p, const int2 *buf
 // prefix over the warp, then into the warp's shared-memory staging buffer, which is flushed with
 // one global atomic per ~STAGE_PAIRS pairs.  A block with more hits than the buffer holds leaves in
 // rounds through the same buffer.  `fill` (warp-uniform) is the number of pairs staged so far.
+// `cand` (kinds with verify_flags only): the columns of `mask` that are candidates; their staged j carries bit 31.
 template <int NQ, bool GROUPED, int VERIFY = VERIFY_NONE, int SP = STAGE_PAIRS>
 __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (&mask)[NQ], int lane, long long i, long long j0,
-                                           int2 *buf, int &fill) {
+                                           int2 *buf, int &fill, const uint32_t *cand = nullptr) {
+    constexpr bool FLAGS = verify_flags(VERIFY);
+    auto flag_of = [&](int q, int c) -> int { return FLAGS ? (int)(((cand[q] >> c) & 1u) << 31) : 0; };
     int cnt = 0;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) cnt += __popc(mask[q]);
@@ -582,12 +596,13 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
                     if (!found && m[q] != 0) {
-                        col = 32 * q + __ffs(m[q]) - 1;
+                        const int c = __ffs(m[q]) - 1;
+                        col = (32 * q + c) | flag_of(q, c);
                         m[q] &= m[q] - 1;
                         found = true;
                     }
                 }
-                buf[pos++] = make_int2(ii, jj + col);
+                buf[pos++] = make_int2(ii, (jj + (col & 0x7fffffff)) | (col & (int)0x80000000));
             }
             remaining -= take;
             __syncwarp();
@@ -607,8 +622,11 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
             int col = 0;
 #pragma unroll
             for (int q = 0; q < NQ; ++q)
-                if (mask[q] != 0) col = 32 * q + __ffs(mask[q]) - 1;
-            buf[fill + incl - 1] = make_int2(ii, jj + col);
+                if (mask[q] != 0) {
+                    const int c = __ffs(mask[q]) - 1;
+                    col = (32 * q + c) | flag_of(q, c);
+                }
+            buf[fill + incl - 1] = make_int2(ii, (jj + (col & 0x7fffffff)) | (col & (int)0x80000000));
         }
         fill += total;
         __syncwarp();
@@ -621,7 +639,7 @@ __device__ __forceinline__ void emit_pairs(const JoinParams &p, const uint32_t (
         while (mk) {
             const int c = __ffs(mk) - 1;
             mk &= mk - 1;
-            buf[pos++] = make_int2(ii, jj + 32 * q + c);
+            buf[pos++] = make_int2(ii, (jj + 32 * q + c) | flag_of(q, c));
         }
     }
     fill += total;
@@ -887,7 +905,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
     if constexpr (IPCOS_FILTER && KIND == KIND_IP) {
         // the filter threshold: t lowered by the error bound at the largest norms (the words hold max |x|^2, max |y|^2)
         const float mx = sqrtf(__uint_as_float(__ldg(p.sel_words))), my = sqrtf(__uint_as_float(__ldg(p.sel_words + 1)));
-        p.thr_f = __fsub_rd(p.thr_f, __fmul_ru(IPCOS_FILTER_MARGIN * p.sel_coef, __fmul_ru(mx, my)));
+        const float margin = __fmul_ru(IPCOS_FILTER_MARGIN * p.sel_coef, __fmul_ru(mx, my));
+        p.thr_hi = __fadd_ru(p.thr_f, margin);      // above it a score passes whatever its rounding error
+        p.thr_f = __fsub_rd(p.thr_f, margin);
     }
     if constexpr (LONGK) {
         p.stationary = 0;
@@ -1055,6 +1075,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             const long long q_end = GROUPED ? (long long)un.qrow0 + un.qrows : p.m;   // end of the Q rows of this unit
             int ri = 0;          // I8/L2: |x|^2 - floor(r^2)
             float rf = 0.f;      // COS: t*|x|;  BF16/L2: (|x|^2 - r^2) / 2
+            float rf_hi = 0.f;   // row-deciding cosine form: the same with the raised threshold
             if (row_ok) {
                 if constexpr (DT == DT_I8 && KIND == KIND_L2) ri = reinterpret_cast<const int *>(p.nx)[i] - p.thr_i;
                 if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
@@ -1066,6 +1087,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     //          s - (-0) = +0 for a score of either zero.
                     rf = p.thr_f * reinterpret_cast<const float *>(p.nx)[i];
                     if (p.thr_f > 0.f && rf == 0.f) rf = 1.401298464e-45f;
+                    if constexpr (IPCOS_FILTER) {
+                        rf_hi = p.thr_hi * reinterpret_cast<const float *>(p.nx)[i];
+                        if (p.thr_hi > 0.f && rf_hi == 0.f) rf_hi = 1.401298464e-45f;
+                    }
                 }
                 if constexpr (DT == DT_I8 && KIND == KIND_COS) {
                     // fp32 filter for s >= t |x| |y|, lowered by 2^-18 relative (the fp32 roundings of t, the two norms,
@@ -1323,8 +1348,9 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     if (!row_ok) gm = 0;
                     const long long j0 = q_base + (long long)qt * TN + ps * TILE_N + coff;
                     uint32_t mask[ECOLS / 32];
+                    uint32_t cand[ECOLS / 32];          // row-deciding inner-product / cosine forms: passing columns that are not sure to pass
 #pragma unroll
-                    for (int q = 0; q < ECOLS / 32; ++q) mask[q] = 0;
+                    for (int q = 0; q < ECOLS / 32; ++q) mask[q] = cand[q] = 0;
                     if constexpr (KIND != KIND_IP) {
                         // the per-column terms go through shared memory: level 2 reads 16 of them per group as four
                         // broadcast loads (a shuffle per term cost four times the instructions)
@@ -1372,6 +1398,22 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
 #pragma unroll
                             for (int q = 0; q < NCH; ++q) fall |= fail[q] << (4 * (NCH - 1 - q));
                             mk = (__brev(~fall) >> (32 - GCOLS)) & GMASK;
+                            if constexpr (IPCOS_FILTER) {
+                                // sure to pass: s > b_hi, the sign bit of fl(b_hi - s) (a score equal to the bound stays a candidate)
+                                uint32_t sure[NCH];
+#pragma unroll
+                                for (int q = 0; q < NCH; ++q) sure[q] = 0;
+#pragma unroll
+                                for (int c = 0; c < GCOLS; ++c) {
+                                    const float bh = KIND == KIND_IP ? p.thr_hi : __fmul_rn(rf_hi, __uint_as_float(yw[c]));
+                                    sure[c >> 2] = __funnelshift_l(__float_as_uint(bh - __uint_as_float(v[k * GCOLS + c])), sure[c >> 2], 1);
+                                }
+                                uint32_t sall = 0;
+#pragma unroll
+                                for (int q = 0; q < NCH; ++q) sall |= sure[q] << (4 * (NCH - 1 - q));
+                                const uint32_t mk_cand = mk & ~((__brev(sall) >> (32 - GCOLS)) & GMASK);
+                                if ((gm >> k) & 1u) cand[(k * GCOLS) >> 5] |= mk_cand << ((k * GCOLS) & 31);
+                            }
                         } else {
 #pragma unroll
                         for (int c = 0; c < GCOLS; ++c) {
@@ -1401,7 +1443,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                             mask[q] &= lq >= 32 ? 0xffffffffu : (lq <= 0 ? 0u : ((1u << (int)lq) - 1u));
                         }
                     }
-                    emit_pairs<ECOLS / 32, GROUPED, VERIFY, SPAIRS>(p, mask, lane, i, j0, stage_buf, stage_fill);
+                    emit_pairs<ECOLS / 32, GROUPED, VERIFY, SPAIRS>(p, mask, lane, i, j0, stage_buf, stage_fill, cand);
                 }
                 }   // passes
                 if constexpr (LONGK) {

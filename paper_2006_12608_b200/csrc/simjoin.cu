@@ -478,6 +478,7 @@ bool cos_row_form(JoinParams &jp, bool i8, simjoin_kind kind) {
     if (i8 || kind != SIMJOIN_COS) return false;
     const bool rows = jp.sel_coef > IPCOS_BAND_SHARE * std::fabs(jp.thr_f);
     if (rows) {
+        jp.thr_hi = std::nextafterf(jp.thr_f + IPCOS_FILTER_MARGIN * jp.sel_coef, INFINITY);
         jp.thr_f = std::nextafterf(jp.thr_f - IPCOS_FILTER_MARGIN * jp.sel_coef, -INFINITY);
         if (jp.thr_f == 0.f) jp.thr_f = -0.0f;
     }
