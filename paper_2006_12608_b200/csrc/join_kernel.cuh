@@ -133,6 +133,7 @@ struct JoinParams {
     int sel_mode;
     float sel_coef;
     float thr_hi;                  // row-deciding inner-product / cosine forms: scores above this threshold pass without a look at the rows
+    float l2_xscale_hi, l2_ycoef_hi, l2_thr_sure;   // the same for the small-radius Euclidean form: the filter's coefficients, raised
     float sel_r2;                  // SEL_L2_RADIUS: r^2 (the kernel's own threshold differs when it runs on transformed operands)
     // When not null: a 64-byte control block that no launch of this call reads or writes.  The kernel zeroes it, so
     // that the caller's next join finds its counter, status and selection words cleared without a memset of its own.
@@ -422,9 +423,9 @@ __device__ __forceinline__ bool ipcos_bf16_passes(const JoinParams &p, long long
 // exact int8 cosine; VERIFY_L2_BF16: the difference-form Euclidean test).  Staged indices are regrouped positions
 // in bucketed mode, else row indices plus the caller's offsets.
 constexpr int VERIFY_NONE = 0, VERIFY_COS_I8 = 1, VERIFY_L2_BF16 = 2, VERIFY_IP_BF16 = 3, VERIFY_COS_BF16 = 4;
-// VERIFY_IP_BF16 / VERIFY_COS_BF16 stage a candidate with bit 31 of j set and a pair that is sure to pass with the bit
+// The bf16 kinds (VERIFY_L2_BF16, VERIFY_IP_BF16, VERIFY_COS_BF16) stage a candidate with bit 31 of j set and a pair that is sure to pass with the bit
 // clear: only candidates are decided from their rows (`candidate`; the other kinds decide every staged pair).
-__host__ __device__ constexpr bool verify_flags(int verify) { return verify == 3 || verify == 4; }
+__host__ __device__ constexpr bool verify_flags(int verify) { return verify == 2 || verify == 3 || verify == 4; }
 template <bool GROUPED, int VERIFY>
 __device__ __forceinline__ bool drop_pair(const JoinParams &p, int i, int j, bool candidate = true) {
     if constexpr (GROUPED) {
@@ -1075,7 +1076,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
             const long long q_end = GROUPED ? (long long)un.qrow0 + un.qrows : p.m;   // end of the Q rows of this unit
             int ri = 0;          // I8/L2: |x|^2 - floor(r^2)
             float rf = 0.f;      // COS: t*|x|;  BF16/L2: (|x|^2 - r^2) / 2
-            float rf_hi = 0.f;   // row-deciding cosine form: the same with the raised threshold
+            float rf_hi = 0.f;   // row-deciding cosine and Euclidean forms: the same with the raised threshold
             if (row_ok) {
                 if constexpr (DT == DT_I8 && KIND == KIND_L2) ri = reinterpret_cast<const int *>(p.nx)[i] - p.thr_i;
                 if constexpr (DT == DT_BF16 && KIND == KIND_COS) {
@@ -1102,7 +1103,10 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                 }
                 // BF16/L2 decides |x|^2 + |y|^2 - 2s <= r^2 as  s >= (|x|^2 - r^2)/2 + |y|^2/2:  one add per element
                 if constexpr (DT == DT_BF16 && KIND == KIND_L2) {
-                    if constexpr (L2_FILTER) rf = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] * p.l2_xscale - p.l2_thr_filter);
+                    if constexpr (L2_FILTER) {
+                        rf = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] * p.l2_xscale - p.l2_thr_filter);
+                        rf_hi = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] * p.l2_xscale_hi - p.l2_thr_sure);
+                    }
                     else rf = 0.5f * (reinterpret_cast<const float *>(p.nx)[i] - p.thr_f);
                 }
             }
@@ -1348,7 +1352,7 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
                     if (!row_ok) gm = 0;
                     const long long j0 = q_base + (long long)qt * TN + ps * TILE_N + coff;
                     uint32_t mask[ECOLS / 32];
-                    uint32_t cand[ECOLS / 32];          // row-deciding inner-product / cosine forms: passing columns that are not sure to pass
+                    uint32_t cand[ECOLS / 32];          // row-deciding forms: passing columns that are not sure to pass
 #pragma unroll
                     for (int q = 0; q < ECOLS / 32; ++q) mask[q] = cand[q] = 0;
                     if constexpr (KIND != KIND_IP) {
@@ -1398,14 +1402,16 @@ join_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CU
 #pragma unroll
                             for (int q = 0; q < NCH; ++q) fall |= fail[q] << (4 * (NCH - 1 - q));
                             mk = (__brev(~fall) >> (32 - GCOLS)) & GMASK;
-                            if constexpr (IPCOS_FILTER) {
+                            if constexpr (IPCOS_FILTER || L2_FILTER) {
                                 // sure to pass: s > b_hi, the sign bit of fl(b_hi - s) (a score equal to the bound stays a candidate)
                                 uint32_t sure[NCH];
 #pragma unroll
                                 for (int q = 0; q < NCH; ++q) sure[q] = 0;
 #pragma unroll
                                 for (int c = 0; c < GCOLS; ++c) {
-                                    const float bh = KIND == KIND_IP ? p.thr_hi : __fmul_rn(rf_hi, __uint_as_float(yw[c]));
+                                    const float bh = KIND == KIND_IP    ? p.thr_hi
+                                                     : KIND == KIND_COS ? __fmul_rn(rf_hi, __uint_as_float(yw[c]))
+                                                                        : __fmaf_rn(p.l2_ycoef_hi, __uint_as_float(yw[c]), rf_hi);
                                     sure[c >> 2] = __funnelshift_l(__float_as_uint(bh - __uint_as_float(v[k * GCOLS + c])), sure[c >> 2], 1);
                                 }
                                 uint32_t sall = 0;

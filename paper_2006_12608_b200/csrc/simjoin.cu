@@ -364,6 +364,11 @@ void set_thresholds(JoinParams &jp, bool i8, simjoin_kind kind, double threshold
             jp.l2_ycoef = (float)(0.5 * (1.0 - eps));
             // the difference form's own error (about d 2^-24 relative) is far inside the 2^-10 added here
             jp.l2_thr_filter = std::nextafterf((float)(threshold * threshold * (1.0 + 1.0 / 1024.0)), INFINITY);
+            // ... and the mirror image: a score above the bound built from these passes whatever its rounding error
+            // (|x|^2 + |y|^2 - 2s, raised by the error bound, is below r^2 (1 - 2^-10)), so its rows are not read
+            jp.l2_xscale_hi = (float)(1.0 + eps);
+            jp.l2_ycoef_hi = (float)(0.5 * (1.0 + eps));
+            jp.l2_thr_sure = std::nextafterf((float)(threshold * threshold * (1.0 - 1.0 / 1024.0)), -INFINITY);
         }
     }
 }
