@@ -75,3 +75,24 @@ def test_generated_inputs_have_the_recorded_hashes(cfg):
     import hashlib
     w = W.make_workload(cfg, **SHA_SIZES[cfg])
     assert (hashlib.sha256(w.P).hexdigest(), hashlib.sha256(w.Q).hexdigest()) == INPUT_SHA256[cfg]
+
+
+def test_full_size_digest_file_is_well_formed_and_names_these_inputs():
+    """The stored digests of the oracle's whole joins (tests/golden/full_size_digests.json): one entry per full-size
+    configuration with the fields the GPU test reads, for the inputs this generator produces (configuration 2 is hashed
+    at full size above; the GPU test regenerates and compares all four)."""
+    import json
+    import os
+    with open(os.path.join(os.path.dirname(__file__), "golden", "full_size_digests.json")) as f:
+        g = json.load(f)
+    assert sorted(g) == ["2", "3", "4", "5"]
+    for cfg, e in g.items():
+        c = W.CONFIGS[int(cfg)]
+        assert (e["n"], e["m"], e["d"], e["threshold"]) == (c["n"], c["m"], c["d"], c["threshold"])
+        assert len(e["inputs_sha256"]["P"]) == len(e["inputs_sha256"]["Q"]) == 64
+        if e["dtype"] == "i8":
+            assert e["count"] > 0 and len(e["sorted_keys_sha256"]) == 64
+        else:
+            assert e["strict_count"] <= e["exact_count"] <= e["loose_count"]
+            assert len(e["band_pairs"]) == e["loose_count"] - e["strict_count"] and len(e["strict_sorted_keys_sha256"]) == 64
+    assert (g["2"]["inputs_sha256"]["P"], g["2"]["inputs_sha256"]["Q"]) == INPUT_SHA256[2]
